@@ -1,0 +1,202 @@
+"""Pins for the CPU oracle's model side (oracle/model.py, oracle/chain.py).
+
+The target forward is checked against library implementations of the same architecture (the transformers
+package's Llama model and its Qwen3 mixture-of-experts block, torch's attention and RMSNorm), the rotary
+embedding through its invariants, and the cached forward against the cache-free one.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import model
+from oracle.chain import ChainOracle
+from paper_2604_26779_b200 import inputs
+
+
+def _tiny_cfg(**over):
+    cfg = inputs.model_config("c1")
+    cfg.update(over)
+    return cfg
+
+
+def test_target_forward_matches_transformers_llama():
+    from transformers import LlamaConfig, LlamaForCausalLM
+    cfg = _tiny_cfg(n_kv_heads=2)                      # grouped-query attention: 4 q heads on 2 KV heads
+    W = inputs.make_target_weights(cfg, seed=11, std=0.05)
+    rng = np.random.default_rng(0)
+    for lw in W["layers"]:                             # non-trivial norm weights
+        lw["attn_norm"] = (1 + 0.1 * rng.standard_normal(cfg["d_model"])).astype(np.float32)
+        lw["mlp_norm"] = (1 + 0.1 * rng.standard_normal(cfg["d_model"])).astype(np.float32)
+    W["final_norm"] = (1 + 0.1 * rng.standard_normal(cfg["d_model"])).astype(np.float32)
+    hf = LlamaConfig(vocab_size=cfg["vocab"], hidden_size=cfg["d_model"], intermediate_size=cfg["d_ffn"],
+                     num_hidden_layers=cfg["n_layers"], num_attention_heads=cfg["n_q_heads"],
+                     num_key_value_heads=cfg["n_kv_heads"], head_dim=cfg["head_dim"], rms_norm_eps=cfg["rms_eps"],
+                     rope_theta=cfg["rope_theta"], attention_bias=False, mlp_bias=False,
+                     tie_word_embeddings=False, max_position_embeddings=512)
+    m = LlamaForCausalLM(hf).double().eval()
+    Hq, Hkv, dh = cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"]
+    sd = {"model.embed_tokens.weight": W["embed"], "model.norm.weight": W["final_norm"], "lm_head.weight": W["lm_head"]}
+    for l, lw in enumerate(W["layers"]):
+        pre = f"model.layers.{l}."
+        sd[pre + "self_attn.q_proj.weight"] = lw["wqkv"][: Hq * dh]
+        sd[pre + "self_attn.k_proj.weight"] = lw["wqkv"][Hq * dh : (Hq + Hkv) * dh]
+        sd[pre + "self_attn.v_proj.weight"] = lw["wqkv"][(Hq + Hkv) * dh :]
+        sd[pre + "self_attn.o_proj.weight"] = lw["wo"]
+        sd[pre + "mlp.gate_proj.weight"] = lw["wgate"]
+        sd[pre + "mlp.up_proj.weight"] = lw["wup"]
+        sd[pre + "mlp.down_proj.weight"] = lw["wdown"]
+        sd[pre + "input_layernorm.weight"] = lw["attn_norm"]
+        sd[pre + "post_attention_layernorm.weight"] = lw["mlp_norm"]
+    missing = m.load_state_dict({k: torch.tensor(np.asarray(v, np.float64)) for k, v in sd.items()}, strict=False)
+    assert not [k for k in missing.missing_keys if "rotary" not in k] and not missing.unexpected_keys
+    toks = inputs.make_prompts(1, 23, cfg["vocab"], seed=3)[0]
+    with torch.no_grad():
+        out = m(torch.tensor(toks[None].astype(np.int64)), output_hidden_states=True)
+    got = model.target_forward(cfg, W, toks, tap_layers=(0, 1, 2))
+    # the library evaluates its rotary cos/sin tables in fp32 even in a double model: agreement stops near 1e-6,
+    # four orders of magnitude below what any structural mistake (pairing, sign, norm, head order) produces
+    assert np.max(np.abs(got["logits"] - out.logits[0].numpy())) < 5e-6
+    assert np.max(np.abs(out.logits[0].numpy())) > 0.5
+    d = cfg["d_model"]
+    # residual stream after 0 and 1 layers = the library's hidden_states[0], [1]
+    assert np.max(np.abs(got["taps"][:, :d] - out.hidden_states[0][0].numpy())) < 1e-12
+    assert np.max(np.abs(got["taps"][:, d : 2 * d] - out.hidden_states[1][0].numpy())) < 5e-6
+
+
+def test_attention_matches_torch_sdpa():
+    rng = np.random.default_rng(1)
+    T, n_past, Hq, Hkv, dh = 5, 37, 8, 2, 32
+    q = rng.standard_normal((T, Hq, dh))
+    k = rng.standard_normal((n_past + T, Hkv, dh))
+    v = rng.standard_normal((n_past + T, Hkv, dh))
+    got = model.attention(q, k, v, n_past)
+    mask = torch.tril(torch.ones(T, n_past + T, dtype=torch.bool), diagonal=n_past)
+    qt = torch.tensor(q).permute(1, 0, 2)[None]
+    kt = torch.tensor(k).permute(1, 0, 2)[None].repeat_interleave(Hq // Hkv, dim=1)
+    vt = torch.tensor(v).permute(1, 0, 2)[None].repeat_interleave(Hq // Hkv, dim=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, attn_mask=mask)[0].permute(1, 0, 2).numpy()
+    assert np.max(np.abs(got - ref)) < 1e-12
+
+
+def test_rmsnorm_matches_torch():
+    rng = np.random.default_rng(2)
+    x, w = rng.standard_normal((6, 96)), rng.standard_normal(96)
+    ref = torch.nn.functional.rms_norm(torch.tensor(x), (96,), torch.tensor(w), eps=1e-5).numpy()
+    assert np.max(np.abs(model.rmsnorm(x, w, 1e-5) - ref)) < 1e-13
+
+
+def test_rope_invariants():
+    rng = np.random.default_rng(3)
+    q, k = rng.standard_normal((1, 2, 64)), rng.standard_normal((1, 2, 64))
+    theta = 10000.0
+    assert np.allclose(model.rope(q, [0], theta), q)                                   # position 0 is the identity
+    assert np.allclose(np.linalg.norm(model.rope(q, [123], theta), axis=-1), np.linalg.norm(q, axis=-1))
+    # scores depend on the position difference only
+    a = np.sum(model.rope(q, [40], theta) * model.rope(k, [33], theta))
+    b = np.sum(model.rope(q, [1007], theta) * model.rope(k, [1000], theta))
+    assert abs(a - b) < 1e-9
+    # the first pair (j = 0, partner j + dh/2) turns by exactly `pos` radians
+    e = np.zeros((1, 1, 64))
+    e[0, 0, 0] = 1.0
+    r = model.rope(e, [0.5], theta)[0, 0]
+    assert np.isclose(r[0], np.cos(0.5)) and np.isclose(r[32], np.sin(0.5)) and np.count_nonzero(r) == 2
+    # the last pair turns by pos * theta^(-(dh-2)/dh)
+    e = np.zeros((1, 1, 64))
+    e[0, 0, 31] = 1.0
+    r = model.rope(e, [100.0], theta)[0, 0]
+    assert np.isclose(r[31], np.cos(100.0 * theta ** (-62 / 64))) and np.isclose(r[63], np.sin(100.0 * theta ** (-62 / 64)))
+
+
+def test_forward_with_past_equals_recompute():
+    cfg = _tiny_cfg()
+    W = inputs.make_target_weights(cfg, seed=5, std=0.05)
+    toks = inputs.make_prompts(1, 20, cfg["vocab"], seed=8)[0]
+    full = model.target_forward(cfg, W, toks, tap_layers=(0, 1, 2))
+    head = model.target_forward(cfg, W, toks[:16])
+    tail = model.target_forward(cfg, W, toks[16:], past=head["new_kv"], start_pos=16, tap_layers=(0, 1, 2))
+    assert np.max(np.abs(tail["logits"] - full["logits"][16:])) < 1e-10
+    assert np.max(np.abs(tail["taps"] - full["taps"][16:])) < 1e-10
+    # k = 0: a one-token verify is plain decode
+    one = model.target_forward(cfg, W, toks[19:], past=[(np.concatenate([a, c[:3]]), np.concatenate([b, e[:3]]))
+                                                       for (a, b), (c, e) in zip(head["new_kv"], tail["new_kv"])],
+                               start_pos=19)
+    assert np.max(np.abs(one["logits"][0] - full["logits"][19])) < 1e-10
+
+
+def test_moe_matches_transformers_block():
+    from transformers.models.qwen3_moe import modeling_qwen3_moe as mq
+    d, E, Fe, topk = 64, 16, 32, 4
+    cfg = dict(inputs.model_config("c5"), d_model=d, n_experts=E, d_expert_ffn=Fe, experts_top_k=topk,
+               n_q_heads=2, n_kv_heads=1, head_dim=32, dtype="f32")
+    lw = inputs.make_layer_weights(cfg, np.random.default_rng(4), std=0.2)
+    lw["router"] = (lw["router"] * 8).astype(np.float32)
+    hf = mq.Qwen3MoeConfig(hidden_size=d, moe_intermediate_size=Fe, num_experts=E, num_experts_per_tok=topk,
+                           norm_topk_prob=True)
+    blk = mq.Qwen3MoeSparseMoeBlock(hf).double().eval()
+    names = dict(blk.named_parameters())
+    with torch.no_grad():
+        names["gate.weight"].copy_(torch.tensor(lw["router"].astype(np.float64)))
+        names["experts.gate_up_proj"].copy_(torch.tensor(
+            np.concatenate([lw["experts_gate"], lw["experts_up"]], axis=1).astype(np.float64)))
+        names["experts.down_proj"].copy_(torch.tensor(lw["experts_down"].astype(np.float64)))
+        x = np.random.default_rng(5).standard_normal((9, d))
+        out = blk(torch.tensor(x)[None])
+        ref = (out[0] if isinstance(out, tuple) else out).reshape(9, d).numpy()
+    got = model.moe_mlp(lw, x, topk)
+    # the library's router takes its softmax in fp32, so the mixture weights agree to fp32 rounding only
+    assert np.max(np.abs(got - ref)) < 1e-5 and np.max(np.abs(ref)) > 0.5
+    # ties go to the lower expert index
+    ids, wts = model.moe_route(np.array([[1.0, 3.0, 3.0, 0.0, 3.0]]), 2)
+    assert ids[0].tolist() == [1, 2] and np.allclose(wts[0], 0.5)
+
+
+@pytest.mark.parametrize("kind", ["eagle3", "mtp"])
+def test_draft_head_consistency(kind):
+    """The heads are this build's own definitions; what can be pinned is structural: proposing k tokens in one
+    call equals proposing them slot by slot through the cached path, and the true-slot part is causal."""
+    cfg = _tiny_cfg(tap_layers=(0, 1, 2) if kind == "eagle3" else (2,))
+    W = inputs.make_target_weights(cfg, seed=5, std=0.05)
+    H = (inputs.make_eagle3_weights if kind == "eagle3" else inputs.make_mtp_weights)(cfg, seed=6, std=0.05)
+    toks = inputs.make_prompts(1, 12, cfg["vocab"], seed=2)[0]
+    feats = model.target_forward(cfg, W, toks[:-1], tap_layers=cfg["tap_layers"])["taps"]
+    u = oracle.uniforms(7, 0, 1, 1, 3)[0]
+
+    def sample_fn(i, lg):
+        q = oracle.softmax(np.asarray(lg, np.float32)[None])[0]
+        return oracle.invcdf(q, u[i])[0], q
+
+    d_all, q_all, _ = model.draft_propose(cfg, W, H, kind, feats, toks[1:], 3, sample_fn)
+    # the same with the first 8 true slots served from a cache built by an earlier call
+    if kind == "eagle3":
+        g = feats[:8] @ H["wfc"].astype(np.float64).T
+        _, pk, pv = model.eagle3_slots(cfg, W, H, g, toks[1:9], np.arange(8))
+    else:
+        _, pk, pv = model.mtp_slots(cfg, W, H, feats[:8], toks[1:9], np.arange(8))
+    d_inc, q_inc, _ = model.draft_propose(cfg, W, H, kind, feats[8:], toks[9:], 3, sample_fn, pk, pv, first_slot=8)
+    assert d_all.tolist() == d_inc.tolist() and np.max(np.abs(q_all - q_inc)) < 1e-7
+    assert np.allclose(q_all.sum(-1), 1.0, atol=1e-5)
+
+
+def test_chain_oracle_emits_between_1_and_k_plus_1_tokens():
+    cfg = _tiny_cfg()
+    W = inputs.make_target_weights(cfg, seed=inputs.sub_seed(1, 0))
+    H = inputs.make_eagle3_weights(cfg, seed=inputs.sub_seed(1, 1))
+    prompt = inputs.make_prompts(1, 16, cfg["vocab"], seed=inputs.sub_seed(1, 2))[0]
+    ch = ChainOracle(cfg, W, H, "eagle3", seed=inputs.BASE_SEED, seq_index=0, prompt=prompt)
+    for _ in range(4):
+        L = len(ch.tokens)
+        rec = ch.step_once(3)
+        assert 1 <= rec["n_emitted"] <= 4 and len(ch.tokens) == L + rec["n_emitted"]
+        assert np.all(rec["out_tokens"][rec["n_emitted"]:] == -1)
+    # draft == target (the head replaced by forced drafts with q = p): every draft token is accepted
+    ch2 = ChainOracle(cfg, W, H, "eagle3", seed=1, seq_index=0, prompt=prompt)
+    toks = list(prompt)
+    drafts, qs = [], []
+    for i in range(3):
+        lg = model.target_forward(cfg, W, toks + drafts)["logits"][-1].astype(np.float32)
+        q = oracle.softmax(lg[None])[0]
+        drafts.append(oracle.invcdf(q, 0.37 + 0.1 * i)[0])
+        qs.append(q)
+    rec = ch2.step_once(3, forced_drafts=(drafts, np.stack(qs)))
+    assert rec["n_emitted"] == 4
