@@ -1,0 +1,238 @@
+/*
+ * spec.h - C ABI of the speculative-decoding step library (CUDA, sm_100a).
+ *
+ * One speculation step of autoregressive rollout generation: a draft head proposes k tokens, the target
+ * model verifies the k+1 positions in one forward against a paged KV cache, a lossless rejection sampler
+ * keeps the target's output distribution, and the KV cache keeps the accepted slots (paper: Introduction,
+ * third paragraph; Section 2.1 "rollouts follow the verifier policy by construction"; Section 2.2 "only the
+ * autoregressive decode phase", "tokens produced per speculation step"; Section 2.3 the two drafting paths).
+ *
+ * Conventions for every function:
+ *   - plain C types only; pointers named *_host are host pointers, every other pointer is a DEVICE pointer;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream);
+ *   - the library never allocates or frees device memory: every buffer is caller-owned and must outlive
+ *     the calls (and the context) that use it;
+ *   - step functions only enqueue work on `stream`; they do not synchronise (spec_get_status does);
+ *   - a host-detectable problem returns a negative spec_status and launches nothing; a problem found on
+ *     the device is recorded in a status word (first error wins) and never traps;
+ *   - a context is not thread-safe.
+ *
+ * Layouts: a weight matrix is [out][in] row-major; token ids, lengths and tables are int32; logits and
+ * probabilities are fp32; activations, weights and KV are bf16 (SPEC_DTYPE_BF16) or fp32 (SPEC_DTYPE_F32).
+ */
+#ifndef SPEC_H_
+#define SPEC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPEC_ABI_VERSION 1u
+
+typedef struct spec_ctx spec_ctx; /* opaque */
+
+typedef enum {
+    SPEC_OK = 0,
+    /* detected on the host, returned immediately, nothing launched */
+    SPEC_ERR_INVALID_ARG = -1,
+    SPEC_ERR_SHAPE = -2,
+    SPEC_ERR_UNSUPPORTED = -3,
+    SPEC_ERR_STATE = -4,
+    SPEC_ERR_CUDA = -5,
+    /* detected on the device, reported through the status word / spec_get_status */
+    SPEC_ERR_KV_EXHAUSTED = -16,
+    SPEC_ERR_TOKEN_RANGE = -17,
+    SPEC_ERR_BAD_PROB = -18,
+    SPEC_ERR_TIMEOUT = -19
+} spec_status;
+
+enum { SPEC_DTYPE_BF16 = 0, SPEC_DTYPE_F32 = 1 };
+enum { SPEC_DRAFT_NONE = 0, SPEC_DRAFT_EAGLE3 = 1, SPEC_DRAFT_MTP = 2 };
+
+/* Model and run description.  n_experts = 0 selects the dense SwiGLU MLP. */
+typedef struct {
+    uint32_t struct_size, abi_version;
+    int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    int32_t n_experts, experts_top_k, d_expert_ffn;
+    float rms_eps, rope_theta;
+    int32_t dtype;              /* SPEC_DTYPE_*: storage type of weights, KV and activations            */
+    int32_t draft_kind;         /* SPEC_DRAFT_*; NONE = the caller supplies draft tokens and draft logits */
+    int32_t draft_d_ffn;        /* FFN width of the draft head's layer                                   */
+    int32_t n_taps, tap_layers[3]; /* residual-stream taps handed to the draft head: tap t = after t layers */
+    int32_t k_max;              /* largest draft length used with this context (<= 7)                    */
+    int32_t max_batch;
+    int32_t kv_block_tokens;    /* tokens per KV block (16)                                              */
+    int32_t kv_num_blocks;      /* physical blocks per layer pool                                        */
+    int32_t max_blocks_per_seq;
+    int32_t kv_layer_pools;     /* physical per-layer pools G <= n_layers; layer l uses pool l mod G.    */
+                                /* G < n_layers aliases layers onto shared pools: a timing-only mode for  */
+                                /* caches larger than the device; results are then not meaningful        */
+    float temperature;          /* > 0; scales the logits of both models before the softmax              */
+    uint64_t seed;              /* Philox key of every uniform the step draws                            */
+} spec_config;
+
+/* Byte sizes of the caller-owned device arenas for a configuration. */
+typedef struct {
+    size_t weights_bytes, draft_weights_bytes, kv_bytes, draft_kv_bytes, workspace_bytes, state_bytes;
+} spec_sizes;
+
+/* The arenas themselves (device pointers, each 256-byte aligned, at least the queried size). */
+typedef struct {
+    void *weights, *draft_weights, *kv, *draft_kv, *workspace, *state;
+} spec_buffers;
+
+/* Tensors addressable through spec_tensor. */
+enum {
+    /* target weights (arena `weights`); per-layer ones take the layer index */
+    SPEC_T_EMBED = 0, SPEC_T_LM_HEAD, SPEC_T_FINAL_NORM,
+    SPEC_T_ATTN_NORM, SPEC_T_WQKV, SPEC_T_WO, SPEC_T_MLP_NORM,
+    SPEC_T_WGATEUP,             /* [2*d_ffn][d]: gate rows, then up rows                              */
+    SPEC_T_WDOWN,
+    SPEC_T_ROUTER,              /* [n_experts][d]                                                      */
+    SPEC_T_EXPERTS_GATEUP,      /* [n_experts][2*d_expert_ffn][d]                                      */
+    SPEC_T_EXPERTS_DOWN,        /* [n_experts][d][d_expert_ffn]                                        */
+    /* draft head weights (arena `draft_weights`) */
+    SPEC_T_D_WFC = 32,          /* EAGLE3: [d][n_taps*d]                                               */
+    SPEC_T_D_WPROJ,             /* MTP: [d][2d] acting on concat(norm_g(g), norm_e(e))                 */
+    SPEC_T_D_NORM_E, SPEC_T_D_NORM_G, SPEC_T_D_NORM_F, SPEC_T_D_ATTN_NORM,
+    SPEC_T_D_WQKV,              /* EAGLE3: [(Hq+2Hkv)dh][2d] acting on concat(norm_e(e), norm_g(g))    */
+    SPEC_T_D_WO, SPEC_T_D_MLP_NORM, SPEC_T_D_WGATEUP, SPEC_T_D_WDOWN, SPEC_T_D_LM_HEAD,
+    /* caches: [block][n_kv_heads][kv_block_tokens][head_dim]; layer = pool index for the target */
+    SPEC_T_KV_K = 64, SPEC_T_KV_V, SPEC_T_DRAFT_KV_K, SPEC_T_DRAFT_KV_V,
+    /* state (int32) */
+    SPEC_T_SEQ_LEN = 96,        /* [max_batch] valid KV entries per sequence                           */
+    SPEC_T_LAST_TOKEN,          /* [max_batch] last committed token, not yet fed to the target         */
+    SPEC_T_BLOCK_TABLE,         /* [max_batch][max_blocks_per_seq], -1 = none                          */
+    SPEC_T_FREE_STACK,          /* [kv_num_blocks]                                                     */
+    SPEC_T_FREE_TOP,            /* [1] number of free blocks                                           */
+    SPEC_T_DRAFT_TOKENS,        /* [max_batch][k_max]                                                  */
+    SPEC_T_OUT_TOKENS,          /* [max_batch][k_max+1], -1 padded                                     */
+    SPEC_T_N_EMITTED,           /* [max_batch]                                                         */
+    SPEC_T_STATUS,              /* [4] device status word: code, detail, 0, 0                          */
+    SPEC_T_STEP,                /* [1] step counter = Philox counter word 0                            */
+    /* step results in the workspace */
+    SPEC_T_LOGITS = 128,        /* [B][k+1][vocab] fp32 target logits of the last verify               */
+    SPEC_T_DRAFT_LOGITS,        /* [B][k][vocab]   fp32 draft logits of the last draft                 */
+    SPEC_T_ROW_STATS,           /* [B*(k+1)][2] fp32 (max, sum exp) of the target rows                 */
+    SPEC_T_DRAFT_ROW_STATS,     /* [B*k][2]                                                            */
+    SPEC_T_TAPS,                /* [B][k+1][n_taps*d] tapped hidden states of the last verify          */
+    SPEC_T_HIDDEN               /* [B*(k+1)][d] fp32 residual stream after the last layer              */
+};
+
+/* Counters returned by spec_get_status (host struct). */
+typedef struct {
+    int32_t device_status;      /* SPEC_OK or the first device-detected error                          */
+    int32_t device_detail;      /* sequence index or row the error refers to                           */
+    int64_t steps;              /* commits since spec_seq_init                                         */
+    int64_t emitted_tokens;     /* sum over sequences and steps of n+1                                 */
+    int64_t accepted_drafts;    /* sum of n                                                            */
+} spec_step_report;
+
+/* ---- context -------------------------------------------------------------------------------------------- */
+
+/* Arena sizes for `cfg`.  Errors: INVALID_ARG (NULL, wrong struct_size/abi_version), SHAPE, UNSUPPORTED. */
+spec_status spec_query_sizes(const spec_config* cfg, spec_sizes* out);
+
+/* Builds a context over caller-owned arenas (nothing is copied or allocated on the device; the context
+ * itself is a small host object freed by spec_destroy).  The state arena must be zero-filled by the caller
+ * or initialised with spec_seq_init before the first step. */
+spec_status spec_create(const spec_config* cfg, const spec_buffers* buffers, spec_ctx** out);
+spec_status spec_destroy(spec_ctx* ctx);
+
+/* Address and byte size of a tensor inside the arenas, so the caller can write weights (also between
+ * steps: overwriting them in place is how refreshed policy weights reach the step, Section 2.3) or cache
+ * contents, and read results. */
+spec_status spec_tensor(spec_ctx* ctx, int tensor_id, int layer, void** dev_ptr, size_t* bytes);
+
+/* Starts B sequences: sequence b has seq_len_host[b] valid KV entries (the caller has filled or will fill
+ * them) and last token last_token_host[b].  free_stack_host[kv_num_blocks] is the initial order of the free
+ * stack (top = last element); blocks for the valid entries are popped in sequence order.  Resets the step
+ * counter.  Errors: INVALID_ARG, SHAPE (B > max_batch, a length that does not fit), KV exhaustion (SHAPE). */
+spec_status spec_seq_init(spec_ctx* ctx, int B, const int32_t* seq_len_host, const int32_t* last_token_host,
+                          const int32_t* free_stack_host, void* stream);
+
+/* ---- one speculation step (Introduction, third paragraph) ------------------------------------------------- */
+
+/* S1 draft propose.  Runs the draft head: pass 0 consumes the (tapped hidden state, next token) pairs of the
+ * positions committed by the previous step, passes 1..k-1 feed the head its own output; fills draft tokens
+ * d_1..d_k (d_i drawn from q_i with the stream-1 uniforms), draft logits and their row statistics.
+ * Errors: STATE (no committed step to draft from, draft_kind NONE), SHAPE (k outside 1..k_max). */
+spec_status spec_draft(spec_ctx* ctx, int k, void* stream);
+
+/* S2 target verify.  One forward over the k+1 tokens [last token, d_1..d_k] of every sequence at positions
+ * seq_len .. seq_len+k, causal among them, against the paged cache; appends their keys/values; writes the
+ * logits of all k+1 positions, their row statistics and the tapped hidden states.  k = 0 is plain decode.
+ * draft_tokens [B][k] overrides the context's draft tokens when not NULL (teacher forcing, external drafts). */
+spec_status spec_verify(spec_ctx* ctx, int k, const int32_t* draft_tokens, void* stream);
+
+/* S3+S4 fused vocabulary softmax and rejection sampling on the context's logits: accept_i = u_i <
+ * min(1, p_i(d_i)/q_i(d_i)); n = accepted prefix length; token n+1 from norm(max(0, p_{n+1}-q_{n+1})) or,
+ * when n = k, the bonus token from p_{k+1}; uniforms Philox(seed; step, sequence, slot 0..k, stream 0).
+ * draft_logits [B][k][vocab] overrides the context's draft logits when not NULL (draft_kind NONE). */
+spec_status spec_reject_sample(spec_ctx* ctx, int k, const float* draft_logits, void* stream);
+
+/* S5 KV commit / rollback: seq_len += n+1, blocks past the new length return to the free stack, the last
+ * token becomes the emitted token, the step counter advances.  force_n / force_token ([B] each, both or
+ * neither) replace the sampler's n and token: teacher-forced prefill through the verify path. */
+spec_status spec_kv_commit(spec_ctx* ctx, const int32_t* force_n, const int32_t* force_token, void* stream);
+
+/* Synchronises `stream`, reads the device status word and counters. */
+spec_status spec_get_status(spec_ctx* ctx, spec_step_report* host_out, void* stream);
+const char* spec_last_error(const spec_ctx* ctx);
+
+/* ---- stateless entry points (same kernels, no context) ------------------------------------------------------ */
+
+/* Row statistics and, optionally, probabilities of `rows` logit rows of width V:
+ * m = max_v l_v, Z = sum_v exp((l_v - m)/T), p_v = exp((l_v - m)/T)/Z.  stats [rows][2] = (m, Z) and probs
+ * [rows][V] may each be NULL. */
+spec_status spec_softmax_rows(int rows, int V, const float* logits, float temperature, float* stats,
+                              float* probs, void* stream);
+
+/* Draws one token per row from fp32 probabilities (not necessarily normalised) by inverse CDF with the
+ * uniform Philox(seed; step, row, slot, stream_tag); tokens [rows]. */
+spec_status spec_sample_rows(int rows, int V, const float* probs, uint64_t seed, uint32_t step, uint32_t slot,
+                             uint32_t stream_tag, int32_t* tokens, int32_t* status, void* stream);
+
+/* Rejection sampling on given probabilities: p [B][k+1][V], q [B][k][V], draft [B][k] ->
+ * out_tokens [B][k+1] (-1 padded), n_emitted [B] in 1..k+1.  status [4] int32 device status word (may be NULL). */
+spec_status spec_reject_sample_probs(int B, int k, int V, const float* p, const float* q, const int32_t* draft,
+                                     uint64_t seed, uint32_t step, int32_t* out_tokens, int32_t* n_emitted,
+                                     int32_t* status, void* stream);
+
+/* The same from logits and their row statistics (p_stats [B*(k+1)][2], q_stats [B*k][2]), probabilities
+ * formed on the fly and never written. */
+spec_status spec_reject_sample_logits(int B, int k, int V, const float* p_logits, const float* p_stats,
+                                      const float* q_logits, const float* q_stats, const int32_t* draft,
+                                      float temperature, uint64_t seed, uint32_t step, int32_t* out_tokens,
+                                      int32_t* n_emitted, int32_t* status, void* stream);
+
+/* Philox uniforms u [n_seq][n_slots] of (seed, step, stream_tag), as the sampler draws them. */
+spec_status spec_uniforms(uint64_t seed, uint32_t step, uint32_t stream_tag, int n_seq, int n_slots, float* u,
+                          void* stream);
+
+/* C[M][N] = A[M][K] * W[N][K]^T (+ C when accumulate != 0).  dtype_in selects bf16 (tensor-core path, fp32
+ * accumulation) or fp32 inputs; out_dtype the type of C.  All leading dimensions are the natural ones.
+ * bf16 requires K % 64 == 0 and N % 8 == 0. */
+spec_status spec_gemm(int M, int N, int K, const void* A, const void* W, void* C, int dtype_in, int out_dtype,
+                      int accumulate, void* stream);
+
+/* Paged attention of R = rows_per_seq query rows per sequence (query row i at position seq_len[b] + i sees
+ * cache positions <= seq_len[b] + i), grouped-query heads.  q [B][R][Hq][dh], out the same shape and type;
+ * k_pool / v_pool [blocks][Hkv][block_tokens][dh]; block_table [B][max_blocks]; scratch: see
+ * spec_attention_scratch_bytes. */
+spec_status spec_attention(int B, int R, int Hq, int Hkv, int dh, int block_tokens, int max_blocks,
+                           const void* q, const void* k_pool, const void* v_pool, const int32_t* block_table,
+                           const int32_t* seq_len, void* out, int dtype, void* scratch, size_t scratch_bytes,
+                           void* stream);
+size_t spec_attention_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int max_kv_len);
+
+/* Version string of the library build. */
+const char* spec_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPEC_H_ */

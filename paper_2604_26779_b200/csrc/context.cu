@@ -1,0 +1,564 @@
+// The context: arena layout over caller-owned device buffers and the host-side sequencing of one speculation step
+// (draft propose -> target verify -> fused softmax + rejection sampling -> KV commit).  Host code only enqueues
+// kernels; everything ragged (lengths, accepted counts, block tables) lives in device metadata, so a step is a fixed
+// sequence of launches.
+#include <string>
+#include <vector>
+
+#include "ops.cuh"
+
+struct Loc { size_t off = 0, bytes = 0; };
+
+struct LayerLoc { Loc attn_norm, wqkv, wo, mlp_norm, wgateup, wdown, router, exp_gateup, exp_down; };
+
+struct spec_ctx {
+    spec_config cfg;
+    spec_buffers buf;
+    int Mmax;                       // max_batch * (k_max + 1)
+    // weights
+    Loc embed, lm_head, final_norm;
+    std::vector<LayerLoc> layers;
+    size_t weights_bytes = 0;
+    // draft weights
+    Loc d_wfc, d_wproj, d_norm_e, d_norm_g, d_norm_f;
+    LayerLoc d_layer;
+    Loc d_lm_head;
+    size_t draft_weights_bytes = 0;
+    // caches
+    size_t kv_pool_bytes = 0, kv_bytes = 0, draft_kv_bytes = 0;
+    // state
+    Loc seq_len, last_token, block_table, free_stack, free_top, draft_tokens, out_tokens, n_emitted, status, step,
+        counters, pending_base;
+    size_t state_bytes = 0;
+    // workspace
+    Loc tokens_in, pos, x, h, qkv, attn_out, gu, act, logits, draft_logits, row_stats, draft_row_stats, taps,
+        attn_scratch, dg, dx, d_hidden, d_tok, d_pos;
+    size_t workspace_bytes = 0;
+    // host-side run state
+    int B = 0;
+    int k_last = -1;                // k of the last verify
+    bool have_pending = false;      // a commit has happened since spec_seq_init
+    bool verified = false;          // a verify has run since the last commit
+    std::string err;
+};
+
+using namespace spec;
+
+namespace {
+
+struct Arena {
+    size_t top = 0;
+    Loc take(size_t bytes) { Loc l{top, bytes}; top = align_up(top + bytes, 256); return l; }
+};
+
+bool has_tap(const spec_config& c, int t)
+{
+    for (int i = 0; i < c.n_taps; ++i) if (c.tap_layers[i] == t) return true;
+    return false;
+}
+int tap_slot(const spec_config& c, int t)
+{
+    for (int i = 0; i < c.n_taps; ++i) if (c.tap_layers[i] == t) return i;
+    return -1;
+}
+
+spec_status check_config(const spec_config* c)
+{
+    if (c == nullptr || c->struct_size != sizeof(spec_config) || c->abi_version != SPEC_ABI_VERSION) return SPEC_ERR_INVALID_ARG;
+    if (c->n_layers <= 0 || c->d_model <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->head_dim <= 0 || c->vocab <= 0)
+        return SPEC_ERR_SHAPE;
+    if (c->n_q_heads % c->n_kv_heads != 0 || c->d_model % 8 != 0 || c->head_dim % 8 != 0 || c->vocab % 4 != 0) return SPEC_ERR_SHAPE;
+    if (c->n_experts == 0 && (c->d_ffn <= 0 || c->d_ffn % 8 != 0)) return SPEC_ERR_SHAPE;
+    if (c->n_experts > 0 && (c->experts_top_k <= 0 || c->experts_top_k > c->n_experts || c->d_expert_ffn <= 0)) return SPEC_ERR_SHAPE;
+    if (c->n_experts > 0) return SPEC_ERR_UNSUPPORTED;
+    if (c->dtype != SPEC_DTYPE_BF16 && c->dtype != SPEC_DTYPE_F32) return SPEC_ERR_UNSUPPORTED;
+    if (c->draft_kind < SPEC_DRAFT_NONE || c->draft_kind > SPEC_DRAFT_MTP) return SPEC_ERR_UNSUPPORTED;
+    if (c->k_max < 0 || c->k_max > 7 || c->max_batch <= 0) return SPEC_ERR_SHAPE;
+    if (c->kv_block_tokens <= 0 || c->kv_num_blocks <= 0 || c->max_blocks_per_seq <= 0) return SPEC_ERR_SHAPE;
+    if (c->kv_layer_pools <= 0 || c->kv_layer_pools > c->n_layers) return SPEC_ERR_SHAPE;
+    if (c->n_taps < 0 || c->n_taps > 3) return SPEC_ERR_SHAPE;
+    for (int i = 0; i < c->n_taps; ++i) if (c->tap_layers[i] < 0 || c->tap_layers[i] > c->n_layers) return SPEC_ERR_SHAPE;
+    if (c->draft_kind == SPEC_DRAFT_EAGLE3 && (c->n_taps < 1 || c->draft_d_ffn <= 0)) return SPEC_ERR_SHAPE;
+    if (c->draft_kind == SPEC_DRAFT_MTP && (c->draft_d_ffn <= 0)) return SPEC_ERR_SHAPE;
+    if (!(c->temperature > 0.f) || !(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return SPEC_ERR_UNSUPPORTED;
+    if (c->vocab > sampler_max_vocab()) return SPEC_ERR_SHAPE;
+    return SPEC_OK;
+}
+
+void build_layout(spec_ctx& x)
+{
+    const spec_config& c = x.cfg;
+    const size_t es = dtype_bytes(c.dtype);
+    const size_t d = c.d_model, qkv_n = (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim, od = (size_t)c.n_q_heads * c.head_dim;
+    x.Mmax = c.max_batch * (c.k_max + 1);
+    {
+        Arena a;
+        x.embed = a.take((size_t)c.vocab * d * es);
+        x.lm_head = a.take((size_t)c.vocab * d * es);
+        x.final_norm = a.take(d * 4);
+        x.layers.resize(c.n_layers);
+        for (auto& L : x.layers) {
+            L.attn_norm = a.take(d * 4);
+            L.wqkv = a.take(qkv_n * d * es);
+            L.wo = a.take(d * od * es);
+            L.mlp_norm = a.take(d * 4);
+            if (c.n_experts > 0) {
+                L.router = a.take((size_t)c.n_experts * d * es);
+                L.exp_gateup = a.take((size_t)c.n_experts * 2 * c.d_expert_ffn * d * es);
+                L.exp_down = a.take((size_t)c.n_experts * d * c.d_expert_ffn * es);
+            } else {
+                L.wgateup = a.take((size_t)2 * c.d_ffn * d * es);
+                L.wdown = a.take(d * (size_t)c.d_ffn * es);
+            }
+        }
+        x.weights_bytes = a.top;
+    }
+    {
+        Arena a;
+        if (c.draft_kind != SPEC_DRAFT_NONE) {
+            const size_t F = c.draft_d_ffn;
+            x.d_norm_e = a.take(d * 4);
+            x.d_norm_g = a.take(d * 4);
+            x.d_layer.mlp_norm = a.take(d * 4);
+            x.d_layer.wo = a.take(d * od * es);
+            x.d_layer.wgateup = a.take(2 * F * d * es);
+            x.d_layer.wdown = a.take(d * F * es);
+            if (c.draft_kind == SPEC_DRAFT_EAGLE3) {
+                x.d_wfc = a.take(d * (size_t)c.n_taps * d * es);
+                x.d_norm_f = a.take(d * 4);
+                x.d_layer.wqkv = a.take(qkv_n * 2 * d * es);
+                x.d_lm_head = a.take((size_t)c.vocab * d * es);
+            } else {
+                x.d_wproj = a.take(d * 2 * d * es);
+                x.d_layer.attn_norm = a.take(d * 4);
+                x.d_layer.wqkv = a.take(qkv_n * d * es);
+            }
+        }
+        x.draft_weights_bytes = a.top;
+    }
+    x.kv_pool_bytes = align_up((size_t)c.kv_num_blocks * c.n_kv_heads * c.kv_block_tokens * c.head_dim * es, 256);
+    x.kv_bytes = x.kv_pool_bytes * 2 * c.kv_layer_pools;
+    x.draft_kv_bytes = c.draft_kind != SPEC_DRAFT_NONE ? x.kv_pool_bytes * 2 : 0;
+    {
+        Arena a;
+        const size_t Bm = c.max_batch;
+        x.seq_len = a.take(Bm * 4);
+        x.last_token = a.take(Bm * 4);
+        x.block_table = a.take(Bm * c.max_blocks_per_seq * 4);
+        x.free_stack = a.take((size_t)c.kv_num_blocks * 4);
+        x.free_top = a.take(4);
+        x.draft_tokens = a.take(Bm * (size_t)(c.k_max > 0 ? c.k_max : 1) * 4);
+        x.out_tokens = a.take(Bm * (c.k_max + 1) * 4);
+        x.n_emitted = a.take(Bm * 4);
+        x.status = a.take(16);
+        x.step = a.take(4);
+        x.counters = a.take(3 * 8);
+        x.pending_base = a.take(Bm * 4);
+        x.state_bytes = a.top;
+    }
+    {
+        Arena a;
+        const size_t M = x.Mmax, Bm = c.max_batch;
+        const size_t Fmax = (size_t)(c.d_ffn > c.draft_d_ffn ? c.d_ffn : c.draft_d_ffn);
+        x.tokens_in = a.take(M * 4);
+        x.pos = a.take(M * 4);
+        x.x = a.take(M * d * 4);
+        x.h = a.take(M * 2 * d * es);
+        x.qkv = a.take(M * qkv_n * es);
+        x.attn_out = a.take(M * od * es);
+        x.gu = a.take(M * 2 * Fmax * es);
+        x.act = a.take(M * Fmax * es);
+        x.logits = a.take(M * (size_t)c.vocab * 4);
+        x.draft_logits = a.take(Bm * (size_t)(c.k_max > 0 ? c.k_max : 1) * c.vocab * 4);
+        x.row_stats = a.take(M * 8);
+        x.draft_row_stats = a.take(Bm * (size_t)(c.k_max > 0 ? c.k_max : 1) * 8);
+        x.taps = a.take(M * (size_t)(c.n_taps > 0 ? c.n_taps : 1) * d * es);
+        x.attn_scratch = a.take(attention_scratch_bytes(c.max_batch, c.k_max + 1, c.n_q_heads, c.n_kv_heads, c.head_dim,
+                                                        c.max_blocks_per_seq * c.kv_block_tokens));
+        x.dg = a.take(M * d * 4);
+        x.dx = a.take(M * d * 4);
+        x.d_hidden = a.take(Bm * d * 4);
+        x.d_tok = a.take(M * 4);
+        x.d_pos = a.take(M * 4);
+        x.workspace_bytes = a.top;
+    }
+}
+
+template <class T = void> T* at(void* base, const Loc& l) { return reinterpret_cast<T*>(static_cast<char*>(base) + l.off); }
+
+struct LayerPtrs { const float* attn_norm; const void* wqkv; const void* wo; const float* mlp_norm; const void* wgateup; const void* wdown; };
+
+LayerPtrs layer_ptrs(void* base, const LayerLoc& L)
+{
+    return {at<const float>(base, L.attn_norm), at<const void>(base, L.wqkv), at<const void>(base, L.wo),
+            at<const float>(base, L.mlp_norm), at<const void>(base, L.wgateup), at<const void>(base, L.wdown)};
+}
+
+#define TRY(expr) do { spec_status s__ = (expr); if (s__ != SPEC_OK) return s__; } while (0)
+
+// attention + MLP of one decoder layer on the fp32 residual `res` [M][d].  `qkv_in` [M][qkv_k] is the already
+// prepared input of the QKV projection.
+spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* res, const void* qkv_in, int qkv_k, int B, int R,
+                           const int32_t* pos, void* k_pool, void* v_pool, cudaStream_t st)
+{
+    const spec_config& g = c.cfg;
+    const int M = B * R, d = g.d_model, dh = g.head_dim, Hq = g.n_q_heads, Hkv = g.n_kv_heads;
+    const int qkv_n = (Hq + 2 * Hkv) * dh, dt = g.dtype;
+    void* ws = c.buf.workspace;
+    TRY(launch_gemm(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt, 0, st));
+    TRY(launch_rope_append(B, R, Hq, Hkv, dh, g.rope_theta, at(ws, c.qkv), pos, k_pool, v_pool,
+                           at<int32_t>(c.buf.state, c.block_table), g.max_blocks_per_seq, g.kv_block_tokens, dt, st));
+    AttnArgs a{B, R, Hq, Hkv, dh, g.kv_block_tokens, g.max_blocks_per_seq, at(ws, c.qkv), qkv_n, k_pool, v_pool,
+               at<int32_t>(c.buf.state, c.block_table), pos, at(ws, c.attn_out), Hq * dh, dt, at(ws, c.attn_scratch),
+               c.attn_scratch.bytes, g.max_blocks_per_seq * g.kv_block_tokens};
+    TRY(launch_attention(a, st));
+    TRY(launch_gemm(M, d, Hq * dh, at(ws, c.attn_out), Hq * dh, W.wo, res, d, dt, SPEC_DTYPE_F32, 1, st));
+    TRY(launch_rmsnorm(M, d, res, W.mlp_norm, g.rms_eps, at(ws, c.h), d, 0, dt, st));
+    TRY(launch_gemm(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.gu), 2 * d_ffn, dt, dt, 0, st));
+    TRY(launch_swiglu(M, d_ffn, at(ws, c.gu), at(ws, c.act), dt, st));
+    TRY(launch_gemm(M, d, d_ffn, at(ws, c.act), d_ffn, W.wdown, res, d, dt, SPEC_DTYPE_F32, 1, st));
+    return SPEC_OK;
+}
+
+__global__ void draft_rows0_kernel(int B, int R, const int32_t* n_emitted, const int32_t* pending_base,
+                                   const int32_t* out_tokens, int32_t* tok, int32_t* pos)
+{
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= B * R) return;
+    const int b = m / R, i = m % R;
+    const bool valid = i < n_emitted[b];
+    pos[m] = valid ? pending_base[b] + i : -1;
+    tok[m] = valid ? out_tokens[m] : -1;
+}
+
+__global__ void draft_rows_kernel(int B, int j, const int32_t* seq_len, const int32_t* draft_tokens, int stride,
+                                  int32_t* tok, int32_t* pos)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    pos[b] = seq_len[b] - 1 + j;
+    tok[b] = draft_tokens[(size_t)b * stride + j - 1];
+}
+
+}  // namespace
+
+extern "C" spec_status spec_query_sizes(const spec_config* cfg, spec_sizes* out)
+{
+    if (out == nullptr) return SPEC_ERR_INVALID_ARG;
+    TRY(check_config(cfg));
+    spec_ctx tmp;
+    tmp.cfg = *cfg;
+    build_layout(tmp);
+    out->weights_bytes = tmp.weights_bytes;
+    out->draft_weights_bytes = tmp.draft_weights_bytes;
+    out->kv_bytes = tmp.kv_bytes;
+    out->draft_kv_bytes = tmp.draft_kv_bytes;
+    out->workspace_bytes = tmp.workspace_bytes;
+    out->state_bytes = tmp.state_bytes;
+    return SPEC_OK;
+}
+
+extern "C" spec_status spec_create(const spec_config* cfg, const spec_buffers* b, spec_ctx** out)
+{
+    if (out == nullptr || b == nullptr) return SPEC_ERR_INVALID_ARG;
+    TRY(check_config(cfg));
+    if (!b->weights || !b->kv || !b->workspace || !b->state) return SPEC_ERR_INVALID_ARG;
+    if (cfg->draft_kind != SPEC_DRAFT_NONE && (!b->draft_weights || !b->draft_kv)) return SPEC_ERR_INVALID_ARG;
+    const void* ptrs[] = {b->weights, b->draft_weights, b->kv, b->draft_kv, b->workspace, b->state};
+    for (const void* p : ptrs) if ((reinterpret_cast<uintptr_t>(p) & 255u) != 0) return SPEC_ERR_INVALID_ARG;
+    spec_ctx* c = new spec_ctx();
+    c->cfg = *cfg;
+    c->buf = *b;
+    build_layout(*c);
+    *out = c;
+    return SPEC_OK;
+}
+
+extern "C" spec_status spec_destroy(spec_ctx* ctx)
+{
+    if (ctx == nullptr) return SPEC_ERR_INVALID_ARG;
+    delete ctx;
+    return SPEC_OK;
+}
+
+extern "C" const char* spec_last_error(const spec_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+extern "C" const char* spec_version(void) { return "spec-step 0.1 (sm_100a)"; }
+
+extern "C" spec_status spec_tensor(spec_ctx* c, int id, int layer, void** dev_ptr, size_t* bytes)
+{
+    if (c == nullptr || dev_ptr == nullptr || bytes == nullptr) return SPEC_ERR_INVALID_ARG;
+    const spec_config& g = c->cfg;
+    void* base = nullptr;
+    Loc l;
+    auto layer_ok = [&]() { return layer >= 0 && layer < g.n_layers; };
+    switch (id) {
+    case SPEC_T_EMBED: base = c->buf.weights; l = c->embed; break;
+    case SPEC_T_LM_HEAD: base = c->buf.weights; l = c->lm_head; break;
+    case SPEC_T_FINAL_NORM: base = c->buf.weights; l = c->final_norm; break;
+    case SPEC_T_ATTN_NORM: case SPEC_T_WQKV: case SPEC_T_WO: case SPEC_T_MLP_NORM: case SPEC_T_WGATEUP: case SPEC_T_WDOWN:
+    case SPEC_T_ROUTER: case SPEC_T_EXPERTS_GATEUP: case SPEC_T_EXPERTS_DOWN: {
+        if (!layer_ok()) return SPEC_ERR_INVALID_ARG;
+        const LayerLoc& L = c->layers[layer];
+        base = c->buf.weights;
+        l = id == SPEC_T_ATTN_NORM ? L.attn_norm : id == SPEC_T_WQKV ? L.wqkv : id == SPEC_T_WO ? L.wo :
+            id == SPEC_T_MLP_NORM ? L.mlp_norm : id == SPEC_T_WGATEUP ? L.wgateup : id == SPEC_T_WDOWN ? L.wdown :
+            id == SPEC_T_ROUTER ? L.router : id == SPEC_T_EXPERTS_GATEUP ? L.exp_gateup : L.exp_down;
+        break;
+    }
+    case SPEC_T_D_WFC: base = c->buf.draft_weights; l = c->d_wfc; break;
+    case SPEC_T_D_WPROJ: base = c->buf.draft_weights; l = c->d_wproj; break;
+    case SPEC_T_D_NORM_E: base = c->buf.draft_weights; l = c->d_norm_e; break;
+    case SPEC_T_D_NORM_G: base = c->buf.draft_weights; l = c->d_norm_g; break;
+    case SPEC_T_D_NORM_F: base = c->buf.draft_weights; l = c->d_norm_f; break;
+    case SPEC_T_D_ATTN_NORM: base = c->buf.draft_weights; l = c->d_layer.attn_norm; break;
+    case SPEC_T_D_WQKV: base = c->buf.draft_weights; l = c->d_layer.wqkv; break;
+    case SPEC_T_D_WO: base = c->buf.draft_weights; l = c->d_layer.wo; break;
+    case SPEC_T_D_MLP_NORM: base = c->buf.draft_weights; l = c->d_layer.mlp_norm; break;
+    case SPEC_T_D_WGATEUP: base = c->buf.draft_weights; l = c->d_layer.wgateup; break;
+    case SPEC_T_D_WDOWN: base = c->buf.draft_weights; l = c->d_layer.wdown; break;
+    case SPEC_T_D_LM_HEAD: base = c->buf.draft_weights; l = c->d_lm_head; break;
+    case SPEC_T_KV_K: case SPEC_T_KV_V:
+        if (layer < 0 || layer >= g.kv_layer_pools) return SPEC_ERR_INVALID_ARG;
+        base = c->buf.kv;
+        l = Loc{((size_t)layer * 2 + (id == SPEC_T_KV_V ? 1 : 0)) * c->kv_pool_bytes, c->kv_pool_bytes};
+        break;
+    case SPEC_T_DRAFT_KV_K: case SPEC_T_DRAFT_KV_V:
+        if (g.draft_kind == SPEC_DRAFT_NONE) return SPEC_ERR_INVALID_ARG;
+        base = c->buf.draft_kv;
+        l = Loc{(id == SPEC_T_DRAFT_KV_V ? 1 : 0) * c->kv_pool_bytes, c->kv_pool_bytes};
+        break;
+    case SPEC_T_SEQ_LEN: base = c->buf.state; l = c->seq_len; break;
+    case SPEC_T_LAST_TOKEN: base = c->buf.state; l = c->last_token; break;
+    case SPEC_T_BLOCK_TABLE: base = c->buf.state; l = c->block_table; break;
+    case SPEC_T_FREE_STACK: base = c->buf.state; l = c->free_stack; break;
+    case SPEC_T_FREE_TOP: base = c->buf.state; l = c->free_top; break;
+    case SPEC_T_DRAFT_TOKENS: base = c->buf.state; l = c->draft_tokens; break;
+    case SPEC_T_OUT_TOKENS: base = c->buf.state; l = c->out_tokens; break;
+    case SPEC_T_N_EMITTED: base = c->buf.state; l = c->n_emitted; break;
+    case SPEC_T_STATUS: base = c->buf.state; l = c->status; break;
+    case SPEC_T_STEP: base = c->buf.state; l = c->step; break;
+    case SPEC_T_LOGITS: base = c->buf.workspace; l = c->logits; break;
+    case SPEC_T_DRAFT_LOGITS: base = c->buf.workspace; l = c->draft_logits; break;
+    case SPEC_T_ROW_STATS: base = c->buf.workspace; l = c->row_stats; break;
+    case SPEC_T_DRAFT_ROW_STATS: base = c->buf.workspace; l = c->draft_row_stats; break;
+    case SPEC_T_TAPS: base = c->buf.workspace; l = c->taps; break;
+    case SPEC_T_HIDDEN: base = c->buf.workspace; l = c->x; break;
+    default: return SPEC_ERR_INVALID_ARG;
+    }
+    if (base == nullptr || l.bytes == 0) return SPEC_ERR_INVALID_ARG;
+    *dev_ptr = static_cast<char*>(base) + l.off;
+    *bytes = l.bytes;
+    return SPEC_OK;
+}
+
+extern "C" spec_status spec_seq_init(spec_ctx* c, int B, const int32_t* seq_len_host, const int32_t* last_token_host,
+                                     const int32_t* free_stack_host, void* stream)
+{
+    if (c == nullptr || B < 0 || (B > 0 && (!seq_len_host || !last_token_host)) || !free_stack_host) return SPEC_ERR_INVALID_ARG;
+    const spec_config& g = c->cfg;
+    if (B > g.max_batch) return SPEC_ERR_SHAPE;
+    const int bt = g.kv_block_tokens, mb = g.max_blocks_per_seq, nb = g.kv_num_blocks;
+    std::vector<int32_t> table((size_t)g.max_batch * mb, -1), stack(free_stack_host, free_stack_host + nb);
+    std::vector<char> seen(nb, 0);
+    for (int i = 0; i < nb; ++i) {
+        if (stack[i] < 0 || stack[i] >= nb || seen[stack[i]]) return SPEC_ERR_INVALID_ARG;
+        seen[stack[i]] = 1;
+    }
+    int top = nb;
+    for (int b = 0; b < B; ++b) {
+        if (seq_len_host[b] < 0 || last_token_host[b] < 0 || last_token_host[b] >= g.vocab) return SPEC_ERR_INVALID_ARG;
+        const int need = (seq_len_host[b] + bt - 1) / bt;
+        if (need > mb || (seq_len_host[b] + g.k_max + 1 + bt - 1) / bt > mb) return SPEC_ERR_SHAPE;
+        if (need > top) return SPEC_ERR_SHAPE;
+        for (int j = 0; j < need; ++j) table[(size_t)b * mb + j] = stack[--top];
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    char* sb = static_cast<char*>(c->buf.state);
+    SPEC_CUDA_OK(cudaMemsetAsync(sb, 0, c->state_bytes, st));
+    SPEC_CUDA_OK(cudaMemcpyAsync(sb + c->seq_len.off, seq_len_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_OK(cudaMemcpyAsync(sb + c->last_token.off, last_token_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_OK(cudaMemcpyAsync(sb + c->block_table.off, table.data(), table.size() * 4, cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_OK(cudaMemcpyAsync(sb + c->free_stack.off, stack.data(), (size_t)nb * 4, cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_OK(cudaMemcpyAsync(sb + c->free_top.off, &top, 4, cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_OK(cudaStreamSynchronize(st));          // the host staging vectors go out of scope here
+    c->B = B;
+    c->k_last = -1;
+    c->have_pending = false;
+    c->verified = false;
+    return SPEC_OK;
+}
+
+extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_tokens, void* stream)
+{
+    if (c == nullptr) return SPEC_ERR_INVALID_ARG;
+    const spec_config& g = c->cfg;
+    if (k < 0 || k > g.k_max) return SPEC_ERR_SHAPE;
+    if (k > 0 && draft_tokens == nullptr && g.draft_kind == SPEC_DRAFT_NONE) return SPEC_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int B = c->B, R = k + 1, M = B * R, d = g.d_model, dt = g.dtype;
+    if (B == 0) return SPEC_OK;
+    void* ws = c->buf.workspace;
+    char* sb = static_cast<char*>(c->buf.state);
+    int32_t* status = at<int32_t>(sb, c->status);
+    int32_t* seq_len = at<int32_t>(sb, c->seq_len);
+    TRY(launch_kv_reserve(B, k, g.kv_block_tokens, g.max_blocks_per_seq, seq_len, at<int32_t>(sb, c->block_table),
+                          at<int32_t>(sb, c->free_stack), at<int32_t>(sb, c->free_top), status, st));
+    StepRows rows{at<int32_t>(ws, c->tokens_in), at<int32_t>(ws, c->pos)};
+    const int32_t* dtok = draft_tokens ? draft_tokens : at<int32_t>(sb, c->draft_tokens);
+    const int dstride = draft_tokens ? k : (g.k_max > 0 ? g.k_max : 1);
+    TRY(launch_verify_rows(B, R, seq_len, at<int32_t>(sb, c->last_token), dtok, dstride, g.vocab, rows, status, st));
+    float* x = at<float>(ws, c->x);
+    TRY(launch_embed(M, d, at(c->buf.weights, c->embed), dt, rows.token, x, st));
+    const int tapw = g.n_taps * d;
+    if (has_tap(g, 0)) TRY(launch_copy_rows_f32_to(M, d, x, at(ws, c->taps), tapw, tap_slot(g, 0) * d, dt, st));
+    for (int l = 0; l < g.n_layers; ++l) {
+        const LayerPtrs W = layer_ptrs(c->buf.weights, c->layers[l]);
+        TRY(launch_rmsnorm(M, d, x, W.attn_norm, g.rms_eps, at(ws, c->h), d, 0, dt, st));
+        const int pool = l % g.kv_layer_pools;
+        char* kp = static_cast<char*>(c->buf.kv) + (size_t)pool * 2 * c->kv_pool_bytes;
+        TRY(run_layer_body(*c, W, g.d_ffn, x, at(ws, c->h), d, B, R, rows.pos, kp, kp + c->kv_pool_bytes, st));
+        if (has_tap(g, l + 1)) TRY(launch_copy_rows_f32_to(M, d, x, at(ws, c->taps), tapw, tap_slot(g, l + 1) * d, dt, st));
+    }
+    TRY(launch_rmsnorm(M, d, x, at<const float>(c->buf.weights, c->final_norm), g.rms_eps, at(ws, c->h), d, 0, dt, st));
+    TRY(launch_gemm(M, g.vocab, d, at(ws, c->h), d, at(c->buf.weights, c->lm_head), at(ws, c->logits), g.vocab, dt,
+                    SPEC_DTYPE_F32, 0, st));
+    TRY(launch_softmax_rows(M, g.vocab, at<float>(ws, c->logits), (size_t)g.vocab, g.temperature, at<float>(ws, c->row_stats),
+                            1, nullptr, st));
+    c->k_last = k;
+    c->verified = true;
+    return SPEC_OK;
+}
+
+extern "C" spec_status spec_reject_sample(spec_ctx* c, int k, const float* draft_logits, void* stream)
+{
+    if (c == nullptr) return SPEC_ERR_INVALID_ARG;
+    const spec_config& g = c->cfg;
+    if (!c->verified || k != c->k_last) return SPEC_ERR_STATE;
+    if (k > 0 && draft_logits == nullptr && g.draft_kind == SPEC_DRAFT_NONE) return SPEC_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int B = c->B;
+    if (B == 0) return SPEC_OK;
+    void* ws = c->buf.workspace;
+    char* sb = static_cast<char*>(c->buf.state);
+    const float* ql = draft_logits ? draft_logits : at<float>(ws, c->draft_logits);
+    float* qs = at<float>(ws, c->draft_row_stats);
+    if (draft_logits != nullptr && k > 0)
+        TRY(launch_softmax_rows(B * k, g.vocab, ql, (size_t)g.vocab, g.temperature, qs, 1, nullptr, st));
+    // draft tokens: those the verify used (rows 1..k of its token list), so an external draft stays consistent
+    return launch_reject_sample(true, B, k, g.vocab, at<float>(ws, c->logits), at<float>(ws, c->row_stats), ql, qs,
+                                at<int32_t>(ws, c->tokens_in) + 1, k + 1, g.temperature, g.seed, at<uint32_t>(sb, c->step), 0, at<int32_t>(sb, c->out_tokens),
+                                at<int32_t>(sb, c->n_emitted), at<int32_t>(sb, c->status), st);
+}
+
+extern "C" spec_status spec_kv_commit(spec_ctx* c, const int32_t* force_n, const int32_t* force_token, void* stream)
+{
+    if (c == nullptr || (force_n == nullptr) != (force_token == nullptr)) return SPEC_ERR_INVALID_ARG;
+    if (!c->verified) return SPEC_ERR_STATE;
+    const spec_config& g = c->cfg;
+    char* sb = static_cast<char*>(c->buf.state);
+    CommitArgs a{};
+    a.B = c->B; a.k = c->k_last; a.block_tokens = g.kv_block_tokens; a.max_blocks = g.max_blocks_per_seq;
+    a.force_n = force_n; a.force_token = force_token;
+    a.verify_tokens = at<int32_t>(c->buf.workspace, c->tokens_in);
+    a.n_emitted = at<int32_t>(sb, c->n_emitted);
+    a.out_tokens = at<int32_t>(sb, c->out_tokens);
+    a.seq_len = at<int32_t>(sb, c->seq_len);
+    a.last_token = at<int32_t>(sb, c->last_token);
+    a.block_table = at<int32_t>(sb, c->block_table);
+    a.free_stack = at<int32_t>(sb, c->free_stack);
+    a.free_top = at<int32_t>(sb, c->free_top);
+    a.pending_base = at<int32_t>(sb, c->pending_base);
+    a.step = at<uint32_t>(sb, c->step);
+    a.counters = at<long long>(sb, c->counters);
+    a.status = at<int32_t>(sb, c->status);
+    TRY(launch_kv_commit(a, (cudaStream_t)stream));
+    c->verified = false;
+    c->have_pending = true;
+    return SPEC_OK;
+}
+
+extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
+{
+    if (c == nullptr) return SPEC_ERR_INVALID_ARG;
+    const spec_config& g = c->cfg;
+    if (g.draft_kind == SPEC_DRAFT_NONE || !c->have_pending || c->verified) return SPEC_ERR_STATE;
+    if (k < 1 || k > g.k_max) return SPEC_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int B = c->B, d = g.d_model, dt = g.dtype, V = g.vocab;
+    if (B == 0) return SPEC_OK;
+    void* ws = c->buf.workspace;
+    void* dw = c->buf.draft_weights;
+    char* sb = static_cast<char*>(c->buf.state);
+    int32_t* status = at<int32_t>(sb, c->status);
+    int32_t* seq_len = at<int32_t>(sb, c->seq_len);
+    const bool eagle = g.draft_kind == SPEC_DRAFT_EAGLE3;
+    TRY(launch_kv_reserve(B, k, g.kv_block_tokens, g.max_blocks_per_seq, seq_len, at<int32_t>(sb, c->block_table),
+                          at<int32_t>(sb, c->free_stack), at<int32_t>(sb, c->free_top), status, st));
+    const LayerPtrs W = layer_ptrs(dw, c->d_layer);
+    char* kp = static_cast<char*>(c->buf.draft_kv);
+    char* vp = kp + c->kv_pool_bytes;
+    int32_t* tok = at<int32_t>(ws, c->d_tok);
+    int32_t* pos = at<int32_t>(ws, c->d_pos);
+    float* dg = at<float>(ws, c->dg);
+    float* dx = at<float>(ws, c->dx);
+    float* hid = at<float>(ws, c->d_hidden);
+    float* dlog = at<float>(ws, c->draft_logits);
+    float* dstats = at<float>(ws, c->draft_row_stats);
+    int32_t* dtoks = at<int32_t>(sb, c->draft_tokens);
+    const int kstride = g.k_max;
+
+    for (int j = 0; j < k; ++j) {
+        const int R = j == 0 ? c->k_last + 1 : 1;
+        const int M = B * R;
+        float* res = j == 0 ? dg : hid;                 // residual stream of this pass
+        if (j == 0) draft_rows0_kernel<<<(M + 255) / 256, 256, 0, st>>>(B, R, at<int32_t>(sb, c->n_emitted), at<int32_t>(sb, c->pending_base),
+                                                                        at<int32_t>(sb, c->out_tokens), tok, pos);
+        else        draft_rows_kernel<<<(B + 255) / 256, 256, 0, st>>>(B, j, seq_len, dtoks, kstride, tok, pos);
+        TRY(launch_status());
+        TRY(launch_embed(M, d, at(c->buf.weights, c->embed), dt, tok, dx, st));
+        if (eagle) {
+            // a = concat(norm_e(e), norm_g(g)); g = W_fc taps (true slots) or the head's previous output
+            if (j == 0) TRY(launch_gemm(M, d, g.n_taps * d, at(ws, c->taps), g.n_taps * d, at(dw, c->d_wfc), dg, d, dt, SPEC_DTYPE_F32, 0, st));
+            TRY(launch_rmsnorm(M, d, dx, at<const float>(dw, c->d_norm_e), g.rms_eps, at(ws, c->h), 2 * d, 0, dt, st));
+            TRY(launch_rmsnorm(M, d, res, at<const float>(dw, c->d_norm_g), g.rms_eps, at(ws, c->h), 2 * d, d, dt, st));
+            TRY(run_layer_body(*c, W, g.draft_d_ffn, res, at(ws, c->h), 2 * d, B, R, pos, kp, vp, st));
+        } else {
+            // h0 = W_proj concat(norm_g(g), norm_e(e)); g = the target's last-layer residual or the head's previous output
+            const float* gsrc = j == 0 ? at<float>(ws, c->x) : hid;
+            TRY(launch_rmsnorm(M, d, gsrc, at<const float>(dw, c->d_norm_g), g.rms_eps, at(ws, c->h), 2 * d, 0, dt, st));
+            TRY(launch_rmsnorm(M, d, dx, at<const float>(dw, c->d_norm_e), g.rms_eps, at(ws, c->h), 2 * d, d, dt, st));
+            TRY(launch_gemm(M, d, 2 * d, at(ws, c->h), 2 * d, at(dw, c->d_wproj), res, d, dt, SPEC_DTYPE_F32, 0, st));
+            TRY(launch_rmsnorm(M, d, res, W.attn_norm, g.rms_eps, at(ws, c->h), d, 0, dt, st));
+            TRY(run_layer_body(*c, W, g.draft_d_ffn, res, at(ws, c->h), d, B, R, pos, kp, vp, st));
+        }
+        if (j == 0) TRY(launch_gather_last_rows(B, R, d, dg, at<int32_t>(sb, c->n_emitted), hid, st));
+        // logits of this slot, their statistics, and the draft token d_{j+1} ~ q_{j+1} (stream-1 uniform, slot j)
+        const float* nf = eagle ? at<const float>(dw, c->d_norm_f) : at<const float>(c->buf.weights, c->final_norm);
+        const void* lm = eagle ? at<const void>(dw, c->d_lm_head) : at<const void>(c->buf.weights, c->lm_head);
+        TRY(launch_rmsnorm(B, d, hid, nf, g.rms_eps, at(ws, c->h), d, 0, dt, st));
+        TRY(launch_gemm(B, V, d, at(ws, c->h), d, lm, dlog + (size_t)j * V, k * V, dt, SPEC_DTYPE_F32, 0, st));
+        TRY(launch_softmax_rows(B, V, dlog + (size_t)j * V, (size_t)k * V, g.temperature, dstats + 2 * j, k, nullptr, st));
+        TRY(launch_sample_logits(B, V, dlog + (size_t)j * V, (size_t)k * V, dstats + 2 * j, k, g.temperature, g.seed,
+                                 at<uint32_t>(sb, c->step), (uint32_t)j, 1u, dtoks + j, kstride, status, st));
+    }
+    return SPEC_OK;
+}
+
+extern "C" spec_status spec_get_status(spec_ctx* c, spec_step_report* out, void* stream)
+{
+    if (c == nullptr || out == nullptr) return SPEC_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    SPEC_CUDA_OK(cudaStreamSynchronize(st));
+    char* sb = static_cast<char*>(c->buf.state);
+    int32_t status[4];
+    long long counters[3];
+    SPEC_CUDA_OK(cudaMemcpy(status, sb + c->status.off, sizeof(status), cudaMemcpyDeviceToHost));
+    SPEC_CUDA_OK(cudaMemcpy(counters, sb + c->counters.off, sizeof(counters), cudaMemcpyDeviceToHost));
+    out->device_status = status[0];
+    out->device_detail = status[1];
+    out->steps = counters[0];
+    out->emitted_tokens = counters[1];
+    out->accepted_drafts = counters[2];
+    return SPEC_OK;
+}

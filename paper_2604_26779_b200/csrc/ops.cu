@@ -1,0 +1,399 @@
+// Element-wise, gather/scatter and bookkeeping kernels of the verify and draft forwards: row metadata, embedding
+// gather, RMSNorm, rotary embedding + paged KV append, SwiGLU, tap copies, and the paged-KV reserve / commit pass
+// (step S5: keep the accepted slots, return the blocks of rejected ones).  All HBM-bound and small next to the
+// attention and GEMM passes; written for coalesced 16-byte accesses where the row width allows.
+#include "ops.cuh"
+
+namespace spec {
+namespace {
+
+template <class T> struct Vec4;     // 4 elements loaded/stored as one access
+template <> struct Vec4<float> {
+    static __device__ __forceinline__ void load(const float* p, float (&v)[4])
+    {
+        const float4 t = *reinterpret_cast<const float4*>(p);
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
+    static __device__ __forceinline__ void store(float* p, const float (&v)[4])
+    {
+        *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+};
+template <> struct Vec4<__nv_bfloat16> {
+    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[4])
+    {
+        const uint2 t = *reinterpret_cast<const uint2*>(p);
+        const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&t.x);
+        const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&t.y);
+        v[0] = __low2float(a); v[1] = __high2float(a); v[2] = __low2float(b); v[3] = __high2float(b);
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&v)[4])
+    {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+        uint2 t;
+        t.x = *reinterpret_cast<uint32_t*>(&a);
+        t.y = *reinterpret_cast<uint32_t*>(&b);
+        *reinterpret_cast<uint2*>(p) = t;
+    }
+};
+
+// ---- row metadata of a verify forward: tokens [last, d_1..d_k] at positions len .. len+k --------------------------
+__global__ void verify_rows_kernel(int B, int R, const int32_t* seq_len, const int32_t* last_token,
+                                   const int32_t* draft, int draft_stride, int vocab, StepRows rows, int32_t* status)
+{
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= B * R) return;
+    const int b = m / R, i = m % R;
+    int tok = (i == 0) ? last_token[b] : draft[(size_t)b * draft_stride + i - 1];
+    if (tok < 0 || tok >= vocab) { set_status(status, SPEC_ERR_TOKEN_RANGE, b); tok = 0; }
+    rows.token[m] = tok;
+    rows.pos[m] = seq_len[b] + i;
+}
+
+template <class T>
+__global__ void embed_kernel(int d, const T* __restrict__ table, const int32_t* __restrict__ token, float* __restrict__ x)
+{
+    const int m = blockIdx.x;
+    const int tok = token[m];
+    float* xr = x + (size_t)m * d;
+    for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
+        if (tok >= 0) Vec4<T>::load(table + (size_t)tok * d + c, v);
+        Vec4<float>::store(xr + c, v);
+    }
+}
+
+template <class T>
+__global__ void __launch_bounds__(256) rmsnorm_kernel(int d, const float* __restrict__ in, const float* __restrict__ w,
+                                                      float eps, T* __restrict__ out, int ld_out, int col0)
+{
+    const int m = blockIdx.x;
+    const float* xr = in + (size_t)m * d;
+    __shared__ float s_part[8];
+    float ss = 0.f;
+    for (int c = threadIdx.x * 4; c < d; c += 256 * 4) {
+        float v[4];
+        Vec4<float>::load(xr + c, v);
+        ss += v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) tot += s_part[i];
+    const float r = rsqrtf(tot / (float)d + eps);
+    T* orow = out + (size_t)m * ld_out + col0;
+    for (int c = threadIdx.x * 4; c < d; c += 256 * 4) {
+        float v[4], g[4];
+        Vec4<float>::load(xr + c, v);
+        Vec4<float>::load(w + c, g);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = v[e] * r * g[e];
+        Vec4<T>::store(orow + c, v);
+    }
+}
+
+// ---- rotary embedding (half-split pairing (j, j+dh/2), angle pos * theta^(-2j/dh)) + paged KV append ------------
+template <class T>
+__global__ void __launch_bounds__(256) rope_append_kernel(int R, int Hq, int Hkv, int dh, float theta,
+                                                          T* __restrict__ qkv, const int32_t* __restrict__ pos,
+                                                          T* __restrict__ k_pool, T* __restrict__ v_pool,
+                                                          const int32_t* __restrict__ block_table, int max_blocks,
+                                                          int block_tokens)
+{
+    extern __shared__ float s_cs[];                       // cos [dh/2], sin [dh/2]
+    const int m = blockIdx.x;
+    const int p = pos[m];
+    if (p < 0) return;
+    const int b = m / R;
+    const int half = dh / 2;
+    for (int j = threadIdx.x; j < half; j += blockDim.x) {
+        // the angle is formed in fp64: at positions of 10^4 an fp32 product would already be off by 10^-3 rad
+        const double inv = exp2(-2.0 * (double)j / (double)dh * log2((double)theta));
+        double s, c;
+        sincos((double)p * inv, &s, &c);
+        s_cs[j] = (float)c;
+        s_cs[half + j] = (float)s;
+    }
+    __syncthreads();
+    T* row = qkv + (size_t)m * (Hq + 2 * Hkv) * dh;
+    const int blk = block_table[(size_t)b * max_blocks + p / block_tokens];
+    const int slot = p % block_tokens;
+    // q and k heads: rotate pairs
+    for (int idx = threadIdx.x; idx < (Hq + Hkv) * half; idx += blockDim.x) {
+        const int h = idx / half, j = idx % half;
+        T* hp = row + (size_t)h * dh;
+        const float a = to_f32(hp[j]), bb = to_f32(hp[j + half]);
+        const float c = s_cs[j], s = s_cs[half + j];
+        const T ra = from_f32<T>(a * c - bb * s), rb = from_f32<T>(bb * c + a * s);
+        if (h < Hq) {
+            hp[j] = ra; hp[j + half] = rb;
+        } else if (blk >= 0) {
+            T* dst = k_pool + (((size_t)blk * Hkv + (h - Hq)) * block_tokens + slot) * dh;
+            dst[j] = ra; dst[j + half] = rb;
+        }
+    }
+    if (blk >= 0) {
+        const T* vsrc = row + (size_t)(Hq + Hkv) * dh;
+        for (int idx = threadIdx.x; idx < Hkv * dh; idx += blockDim.x) {
+            const int h = idx / dh, j = idx % dh;
+            v_pool[(((size_t)blk * Hkv + h) * block_tokens + slot) * dh + j] = vsrc[idx];
+        }
+    }
+}
+
+template <class T>
+__global__ void swiglu_kernel(size_t total4, int F, const T* __restrict__ gu, T* __restrict__ out)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total4) return;
+    const size_t e = i * 4;
+    const size_t m = e / F, c = e % F;
+    float g[4], u[4], o[4];
+    Vec4<T>::load(gu + m * 2 * F + c, g);
+    Vec4<T>::load(gu + m * 2 * F + F + c, u);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) o[j] = g[j] / (1.f + __expf(-g[j])) * u[j];
+    Vec4<T>::store(out + e, o);
+}
+
+template <class T>
+__global__ void copy_rows_kernel(int d, const float* __restrict__ x, T* __restrict__ out, int ld_out, int col0)
+{
+    const int m = blockIdx.x;
+    for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+        float v[4];
+        Vec4<float>::load(x + (size_t)m * d + c, v);
+        Vec4<T>::store(out + (size_t)m * ld_out + col0 + c, v);
+    }
+}
+
+__global__ void gather_last_rows_kernel(int R, int d, const float* __restrict__ src, const int32_t* __restrict__ n_valid,
+                                        float* __restrict__ dst)
+{
+    const int b = blockIdx.x;
+    const int r = n_valid[b] - 1;
+    if (r < 0) return;
+    for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+        float v[4];
+        Vec4<float>::load(src + ((size_t)b * R + r) * d + c, v);
+        Vec4<float>::store(dst + (size_t)b * d + c, v);
+    }
+}
+
+// ---- paged-KV bookkeeping: one CTA, sequences in index order, so the result does not depend on scheduling ------
+constexpr int kBookThreads = 1024;
+
+__device__ int block_exclusive_scan(int v, int* total, int* s_warp /*[33]*/)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    __syncthreads();
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int w = s_warp[lane];
+        int winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += t;
+        }
+        s_warp[lane] = winc - w;
+        if (lane == 31) s_warp[32] = winc;
+    }
+    __syncthreads();
+    *total = s_warp[32];
+    return s_warp[warp] + inc - v;
+}
+
+__global__ void __launch_bounds__(kBookThreads) kv_reserve_kernel(int B, int k, int bt, int max_blocks,
+                                                                  const int32_t* seq_len, int32_t* table,
+                                                                  int32_t* free_stack, int32_t* free_top, int32_t* status)
+{
+    __shared__ int s_warp[33];
+    __shared__ int s_fail;
+    if (threadIdx.x == 0) s_fail = 0;
+    __syncthreads();
+    const int top0 = *free_top;
+    // first sweep: total demand (nothing is changed if it cannot be served)
+    int demand = 0;
+    for (int base = 0; base < B; base += kBookThreads) {
+        const int b = base + threadIdx.x;
+        int need_new = 0;
+        if (b < B) {
+            const int need = (seq_len[b] + k + 1 + bt - 1) / bt;
+            if (need > max_blocks) { s_fail = 1; set_status(status, SPEC_ERR_KV_EXHAUSTED, b); }
+            else for (int j = 0; j < need; ++j) need_new += table[(size_t)b * max_blocks + j] < 0;
+        }
+        int tot;
+        block_exclusive_scan(need_new, &tot, s_warp);
+        demand += tot;
+    }
+    __syncthreads();
+    if (s_fail) return;
+    if (demand > top0) { if (threadIdx.x == 0) set_status(status, SPEC_ERR_KV_EXHAUSTED, -1); return; }
+    int carry = 0;
+    for (int base = 0; base < B; base += kBookThreads) {
+        const int b = base + threadIdx.x;
+        int need = 0, need_new = 0;
+        if (b < B) {
+            need = (seq_len[b] + k + 1 + bt - 1) / bt;
+            for (int j = 0; j < need; ++j) need_new += table[(size_t)b * max_blocks + j] < 0;
+        }
+        int tot;
+        int off = carry + block_exclusive_scan(need_new, &tot, s_warp);
+        if (b < B) {
+            for (int j = 0; j < need; ++j) {
+                int32_t* e = &table[(size_t)b * max_blocks + j];
+                if (*e < 0) { *e = free_stack[top0 - 1 - off]; ++off; }
+            }
+        }
+        carry += tot;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) *free_top = top0 - carry;
+}
+
+__global__ void __launch_bounds__(kBookThreads) kv_commit_kernel(const CommitArgs a)
+{
+    __shared__ int s_warp[33];
+    __shared__ long long s_cnt[2];
+    if (threadIdx.x == 0) { s_cnt[0] = 0; s_cnt[1] = 0; }
+    __syncthreads();
+    const int top0 = *a.free_top;
+    const int R = a.k + 1;
+    int carry = 0;
+    for (int base = 0; base < a.B; base += kBookThreads) {
+        const int b = base + threadIdx.x;
+        int freed = 0, keep = 0;
+        if (b < a.B) {
+            int n1, last;
+            if (a.force_n != nullptr) {
+                n1 = min(max(a.force_n[b], 0), a.k) + 1;
+                last = a.force_token[b];
+                // the committed tokens of a forced step are the verified inputs d_1..d_n followed by the given token
+                for (int i = 0; i < R; ++i)
+                    a.out_tokens[(size_t)b * R + i] = i < n1 - 1 ? a.verify_tokens[(size_t)b * R + i + 1] : (i == n1 - 1 ? last : -1);
+                a.n_emitted[b] = n1;
+            } else {
+                n1 = min(max(a.n_emitted[b], 1), R);
+                last = a.out_tokens[(size_t)b * R + n1 - 1];
+            }
+            a.pending_base[b] = a.seq_len[b];
+            const int len = a.seq_len[b] + n1;
+            a.seq_len[b] = len;
+            a.last_token[b] = last;
+            keep = (len + a.block_tokens - 1) / a.block_tokens;
+            for (int j = keep; j < a.max_blocks; ++j) freed += a.block_table[(size_t)b * a.max_blocks + j] >= 0;
+            atomicAdd((unsigned long long*)&s_cnt[0], (unsigned long long)n1);
+            atomicAdd((unsigned long long*)&s_cnt[1], (unsigned long long)(n1 - 1));
+        }
+        int tot;
+        int off = carry + block_exclusive_scan(freed, &tot, s_warp);
+        if (b < a.B) {
+            for (int j = keep; j < a.max_blocks; ++j) {
+                int32_t* e = &a.block_table[(size_t)b * a.max_blocks + j];
+                if (*e >= 0) { a.free_stack[top0 + off] = *e; ++off; *e = -1; }
+            }
+        }
+        carry += tot;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        *a.free_top = top0 + carry;
+        *a.step += 1u;
+        a.counters[0] += 1;
+        a.counters[1] += s_cnt[0];
+        a.counters[2] += s_cnt[1];
+    }
+}
+
+}  // namespace
+
+#define DISPATCH_T(dtype, ...)                                            \
+    if ((dtype) == SPEC_DTYPE_F32) { using T = float; __VA_ARGS__; }      \
+    else { using T = __nv_bfloat16; __VA_ARGS__; }
+
+spec_status launch_verify_rows(int B, int R, const int32_t* seq_len, const int32_t* last_token,
+                               const int32_t* draft_tokens, int draft_stride, int vocab, StepRows rows,
+                               int32_t* status, cudaStream_t st)
+{
+    const int M = B * R;
+    if (M == 0) return SPEC_OK;
+    verify_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(B, R, seq_len, last_token, draft_tokens, draft_stride, vocab, rows, status);
+    return launch_status();
+}
+
+spec_status launch_embed(int M, int d, const void* table, int dtype, const int32_t* token, float* x, cudaStream_t st)
+{
+    if (M == 0) return SPEC_OK;
+    DISPATCH_T(dtype, embed_kernel<T><<<M, 256, 0, st>>>(d, (const T*)table, token, x));
+    return launch_status();
+}
+
+spec_status launch_rmsnorm(int M, int d, const float* in, const float* w, float eps, void* out, int ld_out, int col0,
+                           int dtype, cudaStream_t st)
+{
+    if (M == 0) return SPEC_OK;
+    DISPATCH_T(dtype, rmsnorm_kernel<T><<<M, 256, 0, st>>>(d, in, w, eps, (T*)out, ld_out, col0));
+    return launch_status();
+}
+
+spec_status launch_rope_append(int B, int R, int Hq, int Hkv, int dh, float theta, void* qkv, const int32_t* pos,
+                               void* k_pool, void* v_pool, const int32_t* block_table, int max_blocks,
+                               int block_tokens, int dtype, cudaStream_t st)
+{
+    if (B * R == 0) return SPEC_OK;
+    DISPATCH_T(dtype, rope_append_kernel<T><<<B * R, 256, dh * sizeof(float), st>>>(
+                          R, Hq, Hkv, dh, theta, (T*)qkv, pos, (T*)k_pool, (T*)v_pool, block_table, max_blocks, block_tokens));
+    return launch_status();
+}
+
+spec_status launch_swiglu(int M, int F, const void* gate_up, void* out, int dtype, cudaStream_t st)
+{
+    const size_t total4 = (size_t)M * F / 4;
+    if (total4 == 0) return SPEC_OK;
+    DISPATCH_T(dtype, swiglu_kernel<T><<<(unsigned)((total4 + 255) / 256), 256, 0, st>>>(total4, F, (const T*)gate_up, (T*)out));
+    return launch_status();
+}
+
+spec_status launch_copy_rows_f32_to(int M, int d, const float* x, void* out, int ld_out, int col0, int dtype,
+                                    cudaStream_t st)
+{
+    if (M == 0) return SPEC_OK;
+    DISPATCH_T(dtype, copy_rows_kernel<T><<<M, 256, 0, st>>>(d, x, (T*)out, ld_out, col0));
+    return launch_status();
+}
+
+spec_status launch_gather_last_rows(int B, int R, int d, const float* src, const int32_t* n_valid, float* dst,
+                                    cudaStream_t st)
+{
+    if (B == 0) return SPEC_OK;
+    gather_last_rows_kernel<<<B, 256, 0, st>>>(R, d, src, n_valid, dst);
+    return launch_status();
+}
+
+spec_status launch_kv_reserve(int B, int k, int block_tokens, int max_blocks, const int32_t* seq_len,
+                              int32_t* block_table, int32_t* free_stack, int32_t* free_top, int32_t* status,
+                              cudaStream_t st)
+{
+    if (B == 0) return SPEC_OK;
+    kv_reserve_kernel<<<1, kBookThreads, 0, st>>>(B, k, block_tokens, max_blocks, seq_len, block_table, free_stack, free_top, status);
+    return launch_status();
+}
+
+spec_status launch_kv_commit(const CommitArgs& a, cudaStream_t st)
+{
+    if (a.B == 0) return SPEC_OK;
+    kv_commit_kernel<<<1, kBookThreads, 0, st>>>(a);
+    return launch_status();
+}
+
+}  // namespace spec

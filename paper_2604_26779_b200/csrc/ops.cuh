@@ -1,0 +1,85 @@
+// Launchers of the library's kernels (internal interface between the translation units).
+#pragma once
+
+#include "common.cuh"
+
+namespace spec {
+
+// sampling.cu
+// row r at logits + r*row_stride; its (max, sum exp) at stats + 2*r*stats_stride; probs (nullable) [rows][V]
+spec_status launch_softmax_rows(int rows, int V, const float* logits, size_t row_stride, float temperature, float* stats,
+                                size_t stats_stride, float* probs, cudaStream_t st);
+spec_status launch_reject_sample(bool from_logits, int B, int k, int V, const float* p, const float* p_stats,
+                                 const float* q, const float* q_stats, const int32_t* draft, int draft_stride,
+                                 float temperature, uint64_t seed, const uint32_t* step_dev, uint32_t step,
+                                 int32_t* out_tokens, int32_t* n_emitted, int32_t* status, cudaStream_t st);
+// one token per row from logits and their statistics: uniform Philox(seed; *step_dev, row, slot, stream_tag)
+spec_status launch_sample_logits(int rows, int V, const float* logits, size_t row_stride, const float* stats,
+                                 size_t stats_stride, float temperature, uint64_t seed, const uint32_t* step_dev,
+                                 uint32_t slot, uint32_t stream_tag, int32_t* tokens, int token_stride, int32_t* status,
+                                 cudaStream_t st);
+int sampler_max_vocab();
+
+// ops.cu: element-wise and bookkeeping kernels.  dtype = SPEC_DTYPE_* of the activation/weight/KV storage.
+struct StepRows {            // per-row metadata of a forward over B sequences x R rows
+    int32_t* token;          // [B*R] input token of each row
+    int32_t* pos;            // [B*R] absolute position, or -1 for a row that does nothing
+};
+spec_status launch_verify_rows(int B, int R, const int32_t* seq_len, const int32_t* last_token,
+                               const int32_t* draft_tokens, int draft_stride, int vocab, StepRows rows,
+                               int32_t* status, cudaStream_t st);
+spec_status launch_embed(int M, int d, const void* table, int dtype, const int32_t* token, float* x, cudaStream_t st);
+// out[m][col0 .. col0+d) = RMSNorm(in[m]) * w, out row stride ld_out elements
+spec_status launch_rmsnorm(int M, int d, const float* in, const float* w, float eps, void* out, int ld_out, int col0,
+                           int dtype, cudaStream_t st);
+// rotates q and k of qkv [M][(Hq+2Hkv)*dh] in place and writes k, v into the paged cache at the rows' positions
+spec_status launch_rope_append(int B, int R, int Hq, int Hkv, int dh, float theta, void* qkv, const int32_t* pos,
+                               void* k_pool, void* v_pool, const int32_t* block_table, int max_blocks,
+                               int block_tokens, int dtype, cudaStream_t st);
+spec_status launch_swiglu(int M, int F, const void* gate_up, void* out, int dtype, cudaStream_t st);
+spec_status launch_copy_rows_f32_to(int M, int d, const float* x, void* out, int ld_out, int col0, int dtype,
+                                    cudaStream_t st);
+// dst[b] = src[b*R + idx[b]-1] rows of width d (fp32); idx = rows valid per sequence
+spec_status launch_gather_last_rows(int B, int R, int d, const float* src, const int32_t* n_valid, float* dst,
+                                    cudaStream_t st);
+
+// KV bookkeeping (single CTA, deterministic order)
+spec_status launch_kv_reserve(int B, int k, int block_tokens, int max_blocks, const int32_t* seq_len,
+                              int32_t* block_table, int32_t* free_stack, int32_t* free_top, int32_t* status,
+                              cudaStream_t st);
+struct CommitArgs {
+    int B, k, block_tokens, max_blocks;
+    const int32_t* force_n;       // nullable
+    const int32_t* force_token;   // nullable
+    const int32_t* verify_tokens; // [B][k+1] input tokens of the last verify (read by a forced commit)
+    int32_t* n_emitted;           // [B] in: sampler's n+1 (ignored when forced); out: committed n+1
+    int32_t* out_tokens;          // [B][k+1]
+    int32_t* seq_len; int32_t* last_token; int32_t* block_table; int32_t* free_stack; int32_t* free_top;
+    int32_t* pending_base;        // [B] first position committed by this step
+    uint32_t* step; long long* counters;   // counters: steps, emitted, accepted
+    int32_t* status;
+};
+spec_status launch_kv_commit(const CommitArgs& a, cudaStream_t st);
+
+// gemm_simt.cu / gemm_tc.cu: C[M][N] (+)= A[M][K] W[N][K]^T, fp32 accumulation
+spec_status launch_gemm_simt(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int dtype_in,
+                             int out_dtype, int accumulate, cudaStream_t st);
+spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int dtype_in,
+                        int out_dtype, int accumulate, cudaStream_t st);
+
+// attention.cu
+struct AttnArgs {
+    int B, R, Hq, Hkv, dh, block_tokens, max_blocks;
+    const void* q; int q_row_stride;   // q row (b, r) at q + (b*R + r) * q_row_stride elements, heads contiguous
+    const void* k_pool; const void* v_pool;
+    const int32_t* block_table;
+    const int32_t* pos;                // [B*R] position of each query row (-1: skip, output zeros)
+    void* out; int out_row_stride;
+    int dtype;
+    void* scratch; size_t scratch_bytes;
+    int max_kv_len;
+};
+spec_status launch_attention(const AttnArgs& a, cudaStream_t st);
+size_t attention_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int max_kv_len);
+
+}  // namespace spec

@@ -1,0 +1,131 @@
+"""GPU parity for the whole speculation step on the tiny fp32 workload (C1): prefill through the verify path, then
+32 steps of draft -> verify -> fused softmax + rejection sampling -> KV commit, in lock-step with the cache-free CPU
+oracle.  Bars: logits within 2e-2 relative (inf-norm per row; the fp32 path sits near 1e-5), tokens / accepted
+lengths / sequence lengths identical except at counted boundary cases (|u - min(1, p/q)| < 1e-4 or the final uniform
+within 1e-6 of a CDF bin edge), after which the oracle is re-seeded from the device's committed tokens.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from oracle import model
+from oracle.chain import ChainOracle
+from paper_2604_26779_b200 import inputs
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def eng_mod():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_26779_b200 import engine
+    return engine
+
+
+def run_chain(engine, cfg, kind, B, prompt_len, k, n_steps, seed):
+    W = inputs.make_target_weights(cfg, seed=inputs.sub_seed(1, 0))
+    H = (inputs.make_eagle3_weights if kind == "eagle3" else inputs.make_mtp_weights)(cfg, seed=inputs.sub_seed(1, 1))
+    prompts = inputs.make_prompts(B, prompt_len, cfg["vocab"], seed=inputs.sub_seed(1, 2))
+    max_blocks = -(-(prompt_len + n_steps * (k + 1) + k + 2) // 16)
+    sc = engine.make_spec_config(cfg, draft_kind=kind, k_max=k, max_batch=B, kv_num_blocks=B * max_blocks + 3,
+                                 max_blocks_per_seq=max_blocks, seed=seed)
+    eng = engine.SpecStep(sc)
+    eng.load_target_weights(W)
+    eng.load_draft_weights(H)
+    eng.seq_init(np.zeros(B, np.int32), prompts[:, 0], inputs.make_block_order(sc.kv_num_blocks, inputs.sub_seed(1, 3)))
+
+    # teacher-forced prefill: chunks of k+1 prompt tokens through the verify path
+    R = k + 1
+    assert prompt_len % R == 0
+    n_chunks = prompt_len // R
+    for c in range(n_chunks):
+        if c > 0:
+            eng.draft(1)                                   # lets the draft head absorb the slots just committed
+        forced = torch.from_numpy(np.ascontiguousarray(prompts[:, c * R + 1 : c * R + R])).cuda()
+        eng.verify(k, forced)
+        last = c == n_chunks - 1
+        fn = torch.full((B,), k - 1 if last else k, dtype=torch.int32, device="cuda")
+        ft = torch.from_numpy(np.ascontiguousarray(prompts[:, -1] if last else prompts[:, (c + 1) * R])).cuda()
+        eng.kv_commit(fn, ft)
+    assert eng.status().device_status == 0
+    assert eng.seq_len().cpu().tolist() == [prompt_len - 1] * B
+
+    chains = [ChainOracle(cfg, W, H, kind, seed, b, prompts[b], step0=n_chunks) for b in range(B)]
+    gpu_tokens = [list(map(int, prompts[b])) for b in range(B)]
+    boundary, max_rel, max_rel_d, emitted = 0, 0.0, 0.0, 0
+    for step in range(n_steps):
+        eng.draft(k)
+        eng.verify(k)
+        eng.reject_sample(k)
+        eng.kv_commit()
+        rep = eng.status()
+        assert rep.device_status == 0
+        g_logits = eng.logits(k).cpu().numpy()
+        g_dlogits = eng.draft_logits(k).cpu().numpy()
+        g_drafts = eng.draft_tokens().cpu().numpy()[:, :k]
+        g_out = eng.out_tokens(k).cpu().numpy()
+        g_n = eng.n_emitted().cpu().numpy()
+        g_len = eng.seq_len().cpu().numpy()
+        for b in range(B):
+            ch = chains[b]
+            rec = ch.step_once(k)
+            same = (np.array_equal(rec["drafts"], g_drafts[b]) and rec["n_emitted"] == g_n[b]
+                    and np.array_equal(rec["out_tokens"], g_out[b]))
+            if np.array_equal(rec["drafts"], g_drafts[b]):
+                max_rel = max(max_rel, float(np.max(np.abs(g_logits[b] - rec["target_logits"]).max(-1) /
+                                                    np.abs(rec["target_logits"]).max(-1))))
+                max_rel_d = max(max_rel_d, float(np.max(np.abs(g_dlogits[b] - rec["draft_logits"]).max(-1) /
+                                                      np.abs(rec["draft_logits"]).max(-1))))
+            if not same:
+                mg = rec["margins"]
+                assert np.any(mg[:k] < 1e-4) or mg[k] < 1e-6 or not np.array_equal(rec["drafts"], g_drafts[b]), \
+                    (step, b, rec["drafts"], g_drafts[b], rec["out_tokens"], g_out[b], mg)
+                boundary += 1
+            gpu_tokens[b] += [int(t) for t in g_out[b, : g_n[b]]]
+            assert 1 <= g_n[b] <= k + 1 and np.all(g_out[b, g_n[b]:] == -1)
+            assert g_len[b] == len(gpu_tokens[b]) - 1                     # committed KV entries = tokens - 1
+            ch.tokens = list(gpu_tokens[b])                                # re-seed (no-op when identical)
+            emitted += int(g_n[b])
+        assert rep.steps == n_chunks + step + 1
+    rep = eng.status()
+    # block conservation after the run
+    table = eng.block_table().cpu().numpy()
+    owned = table[table >= 0]
+    top = int(eng.tensor("FREE_TOP", 0, torch.int32, (1,)).item())
+    free = eng.tensor("FREE_STACK", 0, torch.int32, (sc.kv_num_blocks,)).cpu().numpy()[:top]
+    assert len(set(owned.tolist())) == owned.size and owned.size + top == sc.kv_num_blocks
+    assert set(owned.tolist()).isdisjoint(free.tolist())
+    for b in range(B):
+        assert np.all(table[b, : -(-int(g_len[b]) // 16)] >= 0) and np.all(table[b, -(-int(g_len[b]) // 16):] == -1)
+    eng.close()
+    return dict(boundary=boundary, max_rel=max_rel, max_rel_d=max_rel_d, emitted=emitted, steps=n_steps * B)
+
+
+def test_c1_chain_eagle3_lockstep(eng_mod):
+    cfg = inputs.model_config("c1")
+    r = run_chain(eng_mod, cfg, "eagle3", B=4, prompt_len=64, k=3, n_steps=32, seed=inputs.BASE_SEED)
+    print("C1 eagle3:", r)
+    assert r["max_rel"] < 1e-3 and r["max_rel_d"] < 1e-3            # fp32 path; the bf16 bar is 2e-2
+    assert r["boundary"] <= 2
+    assert r["steps"] <= r["emitted"] <= 4 * r["steps"]
+
+
+def test_tiny_chain_mtp_lockstep(eng_mod):
+    cfg = dict(inputs.model_config("c1"), tap_layers=(2,))
+    r = run_chain(eng_mod, cfg, "mtp", B=3, prompt_len=30, k=2, n_steps=12, seed=5)
+    print("tiny mtp:", r)
+    assert r["max_rel"] < 1e-3 and r["max_rel_d"] < 1e-3 and r["boundary"] <= 2
+
+
+def test_kv_exhaustion_is_reported_not_faulted(eng_mod):
+    cfg = inputs.model_config("c1")
+    sc = eng_mod.make_spec_config(cfg, draft_kind="none", k_max=3, max_batch=2, kv_num_blocks=3, max_blocks_per_seq=4, seed=1)
+    eng = eng_mod.SpecStep(sc)
+    eng.load_target_weights(inputs.make_target_weights(cfg, seed=1))
+    eng.seq_init(np.array([14, 15], np.int32), np.array([1, 2], np.int32), np.arange(3, dtype=np.int32))
+    forced = torch.zeros((2, 3), dtype=torch.int32, device="cuda")
+    eng.verify(3, forced)                      # needs 2 blocks per sequence, only 1 spare
+    assert eng.status().device_status == -16
+    eng.close()

@@ -1,0 +1,232 @@
+"""GPU parity: uniforms, vocabulary softmax and rejection sampling through the C ABI against the CPU oracle.
+
+Bars (written out here): uniforms bit-exact; probabilities within 1e-3 absolute; with identical fp32 probability
+inputs the sampler's accept decisions, accepted lengths and tokens are bit-exact, except draws where the uniform
+lies within 1e-6 of an edge of the chosen CDF bin (counted and reported); the fused from-logits sampler is compared
+with the oracle fed the GPU's own materialised probabilities, under the same rule plus the decision band
+|u - min(1, p/q)| < 1e-4.
+"""
+import numpy as np
+import pytest
+import scipy.stats
+
+import oracle
+from paper_2604_26779_b200 import inputs
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+EDGE = 1e-6
+BAND = 1e-4
+
+
+@pytest.fixture(scope="module")
+def api():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_26779_b200 import binding
+    binding.lib()
+    return binding
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def gpu_reject_probs(api, p, q, drafts, seed, step):
+    B, kp1, V = p.shape
+    out = torch.full((B, kp1), -7, dtype=torch.int32, device="cuda")
+    n = torch.zeros(B, dtype=torch.int32, device="cuda")
+    st = torch.zeros(4, dtype=torch.int32, device="cuda")
+    api.spec_reject_sample_probs(dev(p), dev(q) if kp1 > 1 else None, dev(drafts) if kp1 > 1 else None, seed, step, out, n, st)
+    torch.cuda.synchronize()
+    return out.cpu().numpy(), n.cpu().numpy(), st.cpu().numpy()
+
+
+def compare_with_oracle(out, n, p, q, drafts, seed, step, decision_band=0.0):
+    """Returns the number of tolerated boundary cases; asserts everything else is identical."""
+    o_out, o_n, o_fl, mg = oracle.reject_sample(p, q, drafts, seed, step)
+    k = p.shape[1] - 1
+    boundary = 0
+    for b in range(p.shape[0]):
+        if n[b] == o_n[b] and np.array_equal(out[b], o_out[b]):
+            continue
+        near_decision = decision_band > 0 and np.any(mg[b, :k] < decision_band)
+        near_edge = mg[b, k] < EDGE
+        assert near_decision or (near_edge and n[b] == o_n[b] and np.array_equal(out[b, : n[b] - 1], o_out[b, : n[b] - 1])), \
+            (b, out[b], o_out[b], n[b], o_n[b], mg[b])
+        boundary += 1
+    return boundary
+
+
+def make_case(B, k, V, sigma, tau, seed):
+    t, d = inputs.make_sampler_logits(B, k, V, sigma, tau, seed)
+    p, q = oracle.softmax(t), oracle.softmax(d)
+    if k > 0:
+        ud = oracle.uniforms(seed, 0, 1, B, k)
+        drafts = np.stack([oracle.sample_rows(q[:, i], ud[:, i])[0] for i in range(k)], 1).astype(np.int32)
+    else:
+        drafts = np.zeros((B, 0), np.int32)
+    return t, d, p, q, drafts
+
+
+def test_uniforms_bit_exact(api):
+    u = torch.zeros((50000, 20), dtype=torch.float32, device="cuda")       # 1e6 counters
+    for step, tag, seed in [(0, 0, inputs.BASE_SEED), (12345, 1, 0xFEDCBA9876543210)]:
+        api.spec_uniforms(seed, step, tag, u)
+        assert np.array_equal(u.cpu().numpy(), oracle.uniforms(seed, step, tag, 50000, 20))
+
+
+@pytest.mark.parametrize("V,T", [(8, 1.0), (1000, 0.7), (1027, 1.0), (151936, 1.0), (128256, 2.0)])
+def test_softmax_probabilities_and_stats(api, V, T):
+    rng = np.random.default_rng(V)
+    lg = (rng.standard_normal((5, V)) * 3).astype(np.float32)
+    stats = torch.zeros((5, 2), device="cuda")
+    probs = torch.zeros((5, V), device="cuda")
+    api.spec_softmax_rows(dev(lg), T, stats, probs)
+    torch.cuda.synchronize()
+    ref = oracle.softmax(lg, T)
+    assert np.max(np.abs(probs.cpu().numpy() - ref)) < 1e-3 * 1e-2          # far inside the 1e-3 absolute bar
+    for r in range(5):
+        m, z = oracle.softmax_stats(lg[r], T)
+        assert stats[r, 0].item() == m and abs(stats[r, 1].item() / z - 1) < 1e-5
+    # statistics alone (no probabilities written) give the same numbers
+    stats2 = torch.zeros((5, 2), device="cuda")
+    api.spec_softmax_rows(dev(lg), T, stats2, None)
+    assert torch.equal(stats, stats2)
+
+
+@pytest.mark.parametrize("B,k,V,sigma,tau", [
+    (4096, 3, 8, 1.0, 0.5), (512, 1, 1000, 1.0, 1.0), (256, 5, 1027, 3.0, 0.5), (300, 7, 4100, 1.0, 0.1),
+    (48, 3, 151936, 1.0, 0.5), (24, 7, 151936, 3.0, 1.0), (33, 1, 128256, 1.0, 0.1)])
+def test_reject_sample_probs_bit_exact(api, B, k, V, sigma, tau):
+    _, _, p, q, drafts = make_case(B, k, V, sigma, tau, seed=B + k + V)
+    total_boundary = 0
+    for step in (0, 5):
+        out, n, st = gpu_reject_probs(api, p, q, drafts, inputs.BASE_SEED, step)
+        assert st[0] == 0 and n.min() >= 1 and n.max() <= k + 1
+        total_boundary += compare_with_oracle(out, n, p, q, drafts, inputs.BASE_SEED, step)
+    print(f"boundary cases (|u - CDF edge| < {EDGE}): {total_boundary} of {2 * B}")
+    assert total_boundary <= max(2, 2 * B // 200)
+
+
+def test_empty_and_k0(api):
+    _, _, p, q, drafts = make_case(16, 0, 515, 1.0, 0.5, seed=1)
+    out, n, st = gpu_reject_probs(api, p, q, drafts, 3, 9)                    # k = 0: plain sampling from p_1
+    assert compare_with_oracle(out, n, p, q, drafts, 3, 9) == 0 and np.all(n == 1)
+    e = torch.zeros((0, 4, 64), device="cuda")
+    api.spec_reject_sample_probs(e, torch.zeros((0, 3, 64), device="cuda"), torch.zeros((0, 3), dtype=torch.int32, device="cuda"),
+                                 1, 0, torch.zeros((0, 4), dtype=torch.int32, device="cuda"),
+                                 torch.zeros(0, dtype=torch.int32, device="cuda"))       # B = 0 is a no-op
+
+
+def test_draft_equals_target_accepts_all(api):
+    B, k, V = 128, 3, 5000
+    t, _, p, _, _ = make_case(B, k, V, 1.0, 0.5, seed=2)
+    q = p[:, :k].copy()
+    drafts = np.random.default_rng(0).integers(0, V, (B, k)).astype(np.int32)
+    out, n, st = gpu_reject_probs(api, p, q, drafts, 5, 1)
+    assert np.all(n == k + 1) and np.array_equal(out[:, :k], drafts)
+    assert compare_with_oracle(out, n, p, q, drafts, 5, 1) <= 1
+
+
+def test_one_hot_draft_and_bad_rows(api):
+    B, k, V = 64, 2, 600
+    _, _, p, _, _ = make_case(B, k, V, 1.0, 0.5, seed=3)
+    drafts = np.random.default_rng(1).integers(0, V, (B, k)).astype(np.int32)
+    q = np.zeros((B, k, V), np.float32)
+    for b in range(B):
+        for i in range(k):
+            q[b, i, drafts[b, i]] = 1.0
+    out, n, st = gpu_reject_probs(api, p, q, drafts, 8, 2)
+    assert compare_with_oracle(out, n, p, q, drafts, 8, 2) == 0
+    # an out-of-range draft token is reported through the status word and never dereferenced
+    bad = drafts.copy()
+    bad[7, 0] = V + 5
+    out, n, st = gpu_reject_probs(api, p, q, bad, 8, 2)
+    assert st[0] == -17 and st[1] == 7 and n[7] == 1
+    # residual without mass -> falls back to p_{n+1} and flags it, as the oracle does
+    p2 = np.full((1, 2, 4), 0.1, np.float32)
+    q2 = np.full((1, 1, 4), 0.4, np.float32)
+    for step in range(6):
+        out, n, st = gpu_reject_probs(api, p2, q2, np.array([[1]], np.int32), 4, step)
+        o_out, o_n, o_fl, _ = oracle.reject_sample(p2, q2, np.array([[1]], np.int32), 4, step)
+        assert np.array_equal(out, o_out) and n[0] == o_n[0] and (st[0] == -18) == bool(o_fl[0] & 1)
+
+
+def test_fused_from_logits_matches_oracle_on_gpu_probabilities(api):
+    for (B, k, V, sigma, tau, T) in [(64, 3, 128256, 1.0, 0.5, 1.0), (96, 5, 1027, 3.0, 1.0, 0.8), (512, 3, 8, 1.0, 0.5, 1.0)]:
+        t, d, _, _, _ = make_case(B, k, V, sigma, tau, seed=V + k)
+        tl, dl = dev(t), dev(d)
+        ps, qs = torch.zeros((B * (k + 1), 2), device="cuda"), torch.zeros((B * k, 2), device="cuda")
+        pp, qp = torch.zeros_like(tl), torch.zeros_like(dl)
+        api.spec_softmax_rows(tl, T, ps, pp)
+        api.spec_softmax_rows(dl, T, qs, qp)
+        p, q = pp.cpu().numpy(), qp.cpu().numpy()
+        assert np.max(np.abs(p - oracle.softmax(t, T))) < 1e-3 and np.max(np.abs(q - oracle.softmax(d, T))) < 1e-3
+        ud = oracle.uniforms(7, 0, 1, B, k)
+        drafts = np.stack([oracle.sample_rows(q[:, i], ud[:, i])[0] for i in range(k)], 1).astype(np.int32)
+        out = torch.zeros((B, k + 1), dtype=torch.int32, device="cuda")
+        n = torch.zeros(B, dtype=torch.int32, device="cuda")
+        st = torch.zeros(4, dtype=torch.int32, device="cuda")
+        api.spec_reject_sample_logits(tl, ps, dl, qs, dev(drafts), T, 7, 3, out, n, st)
+        torch.cuda.synchronize()
+        assert st[0].item() == 0
+        nb = compare_with_oracle(out.cpu().numpy(), n.cpu().numpy(), p, q, drafts, 7, 3, decision_band=BAND)
+        print(f"fused sampler V={V}: boundary cases {nb} of {B}")
+        assert nb <= max(2, B // 100)
+
+
+def test_sample_rows_matches_oracle(api):
+    B, V = 200, 3001
+    p = oracle.softmax(np.random.default_rng(5).standard_normal((B, V)).astype(np.float32) * 2)
+    tok = torch.zeros(B, dtype=torch.int32, device="cuda")
+    api.spec_sample_rows(dev(p), 11, 4, 2, 1, tok)
+    u = np.array([oracle.uniform(11, 4, b, 2, 1) for b in range(B)], np.float32)
+    ref, mg = oracle.sample_rows(p, u)
+    diff = tok.cpu().numpy() != ref
+    assert np.all(mg[diff] < EDGE) and diff.sum() <= 2
+
+
+def test_gpu_sampler_chi_square_vocab8(api):
+    """The same distribution-level check as for the oracle, on the CUDA sampler: 1e6 seeded trials at vocab 8, k = 3."""
+    from tests.test_oracle_sampler import _tables, _chain_expected
+    V, k, n_tr = 8, 3, 1_000_000
+    rng = np.random.default_rng(2604)
+    P0, Q0 = _tables(rng, V, 1)[0], _tables(rng, V, 1)[0]
+    P, Q = _tables(rng, V, V), _tables(rng, V, V)
+    Pf, Qf = dev(np.concatenate([P, P0[None]], 0)), dev(np.concatenate([Q, Q0[None]], 0))
+    need = k + 1
+    emitted = torch.full((n_tr, need + k + 1), -1, dtype=torch.int64, device="cuda")
+    count = torch.zeros(n_tr, dtype=torch.int64, device="cuda")
+    prev = torch.full((n_tr,), V, dtype=torch.int64, device="cuda")         # row V = start state
+    ar = torch.arange(n_tr, device="cuda")
+    step = 0
+    seed = inputs.BASE_SEED + 1
+    while int(count.min()) < need:
+        p = torch.zeros((n_tr, k + 1, V), device="cuda")
+        q = torch.zeros((n_tr, k, V), device="cuda")
+        drafts = torch.zeros((n_tr, k), dtype=torch.int32, device="cuda")
+        cur = prev.clone()
+        tok = torch.zeros(n_tr, dtype=torch.int32, device="cuda")
+        for i in range(k):
+            q[:, i] = Qf[cur]
+            p[:, i] = Pf[cur]
+            api.spec_sample_rows(q[:, i].contiguous(), seed, step, i, 1, tok)
+            drafts[:, i] = tok
+            cur = tok.long()
+        p[:, k] = Pf[cur]
+        out = torch.zeros((n_tr, k + 1), dtype=torch.int32, device="cuda")
+        n = torch.zeros(n_tr, dtype=torch.int32, device="cuda")
+        api.spec_reject_sample_probs(p, q, drafts, seed, step, out, n)
+        for j in range(k + 1):
+            live = (j < n) & (count + j < emitted.shape[1])
+            emitted[ar[live], (count + j)[live]] = out[live, j].long()
+        prev = out[ar, (n - 1).long()].long()
+        count += n.long()
+        step += 1
+    toks = emitted[:, :need].cpu().numpy()
+    exp = _chain_expected(P0, P, need).ravel()
+    obs = np.bincount(np.ravel_multi_index(toks.T, (V,) * need), minlength=V ** need)
+    chi = scipy.stats.chisquare(obs, exp / exp.sum() * n_tr)
+    assert chi.pvalue > 1e-4, chi
