@@ -95,13 +95,13 @@ spec_status launch_attention_simt(const AttnArgs& a, cudaStream_t st)
 
 spec_status launch_attention(const AttnArgs& a, cudaStream_t st)
 {
+    if (attention_mma_supported(a)) return launch_attention_mma(a, st);
     return launch_attention_simt(a, st);
 }
 
 size_t attention_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int max_kv_len)
 {
-    (void)B; (void)R; (void)Hq; (void)Hkv; (void)dh; (void)max_kv_len;
-    return 256;
+    return attention_mma_scratch_bytes(B, R, Hq, Hkv, dh, max_kv_len);
 }
 
 }  // namespace spec
@@ -139,6 +139,6 @@ extern "C" spec_status spec_attention(int B, int R, int Hq, int Hkv, int dh, int
     launch_attn_rows(B, R, seq_len, (int32_t*)scratch, st);
     AttnArgs a{B, R, Hq, Hkv, dh, block_tokens, max_blocks, q, Hq * dh, k_pool, v_pool, block_table,
                (const int32_t*)scratch, out, Hq * dh, dtype, (char*)scratch + pos_bytes, scratch_bytes - pos_bytes,
-               max_blocks * block_tokens};
+               max_blocks * block_tokens, 0};
     return launch_attention(a, st);
 }

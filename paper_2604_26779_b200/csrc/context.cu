@@ -199,7 +199,7 @@ LayerPtrs layer_ptrs(void* base, const LayerLoc& L)
 // attention + MLP of one decoder layer on the fp32 residual `res` [M][d].  `qkv_in` [M][qkv_k] is the already
 // prepared input of the QKV projection.
 spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* res, const void* qkv_in, int qkv_k, int B, int R,
-                           const int32_t* pos, void* k_pool, void* v_pool, cudaStream_t st)
+                           const int32_t* pos, void* k_pool, void* v_pool, int launch_index, cudaStream_t st)
 {
     const spec_config& g = c.cfg;
     const int M = B * R, d = g.d_model, dh = g.head_dim, Hq = g.n_q_heads, Hkv = g.n_kv_heads;
@@ -210,7 +210,7 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
                            at<int32_t>(c.buf.state, c.block_table), g.max_blocks_per_seq, g.kv_block_tokens, dt, st));
     AttnArgs a{B, R, Hq, Hkv, dh, g.kv_block_tokens, g.max_blocks_per_seq, at(ws, c.qkv), qkv_n, k_pool, v_pool,
                at<int32_t>(c.buf.state, c.block_table), pos, at(ws, c.attn_out), Hq * dh, dt, at(ws, c.attn_scratch),
-               c.attn_scratch.bytes, g.max_blocks_per_seq * g.kv_block_tokens};
+               c.attn_scratch.bytes, g.max_blocks_per_seq * g.kv_block_tokens, launch_index};
     TRY(launch_attention(a, st));
     TRY(launch_gemm(M, d, Hq * dh, at(ws, c.attn_out), Hq * dh, W.wo, res, d, dt, SPEC_DTYPE_F32, 1, st));
     TRY(launch_rmsnorm(M, d, res, W.mlp_norm, g.rms_eps, at(ws, c.h), d, 0, dt, st));
@@ -417,7 +417,7 @@ extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_toke
         TRY(launch_rmsnorm(M, d, x, W.attn_norm, g.rms_eps, at(ws, c->h), d, 0, dt, st));
         const int pool = l % g.kv_layer_pools;
         char* kp = static_cast<char*>(c->buf.kv) + (size_t)pool * 2 * c->kv_pool_bytes;
-        TRY(run_layer_body(*c, W, g.d_ffn, x, at(ws, c->h), d, B, R, rows.pos, kp, kp + c->kv_pool_bytes, st));
+        TRY(run_layer_body(*c, W, g.d_ffn, x, at(ws, c->h), d, B, R, rows.pos, kp, kp + c->kv_pool_bytes, l, st));
         if (has_tap(g, l + 1)) TRY(launch_copy_rows_f32_to(M, d, x, at(ws, c->taps), tapw, tap_slot(g, l + 1) * d, dt, st));
     }
     TRY(launch_rmsnorm(M, d, x, at<const float>(c->buf.weights, c->final_norm), g.rms_eps, at(ws, c->h), d, 0, dt, st));
@@ -522,7 +522,7 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
             if (j == 0) TRY(launch_gemm(M, d, g.n_taps * d, at(ws, c->taps), g.n_taps * d, at(dw, c->d_wfc), dg, d, dt, SPEC_DTYPE_F32, 0, st));
             TRY(launch_rmsnorm(M, d, dx, at<const float>(dw, c->d_norm_e), g.rms_eps, at(ws, c->h), 2 * d, 0, dt, st));
             TRY(launch_rmsnorm(M, d, res, at<const float>(dw, c->d_norm_g), g.rms_eps, at(ws, c->h), 2 * d, d, dt, st));
-            TRY(run_layer_body(*c, W, g.draft_d_ffn, res, at(ws, c->h), 2 * d, B, R, pos, kp, vp, st));
+            TRY(run_layer_body(*c, W, g.draft_d_ffn, res, at(ws, c->h), 2 * d, B, R, pos, kp, vp, 0, st));
         } else {
             // h0 = W_proj concat(norm_g(g), norm_e(e)); g = the target's last-layer residual or the head's previous output
             const float* gsrc = j == 0 ? at<float>(ws, c->x) : hid;
@@ -530,7 +530,7 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
             TRY(launch_rmsnorm(M, d, dx, at<const float>(dw, c->d_norm_e), g.rms_eps, at(ws, c->h), 2 * d, d, dt, st));
             TRY(launch_gemm(M, d, 2 * d, at(ws, c->h), 2 * d, at(dw, c->d_wproj), res, d, dt, SPEC_DTYPE_F32, 0, st));
             TRY(launch_rmsnorm(M, d, res, W.attn_norm, g.rms_eps, at(ws, c->h), d, 0, dt, st));
-            TRY(run_layer_body(*c, W, g.draft_d_ffn, res, at(ws, c->h), d, B, R, pos, kp, vp, st));
+            TRY(run_layer_body(*c, W, g.draft_d_ffn, res, at(ws, c->h), d, B, R, pos, kp, vp, 0, st));
         }
         if (j == 0) TRY(launch_gather_last_rows(B, R, d, dg, at<int32_t>(sb, c->n_emitted), hid, st));
         // logits of this slot, their statistics, and the draft token d_{j+1} ~ q_{j+1} (stream-1 uniform, slot j)

@@ -78,8 +78,12 @@ struct AttnArgs {
     int dtype;
     void* scratch; size_t scratch_bytes;
     int max_kv_len;
+    int launch_index;                  // 0 plans the work units; later launches of the same step reuse the plan
 };
 spec_status launch_attention(const AttnArgs& a, cudaStream_t st);
 size_t attention_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int max_kv_len);
+bool attention_mma_supported(const AttnArgs& a);
+size_t attention_mma_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int max_kv_len);
+spec_status launch_attention_mma(const AttnArgs& a, cudaStream_t st);
 
 }  // namespace spec

@@ -1,0 +1,113 @@
+"""GPU parity of the two heavy operators through their stateless C entry points: paged grouped-query attention and
+the GEMM, against the CPU oracle / fp64 products on the same seeded bytes.
+
+Bars: bf16 results within 2e-2 of the row's largest magnitude (the same inf-norm-relative bar as for logits), fp32
+results within 1e-4.
+"""
+import numpy as np
+import pytest
+
+from oracle import model
+from paper_2604_26779_b200 import inputs
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def api():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_26779_b200 import binding
+    binding.lib()
+    return binding
+
+
+def paged_case(lens, R, Hq, Hkv, dh, dtype, seed):
+    """Random cache contents in a permuted block pool; returns device tensors and the logical K/V per sequence."""
+    B, bt = len(lens), 16
+    rng = np.random.default_rng(seed)
+    max_blocks = -(-(max(lens) + R) // bt) + 1
+    nblk = sum(-(-(l + R) // bt) for l in lens) + 5
+    order = inputs.make_block_order(nblk, seed)
+    table = np.full((B, max_blocks), -1, np.int32)
+    nxt = 0
+    for b, l in enumerate(lens):
+        for j in range(-(-(l + R) // bt)):
+            table[b, j] = order[nxt]
+            nxt += 1
+    kind = "bf16" if dtype == torch.bfloat16 else "f32"
+    kpool = inputs.make_kv_values((nblk, Hkv, bt, dh), seed + 1, kind)
+    vpool = inputs.make_kv_values((nblk, Hkv, bt, dh), seed + 2, kind)
+    q = inputs.make_kv_values((B, R, Hq, dh), seed + 3, kind)
+    logical = []
+    for b, l in enumerate(lens):
+        n = l + R
+        blocks = table[b, : -(-n // bt)]
+        k = kpool[blocks].transpose(0, 2, 1, 3).reshape(-1, Hkv, dh)[:n]
+        v = vpool[blocks].transpose(0, 2, 1, 3).reshape(-1, Hkv, dh)[:n]
+        logical.append((k, v))
+    return q, kpool, vpool, table, logical
+
+
+@pytest.mark.parametrize("lens,R,Hq,Hkv,dh,dtype", [
+    ([0, 1, 15, 16, 17, 700, 2047, 2048, 2049, 5003], 4, 32, 8, 128, torch.bfloat16),   # 8B shape: 16 rows per KV head
+    ([3, 100, 4100], 1, 32, 8, 128, torch.bfloat16),                                   # plain decode rows
+    ([64, 777, 2500], 5, 16, 4, 128, torch.bfloat16),                                  # k = 4: 20 rows -> two row tiles
+    ([10, 300, 2100], 8, 8, 2, 128, torch.bfloat16),                                   # k = 7: 32 rows
+    ([50, 1234], 4, 32, 2, 128, torch.bfloat16),                                       # group 16: 64 rows (MoE layer shape)
+    ([5, 130, 2300], 4, 8, 4, 64, torch.bfloat16),                                     # head_dim 64
+    ([0, 9, 40, 333], 4, 4, 4, 64, torch.float32),                                     # fp32 reference path
+])
+def test_paged_attention_matches_oracle(api, lens, R, Hq, Hkv, dh, dtype):
+    q, kpool, vpool, table, logical = paged_case(lens, R, Hq, Hkv, dh, dtype, seed=len(lens) * 7 + R)
+    B = len(lens)
+    dq = torch.from_numpy(q).cuda().to(dtype)
+    dk, dv = torch.from_numpy(kpool).cuda().to(dtype), torch.from_numpy(vpool).cuda().to(dtype)
+    out = torch.full((B, R, Hq, dh), 7.0, dtype=dtype, device="cuda")
+    nbytes = api.spec_attention_scratch_bytes(B, R, Hq, Hkv, dh, table.shape[1] * 16)
+    scratch = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    api.spec_attention(dq, dk, dv, torch.from_numpy(table).cuda(), torch.tensor(lens, dtype=torch.int32, device="cuda"),
+                       out, scratch)
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy()
+    tol = 2e-2 if dtype == torch.bfloat16 else 1e-4
+    worst = 0.0
+    for b, l in enumerate(lens):
+        k, v = logical[b]
+        ref = model.attention(q[b].astype(np.float64), k.astype(np.float64), v.astype(np.float64), n_past=l)
+        err = np.abs(got[b] - ref).max(-1) / np.abs(ref).max(-1)
+        worst = max(worst, float(err.max()))
+    print(f"attention R={R} Hq={Hq}/{Hkv} dh={dh} {dtype}: worst row error {worst:.2e}")
+    assert worst < tol
+
+
+@pytest.mark.parametrize("M,N,K,din,dout,acc", [
+    (16, 768, 256, torch.float32, torch.float32, False),
+    (5, 1024, 1024, torch.float32, torch.float32, True),
+    (128, 256, 64, torch.bfloat16, torch.float32, False),          # one tile, one k-step
+    (128, 256, 512, torch.bfloat16, torch.bfloat16, False),
+    (1024, 6144, 4096, torch.bfloat16, torch.bfloat16, False),     # 8B QKV projection
+    (1024, 4096, 14336, torch.bfloat16, torch.float32, True),      # 8B down projection into the fp32 residual
+    (256, 4096, 4096, torch.bfloat16, torch.float32, True),        # decode-sized M
+    (1000, 520, 192, torch.bfloat16, torch.bfloat16, False),       # ragged M and N tails
+    (77, 1000, 4096, torch.bfloat16, torch.float32, False),
+    (1024, 16384, 1024, torch.bfloat16, torch.float32, False),     # LM-head-like slice: fp32 logits
+])
+def test_gemm_matches_fp64(api, M, N, K, din, dout, acc):
+    kind = "bf16" if din == torch.bfloat16 else "f32"
+    A = inputs.make_kv_values((M, K), 1, kind)
+    W = inputs.make_kv_values((N, K), 2, kind) * np.float32(0.05)
+    W = inputs.round_to_bf16(W) if kind == "bf16" else W
+    C0 = inputs.make_kv_values((M, N), 3, "bf16" if dout == torch.bfloat16 else "f32")
+    dA, dW = torch.from_numpy(A).cuda().to(din), torch.from_numpy(W).cuda().to(din)
+    dC = torch.from_numpy(C0).cuda().to(dout)
+    api.spec_gemm(dA, dW, dC, accumulate=acc)
+    torch.cuda.synchronize()
+    # fp64 reference on sampled rows (all rows when small)
+    rows = np.arange(M) if M * N * K < 2e9 else np.unique(np.concatenate([np.arange(0, M, 37), [M - 1, M - 2, 127, 128]]))
+    ref = A[rows].astype(np.float64) @ W.astype(np.float64).T + (C0[rows].astype(np.float64) if acc else 0.0)
+    got = dC.float().cpu().numpy()[rows]
+    err = np.abs(got - ref).max(-1) / np.abs(ref).max(-1)
+    print(f"gemm {M}x{N}x{K} {din}->{dout} acc={acc}: worst row error {err.max():.2e}")
+    assert err.max() < (2e-2 if dout == torch.bfloat16 else (1e-3 if din == torch.bfloat16 else 1e-5))
