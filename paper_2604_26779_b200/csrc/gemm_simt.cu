@@ -80,19 +80,3 @@ spec_status launch_gemm_simt(int M, int N, int K, const void* A, int lda, const 
 
 }  // namespace spec
 
-namespace spec {
-spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int dtype_in,
-                        int out_dtype, int accumulate, cudaStream_t st)
-{
-    return launch_gemm_simt(M, N, K, A, lda, W, C, ldc, dtype_in, out_dtype, accumulate, st);
-}
-}  // namespace spec
-
-extern "C" spec_status spec_gemm(int M, int N, int K, const void* A, const void* W, void* C, int dtype_in, int out_dtype,
-                                 int accumulate, void* stream)
-{
-    if (M < 0 || N < 0 || K <= 0) return SPEC_ERR_INVALID_ARG;
-    if (M == 0 || N == 0) return SPEC_OK;
-    if (!A || !W || !C) return SPEC_ERR_INVALID_ARG;
-    return spec::launch_gemm(M, N, K, A, K, W, C, N, dtype_in, out_dtype, accumulate, (cudaStream_t)stream);
-}

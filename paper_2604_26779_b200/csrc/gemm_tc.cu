@@ -1,0 +1,349 @@
+// bf16 GEMM on the 5th-generation tensor cores:  C[M][N] (+)= A[M][K] * W[N][K]^T, fp32 accumulation.
+//
+// The projections of the verify forward (QKV, O, gate/up, down, LM head) are dense contractions with M = B(k+1)
+// rows, far above the ridge point, so they run on tcgen05:
+//   - persistent CTAs, one per SM, walk 128 x 256 output tiles (tiles that share a weight tile run side by side, so
+//     the weight tile crosses HBM once and the activations stay in L2);
+//   - warp 0 streams A and W tiles of 64 k-columns with TMA (cp.async.bulk.tensor, 128-byte swizzle) into a 4-stage
+//     shared-memory ring, signalled by mbarriers;
+//   - warp 1 issues tcgen05.mma (M=128, N=256, K=16 per instruction) from one thread; the fp32 accumulator lives in
+//     tensor memory, double-buffered (2 x 256 columns) so the epilogue of one tile overlaps the next tile's loads;
+//   - warps 2-5 read the accumulator with tcgen05.ld (one 32-lane quarter each) and store fp32 / bf16, optionally
+//     adding to the fp32 residual stream.
+// Every mbarrier wait is bounded: on a timeout the CTA raises a flag, all roles leave their loops, outstanding
+// tensor-core work is drained with a bounded wait, tensor memory is released and the kernel returns with
+// SPEC_ERR_TIMEOUT in the status word.
+#include <cuda.h>
+
+#include "ops.cuh"
+
+namespace spec {
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr long long kWaitLimit = 300000000LL;            // clock cycles (~0.15 s): far beyond any healthy wait
+
+struct Ctl {
+    uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain;
+    uint32_t tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the CTA is aborting or the limit ran out (which raises the abort flag).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitLimit) { *abort_flag = 1; return false; }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                   "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 64 bf16 (128 bytes) wide, 128-byte swizzle:
+// start address >> 4, leading byte offset 1 (unused for swizzled K-major), stride byte offset = 1024 bytes between
+// 8-row groups, descriptor version 1, layout type 2 (SWIZZLE_128B).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr)
+{
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+struct GemmArgs {
+    int M, N, K;
+    void* C; int ldc;
+    int out_f32, accumulate;
+    int32_t* status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                              const __grid_constant__ CUtensorMap map_b, const GemmArgs g)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;                        // 1024-byte aligned stage ring
+    Ctl* ctl = reinterpret_cast<Ctl*>(smem_raw + (tiles - raw) + STAGES * STAGE_BYTES);
+    volatile int* abort_flag = &ctl->abort;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    const int m_tiles = (g.M + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
+    const int n_work = m_tiles * n_tiles, kb_count = (g.K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&ctl->tmem_full[a]), 1); mbar_init(smem_u32(&ctl->tmem_empty[a]), 128); }
+        mbar_init(smem_u32(&ctl->drain), 1);
+        ctl->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ---- TMA producer ----
+        if (lane == 0) {
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
+                const int mt = w % m_tiles, nt = w / m_tiles;
+                for (int kb = 0; kb < kb_count; ++kb) {
+                    if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t bar = smem_u32(&ctl->full[s]);
+                    mbar_expect_tx(bar, STAGE_BYTES);
+                    tma_load_2d(tiles + s * STAGE_BYTES, &map_a, kb * BK, mt * BM, bar);
+                    tma_load_2d(tiles + s * STAGE_BYTES + A_BYTES, &map_b, kb * BK, nt * BN, bar);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+            }
+            if (!ok) {                                  // give copies in flight time to land before the CTA goes away
+                const long long t0 = clock64();
+                while (clock64() - t0 < 200000) { }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer ----
+        if (lane == 0) {
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            int it = 0;
+            for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++it) {
+                const uint32_t acc = it & 1, acc_ph = (it >> 1) & 1;
+                if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < kb_count; ++kb) {
+                    if (!mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = tiles + s * STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        tc_mma(d_tmem, smem_desc(sa + k * UMMA_K * 2), smem_desc(sb + k * UMMA_K * 2), kIdesc, (kb | k) != 0);
+                    tc_commit(smem_u32(&ctl->empty[s]));            // stage reusable once these MMAs have read it
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (ok) tc_commit(smem_u32(&ctl->tmem_full[acc]));  // accumulator complete
+            }
+            if (!ok) {                                  // drain issued tensor-core work before tensor memory is freed
+                tc_commit(smem_u32(&ctl->drain));
+                const long long t0 = clock64();
+                while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && clock64() - t0 < kWaitLimit) { }
+            }
+        }
+    } else {
+        // ---- epilogue: warps 2..5, each owns the 32-lane quarter (warp % 4) of tensor memory ----
+        const int quarter = warp & 3;
+        bool ok = true;
+        int it = 0;
+        for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++it) {
+            const int mt = w % m_tiles, nt = w / m_tiles;
+            const uint32_t acc = it & 1, acc_ph = (it >> 1) & 1;
+            if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_ph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const int row = mt * BM + quarter * 32 + lane;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                const int col = nt * BN + c0;
+                if (col >= g.N) break;                              // warp-uniform
+                uint32_t v[32];
+                tc_ld32(t_row + c0, v);
+                tc_wait_ld();
+                if (row < g.M) {
+                    if (g.out_f32) {
+                        float* cp = static_cast<float*>(g.C) + (size_t)row * g.ldc + col;
+                        if (col + 32 <= g.N) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                float4 o = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                                       __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                                if (g.accumulate) {
+                                    const float4 p = *reinterpret_cast<const float4*>(cp + 4 * j);
+                                    o.x += p.x; o.y += p.y; o.z += p.z; o.w += p.w;
+                                }
+                                *reinterpret_cast<float4*>(cp + 4 * j) = o;
+                            }
+                        } else {
+                            for (int j = 0; j < 32 && col + j < g.N; ++j)
+                                cp[j] = __uint_as_float(v[j]) + (g.accumulate ? cp[j] : 0.f);
+                        }
+                    } else {
+                        __nv_bfloat16* cp = static_cast<__nv_bfloat16*>(g.C) + (size_t)row * g.ldc + col;
+                        if (col + 32 <= g.N) {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                float f[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * j + e]);
+                                if (g.accumulate) {
+                                    const uint4 p = *reinterpret_cast<const uint4*>(cp + 8 * j);
+                                    const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&p);
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) { f[2 * e] += __low2float(pp[e]); f[2 * e + 1] += __high2float(pp[e]); }
+                                }
+                                uint4 o;
+                                __nv_bfloat162 t0 = __floats2bfloat162_rn(f[0], f[1]), t1 = __floats2bfloat162_rn(f[2], f[3]);
+                                __nv_bfloat162 t2 = __floats2bfloat162_rn(f[4], f[5]), t3 = __floats2bfloat162_rn(f[6], f[7]);
+                                o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
+                                o.z = *reinterpret_cast<uint32_t*>(&t2); o.w = *reinterpret_cast<uint32_t*>(&t3);
+                                *reinterpret_cast<uint4*>(cp + 8 * j) = o;
+                            }
+                        } else {
+                            for (int j = 0; j < 32 && col + j < g.N; ++j)
+                                cp[j] = __float2bfloat16_rn(__uint_as_float(v[j]) + (g.accumulate ? __bfloat162float(cp[j]) : 0.f));
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && ctl->abort) set_status(g.status, SPEC_ERR_TIMEOUT, (int)blockIdx.x);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn g_encode = nullptr;
+int g_sms = 0;
+
+bool init_once()
+{
+    if (g_encode != nullptr) return true;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr) return false;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&g_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (g_sms <= 0) g_sms = 148;
+    constexpr int smem = STAGES * STAGE_BYTES + 1024 + 256;
+    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+    g_encode = reinterpret_cast<EncodeFn>(fn);
+    return true;
+}
+
+// 2-D map over a row-major [rows][cols] bf16 matrix with row pitch ld elements; box = 64 columns x box_rows rows.
+bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows)
+{
+    const cuuint64_t gdim[2] = {cols, rows};
+    const cuuint64_t gstride[1] = {ld * 2};
+    const cuuint32_t box[2] = {BK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool gemm_tc_supported(int M, int N, int K, const void* A, int lda, const void* W, const void* C, int ldc, int dtype_in,
+                       int out_dtype)
+{
+    (void)M;
+    const int cal = out_dtype == SPEC_DTYPE_F32 ? 4 : 8;
+    return dtype_in == SPEC_DTYPE_BF16 && K % 8 == 0 && lda % 8 == 0 && N % cal == 0 && ldc % cal == 0 &&
+           (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && (reinterpret_cast<uintptr_t>(W) & 15u) == 0 &&
+           (reinterpret_cast<uintptr_t>(C) & 15u) == 0;
+}
+
+spec_status launch_gemm_tc(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int out_dtype,
+                           int accumulate, int32_t* status, cudaStream_t st)
+{
+    if (M == 0 || N == 0) return SPEC_OK;
+    if (!init_once()) return SPEC_ERR_CUDA;
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM)) return SPEC_ERR_CUDA;
+    if (!make_map(&mb, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
+    const int n_work = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    GemmArgs g{M, N, K, C, ldc, out_dtype == SPEC_DTYPE_F32 ? 1 : 0, accumulate, status};
+    constexpr int smem = STAGES * STAGE_BYTES + 1024 + 256;
+    gemm_tc_kernel<<<n_work < g_sms ? n_work : g_sms, kThreads, smem, st>>>(ma, mb, g);
+    return launch_status();
+}
+
+spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int dtype_in,
+                        int out_dtype, int accumulate, cudaStream_t st)
+{
+    if (gemm_tc_supported(M, N, K, A, lda, W, C, ldc, dtype_in, out_dtype))
+        return launch_gemm_tc(M, N, K, A, lda, W, C, ldc, out_dtype, accumulate, nullptr, st);
+    return launch_gemm_simt(M, N, K, A, lda, W, C, ldc, dtype_in, out_dtype, accumulate, st);
+}
+
+}  // namespace spec
+
+extern "C" spec_status spec_gemm(int M, int N, int K, const void* A, const void* W, void* C, int dtype_in, int out_dtype,
+                                 int accumulate, void* stream)
+{
+    if (M < 0 || N < 0 || K <= 0) return SPEC_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return SPEC_OK;
+    if (!A || !W || !C) return SPEC_ERR_INVALID_ARG;
+    return spec::launch_gemm(M, N, K, A, K, W, C, N, dtype_in, out_dtype, accumulate, (cudaStream_t)stream);
+}
