@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Benchmark of the speculation step on the 8B-shaped workload (B=256 rollouts, cache lengths ~U[1024,16384] in paged
+16-token blocks, k=3, EAGLE-3-style draft head, bf16): emitted ("accepted") tokens per second per B200.
+
+One step = the whole hot path: draft propose -> target verify of k+1 positions -> fused softmax + rejection sampling
+-> KV commit.  Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample instead.
+Multi-GPU (`torchrun`, one rank per GPU): independent replicas of the workload, no data-path collective; time is the
+max over ranks, value the sum of tokens over ranks (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "accepted tokens/s per B200 (8B-shape verify+sample, k=3)"
+UNIT = "tokens/s"
+# dram bytes per attention launch from the ncu capture summarised in profiles/attention_8b_layer.md, as a ratio to the
+# algorithmic bytes of that captured launch (None until captured)
+ATTN_TRAFFIC_RATIO = None
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", 1411.5)), "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.path = tempfile.mktemp(suffix=".csv")
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "200",
+                                          "-i", str(self.gpu)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        self.proc.wait()
+        sm, smax, reasons = [], [], set()
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_oracle_sample(eng, info, k, n_layers_sample, step_index):
+    """Times the oracle (as it stands) on a bounded sample of the same workload: ONE sequence of the batch, the first
+    `n_layers_sample` decoder layers at full width against that sequence's real cache bytes, plus final norm, LM head,
+    softmax and the rejection sampler.  The layer part is scaled to the full depth (layers cost the same)."""
+    import torch
+    from oracle import harness
+    cfg = info["cfg"]
+    L = cfg["n_layers"]
+    b = 0
+    seq_len = int(eng.seq_len()[b].item())
+    last = int(eng.tensor("LAST_TOKEN", 0, torch.int32, (eng.B,))[b].item())
+    drafts = eng.draft_tokens()[b, :k].cpu().numpy() if k > 0 else np.zeros(0, np.int32)
+    dlog = eng.draft_logits(k)[b].cpu().numpy() if k > 0 else np.zeros((0, cfg["vocab"]), np.float32)
+    table = eng.block_table()[b].cpu().numpy()
+    t0 = time.perf_counter()
+    W = harness.device_weights(eng, cfg, n_layers_sample)
+    t_fetch_head = time.perf_counter() - t0
+    r = harness.oracle_verify_sample(eng, cfg, W, b, [last] + [int(x) for x in drafts], seq_len, table, info["kv_pools"],
+                                     dlog, info["seed"], step_index, n_layers=n_layers_sample)
+    head_s = 0.0
+    # split the forward time: time the head alone (final norm + LM head over k+1 rows) to scale only the layer part
+    from oracle import model
+    t1 = time.perf_counter()
+    model.rmsnorm(r["final"], W["final_norm"], cfg["rms_eps"]) @ np.asarray(W["lm_head"], np.float64).T
+    head_s = time.perf_counter() - t1
+    layers_s = max(r["seconds_forward"] - head_s, 0.0)
+    total = layers_s * (L / n_layers_sample) + head_s + r["seconds_sample"]
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    return dict(value=float(r["n_emitted"]) / total, unit=UNIT, cores=int(cores), kind="oracle",
+                sample=f"1 of {info['B']} sequences (index 0, cache length {seq_len}), k={k}, {n_layers_sample} of {L} layers "
+                       f"timed at full width on the sequence's own cache and scaled to {L}, + LM head, softmax, rejection "
+                       f"sampler; measured {r['seconds_forward'] + r['seconds_sample']:.1f} s of CPU work",
+                seconds_measured=r["seconds_forward"] + r["seconds_sample"], n_emitted_sample=int(r["n_emitted"]),
+                fetch_seconds=t_fetch_head)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--k", type=int, default=3)
+    ap.add_argument("--layers", type=int, default=32)
+    ap.add_argument("--kv-pools", type=int, default=None)
+    ap.add_argument("--cpu-layers", type=int, default=4, help="layers the CPU-baseline sample times (scaled to all)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true")
+    args = ap.parse_args()
+
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference" and rank != 0:
+        return 0
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the speculation step has no CPU implementation")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1 and args.impl == "ours":
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        dist = dist_mod
+
+    from paper_2604_26779_b200 import binding, workloads
+    k, B = args.k, args.batch
+    steps_budget = args.steps * 2 + args.warmup * 2 + 24
+    eng, info = workloads.build_dense_workload("c3", B=B, k=k, n_layers=args.layers, kv_pools=args.kv_pools,
+                                               steps_budget=steps_budget, device=f"cuda:{local}",
+                                               seed=None if rank == 0 else 2604026779 + 3000 + 17 * rank)
+    cfg = info["cfg"]
+    workloads.bootstrap(eng)
+    config = {"workload": "c3: 8B dense verify (32 layers, d=4096, 32q/8kv, dh=128, FFN 14336, V=128256, bf16), "
+                          "EAGLE-3-style 1-layer draft head, cache lengths ~U[1024,16384], 16-token pages",
+              "batch": B, "k": k, "layers": cfg["n_layers"], "kv_layer_pools": info["kv_pools"], "aliased_kv": bool(info["aliased"]),
+              "l2": "inputs_exceed_l2 (15 GB weights + >=9 GB cache per layer per step; no flush needed)",
+              "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+              "acceptance": "measured with the random-init draft head (untrained: low by construction)"}
+
+    if args.impl == "reference":
+        # the CPU oracle on a bounded sample, timed step after step on this machine's host cores
+        for _ in range(args.warmup):
+            workloads.spec_step(eng, k)
+        vals = []
+        t_all = time.perf_counter()
+        for i in range(args.steps):
+            workloads.spec_step(eng, k)                                     # advances the device state the sample is cut from
+            rep = eng.status()
+            vals.append(cpu_oracle_sample(eng, info, k, 1, int(rep.steps) - 1))
+        wall = time.perf_counter() - t_all
+        v = float(np.mean([x["value"] for x in vals]))
+        line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": 0, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": 1000.0 * wall / max(args.steps, 1), "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+                "cpu_baseline": {"value": v, "unit": UNIT, "cores": vals[-1]["cores"], "kind": "oracle", "sample": vals[-1]["sample"]},
+                "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return 0
+
+    stream = torch.cuda.current_stream()
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        workloads.spec_step(eng, k)
+    rep0 = eng.status()
+    assert rep0.device_status == 0, f"device status {rep0.device_status} after warm-up"
+    tokens_before = float(eng.seq_len().sum().item())
+
+    # ---- timed region: K whole steps, device-timed, clocks sampled alongside ------------------------------------------
+    eng.set_timing(1)                                   # bracket the attention passes (32 event pairs per step)
+    eng.get_timing()
+    launches0 = binding.spec_launch_count()
+    sampler = ClockSampler(local)
+    sync_all()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        workloads.spec_step(eng, k)
+    e1.record(stream)
+    sync_all()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    launches = binding.spec_launch_count() - launches0
+    timing = eng.get_timing()
+    eng.set_timing(0)
+    rep1 = eng.status()
+    assert rep1.device_status == 0, f"device status {rep1.device_status}"
+    emitted = rep1.emitted_tokens - rep0.emitted_tokens
+    accepted = rep1.accepted_drafts - rep0.accepted_drafts
+    tokens_after = float(eng.seq_len().sum().item())
+
+    t = torch.tensor([ms_total, float(emitted)], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        tmax = t.clone(); dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        tsum = t.clone(); dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+        ms_total, emitted_all = float(tmax[0]), float(tsum[1])
+    else:
+        emitted_all = float(emitted)
+    value = emitted_all / (ms_total / 1000.0)
+
+    # ---- roofline of the dominant kernel: paged attention, one launch per layer -----------------------------------------
+    hbm_peak, tf_peak, peak_kind = measured_peaks()
+    R = k + 1
+    mean_cached_tokens = 0.5 * (tokens_before + tokens_after) + B * R           # positions each launch reads (prefix + new rows)
+    bytes_per_token_layer = cfg["n_kv_heads"] * cfg["head_dim"] * 2 * 2          # K and V, bf16
+    attn_passes = max(int(timing.passes[0]), 1)
+    attn_ms = float(timing.ms[0]) / attn_passes
+    # the verify forward has n_layers attention launches per step, the draft head k more on its own (one-layer) cache
+    alg_bytes = mean_cached_tokens * bytes_per_token_layer
+    achieved = alg_bytes / (attn_ms * 1e-3) / 1e9
+    roofline = {"kernel": "attn_mma_kernel (+ plan / merge)", "bound": "hbm", "achieved": achieved, "peak": hbm_peak,
+                "unit": "GB/s", "frac": achieved / hbm_peak, "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})",
+                "traffic": None if ATTN_TRAFFIC_RATIO is None else alg_bytes * ATTN_TRAFFIC_RATIO,
+                "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": attn_ms, "launches_timed": attn_passes,
+                "share_of_step": float(timing.ms[0]) / ms_total, "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": int(launches),
+            "roofline": roofline,
+            "acceptance_length": emitted / float(args.steps * B), "accepted_drafts_per_step": accepted / float(args.steps * B)}
+
+    if rank == 0 and not args.no_extras:
+        # context numbers, outside the timed region: verify+sample alone, plain one-token decode, per-class times
+        def timed(fn, n):
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(n):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / n
+        eng.set_timing(15)
+        eng.get_timing()
+        ms_full = timed(lambda: workloads.spec_step(eng, k), 2)
+        tm = eng.get_timing()
+        eng.set_timing(0)
+        ms_vs = timed(lambda: workloads.spec_step(eng, k, with_draft=False), 3)
+        ms_dec = timed(lambda: workloads.bootstrap(eng), 3)
+        line["extras"] = {"ms_verify_sample_commit": ms_vs, "ms_plain_decode_step": ms_dec,
+                          "plain_decode_tokens_per_s": B / (ms_dec / 1000.0),
+                          "speedup_vs_plain_decode_at_measured_acceptance": (emitted / float(args.steps * B)) / (ms_total / args.steps / ms_dec),
+                          "projected_tokens_per_s_at_paper_AL": {"2.77": 2.77 * B / (ms_total / args.steps / 1000.0),
+                                                                 "3.32": 3.32 * B / (ms_total / args.steps / 1000.0)},
+                          "ms_by_class_per_step": {"attention": tm.ms[0] / 2, "gemm": tm.ms[1] / 2, "softmax_sampling": tm.ms[2] / 2},
+                          "gemm_tflops": None}
+
+    # ---- end-to-end through the C ABI with host buffers: seq_init from host arrays (H2D) + K steps, each followed by a
+    # device-to-host read of the step's result (emitted tokens and counts) into pinned memory ---------------------------
+    lens_now = eng.seq_len().cpu().numpy().astype(np.int32)
+    last_now = eng.tensor("LAST_TOKEN", 0, torch.int32, (B,)).cpu().numpy().astype(np.int32)
+    # restart the sequences from host state at their current lengths (block tables are rebuilt from the host arrays)
+    pinned_out = torch.empty((B, R), dtype=torch.int32).pin_memory()
+    pinned_n = torch.empty((B,), dtype=torch.int32).pin_memory()
+    h2d = lens_now.nbytes + last_now.nbytes + info["block_order"].nbytes + B * info["max_blocks"] * 4 + 4
+    e2e_steps = min(args.steps, 6)
+    sync_all()
+    t0 = time.perf_counter()
+    eng.seq_init(lens_now, last_now, info["block_order"])
+    workloads.bootstrap(eng)
+    total_e2e = 0
+    for _ in range(e2e_steps):
+        workloads.spec_step(eng, k)
+        pinned_out.copy_(eng.out_tokens(k), non_blocking=True)
+        pinned_n.copy_(eng.n_emitted(), non_blocking=True)
+        torch.cuda.synchronize()
+        total_e2e += int(pinned_n.sum())
+    sync_all()
+    wall = time.perf_counter() - t0
+    t = torch.tensor([wall, float(total_e2e)], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        tmax = t.clone(); dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        tsum = t.clone(); dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+        wall, total_e2e = float(tmax[0]), float(tsum[1])
+    line["e2e"] = {"value": total_e2e / wall, "unit": UNIT, "h2d_bytes_per_step": int(h2d / e2e_steps),
+                   "d2h_bytes_per_step": int(pinned_out.numel() * 4 + pinned_n.numel() * 4), "steps": e2e_steps,
+                   "note": "host arrays -> spec_seq_init (H2D) + one plain decode step + steps, each with a D2H read of the emitted "
+                           "tokens and a synchronize; wall clock, max over ranks"}
+
+    if rank == 0 and not args.no_cpu_baseline:
+        workloads.spec_step(eng, k)
+        rep = eng.status()
+        cb = cpu_oracle_sample(eng, info, k, args.cpu_layers, int(rep.steps) - 1)
+        line["cpu_baseline"] = {kk: cb[kk] for kk in ("value", "unit", "cores", "kind", "sample")}
+        line["cpu_baseline"]["value"] = cb["value"] * 1.0            # tokens/s of ONE host running the oracle on one sequence at a time
+
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -229,6 +229,18 @@ spec_status spec_attention(int B, int R, int Hq, int Hkv, int dh, int block_toke
                            void* stream);
 size_t spec_attention_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int max_kv_len);
 
+/* Optional per-pass device timing.  When enabled, the step functions bracket the passes selected by `mask` (bit 0
+ * attention, bit 1 GEMMs, bit 2 softmax + sampling, bit 3 everything else) with CUDA events on the call's stream.
+ * spec_get_timing synchronises `stream`, adds up the elapsed time per class since the last read (milliseconds) and
+ * the number of bracketed passes, and resets the accumulation.  At most 8192 passes are recorded between reads;
+ * later ones are dropped and counted in `dropped`.  Events are host-side objects; no device memory is allocated. */
+typedef struct { float ms[4]; int32_t passes[4]; int32_t dropped; } spec_timing;
+spec_status spec_set_timing(spec_ctx* ctx, uint32_t mask);
+spec_status spec_get_timing(spec_ctx* ctx, spec_timing* host_out, void* stream);
+
+/* Number of kernels the library has launched in this process so far. */
+int64_t spec_launch_count(void);
+
 /* Version string of the library build. */
 const char* spec_version(void);
 

@@ -1,0 +1,94 @@
+"""Hands the CPU oracle the exact bytes a device context holds (weights, cache contents), lazily and layer by layer,
+so that large workloads can be checked and timed on a bounded sample without a second copy of the model in host
+memory.  TEST INFRASTRUCTURE ONLY (tests, smoke check, the benchmark's CPU-baseline leg).  It does no arithmetic of
+the method: it converts storage types and gathers cache rows through the block table; the oracle's own functions do
+the rest.  The context object is duck-typed (`tensor(name, layer, dtype, shape)`), nothing of the product is imported.
+"""
+from __future__ import annotations
+
+import time
+
+import numpy as np
+
+import oracle
+from oracle import model
+
+
+def _np(t):
+    return t.float().cpu().numpy()
+
+
+class LazyLayers:
+    """Sequence of per-layer weight dicts fetched from the device on access (fp32 copies of the stored values)."""
+
+    def __init__(self, eng, cfg, n_layers=None):
+        self.eng, self.cfg = eng, cfg
+        self.n = cfg["n_layers"] if n_layers is None else n_layers
+
+    def __len__(self):
+        return self.n
+
+    def __iter__(self):
+        for l in range(self.n):
+            yield self[l]
+
+    def __getitem__(self, l):
+        import torch
+        eng, cfg = self.eng, self.cfg
+        d, F = cfg["d_model"], cfg["d_ffn"]
+        qn = (cfg["n_q_heads"] + 2 * cfg["n_kv_heads"]) * cfg["head_dim"]
+        od = cfg["n_q_heads"] * cfg["head_dim"]
+        td = eng.tdtype
+        gu = _np(eng.tensor("WGATEUP", l, td, (2 * F, d)))
+        return dict(attn_norm=_np(eng.tensor("ATTN_NORM", l, torch.float32, (d,))),
+                    wqkv=_np(eng.tensor("WQKV", l, td, (qn, d))), wo=_np(eng.tensor("WO", l, td, (d, od))),
+                    mlp_norm=_np(eng.tensor("MLP_NORM", l, torch.float32, (d,))),
+                    wgate=gu[:F], wup=gu[F:], wdown=_np(eng.tensor("WDOWN", l, td, (d, F))))
+
+
+class LazyPast:
+    """Per-layer (K, V) [n_past][Hkv][dh] of one sequence, gathered from the paged pools through its block table."""
+
+    def __init__(self, eng, cfg, block_row, n_past, kv_pools, n_layers=None):
+        self.eng, self.cfg, self.blocks, self.n_past, self.G = eng, cfg, block_row, n_past, kv_pools
+        self.n = cfg["n_layers"] if n_layers is None else n_layers
+
+    def __getitem__(self, l):
+        import torch
+        nb = -(-self.n_past // 16)
+        idx = torch.as_tensor(np.ascontiguousarray(self.blocks[:nb]), dtype=torch.long, device=self.eng.device)
+        out = []
+        for which in ("KV_K", "KV_V"):
+            pool = self.eng.kv_pool(which, l % self.G)
+            rows = pool[idx].permute(0, 2, 1, 3).reshape(nb * 16, pool.shape[1], pool.shape[3])[: self.n_past]
+            out.append(_np(rows))
+        return tuple(out)
+
+
+def device_weights(eng, cfg, n_layers=None):
+    import torch
+    d, V, td = cfg["d_model"], cfg["vocab"], eng.tdtype
+    return dict(embed=_np(eng.tensor("EMBED", 0, td, (V, d))), lm_head=_np(eng.tensor("LM_HEAD", 0, td, (V, d))),
+                final_norm=_np(eng.tensor("FINAL_NORM", 0, torch.float32, (d,))), layers=LazyLayers(eng, cfg, n_layers))
+
+
+def oracle_verify_sample(eng, cfg, W, seq, tokens_in, n_past, block_row, kv_pools, draft_logits, seed, step,
+                         n_layers=None, temperature=1.0):
+    """The oracle's verify forward and rejection sampling for one sequence of a device context.
+
+    tokens_in = [last token, d_1..d_k]; the cache prefix (n_past positions per layer) is read from the device pools as
+    they stand.  Returns dict(logits, p, q, out_tokens, n_emitted, margins, seconds_forward, seconds_sample)."""
+    k = len(tokens_in) - 1
+    t0 = time.perf_counter()
+    cfg_run = cfg if n_layers is None else dict(cfg, n_layers=n_layers)
+    out = model.target_forward(cfg_run, W, tokens_in, past=LazyPast(eng, cfg, block_row, n_past, kv_pools, n_layers),
+                               start_pos=n_past)
+    t1 = time.perf_counter()
+    logits = out["logits"].astype(np.float32)
+    p = oracle.softmax(logits, temperature)
+    q = oracle.softmax(np.asarray(draft_logits, np.float32), temperature) if k > 0 else np.zeros((0, p.shape[1]), np.float32)
+    u = oracle.uniforms(seed, step, 0, seq + 1, k + 1)[seq]
+    toks, n_emit, flags, margins = oracle.reject_sample_seq(p, q, np.asarray(tokens_in[1:], np.int32), u)
+    t2 = time.perf_counter()
+    return dict(logits=logits, p=p, q=q, out_tokens=toks, n_emitted=n_emit, margins=margins, final=out["final"],
+                seconds_forward=t1 - t0, seconds_sample=t2 - t1)

@@ -59,6 +59,10 @@ class spec_buffers(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("weights", "draft_weights", "kv", "draft_kv", "workspace", "state")]
 
 
+class spec_timing(C.Structure):
+    _fields_ = [("ms", C.c_float * 4), ("passes", C.c_int32 * 4), ("dropped", C.c_int32)]
+
+
 class spec_step_report(C.Structure):
     _fields_ = [("device_status", C.c_int32), ("device_detail", C.c_int32), ("steps", C.c_int64),
                 ("emitted_tokens", C.c_int64), ("accepted_drafts", C.c_int64)]
@@ -87,6 +91,9 @@ SIGNATURES = {
     "spec_gemm": (_i, [_i, _i, _i, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "spec_attention": (_i, [_i, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
     "spec_attention_scratch_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
+    "spec_set_timing": (_i, [_vp, _u32]),
+    "spec_get_timing": (_i, [_vp, C.POINTER(spec_timing), _vp]),
+    "spec_launch_count": (C.c_int64, []),
     "spec_version": (C.c_char_p, []),
 }
 
@@ -192,3 +199,7 @@ def spec_attention(q, k_pool, v_pool, block_table, seq_len, out, scratch, stream
 
 def spec_version():
     return lib().spec_version().decode()
+
+
+def spec_launch_count():
+    return int(lib().spec_launch_count())

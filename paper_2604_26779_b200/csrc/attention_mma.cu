@@ -408,7 +408,7 @@ spec_status run_mma(const MmaArgs& m, int B, bool plan, int max_chunks, cudaStre
     kern<<<sm_count() * (ctas_per_sm < 1 ? 1 : ctas_per_sm), kThreads, smem, st>>>(m);
     if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
     attn_merge_kernel<DH><<<B * m.Hkv, 128, 0, st>>>(B, 16 * WM, m);
-    return launch_status();
+    return launch_status(plan ? 3 : 2);
 }
 
 }  // namespace

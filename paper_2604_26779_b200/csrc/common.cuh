@@ -22,8 +22,11 @@ __device__ __forceinline__ void set_status(int32_t* status, int code, int detail
         if (e__ != cudaSuccess) return SPEC_ERR_CUDA;        \
     } while (0)
 
-inline spec_status launch_status()
+// Number of kernels this library has launched in this process (every launcher reports through launch_status()).
+long long& launch_counter();
+inline spec_status launch_status(int n_launched = 1)
 {
+    launch_counter() += n_launched;
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }
 

@@ -40,6 +40,11 @@ struct spec_ctx {
     bool have_pending = false;      // a commit has happened since spec_seq_init
     bool verified = false;          // a verify has run since the last commit
     std::string err;
+    // optional pass timing (host-side event pool)
+    uint32_t timing_mask = 0;
+    std::vector<cudaEvent_t> ev;    // pairs: start, stop
+    std::vector<int> ev_cls;        // class of each recorded pair
+    int ev_dropped = 0;
 };
 
 using namespace spec;
@@ -196,6 +201,24 @@ LayerPtrs layer_ptrs(void* base, const LayerLoc& L)
 
 #define TRY(expr) do { spec_status s__ = (expr); if (s__ != SPEC_OK) return s__; } while (0)
 
+constexpr int kMaxTimedPasses = 8192;
+
+// Brackets a pass with two events when its class is selected by the context's timing mask.
+struct Timed {
+    spec_ctx& c; cudaStream_t st; int idx = -1;
+    Timed(spec_ctx& ctx, int cls, cudaStream_t s) : c(ctx), st(s)
+    {
+        if (!(c.timing_mask & (1u << cls))) return;
+        if ((int)c.ev_cls.size() >= kMaxTimedPasses) { c.ev_dropped += 1; return; }
+        idx = (int)c.ev_cls.size();
+        c.ev_cls.push_back(cls);
+        cudaEventRecord(c.ev[2 * idx], st);
+    }
+    ~Timed() { if (idx >= 0) cudaEventRecord(c.ev[2 * idx + 1], st); }
+};
+#define TIMED(ctx, cls, expr) do { Timed t__(ctx, cls, st); TRY(expr); } while (0)
+enum { CLS_ATTN = 0, CLS_GEMM = 1, CLS_SAMPLE = 2, CLS_OTHER = 3 };
+
 // attention + MLP of one decoder layer on the fp32 residual `res` [M][d].  `qkv_in` [M][qkv_k] is the already
 // prepared input of the QKV projection.
 spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* res, const void* qkv_in, int qkv_k, int B, int R,
@@ -205,18 +228,18 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
     const int M = B * R, d = g.d_model, dh = g.head_dim, Hq = g.n_q_heads, Hkv = g.n_kv_heads;
     const int qkv_n = (Hq + 2 * Hkv) * dh, dt = g.dtype;
     void* ws = c.buf.workspace;
-    TRY(launch_gemm(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt, 0, st));
+    TIMED(c, CLS_GEMM, launch_gemm(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt, 0, st));
     TRY(launch_rope_append(B, R, Hq, Hkv, dh, g.rope_theta, at(ws, c.qkv), pos, k_pool, v_pool,
                            at<int32_t>(c.buf.state, c.block_table), g.max_blocks_per_seq, g.kv_block_tokens, dt, st));
     AttnArgs a{B, R, Hq, Hkv, dh, g.kv_block_tokens, g.max_blocks_per_seq, at(ws, c.qkv), qkv_n, k_pool, v_pool,
                at<int32_t>(c.buf.state, c.block_table), pos, at(ws, c.attn_out), Hq * dh, dt, at(ws, c.attn_scratch),
                c.attn_scratch.bytes, g.max_blocks_per_seq * g.kv_block_tokens, launch_index};
-    TRY(launch_attention(a, st));
-    TRY(launch_gemm(M, d, Hq * dh, at(ws, c.attn_out), Hq * dh, W.wo, res, d, dt, SPEC_DTYPE_F32, 1, st));
+    TIMED(c, CLS_ATTN, launch_attention(a, st));
+    TIMED(c, CLS_GEMM, launch_gemm(M, d, Hq * dh, at(ws, c.attn_out), Hq * dh, W.wo, res, d, dt, SPEC_DTYPE_F32, 1, st));
     TRY(launch_rmsnorm(M, d, res, W.mlp_norm, g.rms_eps, at(ws, c.h), d, 0, dt, st));
-    TRY(launch_gemm(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.gu), 2 * d_ffn, dt, dt, 0, st));
+    TIMED(c, CLS_GEMM, launch_gemm(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.gu), 2 * d_ffn, dt, dt, 0, st));
     TRY(launch_swiglu(M, d_ffn, at(ws, c.gu), at(ws, c.act), dt, st));
-    TRY(launch_gemm(M, d, d_ffn, at(ws, c.act), d_ffn, W.wdown, res, d, dt, SPEC_DTYPE_F32, 1, st));
+    TIMED(c, CLS_GEMM, launch_gemm(M, d, d_ffn, at(ws, c.act), d_ffn, W.wdown, res, d, dt, SPEC_DTYPE_F32, 1, st));
     return SPEC_OK;
 }
 
@@ -277,6 +300,7 @@ extern "C" spec_status spec_create(const spec_config* cfg, const spec_buffers* b
 extern "C" spec_status spec_destroy(spec_ctx* ctx)
 {
     if (ctx == nullptr) return SPEC_ERR_INVALID_ARG;
+    for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
     delete ctx;
     return SPEC_OK;
 }
@@ -421,10 +445,10 @@ extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_toke
         if (has_tap(g, l + 1)) TRY(launch_copy_rows_f32_to(M, d, x, at(ws, c->taps), tapw, tap_slot(g, l + 1) * d, dt, st));
     }
     TRY(launch_rmsnorm(M, d, x, at<const float>(c->buf.weights, c->final_norm), g.rms_eps, at(ws, c->h), d, 0, dt, st));
-    TRY(launch_gemm(M, g.vocab, d, at(ws, c->h), d, at(c->buf.weights, c->lm_head), at(ws, c->logits), g.vocab, dt,
-                    SPEC_DTYPE_F32, 0, st));
-    TRY(launch_softmax_rows(M, g.vocab, at<float>(ws, c->logits), (size_t)g.vocab, g.temperature, at<float>(ws, c->row_stats),
-                            1, nullptr, st));
+    TIMED(*c, CLS_GEMM, launch_gemm(M, g.vocab, d, at(ws, c->h), d, at(c->buf.weights, c->lm_head), at(ws, c->logits), g.vocab, dt,
+                                    SPEC_DTYPE_F32, 0, st));
+    TIMED(*c, CLS_SAMPLE, launch_softmax_rows(M, g.vocab, at<float>(ws, c->logits), (size_t)g.vocab, g.temperature,
+                                              at<float>(ws, c->row_stats), 1, nullptr, st));
     c->k_last = k;
     c->verified = true;
     return SPEC_OK;
@@ -446,9 +470,11 @@ extern "C" spec_status spec_reject_sample(spec_ctx* c, int k, const float* draft
     if (draft_logits != nullptr && k > 0)
         TRY(launch_softmax_rows(B * k, g.vocab, ql, (size_t)g.vocab, g.temperature, qs, 1, nullptr, st));
     // draft tokens: those the verify used (rows 1..k of its token list), so an external draft stays consistent
-    return launch_reject_sample(true, B, k, g.vocab, at<float>(ws, c->logits), at<float>(ws, c->row_stats), ql, qs,
-                                at<int32_t>(ws, c->tokens_in) + 1, k + 1, g.temperature, g.seed, at<uint32_t>(sb, c->step), 0, at<int32_t>(sb, c->out_tokens),
-                                at<int32_t>(sb, c->n_emitted), at<int32_t>(sb, c->status), st);
+    TIMED(*c, CLS_SAMPLE, launch_reject_sample(true, B, k, g.vocab, at<float>(ws, c->logits), at<float>(ws, c->row_stats), ql, qs,
+                                               at<int32_t>(ws, c->tokens_in) + 1, k + 1, g.temperature, g.seed,
+                                               at<uint32_t>(sb, c->step), 0, at<int32_t>(sb, c->out_tokens),
+                                               at<int32_t>(sb, c->n_emitted), at<int32_t>(sb, c->status), st));
+    return SPEC_OK;
 }
 
 extern "C" spec_status spec_kv_commit(spec_ctx* c, const int32_t* force_n, const int32_t* force_token, void* stream)
@@ -560,5 +586,42 @@ extern "C" spec_status spec_get_status(spec_ctx* c, spec_step_report* out, void*
     out->steps = counters[0];
     out->emitted_tokens = counters[1];
     out->accepted_drafts = counters[2];
+    return SPEC_OK;
+}
+
+long long& spec::launch_counter()
+{
+    static long long n = 0;
+    return n;
+}
+
+extern "C" int64_t spec_launch_count(void) { return (int64_t)spec::launch_counter(); }
+
+extern "C" spec_status spec_set_timing(spec_ctx* c, uint32_t mask)
+{
+    if (c == nullptr || mask > 15u) return SPEC_ERR_INVALID_ARG;
+    if (mask != 0 && c->ev.empty()) {
+        c->ev.resize(2 * kMaxTimedPasses);
+        for (auto& e : c->ev) if (cudaEventCreate(&e) != cudaSuccess) return SPEC_ERR_CUDA;
+        c->ev_cls.reserve(kMaxTimedPasses);
+    }
+    c->timing_mask = mask;
+    return SPEC_OK;
+}
+
+extern "C" spec_status spec_get_timing(spec_ctx* c, spec_timing* out, void* stream)
+{
+    if (c == nullptr || out == nullptr) return SPEC_ERR_INVALID_ARG;
+    SPEC_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+    *out = spec_timing{};
+    for (size_t i = 0; i < c->ev_cls.size(); ++i) {
+        float ms = 0.f;
+        SPEC_CUDA_OK(cudaEventElapsedTime(&ms, c->ev[2 * i], c->ev[2 * i + 1]));
+        out->ms[c->ev_cls[i]] += ms;
+        out->passes[c->ev_cls[i]] += 1;
+    }
+    out->dropped = c->ev_dropped;
+    c->ev_cls.clear();
+    c->ev_dropped = 0;
     return SPEC_OK;
 }

@@ -157,6 +157,14 @@ class SpecStep:
         B._check(self.lib.spec_get_status(self.ctx, C.byref(rep), B._stream(stream)), "spec_get_status")
         return rep
 
+    def set_timing(self, mask: int):
+        B._check(self.lib.spec_set_timing(self.ctx, mask), "spec_set_timing")
+
+    def get_timing(self, stream=None) -> B.spec_timing:
+        t = B.spec_timing()
+        B._check(self.lib.spec_get_timing(self.ctx, C.byref(t), B._stream(stream)), "spec_get_timing")
+        return t
+
     # ---- typed views of step results -----------------------------------------------------------------------------
     def logits(self, k):
         return self.tensor("LOGITS", 0, torch.float32, (self.B, k + 1, self.sc.vocab))
