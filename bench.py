@@ -148,12 +148,12 @@ def main():
         dist_mod.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
         dist = dist_mod
 
-    from paper_2604_26779_b200 import binding, workloads
+    from paper_2604_26779_b200 import binding, replicas, workloads
     k, B = args.k, args.batch
     steps_budget = args.steps * 2 + args.warmup * 2 + 24
     eng, info = workloads.build_dense_workload("c3", B=B, k=k, n_layers=args.layers, kv_pools=args.kv_pools,
                                                steps_budget=steps_budget, device=f"cuda:{local}",
-                                               seed=None if rank == 0 else 2604026779 + 3000 + 17 * rank)
+                                               seed=replicas.replica_seed(rank))
     cfg = info["cfg"]
     workloads.bootstrap(eng)
     config = {"workload": "c3: 8B dense verify (32 layers, d=4096, 32q/8kv, dh=128, FFN 14336, V=128256, bf16), "
@@ -221,13 +221,7 @@ def main():
     accepted = rep1.accepted_drafts - rep0.accepted_drafts
     tokens_after = float(eng.seq_len().sum().item())
 
-    t = torch.tensor([ms_total, float(emitted)], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        tmax = t.clone(); dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        tsum = t.clone(); dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
-        ms_total, emitted_all = float(tmax[0]), float(tsum[1])
-    else:
-        emitted_all = float(emitted)
+    ms_total, emitted_all = replicas.reduce_job(ms_total, float(emitted), dist, "cuda")
     value = emitted_all / (ms_total / 1000.0)
 
     # ---- roofline of the dominant kernel: paged attention, one launch per layer -----------------------------------------
@@ -237,7 +231,7 @@ def main():
     bytes_per_token_layer = cfg["n_kv_heads"] * cfg["head_dim"] * 2 * 2          # K and V, bf16
     attn_passes = max(int(timing.passes[0]), 1)
     attn_ms = float(timing.ms[0]) / attn_passes
-    # the verify forward has n_layers attention launches per step, the draft head k more on its own (one-layer) cache
+    # n_layers launches per step on the target's cache and k on the draft head's one-layer cache: the same positions each
     alg_bytes = mean_cached_tokens * bytes_per_token_layer
     achieved = alg_bytes / (attn_ms * 1e-3) / 1e9
     roofline = {"kernel": "attn_mma_kernel (+ plan / merge)", "bound": "hbm", "achieved": achieved, "peak": hbm_peak,
@@ -276,7 +270,7 @@ def main():
                           "projected_tokens_per_s_at_paper_AL": {"2.77": 2.77 * B / (ms_total / args.steps / 1000.0),
                                                                  "3.32": 3.32 * B / (ms_total / args.steps / 1000.0)},
                           "ms_by_class_per_step": {"attention": tm.ms[0] / 2, "gemm": tm.ms[1] / 2, "softmax_sampling": tm.ms[2] / 2},
-                          "gemm_tflops": None}
+                          }
 
     # ---- end-to-end through the C ABI with host buffers: seq_init from host arrays (H2D) + K steps, each followed by a
     # device-to-host read of the step's result (emitted tokens and counts) into pinned memory ---------------------------
@@ -300,11 +294,7 @@ def main():
         total_e2e += int(pinned_n.sum())
     sync_all()
     wall = time.perf_counter() - t0
-    t = torch.tensor([wall, float(total_e2e)], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        tmax = t.clone(); dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        tsum = t.clone(); dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
-        wall, total_e2e = float(tmax[0]), float(tsum[1])
+    wall, total_e2e = replicas.reduce_job(wall, float(total_e2e), dist, "cuda")
     line["e2e"] = {"value": total_e2e / wall, "unit": UNIT, "h2d_bytes_per_step": int(h2d / e2e_steps),
                    "d2h_bytes_per_step": int(pinned_out.numel() * 4 + pinned_n.numel() * 4), "steps": e2e_steps,
                    "note": "host arrays -> spec_seq_init (H2D) + one plain decode step + steps, each with a D2H read of the emitted "
