@@ -229,6 +229,27 @@ spec_status spec_attention(int B, int R, int Hq, int Hkv, int dh, int block_toke
                            void* stream);
 size_t spec_attention_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int max_kv_len);
 
+/* spec_attention for callers that cannot allocate device memory.  (The paper has no counterpart: this is a
+ * convenience of the library.)  Some callers of this code run where cudaMalloc is off limits: inside a host
+ * program that has handed all device memory to another allocator and forbids further driver allocations, in a
+ * plug-in that may only enqueue work on a stream it is given, or in a latency-critical loop where an allocation
+ * would serialise the device.  They cannot provide the scratch buffer spec_attention asks for, so this variant
+ * keeps the scratch in a 32 MiB array built into the library image (every GPU that loads the library holds those
+ * 32 MiB until the process exits).  Arguments, layouts and results are those of spec_attention; inputs and outputs
+ * are still the caller's.
+ *   - Sizes: returns SPEC_ERR_SHAPE, launching nothing, when spec_attention_scratch_bytes(B, R, Hq, Hkv, dh,
+ *     max_blocks * block_tokens) exceeds 32 MiB (33554432 bytes); for the 8B head shape with k = 3 that allows,
+ *     for example, 16 sequences of up to 16384 cached positions per call.
+ *   - The first call on each device looks up the array's device address (with that device current); make that
+ *     first call outside any stream capture.  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - All calls share the one array, which keeps whatever the last call left; every call rewrites what it reads
+ *     (row positions, work counters, partial results), so results do not depend on earlier calls.  Two calls that
+ *     overlap on the GPU (different streams, or different host threads) race on the array: serialise them.
+ * Errors: INVALID_ARG, SHAPE (see above), CUDA. */
+spec_status spec_attention_noalloc(int B, int R, int Hq, int Hkv, int dh, int block_tokens, int max_blocks,
+                                   const void* q, const void* k_pool, const void* v_pool, const int32_t* block_table,
+                                   const int32_t* seq_len, void* out, int dtype, void* stream);
+
 /* Optional per-pass device timing.  When enabled, the step functions bracket the passes selected by `mask` (bit 0
  * attention, bit 1 GEMMs, bit 2 softmax + sampling, bit 3 everything else) with CUDA events on the call's stream.
  * spec_get_timing synchronises `stream`, adds up the elapsed time per class since the last read (milliseconds) and

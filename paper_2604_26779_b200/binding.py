@@ -91,6 +91,7 @@ SIGNATURES = {
     "spec_gemm": (_i, [_i, _i, _i, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "spec_attention": (_i, [_i, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
     "spec_attention_scratch_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
+    "spec_attention_noalloc": (_i, [_i, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp]),
     "spec_set_timing": (_i, [_vp, _u32]),
     "spec_get_timing": (_i, [_vp, C.POINTER(spec_timing), _vp]),
     "spec_launch_count": (C.c_int64, []),
@@ -195,6 +196,18 @@ def spec_attention(q, k_pool, v_pool, block_table, seq_len, out, scratch, stream
     _check(lib().spec_attention(B, R, Hq, Hkv, dh, bt, block_table.shape[1], _ptr(q), _ptr(k_pool), _ptr(v_pool),
                                 _ptr(block_table), _ptr(seq_len), _ptr(out), dt, _ptr(scratch),
                                 scratch.numel() * scratch.element_size(), _stream(stream)), "spec_attention")
+
+
+def spec_attention_noalloc(q, k_pool, v_pool, block_table, seq_len, out, stream=None):
+    """spec_attention with the library's built-in 32 MiB scratch: for callers that must not allocate device memory.
+    Raises SpecError(SPEC_ERR_SHAPE) when the shapes need more scratch than that."""
+    import torch
+    B, R, Hq, dh = q.shape
+    _, Hkv, bt, _ = k_pool.shape
+    dt = SPEC_DTYPE_F32 if q.dtype == torch.float32 else SPEC_DTYPE_BF16
+    _check(lib().spec_attention_noalloc(B, R, Hq, Hkv, dh, bt, block_table.shape[1], _ptr(q), _ptr(k_pool), _ptr(v_pool),
+                                        _ptr(block_table), _ptr(seq_len), _ptr(out), dt, _stream(stream)),
+           "spec_attention_noalloc")
 
 
 def spec_version():

@@ -142,3 +142,45 @@ extern "C" spec_status spec_attention(int B, int R, int Hq, int Hkv, int dh, int
                max_blocks * block_tokens, 0};
     return launch_attention(a, st);
 }
+
+// ---- attention without caller-provided scratch ------------------------------------------------------------------------
+// Built-in scratch for spec_attention_noalloc: one array per GPU that loads the library, held until the process exits.
+namespace {
+constexpr size_t kBuiltinScratchBytes = (size_t)32 << 20;                 // 32 MiB
+static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
+constexpr int kMaxDevices = 64;
+void* g_builtin_scratch_addr[kMaxDevices] = {};                          // device address of the array, per device
+}  // namespace
+
+extern "C" spec_status spec_attention_noalloc(int B, int R, int Hq, int Hkv, int dh, int block_tokens, int max_blocks,
+                                              const void* q, const void* k_pool, const void* v_pool,
+                                              const int32_t* block_table, const int32_t* seq_len, void* out, int dtype,
+                                              void* stream)
+{
+    if (B < 0 || R <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || dh <= 0 || dh % 8 != 0 || block_tokens <= 0 ||
+        max_blocks <= 0)
+        return SPEC_ERR_INVALID_ARG;
+    if (B == 0) return SPEC_OK;
+    if (!q || !k_pool || !v_pool || !block_table || !seq_len || !out) return SPEC_ERR_INVALID_ARG;
+    // what spec_attention would ask the caller for must fit the built-in array
+    const size_t pos_bytes = align_up((size_t)B * R * sizeof(int32_t), 256);
+    const size_t need = pos_bytes + attention_scratch_bytes(B, R, Hq, Hkv, dh, max_blocks * block_tokens);
+    if (need > kBuiltinScratchBytes) return SPEC_ERR_SHAPE;
+    // once per device, with that device current: the array's name is a host-side handle, not a device address
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SPEC_ERR_CUDA;
+    if (g_builtin_scratch_addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_builtin_scratch) != cudaSuccess || p == nullptr) return SPEC_ERR_CUDA;
+        g_builtin_scratch_addr[dev] = p;
+    }
+    char* scratch = static_cast<char*>(g_builtin_scratch_addr[dev]);
+    cudaStream_t st = (cudaStream_t)stream;
+    // the row positions are rewritten and the work counters re-zeroed by every call, so nothing depends on what the
+    // previous call left in the array
+    launch_attn_rows(B, R, seq_len, (int32_t*)scratch, st);
+    AttnArgs a{B, R, Hq, Hkv, dh, block_tokens, max_blocks, q, Hq * dh, k_pool, v_pool, block_table,
+               (const int32_t*)scratch, out, Hq * dh, dtype, scratch + pos_bytes, kBuiltinScratchBytes - pos_bytes,
+               max_blocks * block_tokens, 0};
+    return launch_attention(a, st);
+}
