@@ -119,7 +119,10 @@ enum {
     SPEC_T_ROW_STATS,           /* [B*(k+1)][2] fp32 (max, sum exp) of the target rows                 */
     SPEC_T_DRAFT_ROW_STATS,     /* [B*k][2]                                                            */
     SPEC_T_TAPS,                /* [B][k+1][n_taps*d] tapped hidden states of the last verify          */
-    SPEC_T_HIDDEN               /* [B*(k+1)][d] fp32 residual stream after the last layer              */
+    SPEC_T_HIDDEN,              /* [B*(k+1)][d] fp32 residual stream after the last layer              */
+    SPEC_T_MOE_LOGITS,          /* [B*(k+1)][n_experts] fp32 router logits of the last MoE layer run   */
+    SPEC_T_MOE_IDS,             /* [B*(k+1)][experts_top_k] int32 selected experts, best first         */
+    SPEC_T_MOE_WTS              /* [B*(k+1)][experts_top_k] fp32 renormalised mixture weights          */
 };
 
 /* Counters returned by spec_get_status (host struct). */

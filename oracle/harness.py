@@ -18,6 +18,16 @@ def _np(t):
     return t.float().cpu().numpy()
 
 
+class _LazyRows:
+    """Per-expert weight matrices [E][rows][cols] fetched from the device one expert at a time."""
+
+    def __init__(self, dev_tensor, r0, r1):
+        self.t, self.r0, self.r1 = dev_tensor, r0, r1
+
+    def __getitem__(self, e):
+        return _np(self.t[int(e), self.r0 : self.r1])
+
+
 class LazyLayers:
     """Sequence of per-layer weight dicts fetched from the device on access (fp32 copies of the stored values)."""
 
@@ -39,11 +49,19 @@ class LazyLayers:
         qn = (cfg["n_q_heads"] + 2 * cfg["n_kv_heads"]) * cfg["head_dim"]
         od = cfg["n_q_heads"] * cfg["head_dim"]
         td = eng.tdtype
-        gu = _np(eng.tensor("WGATEUP", l, td, (2 * F, d)))
-        return dict(attn_norm=_np(eng.tensor("ATTN_NORM", l, torch.float32, (d,))),
-                    wqkv=_np(eng.tensor("WQKV", l, td, (qn, d))), wo=_np(eng.tensor("WO", l, td, (d, od))),
-                    mlp_norm=_np(eng.tensor("MLP_NORM", l, torch.float32, (d,))),
-                    wgate=gu[:F], wup=gu[F:], wdown=_np(eng.tensor("WDOWN", l, td, (d, F))))
+        lw = dict(attn_norm=_np(eng.tensor("ATTN_NORM", l, torch.float32, (d,))),
+                  wqkv=_np(eng.tensor("WQKV", l, td, (qn, d))), wo=_np(eng.tensor("WO", l, td, (d, od))),
+                  mlp_norm=_np(eng.tensor("MLP_NORM", l, torch.float32, (d,))))
+        if cfg.get("n_experts", 0) > 0:
+            E, Fe = cfg["n_experts"], cfg["d_expert_ffn"]
+            gu = eng.tensor("EXPERTS_GATEUP", l, td, (E, 2 * Fe, d))
+            dn = eng.tensor("EXPERTS_DOWN", l, td, (E, d, Fe))
+            lw.update(router=_np(eng.tensor("ROUTER", l, td, (E, d))), experts_gate=_LazyRows(gu, 0, Fe),
+                      experts_up=_LazyRows(gu, Fe, 2 * Fe), experts_down=_LazyRows(dn, 0, d))
+        else:
+            gu = _np(eng.tensor("WGATEUP", l, td, (2 * F, d)))
+            lw.update(wgate=gu[:F], wup=gu[F:], wdown=_np(eng.tensor("WDOWN", l, td, (d, F))))
+        return lw
 
 
 class LazyPast:

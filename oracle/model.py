@@ -99,8 +99,10 @@ def moe_route(router_logits, top_k):
     return ids, wts
 
 
-def moe_mlp(lw, m, top_k):
-    ids, wts = moe_route(m @ np.asarray(lw["router"], F64).T, top_k)
+def moe_mlp(lw, m, top_k, router_logits=None):
+    """router_logits, when given, replaces W_r m as the input of the top-k decision (used to take that integer
+    decision on the same numbers as an implementation under test)."""
+    ids, wts = moe_route(m @ np.asarray(lw["router"], F64).T if router_logits is None else np.asarray(router_logits, F64), top_k)
     out = np.zeros_like(m)
     for t in range(m.shape[0]):
         for e, w in zip(ids[t], wts[t]):
@@ -111,7 +113,7 @@ def moe_mlp(lw, m, top_k):
     return out
 
 
-def decoder_layer(cfg, lw, x, pos, past_k=None, past_v=None, attn_in=None):
+def decoder_layer(cfg, lw, x, pos, past_k=None, past_v=None, attn_in=None, router_logits=None):
     """One pre-norm decoder layer on rows x [T][d] at absolute positions pos.
 
     past_k / past_v [n_past][Hkv][dh] are cached (already rotated) keys and values, or None.
@@ -133,13 +135,13 @@ def decoder_layer(cfg, lw, x, pos, past_k=None, past_v=None, attn_in=None):
     x = x + att @ np.asarray(lw["wo"], F64).T
     m = rmsnorm(x, lw["mlp_norm"], cfg["rms_eps"])
     if cfg.get("n_experts", 0) > 0:
-        x = x + moe_mlp(lw, m, cfg["experts_top_k"])
+        x = x + moe_mlp(lw, m, cfg["experts_top_k"], router_logits)
     else:
         x = x + dense_mlp(lw, m)
     return x, k, v
 
 
-def target_forward(cfg, W, tokens, past=None, start_pos=0, tap_layers=()):
+def target_forward(cfg, W, tokens, past=None, start_pos=0, tap_layers=(), router_logits=None):
     """Target forward over `tokens` placed at positions start_pos, start_pos+1, ...
 
     past: None (recompute-all, no cache) or a list, per layer, of (K [n_past][Hkv][dh], V likewise).
@@ -155,7 +157,7 @@ def target_forward(cfg, W, tokens, past=None, start_pos=0, tap_layers=()):
     new_kv = []
     for l, lw in enumerate(W["layers"]):
         pk, pv = (None, None) if past is None else past[l]
-        x, k, v = decoder_layer(cfg, lw, x, pos, pk, pv)
+        x, k, v = decoder_layer(cfg, lw, x, pos, pk, pv, router_logits=None if router_logits is None else router_logits[l])
         new_kv.append((k, v))
         if (l + 1) in tap_layers:
             taps[l + 1] = x

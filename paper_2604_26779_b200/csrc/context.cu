@@ -32,7 +32,8 @@ struct spec_ctx {
     size_t state_bytes = 0;
     // workspace
     Loc tokens_in, pos, x, h, qkv, attn_out, gu, act, logits, draft_logits, row_stats, draft_row_stats, taps,
-        attn_scratch, dg, dx, d_hidden, d_tok, d_pos;
+        attn_scratch, dg, dx, d_hidden, d_tok, d_pos,
+        moe_logits, moe_ids, moe_wts, moe_rank, moe_counts, moe_offsets, moe_inv, moe_a, moe_gu, moe_act, moe_out;
     size_t workspace_bytes = 0;
     // host-side run state
     int B = 0;
@@ -75,7 +76,8 @@ spec_status check_config(const spec_config* c)
     if (c->n_q_heads % c->n_kv_heads != 0 || c->d_model % 8 != 0 || c->head_dim % 8 != 0 || c->vocab % 4 != 0) return SPEC_ERR_SHAPE;
     if (c->n_experts == 0 && (c->d_ffn <= 0 || c->d_ffn % 8 != 0)) return SPEC_ERR_SHAPE;
     if (c->n_experts > 0 && (c->experts_top_k <= 0 || c->experts_top_k > c->n_experts || c->d_expert_ffn <= 0)) return SPEC_ERR_SHAPE;
-    if (c->n_experts > 0) return SPEC_ERR_UNSUPPORTED;
+    if (c->n_experts > 0 && (c->dtype != SPEC_DTYPE_BF16 || c->n_experts > 256 || c->experts_top_k > 32 ||
+                             c->d_expert_ffn % 128 != 0 || c->d_model % 256 != 0)) return SPEC_ERR_UNSUPPORTED;
     if (c->dtype != SPEC_DTYPE_BF16 && c->dtype != SPEC_DTYPE_F32) return SPEC_ERR_UNSUPPORTED;
     if (c->draft_kind < SPEC_DRAFT_NONE || c->draft_kind > SPEC_DRAFT_MTP) return SPEC_ERR_UNSUPPORTED;
     if (c->k_max < 0 || c->k_max > 7 || c->max_batch <= 0) return SPEC_ERR_SHAPE;
@@ -185,18 +187,35 @@ void build_layout(spec_ctx& x)
         x.d_hidden = a.take(Bm * d * 4);
         x.d_tok = a.take(M * 4);
         x.d_pos = a.take(M * 4);
+        if (c.n_experts > 0) {
+            const size_t n = M * c.experts_top_k, E = c.n_experts, Fe = c.d_expert_ffn;
+            x.moe_logits = a.take(M * E * 4);
+            x.moe_ids = a.take(n * 4);
+            x.moe_wts = a.take(n * 4);
+            x.moe_rank = a.take(n * 4);
+            x.moe_counts = a.take(E * 4);
+            x.moe_offsets = a.take(E * 4);
+            x.moe_inv = a.take(n * 4);
+            x.moe_a = a.take((n + 128) * d * es);                // + one tile of slack rows for the last group's TMA box
+            x.moe_gu = a.take(n * 2 * Fe * es);
+            x.moe_act = a.take((n + 128) * Fe * es);
+            x.moe_out = a.take(n * d * 4);
+        }
         x.workspace_bytes = a.top;
     }
 }
 
 template <class T = void> T* at(void* base, const Loc& l) { return reinterpret_cast<T*>(static_cast<char*>(base) + l.off); }
 
-struct LayerPtrs { const float* attn_norm; const void* wqkv; const void* wo; const float* mlp_norm; const void* wgateup; const void* wdown; };
+struct LayerPtrs { const float* attn_norm; const void* wqkv; const void* wo; const float* mlp_norm; const void* wgateup; const void* wdown;
+                   const void* router; const void* exp_gateup; const void* exp_down; };
 
 LayerPtrs layer_ptrs(void* base, const LayerLoc& L)
 {
     return {at<const float>(base, L.attn_norm), at<const void>(base, L.wqkv), at<const void>(base, L.wo),
-            at<const float>(base, L.mlp_norm), at<const void>(base, L.wgateup), at<const void>(base, L.wdown)};
+            at<const float>(base, L.mlp_norm), at<const void>(base, L.wgateup), at<const void>(base, L.wdown),
+            L.router.bytes ? at<const void>(base, L.router) : nullptr, at<const void>(base, L.exp_gateup),
+            at<const void>(base, L.exp_down)};
 }
 
 #define TRY(expr) do { spec_status s__ = (expr); if (s__ != SPEC_OK) return s__; } while (0)
@@ -237,6 +256,22 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
     TIMED(c, CLS_ATTN, launch_attention(a, st));
     TIMED(c, CLS_GEMM, launch_gemm(M, d, Hq * dh, at(ws, c.attn_out), Hq * dh, W.wo, res, d, dt, SPEC_DTYPE_F32, 1, st));
     TRY(launch_rmsnorm(M, d, res, W.mlp_norm, g.rms_eps, at(ws, c.h), d, 0, dt, st));
+    if (W.router != nullptr) {
+        // mixture of experts: router -> top-k -> permute into expert order -> grouped gate/up, SwiGLU, grouped down -> combine
+        const int E = g.n_experts, tk = g.experts_top_k, Fe = g.d_expert_ffn, n = M * tk;
+        int32_t* status = at<int32_t>(c.buf.state, c.status);
+        TIMED(c, CLS_GEMM, launch_gemm(M, E, d, at(ws, c.h), d, W.router, at(ws, c.moe_logits), E, dt, SPEC_DTYPE_F32, 0, st));
+        TRY(launch_moe_route(M, E, tk, at<float>(ws, c.moe_logits), at<int32_t>(ws, c.moe_ids), at<float>(ws, c.moe_wts), st));
+        TRY(launch_moe_permute(M, E, tk, d, at<int32_t>(ws, c.moe_ids), at<int32_t>(ws, c.moe_rank), at<int32_t>(ws, c.moe_counts),
+                               at<int32_t>(ws, c.moe_offsets), at<int32_t>(ws, c.moe_inv), at(ws, c.h), at(ws, c.moe_a), st));
+        TIMED(c, CLS_GEMM, launch_gemm_grouped(n, M, E, 2 * Fe, d, at(ws, c.moe_a), W.exp_gateup, at(ws, c.moe_gu), dt,
+                                               at<int32_t>(ws, c.moe_counts), at<int32_t>(ws, c.moe_offsets), status, st));
+        TRY(launch_swiglu(n, Fe, at(ws, c.moe_gu), at(ws, c.moe_act), dt, st));
+        TIMED(c, CLS_GEMM, launch_gemm_grouped(n, M, E, d, Fe, at(ws, c.moe_act), W.exp_down, at(ws, c.moe_out), SPEC_DTYPE_F32,
+                                               at<int32_t>(ws, c.moe_counts), at<int32_t>(ws, c.moe_offsets), status, st));
+        TRY(launch_moe_combine(M, tk, d, at<float>(ws, c.moe_wts), at<int32_t>(ws, c.moe_inv), at<float>(ws, c.moe_out), res, st));
+        return SPEC_OK;
+    }
     TIMED(c, CLS_GEMM, launch_gemm(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.gu), 2 * d_ffn, dt, dt, 0, st));
     TRY(launch_swiglu(M, d_ffn, at(ws, c.gu), at(ws, c.act), dt, st));
     TIMED(c, CLS_GEMM, launch_gemm(M, d, d_ffn, at(ws, c.act), d_ffn, W.wdown, res, d, dt, SPEC_DTYPE_F32, 1, st));
@@ -368,6 +403,9 @@ extern "C" spec_status spec_tensor(spec_ctx* c, int id, int layer, void** dev_pt
     case SPEC_T_DRAFT_ROW_STATS: base = c->buf.workspace; l = c->draft_row_stats; break;
     case SPEC_T_TAPS: base = c->buf.workspace; l = c->taps; break;
     case SPEC_T_HIDDEN: base = c->buf.workspace; l = c->x; break;
+    case SPEC_T_MOE_LOGITS: base = c->buf.workspace; l = c->moe_logits; break;
+    case SPEC_T_MOE_IDS: base = c->buf.workspace; l = c->moe_ids; break;
+    case SPEC_T_MOE_WTS: base = c->buf.workspace; l = c->moe_wts; break;
     default: return SPEC_ERR_INVALID_ARG;
     }
     if (base == nullptr || l.bytes == 0) return SPEC_ERR_INVALID_ARG;

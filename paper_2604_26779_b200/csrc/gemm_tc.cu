@@ -107,7 +107,31 @@ struct GemmArgs {
     void* C; int ldc;
     int out_f32, accumulate;
     int32_t* status;
+    // grouped mode (E > 0): E independent problems that share K and N.  Group e multiplies rows
+    // [offsets[e], offsets[e] + counts[e]) of A by the weight rows [e*N, (e+1)*N) of W; counts/offsets live on the device.
+    int E, max_m_tiles;
+    const int32_t* counts; const int32_t* offsets;
 };
+
+// Decodes work item w into (m-tile, n-tile, group) and the tile's row window.  Returns false for an empty tile.
+struct TileCoord { int a_row, b_row, c_row, rows_valid, col; };
+__device__ __forceinline__ bool tile_coord(const GemmArgs& g, int w, int m_tiles, int n_tiles, TileCoord& t)
+{
+    const int mt = w % m_tiles, nt = (w / m_tiles) % n_tiles;
+    if (g.E > 0) {
+        const int e = w / (m_tiles * n_tiles);
+        const int cnt = g.counts[e];
+        if (mt * BM >= cnt) return false;
+        const int off = g.offsets[e];
+        t.a_row = off + mt * BM; t.c_row = t.a_row; t.rows_valid = cnt - mt * BM;
+        t.b_row = e * g.N + nt * BN;
+    } else {
+        t.a_row = mt * BM; t.c_row = t.a_row; t.rows_valid = g.M - mt * BM;
+        t.b_row = nt * BN;
+    }
+    t.col = nt * BN;
+    return true;
+}
 
 __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a,
                                                               const __grid_constant__ CUtensorMap map_b, const GemmArgs g)
@@ -119,8 +143,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     volatile int* abort_flag = &ctl->abort;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    const int m_tiles = (g.M + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
-    const int n_work = m_tiles * n_tiles, kb_count = (g.K + BK - 1) / BK;
+    const int m_tiles = g.E > 0 ? g.max_m_tiles : (g.M + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
+    const int n_work = m_tiles * n_tiles * (g.E > 0 ? g.E : 1), kb_count = (g.K + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
@@ -145,13 +169,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             uint32_t s = 0, ph = 0;
             bool ok = true;
             for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
-                const int mt = w % m_tiles, nt = w / m_tiles;
+                TileCoord tc;
+                if (!tile_coord(g, w, m_tiles, n_tiles, tc)) continue;
                 for (int kb = 0; kb < kb_count; ++kb) {
                     if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t bar = smem_u32(&ctl->full[s]);
                     mbar_expect_tx(bar, STAGE_BYTES);
-                    tma_load_2d(tiles + s * STAGE_BYTES, &map_a, kb * BK, mt * BM, bar);
-                    tma_load_2d(tiles + s * STAGE_BYTES + A_BYTES, &map_b, kb * BK, nt * BN, bar);
+                    tma_load_2d(tiles + s * STAGE_BYTES, &map_a, kb * BK, tc.a_row, bar);
+                    tma_load_2d(tiles + s * STAGE_BYTES + A_BYTES, &map_b, kb * BK, tc.b_row, bar);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
@@ -166,8 +191,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             uint32_t s = 0, ph = 0;
             bool ok = true;
             int it = 0;
-            for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++it) {
+            for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
+                TileCoord tc;
+                if (!tile_coord(g, w, m_tiles, n_tiles, tc)) continue;
                 const uint32_t acc = it & 1, acc_ph = (it >> 1) & 1;
+                ++it;
                 if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
@@ -194,21 +222,25 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         const int quarter = warp & 3;
         bool ok = true;
         int it = 0;
-        for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++it) {
-            const int mt = w % m_tiles, nt = w / m_tiles;
+        for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
+            TileCoord tc;
+            if (!tile_coord(g, w, m_tiles, n_tiles, tc)) continue;
             const uint32_t acc = it & 1, acc_ph = (it >> 1) & 1;
+            ++it;
             if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_ph, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const int row = mt * BM + quarter * 32 + lane;
+            const int row_in_tile = quarter * 32 + lane;
+            const int row = tc.c_row + row_in_tile;
+            const bool row_ok = row_in_tile < tc.rows_valid;
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
-                const int col = nt * BN + c0;
+                const int col = tc.col + c0;
                 if (col >= g.N) break;                              // warp-uniform
                 uint32_t v[32];
                 tc_ld32(t_row + c0, v);
                 tc_wait_ld();
-                if (row < g.M) {
+                if (row_ok) {
                     if (g.out_f32) {
                         float* cp = static_cast<float*>(g.C) + (size_t)row * g.ldc + col;
                         if (col + 32 <= g.N) {
@@ -323,9 +355,29 @@ spec_status launch_gemm_tc(int M, int N, int K, const void* A, int lda, const vo
     if (!make_map(&ma, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM)) return SPEC_ERR_CUDA;
     if (!make_map(&mb, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
     const int n_work = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-    GemmArgs g{M, N, K, C, ldc, out_dtype == SPEC_DTYPE_F32 ? 1 : 0, accumulate, status};
+    GemmArgs g{M, N, K, C, ldc, out_dtype == SPEC_DTYPE_F32 ? 1 : 0, accumulate, status, 0, 0, nullptr, nullptr};
     constexpr int smem = STAGES * STAGE_BYTES + 1024 + 256;
     gemm_tc_kernel<<<n_work < g_sms ? n_work : g_sms, kThreads, smem, st>>>(ma, mb, g);
+    return launch_status();
+}
+
+// Grouped form: A [rows_total][K] holds the groups' rows back to back (group e at offsets[e], counts[e] rows, both on
+// the device; no group has more than max_rows_per_group rows), W [E][N][K], C [rows_total][N].  N % 256 == 0.
+spec_status launch_gemm_grouped(int rows_total, int max_rows_per_group, int E, int N, int K, const void* A, const void* W,
+                                void* C, int out_dtype, const int32_t* counts, const int32_t* offsets, int32_t* status,
+                                cudaStream_t st)
+{
+    if (rows_total == 0 || E == 0) return SPEC_OK;
+    if (N % BN != 0 || K % 8 != 0) return SPEC_ERR_SHAPE;
+    if (!init_once()) return SPEC_ERR_CUDA;
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, A, (uint64_t)rows_total, (uint64_t)K, (uint64_t)K, BM)) return SPEC_ERR_CUDA;
+    if (!make_map(&mb, W, (uint64_t)E * N, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
+    const int max_m_tiles = (max_rows_per_group + BM - 1) / BM;
+    GemmArgs g{rows_total, N, K, C, N, out_dtype == SPEC_DTYPE_F32 ? 1 : 0, 0, status, E, max_m_tiles, counts, offsets};
+    constexpr int smem = STAGES * STAGE_BYTES + 1024 + 256;
+    const long long n_work = (long long)E * max_m_tiles * (N / BN);
+    gemm_tc_kernel<<<n_work < g_sms ? (int)n_work : g_sms, kThreads, smem, st>>>(ma, mb, g);
     return launch_status();
 }
 

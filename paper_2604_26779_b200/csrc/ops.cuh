@@ -67,6 +67,17 @@ spec_status launch_gemm_simt(int M, int N, int K, const void* A, int lda, const 
 spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int dtype_in,
                         int out_dtype, int accumulate, cudaStream_t st);
 
+spec_status launch_gemm_grouped(int rows_total, int max_rows_per_group, int E, int N, int K, const void* A, const void* W,
+                                void* C, int out_dtype, const int32_t* counts, const int32_t* offsets, int32_t* status,
+                                cudaStream_t st);
+
+// moe.cu: router top-k, permutation into expert order, weighted combination
+spec_status launch_moe_route(int M, int E, int top_k, const float* logits, int32_t* ids, float* wts, cudaStream_t st);
+spec_status launch_moe_permute(int M, int E, int top_k, int d, const int32_t* ids, int32_t* rank, int32_t* counts,
+                               int32_t* offsets, int32_t* inv, const void* h, void* a_perm, cudaStream_t st);
+spec_status launch_moe_combine(int M, int top_k, int d, const float* wts, const int32_t* inv, const float* out_perm,
+                               float* x, cudaStream_t st);
+
 // attention.cu
 struct AttnArgs {
     int B, R, Hq, Hkv, dh, block_tokens, max_blocks;

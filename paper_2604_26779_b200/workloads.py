@@ -19,7 +19,8 @@ def _fill_normal(t: torch.Tensor, std: float, gen: torch.Generator):
 
 
 def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, len_hi=16384, lens=None, draft="eagle3",
-                         kv_pools=None, steps_budget=64, seed=None, device="cuda:0", vocab=None, mem_fraction=0.92):
+                         kv_pools=None, steps_budget=64, seed=None, device="cuda:0", vocab=None, mem_fraction=0.92,
+                         cfg_over=None):
     """Returns (SpecStep, info dict).  The cache of layer l lives in pool l mod G; G < n_layers (chosen so that the
     arenas fit the device) is the aliased, timing-only mode: bytes moved per layer are unchanged because one pool
     (gigabytes) is far larger than L2."""
@@ -28,6 +29,8 @@ def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, l
         cfg = dict(cfg, n_layers=n_layers, tap_layers=inputs.default_tap_layers(n_layers) if draft == "eagle3" else (n_layers,))
     if vocab is not None:
         cfg = dict(cfg, vocab=vocab)
+    if cfg_over:
+        cfg = dict(cfg, **cfg_over)
     seed = inputs.sub_seed(3, 0) if seed is None else seed
     if lens is None:
         lens = inputs.make_seq_lens_uniform(B, len_lo, len_hi, seed + 1)
@@ -69,8 +72,14 @@ def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, l
     for l in range(L):
         eng.tensor("ATTN_NORM", l, f32).fill_(1.0)
         eng.tensor("MLP_NORM", l, f32).fill_(1.0)
-        for nm in ("WQKV", "WO", "WGATEUP", "WDOWN"):
-            _fill_normal(eng.tensor(nm, l, bf), 0.02, gen)
+        if cfg.get("n_experts", 0) > 0:
+            for nm in ("WQKV", "WO", "EXPERTS_GATEUP", "EXPERTS_DOWN"):
+                _fill_normal(eng.tensor(nm, l, bf), 0.02, gen)
+            # router rows ~ N(0, 1/d): unit-RMS inputs give router logits ~ N(0, 1)
+            _fill_normal(eng.tensor("ROUTER", l, bf), float(cfg["d_model"]) ** -0.5, gen)
+        else:
+            for nm in ("WQKV", "WO", "WGATEUP", "WDOWN"):
+                _fill_normal(eng.tensor(nm, l, bf), 0.02, gen)
     if draft != "none":
         for nm in ("D_NORM_E", "D_NORM_G", "D_MLP_NORM") + (("D_NORM_F",) if draft == "eagle3" else ("D_ATTN_NORM",)):
             eng.tensor(nm, 0, f32).fill_(1.0)
