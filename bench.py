@@ -131,6 +131,10 @@ def main():
     ap.add_argument("--cpu-layers", type=int, default=4, help="layers the CPU-baseline sample times (scaled to all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--workload", default="c3", choices=["c3", "c4", "c5"],
+                    help="c3 = the headline 8B + EAGLE-3 workload; c4 = 8B + MTP head, B=512, lognormal lengths; "
+                         "c5 = one 235B-A22B-shaped MoE layer + LM head, B=256, cache length 8192 (measurement of the "
+                         "other configurations; the reported metric line is c3)")
     args = ap.parse_args()
 
     import torch
@@ -151,26 +155,54 @@ def main():
     from paper_2604_26779_b200 import binding, replicas, workloads
     k, B = args.k, args.batch
     steps_budget = args.steps * 2 + args.warmup * 2 + 24
-    eng, info = workloads.build_dense_workload("c3", B=B, k=k, n_layers=args.layers, kv_pools=args.kv_pools,
-                                               steps_budget=steps_budget, device=f"cuda:{local}",
-                                               seed=replicas.replica_seed(rank))
+    ext_drafts = None
+    if args.workload == "c3":
+        eng, info = workloads.build_dense_workload("c3", B=B, k=k, n_layers=args.layers, kv_pools=args.kv_pools,
+                                                   steps_budget=steps_budget, device=f"cuda:{local}",
+                                                   seed=replicas.replica_seed(rank))
+        wl_name = ("c3: 8B dense verify (32 layers, d=4096, 32q/8kv, dh=128, FFN 14336, V=128256, bf16), "
+                   "EAGLE-3-style 1-layer draft head, cache lengths ~U[1024,16384], 16-token pages")
+    elif args.workload == "c4":
+        from paper_2604_26779_b200 import inputs
+        B = 512 if args.batch == 256 else args.batch
+        lens = inputs.make_seq_lens_lognormal(B, 4096, float(np.log(2.0)), 16, 32768, replicas.replica_seed(rank, 4))
+        eng, info = workloads.build_dense_workload("c4", lens=lens, k=k, n_layers=args.layers, kv_pools=args.kv_pools, draft="mtp",
+                                                   steps_budget=steps_budget, device=f"cuda:{local}",
+                                                   seed=replicas.replica_seed(rank, 4))
+        wl_name = "c4: 8B dense verify + MTP head (one decoder layer, shared LM head), cache lengths lognormal(median 4096, sigma ln 2, clip [16, 32768])"
+    else:
+        lens = np.full(B, 8192, np.int32)
+        eng, info = workloads.build_dense_workload("c5", lens=lens, k=k, draft="none", kv_pools=args.kv_pools,
+                                                   steps_budget=steps_budget, device=f"cuda:{local}",
+                                                   seed=replicas.replica_seed(rank, 5))
+        g = torch.Generator(device=f"cuda:{local}"); g.manual_seed(5)
+        ext_drafts = (torch.randint(0, info["cfg"]["vocab"], (B, k), dtype=torch.int32, device="cuda", generator=g),
+                      torch.randn((B, k, info["cfg"]["vocab"]), dtype=torch.float32, device="cuda", generator=g))
+        wl_name = "c5: one MoE decoder layer of 235B-A22B shape (d=4096, 64q/4kv, 128 experts top-8, expert FFN 1536) + LM head V=151936, cache length 8192, external drafts"
     cfg = info["cfg"]
+    if ext_drafts is not None:
+        def step_fn(with_draft=True):
+            eng.verify(k, ext_drafts[0]); eng.reject_sample(k, ext_drafts[1]); eng.kv_commit()
+        workloads_spec_step = lambda e, kk, with_draft=True: step_fn(with_draft)
+    else:
+        workloads_spec_step = workloads.spec_step
     workloads.bootstrap(eng)
-    config = {"workload": "c3: 8B dense verify (32 layers, d=4096, 32q/8kv, dh=128, FFN 14336, V=128256, bf16), "
-                          "EAGLE-3-style 1-layer draft head, cache lengths ~U[1024,16384], 16-token pages",
+    config = {"workload": wl_name,
               "batch": B, "k": k, "layers": cfg["n_layers"], "kv_layer_pools": info["kv_pools"], "aliased_kv": bool(info["aliased"]),
               "l2": "inputs_exceed_l2 (15 GB weights + >=9 GB cache per layer per step; no flush needed)",
               "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
               "acceptance": "measured with the random-init draft head (untrained: low by construction)"}
+    if args.workload != "c3":
+        args.no_cpu_baseline = True
 
     if args.impl == "reference":
         # the CPU oracle on a bounded sample, timed step after step on this machine's host cores
         for _ in range(args.warmup):
-            workloads.spec_step(eng, k)
+            workloads_spec_step(eng, k)
         vals = []
         t_all = time.perf_counter()
         for i in range(args.steps):
-            workloads.spec_step(eng, k)                                     # advances the device state the sample is cut from
+            workloads_spec_step(eng, k)                                     # advances the device state the sample is cut from
             rep = eng.status()
             vals.append(cpu_oracle_sample(eng, info, k, 1, int(rep.steps) - 1))
         wall = time.perf_counter() - t_all
@@ -192,7 +224,7 @@ def main():
             torch.cuda.synchronize()
 
     for _ in range(max(args.warmup, 3)):
-        workloads.spec_step(eng, k)
+        workloads_spec_step(eng, k)
     rep0 = eng.status()
     assert rep0.device_status == 0, f"device status {rep0.device_status} after warm-up"
     tokens_before = float(eng.seq_len().sum().item())
@@ -207,7 +239,7 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
-        workloads.spec_step(eng, k)
+        workloads_spec_step(eng, k)
     e1.record(stream)
     sync_all()
     clocks = sampler.stop()
@@ -259,10 +291,10 @@ def main():
             return a.elapsed_time(b) / n
         eng.set_timing(15)
         eng.get_timing()
-        ms_full = timed(lambda: workloads.spec_step(eng, k), 2)
+        ms_full = timed(lambda: workloads_spec_step(eng, k), 2)
         tm = eng.get_timing()
         eng.set_timing(0)
-        ms_vs = timed(lambda: workloads.spec_step(eng, k, with_draft=False), 3)
+        ms_vs = timed(lambda: workloads_spec_step(eng, k, with_draft=False), 3)
         ms_dec = timed(lambda: workloads.bootstrap(eng), 3)
         line["extras"] = {"ms_verify_sample_commit": ms_vs, "ms_plain_decode_step": ms_dec,
                           "plain_decode_tokens_per_s": B / (ms_dec / 1000.0),
@@ -287,7 +319,7 @@ def main():
     workloads.bootstrap(eng)
     total_e2e = 0
     for _ in range(e2e_steps):
-        workloads.spec_step(eng, k)
+        workloads_spec_step(eng, k)
         pinned_out.copy_(eng.out_tokens(k), non_blocking=True)
         pinned_n.copy_(eng.n_emitted(), non_blocking=True)
         torch.cuda.synchronize()
@@ -301,7 +333,7 @@ def main():
                            "tokens and a synchronize; wall clock, max over ranks"}
 
     if rank == 0 and not args.no_cpu_baseline:
-        workloads.spec_step(eng, k)
+        workloads_spec_step(eng, k)
         rep = eng.status()
         cb = cpu_oracle_sample(eng, info, k, args.cpu_layers, int(rep.steps) - 1)
         line["cpu_baseline"] = {kk: cb[kk] for kk in ("value", "unit", "cores", "kind", "sample")}

@@ -89,10 +89,11 @@ enum {
     /* target weights (arena `weights`); per-layer ones take the layer index */
     SPEC_T_EMBED = 0, SPEC_T_LM_HEAD, SPEC_T_FINAL_NORM,
     SPEC_T_ATTN_NORM, SPEC_T_WQKV, SPEC_T_WO, SPEC_T_MLP_NORM,
-    SPEC_T_WGATEUP,             /* [2*d_ffn][d]: gate rows, then up rows                              */
+    SPEC_T_WGATEUP,             /* [2*d_ffn][d] in 256-row groups: gate rows 128g..128g+127, then up   */
+                                /* rows 128g..128g+127 (d_ffn % 128 == 0)                              */
     SPEC_T_WDOWN,
     SPEC_T_ROUTER,              /* [n_experts][d]                                                      */
-    SPEC_T_EXPERTS_GATEUP,      /* [n_experts][2*d_expert_ffn][d]                                      */
+    SPEC_T_EXPERTS_GATEUP,      /* [n_experts][2*d_expert_ffn][d], each expert grouped like WGATEUP    */
     SPEC_T_EXPERTS_DOWN,        /* [n_experts][d][d_expert_ffn]                                        */
     /* draft head weights (arena `draft_weights`) */
     SPEC_T_D_WFC = 32,          /* EAGLE3: [d][n_taps*d]                                               */

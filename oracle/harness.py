@@ -18,14 +18,23 @@ def _np(t):
     return t.float().cpu().numpy()
 
 
-class _LazyRows:
-    """Per-expert weight matrices [E][rows][cols] fetched from the device one expert at a time."""
+def _split_gate_up(gu):
+    """The device stores gate and up stacked in 256-row groups (128 gate rows, then the matching 128 up rows)."""
+    F2, d = gu.shape
+    t = gu.reshape(F2 // 256, 256, d)
+    return t[:, :128].reshape(F2 // 2, d), t[:, 128:].reshape(F2 // 2, d)
 
-    def __init__(self, dev_tensor, r0, r1):
-        self.t, self.r0, self.r1 = dev_tensor, r0, r1
+
+class _LazyRows:
+    """Per-expert weight matrices [E][rows][cols] fetched from the device one expert at a time; `part` picks the gate
+    (0) or up (1) half of a stacked gate/up matrix, None the whole matrix."""
+
+    def __init__(self, dev_tensor, part=None):
+        self.t, self.part = dev_tensor, part
 
     def __getitem__(self, e):
-        return _np(self.t[int(e), self.r0 : self.r1])
+        m = _np(self.t[int(e)])
+        return m if self.part is None else _split_gate_up(m)[self.part]
 
 
 class LazyLayers:
@@ -56,11 +65,11 @@ class LazyLayers:
             E, Fe = cfg["n_experts"], cfg["d_expert_ffn"]
             gu = eng.tensor("EXPERTS_GATEUP", l, td, (E, 2 * Fe, d))
             dn = eng.tensor("EXPERTS_DOWN", l, td, (E, d, Fe))
-            lw.update(router=_np(eng.tensor("ROUTER", l, td, (E, d))), experts_gate=_LazyRows(gu, 0, Fe),
-                      experts_up=_LazyRows(gu, Fe, 2 * Fe), experts_down=_LazyRows(dn, 0, d))
+            lw.update(router=_np(eng.tensor("ROUTER", l, td, (E, d))), experts_gate=_LazyRows(gu, 0),
+                      experts_up=_LazyRows(gu, 1), experts_down=_LazyRows(dn))
         else:
-            gu = _np(eng.tensor("WGATEUP", l, td, (2 * F, d)))
-            lw.update(wgate=gu[:F], wup=gu[F:], wdown=_np(eng.tensor("WDOWN", l, td, (d, F))))
+            gate, up = _split_gate_up(_np(eng.tensor("WGATEUP", l, td, (2 * F, d))))
+            lw.update(wgate=gate, wup=up, wdown=_np(eng.tensor("WDOWN", l, td, (d, F))))
         return lw
 
 

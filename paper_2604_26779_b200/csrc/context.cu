@@ -28,12 +28,12 @@ struct spec_ctx {
     size_t kv_pool_bytes = 0, kv_bytes = 0, draft_kv_bytes = 0;
     // state
     Loc seq_len, last_token, block_table, free_stack, free_top, draft_tokens, out_tokens, n_emitted, status, step,
-        counters, pending_base;
+        counters, pending_base, owned;
     size_t state_bytes = 0;
     // workspace
     Loc tokens_in, pos, x, h, qkv, attn_out, gu, act, logits, draft_logits, row_stats, draft_row_stats, taps,
         attn_scratch, dg, dx, d_hidden, d_tok, d_pos,
-        moe_logits, moe_ids, moe_wts, moe_rank, moe_counts, moe_offsets, moe_inv, moe_a, moe_gu, moe_act, moe_out;
+        moe_logits, moe_ids, moe_wts, moe_rank, moe_counts, moe_offsets, moe_inv, moe_a, moe_gu, moe_act, moe_out, rope;
     size_t workspace_bytes = 0;
     // host-side run state
     int B = 0;
@@ -74,7 +74,7 @@ spec_status check_config(const spec_config* c)
     if (c->n_layers <= 0 || c->d_model <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->head_dim <= 0 || c->vocab <= 0)
         return SPEC_ERR_SHAPE;
     if (c->n_q_heads % c->n_kv_heads != 0 || c->d_model % 8 != 0 || c->head_dim % 8 != 0 || c->vocab % 4 != 0) return SPEC_ERR_SHAPE;
-    if (c->n_experts == 0 && (c->d_ffn <= 0 || c->d_ffn % 8 != 0)) return SPEC_ERR_SHAPE;
+    if (c->n_experts == 0 && (c->d_ffn <= 0 || c->d_ffn % 128 != 0)) return SPEC_ERR_SHAPE;
     if (c->n_experts > 0 && (c->experts_top_k <= 0 || c->experts_top_k > c->n_experts || c->d_expert_ffn <= 0)) return SPEC_ERR_SHAPE;
     if (c->n_experts > 0 && (c->dtype != SPEC_DTYPE_BF16 || c->n_experts > 256 || c->experts_top_k > 32 ||
                              c->d_expert_ffn % 128 != 0 || c->d_model % 256 != 0)) return SPEC_ERR_UNSUPPORTED;
@@ -85,8 +85,8 @@ spec_status check_config(const spec_config* c)
     if (c->kv_layer_pools <= 0 || c->kv_layer_pools > c->n_layers) return SPEC_ERR_SHAPE;
     if (c->n_taps < 0 || c->n_taps > 3) return SPEC_ERR_SHAPE;
     for (int i = 0; i < c->n_taps; ++i) if (c->tap_layers[i] < 0 || c->tap_layers[i] > c->n_layers) return SPEC_ERR_SHAPE;
-    if (c->draft_kind == SPEC_DRAFT_EAGLE3 && (c->n_taps < 1 || c->draft_d_ffn <= 0)) return SPEC_ERR_SHAPE;
-    if (c->draft_kind == SPEC_DRAFT_MTP && (c->draft_d_ffn <= 0)) return SPEC_ERR_SHAPE;
+    if (c->draft_kind == SPEC_DRAFT_EAGLE3 && (c->n_taps < 1 || c->draft_d_ffn <= 0 || c->draft_d_ffn % 128 != 0)) return SPEC_ERR_SHAPE;
+    if (c->draft_kind == SPEC_DRAFT_MTP && (c->draft_d_ffn <= 0 || c->draft_d_ffn % 128 != 0)) return SPEC_ERR_SHAPE;
     if (!(c->temperature > 0.f) || !(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return SPEC_ERR_UNSUPPORTED;
     if (c->vocab > sampler_max_vocab()) return SPEC_ERR_SHAPE;
     return SPEC_OK;
@@ -161,6 +161,7 @@ void build_layout(spec_ctx& x)
         x.step = a.take(4);
         x.counters = a.take(3 * 8);
         x.pending_base = a.take(Bm * 4);
+        x.owned = a.take(Bm * 4);
         x.state_bytes = a.top;
     }
     {
@@ -187,6 +188,7 @@ void build_layout(spec_ctx& x)
         x.d_hidden = a.take(Bm * d * 4);
         x.d_tok = a.take(M * 4);
         x.d_pos = a.take(M * 4);
+        x.rope = a.take(M * (size_t)(c.head_dim / 2) * 8);
         if (c.n_experts > 0) {
             const size_t n = M * c.experts_top_k, E = c.n_experts, Fe = c.d_expert_ffn;
             x.moe_logits = a.take(M * E * 4);
@@ -243,13 +245,23 @@ enum { CLS_ATTN = 0, CLS_GEMM = 1, CLS_SAMPLE = 2, CLS_OTHER = 3 };
 spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* res, const void* qkv_in, int qkv_k, int B, int R,
                            const int32_t* pos, void* k_pool, void* v_pool, int launch_index, cudaStream_t st)
 {
+    // `pos` rows have their (cos, sin) table in c.rope (filled by the caller for this forward)
     const spec_config& g = c.cfg;
     const int M = B * R, d = g.d_model, dh = g.head_dim, Hq = g.n_q_heads, Hkv = g.n_kv_heads;
     const int qkv_n = (Hq + 2 * Hkv) * dh, dt = g.dtype;
     void* ws = c.buf.workspace;
-    TIMED(c, CLS_GEMM, launch_gemm(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt, 0, st));
-    TRY(launch_rope_append(B, R, Hq, Hkv, dh, g.rope_theta, at(ws, c.qkv), pos, k_pool, v_pool,
-                           at<int32_t>(c.buf.state, c.block_table), g.max_blocks_per_seq, g.kv_block_tokens, dt, st));
+    int32_t* status_word = at<int32_t>(c.buf.state, c.status);
+    const bool tc = gemm_tc_supported(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt);
+    if (tc && (dh == 64 || dh == 128)) {
+        // projection, rotary embedding and the append into the paged cache in one kernel
+        QkvEpilogue e{Hq, Hkv, dh, R, g.max_blocks_per_seq, g.kv_block_tokens, pos, at<int32_t>(c.buf.state, c.block_table),
+                      at<float>(ws, c.rope), k_pool, v_pool};
+        TIMED(c, CLS_GEMM, launch_gemm_qkv_tc(M, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), e, status_word, st));
+    } else {
+        TIMED(c, CLS_GEMM, launch_gemm(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt, 0, st));
+        TRY(launch_rope_append(B, R, Hq, Hkv, dh, g.rope_theta, at(ws, c.qkv), pos, k_pool, v_pool,
+                               at<int32_t>(c.buf.state, c.block_table), g.max_blocks_per_seq, g.kv_block_tokens, dt, st));
+    }
     AttnArgs a{B, R, Hq, Hkv, dh, g.kv_block_tokens, g.max_blocks_per_seq, at(ws, c.qkv), qkv_n, k_pool, v_pool,
                at<int32_t>(c.buf.state, c.block_table), pos, at(ws, c.attn_out), Hq * dh, dt, at(ws, c.attn_scratch),
                c.attn_scratch.bytes, g.max_blocks_per_seq * g.kv_block_tokens, launch_index};
@@ -264,16 +276,19 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
         TRY(launch_moe_route(M, E, tk, at<float>(ws, c.moe_logits), at<int32_t>(ws, c.moe_ids), at<float>(ws, c.moe_wts), st));
         TRY(launch_moe_permute(M, E, tk, d, at<int32_t>(ws, c.moe_ids), at<int32_t>(ws, c.moe_rank), at<int32_t>(ws, c.moe_counts),
                                at<int32_t>(ws, c.moe_offsets), at<int32_t>(ws, c.moe_inv), at(ws, c.h), at(ws, c.moe_a), st));
-        TIMED(c, CLS_GEMM, launch_gemm_grouped(n, M, E, 2 * Fe, d, at(ws, c.moe_a), W.exp_gateup, at(ws, c.moe_gu), dt,
+        TIMED(c, CLS_GEMM, launch_gemm_grouped(n, M, E, 2 * Fe, d, at(ws, c.moe_a), W.exp_gateup, at(ws, c.moe_act), dt, 1,
                                                at<int32_t>(ws, c.moe_counts), at<int32_t>(ws, c.moe_offsets), status, st));
-        TRY(launch_swiglu(n, Fe, at(ws, c.moe_gu), at(ws, c.moe_act), dt, st));
-        TIMED(c, CLS_GEMM, launch_gemm_grouped(n, M, E, d, Fe, at(ws, c.moe_act), W.exp_down, at(ws, c.moe_out), SPEC_DTYPE_F32,
+        TIMED(c, CLS_GEMM, launch_gemm_grouped(n, M, E, d, Fe, at(ws, c.moe_act), W.exp_down, at(ws, c.moe_out), SPEC_DTYPE_F32, 0,
                                                at<int32_t>(ws, c.moe_counts), at<int32_t>(ws, c.moe_offsets), status, st));
         TRY(launch_moe_combine(M, tk, d, at<float>(ws, c.moe_wts), at<int32_t>(ws, c.moe_inv), at<float>(ws, c.moe_out), res, st));
         return SPEC_OK;
     }
-    TIMED(c, CLS_GEMM, launch_gemm(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.gu), 2 * d_ffn, dt, dt, 0, st));
-    TRY(launch_swiglu(M, d_ffn, at(ws, c.gu), at(ws, c.act), dt, st));
+    if (gemm_tc_supported(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.act), d_ffn, dt, dt)) {
+        TIMED(c, CLS_GEMM, launch_gemm_swiglu_tc(M, d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.act), status_word, st));
+    } else {
+        TIMED(c, CLS_GEMM, launch_gemm(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.gu), 2 * d_ffn, dt, dt, 0, st));
+        TRY(launch_swiglu(M, d_ffn, at(ws, c.gu), at(ws, c.act), dt, st));
+    }
     TIMED(c, CLS_GEMM, launch_gemm(M, d, d_ffn, at(ws, c.act), d_ffn, W.wdown, res, d, dt, SPEC_DTYPE_F32, 1, st));
     return SPEC_OK;
 }
@@ -421,7 +436,7 @@ extern "C" spec_status spec_seq_init(spec_ctx* c, int B, const int32_t* seq_len_
     const spec_config& g = c->cfg;
     if (B > g.max_batch) return SPEC_ERR_SHAPE;
     const int bt = g.kv_block_tokens, mb = g.max_blocks_per_seq, nb = g.kv_num_blocks;
-    std::vector<int32_t> table((size_t)g.max_batch * mb, -1), stack(free_stack_host, free_stack_host + nb);
+    std::vector<int32_t> table((size_t)g.max_batch * mb, -1), stack(free_stack_host, free_stack_host + nb), owned(g.max_batch, 0);
     std::vector<char> seen(nb, 0);
     for (int i = 0; i < nb; ++i) {
         if (stack[i] < 0 || stack[i] >= nb || seen[stack[i]]) return SPEC_ERR_INVALID_ARG;
@@ -434,6 +449,7 @@ extern "C" spec_status spec_seq_init(spec_ctx* c, int B, const int32_t* seq_len_
         if (need > mb || (seq_len_host[b] + g.k_max + 1 + bt - 1) / bt > mb) return SPEC_ERR_SHAPE;
         if (need > top) return SPEC_ERR_SHAPE;
         for (int j = 0; j < need; ++j) table[(size_t)b * mb + j] = stack[--top];
+        owned[b] = need;
     }
     cudaStream_t st = (cudaStream_t)stream;
     char* sb = static_cast<char*>(c->buf.state);
@@ -443,6 +459,7 @@ extern "C" spec_status spec_seq_init(spec_ctx* c, int B, const int32_t* seq_len_
     SPEC_CUDA_OK(cudaMemcpyAsync(sb + c->block_table.off, table.data(), table.size() * 4, cudaMemcpyHostToDevice, st));
     SPEC_CUDA_OK(cudaMemcpyAsync(sb + c->free_stack.off, stack.data(), (size_t)nb * 4, cudaMemcpyHostToDevice, st));
     SPEC_CUDA_OK(cudaMemcpyAsync(sb + c->free_top.off, &top, 4, cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_OK(cudaMemcpyAsync(sb + c->owned.off, owned.data(), owned.size() * 4, cudaMemcpyHostToDevice, st));
     SPEC_CUDA_OK(cudaStreamSynchronize(st));          // the host staging vectors go out of scope here
     c->B = B;
     c->k_last = -1;
@@ -464,13 +481,14 @@ extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_toke
     char* sb = static_cast<char*>(c->buf.state);
     int32_t* status = at<int32_t>(sb, c->status);
     int32_t* seq_len = at<int32_t>(sb, c->seq_len);
-    TRY(launch_kv_reserve(B, k, g.kv_block_tokens, g.max_blocks_per_seq, seq_len, at<int32_t>(sb, c->block_table),
+    TRY(launch_kv_reserve(B, k, g.kv_block_tokens, g.max_blocks_per_seq, seq_len, at<int32_t>(sb, c->block_table), at<int32_t>(sb, c->owned),
                           at<int32_t>(sb, c->free_stack), at<int32_t>(sb, c->free_top), status, st));
     StepRows rows{at<int32_t>(ws, c->tokens_in), at<int32_t>(ws, c->pos)};
     const int32_t* dtok = draft_tokens ? draft_tokens : at<int32_t>(sb, c->draft_tokens);
     const int dstride = draft_tokens ? k : (g.k_max > 0 ? g.k_max : 1);
     TRY(launch_verify_rows(B, R, seq_len, at<int32_t>(sb, c->last_token), dtok, dstride, g.vocab, rows, status, st));
     float* x = at<float>(ws, c->x);
+    TRY(launch_rope_table(M, g.head_dim, g.rope_theta, rows.pos, at<float>(ws, c->rope), st));
     TRY(launch_embed(M, d, at(c->buf.weights, c->embed), dt, rows.token, x, st));
     const int tapw = g.n_taps * d;
     if (has_tap(g, 0)) TRY(launch_copy_rows_f32_to(M, d, x, at(ws, c->taps), tapw, tap_slot(g, 0) * d, dt, st));
@@ -530,6 +548,7 @@ extern "C" spec_status spec_kv_commit(spec_ctx* c, const int32_t* force_n, const
     a.seq_len = at<int32_t>(sb, c->seq_len);
     a.last_token = at<int32_t>(sb, c->last_token);
     a.block_table = at<int32_t>(sb, c->block_table);
+    a.owned = at<int32_t>(sb, c->owned);
     a.free_stack = at<int32_t>(sb, c->free_stack);
     a.free_top = at<int32_t>(sb, c->free_top);
     a.pending_base = at<int32_t>(sb, c->pending_base);
@@ -557,7 +576,7 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
     int32_t* status = at<int32_t>(sb, c->status);
     int32_t* seq_len = at<int32_t>(sb, c->seq_len);
     const bool eagle = g.draft_kind == SPEC_DRAFT_EAGLE3;
-    TRY(launch_kv_reserve(B, k, g.kv_block_tokens, g.max_blocks_per_seq, seq_len, at<int32_t>(sb, c->block_table),
+    TRY(launch_kv_reserve(B, k, g.kv_block_tokens, g.max_blocks_per_seq, seq_len, at<int32_t>(sb, c->block_table), at<int32_t>(sb, c->owned),
                           at<int32_t>(sb, c->free_stack), at<int32_t>(sb, c->free_top), status, st));
     const LayerPtrs W = layer_ptrs(dw, c->d_layer);
     char* kp = static_cast<char*>(c->buf.draft_kv);
@@ -580,6 +599,7 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
                                                                         at<int32_t>(sb, c->out_tokens), tok, pos);
         else        draft_rows_kernel<<<(B + 255) / 256, 256, 0, st>>>(B, j, seq_len, dtoks, kstride, tok, pos);
         TRY(launch_status());
+        TRY(launch_rope_table(M, g.head_dim, g.rope_theta, pos, at<float>(ws, c->rope), st));
         TRY(launch_embed(M, d, at(c->buf.weights, c->embed), dt, tok, dx, st));
         if (eagle) {
             // a = concat(norm_e(e), norm_g(g)); g = W_fc taps (true slots) or the head's previous output

@@ -24,6 +24,7 @@ constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;
+constexpr int kSmemBytes = STAGES * STAGE_BYTES + 1024 + 256;
 constexpr long long kWaitLimit = 300000000LL;            // clock cycles (~0.15 s): far beyond any healthy wait
 
 struct Ctl {
@@ -102,6 +103,8 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr)
 // Instruction descriptor: D fp32, A and B bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
+struct TileCoord { int a_row, b_row, c_row, rows_valid, col; };
+
 struct GemmArgs {
     int M, N, K;
     void* C; int ldc;
@@ -111,10 +114,153 @@ struct GemmArgs {
     // [offsets[e], offsets[e] + counts[e]) of A by the weight rows [e*N, (e+1)*N) of W; counts/offsets live on the device.
     int E, max_m_tiles;
     const int32_t* counts; const int32_t* offsets;
+    // EPI_QKV: rotary embedding on q and k heads, k and v written straight into the paged cache
+    int Hq, Hkv, dh, R, max_blocks, block_tokens;
+    const int32_t* pos; const int32_t* block_table; const float2* rope;   // rope [M][dh/2] (cos, sin) of each row's position
+    __nv_bfloat16* k_pool; __nv_bfloat16* v_pool;
 };
 
+enum { EPI_PLAIN = 0, EPI_SWIGLU = 1, EPI_QKV = 2 };
+
+__device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float (&f)[32])
+{
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        uint4 o;
+        __nv_bfloat162 t0 = __floats2bfloat162_rn(f[8 * j], f[8 * j + 1]), t1 = __floats2bfloat162_rn(f[8 * j + 2], f[8 * j + 3]);
+        __nv_bfloat162 t2 = __floats2bfloat162_rn(f[8 * j + 4], f[8 * j + 5]), t3 = __floats2bfloat162_rn(f[8 * j + 6], f[8 * j + 7]);
+        o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
+        o.z = *reinterpret_cast<uint32_t*>(&t2); o.w = *reinterpret_cast<uint32_t*>(&t3);
+        *reinterpret_cast<uint4*>(dst + 8 * j) = o;
+    }
+}
+
+// Plain epilogue: C (+)= accumulator, fp32 or bf16, ragged N handled element-wise.
+__device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok)
+{
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += 32) {
+        const int col = tc.col + c0;
+        if (col >= g.N) break;                              // warp-uniform
+        uint32_t v[32];
+        tc_ld32(t_row + c0, v);
+        tc_wait_ld();
+        if (!row_ok) continue;
+        if (g.out_f32) {
+            float* cp = static_cast<float*>(g.C) + (size_t)row * g.ldc + col;
+            if (col + 32 <= g.N) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    float4 o = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                           __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                    if (g.accumulate) {
+                        const float4 p = *reinterpret_cast<const float4*>(cp + 4 * j);
+                        o.x += p.x; o.y += p.y; o.z += p.z; o.w += p.w;
+                    }
+                    *reinterpret_cast<float4*>(cp + 4 * j) = o;
+                }
+            } else {
+                for (int j = 0; j < 32 && col + j < g.N; ++j)
+                    cp[j] = __uint_as_float(v[j]) + (g.accumulate ? cp[j] : 0.f);
+            }
+        } else {
+            __nv_bfloat16* cp = static_cast<__nv_bfloat16*>(g.C) + (size_t)row * g.ldc + col;
+            if (col + 32 <= g.N) {
+                float f[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(v[e]);
+                if (g.accumulate) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint4 p = *reinterpret_cast<const uint4*>(cp + 8 * j);
+                        const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&p);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) { f[8 * j + 2 * e] += __low2float(pp[e]); f[8 * j + 2 * e + 1] += __high2float(pp[e]); }
+                    }
+                }
+                store_bf16x32(cp, f);
+            } else {
+                for (int j = 0; j < 32 && col + j < g.N; ++j)
+                    cp[j] = __float2bfloat16_rn(__uint_as_float(v[j]) + (g.accumulate ? __bfloat162float(cp[j]) : 0.f));
+            }
+        }
+    }
+}
+
+// SwiGLU epilogue: the tile's first 128 columns are gate rows, the last 128 the matching up rows (the stacked weight is
+// stored in such 256-row groups); writes act = silu(gate) * up, bf16, [rows][N/2].
+__device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok)
+{
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(g.C) + (size_t)row * g.ldc + tc.col / 2;
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN / 2; c0 += 32) {
+        uint32_t gv[32], uv[32];
+        tc_ld32(t_row + c0, gv);
+        tc_ld32(t_row + BN / 2 + c0, uv);
+        tc_wait_ld();
+        if (!row_ok) continue;
+        float f[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const float a = __uint_as_float(gv[e]);
+            f[e] = a / (1.f + __expf(-a)) * __uint_as_float(uv[e]);
+        }
+        store_bf16x32(out + c0, f);
+    }
+}
+
+// QKV epilogue: heads of width dh; q and k heads get the rotary embedding (pairs (j, j + dh/2)); q goes to C (bf16,
+// [rows][N]), k and v go to the paged cache slot of the row's position.  Rows with a negative position write nothing.
+__device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok)
+{
+    const int half = g.dh / 2;
+    int p = -1, blk = -1, slot = 0;
+    if (row_ok) {
+        p = g.pos[row];
+        if (p >= 0) { blk = g.block_table[(size_t)(row / g.R) * g.max_blocks + p / g.block_tokens]; slot = p % g.block_tokens; }
+    }
+    const float2* cs = g.rope + (size_t)(row_ok ? row : 0) * half;
+#pragma unroll 1
+    for (int hb = 0; hb < BN; hb += g.dh) {                              // heads inside this tile
+        const int col = tc.col + hb;
+        if (col >= g.N) break;                                           // warp-uniform
+        const int head = col / g.dh;
+#pragma unroll 1
+        for (int j0 = 0; j0 < half; j0 += 32) {
+            uint32_t lo[32], hi[32];
+            tc_ld32(t_row + hb + j0, lo);
+            tc_ld32(t_row + hb + half + j0, hi);
+            tc_wait_ld();
+            if (p < 0) continue;
+            float a[32], b[32];
+            if (head < g.Hq + g.Hkv) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const float2 t = cs[j0 + e];
+                    const float x = __uint_as_float(lo[e]), y = __uint_as_float(hi[e]);
+                    a[e] = x * t.x - y * t.y;
+                    b[e] = y * t.x + x * t.y;
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) { a[e] = __uint_as_float(lo[e]); b[e] = __uint_as_float(hi[e]); }
+            }
+            __nv_bfloat16* dst;
+            if (head < g.Hq) {
+                dst = static_cast<__nv_bfloat16*>(g.C) + (size_t)row * g.ldc + col;
+            } else {
+                if (blk < 0) continue;
+                const bool is_k = head < g.Hq + g.Hkv;
+                const int kh = is_k ? head - g.Hq : head - g.Hq - g.Hkv;
+                dst = (is_k ? g.k_pool : g.v_pool) + (((size_t)blk * g.Hkv + kh) * g.block_tokens + slot) * g.dh;
+            }
+            store_bf16x32(dst + j0, a);
+            store_bf16x32(dst + half + j0, b);
+        }
+    }
+}
+
 // Decodes work item w into (m-tile, n-tile, group) and the tile's row window.  Returns false for an empty tile.
-struct TileCoord { int a_row, b_row, c_row, rows_valid, col; };
 __device__ __forceinline__ bool tile_coord(const GemmArgs& g, int w, int m_tiles, int n_tiles, TileCoord& t)
 {
     const int mt = w % m_tiles, nt = (w / m_tiles) % n_tiles;
@@ -133,6 +279,7 @@ __device__ __forceinline__ bool tile_coord(const GemmArgs& g, int w, int m_tiles
     return true;
 }
 
+template <int EPI>
 __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a,
                                                               const __grid_constant__ CUtensorMap map_b, const GemmArgs g)
 {
@@ -233,59 +380,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             const int row = tc.c_row + row_in_tile;
             const bool row_ok = row_in_tile < tc.rows_valid;
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                const int col = tc.col + c0;
-                if (col >= g.N) break;                              // warp-uniform
-                uint32_t v[32];
-                tc_ld32(t_row + c0, v);
-                tc_wait_ld();
-                if (row_ok) {
-                    if (g.out_f32) {
-                        float* cp = static_cast<float*>(g.C) + (size_t)row * g.ldc + col;
-                        if (col + 32 <= g.N) {
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                float4 o = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                                       __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-                                if (g.accumulate) {
-                                    const float4 p = *reinterpret_cast<const float4*>(cp + 4 * j);
-                                    o.x += p.x; o.y += p.y; o.z += p.z; o.w += p.w;
-                                }
-                                *reinterpret_cast<float4*>(cp + 4 * j) = o;
-                            }
-                        } else {
-                            for (int j = 0; j < 32 && col + j < g.N; ++j)
-                                cp[j] = __uint_as_float(v[j]) + (g.accumulate ? cp[j] : 0.f);
-                        }
-                    } else {
-                        __nv_bfloat16* cp = static_cast<__nv_bfloat16*>(g.C) + (size_t)row * g.ldc + col;
-                        if (col + 32 <= g.N) {
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                float f[8];
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * j + e]);
-                                if (g.accumulate) {
-                                    const uint4 p = *reinterpret_cast<const uint4*>(cp + 8 * j);
-                                    const __nv_bfloat162* pp = reinterpret_cast<const __nv_bfloat162*>(&p);
-#pragma unroll
-                                    for (int e = 0; e < 4; ++e) { f[2 * e] += __low2float(pp[e]); f[2 * e + 1] += __high2float(pp[e]); }
-                                }
-                                uint4 o;
-                                __nv_bfloat162 t0 = __floats2bfloat162_rn(f[0], f[1]), t1 = __floats2bfloat162_rn(f[2], f[3]);
-                                __nv_bfloat162 t2 = __floats2bfloat162_rn(f[4], f[5]), t3 = __floats2bfloat162_rn(f[6], f[7]);
-                                o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
-                                o.z = *reinterpret_cast<uint32_t*>(&t2); o.w = *reinterpret_cast<uint32_t*>(&t3);
-                                *reinterpret_cast<uint4*>(cp + 8 * j) = o;
-                            }
-                        } else {
-                            for (int j = 0; j < 32 && col + j < g.N; ++j)
-                                cp[j] = __float2bfloat16_rn(__uint_as_float(v[j]) + (g.accumulate ? __bfloat162float(cp[j]) : 0.f));
-                        }
-                    }
-                }
-            }
+            if constexpr (EPI == EPI_SWIGLU) epilogue_swiglu(g, tc, t_row, row, row_ok);
+            else if constexpr (EPI == EPI_QKV) epilogue_qkv(g, tc, t_row, row, row_ok);
+            else epilogue_plain(g, tc, t_row, row, row_ok);
             tc_fence_before();
             mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
         }
@@ -316,10 +413,20 @@ bool init_once()
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&g_sms, cudaDevAttrMultiProcessorCount, dev);
     if (g_sms <= 0) g_sms = 148;
-    constexpr int smem = STAGES * STAGE_BYTES + 1024 + 256;
-    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+    if (cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return false;
+    if (cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return false;
+    if (cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return false;
     g_encode = reinterpret_cast<EncodeFn>(fn);
     return true;
+}
+
+spec_status run_kernel(int epi, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& g, long long n_work, cudaStream_t st)
+{
+    const int grid = n_work < g_sms ? (int)n_work : g_sms;
+    if (epi == EPI_SWIGLU)   gemm_tc_kernel<EPI_SWIGLU><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, g);
+    else if (epi == EPI_QKV) gemm_tc_kernel<EPI_QKV><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, g);
+    else                     gemm_tc_kernel<EPI_PLAIN><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, g);
+    return launch_status();
 }
 
 // 2-D map over a row-major [rows][cols] bf16 matrix with row pitch ld elements; box = 64 columns x box_rows rows.
@@ -355,17 +462,50 @@ spec_status launch_gemm_tc(int M, int N, int K, const void* A, int lda, const vo
     if (!make_map(&ma, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM)) return SPEC_ERR_CUDA;
     if (!make_map(&mb, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
     const int n_work = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-    GemmArgs g{M, N, K, C, ldc, out_dtype == SPEC_DTYPE_F32 ? 1 : 0, accumulate, status, 0, 0, nullptr, nullptr};
-    constexpr int smem = STAGES * STAGE_BYTES + 1024 + 256;
-    gemm_tc_kernel<<<n_work < g_sms ? n_work : g_sms, kThreads, smem, st>>>(ma, mb, g);
-    return launch_status();
+    GemmArgs g{};
+    g.M = M; g.N = N; g.K = K; g.C = C; g.ldc = ldc; g.out_f32 = out_dtype == SPEC_DTYPE_F32 ? 1 : 0; g.accumulate = accumulate;
+    g.status = status;
+    return run_kernel(EPI_PLAIN, ma, mb, g, n_work, st);
+}
+
+// gate/up projection with the SwiGLU applied in the epilogue: W [2F][K] stored in 256-row groups (128 gate rows, then the
+// matching 128 up rows), act [M][F] bf16.
+spec_status launch_gemm_swiglu_tc(int M, int F, int K, const void* A, int lda, const void* W, void* act, int32_t* status,
+                                  cudaStream_t st)
+{
+    if (M == 0 || F == 0) return SPEC_OK;
+    if (!init_once()) return SPEC_ERR_CUDA;
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM)) return SPEC_ERR_CUDA;
+    if (!make_map(&mb, W, (uint64_t)2 * F, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
+    GemmArgs g{};
+    g.M = M; g.N = 2 * F; g.K = K; g.C = act; g.ldc = F; g.status = status;
+    return run_kernel(EPI_SWIGLU, ma, mb, g, (long long)((M + BM - 1) / BM) * (2 * F / BN), st);
+}
+
+// QKV projection with rotary embedding and KV append in the epilogue.
+spec_status launch_gemm_qkv_tc(int M, int K, const void* A, int lda, const void* W, void* qkv, const QkvEpilogue& e,
+                               int32_t* status, cudaStream_t st)
+{
+    const int N = (e.Hq + 2 * e.Hkv) * e.dh;
+    if (M == 0) return SPEC_OK;
+    if (!init_once()) return SPEC_ERR_CUDA;
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM)) return SPEC_ERR_CUDA;
+    if (!make_map(&mb, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
+    GemmArgs g{};
+    g.M = M; g.N = N; g.K = K; g.C = qkv; g.ldc = N; g.status = status;
+    g.Hq = e.Hq; g.Hkv = e.Hkv; g.dh = e.dh; g.R = e.R; g.max_blocks = e.max_blocks; g.block_tokens = e.block_tokens;
+    g.pos = e.pos; g.block_table = e.block_table; g.rope = reinterpret_cast<const float2*>(e.rope);
+    g.k_pool = static_cast<__nv_bfloat16*>(e.k_pool); g.v_pool = static_cast<__nv_bfloat16*>(e.v_pool);
+    return run_kernel(EPI_QKV, ma, mb, g, (long long)((M + BM - 1) / BM) * ((N + BN - 1) / BN), st);
 }
 
 // Grouped form: A [rows_total][K] holds the groups' rows back to back (group e at offsets[e], counts[e] rows, both on
 // the device; no group has more than max_rows_per_group rows), W [E][N][K], C [rows_total][N].  N % 256 == 0.
 spec_status launch_gemm_grouped(int rows_total, int max_rows_per_group, int E, int N, int K, const void* A, const void* W,
-                                void* C, int out_dtype, const int32_t* counts, const int32_t* offsets, int32_t* status,
-                                cudaStream_t st)
+                                void* C, int out_dtype, int swiglu, const int32_t* counts, const int32_t* offsets,
+                                int32_t* status, cudaStream_t st)
 {
     if (rows_total == 0 || E == 0) return SPEC_OK;
     if (N % BN != 0 || K % 8 != 0) return SPEC_ERR_SHAPE;
@@ -374,11 +514,10 @@ spec_status launch_gemm_grouped(int rows_total, int max_rows_per_group, int E, i
     if (!make_map(&ma, A, (uint64_t)rows_total, (uint64_t)K, (uint64_t)K, BM)) return SPEC_ERR_CUDA;
     if (!make_map(&mb, W, (uint64_t)E * N, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
     const int max_m_tiles = (max_rows_per_group + BM - 1) / BM;
-    GemmArgs g{rows_total, N, K, C, N, out_dtype == SPEC_DTYPE_F32 ? 1 : 0, 0, status, E, max_m_tiles, counts, offsets};
-    constexpr int smem = STAGES * STAGE_BYTES + 1024 + 256;
-    const long long n_work = (long long)E * max_m_tiles * (N / BN);
-    gemm_tc_kernel<<<n_work < g_sms ? (int)n_work : g_sms, kThreads, smem, st>>>(ma, mb, g);
-    return launch_status();
+    GemmArgs g{};
+    g.M = rows_total; g.N = N; g.K = K; g.C = C; g.ldc = swiglu ? N / 2 : N; g.out_f32 = out_dtype == SPEC_DTYPE_F32 ? 1 : 0;
+    g.status = status; g.E = E; g.max_m_tiles = max_m_tiles; g.counts = counts; g.offsets = offsets;
+    return run_kernel(swiglu ? EPI_SWIGLU : EPI_PLAIN, ma, mb, g, (long long)E * max_m_tiles * (N / BN), st);
 }
 
 spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int dtype_in,

@@ -143,6 +143,7 @@ __global__ void __launch_bounds__(256) rope_append_kernel(int R, int Hq, int Hkv
     }
 }
 
+// gate_up [M][2F] holds 256-column groups: 128 gate columns, then the matching 128 up columns
 template <class T>
 __global__ void swiglu_kernel(size_t total4, int F, const T* __restrict__ gu, T* __restrict__ out)
 {
@@ -150,12 +151,28 @@ __global__ void swiglu_kernel(size_t total4, int F, const T* __restrict__ gu, T*
     if (i >= total4) return;
     const size_t e = i * 4;
     const size_t m = e / F, c = e % F;
+    const size_t gc = (c / 128) * 256 + c % 128;
     float g[4], u[4], o[4];
-    Vec4<T>::load(gu + m * 2 * F + c, g);
-    Vec4<T>::load(gu + m * 2 * F + F + c, u);
+    Vec4<T>::load(gu + m * 2 * F + gc, g);
+    Vec4<T>::load(gu + m * 2 * F + gc + 128, u);
 #pragma unroll
     for (int j = 0; j < 4; ++j) o[j] = g[j] / (1.f + __expf(-g[j])) * u[j];
     Vec4<T>::store(out + e, o);
+}
+
+// (cos, sin) of pos * theta^(-2j/dh), j < dh/2, per row; formed in fp64 (see rope_append_kernel)
+__global__ void rope_table_kernel(int M, int half, int dh, float theta, const int32_t* __restrict__ pos, float2* __restrict__ table)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M * half) return;
+    const int m = i / half, j = i % half;
+    const int p = pos[m];
+    double s = 0.0, c = 1.0;
+    if (p >= 0) {
+        const double inv = exp2(-2.0 * (double)j / (double)dh * log2((double)theta));
+        sincos((double)p * inv, &s, &c);
+    }
+    table[i] = make_float2((float)c, (float)s);
 }
 
 template <class T>
@@ -214,9 +231,10 @@ __device__ int block_exclusive_scan(int v, int* total, int* s_warp /*[33]*/)
 }
 
 __global__ void __launch_bounds__(kBookThreads) kv_reserve_kernel(int B, int k, int bt, int max_blocks,
-                                                                  const int32_t* seq_len, int32_t* table,
+                                                                  const int32_t* seq_len, int32_t* table, int32_t* owned,
                                                                   int32_t* free_stack, int32_t* free_top, int32_t* status)
 {
+    // owned[b] = number of logical blocks sequence b holds (always the prefix 0..owned-1 of its table row)
     __shared__ int s_warp[33];
     __shared__ int s_fail;
     if (threadIdx.x == 0) s_fail = 0;
@@ -230,7 +248,7 @@ __global__ void __launch_bounds__(kBookThreads) kv_reserve_kernel(int B, int k, 
         if (b < B) {
             const int need = (seq_len[b] + k + 1 + bt - 1) / bt;
             if (need > max_blocks) { s_fail = 1; set_status(status, SPEC_ERR_KV_EXHAUSTED, b); }
-            else for (int j = 0; j < need; ++j) need_new += table[(size_t)b * max_blocks + j] < 0;
+            else need_new = max(0, need - owned[b]);
         }
         int tot;
         block_exclusive_scan(need_new, &tot, s_warp);
@@ -242,18 +260,13 @@ __global__ void __launch_bounds__(kBookThreads) kv_reserve_kernel(int B, int k, 
     int carry = 0;
     for (int base = 0; base < B; base += kBookThreads) {
         const int b = base + threadIdx.x;
-        int need = 0, need_new = 0;
-        if (b < B) {
-            need = (seq_len[b] + k + 1 + bt - 1) / bt;
-            for (int j = 0; j < need; ++j) need_new += table[(size_t)b * max_blocks + j] < 0;
-        }
+        int need = 0, have = 0;
+        if (b < B) { need = (seq_len[b] + k + 1 + bt - 1) / bt; have = owned[b]; }
         int tot;
-        int off = carry + block_exclusive_scan(need_new, &tot, s_warp);
-        if (b < B) {
-            for (int j = 0; j < need; ++j) {
-                int32_t* e = &table[(size_t)b * max_blocks + j];
-                if (*e < 0) { *e = free_stack[top0 - 1 - off]; ++off; }
-            }
+        int off = carry + block_exclusive_scan(max(0, need - have), &tot, s_warp);
+        if (b < B && need > have) {
+            for (int j = have; j < need; ++j) { table[(size_t)b * max_blocks + j] = free_stack[top0 - 1 - off]; ++off; }
+            owned[b] = need;
         }
         carry += tot;
     }
@@ -291,17 +304,18 @@ __global__ void __launch_bounds__(kBookThreads) kv_commit_kernel(const CommitArg
             a.seq_len[b] = len;
             a.last_token[b] = last;
             keep = (len + a.block_tokens - 1) / a.block_tokens;
-            for (int j = keep; j < a.max_blocks; ++j) freed += a.block_table[(size_t)b * a.max_blocks + j] >= 0;
+            freed = max(0, a.owned[b] - keep);
             atomicAdd((unsigned long long*)&s_cnt[0], (unsigned long long)n1);
             atomicAdd((unsigned long long*)&s_cnt[1], (unsigned long long)(n1 - 1));
         }
         int tot;
         int off = carry + block_exclusive_scan(freed, &tot, s_warp);
-        if (b < a.B) {
-            for (int j = keep; j < a.max_blocks; ++j) {
+        if (b < a.B && freed > 0) {
+            for (int j = keep; j < keep + freed; ++j) {
                 int32_t* e = &a.block_table[(size_t)b * a.max_blocks + j];
-                if (*e >= 0) { a.free_stack[top0 + off] = *e; ++off; *e = -1; }
+                a.free_stack[top0 + off] = *e; ++off; *e = -1;
             }
+            a.owned[b] = keep;
         }
         carry += tot;
     }
@@ -364,6 +378,14 @@ spec_status launch_swiglu(int M, int F, const void* gate_up, void* out, int dtyp
     return launch_status();
 }
 
+spec_status launch_rope_table(int M, int dh, float theta, const int32_t* pos, float* table, cudaStream_t st)
+{
+    const int n = M * (dh / 2);
+    if (n == 0) return SPEC_OK;
+    rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(M, dh / 2, dh, theta, pos, reinterpret_cast<float2*>(table));
+    return launch_status();
+}
+
 spec_status launch_copy_rows_f32_to(int M, int d, const float* x, void* out, int ld_out, int col0, int dtype,
                                     cudaStream_t st)
 {
@@ -381,11 +403,11 @@ spec_status launch_gather_last_rows(int B, int R, int d, const float* src, const
 }
 
 spec_status launch_kv_reserve(int B, int k, int block_tokens, int max_blocks, const int32_t* seq_len,
-                              int32_t* block_table, int32_t* free_stack, int32_t* free_top, int32_t* status,
+                              int32_t* block_table, int32_t* owned, int32_t* free_stack, int32_t* free_top, int32_t* status,
                               cudaStream_t st)
 {
     if (B == 0) return SPEC_OK;
-    kv_reserve_kernel<<<1, kBookThreads, 0, st>>>(B, k, block_tokens, max_blocks, seq_len, block_table, free_stack, free_top, status);
+    kv_reserve_kernel<<<1, kBookThreads, 0, st>>>(B, k, block_tokens, max_blocks, seq_len, block_table, owned, free_stack, free_top, status);
     return launch_status();
 }
 

@@ -45,7 +45,7 @@ spec_status launch_gather_last_rows(int B, int R, int d, const float* src, const
 
 // KV bookkeeping (single CTA, deterministic order)
 spec_status launch_kv_reserve(int B, int k, int block_tokens, int max_blocks, const int32_t* seq_len,
-                              int32_t* block_table, int32_t* free_stack, int32_t* free_top, int32_t* status,
+                              int32_t* block_table, int32_t* owned, int32_t* free_stack, int32_t* free_top, int32_t* status,
                               cudaStream_t st);
 struct CommitArgs {
     int B, k, block_tokens, max_blocks;
@@ -54,7 +54,7 @@ struct CommitArgs {
     const int32_t* verify_tokens; // [B][k+1] input tokens of the last verify (read by a forced commit)
     int32_t* n_emitted;           // [B] in: sampler's n+1 (ignored when forced); out: committed n+1
     int32_t* out_tokens;          // [B][k+1]
-    int32_t* seq_len; int32_t* last_token; int32_t* block_table; int32_t* free_stack; int32_t* free_top;
+    int32_t* seq_len; int32_t* last_token; int32_t* block_table; int32_t* owned; int32_t* free_stack; int32_t* free_top;
     int32_t* pending_base;        // [B] first position committed by this step
     uint32_t* step; long long* counters;   // counters: steps, emitted, accepted
     int32_t* status;
@@ -67,9 +67,24 @@ spec_status launch_gemm_simt(int M, int N, int K, const void* A, int lda, const 
 spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int dtype_in,
                         int out_dtype, int accumulate, cudaStream_t st);
 
+// swiglu != 0: W holds [2F] rows per group in 256-row gate/up groups and C is the activation [rows][N/2] (bf16)
 spec_status launch_gemm_grouped(int rows_total, int max_rows_per_group, int E, int N, int K, const void* A, const void* W,
-                                void* C, int out_dtype, const int32_t* counts, const int32_t* offsets, int32_t* status,
-                                cudaStream_t st);
+                                void* C, int out_dtype, int swiglu, const int32_t* counts, const int32_t* offsets,
+                                int32_t* status, cudaStream_t st);
+bool gemm_tc_supported(int M, int N, int K, const void* A, int lda, const void* W, const void* C, int ldc, int dtype_in,
+                       int out_dtype);
+spec_status launch_gemm_swiglu_tc(int M, int F, int K, const void* A, int lda, const void* W, void* act, int32_t* status,
+                                  cudaStream_t st);
+struct QkvEpilogue {
+    int Hq, Hkv, dh, R, max_blocks, block_tokens;
+    const int32_t* pos; const int32_t* block_table;
+    const float* rope;            // [M][dh/2][2] (cos, sin) of each row's position
+    void* k_pool; void* v_pool;
+};
+spec_status launch_gemm_qkv_tc(int M, int K, const void* A, int lda, const void* W, void* qkv, const QkvEpilogue& e,
+                               int32_t* status, cudaStream_t st);
+// (cos, sin) table of the rows' positions for the fused QKV epilogue
+spec_status launch_rope_table(int M, int dh, float theta, const int32_t* pos, float* table, cudaStream_t st);
 
 // moe.cu: router top-k, permutation into expert order, weighted combination
 spec_status launch_moe_route(int M, int E, int top_k, const float* logits, int32_t* ids, float* wts, cudaStream_t st);

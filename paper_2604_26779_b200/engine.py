@@ -36,6 +36,26 @@ def make_spec_config(cfg: dict, *, draft_kind: str = "none", k_max: int = 3, max
     return sc
 
 
+def stack_gate_up(gate, up):
+    """[.., F, d] gate and up -> the library's stacked layout [.., 2F, d]: 256-row groups of 128 gate rows followed by
+    the matching 128 up rows."""
+    gate, up = np.asarray(gate), np.asarray(up)
+    F, d = gate.shape[-2:]
+    lead = gate.shape[:-2]
+    g = gate.reshape(lead + (F // 128, 128, d))
+    u = up.reshape(lead + (F // 128, 128, d))
+    return np.concatenate([g, u], axis=-2).reshape(lead + (2 * F, d))
+
+
+def unstack_gate_up(gu):
+    """Inverse of stack_gate_up: returns (gate, up)."""
+    gu = np.asarray(gu)
+    F2, d = gu.shape[-2:]
+    lead = gu.shape[:-2]
+    t = gu.reshape(lead + (F2 // 256, 256, d))
+    return t[..., :128, :].reshape(lead + (F2 // 2, d)), t[..., 128:, :].reshape(lead + (F2 // 2, d))
+
+
 class SpecStep:
     """One context over arenas allocated here.  Methods mirror the C entry points one to one."""
 
@@ -107,10 +127,10 @@ class SpecStep:
             self.put("MLP_NORM", l, lw["mlp_norm"], f32)
             if "router" in lw:
                 self.put("ROUTER", l, lw["router"])
-                self.put("EXPERTS_GATEUP", l, np.concatenate([lw["experts_gate"], lw["experts_up"]], axis=1))
+                self.put("EXPERTS_GATEUP", l, stack_gate_up(lw["experts_gate"], lw["experts_up"]))
                 self.put("EXPERTS_DOWN", l, lw["experts_down"])
             else:
-                self.put("WGATEUP", l, np.concatenate([lw["wgate"], lw["wup"]], axis=0))
+                self.put("WGATEUP", l, stack_gate_up(lw["wgate"], lw["wup"]))
                 self.put("WDOWN", l, lw["wdown"])
 
     def load_draft_weights(self, H: dict):
@@ -120,7 +140,7 @@ class SpecStep:
         self.put("D_MLP_NORM", 0, H["mlp_norm"], f32)
         self.put("D_WQKV", 0, H["wqkv"])
         self.put("D_WO", 0, H["wo"])
-        self.put("D_WGATEUP", 0, np.concatenate([H["wgate"], H["wup"]], axis=0))
+        self.put("D_WGATEUP", 0, stack_gate_up(H["wgate"], H["wup"]))
         self.put("D_WDOWN", 0, H["wdown"])
         if self.sc.draft_kind == B.SPEC_DRAFT_EAGLE3:
             self.put("D_WFC", 0, H["wfc"])
