@@ -118,6 +118,76 @@ def cpu_oracle_sample(eng, info, k, n_layers_sample, step_index):
                 fetch_seconds=t_fetch_head)
 
 
+def run_sampler_microbench(args):
+    """Rejection-sampling micro-benchmark (B=1024, V=151936, k in {1,3,5,7}; target logits N(0, sigma^2), draft = target +
+    N(0, tau^2)): the stateless sampler on given fp32 probabilities, and the fused from-logits path (row statistics +
+    sampler).  Reports time and GB/s on the algorithmic bytes (one pass over two rows per rejected sequence, one row per
+    fully accepted one), measured acceptance against 2*Phi(-tau/2) and mean tokens per step against (1-a^(k+1))/(1-a)."""
+    import math
+    import torch
+    from paper_2604_26779_b200 import binding as api, report
+    B, V = args.batch if args.batch != 256 else 1024, 151936
+    dev = "cuda"
+    gen = torch.Generator(device=dev); gen.manual_seed(2604026779 + 2000)
+    hbm_peak, _, kind = measured_peaks()
+    rows_out = []
+    cases = [(k, 1.0, 0.5) for k in (1, 3, 5, 7)] + [(3, s, t) for s in (1.0, 3.0) for t in (0.1, 0.5, 1.0)]
+    seen = set()
+    for k, sigma, tau in cases:
+        if (k, sigma, tau) in seen:
+            continue
+        seen.add((k, sigma, tau))
+        tl = torch.empty((B, k + 1, V), dtype=torch.float32, device=dev).normal_(0.0, sigma, generator=gen)
+        dl = tl[:, :k, :] + torch.empty((B, k, V), dtype=torch.float32, device=dev).normal_(0.0, tau, generator=gen)
+        ps, qs = torch.empty((B * (k + 1), 2), device=dev), torch.empty((B * k, 2), device=dev)
+        p, q = torch.empty_like(tl), torch.empty_like(dl)
+        api.spec_softmax_rows(tl, 1.0, ps, p)
+        api.spec_softmax_rows(dl, 1.0, qs, q)
+        drafts = torch.empty((B, k), dtype=torch.int32, device=dev)
+        tok = torch.empty(B, dtype=torch.int32, device=dev)
+        for i in range(k):
+            api.spec_sample_rows(q[:, i, :].contiguous(), 7, 0, i, 1, tok)
+            drafts[:, i] = tok
+        out = torch.empty((B, k + 1), dtype=torch.int32, device=dev)
+        n = torch.empty(B, dtype=torch.int32, device=dev)
+        st = torch.zeros(4, dtype=torch.int32, device=dev)
+        iters = 20
+        for step in range(3):
+            api.spec_reject_sample_probs(p, q, drafts, 7, step, out, n, st)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_sum, rej_rows = 0.0, 0.0
+        e0.record()
+        for step in range(iters):
+            api.spec_reject_sample_probs(p, q, drafts, 7, 100 + step, out, n, st)
+        e1.record(); torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        nn = n.float()
+        rows_read = float(((nn <= k).float() + 1.0).sum())           # last iteration: 2 rows if rejected, 1 if all accepted
+        alg = rows_read * V * 4 + B * 2 * k * 32                       # + one 32-byte sector per gathered probability
+        # fused from logits: statistics over all rows + sampler
+        e0.record()
+        for step in range(iters):
+            api.spec_softmax_rows(tl, 1.0, ps, None)
+            api.spec_softmax_rows(dl, 1.0, qs, None)
+            api.spec_reject_sample_logits(tl, ps, dl, qs, drafts, 1.0, 7, 100 + step, out, n, st)
+        e1.record(); torch.cuda.synchronize()
+        ms_fused = e0.elapsed_time(e1) / iters
+        alg_fused = (2 * k + 1) * B * V * 4 + alg
+        a_closed = 2.0 * 0.5 * math.erfc((tau / 2.0) / math.sqrt(2.0))
+        first_acc = float((nn >= 2).float().mean())
+        rows_out.append({"k": k, "sigma": sigma, "tau": tau, "ms_probs": ms, "GBps_probs": alg / ms / 1e6,
+                         "frac_of_peak_probs": alg / ms / 1e6 / hbm_peak, "ms_from_logits": ms_fused,
+                         "GBps_from_logits": alg_fused / ms_fused / 1e6, "frac_of_peak_from_logits": alg_fused / ms_fused / 1e6 / hbm_peak,
+                         "accept_first_measured": first_acc, "accept_closed_form": a_closed,
+                         "tokens_per_step": float(nn.mean()), "tokens_per_step_iid_formula": report.expected_tokens_per_step(a_closed, k),
+                         "status": int(st[0])})
+        del tl, dl, p, q
+    print(json.dumps({"metric": "rejection-sampling micro-benchmark (B=%d, V=%d)" % (B, V), "unit": "ms / GB/s on algorithmic bytes",
+                      "peak_GBps": hbm_peak, "peak_source": kind, "data": "synthetic", "dtype": "f32", "cases": rows_out}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -131,7 +201,7 @@ def main():
     ap.add_argument("--cpu-layers", type=int, default=4, help="layers the CPU-baseline sample times (scaled to all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
-    ap.add_argument("--workload", default="c3", choices=["c3", "c4", "c5"],
+    ap.add_argument("--workload", default="c3", choices=["c3", "c4", "c5", "c2"],
                     help="c3 = the headline 8B + EAGLE-3 workload; c4 = 8B + MTP head, B=512, lognormal lengths; "
                          "c5 = one 235B-A22B-shaped MoE layer + LM head, B=256, cache length 8192 (measurement of the "
                          "other configurations; the reported metric line is c3)")
@@ -146,6 +216,8 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the speculation step has no CPU implementation")
     torch.cuda.set_device(local)
+    if args.workload == "c2":
+        return run_sampler_microbench(args) if rank == 0 else 0
     dist = None
     if world > 1 and args.impl == "ours":
         import torch.distributed as dist_mod

@@ -96,7 +96,7 @@ __device__ int block_invcdf(const WF& wf, int V, float u, InvCdfSmem& sm)
     __syncthreads();                                         // the shared buffer may still be in use by a previous draw
 
     // pass over the row: one fp64 sum per chunk
-    for (int c = warp; c < nchunks; c += kWarps) {
+    for (int c = warp; c < nchunks; c += (int)(blockDim.x >> 5)) {
         const int base = c * kChunk + lane * 4;
         float w[16];
 #pragma unroll
