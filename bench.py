@@ -368,7 +368,32 @@ def main():
         eng.set_timing(0)
         ms_vs = timed(lambda: workloads_spec_step(eng, k, with_draft=False), 3)
         ms_dec = timed(lambda: workloads.bootstrap(eng), 3)
-        line["extras"] = {"ms_verify_sample_commit": ms_vs, "ms_plain_decode_step": ms_dec,
+        # the same step captured once into a CUDA graph and replayed (the step functions only enqueue, so capture works)
+        ms_graph = None
+        try:
+            gstream = torch.cuda.Stream()
+            gstream.wait_stream(stream)
+            with torch.cuda.stream(gstream):
+                workloads_spec_step(eng, k)
+            gstream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=gstream):
+                workloads_spec_step(eng, k)
+            with torch.cuda.stream(gstream):
+                for _ in range(2):
+                    graph.replay()
+                gstream.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(gstream)
+                for _ in range(5):
+                    graph.replay()
+                b.record(gstream)
+                gstream.synchronize()
+                ms_graph = a.elapsed_time(b) / 5
+            assert eng.status().device_status == 0
+        except Exception as ex:                         # reported, never fatal for the headline number
+            ms_graph = f"capture failed: {ex}"
+        line["extras"] = {"ms_per_step_cuda_graph_replay": ms_graph, "ms_verify_sample_commit": ms_vs, "ms_plain_decode_step": ms_dec,
                           "plain_decode_tokens_per_s": B / (ms_dec / 1000.0),
                           "speedup_vs_plain_decode_at_measured_acceptance": (emitted / float(args.steps * B)) / (ms_total / args.steps / ms_dec),
                           "projected_tokens_per_s_at_paper_AL": {"2.77": 2.77 * B / (ms_total / args.steps / 1000.0),
