@@ -243,7 +243,7 @@ size_t spec_attention_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int m
  * are still the caller's.
  *   - Sizes: returns SPEC_ERR_SHAPE, launching nothing, when spec_attention_scratch_bytes(B, R, Hq, Hkv, dh,
  *     max_blocks * block_tokens) exceeds 32 MiB (33554432 bytes); for the 8B head shape with k = 3 that allows,
- *     for example, 16 sequences of up to 16384 cached positions per call.
+ *     for example, 64 sequences of up to 16384 cached positions per call (24.4 MiB).
  *   - The first call on each device looks up the array's device address (with that device current); make that
  *     first call outside any stream capture.  It calls no cudaMalloc / cudaFree and no allocating library routine.
  *   - All calls share the one array, which keeps whatever the last call left; every call rewrites what it reads
