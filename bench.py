@@ -27,7 +27,7 @@ METRIC = "accepted tokens/s per B200 (8B-shape verify+sample, k=3)"
 UNIT = "tokens/s"
 # dram bytes per attention launch from the ncu capture summarised in profiles/attention_8b_layer.md, as a ratio to the
 # algorithmic bytes of that captured launch (None until captured)
-ATTN_TRAFFIC_RATIO = 1.013
+ATTN_TRAFFIC_RATIO = 1.009
 
 
 def measured_peaks():
