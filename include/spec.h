@@ -114,6 +114,8 @@ enum {
     SPEC_T_N_EMITTED,           /* [max_batch]                                                         */
     SPEC_T_STATUS,              /* [4] device status word: code, detail, 0, 0                          */
     SPEC_T_STEP,                /* [1] step counter = Philox counter word 0                            */
+    SPEC_T_OUT_LOGP,            /* [max_batch][k+1] fp32 log p_target(token) of the emitted tokens     */
+                                /* (the verifier's log-probabilities an RL loss needs, Section 2.3)    */
     /* step results in the workspace */
     SPEC_T_LOGITS = 128,        /* [B][k+1][vocab] fp32 target logits of the last verify               */
     SPEC_T_DRAFT_LOGITS,        /* [B][k][vocab]   fp32 draft logits of the last draft                 */

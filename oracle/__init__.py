@@ -37,6 +37,8 @@ def lib():
         L.spec_oracle_uniforms.argtypes = [c.c_uint64, c.c_uint32, c.c_uint32, c.c_int, c.c_int, f32p]
         L.spec_oracle_softmax.argtypes = [f32p, c.c_int, c.c_int, c.c_double, f32p]
         L.spec_oracle_softmax_row.argtypes = [f32p, c.c_int, c.c_double, f32p, f64p, f64p]
+        L.spec_oracle_logprob.argtypes = [f32p, c.c_int, c.c_double, c.c_int]
+        L.spec_oracle_logprob.restype = c.c_double
         L.spec_oracle_invcdf_f32.argtypes = [f32p, c.c_int, c.c_float, f64p]
         L.spec_oracle_invcdf_f32.restype = c.c_int
         L.spec_oracle_reject_sample_seq.argtypes = [c.c_int, c.c_int, f32p, f32p, i32p, f32p, i32p, i32p, u32p, f64p]
@@ -97,6 +99,11 @@ def softmax_stats(logits_row, temperature=1.0):
     lib().spec_oracle_softmax_row(_p(lg, ctypes.c_float), lg.shape[0], float(temperature), None,
                                   ctypes.byref(m), ctypes.byref(z))
     return m.value, z.value
+
+
+def logprob(logits_row, token, temperature=1.0):
+    lg = _f32(logits_row)
+    return float(lib().spec_oracle_logprob(_p(lg, ctypes.c_float), lg.shape[0], float(temperature), int(token)))
 
 
 def invcdf(weights, u):

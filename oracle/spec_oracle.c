@@ -89,6 +89,15 @@ void spec_oracle_softmax_row(const float* logits, int V, double temperature, flo
     if (row_sumexp) *row_sumexp = Z;
 }
 
+/* log p(token) of one logit row at temperature T: (l_t - m)/T - log sum_v exp((l_v - m)/T), in fp64.  This is the
+ * verifier-side log-probability that an RL loss uses (Section 2.3: it must come from the target, not the draft). */
+double spec_oracle_logprob(const float* logits, int V, double temperature, int token)
+{
+    double m, Z;
+    spec_oracle_softmax_row(logits, V, temperature, NULL, &m, &Z);
+    return ((double)logits[token] - m) / temperature - log(Z);
+}
+
 void spec_oracle_softmax(const float* logits, int rows, int V, double temperature, float* probs)
 {
     for (int r = 0; r < rows; ++r)

@@ -28,7 +28,7 @@ struct spec_ctx {
     size_t kv_pool_bytes = 0, kv_bytes = 0, draft_kv_bytes = 0;
     // state
     Loc seq_len, last_token, block_table, free_stack, free_top, draft_tokens, out_tokens, n_emitted, status, step,
-        counters, pending_base, owned;
+        counters, pending_base, owned, out_logp;
     size_t state_bytes = 0;
     // workspace
     Loc tokens_in, pos, x, h, qkv, attn_out, gu, act, logits, draft_logits, row_stats, draft_row_stats, taps,
@@ -162,6 +162,7 @@ void build_layout(spec_ctx& x)
         x.counters = a.take(3 * 8);
         x.pending_base = a.take(Bm * 4);
         x.owned = a.take(Bm * 4);
+        x.out_logp = a.take(Bm * (c.k_max + 1) * 4);
         x.state_bytes = a.top;
     }
     {
@@ -412,6 +413,7 @@ extern "C" spec_status spec_tensor(spec_ctx* c, int id, int layer, void** dev_pt
     case SPEC_T_N_EMITTED: base = c->buf.state; l = c->n_emitted; break;
     case SPEC_T_STATUS: base = c->buf.state; l = c->status; break;
     case SPEC_T_STEP: base = c->buf.state; l = c->step; break;
+    case SPEC_T_OUT_LOGP: base = c->buf.state; l = c->out_logp; break;
     case SPEC_T_LOGITS: base = c->buf.workspace; l = c->logits; break;
     case SPEC_T_DRAFT_LOGITS: base = c->buf.workspace; l = c->draft_logits; break;
     case SPEC_T_ROW_STATS: base = c->buf.workspace; l = c->row_stats; break;
@@ -529,7 +531,7 @@ extern "C" spec_status spec_reject_sample(spec_ctx* c, int k, const float* draft
     TIMED(*c, CLS_SAMPLE, launch_reject_sample(true, B, k, g.vocab, at<float>(ws, c->logits), at<float>(ws, c->row_stats), ql, qs,
                                                at<int32_t>(ws, c->tokens_in) + 1, k + 1, g.temperature, g.seed,
                                                at<uint32_t>(sb, c->step), 0, at<int32_t>(sb, c->out_tokens),
-                                               at<int32_t>(sb, c->n_emitted), at<int32_t>(sb, c->status), st));
+                                               at<int32_t>(sb, c->n_emitted), at<int32_t>(sb, c->status), at<float>(sb, c->out_logp), st));
     return SPEC_OK;
 }
 

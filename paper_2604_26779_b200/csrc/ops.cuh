@@ -12,7 +12,7 @@ spec_status launch_softmax_rows(int rows, int V, const float* logits, size_t row
 spec_status launch_reject_sample(bool from_logits, int B, int k, int V, const float* p, const float* p_stats,
                                  const float* q, const float* q_stats, const int32_t* draft, int draft_stride,
                                  float temperature, uint64_t seed, const uint32_t* step_dev, uint32_t step,
-                                 int32_t* out_tokens, int32_t* n_emitted, int32_t* status, cudaStream_t st);
+                                 int32_t* out_tokens, int32_t* n_emitted, int32_t* status, float* out_logp, cudaStream_t st);
 // one token per row from logits and their statistics: uniform Philox(seed; *step_dev, row, slot, stream_tag)
 spec_status launch_sample_logits(int rows, int V, const float* logits, size_t row_stride, const float* stats,
                                  size_t stats_stride, float temperature, uint64_t seed, const uint32_t* step_dev,

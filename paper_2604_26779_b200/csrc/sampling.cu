@@ -291,6 +291,7 @@ struct RejectArgs {
     int32_t* out_tokens;       // [B][k+1]
     int32_t* n_emitted;        // [B]
     int32_t* status;
+    float* out_logp;           // [B][k+1] log p_target(emitted token) under the verifier, or nullptr
 };
 
 template <bool kFromLogits>
@@ -377,6 +378,21 @@ __global__ void __launch_bounds__(kThreads) reject_sample_kernel(const RejectArg
         A.out_tokens[(size_t)b * (k + 1) + i] = i < n ? A.draft[(size_t)b * A.draft_stride + i] : (i == n ? token : -1);
     }
     if (threadIdx.x == 0) A.n_emitted[b] = n + 1;
+    // log-probability of every emitted token under the TARGET (the quantity an RL loss needs: never the draft's)
+    if (A.out_logp != nullptr && threadIdx.x <= k) {
+        const int i = threadIdx.x;
+        float lp = 0.f;
+        if (i <= n) {
+            const int t = i < n ? A.draft[(size_t)b * A.draft_stride + i] : token;
+            if constexpr (kFromLogits) {
+                const auto P = p_row(i);
+                lp = __fmul_rn(__fsub_rn(P.l[t], P.m), P.inv_t) - logf(A.p_stats[2 * ((size_t)b * (k + 1) + i) + 1]);
+            } else {
+                lp = logf(prow0[(size_t)i * V + t]);
+            }
+        }
+        A.out_logp[(size_t)b * (k + 1) + i] = lp;
+    }
 }
 
 __global__ void uniforms_kernel(uint64_t seed, uint32_t step, uint32_t stream_tag, int n_seq, int n_slots, float* u)
@@ -399,11 +415,11 @@ spec_status launch_softmax_rows(int rows, int V, const float* logits, size_t row
 spec_status launch_reject_sample(bool from_logits, int B, int k, int V, const float* p, const float* p_stats,
                                  const float* q, const float* q_stats, const int32_t* draft, int draft_stride,
                                  float temperature, uint64_t seed, const uint32_t* step_dev, uint32_t step,
-                                 int32_t* out_tokens, int32_t* n_emitted, int32_t* status, cudaStream_t st)
+                                 int32_t* out_tokens, int32_t* n_emitted, int32_t* status, float* out_logp, cudaStream_t st)
 {
     if (B == 0) return SPEC_OK;
     RejectArgs A{B, k, V, p, q, p_stats, q_stats, draft, draft_stride, 1.0f / temperature, seed, step_dev, step, out_tokens,
-                 n_emitted, status};
+                 n_emitted, status, out_logp};
     if (from_logits) reject_sample_kernel<true><<<B, kThreads, 0, st>>>(A);
     else             reject_sample_kernel<false><<<B, kThreads, 0, st>>>(A);
     return launch_status();
@@ -457,7 +473,7 @@ extern "C" spec_status spec_reject_sample_probs(int B, int k, int V, const float
     if (k > 0 && (q == nullptr || draft == nullptr)) return SPEC_ERR_INVALID_ARG;
     if (V > sampler_max_vocab()) return SPEC_ERR_SHAPE;
     return launch_reject_sample(false, B, k, V, p, nullptr, q, nullptr, draft, k, 1.0f, seed, nullptr, step, out_tokens,
-                                n_emitted, status, (cudaStream_t)stream);
+                                n_emitted, status, nullptr, (cudaStream_t)stream);
 }
 
 extern "C" spec_status spec_reject_sample_logits(int B, int k, int V, const float* p_logits, const float* p_stats,
@@ -472,7 +488,7 @@ extern "C" spec_status spec_reject_sample_logits(int B, int k, int V, const floa
     if (k > 0 && (q_logits == nullptr || q_stats == nullptr || draft == nullptr)) return SPEC_ERR_INVALID_ARG;
     if (V > sampler_max_vocab()) return SPEC_ERR_SHAPE;
     return launch_reject_sample(true, B, k, V, p_logits, p_stats, q_logits, q_stats, draft, k, temperature, seed, nullptr,
-                                step, out_tokens, n_emitted, status, (cudaStream_t)stream);
+                                step, out_tokens, n_emitted, status, nullptr, (cudaStream_t)stream);
 }
 
 extern "C" spec_status spec_uniforms(uint64_t seed, uint32_t step, uint32_t stream_tag, int n_seq, int n_slots,

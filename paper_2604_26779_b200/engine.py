@@ -195,6 +195,9 @@ class SpecStep:
     def out_tokens(self, k):
         return self.tensor("OUT_TOKENS", 0, torch.int32, (self.B, k + 1))
 
+    def out_logp(self, k):
+        return self.tensor("OUT_LOGP", 0, torch.float32, (self.B, k + 1))
+
     def n_emitted(self):
         return self.tensor("N_EMITTED", 0, torch.int32, (self.B,))
 

@@ -34,7 +34,19 @@ def run_chain(engine, cfg, kind, B, prompt_len, k, n_steps, seed):
     eng = engine.SpecStep(sc)
     eng.load_target_weights(W)
     eng.load_draft_weights(H)
-    eng.seq_init(np.zeros(B, np.int32), prompts[:, 0], inputs.make_block_order(sc.kv_num_blocks, inputs.sub_seed(1, 3)))
+    order = inputs.make_block_order(sc.kv_num_blocks, inputs.sub_seed(1, 3))
+    eng.seq_init(np.zeros(B, np.int32), prompts[:, 0], order)
+    # the oracle's paged-KV bookkeeping runs alongside on host copies: integer state must match bit for bit
+    o_len, o_table = np.zeros(B, np.int32), np.full((B, max_blocks), -1, np.int32)
+    o_free, o_top = order.copy(), np.array([sc.kv_num_blocks], np.int32)
+
+    def check_books(n_committed):
+        oracle.kv_commit(16, n_committed, o_len, o_table, o_free, o_top)
+        assert np.array_equal(eng.seq_len().cpu().numpy(), o_len)
+        assert np.array_equal(eng.block_table().cpu().numpy(), o_table)
+        top = int(eng.tensor("FREE_TOP", 0, torch.int32, (1,)).item())
+        assert top == int(o_top[0])
+        assert np.array_equal(eng.tensor("FREE_STACK", 0, torch.int32, (sc.kv_num_blocks,)).cpu().numpy()[:top], o_free[:top])
 
     # teacher-forced prefill: chunks of k+1 prompt tokens through the verify path
     R = k + 1
@@ -43,12 +55,15 @@ def run_chain(engine, cfg, kind, B, prompt_len, k, n_steps, seed):
     for c in range(n_chunks):
         if c > 0:
             eng.draft(1)                                   # lets the draft head absorb the slots just committed
+            assert oracle.kv_reserve(1, 16, o_len, o_table, o_free, o_top) == 0
+        assert oracle.kv_reserve(k, 16, o_len, o_table, o_free, o_top) == 0
         forced = torch.from_numpy(np.ascontiguousarray(prompts[:, c * R + 1 : c * R + R])).cuda()
         eng.verify(k, forced)
         last = c == n_chunks - 1
         fn = torch.full((B,), k - 1 if last else k, dtype=torch.int32, device="cuda")
         ft = torch.from_numpy(np.ascontiguousarray(prompts[:, -1] if last else prompts[:, (c + 1) * R])).cuda()
         eng.kv_commit(fn, ft)
+        check_books(np.full(B, (k - 1 if last else k) + 1, np.int32))
     assert eng.status().device_status == 0
     assert eng.seq_len().cpu().tolist() == [prompt_len - 1] * B
 
@@ -62,12 +77,18 @@ def run_chain(engine, cfg, kind, B, prompt_len, k, n_steps, seed):
         eng.kv_commit()
         rep = eng.status()
         assert rep.device_status == 0
+        assert oracle.kv_reserve(k, 16, o_len, o_table, o_free, o_top) == 0
+        check_books(eng.n_emitted().cpu().numpy())
         g_logits = eng.logits(k).cpu().numpy()
         g_dlogits = eng.draft_logits(k).cpu().numpy()
         g_drafts = eng.draft_tokens().cpu().numpy()[:, :k]
         g_out = eng.out_tokens(k).cpu().numpy()
         g_n = eng.n_emitted().cpu().numpy()
         g_len = eng.seq_len().cpu().numpy()
+        g_lp = eng.out_logp(k).cpu().numpy()
+        for b in range(B):                      # verifier log-probabilities of the emitted tokens, from the device's own logits
+            for i in range(g_n[b]):
+                assert abs(g_lp[b, i] - oracle.logprob(g_logits[b, i], int(g_out[b, i]), cfg.get("temperature", 1.0))) < 1e-4
         for b in range(B):
             ch = chains[b]
             rec = ch.step_once(k)

@@ -53,6 +53,15 @@ def test_softmax_matches_scipy(T):
     assert m == lg[0].max() and np.isclose(np.log(z) + m / T, scipy.special.logsumexp(lg[0].astype(np.float64) / T))
 
 
+def test_logprob_matches_scipy_log_softmax():
+    rng = np.random.default_rng(9)
+    lg = (rng.standard_normal(5000) * 4).astype(np.float32)
+    for T in (1.0, 0.6):
+        ref = scipy.special.log_softmax(lg.astype(np.float64) / T)
+        for t in (0, 17, 4999, int(np.argmax(lg))):
+            assert abs(oracle.logprob(lg, t, T) - ref[t]) < 1e-12
+
+
 # ---- inverse CDF ---------------------------------------------------------------------------------------------
 
 def test_invcdf_edges():
