@@ -198,7 +198,7 @@ def main():
     ap.add_argument("--k", type=int, default=3)
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--kv-pools", type=int, default=None)
-    ap.add_argument("--cpu-layers", type=int, default=4, help="layers the CPU-baseline sample times (scaled to all)")
+    ap.add_argument("--cpu-layers", type=int, default=12, help="layers the CPU-baseline sample times (scaled to all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--workload", default="c3", choices=["c3", "c4", "c5", "c2"],

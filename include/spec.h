@@ -177,7 +177,9 @@ spec_status spec_verify(spec_ctx* ctx, int k, const int32_t* draft_tokens, void*
 /* S3+S4 fused vocabulary softmax and rejection sampling on the context's logits: accept_i = u_i <
  * min(1, p_i(d_i)/q_i(d_i)); n = accepted prefix length; token n+1 from norm(max(0, p_{n+1}-q_{n+1})) or,
  * when n = k, the bonus token from p_{k+1}; uniforms Philox(seed; step, sequence, slot 0..k, stream 0).
- * draft_logits [B][k][vocab] overrides the context's draft logits when not NULL (draft_kind NONE). */
+ * draft_logits [B][k][vocab] overrides the context's draft logits when not NULL.  With draft_kind NONE and
+ * draft_logits NULL the drafts are taken as deterministic (n-gram lookup, greedy drafting): q = one-hot(d), i.e.
+ * accept iff u < p(d), residual = p without the draft token's mass. */
 spec_status spec_reject_sample(spec_ctx* ctx, int k, const float* draft_logits, void* stream);
 
 /* S5 KV commit / rollback: seq_len += n+1, blocks past the new length return to the free stack, the last
@@ -203,7 +205,8 @@ spec_status spec_sample_rows(int rows, int V, const float* probs, uint64_t seed,
                              uint32_t stream_tag, int32_t* tokens, int32_t* status, void* stream);
 
 /* Rejection sampling on given probabilities: p [B][k+1][V], q [B][k][V], draft [B][k] ->
- * out_tokens [B][k+1] (-1 padded), n_emitted [B] in 1..k+1.  status [4] int32 device status word (may be NULL). */
+ * out_tokens [B][k+1] (-1 padded), n_emitted [B] in 1..k+1.  status [4] int32 device status word (may be NULL).
+ * q == NULL means deterministic drafts: q = one-hot(draft). */
 spec_status spec_reject_sample_probs(int B, int k, int V, const float* p, const float* q, const int32_t* draft,
                                      uint64_t seed, uint32_t step, int32_t* out_tokens, int32_t* n_emitted,
                                      int32_t* status, void* stream);

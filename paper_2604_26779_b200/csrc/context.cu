@@ -517,13 +517,13 @@ extern "C" spec_status spec_reject_sample(spec_ctx* c, int k, const float* draft
     if (c == nullptr) return SPEC_ERR_INVALID_ARG;
     const spec_config& g = c->cfg;
     if (!c->verified || k != c->k_last) return SPEC_ERR_STATE;
-    if (k > 0 && draft_logits == nullptr && g.draft_kind == SPEC_DRAFT_NONE) return SPEC_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const int B = c->B;
     if (B == 0) return SPEC_OK;
     void* ws = c->buf.workspace;
     char* sb = static_cast<char*>(c->buf.state);
-    const float* ql = draft_logits ? draft_logits : at<float>(ws, c->draft_logits);
+    // no draft head and no draft logits: the drafts are deterministic (n-gram lookup, greedy), q = one-hot(d)
+    const float* ql = draft_logits ? draft_logits : (g.draft_kind == SPEC_DRAFT_NONE ? nullptr : at<float>(ws, c->draft_logits));
     float* qs = at<float>(ws, c->draft_row_stats);
     if (draft_logits != nullptr && k > 0)
         TRY(launch_softmax_rows(B * k, g.vocab, ql, (size_t)g.vocab, g.temperature, qs, 1, nullptr, st));

@@ -80,6 +80,18 @@ struct ResidualLogits {               // w = max(0, softmax(lp/T) - softmax(lq/T
     }
 };
 
+// Deterministic draft (q = one-hot(d)): the residual is p with the draft token's mass removed.
+template <class Row>
+struct ResidualOneHot {
+    Row P; int d;
+    __device__ void load(int idx, int V, float (&w)[4]) const
+    {
+        P.load(idx, V, w);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) if (idx + e == d) w[e] = 0.f;
+    }
+};
+
 struct InvCdfSmem {
     double chunk_sum[kMaxChunks];
     int token;
@@ -335,12 +347,12 @@ __global__ void __launch_bounds__(kThreads) reject_sample_kernel(const RejectArg
                 float pd, qd;
                 if constexpr (kFromLogits) {
                     const auto P = p_row(i);
-                    const auto Q = q_row(i);
                     pd = prob_from_logit(P.l[d], P.m, P.inv_t, P.inv_z);
-                    qd = prob_from_logit(Q.l[d], Q.m, Q.inv_t, Q.inv_z);
+                    if (A.q != nullptr) { const auto Q = q_row(i); qd = prob_from_logit(Q.l[d], Q.m, Q.inv_t, Q.inv_z); }
+                    else qd = 1.f;                                   // deterministic draft: q = one-hot(d)
                 } else {
                     pd = prow0[(size_t)i * V + d];
-                    qd = qrow0[(size_t)i * V + d];
+                    qd = A.q != nullptr ? qrow0[(size_t)i * V + d] : 1.f;
                 }
                 const float u = philox_uniform(A.seed, step, (uint32_t)b, (uint32_t)i, 0u);
                 double thr;
@@ -357,7 +369,14 @@ __global__ void __launch_bounds__(kThreads) reject_sample_kernel(const RejectArg
     const float u_last = philox_uniform(A.seed, step, (uint32_t)b, (uint32_t)k, 0u);
 
     int token;
-    if (n < k) {
+    if (n < k && A.q == nullptr) {
+        const int dn = A.draft[(size_t)b * A.draft_stride + n];
+        token = block_invcdf(ResidualOneHot<decltype(p_row(n))>{p_row(n), dn}, V, u_last, sm);
+        if (token < 0) {
+            if (threadIdx.x == 0) set_status(A.status, SPEC_ERR_BAD_PROB, b);
+            token = block_invcdf(p_row(n), V, u_last, sm);
+        }
+    } else if (n < k) {
         if constexpr (kFromLogits) token = block_invcdf(ResidualLogits{p_row(n), q_row(n)}, V, u_last, sm);
         else                       token = block_invcdf(ResidualProbs{prow0 + (size_t)n * V, qrow0 + (size_t)n * V,
                                                                       row_vec_ok(prow0 + (size_t)n * V, V) &&
@@ -470,7 +489,7 @@ extern "C" spec_status spec_reject_sample_probs(int B, int k, int V, const float
     if (B < 0 || k < 0 || k > 31 || V <= 0) return SPEC_ERR_INVALID_ARG;
     if (B == 0) return SPEC_OK;
     if (p == nullptr || out_tokens == nullptr || n_emitted == nullptr) return SPEC_ERR_INVALID_ARG;
-    if (k > 0 && (q == nullptr || draft == nullptr)) return SPEC_ERR_INVALID_ARG;
+    if (k > 0 && draft == nullptr) return SPEC_ERR_INVALID_ARG;       // q == NULL: deterministic drafts, q = one-hot(d)
     if (V > sampler_max_vocab()) return SPEC_ERR_SHAPE;
     return launch_reject_sample(false, B, k, V, p, nullptr, q, nullptr, draft, k, 1.0f, seed, nullptr, step, out_tokens,
                                 n_emitted, status, nullptr, (cudaStream_t)stream);
@@ -485,7 +504,7 @@ extern "C" spec_status spec_reject_sample_logits(int B, int k, int V, const floa
     if (B == 0) return SPEC_OK;
     if (p_logits == nullptr || p_stats == nullptr || out_tokens == nullptr || n_emitted == nullptr)
         return SPEC_ERR_INVALID_ARG;
-    if (k > 0 && (q_logits == nullptr || q_stats == nullptr || draft == nullptr)) return SPEC_ERR_INVALID_ARG;
+    if (k > 0 && (draft == nullptr || (q_logits != nullptr && q_stats == nullptr))) return SPEC_ERR_INVALID_ARG;
     if (V > sampler_max_vocab()) return SPEC_ERR_SHAPE;
     return launch_reject_sample(true, B, k, V, p_logits, p_stats, q_logits, q_stats, draft, k, temperature, seed, nullptr,
                                 step, out_tokens, n_emitted, status, nullptr, (cudaStream_t)stream);

@@ -154,6 +154,27 @@ def test_one_hot_draft_and_bad_rows(api):
         assert np.array_equal(out, o_out) and n[0] == o_n[0] and (st[0] == -18) == bool(o_fl[0] & 1)
 
 
+def test_deterministic_drafts_one_hot_mode(api):
+    """q = NULL: drafts are deterministic (n-gram / greedy); must equal the oracle run with an explicit one-hot q."""
+    B, k, V = 200, 3, 3000
+    _, _, p, _, _ = make_case(B, k, V, 2.0, 0.5, seed=13)
+    drafts = np.argsort(-p[:, :k, :], axis=-1)[:, :, 0].astype(np.int32)       # greedy drafts: likely accepted
+    drafts[::3] = np.random.default_rng(2).integers(0, V, (len(drafts[::3]), k))   # and some unlikely ones
+    q = np.zeros((B, k, V), np.float32)
+    for b in range(B):
+        for i in range(k):
+            q[b, i, drafts[b, i]] = 1.0
+    out = torch.zeros((B, k + 1), dtype=torch.int32, device="cuda")
+    n = torch.zeros(B, dtype=torch.int32, device="cuda")
+    st = torch.zeros(4, dtype=torch.int32, device="cuda")
+    for step in (0, 1):
+        api.spec_reject_sample_probs(dev(p), None, dev(drafts), 21, step, out, n, st)
+        torch.cuda.synchronize()
+        assert st[0].item() == 0
+        assert compare_with_oracle(out.cpu().numpy(), n.cpu().numpy(), p, q, drafts, 21, step) <= 1
+    assert 1 < n.float().mean().item() < k + 1
+
+
 def test_fused_from_logits_matches_oracle_on_gpu_probabilities(api):
     for (B, k, V, sigma, tau, T) in [(64, 3, 128256, 1.0, 0.5, 1.0), (96, 5, 1027, 3.0, 1.0, 0.8), (512, 3, 8, 1.0, 0.5, 1.0)]:
         t, d, _, _, _ = make_case(B, k, V, sigma, tau, seed=V + k)
