@@ -132,6 +132,8 @@ def run_sampler_microbench(args):
     hbm_peak, _, kind = measured_peaks()
     rows_out = []
     cases = [(k, 1.0, 0.5) for k in (1, 3, 5, 7)] + [(3, s, t) for s in (1.0, 3.0) for t in (0.1, 0.5, 1.0)]
+    if args.c2_cases == "k3":
+        cases = [(3, 1.0, 0.5)]
     seen = set()
     for k, sigma, tau in cases:
         if (k, sigma, tau) in seen:
@@ -198,6 +200,9 @@ def main():
     ap.add_argument("--k", type=int, default=3)
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--kv-pools", type=int, default=None)
+    ap.add_argument("--len-lo", type=int, default=1024, help="cache length range of the c3 workload (profiling on small footprints)")
+    ap.add_argument("--len-hi", type=int, default=16384)
+    ap.add_argument("--c2-cases", default="all", help="'all' or 'k3' (one case: profiling)")
     ap.add_argument("--cpu-layers", type=int, default=12, help="layers the CPU-baseline sample times (scaled to all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
@@ -230,6 +235,7 @@ def main():
     ext_drafts = None
     if args.workload == "c3":
         eng, info = workloads.build_dense_workload("c3", B=B, k=k, n_layers=args.layers, kv_pools=args.kv_pools,
+                                                   len_lo=args.len_lo, len_hi=args.len_hi,
                                                    steps_budget=steps_budget, device=f"cuda:{local}",
                                                    seed=replicas.replica_seed(rank))
         wl_name = ("c3: 8B dense verify (32 layers, d=4096, 32q/8kv, dh=128, FFN 14336, V=128256, bf16), "
