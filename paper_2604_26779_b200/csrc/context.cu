@@ -223,6 +223,13 @@ LayerPtrs layer_ptrs(void* base, const LayerLoc& L)
 
 #define TRY(expr) do { spec_status s__ = (expr); if (s__ != SPEC_OK) return s__; } while (0)
 
+// Records why a call was refused (read back with spec_last_error) and returns the code.
+spec_status fail(spec_ctx* c, spec_status code, const char* why)
+{
+    if (c != nullptr) c->err = why;
+    return code;
+}
+
 constexpr int kMaxTimedPasses = 8192;
 
 // Brackets a pass with two events when its class is selected by the context's timing mask.
@@ -436,20 +443,21 @@ extern "C" spec_status spec_seq_init(spec_ctx* c, int B, const int32_t* seq_len_
 {
     if (c == nullptr || B < 0 || (B > 0 && (!seq_len_host || !last_token_host)) || !free_stack_host) return SPEC_ERR_INVALID_ARG;
     const spec_config& g = c->cfg;
-    if (B > g.max_batch) return SPEC_ERR_SHAPE;
+    if (B > g.max_batch) return fail(c, SPEC_ERR_SHAPE, "spec_seq_init: B exceeds max_batch");
     const int bt = g.kv_block_tokens, mb = g.max_blocks_per_seq, nb = g.kv_num_blocks;
     std::vector<int32_t> table((size_t)g.max_batch * mb, -1), stack(free_stack_host, free_stack_host + nb), owned(g.max_batch, 0);
     std::vector<char> seen(nb, 0);
     for (int i = 0; i < nb; ++i) {
-        if (stack[i] < 0 || stack[i] >= nb || seen[stack[i]]) return SPEC_ERR_INVALID_ARG;
+        if (stack[i] < 0 || stack[i] >= nb || seen[stack[i]]) return fail(c, SPEC_ERR_INVALID_ARG, "spec_seq_init: free_stack_host is not a permutation of the block ids");
         seen[stack[i]] = 1;
     }
     int top = nb;
     for (int b = 0; b < B; ++b) {
         if (seq_len_host[b] < 0 || last_token_host[b] < 0 || last_token_host[b] >= g.vocab) return SPEC_ERR_INVALID_ARG;
         const int need = (seq_len_host[b] + bt - 1) / bt;
-        if (need > mb || (seq_len_host[b] + g.k_max + 1 + bt - 1) / bt > mb) return SPEC_ERR_SHAPE;
-        if (need > top) return SPEC_ERR_SHAPE;
+        if (need > mb || (seq_len_host[b] + g.k_max + 1 + bt - 1) / bt > mb)
+            return fail(c, SPEC_ERR_SHAPE, "spec_seq_init: a sequence does not fit max_blocks_per_seq");
+        if (need > top) return fail(c, SPEC_ERR_SHAPE, "spec_seq_init: not enough KV blocks for the initial lengths");
         for (int j = 0; j < need; ++j) table[(size_t)b * mb + j] = stack[--top];
         owned[b] = need;
     }
@@ -474,8 +482,9 @@ extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_toke
 {
     if (c == nullptr) return SPEC_ERR_INVALID_ARG;
     const spec_config& g = c->cfg;
-    if (k < 0 || k > g.k_max) return SPEC_ERR_SHAPE;
-    if (k > 0 && draft_tokens == nullptr && g.draft_kind == SPEC_DRAFT_NONE) return SPEC_ERR_INVALID_ARG;
+    if (k < 0 || k > g.k_max) return fail(c, SPEC_ERR_SHAPE, "spec_verify: k outside 0..k_max");
+    if (k > 0 && draft_tokens == nullptr && g.draft_kind == SPEC_DRAFT_NONE)
+        return fail(c, SPEC_ERR_INVALID_ARG, "spec_verify: draft_kind NONE needs draft_tokens");
     cudaStream_t st = (cudaStream_t)stream;
     const int B = c->B, R = k + 1, M = B * R, d = g.d_model, dt = g.dtype;
     if (B == 0) return SPEC_OK;
@@ -516,7 +525,7 @@ extern "C" spec_status spec_reject_sample(spec_ctx* c, int k, const float* draft
 {
     if (c == nullptr) return SPEC_ERR_INVALID_ARG;
     const spec_config& g = c->cfg;
-    if (!c->verified || k != c->k_last) return SPEC_ERR_STATE;
+    if (!c->verified || k != c->k_last) return fail(c, SPEC_ERR_STATE, "spec_reject_sample: no verify with this k since the last commit");
     cudaStream_t st = (cudaStream_t)stream;
     const int B = c->B;
     if (B == 0) return SPEC_OK;
@@ -538,7 +547,7 @@ extern "C" spec_status spec_reject_sample(spec_ctx* c, int k, const float* draft
 extern "C" spec_status spec_kv_commit(spec_ctx* c, const int32_t* force_n, const int32_t* force_token, void* stream)
 {
     if (c == nullptr || (force_n == nullptr) != (force_token == nullptr)) return SPEC_ERR_INVALID_ARG;
-    if (!c->verified) return SPEC_ERR_STATE;
+    if (!c->verified) return fail(c, SPEC_ERR_STATE, "spec_kv_commit: nothing verified since the last commit");
     const spec_config& g = c->cfg;
     char* sb = static_cast<char*>(c->buf.state);
     CommitArgs a{};
@@ -567,8 +576,10 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
 {
     if (c == nullptr) return SPEC_ERR_INVALID_ARG;
     const spec_config& g = c->cfg;
-    if (g.draft_kind == SPEC_DRAFT_NONE || !c->have_pending || c->verified) return SPEC_ERR_STATE;
-    if (k < 1 || k > g.k_max) return SPEC_ERR_SHAPE;
+    if (g.draft_kind == SPEC_DRAFT_NONE) return fail(c, SPEC_ERR_STATE, "spec_draft: the context has no draft head");
+    if (!c->have_pending) return fail(c, SPEC_ERR_STATE, "spec_draft: no committed step to draft from (run one plain decode step first)");
+    if (c->verified) return fail(c, SPEC_ERR_STATE, "spec_draft: a verified step is waiting for its commit");
+    if (k < 1 || k > g.k_max) return fail(c, SPEC_ERR_SHAPE, "spec_draft: k outside 1..k_max");
     cudaStream_t st = (cudaStream_t)stream;
     const int B = c->B, d = g.d_model, dt = g.dtype, V = g.vocab;
     if (B == 0) return SPEC_OK;

@@ -1,0 +1,84 @@
+"""Host-side logic of the library that needs no device: configuration checks, arena sizing, tensor placement."""
+import ctypes as C
+
+import pytest
+
+from paper_2604_26779_b200 import binding as B, engine, inputs
+
+
+def sizes_of(sc):
+    s = B.spec_sizes()
+    return B.lib().spec_query_sizes(C.byref(sc), C.byref(s)), s
+
+
+def test_sizes_of_the_8b_configuration():
+    cfg = inputs.model_config("c3")
+    sc = engine.make_spec_config(cfg, draft_kind="eagle3", k_max=3, max_batch=256, kv_num_blocks=1000, max_blocks_per_seq=64,
+                                 kv_layer_pools=16)
+    code, s = sizes_of(sc)
+    assert code == 0
+    per_layer = 4096 * 6144 + 4096 * 4096 + 3 * 4096 * 14336
+    params = 32 * per_layer + 2 * 128256 * 4096
+    assert params * 2 <= s.weights_bytes <= params * 2 + (32 * 6 + 3) * 256 + 33 * 2 * 4096 * 4 + 4096
+    assert abs(params - 128256 * 4096 - 7.505e9) < 0.01e9                       # 7.5 B parameters besides the embedding table
+    assert s.kv_bytes == 16 * 2 * 1000 * 8 * 16 * 128 * 2                       # pools x (K,V) x blocks x heads x 16 x 128 x bf16
+    assert s.draft_kv_bytes == 2 * 1000 * 8 * 16 * 128 * 2
+    head = 3 * 4096 * 4096 + 6144 * 8192 + 4096 * 4096 + 3 * 4096 * 14336 + 128256 * 4096
+    assert head * 2 <= s.draft_weights_bytes <= head * 2 + 64 * 1024
+    assert s.workspace_bytes > 1024 * 128256 * 4 and s.state_bytes > 256 * 64 * 4
+
+
+@pytest.mark.parametrize("change,code", [
+    (dict(struct_size=8), -1), (dict(abi_version=99), -1), (dict(n_q_heads=30), -2), (dict(k_max=8), -2),
+    (dict(kv_layer_pools=0), -2), (dict(kv_layer_pools=33), -2), (dict(temperature=0.0), -3), (dict(dtype=5), -3),
+    (dict(d_ffn=1000), -2), (dict(vocab=128255), -2), (dict(vocab=1 << 20), -2), (dict(draft_kind=7), -3),
+    (dict(n_experts=4, experts_top_k=8, d_expert_ffn=128), -2), (dict(n_experts=4, experts_top_k=2, d_expert_ffn=100), -3)])
+def test_bad_configurations_are_refused(change, code):
+    cfg = inputs.model_config("c3")
+    sc = engine.make_spec_config(cfg, draft_kind="none", k_max=3, max_batch=8, kv_num_blocks=100, max_blocks_per_seq=16)
+    for k, v in change.items():
+        setattr(sc, k, v)
+    got, _ = sizes_of(sc)
+    assert got == code, (change, got)
+
+
+def test_create_checks_pointers_and_tensors_do_not_overlap():
+    cfg = inputs.model_config("c1")
+    sc = engine.make_spec_config(cfg, draft_kind="eagle3", k_max=3, max_batch=4, kv_num_blocks=32, max_blocks_per_seq=8)
+    code, s = sizes_of(sc)
+    assert code == 0
+    L = B.lib()
+    bufs = B.spec_buffers()
+    base = 1 << 30                                             # fake, aligned, never dereferenced by these calls
+    offs = {}
+    for i, name in enumerate(("weights", "draft_weights", "kv", "draft_kv", "workspace", "state")):
+        offs[name] = base + i * (1 << 32)
+        setattr(bufs, name, offs[name])
+    h = C.c_void_p()
+    bufs.kv = offs["kv"] + 8                                   # misaligned arena
+    assert L.spec_create(C.byref(sc), C.byref(bufs), C.byref(h)) == -1
+    bufs.kv = offs["kv"]
+    assert L.spec_create(C.byref(sc), C.byref(bufs), C.byref(h)) == 0
+    spans = []
+    for name, tid in B.T.items():
+        for layer in range(cfg["n_layers"] if 3 <= tid <= 8 else 1):
+            p, n = C.c_void_p(), C.c_size_t()
+            rc = L.spec_tensor(h, tid, layer, C.byref(p), C.byref(n))
+            if rc != 0:
+                continue                                         # tensors this configuration does not have
+            assert p.value % 256 == 0 and n.value > 0
+            arena = max((a for a in offs.values() if a <= p.value))
+            aname = [k for k, v in offs.items() if v == arena][0]
+            assert p.value + n.value <= arena + getattr(s, aname + "_bytes"), name
+            if name not in ("HIDDEN",):
+                spans.append((p.value, p.value + n.value, name))
+    spans.sort()
+    for (a0, a1, an), (b0, b1, bn) in zip(spans, spans[1:]):
+        assert a1 <= b0, (an, bn)
+    # calls that are out of order are refused with a reason
+    assert L.spec_draft(h, 3, None) == -4 and b"no committed step" in L.spec_last_error(h)
+    assert L.spec_kv_commit(h, None, None, None) == -4
+    assert L.spec_reject_sample(h, 3, None, None) == -4
+    assert L.spec_verify(h, 9, None, None) == -2 and b"k outside" in L.spec_last_error(h)
+    assert L.spec_tensor(h, 9999, 0, C.byref(C.c_void_p()), C.byref(C.c_size_t())) == -1
+    assert L.spec_destroy(h) == 0
