@@ -268,6 +268,12 @@ typedef struct { float ms[4]; int32_t passes[4]; int32_t dropped; } spec_timing;
 spec_status spec_set_timing(spec_ctx* ctx, uint32_t mask);
 spec_status spec_get_timing(spec_ctx* ctx, spec_timing* host_out, void* stream);
 
+/* Self-test of the bounded waits every tensor-core kernel uses: a one-thread kernel waits on a barrier that nothing
+ * signals, gives up after about one millisecond, and records SPEC_ERR_TIMEOUT in status [4] (device) the way the
+ * GEMM roles do; elapsed_kcycles [1] (device) receives the waited time in units of 1024 clock cycles.  Nothing
+ * traps or hangs, and the device context stays usable. */
+spec_status spec_selftest_bounded_wait(int32_t* status, int32_t* elapsed_kcycles, void* stream);
+
 /* Number of kernels the library has launched in this process so far. */
 int64_t spec_launch_count(void);
 

@@ -94,6 +94,7 @@ SIGNATURES = {
     "spec_attention_noalloc": (_i, [_i, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp]),
     "spec_set_timing": (_i, [_vp, _u32]),
     "spec_get_timing": (_i, [_vp, C.POINTER(spec_timing), _vp]),
+    "spec_selftest_bounded_wait": (_i, [_vp, _vp, _vp]),
     "spec_launch_count": (C.c_int64, []),
     "spec_version": (C.c_char_p, []),
 }

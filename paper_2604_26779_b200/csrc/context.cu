@@ -487,7 +487,7 @@ extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_toke
         return fail(c, SPEC_ERR_INVALID_ARG, "spec_verify: draft_kind NONE needs draft_tokens");
     cudaStream_t st = (cudaStream_t)stream;
     const int B = c->B, R = k + 1, M = B * R, d = g.d_model, dt = g.dtype;
-    if (B == 0) return SPEC_OK;
+    if (B == 0) { c->k_last = k; c->verified = true; return SPEC_OK; }
     void* ws = c->buf.workspace;
     char* sb = static_cast<char*>(c->buf.state);
     int32_t* status = at<int32_t>(sb, c->status);

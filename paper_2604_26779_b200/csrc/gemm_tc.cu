@@ -397,6 +397,26 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     }
 }
 
+// Self-test of the bounded wait: waits on an mbarrier that nothing ever arrives on, with a short limit, and reports the
+// outcome exactly as the GEMM roles do (abort flag -> SPEC_ERR_TIMEOUT in the status word).  The context stays usable.
+}  // namespace
+__global__ void bounded_wait_probe_kernel(long long limit_cycles, int32_t* status, int32_t* elapsed_out)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const long long t0 = clock64();
+        bool ok = mbar_try_wait(smem_u32(&bar), 0);
+        while (!ok && clock64() - t0 <= limit_cycles) ok = mbar_try_wait(smem_u32(&bar), 0);
+        if (!ok) { abort_flag = 1; set_status(status, SPEC_ERR_TIMEOUT, 0); }
+        *elapsed_out = (int32_t)((clock64() - t0) >> 10);
+    }
+}
+namespace {
+
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -529,6 +549,13 @@ spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void*
 }
 
 }  // namespace spec
+
+extern "C" spec_status spec_selftest_bounded_wait(int32_t* status, int32_t* elapsed_kcycles, void* stream)
+{
+    if (status == nullptr || elapsed_kcycles == nullptr) return SPEC_ERR_INVALID_ARG;
+    spec::bounded_wait_probe_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(2000000LL, status, elapsed_kcycles);
+    return spec::launch_status();
+}
 
 extern "C" spec_status spec_gemm(int M, int N, int K, const void* A, const void* W, void* C, int dtype_in, int out_dtype,
                                  int accumulate, void* stream)

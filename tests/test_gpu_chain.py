@@ -140,6 +140,26 @@ def test_tiny_chain_mtp_lockstep(eng_mod):
     assert r["max_rel"] < 1e-3 and r["max_rel_d"] < 1e-3 and r["boundary"] <= 2
 
 
+def test_chain_at_other_temperature_and_k1(eng_mod):
+    cfg = dict(inputs.model_config("c1"), temperature=0.7)
+    r = run_chain(eng_mod, cfg, "eagle3", B=2, prompt_len=16, k=1, n_steps=10, seed=77)
+    print("T=0.7 k=1:", r)
+    assert r["max_rel"] < 1e-3 and r["max_rel_d"] < 1e-3 and r["boundary"] <= 1
+
+
+def test_empty_batch_is_a_no_op(eng_mod):
+    cfg = inputs.model_config("c1")
+    sc = eng_mod.make_spec_config(cfg, draft_kind="eagle3", k_max=3, max_batch=2, kv_num_blocks=8, max_blocks_per_seq=4, seed=1)
+    eng = eng_mod.SpecStep(sc)
+    eng.seq_init(np.zeros(0, np.int32), np.zeros(0, np.int32), np.arange(8, dtype=np.int32))
+    eng.verify(0)
+    eng.reject_sample(0)
+    eng.kv_commit()
+    eng.draft(3)
+    assert eng.status().device_status == 0
+    eng.close()
+
+
 def test_kv_exhaustion_is_reported_not_faulted(eng_mod):
     cfg = inputs.model_config("c1")
     sc = eng_mod.make_spec_config(cfg, draft_kind="none", k_max=3, max_batch=2, kv_num_blocks=3, max_blocks_per_seq=4, seed=1)

@@ -111,3 +111,19 @@ def test_gemm_matches_fp64(api, M, N, K, din, dout, acc):
     err = np.abs(got - ref).max(-1) / np.abs(ref).max(-1)
     print(f"gemm {M}x{N}x{K} {din}->{dout} acc={acc}: worst row error {err.max():.2e}")
     assert err.max() < (2e-2 if dout == torch.bfloat16 else (1e-3 if din == torch.bfloat16 else 1e-5))
+
+
+def test_bounded_wait_times_out_cleanly(api):
+    """A wait that nothing satisfies gives up after its limit, reports SPEC_ERR_TIMEOUT, and leaves the device usable."""
+    st = torch.zeros(4, dtype=torch.int32, device="cuda")
+    el = torch.zeros(1, dtype=torch.int32, device="cuda")
+    assert api.lib().spec_selftest_bounded_wait(st.data_ptr(), el.data_ptr(), torch.cuda.current_stream().cuda_stream) == 0
+    torch.cuda.synchronize()
+    assert st[0].item() == -19 and 1500 < el.item() < 200000
+    # the context is intact: a GEMM right after still gives the right answer
+    A = torch.randn((128, 64), device="cuda", dtype=torch.bfloat16)
+    W = torch.randn((256, 64), device="cuda", dtype=torch.bfloat16)
+    Cc = torch.zeros((128, 256), device="cuda", dtype=torch.float32)
+    api.spec_gemm(A, W, Cc)
+    torch.cuda.synchronize()
+    assert torch.allclose(Cc, A.float() @ W.float().t(), atol=1e-2, rtol=1e-3)
