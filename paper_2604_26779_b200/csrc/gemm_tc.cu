@@ -8,8 +8,9 @@
 //     shared-memory ring, signalled by mbarriers;
 //   - warp 1 issues tcgen05.mma (M=128, N=256, K=16 per instruction) from one thread; the fp32 accumulator lives in
 //     tensor memory, double-buffered (2 x 256 columns) so the epilogue of one tile overlaps the next tile's loads;
-//   - warps 2-5 read the accumulator with tcgen05.ld (one 32-lane quarter each) and store fp32 / bf16, optionally
-//     adding to the fp32 residual stream.
+//   - warps 2-9 read the accumulator with tcgen05.ld (two warps per 32-lane quarter, half of the columns each) and store
+//     fp32 / bf16, optionally adding to the fp32 residual stream; the epilogue is a serial ld -> convert -> store chain per
+//     32 columns, so its length is what eight warps instead of four buy.
 // Every mbarrier wait is bounded: on a timeout the CTA raises a flag, all roles leave their loops, outstanding
 // tensor-core work is drained with a bounded wait, tensor memory is released and the kernel returns with
 // SPEC_ERR_TIMEOUT in the status word.
@@ -22,7 +23,8 @@ namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;          // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue (two per tensor-memory lane quarter)
+constexpr int kEpiThreads = 256;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSmemBytes = STAGES * STAGE_BYTES + 1024 + 256;
 constexpr long long kWaitLimit = 300000000LL;            // clock cycles (~0.15 s): far beyond any healthy wait
@@ -136,10 +138,10 @@ __device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float (&
 }
 
 // Plain epilogue: C (+)= accumulator, fp32 or bf16, ragged N handled element-wise.
-__device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok)
+__device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok, int half)
 {
 #pragma unroll 1
-    for (int c0 = 0; c0 < BN; c0 += 32) {
+    for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
         const int col = tc.col + c0;
         if (col >= g.N) break;                              // warp-uniform
         uint32_t v[32];
@@ -189,11 +191,11 @@ __device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoor
 
 // SwiGLU epilogue: the tile's first 128 columns are gate rows, the last 128 the matching up rows (the stacked weight is
 // stored in such 256-row groups); writes act = silu(gate) * up, bf16, [rows][N/2].
-__device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok)
+__device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok, int half)
 {
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(g.C) + (size_t)row * g.ldc + tc.col / 2;
 #pragma unroll 1
-    for (int c0 = 0; c0 < BN / 2; c0 += 32) {
+    for (int c0 = half * (BN / 4); c0 < (half + 1) * (BN / 4); c0 += 32) {
         uint32_t gv[32], uv[32];
         tc_ld32(t_row + c0, gv);
         tc_ld32(t_row + BN / 2 + c0, uv);
@@ -211,7 +213,7 @@ __device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, const TileCoo
 
 // QKV epilogue: heads of width dh; q and k heads get the rotary embedding (pairs (j, j + dh/2)); q goes to C (bf16,
 // [rows][N]), k and v go to the paged cache slot of the row's position.  Rows with a negative position write nothing.
-__device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok)
+__device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok, int part)
 {
     const int half = g.dh / 2;
     int p = -1, blk = -1, slot = 0;
@@ -221,7 +223,7 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord&
     }
     const float2* cs = g.rope + (size_t)(row_ok ? row : 0) * half;
 #pragma unroll 1
-    for (int hb = 0; hb < BN; hb += g.dh) {                              // heads inside this tile
+    for (int hb = part * (BN / 2); hb < (part + 1) * (BN / 2); hb += g.dh) {   // this warp's heads inside the tile
         const int col = tc.col + hb;
         if (col >= g.N) break;                                           // warp-uniform
         const int head = col / g.dh;
@@ -295,7 +297,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&ctl->tmem_full[a]), 1); mbar_init(smem_u32(&ctl->tmem_empty[a]), 128); }
+        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&ctl->tmem_full[a]), 1); mbar_init(smem_u32(&ctl->tmem_empty[a]), kEpiThreads); }
         mbar_init(smem_u32(&ctl->drain), 1);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -365,8 +367,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             }
         }
     } else {
-        // ---- epilogue: warps 2..5, each owns the 32-lane quarter (warp % 4) of tensor memory ----
-        const int quarter = warp & 3;
+        // ---- epilogue: warps 2..9; a warp may only touch the 32-lane quarter (warp % 4) of tensor memory, so two warps
+        // share each quarter and split the tile's columns in halves ----
+        const int quarter = warp & 3, half = (warp - 2) >> 2;
         bool ok = true;
         int it = 0;
         for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
@@ -380,9 +383,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             const int row = tc.c_row + row_in_tile;
             const bool row_ok = row_in_tile < tc.rows_valid;
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-            if constexpr (EPI == EPI_SWIGLU) epilogue_swiglu(g, tc, t_row, row, row_ok);
-            else if constexpr (EPI == EPI_QKV) epilogue_qkv(g, tc, t_row, row, row_ok);
-            else epilogue_plain(g, tc, t_row, row, row_ok);
+            if constexpr (EPI == EPI_SWIGLU) epilogue_swiglu(g, tc, t_row, row, row_ok, half);
+            else if constexpr (EPI == EPI_QKV) epilogue_qkv(g, tc, t_row, row, row_ok, half);
+            else epilogue_plain(g, tc, t_row, row, row_ok, half);
             tc_fence_before();
             mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
         }
