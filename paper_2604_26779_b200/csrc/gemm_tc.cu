@@ -118,7 +118,7 @@ struct GemmArgs {
     const int32_t* counts; const int32_t* offsets;
     // EPI_QKV: rotary embedding on q and k heads, k and v written straight into the paged cache
     int Hq, Hkv, dh, R, max_blocks, block_tokens;
-    const int32_t* pos; const int32_t* block_table; const float2* rope;   // rope [M][dh/2] (cos, sin) of each row's position
+    const int32_t* pos; const int32_t* block_table; const float2* rope;   // rope [dh/2][M] (cos, sin) of each row's position
     __nv_bfloat16* k_pool; __nv_bfloat16* v_pool;
 };
 
@@ -221,7 +221,7 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord&
         p = g.pos[row];
         if (p >= 0) { blk = g.block_table[(size_t)(row / g.R) * g.max_blocks + p / g.block_tokens]; slot = p % g.block_tokens; }
     }
-    const float2* cs = g.rope + (size_t)(row_ok ? row : 0) * half;
+    const float2* cs = g.rope + (row_ok ? row : 0);                      // table is [dh/2][M]: element j of this row at cs[j * M]
 #pragma unroll 1
     for (int hb = part * (BN / 2); hb < (part + 1) * (BN / 2); hb += g.dh) {   // this warp's heads inside the tile
         const int col = tc.col + hb;
@@ -238,7 +238,7 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord&
             if (head < g.Hq + g.Hkv) {
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
-                    const float2 t = cs[j0 + e];
+                    const float2 t = cs[(size_t)(j0 + e) * g.M];
                     const float x = __uint_as_float(lo[e]), y = __uint_as_float(hi[e]);
                     a[e] = x * t.x - y * t.y;
                     b[e] = y * t.x + x * t.y;

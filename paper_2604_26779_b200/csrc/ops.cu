@@ -160,7 +160,7 @@ __global__ void swiglu_kernel(size_t total4, int F, const T* __restrict__ gu, T*
     Vec4<T>::store(out + e, o);
 }
 
-// (cos, sin) of pos * theta^(-2j/dh), j < dh/2, per row; formed in fp64 (see rope_append_kernel)
+// (cos, sin) of pos * theta^(-2j/dh), j < dh/2, per row, stored [dh/2][M]; formed in fp64 (see rope_append_kernel)
 __global__ void rope_table_kernel(int M, int half, int dh, float theta, const int32_t* __restrict__ pos, float2* __restrict__ table)
 {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -172,7 +172,8 @@ __global__ void rope_table_kernel(int M, int half, int dh, float theta, const in
         const double inv = exp2(-2.0 * (double)j / (double)dh * log2((double)theta));
         sincos((double)p * inv, &s, &c);
     }
-    table[i] = make_float2((float)c, (float)s);
+    table[(size_t)j * M + m] = make_float2((float)c, (float)s);      // [dh/2][M]: rows are the fast index, so the GEMM
+                                                                    // epilogue (one row per lane) reads it coalesced
 }
 
 template <class T>

@@ -78,7 +78,7 @@ spec_status launch_gemm_swiglu_tc(int M, int F, int K, const void* A, int lda, c
 struct QkvEpilogue {
     int Hq, Hkv, dh, R, max_blocks, block_tokens;
     const int32_t* pos; const int32_t* block_table;
-    const float* rope;            // [M][dh/2][2] (cos, sin) of each row's position
+    const float* rope;            // [dh/2][M][2] (cos, sin) of each row's position
     void* k_pool; void* v_pool;
 };
 spec_status launch_gemm_qkv_tc(int M, int K, const void* A, int lda, const void* W, void* qkv, const QkvEpilogue& e,
