@@ -78,6 +78,27 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def gemm_flops_per_step(cfg, B, k, draft):
+    """Dense-contraction flops of one step (2*M*N*K per GEMM): verify forward, LM heads and the draft head's passes."""
+    d, F, V = cfg["d_model"], cfg["d_ffn"], cfg["vocab"]
+    qn, od = (cfg["n_q_heads"] + 2 * cfg["n_kv_heads"]) * cfg["head_dim"], cfg["n_q_heads"] * cfg["head_dim"]
+    if cfg.get("n_experts", 0) > 0:
+        mlp = cfg["n_experts"] * d + cfg["experts_top_k"] * 3 * d * cfg["d_expert_ffn"]
+    else:
+        mlp = 3 * d * F
+    layer = d * qn + od * d + mlp
+    M = B * (k + 1)
+    total = 2.0 * M * (cfg["n_layers"] * layer + V * d)
+    if draft == "eagle3":
+        Fd = F or 4 * d
+        head = 2 * d * qn + od * d + 3 * d * Fd
+        total += 2.0 * M * (len(cfg["tap_layers"]) * d * d + head) + 2.0 * B * (k - 1) * head + 2.0 * B * k * V * d
+    elif draft == "mtp":
+        head = 2 * d * d + d * qn + od * d + 3 * d * F
+        total += 2.0 * M * head + 2.0 * B * (k - 1) * head + 2.0 * B * k * V * d
+    return total
+
+
 def cpu_oracle_sample(eng, info, k, n_layers_sample, step_index):
     """Times the oracle (as it stands) on a bounded sample of the same workload: ONE sequence of the batch, the first
     `n_layers_sample` decoder layers at full width against that sequence's real cache bytes, plus final norm, LM head,
@@ -405,6 +426,8 @@ def main():
                           "projected_tokens_per_s_at_paper_AL": {"2.77": 2.77 * B / (ms_total / args.steps / 1000.0),
                                                                  "3.32": 3.32 * B / (ms_total / args.steps / 1000.0)},
                           "ms_by_class_per_step": {"attention": tm.ms[0] / 2, "gemm": tm.ms[1] / 2, "softmax_sampling": tm.ms[2] / 2},
+                          "gemm_tflops_in_step": gemm_flops_per_step(cfg, B, k, info["draft"]) / (tm.ms[1] / 2 * 1e-3) / 1e12,
+                          "gemm_frac_of_measured_sustained_bf16": gemm_flops_per_step(cfg, B, k, info["draft"]) / (tm.ms[1] / 2 * 1e-3) / 1e12 / tf_peak,
                           }
 
     # ---- end-to-end through the C ABI with host buffers: seq_init from host arrays (H2D) + K steps, each followed by a
