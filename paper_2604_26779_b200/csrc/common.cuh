@@ -30,6 +30,10 @@ inline spec_status launch_status(int n_launched = 1)
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }
 
+// Per-thread scratch for split-K GEMMs, set by the context entry points (the stateless spec_gemm has none and never splits).
+struct GemmScratch { void* ptr = nullptr; size_t bytes = 0; };
+GemmScratch& gemm_scratch();
+
 // ---- Philox4x32-10 (Salmon et al., SC'11).  key = (lo, hi) of the seed, counter = (step, seq, slot, stream);
 // the uniform is the top 24 bits of the first output word scaled by 2^-24: in [0,1), exact in fp32. ------------
 __device__ __forceinline__ uint32_t philox_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,

@@ -33,7 +33,7 @@ struct spec_ctx {
     // workspace
     Loc tokens_in, pos, x, h, qkv, attn_out, gu, act, logits, draft_logits, row_stats, draft_row_stats, taps,
         attn_scratch, dg, dx, d_hidden, d_tok, d_pos,
-        moe_logits, moe_ids, moe_wts, moe_rank, moe_counts, moe_offsets, moe_inv, moe_a, moe_gu, moe_act, moe_out, rope;
+        moe_logits, moe_ids, moe_wts, moe_rank, moe_counts, moe_offsets, moe_inv, moe_a, moe_gu, moe_act, moe_out, rope, splitk;
     size_t workspace_bytes = 0;
     // host-side run state
     int B = 0;
@@ -190,6 +190,7 @@ void build_layout(spec_ctx& x)
         x.d_tok = a.take(M * 4);
         x.d_pos = a.take(M * 4);
         x.rope = a.take(M * (size_t)(c.head_dim / 2) * 8);
+        x.splitk = a.take((size_t)32 << 20);
         if (c.n_experts > 0) {
             const size_t n = M * c.experts_top_k, E = c.n_experts, Fe = c.d_expert_ffn;
             x.moe_logits = a.take(M * E * 4);
@@ -229,6 +230,16 @@ spec_status fail(spec_ctx* c, spec_status code, const char* why)
     if (c != nullptr) c->err = why;
     return code;
 }
+
+// Installs the context's split-K scratch for the duration of a step function.
+struct ScratchScope {
+    explicit ScratchScope(spec_ctx* c)
+    {
+        spec::gemm_scratch().ptr = static_cast<char*>(c->buf.workspace) + c->splitk.off;
+        spec::gemm_scratch().bytes = c->splitk.bytes;
+    }
+    ~ScratchScope() { spec::gemm_scratch() = spec::GemmScratch{}; }
+};
 
 constexpr int kMaxTimedPasses = 8192;
 
@@ -488,6 +499,7 @@ extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_toke
     cudaStream_t st = (cudaStream_t)stream;
     const int B = c->B, R = k + 1, M = B * R, d = g.d_model, dt = g.dtype;
     if (B == 0) { c->k_last = k; c->verified = true; return SPEC_OK; }
+    ScratchScope scratch_scope(c);
     void* ws = c->buf.workspace;
     char* sb = static_cast<char*>(c->buf.state);
     int32_t* status = at<int32_t>(sb, c->status);
@@ -583,6 +595,7 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
     cudaStream_t st = (cudaStream_t)stream;
     const int B = c->B, d = g.d_model, dt = g.dtype, V = g.vocab;
     if (B == 0) return SPEC_OK;
+    ScratchScope scratch_scope(c);
     void* ws = c->buf.workspace;
     void* dw = c->buf.draft_weights;
     char* sb = static_cast<char*>(c->buf.state);
@@ -658,6 +671,12 @@ extern "C" spec_status spec_get_status(spec_ctx* c, spec_step_report* out, void*
     out->emitted_tokens = counters[1];
     out->accepted_drafts = counters[2];
     return SPEC_OK;
+}
+
+spec::GemmScratch& spec::gemm_scratch()
+{
+    static thread_local GemmScratch s;
+    return s;
 }
 
 long long& spec::launch_counter()

@@ -27,6 +27,7 @@ constexpr int kThreads = 320;          // warp 0 TMA, warp 1 MMA, warps 2..9 epi
 constexpr int kEpiThreads = 256;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSmemBytes = STAGES * STAGE_BYTES + 1024 + 256;
+#define TRY_LAUNCH(expr) do { spec_status s__ = (expr); if (s__ != SPEC_OK) return s__; } while (0)
 constexpr long long kWaitLimit = 300000000LL;            // clock cycles (~0.15 s): far beyond any healthy wait
 
 struct Ctl {
@@ -105,7 +106,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr)
 // Instruction descriptor: D fp32, A and B bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
-struct TileCoord { int a_row, b_row, c_row, rows_valid, col; };
+struct TileCoord { int a_row, b_row, c_row, rows_valid, col, kb0, kb1; };
 
 struct GemmArgs {
     int M, N, K;
@@ -116,6 +117,9 @@ struct GemmArgs {
     // [offsets[e], offsets[e] + counts[e]) of A by the weight rows [e*N, (e+1)*N) of W; counts/offsets live on the device.
     int E, max_m_tiles;
     const int32_t* counts; const int32_t* offsets;
+    // split-K (splits > 1, plain epilogue only): work item = (tile, split); split s covers k-blocks [s*kb_per, (s+1)*kb_per)
+    // and stores its fp32 partial at C + s * M * ldc (C is then a scratch buffer; a second kernel sums the splits in order)
+    int splits, kb_per;
     // EPI_QKV: rotary embedding on q and k heads, k and v written straight into the paged cache
     int Hq, Hkv, dh, R, max_blocks, block_tokens;
     const int32_t* pos; const int32_t* block_table; const float2* rope;   // rope [dh/2][M] (cos, sin) of each row's position
@@ -265,6 +269,10 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord&
 // Decodes work item w into (m-tile, n-tile, group) and the tile's row window.  Returns false for an empty tile.
 __device__ __forceinline__ bool tile_coord(const GemmArgs& g, int w, int m_tiles, int n_tiles, TileCoord& t)
 {
+    const int kb_count = (g.K + BK - 1) / BK;
+    t.kb0 = 0; t.kb1 = kb_count;
+    int split = 0;
+    if (g.splits > 1) { split = w % g.splits; w /= g.splits; t.kb0 = split * g.kb_per; t.kb1 = min(kb_count, t.kb0 + g.kb_per); }
     const int mt = w % m_tiles, nt = (w / m_tiles) % n_tiles;
     if (g.E > 0) {
         const int e = w / (m_tiles * n_tiles);
@@ -274,7 +282,7 @@ __device__ __forceinline__ bool tile_coord(const GemmArgs& g, int w, int m_tiles
         t.a_row = off + mt * BM; t.c_row = t.a_row; t.rows_valid = cnt - mt * BM;
         t.b_row = e * g.N + nt * BN;
     } else {
-        t.a_row = mt * BM; t.c_row = t.a_row; t.rows_valid = g.M - mt * BM;
+        t.a_row = mt * BM; t.c_row = t.a_row + split * g.M; t.rows_valid = g.M - mt * BM;
         t.b_row = nt * BN;
     }
     t.col = nt * BN;
@@ -293,7 +301,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     const int m_tiles = g.E > 0 ? g.max_m_tiles : (g.M + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
-    const int n_work = m_tiles * n_tiles * (g.E > 0 ? g.E : 1), kb_count = (g.K + BK - 1) / BK;
+    const int n_work = m_tiles * n_tiles * (g.E > 0 ? g.E : 1) * (g.splits > 1 ? g.splits : 1);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
@@ -320,7 +328,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
                 TileCoord tc;
                 if (!tile_coord(g, w, m_tiles, n_tiles, tc)) continue;
-                for (int kb = 0; kb < kb_count; ++kb) {
+                for (int kb = tc.kb0; kb < tc.kb1; ++kb) {
                     if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t bar = smem_u32(&ctl->full[s]);
                     mbar_expect_tx(bar, STAGE_BYTES);
@@ -348,13 +356,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
                 if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < kb_count; ++kb) {
+                for (int kb = tc.kb0; kb < tc.kb1; ++kb) {
                     if (!mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = tiles + s * STAGE_BYTES, sb = sa + A_BYTES;
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k)
-                        tc_mma(d_tmem, smem_desc(sa + k * UMMA_K * 2), smem_desc(sb + k * UMMA_K * 2), kIdesc, (kb | k) != 0);
+                        tc_mma(d_tmem, smem_desc(sa + k * UMMA_K * 2), smem_desc(sb + k * UMMA_K * 2), kIdesc, (kb > tc.kb0 || k > 0) ? 1u : 0u);
                     tc_commit(smem_u32(&ctl->empty[s]));            // stage reusable once these MMAs have read it
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -419,6 +427,24 @@ __global__ void bounded_wait_probe_kernel(long long limit_cycles, int32_t* statu
     }
 }
 namespace {
+
+// Sums the split-K partials in split order (deterministic) into C, optionally on top of C's previous contents.
+template <class TC>
+__global__ void splitk_reduce_kernel(int M, int N, int splits, const float* __restrict__ part, TC* __restrict__ C, int ldc,
+                                     int accumulate)
+{
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i >= (size_t)M * N) return;
+    const int m = (int)(i / N), n = (int)(i % N);
+    float4 acc = *reinterpret_cast<const float4*>(part + i);
+    for (int s = 1; s < splits; ++s) {
+        const float4 v = *reinterpret_cast<const float4*>(part + (size_t)s * M * N + i);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    TC* c = C + (size_t)m * ldc + n;
+    if (accumulate) { acc.x += to_f32(c[0]); acc.y += to_f32(c[1]); acc.z += to_f32(c[2]); acc.w += to_f32(c[3]); }
+    c[0] = from_f32<TC>(acc.x); c[1] = from_f32<TC>(acc.y); c[2] = from_f32<TC>(acc.z); c[3] = from_f32<TC>(acc.w);
+}
 
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -488,6 +514,27 @@ spec_status launch_gemm_tc(int M, int N, int K, const void* A, int lda, const vo
     GemmArgs g{};
     g.M = M; g.N = N; g.K = K; g.C = C; g.ldc = ldc; g.out_f32 = out_dtype == SPEC_DTYPE_F32 ? 1 : 0; g.accumulate = accumulate;
     g.status = status;
+    // Few tiles and a long K (small-M projections: plain decode, draft passes): split K so that every SM streams weights.
+    // Partials go to the caller-provided scratch and are summed in split order by a second kernel.
+    const GemmScratch& sc = gemm_scratch();
+    const int kb_count = (K + BK - 1) / BK;
+    int splits = 1;
+    if (sc.ptr != nullptr && n_work * 2 <= g_sms && N % 4 == 0) {
+        splits = g_sms / n_work;
+        if (splits > 8) splits = 8;
+        while (splits > 1 && (kb_count / splits < 8 || (size_t)splits * M * N * 4 > sc.bytes)) --splits;
+    }
+    if (splits > 1) {
+        g.C = sc.ptr; g.ldc = N; g.out_f32 = 1; g.accumulate = 0;
+        g.splits = splits; g.kb_per = (kb_count + splits - 1) / splits;
+        TRY_LAUNCH(run_kernel(EPI_PLAIN, ma, mb, g, (long long)n_work * splits, st));
+        const size_t n4 = (size_t)M * N / 4;
+        if (out_dtype == SPEC_DTYPE_F32)
+            splitk_reduce_kernel<float><<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(M, N, splits, (const float*)sc.ptr, (float*)C, ldc, accumulate);
+        else
+            splitk_reduce_kernel<__nv_bfloat16><<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(M, N, splits, (const float*)sc.ptr, (__nv_bfloat16*)C, ldc, accumulate);
+        return launch_status();
+    }
     return run_kernel(EPI_PLAIN, ma, mb, g, n_work, st);
 }
 
