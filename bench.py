@@ -25,8 +25,8 @@ sys.path.insert(0, ROOT)
 
 METRIC = "accepted tokens/s per B200 (8B-shape verify+sample, k=3)"
 UNIT = "tokens/s"
-# dram bytes per attention launch from the ncu capture summarised in profiles/attention_8b_layer.md, as a ratio to the
-# algorithmic bytes of that captured launch (None until captured)
+# dram bytes per attention launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture on a 32-sequence case
+# of the same kernel) as a ratio to the algorithmic bytes of that captured launch; traffic grows in proportion to the units
 ATTN_TRAFFIC_RATIO = 1.009
 
 
