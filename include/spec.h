@@ -30,7 +30,7 @@
 extern "C" {
 #endif
 
-#define SPEC_ABI_VERSION 1u
+#define SPEC_ABI_VERSION 2u
 
 typedef struct spec_ctx spec_ctx; /* opaque */
 
@@ -50,7 +50,7 @@ typedef enum {
 } spec_status;
 
 enum { SPEC_DTYPE_BF16 = 0, SPEC_DTYPE_F32 = 1 };
-enum { SPEC_DRAFT_NONE = 0, SPEC_DRAFT_EAGLE3 = 1, SPEC_DRAFT_MTP = 2 };
+enum { SPEC_DRAFT_NONE = 0, SPEC_DRAFT_EAGLE3 = 1, SPEC_DRAFT_MTP = 2, SPEC_DRAFT_NGRAM = 3 };
 
 /* Model and run description.  n_experts = 0 selects the dense SwiGLU MLP. */
 typedef struct {
@@ -72,6 +72,9 @@ typedef struct {
                                 /* caches larger than the device; results are then not meaningful        */
     float temperature;          /* > 0; scales the logits of both models before the softmax              */
     uint64_t seed;              /* Philox key of every uniform the step draws                            */
+    int32_t ngram_n;            /* SPEC_DRAFT_NGRAM: longest trailing n-gram looked up in the sequence's own   */
+                                /* tokens (1..8); the model-free drafting the paper uses as a baseline (Table 2) */
+    int32_t reserved_;
 } spec_config;
 
 /* Byte sizes of the caller-owned device arenas for a configuration. */
@@ -114,6 +117,9 @@ enum {
     SPEC_T_N_EMITTED,           /* [max_batch]                                                         */
     SPEC_T_STATUS,              /* [4] device status word: code, detail, 0, 0                          */
     SPEC_T_STEP,                /* [1] step counter = Philox counter word 0                            */
+    SPEC_T_TOKEN_HISTORY,       /* [max_batch][max_blocks_per_seq*kv_block_tokens] token at every cached    */
+                                /* position (SPEC_DRAFT_NGRAM only); commits append to it, the caller fills  */
+                                /* it for positions that were cached before spec_seq_init                  */
     SPEC_T_OUT_LOGP,            /* [max_batch][k+1] fp32 log p_target(token) of the emitted tokens     */
                                 /* (the verifier's log-probabilities an RL loss needs, Section 2.3)    */
     /* step results in the workspace */
@@ -165,6 +171,8 @@ spec_status spec_seq_init(spec_ctx* ctx, int B, const int32_t* seq_len_host, con
 /* S1 draft propose.  Runs the draft head: pass 0 consumes the (tapped hidden state, next token) pairs of the
  * positions committed by the previous step, passes 1..k-1 feed the head its own output; fills draft tokens
  * d_1..d_k (d_i drawn from q_i with the stream-1 uniforms), draft logits and their row statistics.
+ * With SPEC_DRAFT_NGRAM no model runs: d_1..d_k continue the most recent earlier occurrence of the sequence's trailing
+ * n-gram (n = ngram_n down to 1; without any match the last token is repeated), and q is one-hot.
  * Errors: STATE (no committed step to draft from, draft_kind NONE), SHAPE (k outside 1..k_max). */
 spec_status spec_draft(spec_ctx* ctx, int k, void* stream);
 

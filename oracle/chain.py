@@ -32,7 +32,11 @@ class ChainOracle:
         L = len(t)
         taps_layers = tuple(cfg["tap_layers"])
         rec = {}
-        if forced_drafts is None:
+        if forced_drafts is None and self.kind == "ngram":
+            drafts = model.ngram_propose(t, int(cfg.get("ngram_n", 3)), k)
+            q = np.zeros((k, cfg["vocab"]), np.float32)
+            q[np.arange(k), drafts] = 1.0
+        elif forced_drafts is None:
             feats = model.target_forward(cfg, W, t[: L - 1], tap_layers=taps_layers)["taps"]   # positions 0..L-2
             u_draft = oracle.uniforms(self.seed, self.step, 1, self.seq + 1, max(k, 1))[self.seq]
 

@@ -246,3 +246,26 @@ def draft_propose(cfg, W, H, kind, true_feat, tokens, k, sample_fn, past_k=None,
         k_all = np.concatenate([k_all, kk], axis=0)
         v_all = np.concatenate([v_all, vv], axis=0)
     return np.array(drafts, np.int32), np.stack(q_rows), np.stack(logit_rows)
+
+
+def ngram_propose(tokens, n_max, k):
+    """Model-free drafting (the paper's n-gram baseline, Section 4.2): find the most recent earlier occurrence of the
+    trailing n tokens of `tokens` (n = n_max down to 1; a match must be followed by at least one token), propose the k
+    tokens that followed it, repeating the last proposed token once the sequence ends; without any match the last
+    token is repeated.  The proposal distribution is one-hot."""
+    t = [int(x) for x in tokens]
+    L = len(t)
+    start, n_found = -1, 0
+    for n in range(min(n_max, L - 1), 0, -1):
+        for s in range(L - 1 - n, -1, -1):
+            if t[s : s + n] == t[L - n :]:
+                start, n_found = s, n
+                break
+        if start >= 0:
+            break
+    out, prev = [], t[-1]
+    for i in range(k):
+        p = start + n_found + i
+        prev = t[p] if (start >= 0 and p <= L - 1) else prev
+        out.append(prev)
+    return np.array(out, np.int32)

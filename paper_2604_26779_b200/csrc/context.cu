@@ -28,7 +28,7 @@ struct spec_ctx {
     size_t kv_pool_bytes = 0, kv_bytes = 0, draft_kv_bytes = 0;
     // state
     Loc seq_len, last_token, block_table, free_stack, free_top, draft_tokens, out_tokens, n_emitted, status, step,
-        counters, pending_base, owned, out_logp;
+        counters, pending_base, owned, out_logp, history;
     size_t state_bytes = 0;
     // workspace
     Loc tokens_in, pos, x, h, qkv, attn_out, gu, act, logits, draft_logits, row_stats, draft_row_stats, taps,
@@ -79,7 +79,8 @@ spec_status check_config(const spec_config* c)
     if (c->n_experts > 0 && (c->dtype != SPEC_DTYPE_BF16 || c->n_experts > 256 || c->experts_top_k > 32 ||
                              c->d_expert_ffn % 128 != 0 || c->d_model % 256 != 0)) return SPEC_ERR_UNSUPPORTED;
     if (c->dtype != SPEC_DTYPE_BF16 && c->dtype != SPEC_DTYPE_F32) return SPEC_ERR_UNSUPPORTED;
-    if (c->draft_kind < SPEC_DRAFT_NONE || c->draft_kind > SPEC_DRAFT_MTP) return SPEC_ERR_UNSUPPORTED;
+    if (c->draft_kind < SPEC_DRAFT_NONE || c->draft_kind > SPEC_DRAFT_NGRAM) return SPEC_ERR_UNSUPPORTED;
+    if (c->draft_kind == SPEC_DRAFT_NGRAM && (c->ngram_n < 1 || c->ngram_n > 8)) return SPEC_ERR_SHAPE;
     if (c->k_max < 0 || c->k_max > 7 || c->max_batch <= 0) return SPEC_ERR_SHAPE;
     if (c->kv_block_tokens <= 0 || c->kv_num_blocks <= 0 || c->max_blocks_per_seq <= 0) return SPEC_ERR_SHAPE;
     if (c->kv_layer_pools <= 0 || c->kv_layer_pools > c->n_layers) return SPEC_ERR_SHAPE;
@@ -122,7 +123,7 @@ void build_layout(spec_ctx& x)
     }
     {
         Arena a;
-        if (c.draft_kind != SPEC_DRAFT_NONE) {
+        if (c.draft_kind == SPEC_DRAFT_EAGLE3 || c.draft_kind == SPEC_DRAFT_MTP) {
             const size_t F = c.draft_d_ffn;
             x.d_norm_e = a.take(d * 4);
             x.d_norm_g = a.take(d * 4);
@@ -145,7 +146,7 @@ void build_layout(spec_ctx& x)
     }
     x.kv_pool_bytes = align_up((size_t)c.kv_num_blocks * c.n_kv_heads * c.kv_block_tokens * c.head_dim * es, 256);
     x.kv_bytes = x.kv_pool_bytes * 2 * c.kv_layer_pools;
-    x.draft_kv_bytes = c.draft_kind != SPEC_DRAFT_NONE ? x.kv_pool_bytes * 2 : 0;
+    x.draft_kv_bytes = (c.draft_kind == SPEC_DRAFT_EAGLE3 || c.draft_kind == SPEC_DRAFT_MTP) ? x.kv_pool_bytes * 2 : 0;
     {
         Arena a;
         const size_t Bm = c.max_batch;
@@ -163,6 +164,7 @@ void build_layout(spec_ctx& x)
         x.pending_base = a.take(Bm * 4);
         x.owned = a.take(Bm * 4);
         x.out_logp = a.take(Bm * (c.k_max + 1) * 4);
+        if (c.draft_kind == SPEC_DRAFT_NGRAM) x.history = a.take(Bm * (size_t)c.max_blocks_per_seq * c.kv_block_tokens * 4);
         x.state_bytes = a.top;
     }
     {
@@ -355,7 +357,8 @@ extern "C" spec_status spec_create(const spec_config* cfg, const spec_buffers* b
     if (out == nullptr || b == nullptr) return SPEC_ERR_INVALID_ARG;
     TRY(check_config(cfg));
     if (!b->weights || !b->kv || !b->workspace || !b->state) return SPEC_ERR_INVALID_ARG;
-    if (cfg->draft_kind != SPEC_DRAFT_NONE && (!b->draft_weights || !b->draft_kv)) return SPEC_ERR_INVALID_ARG;
+    if ((cfg->draft_kind == SPEC_DRAFT_EAGLE3 || cfg->draft_kind == SPEC_DRAFT_MTP) && (!b->draft_weights || !b->draft_kv))
+        return SPEC_ERR_INVALID_ARG;
     const void* ptrs[] = {b->weights, b->draft_weights, b->kv, b->draft_kv, b->workspace, b->state};
     for (const void* p : ptrs) if ((reinterpret_cast<uintptr_t>(p) & 255u) != 0) return SPEC_ERR_INVALID_ARG;
     spec_ctx* c = new spec_ctx();
@@ -417,7 +420,7 @@ extern "C" spec_status spec_tensor(spec_ctx* c, int id, int layer, void** dev_pt
         l = Loc{((size_t)layer * 2 + (id == SPEC_T_KV_V ? 1 : 0)) * c->kv_pool_bytes, c->kv_pool_bytes};
         break;
     case SPEC_T_DRAFT_KV_K: case SPEC_T_DRAFT_KV_V:
-        if (g.draft_kind == SPEC_DRAFT_NONE) return SPEC_ERR_INVALID_ARG;
+        if (g.draft_kind != SPEC_DRAFT_EAGLE3 && g.draft_kind != SPEC_DRAFT_MTP) return SPEC_ERR_INVALID_ARG;
         base = c->buf.draft_kv;
         l = Loc{(id == SPEC_T_DRAFT_KV_V ? 1 : 0) * c->kv_pool_bytes, c->kv_pool_bytes};
         break;
@@ -432,6 +435,7 @@ extern "C" spec_status spec_tensor(spec_ctx* c, int id, int layer, void** dev_pt
     case SPEC_T_STATUS: base = c->buf.state; l = c->status; break;
     case SPEC_T_STEP: base = c->buf.state; l = c->step; break;
     case SPEC_T_OUT_LOGP: base = c->buf.state; l = c->out_logp; break;
+    case SPEC_T_TOKEN_HISTORY: base = c->buf.state; l = c->history; break;
     case SPEC_T_LOGITS: base = c->buf.workspace; l = c->logits; break;
     case SPEC_T_DRAFT_LOGITS: base = c->buf.workspace; l = c->draft_logits; break;
     case SPEC_T_ROW_STATS: base = c->buf.workspace; l = c->row_stats; break;
@@ -544,7 +548,8 @@ extern "C" spec_status spec_reject_sample(spec_ctx* c, int k, const float* draft
     void* ws = c->buf.workspace;
     char* sb = static_cast<char*>(c->buf.state);
     // no draft head and no draft logits: the drafts are deterministic (n-gram lookup, greedy), q = one-hot(d)
-    const float* ql = draft_logits ? draft_logits : (g.draft_kind == SPEC_DRAFT_NONE ? nullptr : at<float>(ws, c->draft_logits));
+    const bool has_head = g.draft_kind == SPEC_DRAFT_EAGLE3 || g.draft_kind == SPEC_DRAFT_MTP;
+    const float* ql = draft_logits ? draft_logits : (has_head ? at<float>(ws, c->draft_logits) : nullptr);
     float* qs = at<float>(ws, c->draft_row_stats);
     if (draft_logits != nullptr && k > 0)
         TRY(launch_softmax_rows(B * k, g.vocab, ql, (size_t)g.vocab, g.temperature, qs, 1, nullptr, st));
@@ -575,6 +580,8 @@ extern "C" spec_status spec_kv_commit(spec_ctx* c, const int32_t* force_n, const
     a.free_stack = at<int32_t>(sb, c->free_stack);
     a.free_top = at<int32_t>(sb, c->free_top);
     a.pending_base = at<int32_t>(sb, c->pending_base);
+    a.history = c->history.bytes ? at<int32_t>(sb, c->history) : nullptr;
+    a.max_hist = g.max_blocks_per_seq * g.kv_block_tokens;
     a.step = at<uint32_t>(sb, c->step);
     a.counters = at<long long>(sb, c->counters);
     a.status = at<int32_t>(sb, c->status);
@@ -589,6 +596,14 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
     if (c == nullptr) return SPEC_ERR_INVALID_ARG;
     const spec_config& g = c->cfg;
     if (g.draft_kind == SPEC_DRAFT_NONE) return fail(c, SPEC_ERR_STATE, "spec_draft: the context has no draft head");
+    if (g.draft_kind == SPEC_DRAFT_NGRAM) {
+        if (c->verified) return fail(c, SPEC_ERR_STATE, "spec_draft: a verified step is waiting for its commit");
+        if (k < 1 || k > g.k_max) return fail(c, SPEC_ERR_SHAPE, "spec_draft: k outside 1..k_max");
+        char* sbn = static_cast<char*>(c->buf.state);
+        return launch_ngram_draft(c->B, k, g.ngram_n, at<int32_t>(sbn, c->history), g.max_blocks_per_seq * g.kv_block_tokens,
+                                  at<int32_t>(sbn, c->seq_len), at<int32_t>(sbn, c->last_token), at<int32_t>(sbn, c->draft_tokens),
+                                  g.k_max, (cudaStream_t)stream);
+    }
     if (!c->have_pending) return fail(c, SPEC_ERR_STATE, "spec_draft: no committed step to draft from (run one plain decode step first)");
     if (c->verified) return fail(c, SPEC_ERR_STATE, "spec_draft: a verified step is waiting for its commit");
     if (k < 1 || k > g.k_max) return fail(c, SPEC_ERR_SHAPE, "spec_draft: k outside 1..k_max");

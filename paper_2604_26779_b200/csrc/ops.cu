@@ -300,6 +300,9 @@ __global__ void __launch_bounds__(kBookThreads) kv_commit_kernel(const CommitArg
                 n1 = min(max(a.n_emitted[b], 1), R);
                 last = a.out_tokens[(size_t)b * R + n1 - 1];
             }
+            if (a.history != nullptr)            // the tokens whose cache entries this commit keeps: x_last, d_1..d_n
+                for (int i = 0; i < n1 && a.seq_len[b] + i < a.max_hist; ++i)
+                    a.history[(size_t)b * a.max_hist + a.seq_len[b] + i] = a.verify_tokens[(size_t)b * R + i];
             a.pending_base[b] = a.seq_len[b];
             const int len = a.seq_len[b] + n1;
             a.seq_len[b] = len;
@@ -327,6 +330,44 @@ __global__ void __launch_bounds__(kBookThreads) kv_commit_kernel(const CommitArg
         a.counters[0] += 1;
         a.counters[1] += s_cnt[0];
         a.counters[2] += s_cnt[1];
+    }
+}
+
+// One CTA per sequence.  Context t[0..L-1] = history[0..len-1] followed by the last token.  For n = n_max..1: the trailing
+// n tokens are searched at every earlier start s (s + n <= L - 1, so that at least one token follows the match); the
+// largest such s wins; the draft continues from t[s+n], and once it runs past the end it repeats its last token.
+__global__ void __launch_bounds__(256) ngram_draft_kernel(int k, int n_max, const int32_t* __restrict__ history, int max_hist,
+                                                          const int32_t* __restrict__ seq_len,
+                                                          const int32_t* __restrict__ last_token,
+                                                          int32_t* __restrict__ draft, int draft_stride)
+{
+    __shared__ int s_best;
+    const int b = blockIdx.x;
+    const int32_t* h = history + (size_t)b * max_hist;
+    const int len = min(seq_len[b], max_hist), L = len + 1;
+    const int last = last_token[b];
+    auto tok = [&](int p) { return p < len ? h[p] : last; };
+    int found_s = -1, found_n = 0;
+    for (int n = min(n_max, L - 1); n >= 1 && found_s < 0; --n) {
+        if (threadIdx.x == 0) s_best = -1;
+        __syncthreads();
+        for (int s = threadIdx.x; s + n <= L - 1; s += blockDim.x) {
+            bool eq = true;
+            for (int j = 0; j < n && eq; ++j) eq = tok(s + j) == tok(L - n + j);
+            if (eq) atomicMax(&s_best, s);
+        }
+        __syncthreads();
+        if (s_best >= 0) { found_s = s_best; found_n = n; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        int prev = last;
+        for (int i = 0; i < k; ++i) {
+            const int p = found_s + found_n + i;
+            const int t = (found_s >= 0 && p <= L - 1) ? tok(p) : prev;
+            draft[(size_t)b * draft_stride + i] = t;
+            prev = t;
+        }
     }
 }
 
@@ -409,6 +450,14 @@ spec_status launch_kv_reserve(int B, int k, int block_tokens, int max_blocks, co
 {
     if (B == 0) return SPEC_OK;
     kv_reserve_kernel<<<1, kBookThreads, 0, st>>>(B, k, block_tokens, max_blocks, seq_len, block_table, owned, free_stack, free_top, status);
+    return launch_status();
+}
+
+spec_status launch_ngram_draft(int B, int k, int n_max, const int32_t* history, int max_hist, const int32_t* seq_len,
+                               const int32_t* last_token, int32_t* draft_tokens, int draft_stride, cudaStream_t st)
+{
+    if (B == 0) return SPEC_OK;
+    ngram_draft_kernel<<<B, 256, 0, st>>>(k, n_max, history, max_hist, seq_len, last_token, draft_tokens, draft_stride);
     return launch_status();
 }
 

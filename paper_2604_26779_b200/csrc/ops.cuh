@@ -56,10 +56,15 @@ struct CommitArgs {
     int32_t* out_tokens;          // [B][k+1]
     int32_t* seq_len; int32_t* last_token; int32_t* block_table; int32_t* owned; int32_t* free_stack; int32_t* free_top;
     int32_t* pending_base;        // [B] first position committed by this step
+    int32_t* history; int max_hist;            // nullable: token at every cached position, appended here
     uint32_t* step; long long* counters;   // counters: steps, emitted, accepted
     int32_t* status;
 };
 spec_status launch_kv_commit(const CommitArgs& a, cudaStream_t st);
+
+// model-free drafting: continue the most recent earlier occurrence of the trailing n-gram of (history[0..len), last token)
+spec_status launch_ngram_draft(int B, int k, int n_max, const int32_t* history, int max_hist, const int32_t* seq_len,
+                               const int32_t* last_token, int32_t* draft_tokens, int draft_stride, cudaStream_t st);
 
 // gemm_simt.cu / gemm_tc.cu: C[M][N] (+)= A[M][K] W[N][K]^T, fp32 accumulation
 spec_status launch_gemm_simt(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int dtype_in,

@@ -24,16 +24,19 @@ def eng_mod():
     return engine
 
 
-def run_chain(engine, cfg, kind, B, prompt_len, k, n_steps, seed):
+def run_chain(engine, cfg, kind, B, prompt_len, k, n_steps, seed, prompts=None):
     W = inputs.make_target_weights(cfg, seed=inputs.sub_seed(1, 0))
-    H = (inputs.make_eagle3_weights if kind == "eagle3" else inputs.make_mtp_weights)(cfg, seed=inputs.sub_seed(1, 1))
-    prompts = inputs.make_prompts(B, prompt_len, cfg["vocab"], seed=inputs.sub_seed(1, 2))
+    H = None if kind == "ngram" else \
+        (inputs.make_eagle3_weights if kind == "eagle3" else inputs.make_mtp_weights)(cfg, seed=inputs.sub_seed(1, 1))
+    if prompts is None:
+        prompts = inputs.make_prompts(B, prompt_len, cfg["vocab"], seed=inputs.sub_seed(1, 2))
     max_blocks = -(-(prompt_len + n_steps * (k + 1) + k + 2) // 16)
     sc = engine.make_spec_config(cfg, draft_kind=kind, k_max=k, max_batch=B, kv_num_blocks=B * max_blocks + 3,
                                  max_blocks_per_seq=max_blocks, seed=seed)
     eng = engine.SpecStep(sc)
     eng.load_target_weights(W)
-    eng.load_draft_weights(H)
+    if H is not None:
+        eng.load_draft_weights(H)
     order = inputs.make_block_order(sc.kv_num_blocks, inputs.sub_seed(1, 3))
     eng.seq_init(np.zeros(B, np.int32), prompts[:, 0], order)
     # the oracle's paged-KV bookkeeping runs alongside on host copies: integer state must match bit for bit
@@ -80,7 +83,7 @@ def run_chain(engine, cfg, kind, B, prompt_len, k, n_steps, seed):
         assert oracle.kv_reserve(k, 16, o_len, o_table, o_free, o_top) == 0
         check_books(eng.n_emitted().cpu().numpy())
         g_logits = eng.logits(k).cpu().numpy()
-        g_dlogits = eng.draft_logits(k).cpu().numpy()
+        g_dlogits = eng.draft_logits(k).cpu().numpy() if H is not None else None
         g_drafts = eng.draft_tokens().cpu().numpy()[:, :k]
         g_out = eng.out_tokens(k).cpu().numpy()
         g_n = eng.n_emitted().cpu().numpy()
@@ -97,8 +100,9 @@ def run_chain(engine, cfg, kind, B, prompt_len, k, n_steps, seed):
             if np.array_equal(rec["drafts"], g_drafts[b]):
                 max_rel = max(max_rel, float(np.max(np.abs(g_logits[b] - rec["target_logits"]).max(-1) /
                                                     np.abs(rec["target_logits"]).max(-1))))
-                max_rel_d = max(max_rel_d, float(np.max(np.abs(g_dlogits[b] - rec["draft_logits"]).max(-1) /
-                                                      np.abs(rec["draft_logits"]).max(-1))))
+                if H is not None:
+                    max_rel_d = max(max_rel_d, float(np.max(np.abs(g_dlogits[b] - rec["draft_logits"]).max(-1) /
+                                                          np.abs(rec["draft_logits"]).max(-1))))
             if not same:
                 mg = rec["margins"]
                 assert np.any(mg[:k] < 1e-4) or mg[k] < 1e-6 or not np.array_equal(rec["drafts"], g_drafts[b]), \
@@ -138,6 +142,17 @@ def test_tiny_chain_mtp_lockstep(eng_mod):
     r = run_chain(eng_mod, cfg, "mtp", B=3, prompt_len=30, k=2, n_steps=12, seed=5)
     print("tiny mtp:", r)
     assert r["max_rel"] < 1e-3 and r["max_rel_d"] < 1e-3 and r["boundary"] <= 2
+
+
+def test_chain_ngram_drafting_lockstep(eng_mod):
+    """Model-free drafting: proposals come from the sequence's own tokens, q is one-hot.  Periodic prompts make the first
+    lookups hit; later ones fall back to shorter n-grams or to repeating the last token."""
+    cfg = dict(inputs.model_config("c1"), ngram_n=3)
+    rng = np.random.default_rng(3)
+    prompts = np.stack([np.tile(rng.integers(0, 1024, 5 + b), 20)[:48] for b in range(4)]).astype(np.int32)
+    r = run_chain(eng_mod, cfg, "ngram", B=4, prompt_len=48, k=3, n_steps=16, seed=123, prompts=prompts)
+    print("ngram:", r)
+    assert r["max_rel"] < 1e-3 and r["boundary"] <= 1 and r["emitted"] >= r["steps"]
 
 
 def test_chain_at_other_temperature_and_k1(eng_mod):

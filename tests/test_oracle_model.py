@@ -200,3 +200,29 @@ def test_chain_oracle_emits_between_1_and_k_plus_1_tokens():
         qs.append(q)
     rec = ch2.step_once(3, forced_drafts=(drafts, np.stack(qs)))
     assert rec["n_emitted"] == 4
+
+
+def test_ngram_propose_worked_examples():
+    # trailing [1,2,3] last seen at positions 4..6, followed by 9, 1, 2, 3
+    assert model.ngram_propose([1, 2, 3, 4, 1, 2, 3, 9, 1, 2, 3], 3, 4).tolist() == [9, 1, 2, 3]
+    # the most recent earlier occurrence wins, not the first
+    assert model.ngram_propose([1, 2, 7, 1, 2, 8, 1, 2], 2, 1).tolist() == [8]
+    # no 3- or 2-gram match: falls back to the single token 5 (seen at position 0, followed by 6), then runs off the end
+    assert model.ngram_propose([5, 6, 5], 3, 3).tolist() == [6, 5, 5]
+    # nothing matches: repeat the last token
+    assert model.ngram_propose([5, 6, 7], 3, 3).tolist() == [7, 7, 7]
+    assert model.ngram_propose([7], 3, 2).tolist() == [7, 7]
+    # brute force on random short strings over a tiny alphabet: the proposal continues an occurrence of the longest matching suffix
+    rng = np.random.default_rng(0)
+    for _ in range(300):
+        t = rng.integers(0, 3, rng.integers(2, 12)).tolist()
+        d = model.ngram_propose(t, 3, 1)[0]
+        best = None
+        for n in (3, 2, 1):
+            if n > len(t) - 1:
+                continue
+            hits = [s for s in range(len(t) - n) if t[s : s + n] == t[len(t) - n :]]
+            if hits:
+                best = t[max(hits) + n]
+                break
+        assert d == (best if best is not None else t[-1])
