@@ -166,6 +166,19 @@ spec_status spec_tensor(spec_ctx* ctx, int tensor_id, int layer, void** dev_ptr,
 spec_status spec_seq_init(spec_ctx* ctx, int B, const int32_t* seq_len_host, const int32_t* last_token_host,
                           const int32_t* free_stack_host, void* stream);
 
+/* Replaces finished sequences between steps: rollout responses end at very different lengths (the long tail
+ * of Section 5.1) and a slot whose sequence is done takes the next prompt while the others keep decoding.
+ * For i = 0..n-1, in list order: every block of slot slots_host[i] returns to the free stack (logical
+ * order), blocks for seq_len_host[i] cached positions are popped (the caller fills them, or passes 0 and
+ * prefills through forced verify steps), its last token becomes last_token_host[i] and the draft head has
+ * no pending positions for it.  The step counter and the other slots are untouched, so their random
+ * streams continue.  Host arrays, n <= current batch; synchronises `stream`.
+ * Errors: STATE (between verify and commit), INVALID_ARG (slot out of range or twice, bad token), SHAPE;
+ * a free stack too small for the list leaves the state unchanged and sets the device status
+ * SPEC_ERR_KV_EXHAUSTED. */
+spec_status spec_seq_replace(spec_ctx* ctx, int n, const int32_t* slots_host, const int32_t* seq_len_host,
+                             const int32_t* last_token_host, void* stream);
+
 /* ---- one speculation step (Introduction, third paragraph) ------------------------------------------------- */
 
 /* S1 draft propose.  Runs the draft head: pass 0 consumes the (tapped hidden state, next token) pairs of the
@@ -192,7 +205,8 @@ spec_status spec_reject_sample(spec_ctx* ctx, int k, const float* draft_logits, 
 
 /* S5 KV commit / rollback: seq_len += n+1, blocks past the new length return to the free stack, the last
  * token becomes the emitted token, the step counter advances.  force_n / force_token ([B] each, both or
- * neither) replace the sampler's n and token: teacher-forced prefill through the verify path. */
+ * neither) replace the sampler's n and token: teacher-forced prefill through the verify path; a negative
+ * force_n[b] leaves sequence b to the sampler (a new prompt prefills while the other slots decode). */
 spec_status spec_kv_commit(spec_ctx* ctx, const int32_t* force_n, const int32_t* force_token, void* stream);
 
 /* Synchronises `stream`, reads the device status word and counters. */

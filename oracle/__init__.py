@@ -48,6 +48,8 @@ def lib():
         L.spec_oracle_kv_reserve.argtypes = [c.c_int, c.c_int, c.c_int, c.c_int, i32p, i32p, i32p, i32p]
         L.spec_oracle_kv_reserve.restype = c.c_int
         L.spec_oracle_kv_commit.argtypes = [c.c_int, c.c_int, c.c_int, i32p, i32p, i32p, i32p, i32p]
+        L.spec_oracle_kv_replace.argtypes = [c.c_int, i32p, i32p, c.c_int, c.c_int, i32p, i32p, i32p, i32p]
+        L.spec_oracle_kv_replace.restype = c.c_int
         _lib = L
     return _lib
 
@@ -172,3 +174,11 @@ def kv_commit(block_tokens, n_emitted, seq_len, block_table, free_stack, free_to
     lib().spec_oracle_kv_commit(B, block_tokens, max_blocks, _p(ne, ctypes.c_int32), _p(seq_len, ctypes.c_int32),
                                 _p(block_table, ctypes.c_int32), _p(free_stack, ctypes.c_int32),
                                 _p(free_top, ctypes.c_int32))
+
+
+def kv_replace(slots, new_len, block_tokens, seq_len, block_table, free_stack, free_top):
+    sl, nl = _i32(slots), _i32(new_len)
+    B, max_blocks = block_table.shape
+    return lib().spec_oracle_kv_replace(sl.shape[0], _p(sl, ctypes.c_int32), _p(nl, ctypes.c_int32), block_tokens, max_blocks,
+                                        _p(seq_len, ctypes.c_int32), _p(block_table, ctypes.c_int32),
+                                        _p(free_stack, ctypes.c_int32), _p(free_top, ctypes.c_int32))

@@ -28,7 +28,7 @@ struct spec_ctx {
     size_t kv_pool_bytes = 0, kv_bytes = 0, draft_kv_bytes = 0;
     // state
     Loc seq_len, last_token, block_table, free_stack, free_top, draft_tokens, out_tokens, n_emitted, status, step,
-        counters, pending_base, owned, out_logp, history;
+        counters, pending_base, owned, out_logp, history, replace_args;
     size_t state_bytes = 0;
     // workspace
     Loc tokens_in, pos, x, h, qkv, attn_out, gu, act, logits, draft_logits, row_stats, draft_row_stats, taps,
@@ -165,6 +165,7 @@ void build_layout(spec_ctx& x)
         x.owned = a.take(Bm * 4);
         x.out_logp = a.take(Bm * (c.k_max + 1) * 4);
         if (c.draft_kind == SPEC_DRAFT_NGRAM) x.history = a.take(Bm * (size_t)c.max_blocks_per_seq * c.kv_block_tokens * 4);
+        x.replace_args = a.take(3 * Bm * 4);
         x.state_bytes = a.top;
     }
     {
@@ -325,13 +326,16 @@ __global__ void draft_rows0_kernel(int B, int R, const int32_t* n_emitted, const
     tok[m] = valid ? out_tokens[m] : -1;
 }
 
-__global__ void draft_rows_kernel(int B, int j, const int32_t* seq_len, const int32_t* draft_tokens, int stride,
-                                  int32_t* tok, int32_t* pos)
+__global__ void draft_rows_kernel(int B, int j, const int32_t* seq_len, const int32_t* n_emitted, const int32_t* draft_tokens,
+                                  int stride, int32_t* tok, int32_t* pos)
 {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
-    pos[b] = seq_len[b] - 1 + j;
-    tok[b] = draft_tokens[(size_t)b * stride + j - 1];
+    // a slot that was just replaced has nothing committed to draft from: its rows are inert (zero hidden state, uniform
+    // q) until its first commit, and touch no cache slot
+    const bool fresh = n_emitted[b] == 0;
+    pos[b] = fresh ? -1 : seq_len[b] - 1 + j;
+    tok[b] = fresh ? -1 : draft_tokens[(size_t)b * stride + j - 1];
 }
 
 }  // namespace
@@ -493,6 +497,39 @@ extern "C" spec_status spec_seq_init(spec_ctx* c, int B, const int32_t* seq_len_
     return SPEC_OK;
 }
 
+extern "C" spec_status spec_seq_replace(spec_ctx* c, int n, const int32_t* slots_host, const int32_t* seq_len_host,
+                                        const int32_t* last_token_host, void* stream)
+{
+    if (c == nullptr || n < 0 || (n > 0 && (!slots_host || !seq_len_host || !last_token_host))) return SPEC_ERR_INVALID_ARG;
+    const spec_config& g = c->cfg;
+    if (c->verified) return fail(c, SPEC_ERR_STATE, "spec_seq_replace: a verified step is waiting for its commit");
+    if (n > c->B) return fail(c, SPEC_ERR_SHAPE, "spec_seq_replace: more slots listed than sequences running");
+    if (n == 0) return SPEC_OK;
+    const int bt = g.kv_block_tokens, mb = g.max_blocks_per_seq;
+    std::vector<char> seen(c->B, 0);
+    for (int i = 0; i < n; ++i) {
+        const int b = slots_host[i];
+        if (b < 0 || b >= c->B || seen[b]) return fail(c, SPEC_ERR_INVALID_ARG, "spec_seq_replace: a slot is out of range or listed twice");
+        seen[b] = 1;
+        if (seq_len_host[i] < 0 || last_token_host[i] < 0 || last_token_host[i] >= g.vocab) return SPEC_ERR_INVALID_ARG;
+        if ((seq_len_host[i] + g.k_max + 1 + bt - 1) / bt > mb)
+            return fail(c, SPEC_ERR_SHAPE, "spec_seq_replace: a sequence does not fit max_blocks_per_seq");
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    char* sb = static_cast<char*>(c->buf.state);
+    int32_t* args = at<int32_t>(sb, c->replace_args);
+    const size_t Bm = g.max_batch;
+    SPEC_CUDA_OK(cudaMemcpyAsync(args, slots_host, (size_t)n * 4, cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_OK(cudaMemcpyAsync(args + Bm, seq_len_host, (size_t)n * 4, cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_OK(cudaMemcpyAsync(args + 2 * Bm, last_token_host, (size_t)n * 4, cudaMemcpyHostToDevice, st));
+    TRY(launch_kv_replace(n, args, args + Bm, args + 2 * Bm, bt, mb, at<int32_t>(sb, c->seq_len), at<int32_t>(sb, c->last_token),
+                          at<int32_t>(sb, c->block_table), at<int32_t>(sb, c->owned), at<int32_t>(sb, c->free_stack),
+                          at<int32_t>(sb, c->free_top), at<int32_t>(sb, c->n_emitted), at<int32_t>(sb, c->pending_base),
+                          at<int32_t>(sb, c->status), st));
+    SPEC_CUDA_OK(cudaStreamSynchronize(st));          // the host lists may be reused by the caller from here on
+    return SPEC_OK;
+}
+
 extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_tokens, void* stream)
 {
     if (c == nullptr) return SPEC_ERR_INVALID_ARG;
@@ -638,7 +675,7 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
         float* res = j == 0 ? dg : hid;                 // residual stream of this pass
         if (j == 0) draft_rows0_kernel<<<(M + 255) / 256, 256, 0, st>>>(B, R, at<int32_t>(sb, c->n_emitted), at<int32_t>(sb, c->pending_base),
                                                                         at<int32_t>(sb, c->out_tokens), tok, pos);
-        else        draft_rows_kernel<<<(B + 255) / 256, 256, 0, st>>>(B, j, seq_len, dtoks, kstride, tok, pos);
+        else        draft_rows_kernel<<<(B + 255) / 256, 256, 0, st>>>(B, j, seq_len, at<int32_t>(sb, c->n_emitted), dtoks, kstride, tok, pos);
         TRY(launch_status());
         TRY(launch_rope_table(M, g.head_dim, g.rope_theta, pos, at<float>(ws, c->rope), st));
         TRY(launch_embed(M, d, at(c->buf.weights, c->embed), dt, tok, dx, st));

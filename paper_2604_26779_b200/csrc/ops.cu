@@ -192,10 +192,9 @@ __global__ void gather_last_rows_kernel(int R, int d, const float* __restrict__ 
 {
     const int b = blockIdx.x;
     const int r = n_valid[b] - 1;
-    if (r < 0) return;
     for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
-        float v[4];
-        Vec4<float>::load(src + ((size_t)b * R + r) * d + c, v);
+        float v[4] = {0.f, 0.f, 0.f, 0.f};                      // no valid row: a zero state, not a stale one
+        if (r >= 0) Vec4<float>::load(src + ((size_t)b * R + r) * d + c, v);
         Vec4<float>::store(dst + (size_t)b * d + c, v);
     }
 }
@@ -289,7 +288,7 @@ __global__ void __launch_bounds__(kBookThreads) kv_commit_kernel(const CommitArg
         int freed = 0, keep = 0;
         if (b < a.B) {
             int n1, last;
-            if (a.force_n != nullptr) {
+            if (a.force_n != nullptr && a.force_n[b] >= 0) {     // a negative entry leaves the sequence to the sampler
                 n1 = min(max(a.force_n[b], 0), a.k) + 1;
                 last = a.force_token[b];
                 // the committed tokens of a forced step are the verified inputs d_1..d_n followed by the given token
@@ -369,6 +368,33 @@ __global__ void __launch_bounds__(256) ngram_draft_kernel(int k, int n_max, cons
             prev = t;
         }
     }
+}
+
+// Slot replacement (finished sequences leave, new ones take their slots).  One thread, list order: the bookkeeping is a
+// few integers per sequence and must be deterministic.
+__global__ void kv_replace_kernel(int n, const int32_t* __restrict__ slots, const int32_t* __restrict__ new_len,
+                                  const int32_t* __restrict__ new_last, int bt, int max_blocks, int32_t* seq_len,
+                                  int32_t* last_token, int32_t* table, int32_t* owned, int32_t* free_stack, int32_t* free_top,
+                                  int32_t* n_emitted, int32_t* pending_base, int32_t* status)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int top = *free_top;
+    long avail = top, need = 0;
+    for (int i = 0; i < n; ++i) { avail += owned[slots[i]]; need += (new_len[i] + bt - 1) / bt; }
+    if (need > avail) { set_status(status, SPEC_ERR_KV_EXHAUSTED, -2); return; }
+    for (int i = 0; i < n; ++i) {
+        const int b = slots[i];
+        int32_t* row = table + (size_t)b * max_blocks;
+        for (int j = 0; j < owned[b]; ++j) { free_stack[top++] = row[j]; row[j] = -1; }
+        const int blocks = (new_len[i] + bt - 1) / bt;
+        for (int j = 0; j < blocks; ++j) row[j] = free_stack[--top];
+        owned[b] = blocks;
+        seq_len[b] = new_len[i];
+        last_token[b] = new_last[i];
+        n_emitted[b] = 0;                                       // nothing pending for the draft head
+        pending_base[b] = new_len[i];
+    }
+    *free_top = top;
 }
 
 }  // namespace
@@ -458,6 +484,17 @@ spec_status launch_ngram_draft(int B, int k, int n_max, const int32_t* history, 
 {
     if (B == 0) return SPEC_OK;
     ngram_draft_kernel<<<B, 256, 0, st>>>(k, n_max, history, max_hist, seq_len, last_token, draft_tokens, draft_stride);
+    return launch_status();
+}
+
+spec_status launch_kv_replace(int n, const int32_t* slots, const int32_t* new_len, const int32_t* new_last, int bt,
+                              int max_blocks, int32_t* seq_len, int32_t* last_token, int32_t* table, int32_t* owned,
+                              int32_t* free_stack, int32_t* free_top, int32_t* n_emitted,
+                              int32_t* pending_base, int32_t* status, cudaStream_t st)
+{
+    if (n == 0) return SPEC_OK;
+    kv_replace_kernel<<<1, 32, 0, st>>>(n, slots, new_len, new_last, bt, max_blocks, seq_len, last_token, table, owned,
+                                        free_stack, free_top, n_emitted, pending_base, status);
     return launch_status();
 }
 

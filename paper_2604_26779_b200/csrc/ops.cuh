@@ -61,6 +61,10 @@ struct CommitArgs {
     int32_t* status;
 };
 spec_status launch_kv_commit(const CommitArgs& a, cudaStream_t st);
+spec_status launch_kv_replace(int n, const int32_t* slots, const int32_t* new_len, const int32_t* new_last, int bt,
+                              int max_blocks, int32_t* seq_len, int32_t* last_token, int32_t* table, int32_t* owned,
+                              int32_t* free_stack, int32_t* free_top, int32_t* n_emitted,
+                              int32_t* pending_base, int32_t* status, cudaStream_t st);
 
 // model-free drafting: continue the most recent earlier occurrence of the trailing n-gram of (history[0..len), last token)
 spec_status launch_ngram_draft(int B, int k, int n_max, const int32_t* history, int max_hist, const int32_t* seq_len,

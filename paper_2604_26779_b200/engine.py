@@ -161,6 +161,14 @@ class SpecStep:
                                         B._stream(stream)), "spec_seq_init")
         self.B = sl.shape[0]
 
+    def seq_replace(self, slots, seq_len, last_token, stream=None):
+        sl = np.ascontiguousarray(slots, np.int32)
+        ln = np.ascontiguousarray(seq_len, np.int32)
+        lt = np.ascontiguousarray(last_token, np.int32)
+        assert sl.shape == ln.shape == lt.shape
+        B._check(self.lib.spec_seq_replace(self.ctx, sl.shape[0], sl.ctypes.data, ln.ctypes.data, lt.ctypes.data,
+                                           B._stream(stream)), "spec_seq_replace")
+
     def draft(self, k, stream=None):
         B._check(self.lib.spec_draft(self.ctx, k, B._stream(stream)), "spec_draft")
 

@@ -185,3 +185,113 @@ def test_kv_exhaustion_is_reported_not_faulted(eng_mod):
     eng.verify(3, forced)                      # needs 2 blocks per sequence, only 1 spare
     assert eng.status().device_status == -16
     eng.close()
+
+
+def test_slot_replacement_mid_run(eng_mod):
+    """A finished sequence's slot takes a new prompt between steps; the new prompt prefills through forced verify steps
+    while the other slots keep speculating, then joins them.  All slots stay in lock-step with their cache-free oracle
+    chains, and the block bookkeeping matches the oracle's bit for bit throughout."""
+    engine = eng_mod
+    cfg, kind, B, k, seed = inputs.model_config("c1"), "eagle3", 3, 3, 4242
+    R = k + 1
+    W = inputs.make_target_weights(cfg, seed=inputs.sub_seed(2, 0))
+    H = inputs.make_eagle3_weights(cfg, seed=inputs.sub_seed(2, 1))
+    prompts = inputs.make_prompts(B, 16, cfg["vocab"], seed=inputs.sub_seed(2, 2))
+    new_prompt = inputs.make_prompts(1, 12, cfg["vocab"], seed=inputs.sub_seed(2, 4))[0]
+    max_blocks = 8
+    sc = engine.make_spec_config(cfg, draft_kind=kind, k_max=k, max_batch=B, kv_num_blocks=18,
+                                 max_blocks_per_seq=max_blocks, seed=seed)
+    eng = engine.SpecStep(sc)
+    eng.load_target_weights(W)
+    eng.load_draft_weights(H)
+    order = inputs.make_block_order(sc.kv_num_blocks, inputs.sub_seed(2, 3))
+    eng.seq_init(np.zeros(B, np.int32), prompts[:, 0], order)
+    o_len, o_table = np.zeros(B, np.int32), np.full((B, max_blocks), -1, np.int32)
+    o_free, o_top = order.copy(), np.array([sc.kv_num_blocks], np.int32)
+
+    def books_equal():
+        assert np.array_equal(eng.seq_len().cpu().numpy(), o_len)
+        assert np.array_equal(eng.block_table().cpu().numpy(), o_table)
+        top = int(eng.tensor("FREE_TOP", 0, torch.int32, (1,)).item())
+        assert top == int(o_top[0])
+        assert np.array_equal(eng.tensor("FREE_STACK", 0, torch.int32, (sc.kv_num_blocks,)).cpu().numpy()[:top], o_free[:top])
+
+    def step(forced):
+        """One step; forced maps slot -> (k draft tokens, n, token).  Returns the device's results."""
+        have_pending = eng.status().steps > 0
+        if have_pending:
+            eng.draft(k)
+        drafts = eng.draft_tokens()[:, :k].clone().contiguous()
+        fn = torch.full((B,), -1, dtype=torch.int32)
+        ft = torch.zeros((B,), dtype=torch.int32)
+        for b, (d, n, t) in forced.items():
+            drafts[b] = torch.as_tensor(np.asarray(d, np.int32)).cuda()
+            fn[b], ft[b] = n, int(t)
+        eng.verify(k, drafts)
+        if len(forced) < B:
+            eng.reject_sample(k)
+        eng.kv_commit(fn.cuda(), ft.cuda())
+        assert eng.status().device_status == 0
+        assert oracle.kv_reserve(k, 16, o_len, o_table, o_free, o_top) == 0
+        n_dev = eng.n_emitted().cpu().numpy().copy()
+        oracle.kv_commit(16, n_dev, o_len, o_table, o_free, o_top)
+        books_equal()
+        for b, (d, n, t) in forced.items():
+            assert n_dev[b] == n + 1
+        return drafts.cpu().numpy(), eng.out_tokens(k).cpu().numpy().copy(), n_dev
+
+    def prefill_chunks(p):
+        chunks = []
+        for c in range(len(p) // R):
+            last = c == len(p) // R - 1
+            chunks.append((p[c * R + 1 : c * R + R], k - 1 if last else k, p[-1] if last else p[(c + 1) * R]))
+        return chunks
+
+    # all slots prefill together
+    for c in range(4):
+        step({b: prefill_chunks(prompts[b])[c] for b in range(B)})
+    chains = {b: ChainOracle(cfg, W, H, kind, seed, b, prompts[b], step0=4) for b in range(B)}
+    tokens = {b: list(map(int, prompts[b])) for b in range(B)}
+    boundary = 0
+
+    def lockstep(slots, forced):
+        nonlocal boundary
+        g_drafts, g_out, g_n = step(forced)
+        for b in slots:
+            rec = chains[b].step_once(k)
+            same = (np.array_equal(rec["drafts"], g_drafts[b]) and rec["n_emitted"] == g_n[b]
+                    and np.array_equal(rec["out_tokens"], g_out[b]))
+            if not same:
+                mg = rec["margins"]
+                assert np.any(mg[:k] < 1e-4) or mg[k] < 1e-6 or not np.array_equal(rec["drafts"], g_drafts[b]), (b, rec, g_out[b])
+                boundary += 1
+            tokens[b] += [int(t) for t in g_out[b, : g_n[b]]]
+            chains[b].tokens = list(tokens[b])
+
+    for _ in range(5):
+        lockstep(range(B), {})
+    # slot 1 is done: it takes the new prompt; its blocks go back and come out again in the oracle's order
+    eng.seq_replace([1], [0], [int(new_prompt[0])])
+    assert oracle.kv_replace([1], [0], 16, o_len, o_table, o_free, o_top) == 0
+    books_equal()
+    assert eng.status().device_status == 0
+    for chunk in prefill_chunks(new_prompt):
+        lockstep([0, 2], {1: chunk})
+    assert int(eng.seq_len()[1].item()) == len(new_prompt) - 1
+    chains[1] = ChainOracle(cfg, W, H, kind, seed, 1, new_prompt, step0=chains[0].step)
+    tokens[1] = list(map(int, new_prompt))
+    for _ in range(6):
+        lockstep(range(B), {})
+    for b in range(B):
+        assert int(eng.seq_len()[b].item()) == len(tokens[b]) - 1
+    print("slot replacement: boundary cases", boundary)
+    assert boundary <= 2
+    # a list the free stack cannot serve leaves the state alone and is reported
+    eng.seq_replace([0, 2], [16 * (max_blocks - 1) - 4, 16 * (max_blocks - 1) - 4], [1, 1])
+    assert oracle.kv_replace([0, 2], [16 * (max_blocks - 1) - 4] * 2, 16, o_len, o_table, o_free, o_top) == 0
+    books_equal()
+    eng.seq_replace([1], [16 * (max_blocks - 1) - 4], [1])          # 7 blocks wanted, 4 left even with its own back
+    assert oracle.kv_replace([1], [16 * (max_blocks - 1) - 4], 16, o_len, o_table, o_free, o_top) == -1
+    assert eng.status().device_status == -16
+    books_equal()
+    eng.close()

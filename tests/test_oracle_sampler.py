@@ -377,6 +377,25 @@ def test_kv_reserve_commit_conserves_blocks():
     assert oracle.kv_reserve(k, bt, seq_len, t2, free, top2) == -1 and np.all(t2 == -1)
 
 
+def test_kv_replace_returns_and_reissues_blocks():
+    """Worked by hand: stack [5,4,3,2,1,0] (top last); A holds [0,1], B holds [2]; replacing A by a 40-token sequence
+    pushes 0 then 1 (stack [5,4,3,0,1]) and pops 1, 0, 3 in that order."""
+    bt, maxb = 16, 4
+    seq_len = np.array([20, 7], np.int32)
+    table = np.array([[0, 1, -1, -1], [2, -1, -1, -1]], np.int32)
+    free = np.array([5, 4, 3, 9, 9, 9], np.int32)
+    top = np.array([3], np.int32)
+    assert oracle.kv_replace([0], [40], bt, seq_len, table, free, top) == 0
+    assert table.tolist() == [[1, 0, 3, -1], [2, -1, -1, -1]] and seq_len.tolist() == [40, 7] and top[0] == 2
+    assert free[:2].tolist() == [5, 4]
+    # an empty replacement only returns blocks; asking for more than exist changes nothing
+    assert oracle.kv_replace([1], [0], bt, seq_len, table, free, top) == 0
+    assert table[1].tolist() == [-1] * 4 and top[0] == 3 and free[:3].tolist() == [5, 4, 2] and seq_len[1] == 0
+    before = (seq_len.copy(), table.copy(), free.copy(), top.copy())
+    assert oracle.kv_replace([1], [64], bt, seq_len, table, free, top) == -1
+    assert all(np.array_equal(a, b) for a, b in zip(before, (seq_len, table, free, top)))
+
+
 # ---- the paper's reporting formula (Section 2.2) against its own tables ---------------------------------------
 
 def test_amdahl_bound_against_paper_tables(golden_dir):
