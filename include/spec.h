@@ -171,7 +171,9 @@ spec_status spec_seq_init(spec_ctx* ctx, int B, const int32_t* seq_len_host, con
  * For i = 0..n-1, in list order: every block of slot slots_host[i] returns to the free stack (logical
  * order), blocks for seq_len_host[i] cached positions are popped (the caller fills them, or passes 0 and
  * prefills through forced verify steps), its last token becomes last_token_host[i] and the draft head has
- * no pending positions for it.  The step counter and the other slots are untouched, so their random
+ * no pending positions for it.  seq_len_host[i] < 0 retires the slot instead (no prompt left): it keeps
+ * no block, its rows of later steps are inert (no cache access, nothing emitted: N_EMITTED 0, SEQ_LEN -1)
+ * until it is replaced again.  The step counter and the other slots are untouched, so their random
  * streams continue.  Host arrays, n <= current batch; synchronises `stream`.
  * Errors: STATE (between verify and commit), INVALID_ARG (slot out of range or twice, bad token), SHAPE;
  * a free stack too small for the list leaves the state unchanged and sets the device status

@@ -247,12 +247,14 @@ int spec_oracle_kv_reserve(int B, int k, int block_tokens, int max_blocks, const
 {
     long need_total = 0;
     for (int b = 0; b < B; ++b) {
+        if (seq_len[b] < 0) continue;                      /* retired slot */
         int need = (seq_len[b] + k + 1 + block_tokens - 1) / block_tokens;
         if (need > max_blocks) return -2;
         for (int j = 0; j < need; ++j) if (block_table[(size_t)b * max_blocks + j] < 0) need_total += 1;
     }
     if (need_total > *free_top) return -1;
     for (int b = 0; b < B; ++b) {
+        if (seq_len[b] < 0) continue;
         int need = (seq_len[b] + k + 1 + block_tokens - 1) / block_tokens;
         for (int j = 0; j < need; ++j) {
             int32_t* e = &block_table[(size_t)b * max_blocks + j];
@@ -266,6 +268,7 @@ void spec_oracle_kv_commit(int B, int block_tokens, int max_blocks, const int32_
                            int32_t* seq_len, int32_t* block_table, int32_t* free_stack, int32_t* free_top)
 {
     for (int b = 0; b < B; ++b) {
+        if (seq_len[b] < 0) continue;                      /* retired slot: holds nothing, commits nothing */
         seq_len[b] += n_emitted[b];
         int keep = (seq_len[b] + block_tokens - 1) / block_tokens;
         for (int j = keep; j < max_blocks; ++j) {
@@ -277,23 +280,25 @@ void spec_oracle_kv_commit(int B, int block_tokens, int max_blocks, const int32_
 
 /* replace: sequences finish at different lengths (the long tail of response lengths, Section 5.1) and their slots are
  * refilled.  For every listed slot, in list order: all its blocks go back to the free stack (logical order), then blocks
- * for new_len[i] cached positions are popped.  Returns -1 (nothing changed) if the stack cannot serve the list. */
+ * for new_len[i] cached positions are popped.  new_len[i] < 0 retires the slot: it keeps no block, its length stays -1
+ * and reserve / commit pass it over until it is replaced again.  Returns -1 (nothing changed) if the stack cannot
+ * serve the list. */
 int spec_oracle_kv_replace(int n, const int32_t* slots, const int32_t* new_len, int block_tokens, int max_blocks,
                            int32_t* seq_len, int32_t* block_table, int32_t* free_stack, int32_t* free_top)
 {
     long avail = *free_top, need = 0;
     for (int i = 0; i < n; ++i) {
         for (int j = 0; j < max_blocks; ++j) if (block_table[(size_t)slots[i] * max_blocks + j] >= 0) avail += 1;
-        need += (new_len[i] + block_tokens - 1) / block_tokens;
+        need += new_len[i] < 0 ? 0 : (new_len[i] + block_tokens - 1) / block_tokens;
     }
     if (need > avail) return -1;
     for (int i = 0; i < n; ++i) {
         int32_t* row = block_table + (size_t)slots[i] * max_blocks;
         for (int j = 0; j < max_blocks; ++j)
             if (row[j] >= 0) { free_stack[*free_top] = row[j]; *free_top += 1; row[j] = -1; }
-        int blocks = (new_len[i] + block_tokens - 1) / block_tokens;
+        int blocks = new_len[i] < 0 ? 0 : (new_len[i] + block_tokens - 1) / block_tokens;
         for (int j = 0; j < blocks; ++j) { *free_top -= 1; row[j] = free_stack[*free_top]; }
-        seq_len[slots[i]] = new_len[i];
+        seq_len[slots[i]] = new_len[i] < 0 ? -1 : new_len[i];
     }
     return 0;
 }

@@ -511,7 +511,8 @@ extern "C" spec_status spec_seq_replace(spec_ctx* c, int n, const int32_t* slots
         const int b = slots_host[i];
         if (b < 0 || b >= c->B || seen[b]) return fail(c, SPEC_ERR_INVALID_ARG, "spec_seq_replace: a slot is out of range or listed twice");
         seen[b] = 1;
-        if (seq_len_host[i] < 0 || last_token_host[i] < 0 || last_token_host[i] >= g.vocab) return SPEC_ERR_INVALID_ARG;
+        if (seq_len_host[i] < 0) continue;                  // retire: the slot stays empty until it is replaced again
+        if (last_token_host[i] < 0 || last_token_host[i] >= g.vocab) return SPEC_ERR_INVALID_ARG;
         if ((seq_len_host[i] + g.k_max + 1 + bt - 1) / bt > mb)
             return fail(c, SPEC_ERR_SHAPE, "spec_seq_replace: a sequence does not fit max_blocks_per_seq");
     }

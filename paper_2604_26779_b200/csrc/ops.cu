@@ -44,6 +44,7 @@ __global__ void verify_rows_kernel(int B, int R, const int32_t* seq_len, const i
     const int m = blockIdx.x * blockDim.x + threadIdx.x;
     if (m >= B * R) return;
     const int b = m / R, i = m % R;
+    if (seq_len[b] < 0) { rows.token[m] = 0; rows.pos[m] = -1; return; }     // retired slot: inert rows, no cache access
     int tok = (i == 0) ? last_token[b] : draft[(size_t)b * draft_stride + i - 1];
     if (tok < 0 || tok >= vocab) { set_status(status, SPEC_ERR_TOKEN_RANGE, b); tok = 0; }
     rows.token[m] = tok;
@@ -245,7 +246,7 @@ __global__ void __launch_bounds__(kBookThreads) kv_reserve_kernel(int B, int k, 
     for (int base = 0; base < B; base += kBookThreads) {
         const int b = base + threadIdx.x;
         int need_new = 0;
-        if (b < B) {
+        if (b < B && seq_len[b] >= 0) {                           // a retired slot (negative length) asks for nothing
             const int need = (seq_len[b] + k + 1 + bt - 1) / bt;
             if (need > max_blocks) { s_fail = 1; set_status(status, SPEC_ERR_KV_EXHAUSTED, b); }
             else need_new = max(0, need - owned[b]);
@@ -261,7 +262,7 @@ __global__ void __launch_bounds__(kBookThreads) kv_reserve_kernel(int B, int k, 
     for (int base = 0; base < B; base += kBookThreads) {
         const int b = base + threadIdx.x;
         int need = 0, have = 0;
-        if (b < B) { need = (seq_len[b] + k + 1 + bt - 1) / bt; have = owned[b]; }
+        if (b < B && seq_len[b] >= 0) { need = (seq_len[b] + k + 1 + bt - 1) / bt; have = owned[b]; }
         int tot;
         int off = carry + block_exclusive_scan(max(0, need - have), &tot, s_warp);
         if (b < B && need > have) {
@@ -286,7 +287,10 @@ __global__ void __launch_bounds__(kBookThreads) kv_commit_kernel(const CommitArg
     for (int base = 0; base < a.B; base += kBookThreads) {
         const int b = base + threadIdx.x;
         int freed = 0, keep = 0;
-        if (b < a.B) {
+        if (b < a.B && a.seq_len[b] < 0) {                       // retired slot: nothing emitted, nothing kept
+            a.n_emitted[b] = 0;
+            for (int i = 0; i < R; ++i) a.out_tokens[(size_t)b * R + i] = -1;
+        } else if (b < a.B) {
             int n1, last;
             if (a.force_n != nullptr && a.force_n[b] >= 0) {     // a negative entry leaves the sequence to the sampler
                 n1 = min(max(a.force_n[b], 0), a.k) + 1;
@@ -380,19 +384,19 @@ __global__ void kv_replace_kernel(int n, const int32_t* __restrict__ slots, cons
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     int top = *free_top;
     long avail = top, need = 0;
-    for (int i = 0; i < n; ++i) { avail += owned[slots[i]]; need += (new_len[i] + bt - 1) / bt; }
+    for (int i = 0; i < n; ++i) { avail += owned[slots[i]]; need += new_len[i] < 0 ? 0 : (new_len[i] + bt - 1) / bt; }
     if (need > avail) { set_status(status, SPEC_ERR_KV_EXHAUSTED, -2); return; }
     for (int i = 0; i < n; ++i) {
         const int b = slots[i];
         int32_t* row = table + (size_t)b * max_blocks;
         for (int j = 0; j < owned[b]; ++j) { free_stack[top++] = row[j]; row[j] = -1; }
-        const int blocks = (new_len[i] + bt - 1) / bt;
+        const int blocks = new_len[i] < 0 ? 0 : (new_len[i] + bt - 1) / bt;      // negative: the slot is retired
         for (int j = 0; j < blocks; ++j) row[j] = free_stack[--top];
         owned[b] = blocks;
-        seq_len[b] = new_len[i];
+        seq_len[b] = new_len[i] < 0 ? -1 : new_len[i];
         last_token[b] = new_last[i];
         n_emitted[b] = 0;                                       // nothing pending for the draft head
-        pending_base[b] = new_len[i];
+        pending_base[b] = new_len[i] < 0 ? 0 : new_len[i];
     }
     *free_top = top;
 }

@@ -1,6 +1,7 @@
 """Host-side logic of the library that needs no device: configuration checks, arena sizing, tensor placement."""
 import ctypes as C
 
+import numpy as np
 import pytest
 
 from paper_2604_26779_b200 import binding as B, engine, inputs
@@ -82,3 +83,26 @@ def test_create_checks_pointers_and_tensors_do_not_overlap():
     assert L.spec_verify(h, 9, None, None) == -2 and b"k outside" in L.spec_last_error(h)
     assert L.spec_tensor(h, 9999, 0, C.byref(C.c_void_p()), C.byref(C.c_size_t())) == -1
     assert L.spec_destroy(h) == 0
+
+
+def test_k_policy_arithmetic():
+    """Expected tokens per step under independent acceptance is the geometric sum; the chosen k is the brute-force best."""
+    from paper_2604_26779_b200 import rollout
+    for a in (0.0, 0.3, 0.8, 1.0):
+        for k in (0, 1, 3, 7):
+            assert abs(rollout.expected_tokens_per_step(a, k) - sum(a ** i for i in range(k + 1))) < 1e-12
+    # Monte Carlo check of the same quantity: the accepted prefix of k Bernoulli(a) trials plus one token
+    rng = np.random.default_rng(0)
+    acc = rng.random((200000, 5)) < 0.6
+    n = np.where(acc.all(1), 5, np.argmin(acc, 1))
+    assert abs((n + 1).mean() - rollout.expected_tokens_per_step(0.6, 5)) < 0.02
+    assert rollout.acceptance_rate(30, 50) == 0.6 and rollout.acceptance_rate(0, 0) == 0.0
+    # cost linear in rows: a thin batch prefers long drafts, a full one short drafts
+    cost = lambda B, k: 10.0 + 0.05 * B * (k + 1)
+    assert rollout.choose_k(0.7, 4, cost, range(1, 8)) == 7
+    assert rollout.choose_k(0.7, 2048, cost, range(1, 8)) <= 2
+    for a in (0.2, 0.5, 0.9):
+        for B in (1, 64, 1024):
+            ks = list(range(1, 8))
+            rates = [rollout.expected_tokens_per_step(a, k) / cost(B, k) for k in ks]
+            assert rollout.choose_k(a, B, cost, ks) == ks[int(np.argmax(rates))]
