@@ -139,6 +139,48 @@ def cpu_oracle_sample(eng, info, k, n_layers_sample, step_index):
                 fetch_seconds=t_fetch_head)
 
 
+def controlled_acceptance(eng, k, temperature, taus, n_steps, stream):
+    """Harness-only mode (flagged synthetic_q): the draft head is bypassed and the drafts are built the way the sampler
+    micro-benchmark builds them, q_i = softmax(target logits of position i + N(0, tau^2)), d_i ~ q_i, so that verify +
+    sample + commit can be timed at acceptance rates that bracket a trained draft's.  Position i's target logits depend
+    on d_1..d_{i-1}, so each step needs k untimed dry-run verifies to build a consistent draft; only the final verify,
+    the sampler and the commit are timed."""
+    import math
+    import torch
+    B, V = eng.B, eng.sc.vocab
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(2604026779 + 7)
+    out = []
+    for tau in taus:
+        ms, emitted, accepted = [], 0, 0
+        for _ in range(n_steps):
+            drafts = torch.zeros((B, k), dtype=torch.int32, device="cuda")
+            ql = torch.empty((B, k, V), dtype=torch.float32, device="cuda")
+            for i in range(k):
+                eng.verify(k, drafts)                                   # rows 0..i are final given d_1..d_i
+                ql[:, i] = eng.logits(k)[:, i] + tau * torch.randn((B, V), device="cuda", generator=gen)
+                probs = torch.softmax(ql[:, i] / temperature, -1)
+                drafts[:, i] = torch.multinomial(probs, 1, generator=gen)[:, 0].to(torch.int32)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            eng.verify(k, drafts)
+            eng.reject_sample(k, ql)
+            eng.kv_commit()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms.append(a.elapsed_time(b))
+            n = eng.n_emitted()
+            emitted += int(n.sum().item())
+            accepted += int((n - 1).sum().item())
+        med = float(np.median(ms))
+        al = emitted / float(n_steps * B)
+        out.append({"tau": tau, "acceptance_expected_2Phi(-tau/2)": math.erfc(tau / 2 / math.sqrt(2.0)),
+                    "acceptance_length": al, "accepted_drafts_per_step": accepted / float(n_steps * B),
+                    "ms_verify_sample_commit_median": med, "tokens_per_s": al * B / (med / 1000.0), "steps": n_steps})
+    return out
+
+
 def run_sampler_microbench(args):
     """Rejection-sampling micro-benchmark (B=1024, V=151936, k in {1,3,5,7}; target logits N(0, sigma^2), draft = target +
     N(0, tau^2)): the stateless sampler on given fp32 probabilities, and the fused from-logits path (row statistics +
@@ -252,7 +294,7 @@ def main():
 
     from paper_2604_26779_b200 import binding, replicas, workloads
     k, B = args.k, args.batch
-    steps_budget = args.steps * 2 + args.warmup * 2 + 24
+    steps_budget = args.steps * 2 + args.warmup * 2 + 48
     ext_drafts = None
     if args.workload == "c3":
         eng, info = workloads.build_dense_workload("c3", B=B, k=k, n_layers=args.layers, kv_pools=args.kv_pools,
@@ -429,6 +471,11 @@ def main():
                           "gemm_tflops_in_step": gemm_flops_per_step(cfg, B, k, info["draft"]) / (tm.ms[1] / 2 * 1e-3) / 1e12,
                           "gemm_frac_of_measured_sustained_bf16": gemm_flops_per_step(cfg, B, k, info["draft"]) / (tm.ms[1] / 2 * 1e-3) / 1e12 / tf_peak,
                           }
+
+        if args.workload == "c3":
+            line["extras"]["controlled_acceptance_synthetic_q"] = controlled_acceptance(
+                eng, k, float(cfg.get("temperature", 1.0)), (0.1, 0.5, 1.0), 5, stream)
+            assert eng.status().device_status == 0
 
     # ---- end-to-end through the C ABI with host buffers: seq_init from host arrays (H2D) + K steps, each followed by a
     # device-to-host read of the step's result (emitted tokens and counts) into pinned memory ---------------------------

@@ -77,6 +77,28 @@ def test_uniforms_bit_exact(api):
         assert np.array_equal(u.cpu().numpy(), oracle.uniforms(seed, step, tag, 50000, 20))
 
 
+def test_uniforms_match_curand_device_philox(api):
+    """Both the library's and the oracle's uniforms equal (word >> 8) * 2^-24 of cuRAND's own Philox4x32-10 on 1e6
+    counters: an implementation neither shares code with."""
+    import ctypes
+    import os
+    import __graft_entry__ as entry
+    helper = ctypes.CDLL(entry.build_test_helpers())
+    helper.curand_philox_words.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_int, ctypes.c_int,
+                                           ctypes.c_void_p]
+    n_seq, n_slots = 50000, 20
+    words = torch.zeros((n_seq, n_slots), dtype=torch.int32, device="cuda")
+    u = torch.zeros((n_seq, n_slots), dtype=torch.float32, device="cuda")
+    for step, tag, seed in [(0, 0, inputs.BASE_SEED), (7, 1, 0xFEDCBA9876543210), (4000000000, 0, 3)]:
+        torch.cuda.synchronize()
+        assert helper.curand_philox_words(seed, step, tag, n_seq, n_slots, words.data_ptr()) == 0
+        w = words.cpu().numpy().view(np.uint32)
+        ref = ((w >> 8).astype(np.float64) * 2.0 ** -24).astype(np.float32)
+        api.spec_uniforms(seed, step, tag, u)
+        assert np.array_equal(u.cpu().numpy(), ref)
+        assert np.array_equal(oracle.uniforms(seed, step, tag, n_seq, n_slots), ref)
+
+
 @pytest.mark.parametrize("V,T", [(8, 1.0), (1000, 0.7), (1027, 1.0), (151936, 1.0), (128256, 2.0)])
 def test_softmax_probabilities_and_stats(api, V, T):
     rng = np.random.default_rng(V)
