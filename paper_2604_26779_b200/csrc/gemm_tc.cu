@@ -273,9 +273,15 @@ __device__ __forceinline__ bool tile_coord(const GemmArgs& g, int w, int m_tiles
     t.kb0 = 0; t.kb1 = kb_count;
     int split = 0;
     if (g.splits > 1) { split = w % g.splits; w /= g.splits; t.kb0 = split * g.kb_per; t.kb1 = min(kb_count, t.kb0 + g.kb_per); }
-    const int mt = w % m_tiles, nt = (w / m_tiles) % n_tiles;
+    int mt = w % m_tiles, nt = (w / m_tiles) % n_tiles;
     if (g.E > 0) {
-        const int e = w / (m_tiles * n_tiles);
+        // grouped: m-tile index slowest.  Most groups fill only their first m-tile, so the non-empty items are the first
+        // E * n_tiles ones and the round-robin over CTAs spreads them evenly (with the m-tile fastest, a stride of 148
+        // would hand every non-empty item to a quarter of the CTAs)
+        const int per = n_tiles * g.E, rem = w % per;
+        mt = w / per;
+        nt = rem % n_tiles;
+        const int e = rem / n_tiles;
         const int cnt = g.counts[e];
         if (mt * BM >= cnt) return false;
         const int off = g.offsets[e];
