@@ -3,7 +3,7 @@
 //
 // This file holds the plain SIMT kernel (any element type, any head shape): the reference-precision path of fp32
 // models and the fallback for shapes the tensor-core kernel does not take.
-#include "ops.cuh"
+#include "attention_plan.cuh"
 
 namespace spec {
 namespace {
@@ -95,6 +95,7 @@ spec_status launch_attention_simt(const AttnArgs& a, cudaStream_t st)
 
 spec_status launch_attention(const AttnArgs& a, cudaStream_t st)
 {
+    if (attn::attention_tc_supported(a)) return attn::launch_attention_tc(a, st);
     if (attention_mma_supported(a)) return launch_attention_mma(a, st);
     return launch_attention_simt(a, st);
 }

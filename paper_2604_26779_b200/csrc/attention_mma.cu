@@ -9,29 +9,14 @@
 // ldmatrix (transposed for V), softmax is online in fp32 (exp2 domain), and units of one sequence are merged by a
 // log-sum-exp kernel (skipped for single-chunk sequences, which write their output directly).
 // Causality among the new rows: row (i, head j) sees cache positions <= pos[b*R + i].
-#include "ops.cuh"
+#include "attention_plan.cuh"
 
 namespace spec {
+using namespace attn;
 namespace {
 
-constexpr int kChunk = 4096;        // KV tokens per unit (upper bound); 4096 measured 3 % faster than 2048 and 1 % faster than 8192
-constexpr int kTileTok = 64;        // tokens per pipeline stage
-constexpr int kBT = 16;             // tokens per KV block
 constexpr int kThreads = 128;
 constexpr int kPlanThreads = 1024;
-constexpr int kCounters = 64;
-
-struct Unit { int b, t0, t1, slot; };      // slot: index of this (sequence, chunk) among all; -1 when the sequence has one chunk
-
-struct PlanView {                    // carved out of the scratch buffer
-    int* counters;                   // [kCounters] work counters, one per launch index
-    int* n_entries;                  // [1]
-    int* first;                      // [B] first entry of the sequence
-    int* nc;                         // [B] number of chunks of the sequence
-    Unit* entries;                   // [B * max_chunks]
-    float* part_o;                   // [entries * Hkv][rows][dh]
-    float* part_ml;                  // [entries * Hkv][rows][2]
-};
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes)
@@ -422,31 +407,34 @@ bool attention_mma_supported(const AttnArgs& a)
 
 size_t attention_mma_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int max_kv_len)
 {
-    const int rows = R * (Hq / Hkv);
-    const int rows_alloc = rows <= 16 ? 16 : rows <= 32 ? 32 : 64;
-    const int max_chunks = (max_kv_len + kTileTok + kChunk - 1) / kChunk + 1;
-    const size_t entries = (size_t)B * max_chunks;
+    const int rows_alloc = rows_alloc_for(R * (Hq / Hkv));
+    const size_t entries = (size_t)B * max_chunks_for(max_kv_len);
     return align_up((size_t)kCounters * 4 + 4, 256) + 2 * align_up((size_t)B * 4, 256) + align_up(entries * sizeof(Unit), 256) +
            align_up(entries * Hkv * rows_alloc * dh * 4, 256) + align_up(entries * Hkv * rows_alloc * 8, 256);
+}
+
+spec_status attn::launch_attn_plan(int B, int R, const int32_t* pos, int max_chunks, const PlanView& pv, cudaStream_t st)
+{
+    attn_plan_kernel<<<1, kPlanThreads, 0, st>>>(B, R, pos, max_chunks, pv);
+    return launch_status();
+}
+
+spec_status attn::launch_attn_merge128(int B, int rows_alloc, int Hkv, int R, int group, void* out, int out_row_stride,
+                                       const PlanView& pv, cudaStream_t st)
+{
+    MmaArgs m{};
+    m.R = R; m.group = group; m.Hkv = Hkv; m.out = static_cast<__nv_bfloat16*>(out); m.out_row_stride = out_row_stride; m.pv = pv;
+    attn_merge_kernel<128><<<B * Hkv, 128, 0, st>>>(B, rows_alloc, m);
+    return launch_status();
 }
 
 spec_status launch_attention_mma(const AttnArgs& a, cudaStream_t st)
 {
     const int group = a.Hq / a.Hkv, rows = a.R * group;
-    const int rows_alloc = rows <= 16 ? 16 : rows <= 32 ? 32 : 64;
-    const int max_chunks = (a.max_kv_len + kTileTok + kChunk - 1) / kChunk + 1;
+    const int rows_alloc = rows_alloc_for(rows);
+    const int max_chunks = max_chunks_for(a.max_kv_len);
     if (a.scratch_bytes < attention_mma_scratch_bytes(a.B, a.R, a.Hq, a.Hkv, a.dh, a.max_kv_len)) return SPEC_ERR_SHAPE;
-    const size_t entries = (size_t)a.B * max_chunks;
-    char* p = static_cast<char*>(a.scratch);
-    PlanView pv;
-    pv.counters = reinterpret_cast<int*>(p);
-    pv.n_entries = pv.counters + kCounters;
-    p += align_up((size_t)kCounters * 4 + 4, 256);
-    pv.first = reinterpret_cast<int*>(p); p += align_up((size_t)a.B * 4, 256);
-    pv.nc = reinterpret_cast<int*>(p); p += align_up((size_t)a.B * 4, 256);
-    pv.entries = reinterpret_cast<Unit*>(p); p += align_up(entries * sizeof(Unit), 256);
-    pv.part_o = reinterpret_cast<float*>(p); p += align_up(entries * a.Hkv * rows_alloc * a.dh * 4, 256);
-    pv.part_ml = reinterpret_cast<float*>(p);
+    const PlanView pv = carve_plan(a.scratch, a.B, a.Hkv, rows_alloc, a.dh, max_chunks);
     MmaArgs m{(const __nv_bfloat16*)a.q, a.q_row_stride, (const __nv_bfloat16*)a.k_pool, (const __nv_bfloat16*)a.v_pool,
               a.block_table, a.max_blocks, a.pos, a.R, group, a.Hkv, (__nv_bfloat16*)a.out, a.out_row_stride,
               1.4426950408889634f / sqrtf((float)a.dh), pv, a.launch_index % kCounters};

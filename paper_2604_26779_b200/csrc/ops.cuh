@@ -114,6 +114,7 @@ struct AttnArgs {
     void* scratch; size_t scratch_bytes;
     int max_kv_len;
     int launch_index;                  // 0 plans the work units; later launches of the same step reuse the plan
+    int32_t* status = nullptr;         // device status word for kernels with bounded waits (may be null)
 };
 spec_status launch_attention(const AttnArgs& a, cudaStream_t st);
 size_t attention_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int max_kv_len);

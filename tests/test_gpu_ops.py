@@ -56,6 +56,9 @@ def paged_case(lens, R, Hq, Hkv, dh, dtype, seed):
     ([64, 777, 2500], 5, 16, 4, 128, torch.bfloat16),                                  # k = 4: 20 rows -> two row tiles
     ([10, 300, 2100], 8, 8, 2, 128, torch.bfloat16),                                   # k = 7: 32 rows
     ([50, 1234], 4, 32, 2, 128, torch.bfloat16),                                       # group 16: 64 rows (MoE layer shape)
+    ([0, 7, 127, 128, 129, 4093, 4100, 9001], 4, 32, 2, 128, torch.bfloat16),          # 64 rows, tile edges, several chunks
+    ([33, 640, 5000], 8, 32, 2, 128, torch.bfloat16),                                  # k = 7 on a 16-head group: 128 rows
+    ([100, 3000], 17, 2, 2, 128, torch.bfloat16),                                      # 17 rows: just past the 16-row kernel
     ([5, 130, 2300], 4, 8, 4, 64, torch.bfloat16),                                     # head_dim 64
     ([0, 9, 40, 333], 4, 4, 4, 64, torch.float32),                                     # fp32 reference path
 ])
