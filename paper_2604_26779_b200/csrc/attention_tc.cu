@@ -6,13 +6,14 @@
 // its operands from shared memory once per tile whatever M is:
 //   - work units (sequence, KV head, chunk of <= 4096 tokens) come from the same plan and atomic counter as the
 //     register-fragment kernel; one persistent CTA per SM;
-//   - warp 0 pulls units and streams their K and V tiles of 128 tokens with TMA straight from the paged pools: one
-//     64-column x 16-row box per (block, half of head_dim), 128-byte swizzle, so a tile lands as [half][token][64] -
-//     K-major for S = Q K^T and MN-major for O += P V - in two 2-stage rings (K and V are released separately);
+//   - warp 0 pulls units and streams their K tiles of 128 tokens with TMA straight from the paged pool, warp 6 the V
+//     tiles: one 64-column x 16-row box per (block, half of head_dim), 128-byte swizzle, so a tile lands as
+//     [half][token][64] - K-major for S = Q K^T and MN-major for O += P V - in two 2-stage rings;
 //   - warp 1 issues the MMAs from one thread: S (128 x 128, fp32) into one of two tensor-memory buffers, O (128 x 128)
 //     accumulated in a third;
-//   - warps 2..5 are the softmax: thread = query row = tensor-memory lane (rows are dealt round-robin over the four
-//     32-lane quarters so that few rows still use all four warps).  Row maximum and exponentials in the exp2 domain; the
+//   - warps 2..5 are the softmax; query rows are dealt round-robin over the four 32-lane quarters of tensor memory and
+//     the scores are read in the 16-lane fragment shape, so the 32 threads of a warp share the columns of 16 rows (the
+//     exponentials, 4 per clock and scheduler whatever the number of active lanes, are what a tile costs).  Row maximum and exponentials in the exp2 domain; the
 //     running maximum is only raised when a tile exceeds it by more than 2^8 (the accumulator and the row sum are then
 //     rescaled in tensor memory), otherwise the stale maximum is kept - the final division makes both exact; P is
 //     written to shared memory as bf16 in the K-major swizzled layout the second MMA reads;
@@ -30,7 +31,7 @@ namespace attn {
 namespace {
 
 constexpr int DH = 128, T = 128;                  // head_dim; KV tokens per tile
-constexpr int kThreadsTc = 192;
+constexpr int kThreadsTc = 224;                  // warps: 0 K producer, 1 MMA, 2..5 softmax, 6 V producer
 constexpr int kSoftmaxThreads = 128;
 constexpr int kHalfBytes = 128 * 128;             // [128 rows][64 bf16], 128-byte rows, swizzled
 constexpr int kTileBytes = 2 * kHalfBytes;        // Q, P, one K tile, one V tile
@@ -74,12 +75,23 @@ __device__ __forceinline__ uint64_t tile_desc(uint32_t saddr, uint32_t lbo_bytes
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
 
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void stmatrix_x4(uint32_t addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3)
+{
+    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
+}
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+template <int H>
 __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap map_k,
                                                                 const __grid_constant__ CUtensorMap map_v, const TcArgs a)
 {
@@ -104,7 +116,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
         mbar_init(smem_u32(&ctl->p_full), kSoftmaxThreads);
         mbar_init(smem_u32(&ctl->pv_done), 1);
         mbar_init(smem_u32(&ctl->q_ready), kSoftmaxThreads);
-        for (int s = 0; s < NQ; ++s) { mbar_init(smem_u32(&ctl->uq_full[s]), 1); mbar_init(smem_u32(&ctl->uq_empty[s]), 5); }
+        for (int s = 0; s < NQ; ++s) { mbar_init(smem_u32(&ctl->uq_full[s]), 1); mbar_init(smem_u32(&ctl->uq_empty[s]), 6); }
         mbar_init(smem_u32(&ctl->drain), 1);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -120,23 +132,35 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     const uint32_t tmem_base = ctl->tmem_base;
     const int rows_valid = a.R * a.group;
 
-    if (warp == 0) {
-        // ---- producer: unit queue + TMA ring ----
+    if (warp == 0 || warp == 6) {
+        // ---- producers: warp 0 pulls units, publishes them and streams the K tiles; warp 6 streams the V tiles (the issue
+        // cost of the 16 TMA boxes a tile needs per operand is what one thread can sustain) ----
         if (lane == 0) {
-            uint32_t ks = 0, kph = 0, vs = 0, vph = 0;
+            const bool is_k = warp == 0;
+            const CUtensorMap* map = is_k ? &map_k : &map_v;
+            uint64_t* full = is_k ? ctl->k_full : ctl->v_full;
+            uint64_t* empty = is_k ? ctl->k_empty : ctl->v_empty;
+            const uint32_t ring = is_k ? k_s : v_s;
+            uint32_t st = 0, ph = 0;
             bool ok = true;
             const int n_units = *a.pv.n_entries * a.Hkv;
             for (int n = 0; ok; ++n) {
                 const int slot_q = n % NQ;
-                if (!mbar_wait(smem_u32(&ctl->uq_empty[slot_q]), (((uint32_t)(n / NQ)) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-                const int u = atomicAdd(&a.pv.counters[a.counter_index], 1);
                 UnitMsg msg{0, 0, 0, -1, -1, 0, 0, 0};
-                if (u < n_units) {
-                    const Unit un = a.pv.entries[u / a.Hkv];
-                    msg.b = un.b; msg.g = u % a.Hkv; msg.t0 = un.t0; msg.t1 = un.t1; msg.slot = un.slot;
+                if (is_k) {
+                    if (!mbar_wait(smem_u32(&ctl->uq_empty[slot_q]), (((uint32_t)(n / NQ)) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                    const int u = atomicAdd(&a.pv.counters[a.counter_index], 1);
+                    if (u < n_units) {
+                        const Unit un = a.pv.entries[u / a.Hkv];
+                        msg.b = un.b; msg.g = u % a.Hkv; msg.t0 = un.t0; msg.t1 = un.t1; msg.slot = un.slot;
+                    }
+                    ctl->uq[slot_q] = msg;
+                    mbar_arrive(smem_u32(&ctl->uq_full[slot_q]));
+                } else {
+                    if (!mbar_wait(smem_u32(&ctl->uq_full[slot_q]), ((uint32_t)(n / NQ)) & 1u, abort_flag)) { ok = false; break; }
+                    msg = ctl->uq[slot_q];
+                    mbar_arrive(smem_u32(&ctl->uq_empty[slot_q]));
                 }
-                ctl->uq[slot_q] = msg;
-                mbar_arrive(smem_u32(&ctl->uq_full[slot_q]));
                 if (msg.t1 < 0) break;
                 const int32_t* table = a.block_table + (size_t)msg.b * a.max_blocks;
                 const int n_tiles = (msg.t1 - msg.t0 + T - 1) / T;
@@ -150,36 +174,18 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                         phys[bb] = (bi * kBT < msg.t1 && bi < a.max_blocks) ? table[bi] : -1;
                         n_ok += phys[bb] >= 0;
                     }
-                    // K tile
-                    if (!mbar_wait(smem_u32(&ctl->k_empty[ks]), kph ^ 1u, abort_flag)) { ok = false; break; }
-                    {
-                        const uint32_t bar = smem_u32(&ctl->k_full[ks]);
-                        mbar_expect_tx(bar, (uint32_t)n_ok * 2u * (kBT * 128));
-                        const uint32_t dst = k_s + ks * kTileBytes;
+                    if (!mbar_wait(smem_u32(&empty[st]), ph ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t bar = smem_u32(&full[st]);
+                    mbar_expect_tx(bar, (uint32_t)n_ok * 2u * (kBT * 128));
+                    const uint32_t dst = ring + st * kTileBytes;
 #pragma unroll
-                        for (int bb = 0; bb < T / kBT; ++bb) {
-                            if (phys[bb] < 0) continue;
-                            const int row = (phys[bb] * a.Hkv + msg.g) * kBT;
-                            tma_load_2d(dst + bb * (kBT * 128), &map_k, 0, row, bar);
-                            tma_load_2d(dst + kHalfBytes + bb * (kBT * 128), &map_k, 64, row, bar);
-                        }
-                        if (++ks == kStages) { ks = 0; kph ^= 1u; }
+                    for (int bb = 0; bb < T / kBT; ++bb) {
+                        if (phys[bb] < 0) continue;
+                        const int row = (phys[bb] * a.Hkv + msg.g) * kBT;
+                        tma_load_2d(dst + bb * (kBT * 128), map, 0, row, bar);
+                        tma_load_2d(dst + kHalfBytes + bb * (kBT * 128), map, 64, row, bar);
                     }
-                    // V tile
-                    if (!mbar_wait(smem_u32(&ctl->v_empty[vs]), vph ^ 1u, abort_flag)) { ok = false; break; }
-                    {
-                        const uint32_t bar = smem_u32(&ctl->v_full[vs]);
-                        mbar_expect_tx(bar, (uint32_t)n_ok * 2u * (kBT * 128));
-                        const uint32_t dst = v_s + vs * kTileBytes;
-#pragma unroll
-                        for (int bb = 0; bb < T / kBT; ++bb) {
-                            if (phys[bb] < 0) continue;
-                            const int row = (phys[bb] * a.Hkv + msg.g) * kBT;
-                            tma_load_2d(dst + bb * (kBT * 128), &map_v, 0, row, bar);
-                            tma_load_2d(dst + kHalfBytes + bb * (kBT * 128), &map_v, 64, row, bar);
-                        }
-                        if (++vs == kStages) { vs = 0; vph ^= 1u; }
-                    }
+                    if (++st == kStages) { st = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {                                  // give copies in flight time to land before the CTA goes away
@@ -243,15 +249,35 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && clock64() - t0c < kWaitLimit) { }
             }
         }
-    } else {
-        // ---- softmax warps: thread = MMA row m = quarter * 32 + lane; query row r = lane * 4 + quarter ----
+    } else if (warp < 6) {
+        // ---- softmax warps.  Query row r lives in MMA row / tensor-memory lane (r % 4) * 32 + r / 4, so every quarter (one
+        // warp each) holds rows_valid / 4 rows in its first lanes.  The scores are read in the 16-lane fragment shape
+        // (16x256b: a row's 8 consecutive columns over the 4 threads of a quad, rows g4 and g4 + 8 per thread, as in an
+        // mma accumulator), so all 32 threads share the columns of 16 rows: with up to 64 query rows (H = 1) a thread
+        // handles 64 scores per tile, with up to 128 (H = 2: both 16-lane halves) 128.  The exponentials are the critical
+        // path: 4 per clock and scheduler whatever the number of active lanes.
         const int quarter = warp & 3;
-        const int m = quarter * 32 + lane;
-        const int r = lane * 4 + quarter;
-        const bool row_ok = r < rows_valid;
-        const int ri = row_ok ? r / a.group : 0, rj = row_ok ? r % a.group : 0;
+        const int g4 = lane >> 2, q4 = lane & 3;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const uint32_t o_tmem = t_lane + 256;
+        // staging / result mapping: thread = tensor-memory lane
+        const int r_st = lane * 4 + quarter;
+        const bool st_ok = r_st < rows_valid;
+        const int st_i = st_ok ? r_st / a.group : 0, st_j = st_ok ? r_st % a.group : 0;
+        const int m_st = quarter * 32 + lane;
+        // score mapping: rows (h, hh) -> lane-in-quarter h * 16 + g4 + 8 * hh
+        bool rok[H][2];
+        int ri[H][2];
+#pragma unroll
+        for (int h = 0; h < H; ++h)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int r = (h * 16 + g4 + 8 * hh) * 4 + quarter;
+                rok[h][hh] = r < rows_valid;
+                ri[h][hh] = rok[h][hh] ? r / a.group : 0;
+            }
+        // P row address pieces for stmatrix: lane supplies the address of row (k & 1) * 8 + rr of matrix k = lane / 8
+        const int sm_k = lane >> 3, sm_rr = lane & 7;
         uint32_t n_tile = 0;                          // running tile counter (same sequence as the MMA warp's)
         bool ok = true;
         for (int n = 0; ok; ++n) {
@@ -263,112 +289,168 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
             if (un.t1 < 0) break;
             const int n_tiles = (un.t1 - un.t0 + T - 1) / T;
             // stage Q: the previous unit's S tiles have all been read, so no MMA still reads the buffer
-            int lim = -1;
-            if (row_ok) {
-                lim = a.pos[(size_t)un.b * a.R + ri];
-                const uint4* qp = reinterpret_cast<const uint4*>(a.q + ((size_t)un.b * a.R + ri) * a.q_row_stride +
-                                                                 (size_t)(un.g * a.group + rj) * DH);
+            if (st_ok) {
+                const uint4* qp = reinterpret_cast<const uint4*>(a.q + ((size_t)un.b * a.R + st_i) * a.q_row_stride +
+                                                                 (size_t)(un.g * a.group + st_j) * DH);
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
                     const uint4 v = qp[c];
-                    const uint32_t off = (uint32_t)((c >> 3) * kHalfBytes + m * 128 + (((c & 7) ^ (m & 7)) << 4));
+                    const uint32_t off = (uint32_t)((c >> 3) * kHalfBytes + m_st * 128 + (((c & 7) ^ (m_st & 7)) << 4));
                     *reinterpret_cast<uint4*>(base_ptr + off) = v;
                 }
             }
             fence_proxy_async();
             mbar_arrive(smem_u32(&ctl->q_ready));
+            int lim[H][2];
+            float m_used[H][2], l_run[H][2];          // l_run: this thread's share of the row sum (its columns)
+#pragma unroll
+            for (int h = 0; h < H; ++h)
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    lim[h][hh] = rok[h][hh] ? a.pos[(size_t)un.b * a.R + ri[h][hh]] : -1;
+                    m_used[h][hh] = -INFINITY;
+                    l_run[h][hh] = 0.f;
+                }
 
-            float m_used = -INFINITY, l_run = 0.f;
             for (int j = 0; j < n_tiles; ++j, ++n_tile) {
                 const uint32_t buf = n_tile & 1u;
                 if (!mbar_wait(smem_u32(&ctl->s_full[buf]), (n_tile >> 1) & 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const int tok0 = un.t0 + j * T;
-                const int vis = min(lim + 1, un.t1) - tok0;       // this row sees tile columns [0, vis)
-                // pass 1: row maximum
-                float mx = -INFINITY;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tc_ld32(t_lane + buf * 128 + c * 32, v);
-                    tc_wait_ld();
-                    if (row_ok) {
+                int vis[H][2];                                    // the row sees tile columns [0, vis)
+                bool all_vis = true;
 #pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (c * 32 + e < vis) mx = fmaxf(mx, __uint_as_float(v[e]));
+                for (int h = 0; h < H; ++h)
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        vis[h][hh] = min(lim[h][hh] + 1, un.t1) - tok0;
+                        all_vis = all_vis && (vis[h][hh] >= T || !rok[h][hh]);
                     }
+                if (__all_sync(0xffffffffu, all_vis)) {           // most tiles need no masking: lift the limits out of reach
+#pragma unroll
+                    for (int h = 0; h < H; ++h) { vis[h][0] = 0x7fffffff; vis[h][1] = 0x7fffffff; }
                 }
-                mx *= a.scale_log2;                               // scale > 0; -inf stays -inf
-                float alpha = 1.f;
+                uint32_t pk[H][32];                               // bf16 pairs: [x * 16 + 2 * jc + hh]
+                float alpha[H][2];
                 bool raise = false;
-                if (row_ok && mx > -INFINITY && (m_used == -INFINITY || mx > m_used + kRescaleGap)) {
-                    alpha = m_used == -INFINITY ? 0.f : exp2f(m_used - mx);
-                    raise = j > 0;                                // the first tile overwrites the accumulator
-                    m_used = mx;
-                    l_run *= alpha;
-                }
-                const float ms = m_used == -INFINITY ? 0.f : m_used;
-                // pass 2: probabilities, packed to bf16
-                uint32_t pk[64];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tc_ld32(t_lane + buf * 128 + c * 32, v);
+                for (int h = 0; h < H; ++h) {
+                    const uint32_t s_addr = t_lane + ((uint32_t)(h * 16) << 16) + buf * 128;
+                    // both 64-column loads are issued before the one wait: a tensor-memory load takes a few hundred
+                    // cycles and this warp is alone on its scheduler, so nothing else would hide them
+                    uint32_t v[2][32];
+                    tc_ld_16x256b_x8(s_addr, v[0]);
+                    tc_ld_16x256b_x8(s_addr + 64, v[1]);
                     tc_wait_ld();
-                    if (c == 3) { tc_fence_before(); mbar_arrive(smem_u32(&ctl->s_empty[buf])); }
+                    if (h == H - 1) { tc_fence_before(); mbar_arrive(smem_u32(&ctl->s_empty[buf])); }
+                    // row maxima over this thread's columns, then over the quad
+                    float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        float p0 = 0.f, p1 = 0.f;
-                        if (row_ok) {
-                            if (c * 32 + e < vis) p0 = exp2f(fmaf(__uint_as_float(v[e]), a.scale_log2, -ms));
-                            if (c * 32 + e + 1 < vis) p1 = exp2f(fmaf(__uint_as_float(v[e + 1]), a.scale_log2, -ms));
+                    for (int x = 0; x < 2; ++x)
+#pragma unroll
+                        for (int jc = 0; jc < 8; ++jc)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const int col = x * 64 + jc * 8 + 2 * q4 + (e & 1);
+                                if (col >= vis[h][e >> 1]) v[x][4 * jc + e] = 0xff800000u;      // -inf: the exponential is an exact zero
+                                mx[e >> 1] = fmaxf(mx[e >> 1], __uint_as_float(v[x][4 * jc + e]));
+                            }
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 1));
+                        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 2));
+                        mx[hh] *= a.scale_log2;                   // scale > 0; -inf stays -inf
+                        alpha[h][hh] = 1.f;
+                        if (rok[h][hh] && mx[hh] > -INFINITY && (m_used[h][hh] == -INFINITY || mx[hh] > m_used[h][hh] + kRescaleGap)) {
+                            alpha[h][hh] = m_used[h][hh] == -INFINITY ? 0.f : exp2f(m_used[h][hh] - mx[hh]);
+                            raise = raise || j > 0;               // the first tile overwrites the accumulator
+                            m_used[h][hh] = mx[hh];
+                            l_run[h][hh] *= alpha[h][hh];
                         }
-                        l_run += p0 + p1;
-                        pk[c * 16 + e / 2] = pack2(p0, p1);
                     }
+                    const float ms0 = m_used[h][0] == -INFINITY ? 0.f : m_used[h][0];
+                    const float ms1 = m_used[h][1] == -INFINITY ? 0.f : m_used[h][1];
+                    // probabilities, bf16 pairs
+                    float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+                    for (int x = 0; x < 2; ++x)
+#pragma unroll
+                        for (int jc = 0; jc < 8; ++jc) {
+                            float p[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                p[e] = ex2_approx(fmaf(__uint_as_float(v[x][4 * jc + e]), a.scale_log2, (e >> 1) ? -ms1 : -ms0));
+                            l0 += p[0] + p[1];
+                            l1 += p[2] + p[3];
+                            pk[h][x * 16 + 2 * jc] = pack2(p[0], p[1]);
+                            pk[h][x * 16 + 2 * jc + 1] = pack2(p[2], p[3]);
+                        }
+                    l_run[h][0] += l0;
+                    l_run[h][1] += l1;
                 }
                 // the previous tile's P V has finished: P may be overwritten and the accumulator is at rest
                 if (n_tile > 0 && !mbar_wait(smem_u32(&ctl->pv_done), (n_tile - 1u) & 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 if (__any_sync(0xffffffffu, raise)) {
-                    const float f = raise ? alpha : 1.f;
-#pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t v[32];
-                        tc_ld32(o_tmem + c * 32, v);
-                        tc_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * f);
-                        tc_st32(o_tmem + c * 32, v);
-                    }
+                    for (int h = 0; h < H; ++h)
+#pragma unroll 1
+                        for (int x = 0; x < 2; ++x) {
+                            uint32_t v[32];
+                            const uint32_t o_addr = o_tmem + ((uint32_t)(h * 16) << 16) + x * 64;
+                            tc_ld_16x256b_x8(o_addr, v);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha[h][(e >> 1) & 1]);
+                            tc_st_16x256b_x8(o_addr, v);
+                        }
                     tc_wait_st();
                 }
-                if (row_ok) {
+                // P: two 8 x 8 column groups of both row halves per stmatrix (matrix k: rows (k & 1) * 8.., chunk + (k >> 1))
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {                // 16-byte chunk c holds tokens 8c .. 8c+7
-                        const uint32_t off = (uint32_t)(kTileBytes + (c >> 3) * kHalfBytes + m * 128 + (((c & 7) ^ (m & 7)) << 4));
-                        *reinterpret_cast<uint4*>(base_ptr + off) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-                    }
+                for (int h = 0; h < H; ++h) {
+                    const int mrow = quarter * 32 + h * 16 + (sm_k & 1) * 8 + sm_rr;
+#pragma unroll
+                    for (int x = 0; x < 2; ++x)
+#pragma unroll
+                        for (int jj = 0; jj < 4; ++jj) {
+                            const int c16 = x * 8 + 2 * jj + (sm_k >> 1);
+                            const uint32_t addr = p_s + (uint32_t)((c16 >> 3) * kHalfBytes + mrow * 128 + (((c16 & 7) ^ (mrow & 7)) << 4));
+                            stmatrix_x4(addr, pk[h][x * 16 + 4 * jj], pk[h][x * 16 + 4 * jj + 1], pk[h][x * 16 + 4 * jj + 2],
+                                        pk[h][x * 16 + 4 * jj + 3]);
+                        }
                 }
                 fence_proxy_async();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&ctl->p_full));
             }
             if (!ok) break;
-            // ---- unit result ----
+            // ---- unit result: thread = tensor-memory lane; the row's maximum and sum come from the quad that tracked it ----
             if (!mbar_wait(smem_u32(&ctl->pv_done), (n_tile - 1u) & 1u, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            float row_m = -INFINITY, row_l = 0.f;
+#pragma unroll
+            for (int h = 0; h < H; ++h)
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    float l = l_run[h][hh];
+                    l += __shfl_xor_sync(0xffffffffu, l, 1);
+                    l += __shfl_xor_sync(0xffffffffu, l, 2);
+                    const float tm = __shfl_sync(0xffffffffu, m_used[h][hh], 4 * (lane & 7));
+                    const float tl = __shfl_sync(0xffffffffu, l, 4 * (lane & 7));
+                    if ((lane >> 4) == h && ((lane >> 3) & 1) == hh) { row_m = tm; row_l = tl; }
+                }
+            const float inv = row_l > 0.f ? 1.f / row_l : 0.f;
             float* part = nullptr;
             __nv_bfloat16* op = nullptr;
-            if (row_ok) {
+            if (st_ok) {
                 if (un.slot >= 0) {
-                    const size_t ps = ((size_t)un.slot * a.Hkv + un.g) * a.rows_alloc + r;
+                    const size_t ps = ((size_t)un.slot * a.Hkv + un.g) * a.rows_alloc + r_st;
                     part = a.pv.part_o + ps * DH;
-                    a.pv.part_ml[ps * 2] = m_used;
-                    a.pv.part_ml[ps * 2 + 1] = l_run;
+                    a.pv.part_ml[ps * 2] = row_m;
+                    a.pv.part_ml[ps * 2 + 1] = row_l;
                 } else {
-                    op = a.out + ((size_t)un.b * a.R + ri) * a.out_row_stride + (size_t)(un.g * a.group + rj) * DH;
+                    op = a.out + ((size_t)un.b * a.R + st_i) * a.out_row_stride + (size_t)(un.g * a.group + st_j) * DH;
                 }
             }
 #pragma unroll 1
@@ -426,7 +508,9 @@ spec_status launch_attention_tc(const AttnArgs& a, cudaStream_t st)
     const PlanView pv = carve_plan(a.scratch, a.B, a.Hkv, rows_alloc, a.dh, max_chunks);
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc) != cudaSuccess) return SPEC_ERR_CUDA;
+        if (cudaFuncSetAttribute(attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc) != cudaSuccess ||
+            cudaFuncSetAttribute(attn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc) != cudaSuccess)
+            return SPEC_ERR_CUDA;
         configured = true;
     }
     // the pools as matrices of 128-column rows ((block, head, token) flattened); one box = 64 columns x 16 tokens
@@ -441,7 +525,8 @@ spec_status launch_attention_tc(const AttnArgs& a, cudaStream_t st)
         spec_status s = launch_attn_plan(a.B, a.R, a.pos, max_chunks, pv, st);
         if (s != SPEC_OK) return s;
     }
-    attn_tc_kernel<<<tc_sm_count(), kThreadsTc, kSmemTc, st>>>(mk, mv, t);
+    if (rows <= 64) attn_tc_kernel<1><<<tc_sm_count(), kThreadsTc, kSmemTc, st>>>(mk, mv, t);
+    else            attn_tc_kernel<2><<<tc_sm_count(), kThreadsTc, kSmemTc, st>>>(mk, mv, t);
     if (launch_status() != SPEC_OK) return SPEC_ERR_CUDA;
     return launch_attn_merge128(a.B, rows_alloc, a.Hkv, a.R, group, a.out, a.out_row_stride, pv, st);
 }
