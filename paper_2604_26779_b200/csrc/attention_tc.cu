@@ -6,9 +6,9 @@
 // its operands from shared memory once per tile whatever M is:
 //   - work units (sequence, KV head, chunk of <= 4096 tokens) come from the same plan and atomic counter as the
 //     register-fragment kernel; one persistent CTA per SM;
-//   - warp 0 pulls units and streams their K tiles of 128 tokens with TMA straight from the paged pool, warp 6 the V
-//     tiles: one 64-column x 16-row box per (block, half of head_dim), 128-byte swizzle, so a tile lands as
-//     [half][token][64] - K-major for S = Q K^T and MN-major for O += P V - in two 2-stage rings;
+//   - four producer warps stream the K and V tiles of 128 tokens with TMA straight from the paged pools: one 64-column
+//     x 16-row box per (block, half of head_dim), 128-byte swizzle, so a tile lands as [half][token][64] - K-major for
+//     S = Q K^T and MN-major for O += P V - in two 2-stage rings; warp 0 also pulls the units and publishes them;
 //   - warp 1 issues the MMAs from one thread: S (128 x 128, fp32) into one of two tensor-memory buffers, O (128 x 128)
 //     accumulated in a third;
 //   - warps 2..5 are the softmax; query rows are dealt round-robin over the four 32-lane quarters of tensor memory and
@@ -31,7 +31,7 @@ namespace attn {
 namespace {
 
 constexpr int DH = 128, T = 128;                  // head_dim; KV tokens per tile
-constexpr int kThreadsTc = 224;                  // warps: 0 K producer, 1 MMA, 2..5 softmax, 6 V producer
+constexpr int kThreadsTc = 288;                  // warps: 0, 7 K producers; 6, 8 V producers; 1 MMA; 2..5 softmax
 constexpr int kSoftmaxThreads = 128;
 constexpr int kHalfBytes = 128 * 128;             // [128 rows][64 bf16], 128-byte rows, swizzled
 constexpr int kTileBytes = 2 * kHalfBytes;        // Q, P, one K tile, one V tile
@@ -109,14 +109,14 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
         reinterpret_cast<uint4*>(base_ptr)[i] = make_uint4(0u, 0u, 0u, 0u);
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1);
-            mbar_init(smem_u32(&ctl->v_full[s]), 1); mbar_init(smem_u32(&ctl->v_empty[s]), 1);
+            mbar_init(smem_u32(&ctl->k_full[s]), 2); mbar_init(smem_u32(&ctl->k_empty[s]), 1);
+            mbar_init(smem_u32(&ctl->v_full[s]), 2); mbar_init(smem_u32(&ctl->v_empty[s]), 1);
         }
         for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->s_full[s]), 1); mbar_init(smem_u32(&ctl->s_empty[s]), kSoftmaxThreads); }
         mbar_init(smem_u32(&ctl->p_full), kSoftmaxThreads);
         mbar_init(smem_u32(&ctl->pv_done), 1);
         mbar_init(smem_u32(&ctl->q_ready), kSoftmaxThreads);
-        for (int s = 0; s < NQ; ++s) { mbar_init(smem_u32(&ctl->uq_full[s]), 1); mbar_init(smem_u32(&ctl->uq_empty[s]), 6); }
+        for (int s = 0; s < NQ; ++s) { mbar_init(smem_u32(&ctl->uq_full[s]), 1); mbar_init(smem_u32(&ctl->uq_empty[s]), 8); }
         mbar_init(smem_u32(&ctl->drain), 1);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -132,11 +132,13 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     const uint32_t tmem_base = ctl->tmem_base;
     const int rows_valid = a.R * a.group;
 
-    if (warp == 0 || warp == 6) {
-        // ---- producers: warp 0 pulls units, publishes them and streams the K tiles; warp 6 streams the V tiles (the issue
-        // cost of the 16 TMA boxes a tile needs per operand is what one thread can sustain) ----
+    if (warp == 0 || warp >= 6) {
+        // ---- producers: one thread issues a TMA box in ~100 cycles and a tile needs 16 per operand, so four warps share
+        // them: warps 0 and 7 the even and odd blocks of the K tiles, warps 6 and 8 those of the V tiles.  Warp 0 also pulls
+        // the units and publishes them to everyone else. ----
         if (lane == 0) {
-            const bool is_k = warp == 0;
+            const bool is_k = warp == 0 || warp == 7;
+            const int parity_b = warp >= 7 ? 1 : 0;
             const CUtensorMap* map = is_k ? &map_k : &map_v;
             uint64_t* full = is_k ? ctl->k_full : ctl->v_full;
             uint64_t* empty = is_k ? ctl->k_empty : ctl->v_empty;
@@ -147,7 +149,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
             for (int n = 0; ok; ++n) {
                 const int slot_q = n % NQ;
                 UnitMsg msg{0, 0, 0, -1, -1, 0, 0, 0};
-                if (is_k) {
+                if (warp == 0) {
                     if (!mbar_wait(smem_u32(&ctl->uq_empty[slot_q]), (((uint32_t)(n / NQ)) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                     const int u = atomicAdd(&a.pv.counters[a.counter_index], 1);
                     if (u < n_units) {
@@ -166,22 +168,23 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 const int n_tiles = (msg.t1 - msg.t0 + T - 1) / T;
                 for (int j = 0; j < n_tiles && ok; ++j) {
                     const int blk0 = (msg.t0 + j * T) / kBT;
-                    int phys[T / kBT];
+                    int phys[T / kBT / 2];
                     int n_ok = 0;
 #pragma unroll
-                    for (int bb = 0; bb < T / kBT; ++bb) {
-                        const int bi = blk0 + bb;
-                        phys[bb] = (bi * kBT < msg.t1 && bi < a.max_blocks) ? table[bi] : -1;
-                        n_ok += phys[bb] >= 0;
+                    for (int hb = 0; hb < T / kBT / 2; ++hb) {
+                        const int bi = blk0 + 2 * hb + parity_b;
+                        phys[hb] = (bi * kBT < msg.t1 && bi < a.max_blocks) ? table[bi] : -1;
+                        n_ok += phys[hb] >= 0;
                     }
                     if (!mbar_wait(smem_u32(&empty[st]), ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t bar = smem_u32(&full[st]);
                     mbar_expect_tx(bar, (uint32_t)n_ok * 2u * (kBT * 128));
                     const uint32_t dst = ring + st * kTileBytes;
 #pragma unroll
-                    for (int bb = 0; bb < T / kBT; ++bb) {
-                        if (phys[bb] < 0) continue;
-                        const int row = (phys[bb] * a.Hkv + msg.g) * kBT;
+                    for (int hb = 0; hb < T / kBT / 2; ++hb) {
+                        if (phys[hb] < 0) continue;
+                        const int bb = 2 * hb + parity_b;
+                        const int row = (phys[hb] * a.Hkv + msg.g) * kBT;
                         tma_load_2d(dst + bb * (kBT * 128), map, 0, row, bar);
                         tma_load_2d(dst + kHalfBytes + bb * (kBT * 128), map, 64, row, bar);
                     }
@@ -453,25 +456,29 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                     op = a.out + ((size_t)un.b * a.R + st_i) * a.out_row_stride + (size_t)(un.g * a.group + st_j) * DH;
                 }
             }
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tc_ld32(o_tmem + c * 32, v);
+            {
+                uint32_t o[4][32];                    // the whole row in one round trip to tensor memory
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tc_ld32(o_tmem + c * 32, o[c]);
                 tc_wait_ld();
-                if (part != nullptr) {
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4)
-                        *reinterpret_cast<float4*>(part + c * 32 + e) =
-                            make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]), __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
-                } else if (op != nullptr) {
+                for (int c = 0; c < 4; ++c) {
+                    if (part != nullptr) {
 #pragma unroll
-                    for (int e = 0; e < 32; e += 8) {
-                        uint4 o;
-                        o.x = pack2(__uint_as_float(v[e]) * inv, __uint_as_float(v[e + 1]) * inv);
-                        o.y = pack2(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv);
-                        o.z = pack2(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv);
-                        o.w = pack2(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv);
-                        *reinterpret_cast<uint4*>(op + c * 32 + e) = o;
+                        for (int e = 0; e < 32; e += 4)
+                            *reinterpret_cast<float4*>(part + c * 32 + e) =
+                                make_float4(__uint_as_float(o[c][e]), __uint_as_float(o[c][e + 1]), __uint_as_float(o[c][e + 2]),
+                                            __uint_as_float(o[c][e + 3]));
+                    } else if (op != nullptr) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8) {
+                            uint4 w;
+                            w.x = pack2(__uint_as_float(o[c][e]) * inv, __uint_as_float(o[c][e + 1]) * inv);
+                            w.y = pack2(__uint_as_float(o[c][e + 2]) * inv, __uint_as_float(o[c][e + 3]) * inv);
+                            w.z = pack2(__uint_as_float(o[c][e + 4]) * inv, __uint_as_float(o[c][e + 5]) * inv);
+                            w.w = pack2(__uint_as_float(o[c][e + 6]) * inv, __uint_as_float(o[c][e + 7]) * inv);
+                            *reinterpret_cast<uint4*>(op + c * 32 + e) = w;
+                        }
                     }
                 }
             }
