@@ -16,8 +16,9 @@
 //     exponentials, 4 per clock and scheduler whatever the number of active lanes, are what a tile costs).  Row maximum and exponentials in the exp2 domain; the
 //     running maximum is only raised when a tile exceeds it by more than 2^8 (the accumulator and the row sum are then
 //     rescaled in tensor memory), otherwise the stale maximum is kept - the final division makes both exact; P is
-//     written to shared memory as bf16 in the K-major swizzled layout the second MMA reads;
-//   - per unit the softmax threads stage Q (zero-padded to 128 rows) and write the result: normalised bf16 for
+//     written back to tensor memory as bf16 pairs, from where the second MMA takes it as its A operand;
+//   - per unit the softmax threads stage Q (zero-padded to 128 rows) in tensor memory, from where the first MMA takes it
+//     as its A operand, and write the result: normalised bf16 for
 //     single-chunk sequences, (max, sum, unnormalised fp32 row) partials for the merge kernel otherwise.
 // Every mbarrier wait is bounded (abort flag -> SPEC_ERR_TIMEOUT, tensor memory released, kernel returns).
 #include <cuda.h>
@@ -35,10 +36,10 @@ constexpr int kThreadsTc = 288;                  // warps: 0, 7 K producers; 6, 
 constexpr int kSoftmaxThreads = 128;
 constexpr int kHalfBytes = 128 * 128;             // [128 rows][64 bf16], 128-byte rows, swizzled
 constexpr int kTileBytes = 2 * kHalfBytes;        // Q, P, one K tile, one V tile
-constexpr int kStages = 2;
+constexpr int kStages = 3;                        // per ring (K and V)
 constexpr int NQ = 4;                             // unit queue depth (the producer runs ahead of the consumers)
-constexpr uint32_t kTmemCols = 512;               // S0 [0,128), S1 [128,256), O [256,384)
-constexpr int kSmemTc = (2 + 2 * kStages) * kTileBytes + 1024 + 512;
+constexpr uint32_t kTmemCols = 512;               // S0 [0,128), S1 [128,256), O [256,384), Q [384,448) and P [448,512) as bf16 pairs
+constexpr int kSmemTc = 2 * kStages * kTileBytes + 1024 + 512;
 constexpr float kRescaleGap = 8.f;                // log2 units
 
 struct UnitMsg { int b, g, t0, t1, slot, pad0, pad1, pad2; };
@@ -81,10 +82,6 @@ __device__ __forceinline__ float ex2_approx(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void stmatrix_x4(uint32_t addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3)
-{
-    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
-}
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -99,13 +96,13 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - raw);
-    const uint32_t q_s = base, p_s = base + kTileBytes, k_s = base + 2 * kTileBytes, v_s = k_s + kStages * kTileBytes;
-    Ctl* ctl = reinterpret_cast<Ctl*>(base_ptr + (2 + 2 * kStages) * kTileBytes);
+    const uint32_t k_s = base, v_s = k_s + kStages * kTileBytes;
+    Ctl* ctl = reinterpret_cast<Ctl*>(base_ptr + 2 * kStages * kTileBytes);
     volatile int* abort_flag = &ctl->abort;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     // finite contents everywhere: masked probabilities are exact zeros, and 0 x (stale but finite) stays 0
-    for (int i = threadIdx.x; i < (2 + 2 * kStages) * kTileBytes / 16; i += kThreadsTc)
+    for (int i = threadIdx.x; i < 2 * kStages * kTileBytes / 16; i += kThreadsTc)
         reinterpret_cast<uint4*>(base_ptr)[i] = make_uint4(0u, 0u, 0u, 0u);
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -213,8 +210,8 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 for (int h = 0; h < 2; ++h)
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        tc_mma(tmem_base + buf * 128, tile_desc(q_s + h * kHalfBytes + kk * 32, 16, 1024),
-                               tile_desc(kb + h * kHalfBytes + kk * 32, 16, 1024), kIdescQK, (h | kk) ? 1u : 0u);
+                        tc_mma_ta(tmem_base + buf * 128, tmem_base + 384 + (h * 4 + kk) * 8,
+                                  tile_desc(kb + h * kHalfBytes + kk * 32, 16, 1024), kIdescQK, (h | kk) ? 1u : 0u);
                 tc_commit(smem_u32(&ctl->k_empty[ks]));
                 tc_commit(smem_u32(&ctl->s_full[buf]));
                 if (++ks == kStages) { ks = 0; kph ^= 1u; }
@@ -238,8 +235,8 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                     const uint32_t vb = v_s + vs * kTileBytes;
 #pragma unroll
                     for (int kk = 0; kk < T / 16; ++kk)      // 16 tokens per instruction: two 8-token groups of the V tile
-                        tc_mma(o_tmem, tile_desc(p_s + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024),
-                               tile_desc(vb + kk * 2048, kHalfBytes, 1024), kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+                        tc_mma_ta(o_tmem, tmem_base + 448 + kk * 8, tile_desc(vb + kk * 2048, kHalfBytes, 1024), kIdescPV,
+                                  (j > 0 || kk > 0) ? 1u : 0u);
                     tc_commit(smem_u32(&ctl->v_empty[vs]));
                     tc_commit(smem_u32(&ctl->pv_done));
                     if (++vs == kStages) { vs = 0; vph ^= 1u; }
@@ -279,8 +276,14 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 rok[h][hh] = r < rows_valid;
                 ri[h][hh] = rok[h][hh] ? r / a.group : 0;
             }
-        // P row address pieces for stmatrix: lane supplies the address of row (k & 1) * 8 + rr of matrix k = lane / 8
-        const int sm_k = lane >> 3, sm_rr = lane & 7;
+        {   // rows without a query row hold zeros in Q and P for the whole launch
+            uint32_t z[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) z[e] = 0u;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tc_st32(t_lane + 384 + c * 32, z);
+            tc_wait_st();
+        }
         uint32_t n_tile = 0;                          // running tile counter (same sequence as the MMA warp's)
         bool ok = true;
         for (int n = 0; ok; ++n) {
@@ -291,18 +294,23 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
             if (lane == 0) mbar_arrive(smem_u32(&ctl->uq_empty[slot_q]));
             if (un.t1 < 0) break;
             const int n_tiles = (un.t1 - un.t0 + T - 1) / T;
-            // stage Q: the previous unit's S tiles have all been read, so no MMA still reads the buffer
-            if (st_ok) {
+            // stage Q in tensor memory (the A operand of S = Q K^T): thread = row, 64 columns of bf16 pairs.  The previous
+            // unit's S tiles have all been read, so no MMA still reads it.
+            {
+                uint32_t qv[2][32];
                 const uint4* qp = reinterpret_cast<const uint4*>(a.q + ((size_t)un.b * a.R + st_i) * a.q_row_stride +
                                                                  (size_t)(un.g * a.group + st_j) * DH);
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
-                    const uint4 v = qp[c];
-                    const uint32_t off = (uint32_t)((c >> 3) * kHalfBytes + m_st * 128 + (((c & 7) ^ (m_st & 7)) << 4));
-                    *reinterpret_cast<uint4*>(base_ptr + off) = v;
+                    const uint4 v = st_ok ? qp[c] : make_uint4(0u, 0u, 0u, 0u);
+                    qv[c >> 3][(c & 7) * 4] = v.x; qv[c >> 3][(c & 7) * 4 + 1] = v.y;
+                    qv[c >> 3][(c & 7) * 4 + 2] = v.z; qv[c >> 3][(c & 7) * 4 + 3] = v.w;
                 }
+                tc_st32(t_lane + 384, qv[0]);
+                tc_st32(t_lane + 384 + 32, qv[1]);
+                tc_wait_st();
             }
-            fence_proxy_async();
+            tc_fence_before();
             mbar_arrive(smem_u32(&ctl->q_ready));
             int lim[H][2];
             float m_used[H][2], l_run[H][2];          // l_run: this thread's share of the row sum (its columns)
@@ -409,21 +417,10 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                         }
                     tc_wait_st();
                 }
-                // P: two 8 x 8 column groups of both row halves per stmatrix (matrix k: rows (k & 1) * 8.., chunk + (k >> 1))
+                // P goes to tensor memory as bf16 pairs (the A operand of O += P V): one store per 16-lane half
 #pragma unroll
-                for (int h = 0; h < H; ++h) {
-                    const int mrow = quarter * 32 + h * 16 + (sm_k & 1) * 8 + sm_rr;
-#pragma unroll
-                    for (int x = 0; x < 2; ++x)
-#pragma unroll
-                        for (int jj = 0; jj < 4; ++jj) {
-                            const int c16 = x * 8 + 2 * jj + (sm_k >> 1);
-                            const uint32_t addr = p_s + (uint32_t)((c16 >> 3) * kHalfBytes + mrow * 128 + (((c16 & 7) ^ (mrow & 7)) << 4));
-                            stmatrix_x4(addr, pk[h][x * 16 + 4 * jj], pk[h][x * 16 + 4 * jj + 1], pk[h][x * 16 + 4 * jj + 2],
-                                        pk[h][x * 16 + 4 * jj + 3]);
-                        }
-                }
-                fence_proxy_async();
+                for (int h = 0; h < H; ++h) tc_st_16x128b_x16(t_lane + ((uint32_t)(h * 16) << 16) + 448, pk[h]);
+                tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&ctl->p_full));
             }
