@@ -36,16 +36,16 @@ constexpr int kThreadsTc = 288;                  // warps: 0, 7 K producers; 6, 
 constexpr int kSoftmaxThreads = 128;
 constexpr int kHalfBytes = 128 * 128;             // [128 rows][64 bf16], 128-byte rows, swizzled
 constexpr int kTileBytes = 2 * kHalfBytes;        // Q, P, one K tile, one V tile
-constexpr int kStages = 3;                        // per ring (K and V)
+constexpr int kStagesK = 4, kStagesV = 3;         // K is needed a tile earlier than V
 constexpr int NQ = 4;                             // unit queue depth (the producer runs ahead of the consumers)
 constexpr uint32_t kTmemCols = 512;               // S0 [0,128), S1 [128,256), O [256,384), Q [384,448) and P [448,512) as bf16 pairs
-constexpr int kSmemTc = 2 * kStages * kTileBytes + 1024 + 512;
+constexpr int kSmemTc = (kStagesK + kStagesV) * kTileBytes + 1024 + 512;
 constexpr float kRescaleGap = 8.f;                // log2 units
 
 struct UnitMsg { int b, g, t0, t1, slot, pad0, pad1, pad2; };
 
 struct Ctl {
-    uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+    uint64_t k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
     uint64_t s_full[2], s_empty[2], p_full, pv_done, q_ready, uq_full[NQ], uq_empty[NQ], drain;
     UnitMsg uq[NQ];
     uint32_t tmem_base;
@@ -96,19 +96,17 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - raw);
-    const uint32_t k_s = base, v_s = k_s + kStages * kTileBytes;
-    Ctl* ctl = reinterpret_cast<Ctl*>(base_ptr + 2 * kStages * kTileBytes);
+    const uint32_t k_s = base, v_s = k_s + kStagesK * kTileBytes;
+    Ctl* ctl = reinterpret_cast<Ctl*>(base_ptr + (kStagesK + kStagesV) * kTileBytes);
     volatile int* abort_flag = &ctl->abort;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     // finite contents everywhere: masked probabilities are exact zeros, and 0 x (stale but finite) stays 0
-    for (int i = threadIdx.x; i < 2 * kStages * kTileBytes / 16; i += kThreadsTc)
+    for (int i = threadIdx.x; i < (kStagesK + kStagesV) * kTileBytes / 16; i += kThreadsTc)
         reinterpret_cast<uint4*>(base_ptr)[i] = make_uint4(0u, 0u, 0u, 0u);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&ctl->k_full[s]), 2); mbar_init(smem_u32(&ctl->k_empty[s]), 1);
-            mbar_init(smem_u32(&ctl->v_full[s]), 2); mbar_init(smem_u32(&ctl->v_empty[s]), 1);
-        }
+        for (int s = 0; s < kStagesK; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 2); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
+        for (int s = 0; s < kStagesV; ++s) { mbar_init(smem_u32(&ctl->v_full[s]), 2); mbar_init(smem_u32(&ctl->v_empty[s]), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->s_full[s]), 1); mbar_init(smem_u32(&ctl->s_empty[s]), kSoftmaxThreads); }
         mbar_init(smem_u32(&ctl->p_full), kSoftmaxThreads);
         mbar_init(smem_u32(&ctl->pv_done), 1);
@@ -185,7 +183,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                         tma_load_2d(dst + bb * (kBT * 128), map, 0, row, bar);
                         tma_load_2d(dst + kHalfBytes + bb * (kBT * 128), map, 64, row, bar);
                     }
-                    if (++st == kStages) { st = 0; ph ^= 1u; }
+                    if (++st == (is_k ? kStagesK : kStagesV)) { st = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {                                  // give copies in flight time to land before the CTA goes away
@@ -214,7 +212,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                                   tile_desc(kb + h * kHalfBytes + kk * 32, 16, 1024), kIdescQK, (h | kk) ? 1u : 0u);
                 tc_commit(smem_u32(&ctl->k_empty[ks]));
                 tc_commit(smem_u32(&ctl->s_full[buf]));
-                if (++ks == kStages) { ks = 0; kph ^= 1u; }
+                if (++ks == kStagesK) { ks = 0; kph ^= 1u; }
                 ++n_qk;
                 return true;
             };
@@ -239,7 +237,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                                   (j > 0 || kk > 0) ? 1u : 0u);
                     tc_commit(smem_u32(&ctl->v_empty[vs]));
                     tc_commit(smem_u32(&ctl->pv_done));
-                    if (++vs == kStages) { vs = 0; vph ^= 1u; }
+                    if (++vs == kStagesV) { vs = 0; vph ^= 1u; }
                     ++n_pv;
                 }
             }
