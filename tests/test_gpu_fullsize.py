@@ -91,3 +91,67 @@ def test_full_size_step_sampled_against_oracle():
         keep = -(-int(new_len[bb]) // 16)
         assert np.all(t2[bb, :keep] >= 0) and np.all(t2[bb, keep:] == -1) and np.array_equal(t2[bb, : -(-int(pre_len[bb]) // 16)], table[bb, : -(-int(pre_len[bb]) // 16)])
     eng.close()
+
+
+@pytest.mark.parametrize("name,B,R,Hq,Hkv,lens_kind", [
+    ("MoE layer shape, 64 query rows per KV head", 256, 4, 64, 4, "fixed8192"),
+    ("8B shape at k=4, 20 query rows per KV head", 512, 5, 32, 8, "lognormal"),
+])
+def test_attention_at_bench_sizes_sampled(name, B, R, Hq, Hkv, lens_kind):
+    """The attention launch of the other benchmark configurations at their full batch and cache lengths (the launch
+    configuration bench.py times for them): sampled (sequence, KV head) pairs are recomputed by the oracle from the
+    device's own bytes, every output of the launch must be finite, and rows of sequences that differ only in their block
+    placement must agree bit for bit."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40e9:
+        pytest.skip("needs a device with > 40 GB free")
+    from oracle import model
+    from paper_2604_26779_b200 import binding as api, inputs
+    dh, bt = 128, 16
+    if lens_kind == "fixed8192":
+        lens = np.full(B, 8192, np.int32)
+    else:
+        lens = inputs.make_seq_lens_lognormal(B, 4096, float(np.log(2.0)), 16, 32768, 77)
+    lens[1] = lens[0]                                           # sequence 1 repeats sequence 0 in other blocks
+    nb_seq = [-(-(int(l) + R) // bt) for l in lens]
+    max_blocks = max(nb_seq) + 1
+    nblk = int(sum(nb_seq)) + 7
+    gen = torch.Generator(device="cuda"); gen.manual_seed(2604)
+    kpool = torch.randn((nblk, Hkv, bt, dh), device="cuda", generator=gen).to(torch.bfloat16)
+    vpool = torch.randn((nblk, Hkv, bt, dh), device="cuda", generator=gen).to(torch.bfloat16)
+    q = torch.randn((B, R, Hq, dh), device="cuda", generator=gen).to(torch.bfloat16)
+    order = inputs.make_block_order(nblk, 5)
+    table = np.full((B, max_blocks), -1, np.int32)
+    nxt = 0
+    for b in range(B):
+        table[b, : nb_seq[b]] = order[nxt : nxt + nb_seq[b]]
+        nxt += nb_seq[b]
+    dtable = torch.from_numpy(table).cuda()
+    # sequence 1 = sequence 0: same query rows, same cache contents, different physical blocks
+    q[1] = q[0]
+    i0 = torch.as_tensor(table[0, : nb_seq[0]].astype(np.int64), device="cuda")
+    i1 = torch.as_tensor(table[1, : nb_seq[1]].astype(np.int64), device="cuda")
+    kpool[i1] = kpool[i0]
+    vpool[i1] = vpool[i0]
+    out = torch.full((B, R, Hq, dh), float("nan"), dtype=torch.bfloat16, device="cuda")
+    scratch = torch.zeros(api.spec_attention_scratch_bytes(B, R, Hq, Hkv, dh, max_blocks * bt), dtype=torch.uint8, device="cuda")
+    api.spec_attention(q, kpool, vpool, dtable, torch.from_numpy(lens).cuda(), out, scratch)
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(out.float()).all())
+    assert torch.equal(out[0], out[1])
+    group = Hq // Hkv
+    worst = 0.0
+    picks = [(0, 0), (B // 2, Hkv - 1), (B - 1, 1), (int(np.argmax(lens)), 0), (int(np.argmin(lens)), Hkv - 1)]
+    for b, g in picks:
+        n = int(lens[b]) + R
+        idx = torch.as_tensor(table[b, : -(-n // bt)].astype(np.int64), device="cuda")
+        kk = kpool[idx, g].reshape(-1, dh)[:n].float().cpu().numpy().astype(np.float64)[:, None, :]
+        vv = vpool[idx, g].reshape(-1, dh)[:n].float().cpu().numpy().astype(np.float64)[:, None, :]
+        qq = q[b, :, g * group : (g + 1) * group].float().cpu().numpy().astype(np.float64)
+        ref = model.attention(qq, kk, vv, n_past=int(lens[b]))
+        got = out[b, :, g * group : (g + 1) * group].float().cpu().numpy()
+        worst = max(worst, float((np.abs(got - ref).max(-1) / np.abs(ref).max(-1)).max()))
+    print(f"{name}: B={B}, {R * group} rows, worst sampled row error {worst:.2e}")
+    assert worst < 2e-2

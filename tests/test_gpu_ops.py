@@ -92,7 +92,9 @@ def test_paged_attention_matches_oracle(api, lens, R, Hq, Hkv, dh, dtype):
     (128, 256, 512, torch.bfloat16, torch.bfloat16, False),
     (1024, 6144, 4096, torch.bfloat16, torch.bfloat16, False),     # 8B QKV projection
     (1024, 4096, 14336, torch.bfloat16, torch.float32, True),      # 8B down projection into the fp32 residual
-    (256, 4096, 4096, torch.bfloat16, torch.float32, True),        # decode-sized M
+    (256, 4096, 4096, torch.bfloat16, torch.float32, True),        # decode-sized M: two m-tiles per CTA
+    (200, 1000, 2048, torch.bfloat16, torch.bfloat16, False),      # the same variant with ragged M and N
+    (129, 512, 320, torch.bfloat16, torch.float32, False),
     (1000, 520, 192, torch.bfloat16, torch.bfloat16, False),       # ragged M and N tails
     (77, 1000, 4096, torch.bfloat16, torch.float32, False),
     (1024, 16384, 1024, torch.bfloat16, torch.float32, False),     # LM-head-like slice: fp32 logits
