@@ -43,12 +43,16 @@ def draft_head_weights(eng, cfg, kind):
     return H
 
 
-@pytest.mark.parametrize("kind,k", [("eagle3", 3), ("mtp", 2), ("eagle3", 7)])
-def test_bf16_steps_stage_by_stage(kind, k):
+@pytest.mark.parametrize("kind,k,head_dim", [("eagle3", 3, 64), ("mtp", 2, 64), ("eagle3", 7, 64),
+                                              ("eagle3", 5, 128), ("mtp", 7, 128)])
+def test_bf16_steps_stage_by_stage(kind, k, head_dim):
+    """head_dim 64: 16 or 32 query rows per KV head on the register-fragment attention kernel; head_dim 128 with k = 5 / 7:
+    24 / 32 rows on the tcgen05 kernel, including the draft head's first pass, whose rows past the committed count carry
+    position -1."""
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from paper_2604_26779_b200 import workloads
-    over = dict(d_model=512, n_q_heads=8, n_kv_heads=2, head_dim=64, d_ffn=1024)
+    over = dict(d_model=512, n_q_heads=8, n_kv_heads=2, head_dim=head_dim, d_ffn=1024)
     n_layers = 3
     lens = np.array([5, 40, 100, 17, 300], np.int32)
     eng, info = workloads.build_dense_workload("c3", lens=lens, k=k, draft=kind, steps_budget=8, n_layers=n_layers,
@@ -108,6 +112,6 @@ def test_bf16_steps_stage_by_stage(kind, k):
         assert eng.status().device_status == 0
         assert np.array_equal(eng.seq_len().cpu().numpy(), seq_len + g_n)
         k_prev = k
-    print(f"bf16 {kind} k={k}: draft logits {worst_d:.2e}, verify logits {worst_v:.2e}, boundary cases {boundary}")
+    print(f"bf16 {kind} k={k} dh={head_dim}: draft logits {worst_d:.2e}, verify logits {worst_v:.2e}, boundary cases {boundary}")
     assert worst_d < 2e-2 and worst_v < 2e-2 and boundary <= 2
     eng.close()
