@@ -74,7 +74,9 @@ typedef struct {
     uint64_t seed;              /* Philox key of every uniform the step draws                            */
     int32_t ngram_n;            /* SPEC_DRAFT_NGRAM: longest trailing n-gram looked up in the sequence's own   */
                                 /* tokens (1..8); the model-free drafting the paper uses as a baseline (Table 2) */
-    int32_t reserved_;
+    int32_t draft_greedy;       /* 1: the draft head proposes d_i = argmax of its logits (ties: lowest id)      */
+                                /* and q_i is taken as one-hot(d_i): accept iff u < p_i(d_i), residual = p_i    */
+                                /* without d_i's mass (the deterministic-draft special case of the rule)        */
 } spec_config;
 
 /* Byte sizes of the caller-owned device arenas for a configuration. */
@@ -186,6 +188,7 @@ spec_status spec_seq_replace(spec_ctx* ctx, int n, const int32_t* slots_host, co
 /* S1 draft propose.  Runs the draft head: pass 0 consumes the (tapped hidden state, next token) pairs of the
  * positions committed by the previous step, passes 1..k-1 feed the head its own output; fills draft tokens
  * d_1..d_k (d_i drawn from q_i with the stream-1 uniforms), draft logits and their row statistics.
+ * With draft_greedy = 1 the head's tokens are the arg-maxima of its logits and no draft uniform is consumed.
  * With SPEC_DRAFT_NGRAM no model runs: d_1..d_k continue the most recent earlier occurrence of the sequence's trailing
  * n-gram (n = ngram_n down to 1; without any match the last token is repeated), and q is one-hot.
  * Errors: STATE (no committed step to draft from, draft_kind NONE), SHAPE (k outside 1..k_max). */

@@ -41,7 +41,13 @@ class ChainOracle:
             u_draft = oracle.uniforms(self.seed, self.step, 1, self.seq + 1, max(k, 1))[self.seq]
 
             def sample_fn(i, logits_row):
-                q = oracle.softmax(np.asarray(logits_row, np.float32)[None, :], self.T)[0]
+                lg = np.asarray(logits_row, np.float32)
+                if cfg.get("draft_greedy"):                 # deterministic draft: arg-max (lowest id among equals), q = one-hot
+                    tok = int(np.argmax(lg))
+                    q = np.zeros(lg.shape[0], np.float32)
+                    q[tok] = 1.0
+                    return tok, q
+                q = oracle.softmax(lg[None, :], self.T)[0]
                 tok, _ = oracle.invcdf(q, u_draft[i])
                 return tok, q
 

@@ -47,7 +47,7 @@ class spec_config(C.Structure):
                 ("n_taps", C.c_int32), ("tap_layers", C.c_int32 * 3),
                 ("k_max", C.c_int32), ("max_batch", C.c_int32), ("kv_block_tokens", C.c_int32),
                 ("kv_num_blocks", C.c_int32), ("max_blocks_per_seq", C.c_int32), ("kv_layer_pools", C.c_int32),
-                ("temperature", C.c_float), ("seed", C.c_uint64), ("ngram_n", C.c_int32), ("reserved_", C.c_int32)]
+                ("temperature", C.c_float), ("seed", C.c_uint64), ("ngram_n", C.c_int32), ("draft_greedy", C.c_int32)]
 
 
 class spec_sizes(C.Structure):

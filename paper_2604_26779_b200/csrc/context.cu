@@ -586,8 +586,8 @@ extern "C" spec_status spec_reject_sample(spec_ctx* c, int k, const float* draft
     if (B == 0) return SPEC_OK;
     void* ws = c->buf.workspace;
     char* sb = static_cast<char*>(c->buf.state);
-    // no draft head and no draft logits: the drafts are deterministic (n-gram lookup, greedy), q = one-hot(d)
-    const bool has_head = g.draft_kind == SPEC_DRAFT_EAGLE3 || g.draft_kind == SPEC_DRAFT_MTP;
+    // no sampled draft and no draft logits given: the drafts are deterministic (n-gram lookup, greedy head), q = one-hot(d)
+    const bool has_head = (g.draft_kind == SPEC_DRAFT_EAGLE3 || g.draft_kind == SPEC_DRAFT_MTP) && !g.draft_greedy;
     const float* ql = draft_logits ? draft_logits : (has_head ? at<float>(ws, c->draft_logits) : nullptr);
     float* qs = at<float>(ws, c->draft_row_stats);
     if (draft_logits != nullptr && k > 0)
@@ -702,9 +702,13 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
         const void* lm = eagle ? at<const void>(dw, c->d_lm_head) : at<const void>(c->buf.weights, c->lm_head);
         TRY(launch_rmsnorm(B, d, hid, nf, g.rms_eps, at(ws, c->h), d, 0, dt, st));
         TRY(launch_gemm(B, V, d, at(ws, c->h), d, lm, dlog + (size_t)j * V, k * V, dt, SPEC_DTYPE_F32, 0, st));
-        TRY(launch_softmax_rows(B, V, dlog + (size_t)j * V, (size_t)k * V, g.temperature, dstats + 2 * j, k, nullptr, st));
-        TRY(launch_sample_logits(B, V, dlog + (size_t)j * V, (size_t)k * V, dstats + 2 * j, k, g.temperature, g.seed,
-                                 at<uint32_t>(sb, c->step), (uint32_t)j, 1u, dtoks + j, kstride, status, st));
+        if (g.draft_greedy) {
+            TRY(launch_argmax_rows(B, V, dlog + (size_t)j * V, (size_t)k * V, dtoks + j, kstride, st));
+        } else {
+            TRY(launch_softmax_rows(B, V, dlog + (size_t)j * V, (size_t)k * V, g.temperature, dstats + 2 * j, k, nullptr, st));
+            TRY(launch_sample_logits(B, V, dlog + (size_t)j * V, (size_t)k * V, dstats + 2 * j, k, g.temperature, g.seed,
+                                     at<uint32_t>(sb, c->step), (uint32_t)j, 1u, dtoks + j, kstride, status, st));
+        }
     }
     return SPEC_OK;
 }

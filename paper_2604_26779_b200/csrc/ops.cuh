@@ -18,6 +18,8 @@ spec_status launch_sample_logits(int rows, int V, const float* logits, size_t ro
                                  size_t stats_stride, float temperature, uint64_t seed, const uint32_t* step_dev,
                                  uint32_t slot, uint32_t stream_tag, int32_t* tokens, int token_stride, int32_t* status,
                                  cudaStream_t st);
+spec_status launch_argmax_rows(int rows, int V, const float* logits, size_t row_stride, int32_t* tokens, int token_stride,
+                               cudaStream_t st);
 int sampler_max_vocab();
 
 // ops.cu: element-wise and bookkeeping kernels.  dtype = SPEC_DTYPE_* of the activation/weight/KV storage.

@@ -287,6 +287,34 @@ __global__ void __launch_bounds__(kThreads) sample_logits_kernel(int V, const fl
     }
 }
 
+// arg-maximum per row (greedy drafting): the largest logit, the lowest index among equals
+__global__ void __launch_bounds__(kThreads) argmax_rows_kernel(int V, const float* __restrict__ logits, size_t row_stride,
+                                                               int32_t* __restrict__ tokens, int token_stride)
+{
+    __shared__ float s_v[kThreads / 32];
+    __shared__ int s_i[kThreads / 32];
+    const float* l = logits + (size_t)blockIdx.x * row_stride;
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int v = threadIdx.x; v < V; v += kThreads) {
+        const float x = l[v];
+        if (x > bv || (x == bv && v < bi)) { bv = x; bi = v; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { s_v[threadIdx.x >> 5] = bv; s_i[threadIdx.x >> 5] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kThreads / 32; ++w)
+            if (s_v[w] > bv || (s_v[w] == bv && s_i[w] < bi)) { bv = s_v[w]; bi = s_i[w]; }
+        tokens[(size_t)blockIdx.x * token_stride] = bi == 0x7fffffff ? 0 : bi;
+    }
+}
+
 // ---- rejection sampling ---------------------------------------------------------------------------------------------
 struct RejectArgs {
     int B, k, V;
@@ -452,6 +480,14 @@ spec_status launch_sample_logits(int rows, int V, const float* logits, size_t ro
     if (rows == 0) return SPEC_OK;
     sample_logits_kernel<<<rows, kThreads, 0, st>>>(V, logits, row_stride, stats, stats_stride, 1.0f / temperature, seed,
                                                     step_dev, slot, stream_tag, tokens, token_stride, status);
+    return launch_status();
+}
+
+spec_status launch_argmax_rows(int rows, int V, const float* logits, size_t row_stride, int32_t* tokens, int token_stride,
+                               cudaStream_t st)
+{
+    if (rows == 0) return SPEC_OK;
+    argmax_rows_kernel<<<rows, kThreads, 0, st>>>(V, logits, row_stride, tokens, token_stride);
     return launch_status();
 }
 

@@ -15,7 +15,7 @@ from .binding import T
 
 def make_spec_config(cfg: dict, *, draft_kind: str = "none", k_max: int = 3, max_batch: int = 4, kv_num_blocks: int = 64,
                      max_blocks_per_seq: int = 16, kv_block_tokens: int = 16, kv_layer_pools: int | None = None,
-                     seed: int = 0, draft_d_ffn: int | None = None, ngram_n: int = 3) -> B.spec_config:
+                     seed: int = 0, draft_d_ffn: int | None = None, ngram_n: int = 3, draft_greedy: bool = False) -> B.spec_config:
     sc = B.spec_config()
     sc.struct_size, sc.abi_version = C.sizeof(B.spec_config), B.SPEC_ABI_VERSION
     for name in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab", "n_experts",
@@ -26,6 +26,7 @@ def make_spec_config(cfg: dict, *, draft_kind: str = "none", k_max: int = 3, max
     sc.draft_kind = {"none": B.SPEC_DRAFT_NONE, "eagle3": B.SPEC_DRAFT_EAGLE3, "mtp": B.SPEC_DRAFT_MTP, "ngram": B.SPEC_DRAFT_NGRAM}[draft_kind]
     sc.draft_d_ffn = int(draft_d_ffn if draft_d_ffn is not None else (cfg["d_ffn"] or 4 * cfg["d_model"])) if draft_kind in ("eagle3", "mtp") else 0
     sc.ngram_n = int(ngram_n) if draft_kind == "ngram" else 0
+    sc.draft_greedy = 1 if draft_greedy else 0
     taps = tuple(cfg.get("tap_layers", ())) if draft_kind == "eagle3" else ()
     sc.n_taps = len(taps)
     for i, t in enumerate(taps):

@@ -32,7 +32,7 @@ def run_chain(engine, cfg, kind, B, prompt_len, k, n_steps, seed, prompts=None):
         prompts = inputs.make_prompts(B, prompt_len, cfg["vocab"], seed=inputs.sub_seed(1, 2))
     max_blocks = -(-(prompt_len + n_steps * (k + 1) + k + 2) // 16)
     sc = engine.make_spec_config(cfg, draft_kind=kind, k_max=k, max_batch=B, kv_num_blocks=B * max_blocks + 3,
-                                 max_blocks_per_seq=max_blocks, seed=seed)
+                                 max_blocks_per_seq=max_blocks, seed=seed, draft_greedy=bool(cfg.get("draft_greedy")))
     eng = engine.SpecStep(sc)
     eng.load_target_weights(W)
     if H is not None:
@@ -153,6 +153,17 @@ def test_chain_ngram_drafting_lockstep(eng_mod):
     r = run_chain(eng_mod, cfg, "ngram", B=4, prompt_len=48, k=3, n_steps=16, seed=123, prompts=prompts)
     print("ngram:", r)
     assert r["max_rel"] < 1e-3 and r["boundary"] <= 1 and r["emitted"] >= r["steps"]
+
+
+def test_chain_greedy_head_drafts_lockstep(eng_mod):
+    """Greedy drafting: the head's arg-max tokens with q = one-hot; the emitted tokens are still exact samples of the
+    target (accept iff u < p(d), residual = p without d)."""
+    cfg = dict(inputs.model_config("c1"), draft_greedy=True)
+    r = run_chain(eng_mod, cfg, "eagle3", B=3, prompt_len=32, k=3, n_steps=20, seed=31)
+    print("greedy eagle3:", r)
+    assert r["max_rel"] < 1e-3 and r["max_rel_d"] < 1e-3 and r["boundary"] <= 2
+    assert r["emitted"] >= r["steps"]      # a random target accepts an arg-max draft with probability ~1/vocab: the accepted
+                                           # branch of the one-hot rule is covered by the sampler tests
 
 
 def test_chain_at_other_temperature_and_k1(eng_mod):
