@@ -9,6 +9,8 @@
 // ldmatrix (transposed for V), softmax is online in fp32 (exp2 domain), and units of one sequence are merged by a
 // log-sum-exp kernel (skipped for single-chunk sequences, which write their output directly).
 // Causality among the new rows: row (i, head j) sees cache positions <= pos[b*R + i].
+// This is the kernel for up to 16 query rows per KV head (and for head_dim 64); wider row groups at head_dim 128 go to the
+// tcgen05 kernel, which shares the plan and the merge pass defined here.
 #include "attention_plan.cuh"
 
 namespace spec {
