@@ -28,6 +28,8 @@ UNIT = "tokens/s"
 # dram bytes per attention launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture on a 32-sequence case
 # of the same kernel) as a ratio to the algorithmic bytes of that captured launch; traffic grows in proportion to the units
 ATTN_TRAFFIC_RATIO = 1.009
+# the same for the tcgen05 attention kernel (64-sequence case of the MoE layer shape; split-KV partials included)
+ATTN_TC_TRAFFIC_RATIO = 1.028
 
 
 def measured_peaks():
@@ -407,9 +409,12 @@ def main():
     # n_layers launches per step on the target's cache and k on the draft head's one-layer cache: the same positions each
     alg_bytes = mean_cached_tokens * bytes_per_token_layer
     achieved = alg_bytes / (attn_ms * 1e-3) / 1e9
-    roofline = {"kernel": "attn_mma_kernel (+ plan / merge)", "bound": "hbm", "achieved": achieved, "peak": hbm_peak,
+    rows_per_kv_head = R * (cfg["n_q_heads"] // cfg["n_kv_heads"])
+    tc_attention = rows_per_kv_head > 16 and cfg["head_dim"] == 128       # the library's dispatch rule
+    traffic_ratio = ATTN_TC_TRAFFIC_RATIO if tc_attention else ATTN_TRAFFIC_RATIO
+    roofline = {"kernel": ("attn_tc_kernel" if tc_attention else "attn_mma_kernel") + " (+ plan / merge)", "bound": "hbm", "achieved": achieved, "peak": hbm_peak,
                 "unit": "GB/s", "frac": achieved / hbm_peak, "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({peak_kind})",
-                "traffic": None if ATTN_TRAFFIC_RATIO is None else alg_bytes * ATTN_TRAFFIC_RATIO,
+                "traffic": None if traffic_ratio is None else alg_bytes * traffic_ratio,
                 "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": attn_ms, "launches_timed": attn_passes,
                 "share_of_step": float(timing.ms[0]) / ms_total, "frac_of_nominal_8TBs": achieved / 8000.0}
 

@@ -43,3 +43,12 @@ def test_host_side_argument_checks(built_lib):
     assert L.spec_softmax_rows(1, 8, None, 1.0, None, None, None) == -1
     assert L.spec_reject_sample_probs(1, 40, 8, None, None, None, 0, 0, None, None, None, None) == -1
     assert L.spec_query_sizes(None, None) < 0
+    # context entry points refuse a missing context before touching anything
+    assert L.spec_seq_replace(None, 1, None, None, None, None) == -1
+    assert L.spec_seq_init(None, 1, None, None, None, None) == -1
+    assert L.spec_verify(None, 0, None, None) == -1
+    assert L.spec_draft(None, 1, None) == -1
+    assert L.spec_reject_sample(None, 0, None, None) == -1
+    assert L.spec_kv_commit(None, None, None, None) == -1
+    assert L.spec_attention(1, 0, 8, 2, 128, 16, 4, None, None, None, None, None, None, 1, None, 0, None) == -1
+    assert L.spec_gemm(4, 4, 0, None, None, None, 1, 1, 0, None) == -1
