@@ -183,6 +183,55 @@ def controlled_acceptance(eng, k, temperature, taus, n_steps, stream):
     return out
 
 
+# Acceptance lengths the paper measured for its trained EAGLE-3 drafts at each draft length (its draft-length ablation, Table 4;
+# RL-Zero / RL-Think), used only to convert this build's step cost into a labelled projection.
+PAPER_AL_BY_K = {3: (3.32, 2.77), 5: (4.35, 3.23), 7: (5.06, 3.48)}
+
+
+def run_k_sweep(args, ks):
+    """Step cost against draft length on the headline workload: c(k) = t_step(k) / t_decode and the speed-up over plain
+    decode that an acceptance length AL would give, AL / c(k) - the mechanism behind the paper's finding that longer
+    drafts raise AL but can lower the speed-up (Section 4.2)."""
+    import torch
+    from paper_2604_26779_b200 import workloads
+    kmax = max(ks)
+    eng, info = workloads.build_dense_workload("c3", B=args.batch, k=kmax, n_layers=args.layers, kv_pools=args.kv_pools,
+                                               len_lo=args.len_lo, len_hi=args.len_hi, steps_budget=12 * len(ks) + 24)
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, n):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(n):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+    workloads.bootstrap(eng)
+    ms_dec = timed(lambda: workloads.bootstrap(eng), 4)
+    rows = []
+    for k in ks:
+        rep0 = eng.status()
+        ms = timed(lambda: workloads.spec_step(eng, k), 4)
+        rep1 = eng.status()
+        al = (rep1.emitted_tokens - rep0.emitted_tokens) / float(6 * args.batch)
+        row = {"k": k, "ms_per_step": ms, "cost_ratio_vs_decode": ms / ms_dec, "acceptance_length_random_head": al,
+               "query_rows_per_kv_head": (k + 1) * (info["cfg"]["n_q_heads"] // info["cfg"]["n_kv_heads"])}
+        if k in PAPER_AL_BY_K:
+            row["projected_speedup_at_paper_AL"] = {f"{a:.2f}": a / (ms / ms_dec) for a in PAPER_AL_BY_K[k]}
+        rows.append(row)
+    assert eng.status().device_status == 0
+    print(json.dumps({"metric": "step cost vs draft length (c3 workload)", "ms_plain_decode_step": ms_dec, "k_sweep": rows,
+                      "config": {"workload": "c3", "batch": args.batch, "layers": info["cfg"]["n_layers"],
+                                 "kv_layer_pools": info["kv_pools"], "aliased_kv": bool(info["aliased"])},
+                      "note": "projections divide the paper's measured acceptance lengths by this build's kernel-level cost "
+                              "ratio; the paper's own speed-ups include prefill, scheduling and sampling overheads of its stack"}))
+    return 0
+
+
 def run_sampler_microbench(args):
     """Rejection-sampling micro-benchmark (B=1024, V=151936, k in {1,3,5,7}; target logits N(0, sigma^2), draft = target +
     N(0, tau^2)): the stateless sampler on given fp32 probabilities, and the fused from-logits path (row statistics +
@@ -271,6 +320,9 @@ def main():
     ap.add_argument("--cpu-layers", type=int, default=12, help="layers the CPU-baseline sample times (scaled to all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--k-sweep", default=None,
+                    help="comma-separated draft lengths, e.g. 1,3,5,7: times the c3 step at each k on one engine built for the "
+                         "largest (not the headline run: prints its own JSON line)")
     ap.add_argument("--workload", default="c3", choices=["c3", "c4", "c5", "c2"],
                     help="c3 = the headline 8B + EAGLE-3 workload; c4 = 8B + MTP head, B=512, lognormal lengths; "
                          "c5 = one 235B-A22B-shaped MoE layer + LM head, B=256, cache length 8192 (measurement of the "
@@ -288,6 +340,8 @@ def main():
     torch.cuda.set_device(local)
     if args.workload == "c2":
         return run_sampler_microbench(args) if rank == 0 else 0
+    if args.k_sweep:
+        return run_k_sweep(args, [int(x) for x in args.k_sweep.split(",")]) if rank == 0 else 0
     dist = None
     if world > 1 and args.impl == "ours":
         import torch.distributed as dist_mod
