@@ -383,6 +383,9 @@ def main():
         workloads_spec_step = lambda e, kk, with_draft=True: step_fn(with_draft)
     else:
         workloads_spec_step = workloads.spec_step
+    if dist is not None:
+        # replicas of one model: rank 0's weights reach every rank by one broadcast over NCCL (outside the timed region)
+        replicas.broadcast_weights([eng.arenas["weights"], eng.arenas["draft_weights"]], dist, src=0)
     workloads.bootstrap(eng)
     config = {"workload": wl_name,
               "batch": B, "k": k, "layers": cfg["n_layers"], "kv_layer_pools": info["kv_pools"], "aliased_kv": bool(info["aliased"]),

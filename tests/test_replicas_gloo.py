@@ -14,8 +14,14 @@ def _worker(rank, world, port, out):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     dist.init_process_group("gloo", rank=rank, world_size=world)
     ms, tok = replicas.reduce_job(10.0 + 5.0 * rank, 100.0 * (rank + 1), dist)
+    # weight refresh: every rank ends up with rank 0's bytes, arenas of odd sizes, several chunks
+    g = torch.Generator().manual_seed(100 + rank)
+    arenas = [torch.randint(0, 256, (n,), dtype=torch.uint8, generator=g) for n in (1000, 37, 4096)]
+    sent = replicas.broadcast_weights(arenas, dist, src=0, chunk_bytes=300)
+    g0 = torch.Generator().manual_seed(100)
+    same = all(torch.equal(a, torch.randint(0, 256, (n,), dtype=torch.uint8, generator=g0)) for a, n in zip(arenas, (1000, 37, 4096)))
     dist.barrier()
-    out[rank] = (ms, tok, replicas.replica_seed(rank))
+    out[rank] = (ms, tok, replicas.replica_seed(rank), sent, same)
     dist.destroy_process_group()
 
 
@@ -26,6 +32,7 @@ def test_reduce_job_two_ranks():
         mp.spawn(_worker, args=(2, port, out), nprocs=2, join=True)
         assert out[0][:2] == (15.0, 300.0) and out[1][:2] == (15.0, 300.0)      # max time, summed tokens, on every rank
         assert out[0][2] != out[1][2] and out[0][2] == inputs.sub_seed(3, 0)
+        assert out[0][3] == out[1][3] == 1000 + 37 + 4096 and out[0][4] and out[1][4]
 
 
 def test_shard_by_tokens_balances_long_tail():
