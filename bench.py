@@ -320,6 +320,8 @@ def main():
     ap.add_argument("--cpu-layers", type=int, default=12, help="layers the CPU-baseline sample times (scaled to all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--draft-vocab", type=int, default=0,
+                    help="c3 only: give the EAGLE-3-style head its own vocabulary of this many rows (0 = whole vocabulary, the headline)")
     ap.add_argument("--k-sweep", default=None,
                     help="comma-separated draft lengths, e.g. 1,3,5,7: times the c3 step at each k on one engine built for the "
                          "largest (not the headline run: prints its own JSON line)")
@@ -356,7 +358,8 @@ def main():
         eng, info = workloads.build_dense_workload("c3", B=B, k=k, n_layers=args.layers, kv_pools=args.kv_pools,
                                                    len_lo=args.len_lo, len_hi=args.len_hi,
                                                    steps_budget=steps_budget, device=f"cuda:{local}",
-                                                   seed=replicas.replica_seed(rank))
+                                                   seed=replicas.replica_seed(rank),
+                                                   cfg_over=dict(draft_vocab=args.draft_vocab) if args.draft_vocab else None)
         wl_name = ("c3: 8B dense verify (32 layers, d=4096, 32q/8kv, dh=128, FFN 14336, V=128256, bf16), "
                    "EAGLE-3-style 1-layer draft head, cache lengths ~U[1024,16384], 16-token pages")
     elif args.workload == "c4":
@@ -392,6 +395,8 @@ def main():
               "l2": "inputs_exceed_l2 (15 GB weights + >=9 GB cache per layer per step; no flush needed)",
               "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
               "acceptance": "measured with the random-init draft head (untrained: low by construction)"}
+    if args.workload == "c3" and args.draft_vocab:
+        config["draft_vocab"] = args.draft_vocab
     if args.workload != "c3":
         args.no_cpu_baseline = True
 

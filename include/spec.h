@@ -30,7 +30,7 @@
 extern "C" {
 #endif
 
-#define SPEC_ABI_VERSION 2u
+#define SPEC_ABI_VERSION 3u
 
 typedef struct spec_ctx spec_ctx; /* opaque */
 
@@ -77,6 +77,10 @@ typedef struct {
     int32_t draft_greedy;       /* 1: the draft head proposes d_i = argmax of its logits (ties: lowest id)      */
                                 /* and q_i is taken as one-hot(d_i): accept iff u < p_i(d_i), residual = p_i    */
                                 /* without d_i's mass (the deterministic-draft special case of the rule)        */
+    int32_t draft_vocab;        /* EAGLE3 only: 0 = the head's LM head covers the whole vocabulary; else its    */
+                                /* number of rows (a multiple of 8, <= vocab): row r scores target token        */
+                                /* D_D2T[r] (strictly increasing ids), q is zero outside that set                */
+    int32_t reserved_;
 } spec_config;
 
 /* Byte sizes of the caller-owned device arenas for a configuration. */
@@ -105,7 +109,9 @@ enum {
     SPEC_T_D_WPROJ,             /* MTP: [d][2d] acting on concat(norm_g(g), norm_e(e))                 */
     SPEC_T_D_NORM_E, SPEC_T_D_NORM_G, SPEC_T_D_NORM_F, SPEC_T_D_ATTN_NORM,
     SPEC_T_D_WQKV,              /* EAGLE3: [(Hq+2Hkv)dh][2d] acting on concat(norm_e(e), norm_g(g))    */
-    SPEC_T_D_WO, SPEC_T_D_MLP_NORM, SPEC_T_D_WGATEUP, SPEC_T_D_WDOWN, SPEC_T_D_LM_HEAD,
+    SPEC_T_D_WO, SPEC_T_D_MLP_NORM, SPEC_T_D_WGATEUP, SPEC_T_D_WDOWN,
+    SPEC_T_D_LM_HEAD,           /* EAGLE3: [draft_vocab or vocab][d]                                   */
+    SPEC_T_D_D2T,               /* EAGLE3 with draft_vocab: [draft_vocab] int32 target id of each row  */
     /* caches: [block][n_kv_heads][kv_block_tokens][head_dim]; layer = pool index for the target */
     SPEC_T_KV_K = 64, SPEC_T_KV_V, SPEC_T_DRAFT_KV_K, SPEC_T_DRAFT_KV_V,
     /* state (int32) */
@@ -126,7 +132,7 @@ enum {
                                 /* (the verifier's log-probabilities an RL loss needs, Section 2.3)    */
     /* step results in the workspace */
     SPEC_T_LOGITS = 128,        /* [B][k+1][vocab] fp32 target logits of the last verify               */
-    SPEC_T_DRAFT_LOGITS,        /* [B][k][vocab]   fp32 draft logits of the last draft                 */
+    SPEC_T_DRAFT_LOGITS,        /* [B][k][draft_vocab or vocab] fp32 draft logits of the last draft    */
     SPEC_T_ROW_STATS,           /* [B*(k+1)][2] fp32 (max, sum exp) of the target rows                 */
     SPEC_T_DRAFT_ROW_STATS,     /* [B*k][2]                                                            */
     SPEC_T_TAPS,                /* [B][k+1][n_taps*d] tapped hidden states of the last verify          */
@@ -203,7 +209,7 @@ spec_status spec_verify(spec_ctx* ctx, int k, const int32_t* draft_tokens, void*
 /* S3+S4 fused vocabulary softmax and rejection sampling on the context's logits: accept_i = u_i <
  * min(1, p_i(d_i)/q_i(d_i)); n = accepted prefix length; token n+1 from norm(max(0, p_{n+1}-q_{n+1})) or,
  * when n = k, the bonus token from p_{k+1}; uniforms Philox(seed; step, sequence, slot 0..k, stream 0).
- * draft_logits [B][k][vocab] overrides the context's draft logits when not NULL.  With draft_kind NONE and
+ * draft_logits [B][k][vocab] (always over the whole vocabulary) overrides the context's draft logits when not NULL.  With draft_kind NONE and
  * draft_logits NULL the drafts are taken as deterministic (n-gram lookup, greedy drafting): q = one-hot(d), i.e.
  * accept iff u < p(d), residual = p without the draft token's mass. */
 spec_status spec_reject_sample(spec_ctx* ctx, int k, const float* draft_logits, void* stream);

@@ -216,7 +216,7 @@ def draft_propose(cfg, W, H, kind, true_feat, tokens, k, sample_fn, past_k=None,
     most recent committed token).  past_k/past_v: the head's cached keys/values of slots < first_slot, or
     None.  sample_fn(i, logits_row) -> (token d_{i+1}, q_{i+1} as the fp32 probabilities it was drawn from);
     the caller supplies it so that the softmax and the inverse CDF are the C oracle's.
-    Returns (draft tokens [k], q [k][V] fp32 probabilities, logits [k][V] fp64)."""
+    Returns (draft tokens [k], q [k][V] fp32 probabilities, logits [k][V or draft vocabulary] fp64)."""
     S = true_feat.shape[0]
     pos = first_slot + np.arange(S)
     if kind == "eagle3":
@@ -233,6 +233,11 @@ def draft_propose(cfg, W, H, kind, true_feat, tokens, k, sample_fn, past_k=None,
     for i in range(k):
         lg = eagle3_logits(cfg, H, h_last)[0] if kind == "eagle3" else mtp_logits(cfg, W, h_last)[0]
         d, q = sample_fn(i, lg)
+        if H.get("d2t") is not None:        # the head's own vocabulary: row r scores target token d2t[r], q is zero elsewhere
+            d2t = np.asarray(H["d2t"], np.int64)
+            q_full = np.zeros(cfg["vocab"], np.float32)
+            q_full[d2t] = q
+            d, q = int(d2t[int(d)]), q_full
         drafts.append(int(d))
         q_rows.append(q)
         logit_rows.append(lg)

@@ -12,7 +12,7 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libspec.so")
 
-SPEC_ABI_VERSION = 2
+SPEC_ABI_VERSION = 3
 SPEC_DTYPE_BF16, SPEC_DTYPE_F32 = 0, 1
 SPEC_DRAFT_NONE, SPEC_DRAFT_EAGLE3, SPEC_DRAFT_MTP, SPEC_DRAFT_NGRAM = 0, 1, 2, 3
 
@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "SPEC_OK", -1: "SPEC_ERR_INVALID_ARG", -2: "SPEC_ERR_SHAPE", 
 T = dict(EMBED=0, LM_HEAD=1, FINAL_NORM=2, ATTN_NORM=3, WQKV=4, WO=5, MLP_NORM=6, WGATEUP=7, WDOWN=8, ROUTER=9,
          EXPERTS_GATEUP=10, EXPERTS_DOWN=11,
          D_WFC=32, D_WPROJ=33, D_NORM_E=34, D_NORM_G=35, D_NORM_F=36, D_ATTN_NORM=37, D_WQKV=38, D_WO=39,
-         D_MLP_NORM=40, D_WGATEUP=41, D_WDOWN=42, D_LM_HEAD=43,
+         D_MLP_NORM=40, D_WGATEUP=41, D_WDOWN=42, D_LM_HEAD=43, D_D2T=44,
          KV_K=64, KV_V=65, DRAFT_KV_K=66, DRAFT_KV_V=67,
          SEQ_LEN=96, LAST_TOKEN=97, BLOCK_TABLE=98, FREE_STACK=99, FREE_TOP=100, DRAFT_TOKENS=101, OUT_TOKENS=102,
          N_EMITTED=103, STATUS=104, STEP=105, TOKEN_HISTORY=106, OUT_LOGP=107,
@@ -47,7 +47,7 @@ class spec_config(C.Structure):
                 ("n_taps", C.c_int32), ("tap_layers", C.c_int32 * 3),
                 ("k_max", C.c_int32), ("max_batch", C.c_int32), ("kv_block_tokens", C.c_int32),
                 ("kv_num_blocks", C.c_int32), ("max_blocks_per_seq", C.c_int32), ("kv_layer_pools", C.c_int32),
-                ("temperature", C.c_float), ("seed", C.c_uint64), ("ngram_n", C.c_int32), ("draft_greedy", C.c_int32)]
+                ("temperature", C.c_float), ("seed", C.c_uint64), ("ngram_n", C.c_int32), ("draft_greedy", C.c_int32), ("draft_vocab", C.c_int32), ("reserved_", C.c_int32)]
 
 
 class spec_sizes(C.Structure):

@@ -22,7 +22,7 @@ struct spec_ctx {
     // draft weights
     Loc d_wfc, d_wproj, d_norm_e, d_norm_g, d_norm_f;
     LayerLoc d_layer;
-    Loc d_lm_head;
+    Loc d_lm_head, d_d2t;
     size_t draft_weights_bytes = 0;
     // caches
     size_t kv_pool_bytes = 0, kv_bytes = 0, draft_kv_bytes = 0;
@@ -33,7 +33,8 @@ struct spec_ctx {
     // workspace
     Loc tokens_in, pos, x, h, qkv, attn_out, gu, act, logits, draft_logits, row_stats, draft_row_stats, taps,
         attn_scratch, dg, dx, d_hidden, d_tok, d_pos,
-        moe_logits, moe_ids, moe_wts, moe_rank, moe_counts, moe_offsets, moe_inv, moe_a, moe_gu, moe_act, moe_out, rope, splitk;
+        moe_logits, moe_ids, moe_wts, moe_rank, moe_counts, moe_offsets, moe_inv, moe_a, moe_gu, moe_act, moe_out, rope, splitk,
+        t2d, draft_red;
     size_t workspace_bytes = 0;
     // host-side run state
     int B = 0;
@@ -90,6 +91,8 @@ spec_status check_config(const spec_config* c)
     if (c->draft_kind == SPEC_DRAFT_MTP && (c->draft_d_ffn <= 0 || c->draft_d_ffn % 128 != 0)) return SPEC_ERR_SHAPE;
     if (!(c->temperature > 0.f) || !(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return SPEC_ERR_UNSUPPORTED;
     if (c->vocab > sampler_max_vocab()) return SPEC_ERR_SHAPE;
+    if (c->draft_vocab != 0 && (c->draft_kind != SPEC_DRAFT_EAGLE3 || c->draft_vocab < 8 || c->draft_vocab > c->vocab ||
+                                c->draft_vocab % 8 != 0)) return SPEC_ERR_SHAPE;
     return SPEC_OK;
 }
 
@@ -135,7 +138,8 @@ void build_layout(spec_ctx& x)
                 x.d_wfc = a.take(d * (size_t)c.n_taps * d * es);
                 x.d_norm_f = a.take(d * 4);
                 x.d_layer.wqkv = a.take(qkv_n * 2 * d * es);
-                x.d_lm_head = a.take((size_t)c.vocab * d * es);
+                x.d_lm_head = a.take((size_t)(c.draft_vocab ? c.draft_vocab : c.vocab) * d * es);
+                if (c.draft_vocab) x.d_d2t = a.take((size_t)c.draft_vocab * 4);
             } else {
                 x.d_wproj = a.take(d * 2 * d * es);
                 x.d_layer.attn_norm = a.take(d * 4);
@@ -181,7 +185,11 @@ void build_layout(spec_ctx& x)
         x.gu = a.take(M * 2 * Fmax * es);
         x.act = a.take(M * Fmax * es);
         x.logits = a.take(M * (size_t)c.vocab * 4);
-        x.draft_logits = a.take(Bm * (size_t)(c.k_max > 0 ? c.k_max : 1) * c.vocab * 4);
+        x.draft_logits = a.take(Bm * (size_t)(c.k_max > 0 ? c.k_max : 1) * c.vocab * 4);   // sized for the whole vocabulary
+        if (c.draft_vocab) {
+            x.t2d = a.take((size_t)c.vocab * 4);
+            x.draft_red = a.take(Bm * (size_t)(c.k_max > 0 ? c.k_max : 1) * 4);
+        }
         x.row_stats = a.take(M * 8);
         x.draft_row_stats = a.take(Bm * (size_t)(c.k_max > 0 ? c.k_max : 1) * 8);
         x.taps = a.take(M * (size_t)(c.n_taps > 0 ? c.n_taps : 1) * d * es);
@@ -419,6 +427,7 @@ extern "C" spec_status spec_tensor(spec_ctx* c, int id, int layer, void** dev_pt
     case SPEC_T_D_WGATEUP: base = c->buf.draft_weights; l = c->d_layer.wgateup; break;
     case SPEC_T_D_WDOWN: base = c->buf.draft_weights; l = c->d_layer.wdown; break;
     case SPEC_T_D_LM_HEAD: base = c->buf.draft_weights; l = c->d_lm_head; break;
+    case SPEC_T_D_D2T: base = c->buf.draft_weights; l = c->d_d2t; break;
     case SPEC_T_KV_K: case SPEC_T_KV_V:
         if (layer < 0 || layer >= g.kv_layer_pools) return SPEC_ERR_INVALID_ARG;
         base = c->buf.kv;
@@ -593,7 +602,10 @@ extern "C" spec_status spec_reject_sample(spec_ctx* c, int k, const float* draft
     if (draft_logits != nullptr && k > 0)
         TRY(launch_softmax_rows(B * k, g.vocab, ql, (size_t)g.vocab, g.temperature, qs, 1, nullptr, st));
     // draft tokens: those the verify used (rows 1..k of its token list), so an external draft stays consistent
+    // a draft head with its own smaller vocabulary: q rows are draft_vocab wide and looked up through the target-to-draft map
+    const bool mapped = draft_logits == nullptr && has_head && g.draft_vocab != 0;
     TIMED(*c, CLS_SAMPLE, launch_reject_sample(true, B, k, g.vocab, at<float>(ws, c->logits), at<float>(ws, c->row_stats), ql, qs,
+                                               mapped ? g.draft_vocab : g.vocab, mapped ? at<int32_t>(ws, c->t2d) : nullptr,
                                                at<int32_t>(ws, c->tokens_in) + 1, k + 1, g.temperature, g.seed,
                                                at<uint32_t>(sb, c->step), 0, at<int32_t>(sb, c->out_tokens),
                                                at<int32_t>(sb, c->n_emitted), at<int32_t>(sb, c->status), at<float>(sb, c->out_logp), st));
@@ -670,6 +682,10 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
     float* dstats = at<float>(ws, c->draft_row_stats);
     int32_t* dtoks = at<int32_t>(sb, c->draft_tokens);
     const int kstride = g.k_max;
+    const bool mapped = eagle && g.draft_vocab != 0;
+    const int Vd = mapped ? g.draft_vocab : V;
+    int32_t* dred = mapped ? at<int32_t>(ws, c->draft_red) : nullptr;
+    if (mapped) TRY(launch_build_t2d(V, Vd, at<const int32_t>(dw, c->d_d2t), at<int32_t>(ws, c->t2d), st));
 
     for (int j = 0; j < k; ++j) {
         const int R = j == 0 ? c->k_last + 1 : 1;
@@ -701,14 +717,16 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
         const float* nf = eagle ? at<const float>(dw, c->d_norm_f) : at<const float>(c->buf.weights, c->final_norm);
         const void* lm = eagle ? at<const void>(dw, c->d_lm_head) : at<const void>(c->buf.weights, c->lm_head);
         TRY(launch_rmsnorm(B, d, hid, nf, g.rms_eps, at(ws, c->h), d, 0, dt, st));
-        TRY(launch_gemm(B, V, d, at(ws, c->h), d, lm, dlog + (size_t)j * V, k * V, dt, SPEC_DTYPE_F32, 0, st));
+        TRY(launch_gemm(B, Vd, d, at(ws, c->h), d, lm, dlog + (size_t)j * Vd, k * Vd, dt, SPEC_DTYPE_F32, 0, st));
+        int32_t* tok_out = mapped ? dred + j : dtoks + j;          // reduced ids first when the head has its own vocabulary
         if (g.draft_greedy) {
-            TRY(launch_argmax_rows(B, V, dlog + (size_t)j * V, (size_t)k * V, dtoks + j, kstride, st));
+            TRY(launch_argmax_rows(B, Vd, dlog + (size_t)j * Vd, (size_t)k * Vd, tok_out, kstride, st));
         } else {
-            TRY(launch_softmax_rows(B, V, dlog + (size_t)j * V, (size_t)k * V, g.temperature, dstats + 2 * j, k, nullptr, st));
-            TRY(launch_sample_logits(B, V, dlog + (size_t)j * V, (size_t)k * V, dstats + 2 * j, k, g.temperature, g.seed,
-                                     at<uint32_t>(sb, c->step), (uint32_t)j, 1u, dtoks + j, kstride, status, st));
+            TRY(launch_softmax_rows(B, Vd, dlog + (size_t)j * Vd, (size_t)k * Vd, g.temperature, dstats + 2 * j, k, nullptr, st));
+            TRY(launch_sample_logits(B, Vd, dlog + (size_t)j * Vd, (size_t)k * Vd, dstats + 2 * j, k, g.temperature, g.seed,
+                                     at<uint32_t>(sb, c->step), (uint32_t)j, 1u, tok_out, kstride, status, st));
         }
+        if (mapped) TRY(launch_map_tokens(B, dred + j, kstride, at<const int32_t>(dw, c->d_d2t), dtoks + j, kstride, st));
     }
     return SPEC_OK;
 }

@@ -9,8 +9,10 @@ namespace spec {
 // row r at logits + r*row_stride; its (max, sum exp) at stats + 2*r*stats_stride; probs (nullable) [rows][V]
 spec_status launch_softmax_rows(int rows, int V, const float* logits, size_t row_stride, float temperature, float* stats,
                                 size_t stats_stride, float* probs, cudaStream_t st);
+// q rows are q_width wide; with t2d (target id -> row of q, or -1) the draft distribution lives on a subset of the vocabulary
 spec_status launch_reject_sample(bool from_logits, int B, int k, int V, const float* p, const float* p_stats,
-                                 const float* q, const float* q_stats, const int32_t* draft, int draft_stride,
+                                 const float* q, const float* q_stats, int q_width, const int32_t* t2d,
+                                 const int32_t* draft, int draft_stride,
                                  float temperature, uint64_t seed, const uint32_t* step_dev, uint32_t step,
                                  int32_t* out_tokens, int32_t* n_emitted, int32_t* status, float* out_logp, cudaStream_t st);
 // one token per row from logits and their statistics: uniform Philox(seed; *step_dev, row, slot, stream_tag)
@@ -20,6 +22,9 @@ spec_status launch_sample_logits(int rows, int V, const float* logits, size_t ro
                                  cudaStream_t st);
 spec_status launch_argmax_rows(int rows, int V, const float* logits, size_t row_stride, int32_t* tokens, int token_stride,
                                cudaStream_t st);
+spec_status launch_build_t2d(int V, int Vd, const int32_t* d2t, int32_t* t2d, cudaStream_t st);
+spec_status launch_map_tokens(int B, const int32_t* src, int src_stride, const int32_t* d2t, int32_t* dst, int dst_stride,
+                              cudaStream_t st);
 int sampler_max_vocab();
 
 // ops.cu: element-wise and bookkeeping kernels.  dtype = SPEC_DTYPE_* of the activation/weight/KV storage.

@@ -80,6 +80,30 @@ struct ResidualLogits {               // w = max(0, softmax(lp/T) - softmax(lq/T
     }
 };
 
+// A draft distribution over a subset of the vocabulary: q(x) = softmax(lq / T)[t2d[x]] where t2d[x] >= 0, else 0.
+struct MappedLogitRow {
+    LogitRow Q; const int32_t* t2d;
+    __device__ void load(int idx, int V, float (&w)[4]) const
+    {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int t = (idx + e < V) ? t2d[idx + e] : -1;
+            w[e] = t >= 0 ? prob_from_logit(Q.l[t], Q.m, Q.inv_t, Q.inv_z) : 0.f;
+        }
+    }
+};
+struct ResidualLogitsMapped {
+    LogitRow P; MappedLogitRow Q;
+    __device__ void load(int idx, int V, float (&w)[4]) const
+    {
+        float a[4], b[4];
+        P.load(idx, V, a);
+        Q.load(idx, V, b);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) w[e] = fmaxf(0.f, __fsub_rn(a[e], b[e]));
+    }
+};
+
 // Deterministic draft (q = one-hot(d)): the residual is p with the draft token's mass removed.
 template <class Row>
 struct ResidualOneHot {
@@ -322,6 +346,8 @@ struct RejectArgs {
     const float* q;            // [B][k][V]
     const float* p_stats;      // [B*(k+1)][2] (max, sum exp) when logits, else unused
     const float* q_stats;      // [B*k][2]
+    int Vq;                    // width of a q row (V unless the draft head has its own vocabulary)
+    const int32_t* t2d;        // [V] target id -> column of q, -1 outside the draft vocabulary; nullptr: identity
     const int32_t* draft;      // d_i of sequence b at draft[b*draft_stride + i]
     int draft_stride;
     float inv_t;
@@ -342,7 +368,8 @@ __global__ void __launch_bounds__(kThreads) reject_sample_kernel(const RejectArg
     const int b = blockIdx.x, k = A.k, V = A.V;
     const uint32_t step = A.step_dev ? *A.step_dev : A.step;
     const float* prow0 = A.p + (size_t)b * (k + 1) * V;
-    const float* qrow0 = A.q + (size_t)b * k * V;
+    const int Vq = A.Vq;
+    const float* qrow0 = A.q + (size_t)b * k * Vq;
 
     auto p_row = [&](int i) {
         const float* l = prow0 + (size_t)i * V;
@@ -354,10 +381,10 @@ __global__ void __launch_bounds__(kThreads) reject_sample_kernel(const RejectArg
         }
     };
     auto q_row = [&](int i) {
-        const float* l = qrow0 + (size_t)i * V;
+        const float* l = qrow0 + (size_t)i * Vq;
         if constexpr (kFromLogits) {
             const float* st = A.q_stats + 2 * ((size_t)b * k + i);
-            return LogitRow{l, st[0], __frcp_rn(st[1]), A.inv_t, row_vec_ok(l, V)};
+            return LogitRow{l, st[0], __frcp_rn(st[1]), A.inv_t, row_vec_ok(l, Vq)};
         } else {
             return ProbRow{l, row_vec_ok(l, V)};
         }
@@ -376,8 +403,11 @@ __global__ void __launch_bounds__(kThreads) reject_sample_kernel(const RejectArg
                 if constexpr (kFromLogits) {
                     const auto P = p_row(i);
                     pd = prob_from_logit(P.l[d], P.m, P.inv_t, P.inv_z);
-                    if (A.q != nullptr) { const auto Q = q_row(i); qd = prob_from_logit(Q.l[d], Q.m, Q.inv_t, Q.inv_z); }
-                    else qd = 1.f;                                   // deterministic draft: q = one-hot(d)
+                    if (A.q != nullptr) {
+                        const auto Q = q_row(i);
+                        const int dq = A.t2d != nullptr ? A.t2d[d] : d;            // a token outside the draft vocabulary has q = 0
+                        qd = dq >= 0 ? prob_from_logit(Q.l[dq], Q.m, Q.inv_t, Q.inv_z) : 0.f;
+                    } else qd = 1.f;                                 // deterministic draft: q = one-hot(d)
                 } else {
                     pd = prow0[(size_t)i * V + d];
                     qd = A.q != nullptr ? qrow0[(size_t)i * V + d] : 1.f;
@@ -405,7 +435,10 @@ __global__ void __launch_bounds__(kThreads) reject_sample_kernel(const RejectArg
             token = block_invcdf(p_row(n), V, u_last, sm);
         }
     } else if (n < k) {
-        if constexpr (kFromLogits) token = block_invcdf(ResidualLogits{p_row(n), q_row(n)}, V, u_last, sm);
+        if constexpr (kFromLogits) {
+            if (A.t2d != nullptr) token = block_invcdf(ResidualLogitsMapped{p_row(n), MappedLogitRow{q_row(n), A.t2d}}, V, u_last, sm);
+            else                  token = block_invcdf(ResidualLogits{p_row(n), q_row(n)}, V, u_last, sm);
+        }
         else                       token = block_invcdf(ResidualProbs{prow0 + (size_t)n * V, qrow0 + (size_t)n * V,
                                                                       row_vec_ok(prow0 + (size_t)n * V, V) &&
                                                                       row_vec_ok(qrow0 + (size_t)n * V, V)}, V, u_last, sm);
@@ -460,12 +493,13 @@ spec_status launch_softmax_rows(int rows, int V, const float* logits, size_t row
 }
 
 spec_status launch_reject_sample(bool from_logits, int B, int k, int V, const float* p, const float* p_stats,
-                                 const float* q, const float* q_stats, const int32_t* draft, int draft_stride,
+                                 const float* q, const float* q_stats, int q_width, const int32_t* t2d,
+                                 const int32_t* draft, int draft_stride,
                                  float temperature, uint64_t seed, const uint32_t* step_dev, uint32_t step,
                                  int32_t* out_tokens, int32_t* n_emitted, int32_t* status, float* out_logp, cudaStream_t st)
 {
     if (B == 0) return SPEC_OK;
-    RejectArgs A{B, k, V, p, q, p_stats, q_stats, draft, draft_stride, 1.0f / temperature, seed, step_dev, step, out_tokens,
+    RejectArgs A{B, k, V, p, q, p_stats, q_stats, q_width, t2d, draft, draft_stride, 1.0f / temperature, seed, step_dev, step, out_tokens,
                  n_emitted, status, out_logp};
     if (from_logits) reject_sample_kernel<true><<<B, kThreads, 0, st>>>(A);
     else             reject_sample_kernel<false><<<B, kThreads, 0, st>>>(A);
@@ -488,6 +522,35 @@ spec_status launch_argmax_rows(int rows, int V, const float* logits, size_t row_
 {
     if (rows == 0) return SPEC_OK;
     argmax_rows_kernel<<<rows, kThreads, 0, st>>>(V, logits, row_stride, tokens, token_stride);
+    return launch_status();
+}
+
+// target-to-draft map of a draft head with its own vocabulary: t2d[x] = r where d2t[r] = x, -1 elsewhere
+__global__ void build_t2d_kernel(int V, int Vd, const int32_t* __restrict__ d2t, int32_t* __restrict__ t2d, int phase)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (phase == 0) { if (i < V) t2d[i] = -1; }
+    else if (i < Vd) { const int x = d2t[i]; if (x >= 0 && x < V) t2d[x] = i; }
+}
+__global__ void map_tokens_kernel(int B, const int32_t* __restrict__ src, int src_stride, const int32_t* __restrict__ d2t,
+                                  int32_t* __restrict__ dst, int dst_stride)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B) dst[(size_t)b * dst_stride] = d2t[src[(size_t)b * src_stride]];
+}
+
+spec_status launch_build_t2d(int V, int Vd, const int32_t* d2t, int32_t* t2d, cudaStream_t st)
+{
+    build_t2d_kernel<<<(V + 255) / 256, 256, 0, st>>>(V, Vd, d2t, t2d, 0);
+    build_t2d_kernel<<<(Vd + 255) / 256, 256, 0, st>>>(V, Vd, d2t, t2d, 1);
+    return launch_status(2);
+}
+
+spec_status launch_map_tokens(int B, const int32_t* src, int src_stride, const int32_t* d2t, int32_t* dst, int dst_stride,
+                              cudaStream_t st)
+{
+    if (B == 0) return SPEC_OK;
+    map_tokens_kernel<<<(B + 255) / 256, 256, 0, st>>>(B, src, src_stride, d2t, dst, dst_stride);
     return launch_status();
 }
 
@@ -527,7 +590,7 @@ extern "C" spec_status spec_reject_sample_probs(int B, int k, int V, const float
     if (p == nullptr || out_tokens == nullptr || n_emitted == nullptr) return SPEC_ERR_INVALID_ARG;
     if (k > 0 && draft == nullptr) return SPEC_ERR_INVALID_ARG;       // q == NULL: deterministic drafts, q = one-hot(d)
     if (V > sampler_max_vocab()) return SPEC_ERR_SHAPE;
-    return launch_reject_sample(false, B, k, V, p, nullptr, q, nullptr, draft, k, 1.0f, seed, nullptr, step, out_tokens,
+    return launch_reject_sample(false, B, k, V, p, nullptr, q, nullptr, V, nullptr, draft, k, 1.0f, seed, nullptr, step, out_tokens,
                                 n_emitted, status, nullptr, (cudaStream_t)stream);
 }
 
@@ -542,7 +605,7 @@ extern "C" spec_status spec_reject_sample_logits(int B, int k, int V, const floa
         return SPEC_ERR_INVALID_ARG;
     if (k > 0 && (draft == nullptr || (q_logits != nullptr && q_stats == nullptr))) return SPEC_ERR_INVALID_ARG;
     if (V > sampler_max_vocab()) return SPEC_ERR_SHAPE;
-    return launch_reject_sample(true, B, k, V, p_logits, p_stats, q_logits, q_stats, draft, k, temperature, seed, nullptr,
+    return launch_reject_sample(true, B, k, V, p_logits, p_stats, q_logits, q_stats, V, nullptr, draft, k, temperature, seed, nullptr,
                                 step, out_tokens, n_emitted, status, nullptr, (cudaStream_t)stream);
 }
 

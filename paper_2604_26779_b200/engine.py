@@ -15,7 +15,8 @@ from .binding import T
 
 def make_spec_config(cfg: dict, *, draft_kind: str = "none", k_max: int = 3, max_batch: int = 4, kv_num_blocks: int = 64,
                      max_blocks_per_seq: int = 16, kv_block_tokens: int = 16, kv_layer_pools: int | None = None,
-                     seed: int = 0, draft_d_ffn: int | None = None, ngram_n: int = 3, draft_greedy: bool = False) -> B.spec_config:
+                     seed: int = 0, draft_d_ffn: int | None = None, ngram_n: int = 3, draft_greedy: bool = False,
+                     draft_vocab: int = 0) -> B.spec_config:
     sc = B.spec_config()
     sc.struct_size, sc.abi_version = C.sizeof(B.spec_config), B.SPEC_ABI_VERSION
     for name in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab", "n_experts",
@@ -27,6 +28,7 @@ def make_spec_config(cfg: dict, *, draft_kind: str = "none", k_max: int = 3, max
     sc.draft_d_ffn = int(draft_d_ffn if draft_d_ffn is not None else (cfg["d_ffn"] or 4 * cfg["d_model"])) if draft_kind in ("eagle3", "mtp") else 0
     sc.ngram_n = int(ngram_n) if draft_kind == "ngram" else 0
     sc.draft_greedy = 1 if draft_greedy else 0
+    sc.draft_vocab = int(draft_vocab) if draft_kind == "eagle3" else 0
     taps = tuple(cfg.get("tap_layers", ())) if draft_kind == "eagle3" else ()
     sc.n_taps = len(taps)
     for i, t in enumerate(taps):
@@ -148,6 +150,9 @@ class SpecStep:
             self.put("D_WFC", 0, H["wfc"])
             self.put("D_NORM_F", 0, H["norm_f"], f32)
             self.put("D_LM_HEAD", 0, H["lm_head"])
+            if self.sc.draft_vocab:
+                assert H["lm_head"].shape[0] == self.sc.draft_vocab and len(H["d2t"]) == self.sc.draft_vocab
+                self.put("D_D2T", 0, np.asarray(H["d2t"], np.int32), torch.int32)
         else:
             self.put("D_WPROJ", 0, H["wproj"])
             self.put("D_ATTN_NORM", 0, H["attn_norm"], f32)
@@ -200,7 +205,7 @@ class SpecStep:
         return self.tensor("LOGITS", 0, torch.float32, (self.B, k + 1, self.sc.vocab))
 
     def draft_logits(self, k):
-        return self.tensor("DRAFT_LOGITS", 0, torch.float32, (self.B, k, self.sc.vocab))
+        return self.tensor("DRAFT_LOGITS", 0, torch.float32, (self.B, k, self.sc.draft_vocab or self.sc.vocab))
 
     def out_tokens(self, k):
         return self.tensor("OUT_TOKENS", 0, torch.int32, (self.B, k + 1))

@@ -113,9 +113,12 @@ def make_eagle3_weights(cfg: dict, seed: int, std=0.02) -> dict:
     dense = dict(cfg, n_experts=0, d_ffn=cfg["d_ffn"] or 4 * d)
     H = make_layer_weights(dense, rng, std, qkv_in=2 * d)
     del H["attn_norm"]
+    Vd = int(cfg.get("draft_vocab") or 0)
     H.update(wfc=_normal(rng, (d, len(cfg["tap_layers"]) * d), std, dt),
              norm_e=np.ones(d, np.float32), norm_g=np.ones(d, np.float32), norm_f=np.ones(d, np.float32),
-             lm_head=_normal(rng, (V, d), std, dt))
+             lm_head=_normal(rng, (Vd or V, d), std, dt))
+    if Vd:      # the head's own vocabulary: a seeded subset of the target's ids, in increasing order
+        H["d2t"] = np.sort(rng.choice(V, size=Vd, replace=False)).astype(np.int32)
     return H
 
 

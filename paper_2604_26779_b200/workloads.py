@@ -45,7 +45,8 @@ def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, l
 
     def sizes_for(G):
         sc = engine.make_spec_config(cfg, draft_kind=draft, k_max=k, max_batch=B, kv_num_blocks=num_blocks,
-                                     max_blocks_per_seq=max_blocks, kv_layer_pools=G, seed=seed)
+                                     max_blocks_per_seq=max_blocks, kv_layer_pools=G, seed=seed,
+                                     draft_vocab=int(cfg.get("draft_vocab") or 0), draft_greedy=bool(cfg.get("draft_greedy")))
         from . import binding as Bd
         import ctypes as C
         s = Bd.spec_sizes()
@@ -85,6 +86,10 @@ def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, l
             eng.tensor(nm, 0, f32).fill_(1.0)
         for nm in ("D_WQKV", "D_WO", "D_WGATEUP", "D_WDOWN") + (("D_WFC", "D_LM_HEAD") if draft == "eagle3" else ("D_WPROJ",)):
             _fill_normal(eng.tensor(nm, 0, bf), 0.02, gen)
+        if draft == "eagle3" and cfg.get("draft_vocab"):      # the head's id set: a seeded subset of the vocabulary, increasing
+            rng = np.random.Generator(np.random.PCG64(seed + 4))
+            d2t = np.sort(rng.choice(cfg["vocab"], size=int(cfg["draft_vocab"]), replace=False)).astype(np.int32)
+            eng.tensor("D_D2T", 0, torch.int32).copy_(torch.from_numpy(d2t).to(device))
         _fill_normal(eng.tensor("DRAFT_KV_K", 0, bf), 1.0, gen)
         _fill_normal(eng.tensor("DRAFT_KV_V", 0, bf), 1.0, gen)
     for p in range(G):

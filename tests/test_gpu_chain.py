@@ -32,7 +32,8 @@ def run_chain(engine, cfg, kind, B, prompt_len, k, n_steps, seed, prompts=None):
         prompts = inputs.make_prompts(B, prompt_len, cfg["vocab"], seed=inputs.sub_seed(1, 2))
     max_blocks = -(-(prompt_len + n_steps * (k + 1) + k + 2) // 16)
     sc = engine.make_spec_config(cfg, draft_kind=kind, k_max=k, max_batch=B, kv_num_blocks=B * max_blocks + 3,
-                                 max_blocks_per_seq=max_blocks, seed=seed, draft_greedy=bool(cfg.get("draft_greedy")))
+                                 max_blocks_per_seq=max_blocks, seed=seed, draft_greedy=bool(cfg.get("draft_greedy")),
+                                 draft_vocab=int(cfg.get("draft_vocab") or 0))
     eng = engine.SpecStep(sc)
     eng.load_target_weights(W)
     if H is not None:
@@ -164,6 +165,17 @@ def test_chain_greedy_head_drafts_lockstep(eng_mod):
     assert r["max_rel"] < 1e-3 and r["max_rel_d"] < 1e-3 and r["boundary"] <= 2
     assert r["emitted"] >= r["steps"]      # a random target accepts an arg-max draft with probability ~1/vocab: the accepted
                                            # branch of the one-hot rule is covered by the sampler tests
+
+
+def test_chain_draft_head_with_its_own_vocabulary(eng_mod):
+    """EAGLE-3-style head whose LM head covers a quarter of the vocabulary: q is zero outside its id set, the residual
+    still runs over the whole vocabulary; sampled and greedy drafting."""
+    cfg = dict(inputs.model_config("c1"), draft_vocab=256)
+    r = run_chain(eng_mod, cfg, "eagle3", B=3, prompt_len=32, k=3, n_steps=24, seed=909)
+    print("reduced draft vocabulary:", r)
+    assert r["max_rel"] < 1e-3 and r["max_rel_d"] < 1e-3 and r["boundary"] <= 2 and r["emitted"] > r["steps"]
+    r = run_chain(eng_mod, dict(cfg, draft_greedy=True), "eagle3", B=2, prompt_len=18, k=2, n_steps=8, seed=910)
+    assert r["max_rel"] < 1e-3 and r["boundary"] <= 1
 
 
 def test_chain_at_other_temperature_and_k1(eng_mod):
