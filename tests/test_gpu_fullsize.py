@@ -22,6 +22,9 @@ pytestmark = pytest.mark.gpu
 def test_full_size_step_sampled_against_oracle():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < 60e9:
         pytest.skip("needs a device with > 60 GB free")
@@ -104,6 +107,9 @@ def test_attention_at_bench_sizes_sampled(name, B, R, Hq, Hkv, lens_kind):
     placement must agree bit for bit."""
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()                                    # memory cached by earlier tests of this process counts as free
     free, _ = torch.cuda.mem_get_info()
     if free < 40e9:
         pytest.skip("needs a device with > 40 GB free")
