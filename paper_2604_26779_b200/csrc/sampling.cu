@@ -124,27 +124,82 @@ struct InvCdfSmem {
 // Block-wide inverse CDF: the smallest v with  sum_{j<=v} w_j > u * sum_j w_j  (strict; a zero-weight bin is never
 // chosen); if rounding leaves every prefix at or below the target, the last positive bin.  Returns -1 when the row
 // has no positive finite mass.  All threads of the block must call it; all get the result.
+// The fp64 sum of one 512-element chunk of weights (one warp; the same fp32 tree in every caller, so that whoever computes
+// a chunk gets the same number).
+template <class WF>
+__device__ __forceinline__ double chunk_sum_of(const WF& wf, int V, int c, int lane)
+{
+    const int base = c * kChunk + lane * 4;
+    float w[16];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) wf.load(base + s * 128, V, *reinterpret_cast<float(*)[4]>(&w[4 * s]));
+    float part[4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) part[s] = (w[4 * s] + w[4 * s + 1]) + (w[4 * s + 2] + w[4 * s + 3]);
+    return warp_sum((double)((part[0] + part[1]) + (part[2] + part[3])));
+}
+
+template <class WF> __device__ int invcdf_select(const WF& wf, int V, float u, InvCdfSmem& sm);
+
 template <class WF>
 __device__ int block_invcdf(const WF& wf, int V, float u, InvCdfSmem& sm)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nchunks = (V + kChunk - 1) / kChunk;
     __syncthreads();                                         // the shared buffer may still be in use by a previous draw
-
     // pass over the row: one fp64 sum per chunk
     for (int c = warp; c < nchunks; c += (int)(blockDim.x >> 5)) {
-        const int base = c * kChunk + lane * 4;
-        float w[16];
-#pragma unroll
-        for (int s = 0; s < 4; ++s) wf.load(base + s * 128, V, *reinterpret_cast<float(*)[4]>(&w[4 * s]));
-        float part[4];
-#pragma unroll
-        for (int s = 0; s < 4; ++s) part[s] = (w[4 * s] + w[4 * s + 1]) + (w[4 * s + 2] + w[4 * s + 3]);
-        const double d = warp_sum((double)((part[0] + part[1]) + (part[2] + part[3])));
+        const double d = chunk_sum_of(wf, V, c, lane);
         if (lane == 0) sm.chunk_sum[c] = d;
     }
     __syncthreads();
+    return invcdf_select(wf, V, u, sm);
+}
 
+// ---- the same draw by a cluster of CTAs: with a few hundred sequences one CTA per sequence leaves most of the machine
+// idle, so kClusterCtas CTAs share the pass over the row; each writes its chunk sums straight into the first CTA's table
+// through distributed shared memory, and that CTA scans them and takes the second look.  The sums are the same numbers
+// whoever computes them, so the drawn token does not depend on the cluster size.
+constexpr int kClusterCtas = 4;
+__device__ __forceinline__ uint32_t cluster_cta_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_cluster_f64(uint32_t local_saddr, uint32_t target_rank, double v)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_saddr), "r"(target_rank));
+    asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(remote), "d"(v) : "memory");
+}
+// All CTAs of the cluster must call it with the same functor; returns the token in the first CTA and -2 in the others
+// (which have nothing left to do).
+template <class WF>
+__device__ int cluster_invcdf(const WF& wf, int V, float u, InvCdfSmem& sm)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nchunks = (V + kChunk - 1) / kChunk;
+    const uint32_t rank = cluster_cta_rank();
+    const uint32_t table = (uint32_t)__cvta_generic_to_shared(&sm.chunk_sum[0]);
+    for (int c = (int)rank * kWarps + warp; c < nchunks; c += kClusterCtas * kWarps) {
+        const double d = chunk_sum_of(wf, V, c, lane);
+        if (lane == 0) st_cluster_f64(table + (uint32_t)c * 8u, 0u, d);
+    }
+    cluster_sync_all();                                      // every sum has landed in the first CTA's table
+    if (rank != 0) return -2;
+    return invcdf_select(wf, V, u, sm);
+}
+
+template <class WF>
+__device__ int invcdf_select(const WF& wf, int V, float u, InvCdfSmem& sm)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nchunks = (V + kChunk - 1) / kChunk;
     if (warp == 0) {
         // scan of the chunk sums: every lane owns a contiguous range of chunks
         const int per = (nchunks + 31) / 32;
@@ -292,6 +347,7 @@ __global__ void __launch_bounds__(kThreads) sample_rows_kernel(int V, const floa
 }
 
 // one token per row from logits and their statistics (the draft head's d_i ~ q_i)
+template <bool kCluster>
 __global__ void __launch_bounds__(kThreads) sample_logits_kernel(int V, const float* __restrict__ logits, size_t row_stride,
                                                                  const float* __restrict__ stats, size_t stats_stride,
                                                                  float inv_t, uint64_t seed, const uint32_t* step_dev,
@@ -300,11 +356,19 @@ __global__ void __launch_bounds__(kThreads) sample_logits_kernel(int V, const fl
                                                                  int32_t* status)
 {
     __shared__ InvCdfSmem sm;
-    const int row = blockIdx.x;
+    const int row = kCluster ? blockIdx.x / kClusterCtas : blockIdx.x;
     const float* l = logits + (size_t)row * row_stride;
     const float* st = stats + 2 * (size_t)row * stats_stride;
     const float u = philox_uniform(seed, *step_dev, (uint32_t)row, slot, stream_tag);
-    int t = block_invcdf(LogitRow{l, st[0], __frcp_rn(st[1]), inv_t, row_vec_ok(l, V)}, V, u, sm);
+    const LogitRow wf{l, st[0], __frcp_rn(st[1]), inv_t, row_vec_ok(l, V)};
+    int t;
+    if constexpr (kCluster) {
+        cluster_sync_all();                                  // the first CTA's table exists before anyone writes to it
+        t = cluster_invcdf(wf, V, u, sm);
+        if (t == -2) return;
+    } else {
+        t = block_invcdf(wf, V, u, sm);
+    }
     if (threadIdx.x == 0) {
         if (t < 0) { set_status(status, SPEC_ERR_BAD_PROB, row); t = 0; }
         tokens[(size_t)row * token_stride] = t;
@@ -360,12 +424,19 @@ struct RejectArgs {
     float* out_logp;           // [B][k+1] log p_target(emitted token) under the verifier, or nullptr
 };
 
-template <bool kFromLogits>
+template <bool kFromLogits, bool kCluster>
 __global__ void __launch_bounds__(kThreads) reject_sample_kernel(const RejectArgs A)
 {
     __shared__ InvCdfSmem sm;
     __shared__ int s_n;
-    const int b = blockIdx.x, k = A.k, V = A.V;
+    const int b = kCluster ? blockIdx.x / kClusterCtas : blockIdx.x, k = A.k, V = A.V;
+    if constexpr (kCluster) cluster_sync_all();              // the first CTA's table exists before anyone writes to it
+    // the first draw is shared by the CTAs of a cluster (every CTA takes the same branch: the accept tests below are
+    // recomputed by each); whatever follows it is the first CTA's alone
+    auto draw = [&](const auto& wf, float u) {
+        if constexpr (kCluster) return cluster_invcdf(wf, V, u, sm);
+        else                    return block_invcdf(wf, V, u, sm);
+    };
     const uint32_t step = A.step_dev ? *A.step_dev : A.step;
     const float* prow0 = A.p + (size_t)b * (k + 1) * V;
     const int Vq = A.Vq;
@@ -429,25 +500,28 @@ __global__ void __launch_bounds__(kThreads) reject_sample_kernel(const RejectArg
     int token;
     if (n < k && A.q == nullptr) {
         const int dn = A.draft[(size_t)b * A.draft_stride + n];
-        token = block_invcdf(ResidualOneHot<decltype(p_row(n))>{p_row(n), dn}, V, u_last, sm);
+        token = draw(ResidualOneHot<decltype(p_row(n))>{p_row(n), dn}, u_last);
+        if (token == -2) return;
         if (token < 0) {
             if (threadIdx.x == 0) set_status(A.status, SPEC_ERR_BAD_PROB, b);
             token = block_invcdf(p_row(n), V, u_last, sm);
         }
     } else if (n < k) {
         if constexpr (kFromLogits) {
-            if (A.t2d != nullptr) token = block_invcdf(ResidualLogitsMapped{p_row(n), MappedLogitRow{q_row(n), A.t2d}}, V, u_last, sm);
-            else                  token = block_invcdf(ResidualLogits{p_row(n), q_row(n)}, V, u_last, sm);
+            if (A.t2d != nullptr) token = draw(ResidualLogitsMapped{p_row(n), MappedLogitRow{q_row(n), A.t2d}}, u_last);
+            else                  token = draw(ResidualLogits{p_row(n), q_row(n)}, u_last);
         }
-        else                       token = block_invcdf(ResidualProbs{prow0 + (size_t)n * V, qrow0 + (size_t)n * V,
-                                                                      row_vec_ok(prow0 + (size_t)n * V, V) &&
-                                                                      row_vec_ok(qrow0 + (size_t)n * V, V)}, V, u_last, sm);
+        else                       token = draw(ResidualProbs{prow0 + (size_t)n * V, qrow0 + (size_t)n * V,
+                                                              row_vec_ok(prow0 + (size_t)n * V, V) &&
+                                                              row_vec_ok(qrow0 + (size_t)n * V, V)}, u_last);
+        if (token == -2) return;
         if (token < 0) {                                       // residual without mass: garbage input
             if (threadIdx.x == 0) set_status(A.status, SPEC_ERR_BAD_PROB, b);
             token = block_invcdf(p_row(n), V, u_last, sm);
         }
     } else {
-        token = block_invcdf(p_row(k), V, u_last, sm);
+        token = draw(p_row(k), u_last);
+        if (token == -2) return;
     }
     if (token < 0) {
         if (threadIdx.x == 0) set_status(A.status, SPEC_ERR_BAD_PROB, b);
@@ -492,6 +566,26 @@ spec_status launch_softmax_rows(int rows, int V, const float* logits, size_t row
     return launch_status();
 }
 
+namespace {
+constexpr int kClusterBatchLimit = 512;          // above this one CTA per sequence already fills the machine
+template <class... KArgs, class... Args>
+spec_status launch_clustered(void (*kernel)(KArgs...), int n_seq, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)n_seq * kClusterCtas);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = kClusterCtas; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) != cudaSuccess) { cudaGetLastError(); return SPEC_ERR_CUDA; }
+    return launch_status();
+}
+}  // namespace
+
 spec_status launch_reject_sample(bool from_logits, int B, int k, int V, const float* p, const float* p_stats,
                                  const float* q, const float* q_stats, int q_width, const int32_t* t2d,
                                  const int32_t* draft, int draft_stride,
@@ -501,8 +595,13 @@ spec_status launch_reject_sample(bool from_logits, int B, int k, int V, const fl
     if (B == 0) return SPEC_OK;
     RejectArgs A{B, k, V, p, q, p_stats, q_stats, q_width, t2d, draft, draft_stride, 1.0f / temperature, seed, step_dev, step, out_tokens,
                  n_emitted, status, out_logp};
-    if (from_logits) reject_sample_kernel<true><<<B, kThreads, 0, st>>>(A);
-    else             reject_sample_kernel<false><<<B, kThreads, 0, st>>>(A);
+    // few sequences: a cluster of CTAs per sequence, so that the pass over the vocabulary uses the whole machine
+    if (B <= kClusterBatchLimit) {
+        if (from_logits) return launch_clustered(reject_sample_kernel<true, true>, B, st, A);
+        return launch_clustered(reject_sample_kernel<false, true>, B, st, A);
+    }
+    if (from_logits) reject_sample_kernel<true, false><<<B, kThreads, 0, st>>>(A);
+    else             reject_sample_kernel<false, false><<<B, kThreads, 0, st>>>(A);
     return launch_status();
 }
 
@@ -512,8 +611,11 @@ spec_status launch_sample_logits(int rows, int V, const float* logits, size_t ro
                                  cudaStream_t st)
 {
     if (rows == 0) return SPEC_OK;
-    sample_logits_kernel<<<rows, kThreads, 0, st>>>(V, logits, row_stride, stats, stats_stride, 1.0f / temperature, seed,
-                                                    step_dev, slot, stream_tag, tokens, token_stride, status);
+    if (rows <= kClusterBatchLimit)
+        return launch_clustered(sample_logits_kernel<true>, rows, st, V, logits, row_stride, stats, stats_stride, 1.0f / temperature,
+                                seed, step_dev, slot, stream_tag, tokens, token_stride, status);
+    sample_logits_kernel<false><<<rows, kThreads, 0, st>>>(V, logits, row_stride, stats, stats_stride, 1.0f / temperature, seed,
+                                                           step_dev, slot, stream_tag, tokens, token_stride, status);
     return launch_status();
 }
 
