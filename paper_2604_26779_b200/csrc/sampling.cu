@@ -6,7 +6,8 @@
 // statistics) or one sequence (sampling); lanes read 16 bytes at consecutive addresses; the row of weights is
 // reduced to one fp64 sum per 512-element chunk in shared memory, the chunk holding the u-quantile is found by a
 // scan over those sums, and only that chunk is read a second time to locate the token.  So a draw costs one pass
-// over the row(s) it samples from, not two.
+// over the row(s) it samples from, not two.  With at most a few hundred sequences a cluster of four CTAs shares that pass
+// (distributed shared memory carries the chunk sums to the CTA that scans them).
 #include "ops.cuh"
 
 namespace spec {
