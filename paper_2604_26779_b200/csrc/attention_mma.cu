@@ -61,7 +61,9 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(int B, int R, c
         int ntok = 0, nc = 0, per = 0;
         if (b < B) {
             for (int i = 0; i < R; ++i) ntok = max(ntok, pos[(size_t)b * R + i] + 1);
-            nc = (ntok + kChunk - 1) / kChunk;
+            // a few tokens past a multiple of the chunk length (the k+1 new rows on top of a round cache length) do not
+            // open another chunk: a chunk may run up to kChunkSlack tokens over
+            nc = ntok > 0 ? max(1, (ntok - kChunkSlack + kChunk - 1) / kChunk) : 0;
             if (nc > 0) {
                 per = ((ntok + nc - 1) / nc + kTileTok - 1) / kTileTok * kTileTok;
                 nc = (ntok + per - 1) / per;
