@@ -412,3 +412,39 @@ def test_amdahl_bound_against_paper_tables(golden_dir):
         ro, e2e = g[f"sim_rollout_{s}"], g[f"sim_e2e_{s}"]
         shares.append((1 - 1 / e2e) / (1 - 1 / ro))
     assert max(shares) - min(shares) < 0.005 and abs(np.mean(shares) - 0.65) < 0.005
+
+
+def test_kv_bookkeeping_random_walk_with_replacement():
+    """Random sequences of reserve / commit / replace / retire: blocks are conserved, no block is owned twice, every live
+    sequence owns exactly the blocks its length needs after a commit, retired slots own nothing and are passed over."""
+    rng = np.random.default_rng(12)
+    B, bt, maxb, nblk, k = 6, 16, 10, 40, 3
+    seq_len = np.zeros(B, np.int32)
+    table = np.full((B, maxb), -1, np.int32)
+    free = inputs.make_block_order(nblk, 9)
+    top = np.array([nblk], np.int32)
+    everything = set(free.tolist())
+    for it in range(400):
+        live = seq_len >= 0
+        if oracle.kv_reserve(k, bt, seq_len, table, free, top) == 0:
+            n = rng.integers(1, k + 2, B).astype(np.int32)
+            before = seq_len.copy()
+            oracle.kv_commit(bt, n, seq_len, table, free, top)
+            assert np.all(seq_len[live] == before[live] + n[live]) and np.all(seq_len[~live] == -1)
+        owned = table[table >= 0]
+        assert len(set(owned.tolist())) == owned.size and owned.size + top[0] == nblk
+        assert set(owned.tolist()) | set(free[: top[0]].tolist()) == everything
+        for b in range(B):
+            keep = 0 if seq_len[b] < 0 else -(-int(seq_len[b]) // bt)
+            assert np.all(table[b, :keep] >= 0) and np.all(table[b, keep:] == -1)
+        # finished or overlong sequences leave; their slot gets a new prompt, or retires
+        leave = [b for b in range(B) if seq_len[b] >= 0 and (seq_len[b] + k + 1 > (maxb - 1) * bt or rng.random() < 0.05)]
+        back = [b for b in range(B) if seq_len[b] < 0 and rng.random() < 0.3]
+        if leave or back:
+            slots = leave + back
+            new_len = [int(rng.choice([-1, 0, 5, 33])) for _ in leave] + [int(rng.choice([0, 17])) for _ in back]
+            r = oracle.kv_replace(slots, new_len, bt, seq_len, table, free, top)
+            assert r in (0, -1)
+            if r == 0:
+                for s_, nl in zip(slots, new_len):
+                    assert seq_len[s_] == (nl if nl >= 0 else -1)
