@@ -3,23 +3,23 @@
 // With more than 16 query rows per KV head (long drafts, wide query groups: 64 rows for a 16-head group at k = 3) the
 // register-fragment kernel re-reads every K/V tile from shared memory once per 16 rows and runs out of shared-memory
 // bandwidth and issue slots before it runs out of HBM.  Here the rows are the M dimension of tcgen05.mma, which reads
-// its operands from shared memory once per tile whatever M is:
-//   - work units (sequence, KV head, chunk of <= 4096 tokens) come from the same plan and atomic counter as the
+// its operands once per tile whatever M is:
+//   - work units (sequence, KV head, chunk of about 4096 tokens) come from the same plan and atomic counter as the
 //     register-fragment kernel; one persistent CTA per SM;
 //   - four producer warps stream the K and V tiles of 128 tokens with TMA straight from the paged pools: one 64-column
 //     x 16-row box per (block, half of head_dim), 128-byte swizzle, so a tile lands as [half][token][64] - K-major for
-//     S = Q K^T and MN-major for O += P V - in two 2-stage rings; warp 0 also pulls the units and publishes them;
+//     S = Q K^T and MN-major for O += P V - in a 4-stage K ring and a 3-stage V ring, which is all that shared memory
+//     holds; warp 0 also pulls the units and publishes them to the other roles through a small queue;
 //   - warp 1 issues the MMAs from one thread: S (128 x 128, fp32) into one of two tensor-memory buffers, O (128 x 128)
-//     accumulated in a third;
+//     accumulated in a third; both A operands, Q and P, are read from tensor memory (bf16 pairs);
 //   - warps 2..5 are the softmax; query rows are dealt round-robin over the four 32-lane quarters of tensor memory and
 //     the scores are read in the 16-lane fragment shape, so the 32 threads of a warp share the columns of 16 rows (the
-//     exponentials, 4 per clock and scheduler whatever the number of active lanes, are what a tile costs).  Row maximum and exponentials in the exp2 domain; the
-//     running maximum is only raised when a tile exceeds it by more than 2^8 (the accumulator and the row sum are then
-//     rescaled in tensor memory), otherwise the stale maximum is kept - the final division makes both exact; P is
-//     written back to tensor memory as bf16 pairs, from where the second MMA takes it as its A operand;
-//   - per unit the softmax threads stage Q (zero-padded to 128 rows) in tensor memory, from where the first MMA takes it
-//     as its A operand, and write the result: normalised bf16 for
-//     single-chunk sequences, (max, sum, unnormalised fp32 row) partials for the merge kernel otherwise.
+//     exponentials, 4 per clock and scheduler whatever the number of active lanes, are what a tile costs).  Row maximum
+//     and exponentials in the exp2 domain; the running maximum is only raised when a tile exceeds it by more than 2^8
+//     (the accumulator and the row sum are then rescaled in tensor memory), otherwise the stale maximum is kept - the
+//     final division makes both exact; P goes back to tensor memory with one store per 16 rows;
+//   - per unit the softmax threads stage Q (zero-padded to 128 rows) in tensor memory and write the result: normalised
+//     bf16 for single-chunk sequences, (max, sum, unnormalised fp32 row) partials for the merge kernel otherwise.
 // Every mbarrier wait is bounded (abort flag -> SPEC_ERR_TIMEOUT, tensor memory released, kernel returns).
 #include <cuda.h>
 
@@ -35,7 +35,7 @@ constexpr int DH = 128, T = 128;                  // head_dim; KV tokens per til
 constexpr int kThreadsTc = 288;                  // warps: 0, 7 K producers; 6, 8 V producers; 1 MMA; 2..5 softmax
 constexpr int kSoftmaxThreads = 128;
 constexpr int kHalfBytes = 128 * 128;             // [128 rows][64 bf16], 128-byte rows, swizzled
-constexpr int kTileBytes = 2 * kHalfBytes;        // Q, P, one K tile, one V tile
+constexpr int kTileBytes = 2 * kHalfBytes;        // one K tile or one V tile of 128 tokens
 constexpr int kStagesK = 4, kStagesV = 3;         // K is needed a tile earlier than V
 constexpr int NQ = 4;                             // unit queue depth (the producer runs ahead of the consumers)
 constexpr uint32_t kTmemCols = 512;               // S0 [0,128), S1 [128,256), O [256,384), Q [384,448) and P [448,512) as bf16 pairs
