@@ -32,14 +32,14 @@ namespace attn {
 namespace {
 
 constexpr int DH = 128, T = 128;                  // head_dim; KV tokens per tile
-constexpr int kThreadsTc = 288;                  // warps: 0, 7 K producers; 6, 8 V producers; 1 MMA; 2..5 softmax
-constexpr int kSoftmaxThreads = 128;
+constexpr int kThreadsTc = 416;                  // warps: 0, 7 K producers; 6, 8 V producers; 1 MMA; 2..5 and 9..12 softmax
+constexpr int kSoftmaxThreads = 256;
 constexpr int kHalfBytes = 128 * 128;             // [128 rows][64 bf16], 128-byte rows, swizzled
 constexpr int kTileBytes = 2 * kHalfBytes;        // one K tile or one V tile of 128 tokens
-constexpr int kStagesK = 4, kStagesV = 3;         // K is needed a tile earlier than V
+constexpr int kStagesK = 3, kStagesV = 3;
 constexpr int NQ = 4;                             // unit queue depth (the producer runs ahead of the consumers)
 constexpr uint32_t kTmemCols = 512;               // S0 [0,128), S1 [128,256), O [256,384), Q [384,448) and P [448,512) as bf16 pairs
-constexpr int kSmemTc = (kStagesK + kStagesV) * kTileBytes + 1024 + 512;
+constexpr int kSmemTc = (kStagesK + kStagesV) * kTileBytes + 1024 + 4096;
 constexpr float kRescaleGap = 8.f;                // log2 units
 
 struct UnitMsg { int b, g, t0, t1, slot, pad0, pad1, pad2; };
@@ -48,10 +48,12 @@ struct Ctl {
     uint64_t k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
     uint64_t s_full[2], s_empty[2], p_full, pv_done, q_ready, uq_full[NQ], uq_empty[NQ], drain;
     UnitMsg uq[NQ];
+    float xmax[2][4][2][2][16];      // [tile parity][quarter][side][half][row]: row maxima exchanged by the two sides
+    float xsum[4][2][32];            // [quarter][side][lane]: row sums at the end of a unit
     uint32_t tmem_base;
     int abort;
 };
-static_assert(sizeof(Ctl) <= 512, "control block fits its slot");
+static_assert(sizeof(Ctl) <= 4096, "control block fits its slot");
 
 struct TcArgs {
     const __nv_bfloat16* q; int q_row_stride;
@@ -111,7 +113,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
         mbar_init(smem_u32(&ctl->p_full), kSoftmaxThreads);
         mbar_init(smem_u32(&ctl->pv_done), 1);
         mbar_init(smem_u32(&ctl->q_ready), kSoftmaxThreads);
-        for (int s = 0; s < NQ; ++s) { mbar_init(smem_u32(&ctl->uq_full[s]), 1); mbar_init(smem_u32(&ctl->uq_empty[s]), 8); }
+        for (int s = 0; s < NQ; ++s) { mbar_init(smem_u32(&ctl->uq_full[s]), 1); mbar_init(smem_u32(&ctl->uq_empty[s]), 12); }
         mbar_init(smem_u32(&ctl->drain), 1);
         ctl->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -127,7 +129,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
     const uint32_t tmem_base = ctl->tmem_base;
     const int rows_valid = a.R * a.group;
 
-    if (warp == 0 || warp >= 6) {
+    if (warp == 0 || (warp >= 6 && warp <= 8)) {
         // ---- producers: one thread issues a TMA box in ~100 cycles and a tile needs 16 per operand, so four warps share
         // them: warps 0 and 7 the even and odd blocks of the K tiles, warps 6 and 8 those of the V tiles.  Warp 0 also pulls
         // the units and publishes them to everyone else. ----
@@ -247,22 +249,24 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && clock64() - t0c < kWaitLimit) { }
             }
         }
-    } else if (warp < 6) {
-        // ---- softmax warps.  Query row r lives in MMA row / tensor-memory lane (r % 4) * 32 + r / 4, so every quarter (one
-        // warp each) holds rows_valid / 4 rows in its first lanes.  The scores are read in the 16-lane fragment shape
-        // (16x256b: a row's 8 consecutive columns over the 4 threads of a quad, rows g4 and g4 + 8 per thread, as in an
-        // mma accumulator), so all 32 threads share the columns of 16 rows: with up to 64 query rows (H = 1) a thread
-        // handles 64 scores per tile, with up to 128 (H = 2: both 16-lane halves) 128.  The exponentials are the critical
-        // path: 4 per clock and scheduler whatever the number of active lanes.
+    } else {
+        // ---- softmax warps: 2..5 (columns 0..63 of every score tile) and 9..12 (columns 64..127).  Query row r lives in MMA
+        // row / tensor-memory lane (r % 4) * 32 + r / 4, so every 32-lane quarter - which one warp of each side may touch -
+        // holds rows_valid / 4 rows in its first lanes.  The scores are read in the 16-lane fragment shape (16x256b: a row's
+        // 8 consecutive columns over the 4 threads of a quad, rows g4 and g4 + 8 per thread, as in an mma accumulator), so
+        // the 32 threads of a warp share its 64 columns of 16 rows: 32 scores per thread and tile with up to 64 query rows
+        // (H = 1), 64 with up to 128 (H = 2: both 16-lane halves).  The two warps of a quarter exchange their row maxima
+        // through shared memory (a 64-thread named barrier per tile) and otherwise work on their own columns of S, P and O.
+        // The exponentials are what a tile costs: 4 per clock and scheduler whatever the number of active lanes.
         const int quarter = warp & 3;
+        const int x = warp >= 9 ? 1 : 0;              // column half
         const int g4 = lane >> 2, q4 = lane & 3;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const uint32_t o_tmem = t_lane + 256;
-        // staging / result mapping: thread = tensor-memory lane
+        // staging / result mapping: thread = tensor-memory lane, this side's half of the row
         const int r_st = lane * 4 + quarter;
         const bool st_ok = r_st < rows_valid;
         const int st_i = st_ok ? r_st / a.group : 0, st_j = st_ok ? r_st % a.group : 0;
-        const int m_st = quarter * 32 + lane;
         // score mapping: rows (h, hh) -> lane-in-quarter h * 16 + g4 + 8 * hh
         bool rok[H][2];
         int ri[H][2];
@@ -274,12 +278,13 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                 rok[h][hh] = r < rows_valid;
                 ri[h][hh] = rok[h][hh] ? r / a.group : 0;
             }
+        auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + quarter) : "memory"); };
         {   // rows without a query row hold zeros in Q and P for the whole launch
             uint32_t z[32];
 #pragma unroll
             for (int e = 0; e < 32; ++e) z[e] = 0u;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tc_st32(t_lane + 384 + c * 32, z);
+            tc_st32(t_lane + 384 + x * 32, z);
+            tc_st32(t_lane + 448 + x * 32, z);
             tc_wait_st();
         }
         uint32_t n_tile = 0;                          // running tile counter (same sequence as the MMA warp's)
@@ -292,20 +297,18 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
             if (lane == 0) mbar_arrive(smem_u32(&ctl->uq_empty[slot_q]));
             if (un.t1 < 0) break;
             const int n_tiles = (un.t1 - un.t0 + T - 1) / T;
-            // stage Q in tensor memory (the A operand of S = Q K^T): thread = row, 64 columns of bf16 pairs.  The previous
-            // unit's S tiles have all been read, so no MMA still reads it.
+            // stage this side's half of Q in tensor memory (the A operand of S = Q K^T): thread = row, 32 columns of bf16
+            // pairs.  The previous unit's S tiles have all been read, so no MMA still reads it.
             {
-                uint32_t qv[2][32];
+                uint32_t qv[32];
                 const uint4* qp = reinterpret_cast<const uint4*>(a.q + ((size_t)un.b * a.R + st_i) * a.q_row_stride +
-                                                                 (size_t)(un.g * a.group + st_j) * DH);
+                                                                 (size_t)(un.g * a.group + st_j) * DH) + x * 8;
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
+                for (int c = 0; c < 8; ++c) {
                     const uint4 v = st_ok ? qp[c] : make_uint4(0u, 0u, 0u, 0u);
-                    qv[c >> 3][(c & 7) * 4] = v.x; qv[c >> 3][(c & 7) * 4 + 1] = v.y;
-                    qv[c >> 3][(c & 7) * 4 + 2] = v.z; qv[c >> 3][(c & 7) * 4 + 3] = v.w;
+                    qv[c * 4] = v.x; qv[c * 4 + 1] = v.y; qv[c * 4 + 2] = v.z; qv[c * 4 + 3] = v.w;
                 }
-                tc_st32(t_lane + 384, qv[0]);
-                tc_st32(t_lane + 384 + 32, qv[1]);
+                tc_st32(t_lane + 384 + x * 32, qv);
                 tc_wait_st();
             }
             tc_fence_before();
@@ -339,91 +342,93 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
 #pragma unroll
                     for (int h = 0; h < H; ++h) { vis[h][0] = 0x7fffffff; vis[h][1] = 0x7fffffff; }
                 }
-                uint32_t pk[H][32];                               // bf16 pairs: [x * 16 + 2 * jc + hh]
+                // this side's 64 columns of every half, all loads before the one wait (a tensor-memory load takes a few
+                // hundred cycles and this warp shares its scheduler with one other softmax warp at most)
+                uint32_t v[H][32];
+#pragma unroll
+                for (int h = 0; h < H; ++h) tc_ld_16x256b_x8(t_lane + ((uint32_t)(h * 16) << 16) + buf * 128 + x * 64, v[h]);
+                tc_wait_ld();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&ctl->s_empty[buf]));
+                // row maxima: this thread's columns, the quad, then the other side's
+                float mx[H][2];
+#pragma unroll
+                for (int h = 0; h < H; ++h) {
+                    mx[h][0] = -INFINITY; mx[h][1] = -INFINITY;
+#pragma unroll
+                    for (int jc = 0; jc < 8; ++jc)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int col = x * 64 + jc * 8 + 2 * q4 + (e & 1);
+                            if (col >= vis[h][e >> 1]) v[h][4 * jc + e] = 0xff800000u;          // -inf: the exponential is an exact zero
+                            mx[h][e >> 1] = fmaxf(mx[h][e >> 1], __uint_as_float(v[h][4 * jc + e]));
+                        }
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        mx[h][hh] = fmaxf(mx[h][hh], __shfl_xor_sync(0xffffffffu, mx[h][hh], 1));
+                        mx[h][hh] = fmaxf(mx[h][hh], __shfl_xor_sync(0xffffffffu, mx[h][hh], 2));
+                        if (q4 == 0) ctl->xmax[buf][quarter][x][h][g4 + 8 * hh] = mx[h][hh];
+                    }
+                }
+                pair_sync();
+                uint32_t pk[H][16];                               // bf16 pairs: [2 * jc + hh]
                 float alpha[H][2];
                 bool raise = false;
 #pragma unroll
                 for (int h = 0; h < H; ++h) {
-                    const uint32_t s_addr = t_lane + ((uint32_t)(h * 16) << 16) + buf * 128;
-                    // both 64-column loads are issued before the one wait: a tensor-memory load takes a few hundred
-                    // cycles and this warp is alone on its scheduler, so nothing else would hide them
-                    uint32_t v[2][32];
-                    tc_ld_16x256b_x8(s_addr, v[0]);
-                    tc_ld_16x256b_x8(s_addr + 64, v[1]);
-                    tc_wait_ld();
-                    if (h == H - 1) { tc_fence_before(); mbar_arrive(smem_u32(&ctl->s_empty[buf])); }
-                    // row maxima over this thread's columns, then over the quad
-                    float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-                    for (int x = 0; x < 2; ++x)
-#pragma unroll
-                        for (int jc = 0; jc < 8; ++jc)
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const int col = x * 64 + jc * 8 + 2 * q4 + (e & 1);
-                                if (col >= vis[h][e >> 1]) v[x][4 * jc + e] = 0xff800000u;      // -inf: the exponential is an exact zero
-                                mx[e >> 1] = fmaxf(mx[e >> 1], __uint_as_float(v[x][4 * jc + e]));
-                            }
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh) {
-                        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 1));
-                        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 2));
-                        mx[hh] *= a.scale_log2;                   // scale > 0; -inf stays -inf
+                        float m2 = fmaxf(mx[h][hh], ctl->xmax[buf][quarter][x ^ 1][h][g4 + 8 * hh]) * a.scale_log2;   // -inf stays -inf
                         alpha[h][hh] = 1.f;
-                        if (rok[h][hh] && mx[hh] > -INFINITY && (m_used[h][hh] == -INFINITY || mx[hh] > m_used[h][hh] + kRescaleGap)) {
-                            alpha[h][hh] = m_used[h][hh] == -INFINITY ? 0.f : exp2f(m_used[h][hh] - mx[hh]);
+                        if (rok[h][hh] && m2 > -INFINITY && (m_used[h][hh] == -INFINITY || m2 > m_used[h][hh] + kRescaleGap)) {
+                            alpha[h][hh] = m_used[h][hh] == -INFINITY ? 0.f : exp2f(m_used[h][hh] - m2);
                             raise = raise || j > 0;               // the first tile overwrites the accumulator
-                            m_used[h][hh] = mx[hh];
+                            m_used[h][hh] = m2;
                             l_run[h][hh] *= alpha[h][hh];
                         }
                     }
                     const float ms0 = m_used[h][0] == -INFINITY ? 0.f : m_used[h][0];
                     const float ms1 = m_used[h][1] == -INFINITY ? 0.f : m_used[h][1];
-                    // probabilities, bf16 pairs
                     float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-                    for (int x = 0; x < 2; ++x)
+                    for (int jc = 0; jc < 8; ++jc) {
+                        float p[4];
 #pragma unroll
-                        for (int jc = 0; jc < 8; ++jc) {
-                            float p[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                p[e] = ex2_approx(fmaf(__uint_as_float(v[x][4 * jc + e]), a.scale_log2, (e >> 1) ? -ms1 : -ms0));
-                            l0 += p[0] + p[1];
-                            l1 += p[2] + p[3];
-                            pk[h][x * 16 + 2 * jc] = pack2(p[0], p[1]);
-                            pk[h][x * 16 + 2 * jc + 1] = pack2(p[2], p[3]);
-                        }
+                        for (int e = 0; e < 4; ++e)
+                            p[e] = ex2_approx(fmaf(__uint_as_float(v[h][4 * jc + e]), a.scale_log2, (e >> 1) ? -ms1 : -ms0));
+                        l0 += p[0] + p[1];
+                        l1 += p[2] + p[3];
+                        pk[h][2 * jc] = pack2(p[0], p[1]);
+                        pk[h][2 * jc + 1] = pack2(p[2], p[3]);
+                    }
                     l_run[h][0] += l0;
                     l_run[h][1] += l1;
                 }
                 // the previous tile's P V has finished: P may be overwritten and the accumulator is at rest
                 if (n_tile > 0 && !mbar_wait(smem_u32(&ctl->pv_done), (n_tile - 1u) & 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, raise)) {
+                if (__any_sync(0xffffffffu, raise)) {             // this side's 64 columns of the accumulator
 #pragma unroll
-                    for (int h = 0; h < H; ++h)
-#pragma unroll 1
-                        for (int x = 0; x < 2; ++x) {
-                            uint32_t v[32];
-                            const uint32_t o_addr = o_tmem + ((uint32_t)(h * 16) << 16) + x * 64;
-                            tc_ld_16x256b_x8(o_addr, v);
-                            tc_wait_ld();
+                    for (int h = 0; h < H; ++h) {
+                        uint32_t o[32];
+                        const uint32_t o_addr = o_tmem + ((uint32_t)(h * 16) << 16) + x * 64;
+                        tc_ld_16x256b_x8(o_addr, o);
+                        tc_wait_ld();
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha[h][(e >> 1) & 1]);
-                            tc_st_16x256b_x8(o_addr, v);
-                        }
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha[h][(e >> 1) & 1]);
+                        tc_st_16x256b_x8(o_addr, o);
+                    }
                     tc_wait_st();
                 }
-                // P goes to tensor memory as bf16 pairs (the A operand of O += P V): one store per 16-lane half
+                // P goes to tensor memory as bf16 pairs (the A operand of O += P V): this side's 32 packed columns
 #pragma unroll
-                for (int h = 0; h < H; ++h) tc_st_16x128b_x16(t_lane + ((uint32_t)(h * 16) << 16) + 448, pk[h]);
+                for (int h = 0; h < H; ++h) tc_st_16x128b_x8(t_lane + ((uint32_t)(h * 16) << 16) + 448 + x * 32, pk[h]);
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&ctl->p_full));
             }
             if (!ok) break;
-            // ---- unit result: thread = tensor-memory lane; the row's maximum and sum come from the quad that tracked it ----
+            // ---- unit result: thread = tensor-memory lane; the row's maximum and sum come from the quads that tracked it ----
             if (!mbar_wait(smem_u32(&ctl->pv_done), (n_tile - 1u) & 1u, abort_flag)) { ok = false; break; }
             tc_fence_after();
             float row_m = -INFINITY, row_l = 0.f;
@@ -438,26 +443,28 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                     const float tl = __shfl_sync(0xffffffffu, l, 4 * (lane & 7));
                     if ((lane >> 4) == h && ((lane >> 3) & 1) == hh) { row_m = tm; row_l = tl; }
                 }
+            ctl->xsum[quarter][x][lane] = row_l;                  // the row sum is the two sides' together
+            pair_sync();
+            row_l += ctl->xsum[quarter][x ^ 1][lane];
             const float inv = row_l > 0.f ? 1.f / row_l : 0.f;
             float* part = nullptr;
             __nv_bfloat16* op = nullptr;
             if (st_ok) {
                 if (un.slot >= 0) {
                     const size_t ps = ((size_t)un.slot * a.Hkv + un.g) * a.rows_alloc + r_st;
-                    part = a.pv.part_o + ps * DH;
-                    a.pv.part_ml[ps * 2] = row_m;
-                    a.pv.part_ml[ps * 2 + 1] = row_l;
+                    part = a.pv.part_o + ps * DH + x * 64;
+                    if (x == 0) { a.pv.part_ml[ps * 2] = row_m; a.pv.part_ml[ps * 2 + 1] = row_l; }
                 } else {
-                    op = a.out + ((size_t)un.b * a.R + st_i) * a.out_row_stride + (size_t)(un.g * a.group + st_j) * DH;
+                    op = a.out + ((size_t)un.b * a.R + st_i) * a.out_row_stride + (size_t)(un.g * a.group + st_j) * DH + x * 64;
                 }
             }
             {
-                uint32_t o[4][32];                    // the whole row in one round trip to tensor memory
+                uint32_t o[2][32];                    // this side's half of the row in one round trip to tensor memory
 #pragma unroll
-                for (int c = 0; c < 4; ++c) tc_ld32(o_tmem + c * 32, o[c]);
+                for (int c = 0; c < 2; ++c) tc_ld32(o_tmem + x * 64 + c * 32, o[c]);
                 tc_wait_ld();
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     if (part != nullptr) {
 #pragma unroll
                         for (int e = 0; e < 32; e += 4)
@@ -477,6 +484,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) attn_tc_kernel(const __grid_con
                     }
                 }
             }
+            pair_sync();                                          // the exchange slots are free for the next unit
             tc_fence_before();
         }
     }
