@@ -318,3 +318,27 @@ def test_slot_replacement_mid_run(eng_mod):
     assert eng.status().device_status == -16
     books_equal()
     eng.close()
+
+
+def test_seq_replace_argument_and_state_errors(eng_mod):
+    """Host-detectable misuse of slot replacement is refused with an error code and changes nothing."""
+    cfg = inputs.model_config("c1")
+    sc = eng_mod.make_spec_config(cfg, draft_kind="none", k_max=1, max_batch=2, kv_num_blocks=8, max_blocks_per_seq=4, seed=1)
+    eng = eng_mod.SpecStep(sc)
+    eng.load_target_weights(inputs.make_target_weights(cfg, seed=1))
+    eng.seq_init(np.array([3, 5], np.int32), np.array([1, 2], np.int32), np.arange(8, dtype=np.int32))
+    before = (eng.seq_len().cpu().numpy().copy(), eng.block_table().cpu().numpy().copy())
+    for slots, lens, lasts in [([2], [0], [1]), ([0, 0], [0, 0], [1, 1]), ([1], [0], [cfg["vocab"]]), ([0], [16 * 4], [1])]:
+        with pytest.raises(RuntimeError):
+            eng.seq_replace(slots, lens, lasts)
+    eng.verify(0)
+    with pytest.raises(RuntimeError):                       # a verified step is waiting for its commit
+        eng.seq_replace([0], [0], [1])
+    eng.reject_sample(0)
+    eng.kv_commit()
+    assert np.array_equal(eng.seq_len().cpu().numpy(), before[0] + 1)
+    eng.seq_replace([1], [-1], [0])                         # retire
+    assert eng.seq_len().cpu().tolist() == [4, -1] and eng.status().device_status == 0
+    eng.verify(0); eng.reject_sample(0); eng.kv_commit()    # the retired slot is passed over
+    assert eng.seq_len().cpu().tolist() == [5, -1] and eng.n_emitted().cpu().tolist() == [1, 0]
+    eng.close()
