@@ -30,7 +30,7 @@
 extern "C" {
 #endif
 
-#define SPEC_ABI_VERSION 3u
+#define SPEC_ABI_VERSION 4u
 
 typedef struct spec_ctx spec_ctx; /* opaque */
 
@@ -50,6 +50,7 @@ typedef enum {
 } spec_status;
 
 enum { SPEC_DTYPE_BF16 = 0, SPEC_DTYPE_F32 = 1 };
+enum { SPEC_KV_MODEL = 0, SPEC_KV_E4M3 = 1 };
 enum { SPEC_DRAFT_NONE = 0, SPEC_DRAFT_EAGLE3 = 1, SPEC_DRAFT_MTP = 2, SPEC_DRAFT_NGRAM = 3 };
 
 /* Model and run description.  n_experts = 0 selects the dense SwiGLU MLP. */
@@ -80,6 +81,11 @@ typedef struct {
     int32_t draft_vocab;        /* EAGLE3 only: 0 = the head's LM head covers the whole vocabulary; else its    */
                                 /* number of rows (a multiple of 8, <= vocab): row r scores target token        */
                                 /* D_D2T[r] (strictly increasing ids), q is zero outside that set                */
+    int32_t kv_dtype;           /* SPEC_KV_MODEL: the cache holds `dtype`; SPEC_KV_E4M3: one byte per element, the e4m3    */
+                                /* code (round to nearest even, saturating at 448) of x / scale, read back as code * scale */
+                                /* (the precision of the paper's deployment simulator, Section 5.1).  bf16 models with     */
+                                /* head_dim 128 and at most 16 query rows per KV head; a reduced-precision mode            */
+    float kv_scale_k, kv_scale_v; /* > 0 with SPEC_KV_E4M3: one scale for all keys (after the rotary embedding), one for values */
     int32_t reserved_;
 } spec_config;
 

@@ -50,6 +50,8 @@ def lib():
         L.spec_oracle_kv_commit.argtypes = [c.c_int, c.c_int, c.c_int, i32p, i32p, i32p, i32p, i32p]
         L.spec_oracle_kv_replace.argtypes = [c.c_int, i32p, i32p, c.c_int, c.c_int, i32p, i32p, i32p, i32p]
         L.spec_oracle_kv_replace.restype = c.c_int
+        L.spec_oracle_e4m3_quantize.argtypes = [c.c_size_t, c.POINTER(c.c_float), c.c_float, c.POINTER(c.c_uint8)]
+        L.spec_oracle_e4m3_dequantize.argtypes = [c.c_size_t, c.POINTER(c.c_uint8), c.c_float, c.POINTER(c.c_float)]
         _lib = L
     return _lib
 
@@ -182,3 +184,22 @@ def kv_replace(slots, new_len, block_tokens, seq_len, block_table, free_stack, f
     return lib().spec_oracle_kv_replace(sl.shape[0], _p(sl, ctypes.c_int32), _p(nl, ctypes.c_int32), block_tokens, max_blocks,
                                         _p(seq_len, ctypes.c_int32), _p(block_table, ctypes.c_int32),
                                         _p(free_stack, ctypes.c_int32), _p(free_top, ctypes.c_int32))
+
+
+def e4m3_quantize(x, scale=1.0):
+    """e4m3 codes (uint8) of x / scale: round to nearest even, saturating at 448."""
+    xf = _f32(x)
+    out = np.empty(xf.shape, np.uint8)
+    lib().spec_oracle_e4m3_quantize(xf.size, _p(xf, ctypes.c_float), float(scale), _p(out, ctypes.c_uint8))
+    return out
+
+
+def e4m3_dequantize(codes, scale=1.0):
+    cc = np.ascontiguousarray(codes, np.uint8)
+    out = np.empty(cc.shape, np.float32)
+    lib().spec_oracle_e4m3_dequantize(cc.size, _p(cc, ctypes.c_uint8), float(scale), _p(out, ctypes.c_float))
+    return out
+
+
+def e4m3_roundtrip(x, scale=1.0):
+    return e4m3_dequantize(e4m3_quantize(x, scale), scale)

@@ -88,6 +88,9 @@ class LazyPast:
         for which in ("KV_K", "KV_V"):
             pool = self.eng.kv_pool(which, l % self.G)
             rows = pool[idx].permute(0, 2, 1, 3).reshape(nb * 16, pool.shape[1], pool.shape[3])[: self.n_past]
+            if pool.dtype == torch.uint8:       # 8-bit cache: e4m3 codes times the scale (torch's cast reads the codes back exactly)
+                sc = self.eng.sc
+                rows = rows.contiguous().view(torch.float8_e4m3fn).float() * (sc.kv_scale_k if which.endswith("_K") else sc.kv_scale_v)
             out.append(_np(rows))
         return tuple(out)
 

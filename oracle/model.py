@@ -113,6 +113,18 @@ def moe_mlp(lw, m, top_k, router_logits=None):
     return out
 
 
+def kv_as_cached(cfg, k, v):
+    """What the attention reads back for freshly computed keys and values: themselves, or, with an 8-bit cache
+    (cfg["kv_fp8"] = (k_scale, v_scale)), their e4m3 codes times the scale - for the new positions as for the old ones,
+    since every position is attended to through the cache."""
+    if not cfg.get("kv_fp8"):
+        return k, v
+    import oracle
+    ks, vs = cfg["kv_fp8"]
+    return (oracle.e4m3_roundtrip(np.asarray(k, np.float32), ks).astype(F64),
+            oracle.e4m3_roundtrip(np.asarray(v, np.float32), vs).astype(F64))
+
+
 def decoder_layer(cfg, lw, x, pos, past_k=None, past_v=None, attn_in=None, router_logits=None):
     """One pre-norm decoder layer on rows x [T][d] at absolute positions pos.
 
@@ -128,6 +140,7 @@ def decoder_layer(cfg, lw, x, pos, past_k=None, past_v=None, attn_in=None, route
     v = qkv[:, (Hq + Hkv) * dh :].reshape(T, Hkv, dh)
     q = rope(q, pos, cfg["rope_theta"])
     k = rope(k, pos, cfg["rope_theta"])
+    k, v = kv_as_cached(cfg, k, v)
     n_past = 0 if past_k is None else past_k.shape[0]
     k_all = k if n_past == 0 else np.concatenate([np.asarray(past_k, F64), k], axis=0)
     v_all = v if n_past == 0 else np.concatenate([np.asarray(past_v, F64), v], axis=0)
@@ -183,6 +196,7 @@ def eagle3_slots(cfg, W, H, g, tokens_next, pos, past_k=None, past_v=None):
     q = rope(qkv[:, : Hq * dh].reshape(T, Hq, dh), pos, cfg["rope_theta"])
     k = rope(qkv[:, Hq * dh : (Hq + Hkv) * dh].reshape(T, Hkv, dh), pos, cfg["rope_theta"])
     v = qkv[:, (Hq + Hkv) * dh :].reshape(T, Hkv, dh)
+    k, v = kv_as_cached(cfg, k, v)
     n_past = 0 if past_k is None else past_k.shape[0]
     k_all = k if n_past == 0 else np.concatenate([past_k, k], axis=0)
     v_all = v if n_past == 0 else np.concatenate([past_v, v], axis=0)

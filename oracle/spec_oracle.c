@@ -302,3 +302,48 @@ int spec_oracle_kv_replace(int n, const int32_t* slots, const int32_t* new_len, 
     }
     return 0;
 }
+
+/* ------------------------------------------------------------------------------------------------------
+ * 8-bit KV cache (the precision the paper's deployment simulator assumes, Section 5.1): a cached value x is stored
+ * as e4m3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities, largest finite value 448,
+ * smallest subnormal 2^-9) of x / scale, rounded to nearest with ties to even and saturating at +-448; the
+ * attention reads it back as code * scale.  NaN maps to the NaN code 0x7f.
+ * ---------------------------------------------------------------------------------------------------- */
+static uint8_t e4m3_from_float(float x)
+{
+    if (x != x) return 0x7f;
+    const uint8_t sign = signbit(x) ? 0x80 : 0x00;
+    const double a = fabs((double)x);
+    if (a >= 448.0) return (uint8_t)(sign | 0x7e);                 /* saturate: 0x7e is 448 */
+    if (a < 0.015625) {                                             /* below 2^-6: subnormal grid, spacing 2^-9 */
+        const double r = nearbyint(a * 512.0);                      /* default rounding mode: ties to even */
+        return (uint8_t)(sign | (uint8_t)r);                        /* r = 8 is the code of the first normal, 2^-6 */
+    }
+    int e;
+    (void)frexp(a, &e);                                             /* a = m * 2^e with m in [0.5, 1): a = 1.f * 2^(e-1) */
+    int exp_field = e - 1 + 7;
+    double r = nearbyint(ldexp(a, -(e - 1)) * 8.0);                 /* 8 + mantissa, in [8, 16] */
+    if (r >= 16.0) { r = 8.0; exp_field += 1; }
+    if (exp_field > 15 || (exp_field == 15 && r > 14.0)) return (uint8_t)(sign | 0x7e);
+    return (uint8_t)(sign | (uint8_t)(exp_field << 3) | (uint8_t)((int)r - 8));
+}
+
+static float e4m3_to_float(uint8_t c)
+{
+    int sign = c & 0x80, ef = (c >> 3) & 0xf, mf = c & 7;
+    double v;
+    if (ef == 15 && mf == 7) return NAN;
+    if (ef == 0) v = mf / 512.0;
+    else v = ldexp(1.0 + mf / 8.0, ef - 7);
+    return (float)(sign ? -v : v);
+}
+
+void spec_oracle_e4m3_quantize(size_t n, const float* x, float scale, uint8_t* codes)
+{
+    for (size_t i = 0; i < n; ++i) codes[i] = e4m3_from_float(x[i] / scale);
+}
+
+void spec_oracle_e4m3_dequantize(size_t n, const uint8_t* codes, float scale, float* x)
+{
+    for (size_t i = 0; i < n; ++i) x[i] = e4m3_to_float(codes[i]) * scale;
+}

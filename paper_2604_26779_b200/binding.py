@@ -12,8 +12,9 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libspec.so")
 
-SPEC_ABI_VERSION = 3
+SPEC_ABI_VERSION = 4
 SPEC_DTYPE_BF16, SPEC_DTYPE_F32 = 0, 1
+SPEC_KV_MODEL, SPEC_KV_E4M3 = 0, 1
 SPEC_DRAFT_NONE, SPEC_DRAFT_EAGLE3, SPEC_DRAFT_MTP, SPEC_DRAFT_NGRAM = 0, 1, 2, 3
 
 STATUS_NAMES = {0: "SPEC_OK", -1: "SPEC_ERR_INVALID_ARG", -2: "SPEC_ERR_SHAPE", -3: "SPEC_ERR_UNSUPPORTED",
@@ -47,7 +48,8 @@ class spec_config(C.Structure):
                 ("n_taps", C.c_int32), ("tap_layers", C.c_int32 * 3),
                 ("k_max", C.c_int32), ("max_batch", C.c_int32), ("kv_block_tokens", C.c_int32),
                 ("kv_num_blocks", C.c_int32), ("max_blocks_per_seq", C.c_int32), ("kv_layer_pools", C.c_int32),
-                ("temperature", C.c_float), ("seed", C.c_uint64), ("ngram_n", C.c_int32), ("draft_greedy", C.c_int32), ("draft_vocab", C.c_int32), ("reserved_", C.c_int32)]
+                ("temperature", C.c_float), ("seed", C.c_uint64), ("ngram_n", C.c_int32), ("draft_greedy", C.c_int32), ("draft_vocab", C.c_int32), ("kv_dtype", C.c_int32),
+                ("kv_scale_k", C.c_float), ("kv_scale_v", C.c_float), ("reserved_", C.c_int32)]
 
 
 class spec_sizes(C.Structure):

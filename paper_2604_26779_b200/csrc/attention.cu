@@ -95,6 +95,7 @@ spec_status launch_attention_simt(const AttnArgs& a, cudaStream_t st)
 
 spec_status launch_attention(const AttnArgs& a, cudaStream_t st)
 {
+    if (a.kv_fp8) return attn::attention_fp8_supported(a) ? attn::launch_attention_fp8(a, st) : SPEC_ERR_UNSUPPORTED;
     if (attn::attention_tc_supported(a)) return attn::launch_attention_tc(a, st);
     if (attention_mma_supported(a)) return launch_attention_mma(a, st);
     return launch_attention_simt(a, st);

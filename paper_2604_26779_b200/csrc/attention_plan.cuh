@@ -49,6 +49,8 @@ spec_status launch_attn_plan(int B, int R, const int32_t* pos, int max_chunks, c
 spec_status launch_attn_merge128(int B, int rows_alloc, int Hkv, int R, int group, void* out, int out_row_stride,
                                  const PlanView& pv, cudaStream_t st);
 
+bool attention_fp8_supported(const AttnArgs& a);
+spec_status launch_attention_fp8(const AttnArgs& a, cudaStream_t st);
 bool attention_tc_supported(const AttnArgs& a);
 spec_status launch_attention_tc(const AttnArgs& a, cudaStream_t st);
 

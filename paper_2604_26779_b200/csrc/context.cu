@@ -91,6 +91,9 @@ spec_status check_config(const spec_config* c)
     if (c->draft_kind == SPEC_DRAFT_MTP && (c->draft_d_ffn <= 0 || c->draft_d_ffn % 128 != 0)) return SPEC_ERR_SHAPE;
     if (!(c->temperature > 0.f) || !(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return SPEC_ERR_UNSUPPORTED;
     if (c->vocab > sampler_max_vocab()) return SPEC_ERR_SHAPE;
+    if (c->kv_dtype != SPEC_KV_MODEL && (c->kv_dtype != SPEC_KV_E4M3 || c->dtype != SPEC_DTYPE_BF16 || c->head_dim != 128 ||
+                                         !(c->kv_scale_k > 0.f) || !(c->kv_scale_v > 0.f) ||
+                                         (c->k_max + 1) * (c->n_q_heads / c->n_kv_heads) > 16)) return SPEC_ERR_UNSUPPORTED;
     if (c->draft_vocab != 0 && (c->draft_kind != SPEC_DRAFT_EAGLE3 || c->draft_vocab < 8 || c->draft_vocab > c->vocab ||
                                 c->draft_vocab % 8 != 0)) return SPEC_ERR_SHAPE;
     return SPEC_OK;
@@ -148,7 +151,8 @@ void build_layout(spec_ctx& x)
         }
         x.draft_weights_bytes = a.top;
     }
-    x.kv_pool_bytes = align_up((size_t)c.kv_num_blocks * c.n_kv_heads * c.kv_block_tokens * c.head_dim * es, 256);
+    x.kv_pool_bytes = align_up((size_t)c.kv_num_blocks * c.n_kv_heads * c.kv_block_tokens * c.head_dim *
+                               (c.kv_dtype == SPEC_KV_E4M3 ? 1 : es), 256);
     x.kv_bytes = x.kv_pool_bytes * 2 * c.kv_layer_pools;
     x.draft_kv_bytes = (c.draft_kind == SPEC_DRAFT_EAGLE3 || c.draft_kind == SPEC_DRAFT_MTP) ? x.kv_pool_bytes * 2 : 0;
     {
@@ -286,8 +290,10 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
         // projection, rotary embedding and the append into the paged cache in one kernel
         QkvEpilogue e{Hq, Hkv, dh, R, g.max_blocks_per_seq, g.kv_block_tokens, pos, at<int32_t>(c.buf.state, c.block_table),
                       at<float>(ws, c.rope), k_pool, v_pool};
+        if (g.kv_dtype == SPEC_KV_E4M3) { e.kv_fp8 = 1; e.k_scale = g.kv_scale_k; e.v_scale = g.kv_scale_v; }
         TIMED(c, CLS_GEMM, launch_gemm_qkv_tc(M, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), e, status_word, st));
     } else {
+        if (g.kv_dtype == SPEC_KV_E4M3) return SPEC_ERR_UNSUPPORTED;    // the 8-bit cache is written by the fused epilogue only
         TIMED(c, CLS_GEMM, launch_gemm(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt, 0, st));
         TRY(launch_rope_append(B, R, Hq, Hkv, dh, g.rope_theta, at(ws, c.qkv), pos, k_pool, v_pool,
                                at<int32_t>(c.buf.state, c.block_table), g.max_blocks_per_seq, g.kv_block_tokens, dt, st));
@@ -296,6 +302,7 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
                at<int32_t>(c.buf.state, c.block_table), pos, at(ws, c.attn_out), Hq * dh, dt, at(ws, c.attn_scratch),
                c.attn_scratch.bytes, g.max_blocks_per_seq * g.kv_block_tokens, launch_index};
     a.status = status_word;
+    if (g.kv_dtype == SPEC_KV_E4M3) { a.kv_fp8 = 1; a.k_scale = g.kv_scale_k; a.v_scale = g.kv_scale_v; }
     TIMED(c, CLS_ATTN, launch_attention(a, st));
     TIMED(c, CLS_GEMM, launch_gemm(M, d, Hq * dh, at(ws, c.attn_out), Hq * dh, W.wo, res, d, dt, SPEC_DTYPE_F32, 1, st));
     TRY(launch_rmsnorm(M, d, res, W.mlp_norm, g.rms_eps, at(ws, c.h), d, 0, dt, st));

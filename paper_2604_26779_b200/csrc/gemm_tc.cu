@@ -65,6 +65,7 @@ struct GemmArgs {
     int Hq, Hkv, dh, R, max_blocks, block_tokens;
     const int32_t* pos; const int32_t* block_table; const float2* rope;   // rope [dh/2][M] (cos, sin) of each row's position
     __nv_bfloat16* k_pool; __nv_bfloat16* v_pool;
+    int kv_fp8; float k_scale, v_scale;           // 8-bit cache: k and v are stored as e4m3 codes of x / scale
 };
 
 enum { EPI_PLAIN = 0, EPI_SWIGLU = 1, EPI_QKV = 2 };
@@ -80,6 +81,21 @@ __device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float (&
         o.z = *reinterpret_cast<uint32_t*>(&t2); o.w = *reinterpret_cast<uint32_t*>(&t3);
         *reinterpret_cast<uint4*>(dst + 8 * j) = o;
     }
+}
+
+// 32 consecutive values as e4m3 codes (round to nearest even, saturating), 32 bytes.
+__device__ __forceinline__ void store_e4m3x32(unsigned char* dst, const float (&f)[32], float scale)
+{
+    uint32_t w[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        unsigned short lo, hi;                       // cvt packs its first source into the upper byte
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(__fdiv_rn(f[4 * j + 1], scale)), "f"(__fdiv_rn(f[4 * j], scale)));
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(__fdiv_rn(f[4 * j + 3], scale)), "f"(__fdiv_rn(f[4 * j + 2], scale)));
+        w[j] = (uint32_t)lo | ((uint32_t)hi << 16);
+    }
+    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+    *reinterpret_cast<uint4*>(dst + 16) = make_uint4(w[4], w[5], w[6], w[7]);
 }
 
 // Plain epilogue: C (+)= accumulator, fp32 or bf16, ragged N handled element-wise.
@@ -199,7 +215,15 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord&
                 if (blk < 0) continue;
                 const bool is_k = head < g.Hq + g.Hkv;
                 const int kh = is_k ? head - g.Hq : head - g.Hq - g.Hkv;
-                dst = (is_k ? g.k_pool : g.v_pool) + (((size_t)blk * g.Hkv + kh) * g.block_tokens + slot) * g.dh;
+                const size_t at = (((size_t)blk * g.Hkv + kh) * g.block_tokens + slot) * g.dh;
+                if (g.kv_fp8) {
+                    unsigned char* d8 = reinterpret_cast<unsigned char*>(is_k ? g.k_pool : g.v_pool) + at;
+                    const float sc = is_k ? g.k_scale : g.v_scale;
+                    store_e4m3x32(d8 + j0, a, sc);
+                    store_e4m3x32(d8 + half + j0, b, sc);
+                    continue;
+                }
+                dst = (is_k ? g.k_pool : g.v_pool) + at;
             }
             store_bf16x32(dst + j0, a);
             store_bf16x32(dst + half + j0, b);
@@ -530,6 +554,7 @@ spec_status launch_gemm_qkv_tc(int M, int K, const void* A, int lda, const void*
     g.Hq = e.Hq; g.Hkv = e.Hkv; g.dh = e.dh; g.R = e.R; g.max_blocks = e.max_blocks; g.block_tokens = e.block_tokens;
     g.pos = e.pos; g.block_table = e.block_table; g.rope = reinterpret_cast<const float2*>(e.rope);
     g.k_pool = static_cast<__nv_bfloat16*>(e.k_pool); g.v_pool = static_cast<__nv_bfloat16*>(e.v_pool);
+    g.kv_fp8 = e.kv_fp8; g.k_scale = e.k_scale; g.v_scale = e.v_scale;
     return run_kernel(EPI_QKV, ma, mb, g, (long long)((M + BM - 1) / BM) * ((N + BN - 1) / BN), st);
 }
 

@@ -96,6 +96,8 @@ struct QkvEpilogue {
     const int32_t* pos; const int32_t* block_table;
     const float* rope;            // [dh/2][M][2] (cos, sin) of each row's position
     void* k_pool; void* v_pool;
+    int kv_fp8 = 0;               // write e4m3 codes of k / k_scale and v / v_scale instead of bf16
+    float k_scale = 1.f, v_scale = 1.f;
 };
 spec_status launch_gemm_qkv_tc(int M, int K, const void* A, int lda, const void* W, void* qkv, const QkvEpilogue& e,
                                int32_t* status, cudaStream_t st);
@@ -122,6 +124,8 @@ struct AttnArgs {
     int max_kv_len;
     int launch_index;                  // 0 plans the work units; later launches of the same step reuse the plan
     int32_t* status = nullptr;         // device status word for kernels with bounded waits (may be null)
+    int kv_fp8 = 0;                    // the pools hold e4m3 codes of x / scale (one byte per element)
+    float k_scale = 1.f, v_scale = 1.f;
 };
 spec_status launch_attention(const AttnArgs& a, cudaStream_t st);
 size_t attention_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int max_kv_len);

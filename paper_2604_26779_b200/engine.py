@@ -16,7 +16,8 @@ from .binding import T
 def make_spec_config(cfg: dict, *, draft_kind: str = "none", k_max: int = 3, max_batch: int = 4, kv_num_blocks: int = 64,
                      max_blocks_per_seq: int = 16, kv_block_tokens: int = 16, kv_layer_pools: int | None = None,
                      seed: int = 0, draft_d_ffn: int | None = None, ngram_n: int = 3, draft_greedy: bool = False,
-                     draft_vocab: int = 0) -> B.spec_config:
+                     draft_vocab: int = 0, kv_fp8=None) -> B.spec_config:
+    """kv_fp8: None for a cache in the model's dtype, or (k_scale, v_scale) for the 8-bit e4m3 cache."""
     sc = B.spec_config()
     sc.struct_size, sc.abi_version = C.sizeof(B.spec_config), B.SPEC_ABI_VERSION
     for name in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab", "n_experts",
@@ -29,6 +30,8 @@ def make_spec_config(cfg: dict, *, draft_kind: str = "none", k_max: int = 3, max
     sc.ngram_n = int(ngram_n) if draft_kind == "ngram" else 0
     sc.draft_greedy = 1 if draft_greedy else 0
     sc.draft_vocab = int(draft_vocab) if draft_kind == "eagle3" else 0
+    if kv_fp8:
+        sc.kv_dtype, sc.kv_scale_k, sc.kv_scale_v = B.SPEC_KV_E4M3, float(kv_fp8[0]), float(kv_fp8[1])
     taps = tuple(cfg.get("tap_layers", ())) if draft_kind == "eagle3" else ()
     sc.n_taps = len(taps)
     for i, t in enumerate(taps):
@@ -227,4 +230,14 @@ class SpecStep:
 
     def kv_pool(self, which: str, pool: int = 0):
         sc = self.sc
-        return self.tensor(which, pool, self.tdtype, (sc.kv_num_blocks, sc.n_kv_heads, sc.kv_block_tokens, sc.head_dim))
+        dt = torch.uint8 if sc.kv_dtype == B.SPEC_KV_E4M3 else self.tdtype           # e4m3 codes are handed out as bytes
+        return self.tensor(which, pool, dt, (sc.kv_num_blocks, sc.n_kv_heads, sc.kv_block_tokens, sc.head_dim))
+
+    def kv_pool_values(self, which: str, pool: int = 0):
+        """The pool as fp32 values (codes times the scale for the 8-bit cache)."""
+        sc = self.sc
+        p = self.kv_pool(which, pool)
+        if sc.kv_dtype != B.SPEC_KV_E4M3:
+            return p.float()
+        scale = sc.kv_scale_k if which.endswith("_K") else sc.kv_scale_v
+        return p.view(torch.float8_e4m3fn).float() * scale

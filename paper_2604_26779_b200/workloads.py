@@ -18,6 +18,16 @@ def _fill_normal(t: torch.Tensor, std: float, gen: torch.Generator):
         flat[i : i + step].normal_(0.0, std, generator=gen)
 
 
+def _fill_normal_e4m3(t: torch.Tensor, std: float, scale: float, gen: torch.Generator):
+    """In-place fill of a uint8 view with the e4m3 codes of N(0, std) / scale (input data for the 8-bit cache)."""
+    flat = t.reshape(-1)
+    step = 1 << 27
+    for i in range(0, flat.numel(), step):
+        n = min(step, flat.numel() - i)
+        x = torch.empty(n, dtype=torch.float32, device=flat.device).normal_(0.0, std, generator=gen) / scale
+        flat[i : i + n].copy_(x.to(torch.float8_e4m3fn).view(torch.uint8))
+
+
 def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, len_hi=16384, lens=None, draft="eagle3",
                          kv_pools=None, steps_budget=64, seed=None, device="cuda:0", vocab=None, mem_fraction=0.92,
                          cfg_over=None):
@@ -46,7 +56,8 @@ def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, l
     def sizes_for(G):
         sc = engine.make_spec_config(cfg, draft_kind=draft, k_max=k, max_batch=B, kv_num_blocks=num_blocks,
                                      max_blocks_per_seq=max_blocks, kv_layer_pools=G, seed=seed,
-                                     draft_vocab=int(cfg.get("draft_vocab") or 0), draft_greedy=bool(cfg.get("draft_greedy")))
+                                     draft_vocab=int(cfg.get("draft_vocab") or 0), draft_greedy=bool(cfg.get("draft_greedy")),
+                                     kv_fp8=cfg.get("kv_fp8"))
         from . import binding as Bd
         import ctypes as C
         s = Bd.spec_sizes()
@@ -90,11 +101,19 @@ def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, l
             rng = np.random.Generator(np.random.PCG64(seed + 4))
             d2t = np.sort(rng.choice(cfg["vocab"], size=int(cfg["draft_vocab"]), replace=False)).astype(np.int32)
             eng.tensor("D_D2T", 0, torch.int32).copy_(torch.from_numpy(d2t).to(device))
-        _fill_normal(eng.tensor("DRAFT_KV_K", 0, bf), 1.0, gen)
-        _fill_normal(eng.tensor("DRAFT_KV_V", 0, bf), 1.0, gen)
+        if cfg.get("kv_fp8"):
+            _fill_normal_e4m3(eng.kv_pool("DRAFT_KV_K", 0), 1.0, cfg["kv_fp8"][0], gen)
+            _fill_normal_e4m3(eng.kv_pool("DRAFT_KV_V", 0), 1.0, cfg["kv_fp8"][1], gen)
+        else:
+            _fill_normal(eng.tensor("DRAFT_KV_K", 0, bf), 1.0, gen)
+            _fill_normal(eng.tensor("DRAFT_KV_V", 0, bf), 1.0, gen)
     for p in range(G):
-        _fill_normal(eng.tensor("KV_K", p, bf), 1.0, gen)
-        _fill_normal(eng.tensor("KV_V", p, bf), 1.0, gen)
+        if cfg.get("kv_fp8"):
+            _fill_normal_e4m3(eng.kv_pool("KV_K", p), 1.0, cfg["kv_fp8"][0], gen)
+            _fill_normal_e4m3(eng.kv_pool("KV_V", p), 1.0, cfg["kv_fp8"][1], gen)
+        else:
+            _fill_normal(eng.tensor("KV_K", p, bf), 1.0, gen)
+            _fill_normal(eng.tensor("KV_V", p, bf), 1.0, gen)
     last = inputs.make_prompts(B, 1, cfg["vocab"], seed + 2)[:, 0]
     order = inputs.make_block_order(num_blocks, seed + 3)
     torch.cuda.synchronize()

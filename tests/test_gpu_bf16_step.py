@@ -23,7 +23,10 @@ def gather_pool(eng, which, blocks, n):
     pool = eng.kv_pool(which, 0)
     nb = -(-n // 16)
     idx = torch.as_tensor(np.ascontiguousarray(blocks[:nb]), dtype=torch.long, device="cuda")
-    return pool[idx].permute(0, 2, 1, 3).reshape(nb * 16, pool.shape[1], pool.shape[3])[:n].float().cpu().numpy()
+    rows = pool[idx].permute(0, 2, 1, 3).reshape(nb * 16, pool.shape[1], pool.shape[3])[:n]
+    if pool.dtype == torch.uint8:                # 8-bit cache: codes times the scale
+        rows = rows.contiguous().view(torch.float8_e4m3fn).float() * (eng.sc.kv_scale_k if which.endswith("_K") else eng.sc.kv_scale_v)
+    return rows.float().cpu().numpy()
 
 
 def draft_head_weights(eng, cfg, kind):
@@ -43,9 +46,10 @@ def draft_head_weights(eng, cfg, kind):
     return H
 
 
-@pytest.mark.parametrize("kind,k,head_dim", [("eagle3", 3, 64), ("mtp", 2, 64), ("eagle3", 7, 64),
-                                              ("eagle3", 5, 128), ("mtp", 7, 128)])
-def test_bf16_steps_stage_by_stage(kind, k, head_dim):
+@pytest.mark.parametrize("kind,k,head_dim,kv_fp8", [("eagle3", 3, 64, None), ("mtp", 2, 64, None), ("eagle3", 7, 64, None),
+                                                     ("eagle3", 5, 128, None), ("mtp", 7, 128, None),
+                                                     ("eagle3", 3, 128, (1.0, 1.0)), ("mtp", 3, 128, (0.05, 0.03))])
+def test_bf16_steps_stage_by_stage(kind, k, head_dim, kv_fp8):
     """head_dim 64: 16 or 32 query rows per KV head on the register-fragment attention kernel; head_dim 128 with k = 5 / 7:
     24 / 32 rows on the tcgen05 kernel, including the draft head's first pass, whose rows past the committed count carry
     position -1."""
@@ -53,6 +57,8 @@ def test_bf16_steps_stage_by_stage(kind, k, head_dim):
         pytest.skip("no CUDA device")
     from paper_2604_26779_b200 import workloads
     over = dict(d_model=512, n_q_heads=8, n_kv_heads=2, head_dim=head_dim, d_ffn=1024)
+    if kv_fp8:                 # 8-bit cache: the oracle rounds every key and value to e4m3 exactly where the device stores it
+        over["kv_fp8"] = kv_fp8
     n_layers = 3
     lens = np.array([5, 40, 100, 17, 300], np.int32)
     eng, info = workloads.build_dense_workload("c3", lens=lens, k=k, draft=kind, steps_budget=8, n_layers=n_layers,
@@ -102,6 +108,22 @@ def test_bf16_steps_stage_by_stage(kind, k, head_dim):
             r = harness.oracle_verify_sample(eng, cfg, W, b, [int(last[b])] + [int(x) for x in g_drafts[b]], int(seq_len[b]),
                                              table[b], info["kv_pools"], g_dlog[b], info["seed"], draft_step)
             worst_v = max(worst_v, float((np.abs(g_logits[b] - r["logits"]).max(-1) / np.abs(r["logits"]).max(-1)).max()))
+            if kv_fp8 and b == 1:
+                # what the step appended to the 8-bit cache of the first layer: the oracle's keys and values of the k+1 new
+                # positions, rounded to e4m3 by the oracle.  The device rounds fp32 results of bf16 GEMMs, the oracle fp64 ones,
+                # so a value near a rounding boundary (small values above all) may land on the neighbouring code: most codes equal, none further
+                # than one step (2^-3 relative) away.
+                tokens_in = [int(last[b])] + [int(x) for x in g_drafts[b]]
+                fw = model.target_forward(dict(cfg, n_layers=1), dict(W, layers=[W["layers"][0]]), tokens_in,
+                                          past=harness.LazyPast(eng, cfg, table[b], int(seq_len[b]), info["kv_pools"], 1),
+                                          start_pos=int(seq_len[b]))
+                for which, ref in (("KV_K", fw["new_kv"][0][0]), ("KV_V", fw["new_kv"][0][1])):
+                    n_all = int(seq_len[b]) + k + 1
+                    dev = gather_pool(eng, which, eng.block_table().cpu().numpy()[b], n_all)[int(seq_len[b]):]
+                    same = np.mean(dev == ref.astype(np.float32))
+                    # one code step (2^-3 of the value) plus the absolute error of the bf16 computation that fed the rounding
+                    step_ok = np.all(np.abs(dev - ref) <= 0.126 * np.abs(ref) + 8e-3 * np.sqrt(np.mean(ref ** 2)))
+                    assert same > 0.85 and step_ok, (which, same)
             p, q = oracle.softmax(g_logits[b]), oracle.softmax(g_dlog[b])
             u = oracle.uniforms(info["seed"], draft_step, 0, b + 1, k + 1)[b]
             toks, n_o, _, mg = oracle.reject_sample_seq(p, q, g_drafts[b], u)
@@ -112,6 +134,6 @@ def test_bf16_steps_stage_by_stage(kind, k, head_dim):
         assert eng.status().device_status == 0
         assert np.array_equal(eng.seq_len().cpu().numpy(), seq_len + g_n)
         k_prev = k
-    print(f"bf16 {kind} k={k} dh={head_dim}: draft logits {worst_d:.2e}, verify logits {worst_v:.2e}, boundary cases {boundary}")
+    print(f"bf16 {kind} k={k} dh={head_dim} kv_fp8={kv_fp8}: draft logits {worst_d:.2e}, verify logits {worst_v:.2e}, boundary cases {boundary}")
     assert worst_d < 2e-2 and worst_v < 2e-2 and boundary <= 2
     eng.close()

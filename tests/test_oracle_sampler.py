@@ -448,3 +448,32 @@ def test_kv_bookkeeping_random_walk_with_replacement():
             if r == 0:
                 for s_, nl in zip(slots, new_len):
                     assert seq_len[s_] == (nl if nl >= 0 else -1)
+
+
+# ---- 8-bit KV cache codes ------------------------------------------------------------------------------------
+
+def test_e4m3_codes_match_the_library_cast():
+    """The oracle's e4m3 rounding (nearest even, saturating at 448) against torch's float8_e4m3fn cast on every code's
+    value, on the midpoints between neighbouring codes, and on random values; the read-back is exact."""
+    import torch
+    codes = np.arange(256, dtype=np.uint8)
+    vals = oracle.e4m3_dequantize(codes)
+    ref_vals = torch.from_numpy(codes).view(torch.float8_e4m3fn).float().numpy()
+    finite = np.isfinite(ref_vals)
+    assert np.array_equal(vals[finite], ref_vals[finite]) and np.all(np.isnan(vals[~finite]))
+    assert vals[0x7e] == 448.0 and vals[0x01] == 2.0 ** -9 and vals[0x08] == 2.0 ** -6
+    pos = np.sort(vals[finite & (vals >= 0)])
+    mids = ((pos[:-1].astype(np.float64) + pos[1:].astype(np.float64)) / 2).astype(np.float32)     # exact in fp32
+    rng = np.random.default_rng(5)
+    xs = np.concatenate([pos, -pos, mids, -mids, rng.normal(0, 1, 20000).astype(np.float32),
+                         rng.normal(0, 100, 20000).astype(np.float32), (rng.normal(0, 1e-3, 5000)).astype(np.float32),
+                         np.array([447.9, 448.0, 463.9], np.float32)])
+    xs = xs[np.abs(xs) < 464.0]                                   # beyond the last rounding boundary torch returns NaN, we saturate
+    got = oracle.e4m3_quantize(xs)
+    ref = torch.from_numpy(xs).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(got, ref)
+    assert oracle.e4m3_quantize(np.array([1e9, -1e9], np.float32)).tolist() == [0x7e, 0xfe]      # saturation, not NaN
+    # a scale divides before rounding and multiplies after
+    x = rng.normal(0, 3, 1000).astype(np.float32)
+    assert np.array_equal(oracle.e4m3_roundtrip(x, 0.25), oracle.e4m3_dequantize(oracle.e4m3_quantize(x / np.float32(0.25))) * np.float32(0.25))
+    assert np.max(np.abs(oracle.e4m3_roundtrip(x) - x) / np.maximum(np.abs(x), 2.0 ** -6)) <= 2.0 ** -4 + 1e-7
