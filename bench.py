@@ -322,6 +322,9 @@ def main():
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--draft-vocab", type=int, default=0,
                     help="c3 only: give the EAGLE-3-style head its own vocabulary of this many rows (0 = whole vocabulary, the headline)")
+    ap.add_argument("--kv-fp8", action="store_true",
+                    help="c3 only: 8-bit (e4m3) KV cache, scales 1/16 - a reduced-precision variant, reported under its own "
+                         "metric name and never the headline")
     ap.add_argument("--k-sweep", default=None,
                     help="comma-separated draft lengths, e.g. 1,3,5,7: times the c3 step at each k on one engine built for the "
                          "largest (not the headline run: prints its own JSON line)")
@@ -359,7 +362,8 @@ def main():
                                                    len_lo=args.len_lo, len_hi=args.len_hi,
                                                    steps_budget=steps_budget, device=f"cuda:{local}",
                                                    seed=replicas.replica_seed(rank),
-                                                   cfg_over=dict(draft_vocab=args.draft_vocab) if args.draft_vocab else None)
+                                                   cfg_over=dict(**(dict(draft_vocab=args.draft_vocab) if args.draft_vocab else {}),
+                                                                 **(dict(kv_fp8=(0.0625, 0.0625)) if args.kv_fp8 else {})) or None)
         wl_name = ("c3: 8B dense verify (32 layers, d=4096, 32q/8kv, dh=128, FFN 14336, V=128256, bf16), "
                    "EAGLE-3-style 1-layer draft head, cache lengths ~U[1024,16384], 16-token pages")
     elif args.workload == "c4":
@@ -397,6 +401,8 @@ def main():
               "acceptance": "measured with the random-init draft head (untrained: low by construction)"}
     if args.workload == "c3" and args.draft_vocab:
         config["draft_vocab"] = args.draft_vocab
+    if args.workload == "c3" and args.kv_fp8:
+        config["kv_cache"] = "e4m3 codes, scales 1/16 (REDUCED PRECISION: not the headline configuration)"
     if args.workload != "c3":
         args.no_cpu_baseline = True
 
@@ -465,7 +471,7 @@ def main():
     hbm_peak, tf_peak, peak_kind = measured_peaks()
     R = k + 1
     mean_cached_tokens = 0.5 * (tokens_before + tokens_after) + B * R           # positions each launch reads (prefix + new rows)
-    bytes_per_token_layer = cfg["n_kv_heads"] * cfg["head_dim"] * 2 * 2          # K and V, bf16
+    bytes_per_token_layer = cfg["n_kv_heads"] * cfg["head_dim"] * 2 * (1 if cfg.get("kv_fp8") else 2)   # K and V, bf16 or e4m3
     attn_passes = max(int(timing.passes[0]), 1)
     attn_ms = float(timing.ms[0]) / attn_passes
     # n_layers launches per step on the target's cache and k on the draft head's one-layer cache: the same positions each
@@ -480,7 +486,7 @@ def main():
                 "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": attn_ms, "launches_timed": attn_passes,
                 "share_of_step": float(timing.ms[0]) / ms_total, "frac_of_nominal_8TBs": achieved / 8000.0}
 
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+    line = {"metric": METRIC + (" [8-bit KV cache variant]" if cfg.get("kv_fp8") else ""), "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": int(launches),
             "roofline": roofline,
