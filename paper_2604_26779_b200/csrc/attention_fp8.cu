@@ -1,10 +1,16 @@
 // Paged grouped-query attention over an 8-bit (e4m3) KV cache, up to 16 query rows per KV head, head_dim 128.
 //
 // The cache holds one byte per element (code = round_e4m3(x / scale), one scale for keys and one for values), so the pass
-// that dominates a verify forward moves half the bytes.  The kernel is the register-fragment kernel of the bf16 cache with
-// one more stage in front of the fragments: tiles of codes arrive by 16-byte cp.async (three stages of 16 KB), every warp
-// converts its own 16-token block of the tile to fp16 - the conversion is exact - into the swizzled rows that ldmatrix
-// reads, and the two MMAs run in fp16 (Q converted from bf16 once per unit, P packed to fp16) with fp32 accumulation.
+// that dominates a verify forward moves half the bytes.  The kernel is the register-fragment kernel of the bf16 cache
+// with the fragments taken straight from the code tiles: tiles of codes arrive by 16-byte cp.async (stages of 16 KB,
+// 16-byte chunks XOR-swizzled by token), ldmatrix reads them as if two codes were one 16-bit element, and the codes are
+// converted to fp16 - exactly - in registers; both MMAs run in fp16 (Q converted from bf16 once per unit, P packed to
+// fp16) with fp32 accumulation.  Two index permutations make the register contents fit the MMA fragments:
+//   keys    a thread's ldmatrix register holds four consecutive head_dim codes of one token, so inside every 16-wide
+//           k-block the MMA's k index 2t, 2t+1, 2t+8, 2t+9 is mapped to head_dim 4t .. 4t+3 (Q is loaded the same way);
+//   values  the transposing ldmatrix delivers codes (token 2t, dims 2g, 2g+1) and (token 2t+1, dims 2g, 2g+1); a byte
+//           permute pairs equal dims of the two tokens, which makes one MMA n-tile the even dims of a 16-wide block and
+//           the next one the odd dims; the accumulator columns are put back in order when the result is written.
 // The scales never touch the tile: the key scale multiplies the softmax scale, the value scale the final normalisation.
 // Work units, the atomic work counter and the merge pass are the bf16 kernel's.
 #include <cuda_fp16.h>
@@ -75,18 +81,12 @@ __device__ __forceinline__ void e4m3x4_to_f16x4(uint32_t w, uint32_t& lo, uint32
     asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(lo) : "h"(a));
     asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(hi) : "h"(b));
 }
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint4& v)
-{
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
 // One CTA = 4 warps, each taking one 16-token block of every 64-token tile (16 query rows per KV head at most).
 template <int STAGES>
 __global__ void __launch_bounds__(kThreads) attn_fp8_kernel(const Fp8Args a)
 {
     constexpr int DH = 128, WM = 1, WN = 4;
     constexpr int CH = DH / 8;                               // 16-byte chunks per fp16 row
-    constexpr int kBlkBytes = kBT * DH * 2;                  // one block of one head as fp16
     constexpr int kCodeBlk = kBT * DH;                       // the same block as e4m3 codes
     constexpr int kStageBytes = 4 * kCodeBlk * 2;            // 4 blocks, K and V, as codes
     constexpr int ROWS = 16 * WM;
@@ -97,7 +97,6 @@ __global__ void __launch_bounds__(kThreads) attn_fp8_kernel(const Fp8Args a)
     const int wm = warp / WN, wn = warp % WN;
     const int g4 = lane >> 2, q4 = lane & 3;
     const uint32_t smem_base = smem_u32(smem);
-    const uint32_t work = smem_base + STAGES * kStageBytes;   // this tile converted to fp16: the layout the fragments expect
     const int n_rows_valid = a.R * a.group;
 
     for (;;) {
@@ -122,9 +121,9 @@ __global__ void __launch_bounds__(kThreads) attn_fp8_kernel(const Fp8Args a)
             const __nv_bfloat16* qp = a.q + ((size_t)b * a.R + i) * a.q_row_stride + (size_t)(g * a.group + j) * DH;
 #pragma unroll
             for (int ks = 0; ks < DH / 16; ++ks) {
-                // A fragment: regs {hh, hh+2} hold (row, k = 16 ks + 2 q4 + {0,1}) and (row, the same + 8)
-                qf[ks][hh] = valid ? bf16x2_to_f16x2(*reinterpret_cast<const uint32_t*>(qp + 16 * ks + 2 * q4)) : 0u;
-                qf[ks][hh + 2] = valid ? bf16x2_to_f16x2(*reinterpret_cast<const uint32_t*>(qp + 16 * ks + 8 + 2 * q4)) : 0u;
+                // A fragment under the key permutation: regs {hh, hh+2} hold (row, head_dim 16 ks + 4 q4 + {0,1}) and (+ {2,3})
+                qf[ks][hh] = valid ? bf16x2_to_f16x2(*reinterpret_cast<const uint32_t*>(qp + 16 * ks + 4 * q4)) : 0u;
+                qf[ks][hh + 2] = valid ? bf16x2_to_f16x2(*reinterpret_cast<const uint32_t*>(qp + 16 * ks + 4 * q4 + 2)) : 0u;
             }
         }
         int min_lim = min(lim[0], lim[1]);
@@ -147,8 +146,9 @@ __global__ void __launch_bounds__(kThreads) attn_fp8_kernel(const Fp8Args a)
                 const size_t goff = ((size_t)(phys < 0 ? 0 : phys) * a.Hkv + g) * (size_t)kCodeBlk;      // bytes
                 const int nbytes = phys < 0 ? 0 : 16;
                 // 128 chunks of 16 codes per block: one per thread and tensor
-                cp_async16(stage + bb * kCodeBlk + tid * 16, a.k_pool + goff + (size_t)tid * 16, nbytes);
-                cp_async16(stage + 4 * kCodeBlk + bb * kCodeBlk + tid * 16, a.v_pool + goff + (size_t)tid * 16, nbytes);
+                const uint32_t soff = (uint32_t)(bb * kCodeBlk + (tid >> 3) * 128 + (((tid & 7) ^ ((tid >> 3) & 7)) << 4));   // token tid/8, chunk tid%8
+                cp_async16(stage + soff, a.k_pool + goff + (size_t)tid * 16, nbytes);
+                cp_async16(stage + 4 * kCodeBlk + soff, a.v_pool + goff + (size_t)tid * 16, nbytes);
             }
         };
 
@@ -160,41 +160,26 @@ __global__ void __launch_bounds__(kThreads) attn_fp8_kernel(const Fp8Args a)
             __syncthreads();
             if (j + STAGES - 1 < n_tiles) issue_tile(j + STAGES - 1);
             cp_async_commit();
-            const unsigned char* codes = smem + (size_t)(j % STAGES) * kStageBytes;
+            const uint32_t stage = smem_base + (uint32_t)(j % STAGES) * kStageBytes;
 #pragma unroll
             for (int bb = wn; bb < 4; bb += WN) {
                 const int tok0 = t0 + j * kTileTok + bb * kBT;
                 if (tok0 >= t1) continue;
-                const uint32_t kb_base = work + bb * kBlkBytes, vb_base = kb_base + 4 * kBlkBytes;
-                // this warp's block, codes -> fp16 (exact), into the swizzled rows the fragment loads read: 256 chunks of 16
-                // codes (K then V), eight per lane; the scales are applied to the scores and to the result instead
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int ci = lane + 32 * i, tensor = ci >> 7, idx = ci & 127;
-                    const int r = idx >> 3, c = idx & 7;
-                    const uint4 w = *reinterpret_cast<const uint4*>(codes + tensor * 4 * kCodeBlk + bb * kCodeBlk + idx * 16);
-                    uint4 lo, hi;
-                    e4m3x4_to_f16x4(w.x, lo.x, lo.y); e4m3x4_to_f16x4(w.y, lo.z, lo.w);
-                    e4m3x4_to_f16x4(w.z, hi.x, hi.y); e4m3x4_to_f16x4(w.w, hi.z, hi.w);
-                    const uint32_t base = (tensor ? vb_base : kb_base) + r * (DH * 2);
-                    const int c0 = 2 * c, c1 = 2 * c + 1;
-                    st_shared_v4(base + (((c0 & ~7) | ((c0 ^ r) & 7)) << 4), lo);
-                    st_shared_v4(base + (((c1 & ~7) | ((c1 ^ r) & 7)) << 4), hi);
-                }
-                __syncwarp();
+                const uint32_t kb_base = stage + bb * kCodeBlk, vb_base = kb_base + 4 * kCodeBlk;
+                // this lane's row of the four 8 x 8 matrices an ldmatrix.x4 reads: matrix m = lane / 8 covers tokens
+                // (m & 1) * 8 .. + 7 and the 16-code chunk (first chunk of the pair) + (m >> 1)
+                const int l_tok = ((lane >> 3) & 1) * 8 + (lane & 7), l_chunk = lane >> 4;
                 // S = Q K^T for 16 tokens
                 float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-                {
-                    const int mat = lane >> 3, rr = lane & 7;
-                    const int row = rr + 8 * (mat >> 1);
 #pragma unroll
-                    for (int ks = 0; ks < DH / 16; ++ks) {
-                        const int c = 2 * ks + (mat & 1);
-                        uint32_t kb[4];
-                        ldmatrix_x4(kb, kb_base + row * (DH * 2) + (((c & ~7) | ((c ^ row) & 7)) << 4));
-                        mma_f16(s[0], qf[ks], kb[0], kb[1]);
-                        mma_f16(s[1], qf[ks], kb[2], kb[3]);
-                    }
+                for (int kp = 0; kp < DH / 32; ++kp) {               // two 16-wide k-blocks per load
+                    uint32_t kb[4];
+                    ldmatrix_x4(kb, kb_base + l_tok * 128 + (((2 * kp + l_chunk) ^ (l_tok & 7)) << 4));
+                    uint32_t b0, b1;
+                    e4m3x4_to_f16x4(kb[0], b0, b1); mma_f16(s[0], qf[2 * kp], b0, b1);          // tokens 0..7, k-block 2 kp
+                    e4m3x4_to_f16x4(kb[1], b0, b1); mma_f16(s[1], qf[2 * kp], b0, b1);          // tokens 8..15
+                    e4m3x4_to_f16x4(kb[2], b0, b1); mma_f16(s[0], qf[2 * kp + 1], b0, b1);      // k-block 2 kp + 1
+                    e4m3x4_to_f16x4(kb[3], b0, b1); mma_f16(s[1], qf[2 * kp + 1], b0, b1);
                 }
                 // causal limit of the new rows and the end of this unit's range
                 if (tok0 + kBT - 1 > min_lim || tok0 + kBT > t1) {
@@ -246,17 +231,18 @@ __global__ void __launch_bounds__(kThreads) attn_fp8_kernel(const Fp8Args a)
                     pf[2] = pack_f16(p[1][0], p[1][1]);
                     pf[3] = pack_f16(p[1][2], p[1][3]);
                 }
-                // O += P V
-                {
-                    const int mat = lane >> 3, rr = lane & 7;
-                    const int row = rr + 8 * (mat & 1);
+                // O += P V: per 32 head dims one transposing load; even dims and odd dims of a 16-wide block are two n-tiles
 #pragma unroll
-                    for (int nd = 0; nd < DH / 16; ++nd) {
-                        const int c = 2 * nd + (mat >> 1);
-                        uint32_t vb[4];
-                        ldmatrix_x4_trans(vb, vb_base + row * (DH * 2) + (((c & ~7) | ((c ^ row) & 7)) << 4));
-                        mma_f16(o_acc[2 * nd], pf, vb[0], vb[1]);
-                        mma_f16(o_acc[2 * nd + 1], pf, vb[2], vb[3]);
+                for (int dp = 0; dp < DH / 32; ++dp) {
+                    uint32_t vb[4];
+                    ldmatrix_x4_trans(vb, vb_base + l_tok * 128 + (((2 * dp + l_chunk) ^ (l_tok & 7)) << 4));
+#pragma unroll
+                    for (int h2 = 0; h2 < 2; ++h2) {                  // block 2 dp + h2: registers vb[2 h2] (tokens 0..7) and vb[2 h2 + 1] (8..15)
+                        uint32_t b0, b1;
+                        e4m3x4_to_f16x4(__byte_perm(vb[2 * h2], vb[2 * h2 + 1], 0x6420), b0, b1);
+                        mma_f16(o_acc[2 * (2 * dp + h2)], pf, b0, b1);                       // even dims
+                        e4m3x4_to_f16x4(__byte_perm(vb[2 * h2], vb[2 * h2 + 1], 0x7531), b0, b1);
+                        mma_f16(o_acc[2 * (2 * dp + h2) + 1], pf, b0, b1);                   // odd dims
                     }
                 }
             }
@@ -277,8 +263,9 @@ __global__ void __launch_bounds__(kThreads) attn_fp8_kernel(const Fp8Args a)
             const int r = 16 * wm + g4 + 8 * hh;
             float* orow = mrg_o + ((size_t)wn * ROWS + r) * DH;
 #pragma unroll
-            for (int n = 0; n < NT_O; ++n)
-                *reinterpret_cast<float2*>(orow + 8 * n + 2 * q4) = make_float2(o_acc[n][2 * hh], o_acc[n][2 * hh + 1]);
+            for (int d = 0; d < NT_O / 2; ++d)        // block d: n-tile 2d holds dims 16 d + 4 q4 + {0, 2}, n-tile 2d + 1 the dims + {1, 3}
+                *reinterpret_cast<float4*>(orow + 16 * d + 4 * q4) =
+                    make_float4(o_acc[2 * d][2 * hh], o_acc[2 * d + 1][2 * hh], o_acc[2 * d][2 * hh + 1], o_acc[2 * d + 1][2 * hh + 1]);
             if (q4 == 0) { mrg_ml[((size_t)wn * ROWS + r) * 2] = m_run[hh]; mrg_ml[((size_t)wn * ROWS + r) * 2 + 1] = l_run[hh]; }
         }
         __syncthreads();
@@ -329,7 +316,8 @@ bool attention_fp8_supported(const AttnArgs& a)
 spec_status launch_attention_fp8(const AttnArgs& a, cudaStream_t st)
 {
     constexpr int STAGES = 3;
-    constexpr int smem = STAGES * (4 * kBT * 128 * 2) + 4 * kBT * 128 * 2 * 2;       // code stages + one fp16 tile (K and V)
+    constexpr int kStages = STAGES * (4 * kBT * 128 * 2), kMerge = 4 * 16 * 130 * 4;
+    constexpr int smem = kStages > kMerge ? kStages : kMerge;      // code stages; the unit-end merge of the four warps reuses them
     const int group = a.Hq / a.Hkv;
     const int max_chunks = max_chunks_for(a.max_kv_len);
     if (a.scratch_bytes < attention_mma_scratch_bytes(a.B, a.R, a.Hq, a.Hkv, a.dh, a.max_kv_len)) return SPEC_ERR_SHAPE;
