@@ -28,7 +28,9 @@ constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTE
 constexpr int kThreads = 320;          // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue (two per tensor-memory lane quarter)
 constexpr int kEpiThreads = 256;
 constexpr uint32_t kTmemCols = 512;
-constexpr int kSmemBytes = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int kOutStageBytes = 32 * 128;  // per epilogue warp: 32 rows x 128 bytes, where a warp turns its row-per-thread
+                                          // accumulator fragments into row-contiguous 128-byte pieces before they go to memory
+constexpr int kSmemBytes = STAGES * STAGE_BYTES + (kEpiThreads / 32) * kOutStageBytes + 1024 + 256;
 #define TRY_LAUNCH(expr) do { spec_status s__ = (expr); if (s__ != SPEC_OK) return s__; } while (0)
 
 struct Ctl {
@@ -98,16 +100,115 @@ __device__ __forceinline__ void store_e4m3x32(unsigned char* dst, const float (&
     *reinterpret_cast<uint4*>(dst + 16) = make_uint4(w[4], w[5], w[6], w[7]);
 }
 
-// Plain epilogue: C (+)= accumulator, fp32 or bf16, ragged N handled element-wise.
-__device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok, int half)
+// Output staging.  After tcgen05.ld a thread holds 32 consecutive columns of ONE row, so a direct store makes every warp
+// instruction touch 32 different lines, 16 bytes each.  Instead each thread writes its 128 bytes into the warp's staging
+// area (16-byte pieces XOR-swizzled by the row, conflict-free both ways) and the warp reads it back four rows at a time,
+// eight lanes per row: every store (and every residual load) instruction then covers four whole 128-byte lines.
+__device__ __forceinline__ void stage_put(uint32_t stage, int lane, int piece, const uint4& v)
 {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + lane * 128 + ((piece ^ (lane & 7)) << 4)),
+                 "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 stage_get(uint32_t stage, int row, int piece)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(stage + row * 128 + ((piece ^ (row & 7)) << 4)) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint4 pack_bf16x8(const float* f)
+{
+    __nv_bfloat162 t0 = __floats2bfloat162_rn(f[0], f[1]), t1 = __floats2bfloat162_rn(f[2], f[3]);
+    __nv_bfloat162 t2 = __floats2bfloat162_rn(f[4], f[5]), t3 = __floats2bfloat162_rn(f[6], f[7]);
+    return make_uint4(*reinterpret_cast<uint32_t*>(&t0), *reinterpret_cast<uint32_t*>(&t1),
+                      *reinterpret_cast<uint32_t*>(&t2), *reinterpret_cast<uint32_t*>(&t3));
+}
+// The 32 x 128-byte block of the residual that a staged block will be added to: this lane's eight 16-byte pieces.
+__device__ __forceinline__ void residual_get(uint4 (&o)[8], int lane, const unsigned char* src, size_t row_stride_bytes, int rows_ok)
+{
+    const unsigned char* base = src + (lane & 7) * 16;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = i * 4 + (lane >> 3);
+        if (r < rows_ok) o[i] = __ldcg(reinterpret_cast<const uint4*>(base + (size_t)r * row_stride_bytes));
+    }
+}
+// Writes the staged 32 x 128-byte block: row r of the block goes to dst + r * row_stride_bytes; rows >= rows_ok are skipped.
+// kAddF32: the block is fp32 and o (from residual_get on the same rows) is added first.
+template <bool kAddF32>
+__device__ __forceinline__ void stage_flush(uint32_t stage, int lane, unsigned char* dst, size_t row_stride_bytes, int rows_ok,
+                                            const uint4 (&o)[8])
+{
+    __syncwarp();
+    const int piece = lane & 7, r0 = lane >> 3;
+    unsigned char* base = dst + piece * 16;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = i * 4 + r0;
+        if (r < rows_ok) {
+            uint4 v = stage_get(stage, r, piece);
+            if (kAddF32) {
+                v.x = __float_as_uint(__uint_as_float(v.x) + __uint_as_float(o[i].x));
+                v.y = __float_as_uint(__uint_as_float(v.y) + __uint_as_float(o[i].y));
+                v.z = __float_as_uint(__uint_as_float(v.z) + __uint_as_float(o[i].z));
+                v.w = __float_as_uint(__uint_as_float(v.w) + __uint_as_float(o[i].w));
+            }
+            *reinterpret_cast<uint4*>(base + (size_t)r * row_stride_bytes) = v;
+        }
+    }
+    __syncwarp();
+}
+__device__ __forceinline__ void stage_flush(uint32_t stage, int lane, unsigned char* dst, size_t row_stride_bytes, int rows_ok)
+{
+    uint4 none[8];
+    stage_flush<false>(stage, lane, dst, row_stride_bytes, rows_ok, none);
+}
+
+// Plain epilogue: C (+)= accumulator, fp32 or bf16, ragged N handled element-wise.
+__device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok, int half,
+                                               uint32_t stage, int lane, int rows_ok, uint4 (&resid)[8])
+{
+    // resid (fp32 output added to what C holds, whole 32-column blocks): the residual block of the first 32 columns, loaded by the caller before it
+    // waited for the accumulator; each later block is requested as soon as the previous one has been stored
+    const int row0 = row - lane;                            // first row of this warp's 32
 #pragma unroll 1
     for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
         const int col = tc.col + c0;
         if (col >= g.N) break;                              // warp-uniform
         uint32_t v[32];
         tc_ld32(t_row + c0, v);
+        if (!g.out_f32 && !g.accumulate && col + 64 <= g.N) {          // bf16: 64 columns = 128 bytes per row
+            uint32_t v2[32];
+            tc_ld32(t_row + c0 + 32, v2);
+            tc_wait_ld();
+            float f[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * j + e]);
+                stage_put(stage, lane, j, pack_bf16x8(f));
+#pragma unroll
+                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v2[8 * j + e]);
+                stage_put(stage, lane, 4 + j, pack_bf16x8(f));
+            }
+            stage_flush(stage, lane, reinterpret_cast<unsigned char*>(static_cast<__nv_bfloat16*>(g.C) + (size_t)row0 * g.ldc + col),
+                               (size_t)g.ldc * 2, rows_ok);
+            c0 += 32;
+            continue;
+        }
         tc_wait_ld();
+        if (g.out_f32 && col + 32 <= g.N) {                 // fp32: 32 columns = 128 bytes per row
+#pragma unroll
+            for (int j = 0; j < 8; ++j) stage_put(stage, lane, j, make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]));
+            unsigned char* dst = reinterpret_cast<unsigned char*>(static_cast<float*>(g.C) + (size_t)row0 * g.ldc + col);
+            if (g.accumulate) {
+                stage_flush<true>(stage, lane, dst, (size_t)g.ldc * 4, rows_ok, resid);
+                if (c0 + 32 < (half + 1) * (BN / 2) && col + 64 <= g.N) residual_get(resid, lane, dst + 128, (size_t)g.ldc * 4, rows_ok);
+            } else {
+                stage_flush(stage, lane, dst, (size_t)g.ldc * 4, rows_ok);
+            }
+            continue;
+        }
         if (!row_ok) continue;
         if (g.out_f32) {
             float* cp = static_cast<float*>(g.C) + (size_t)row * g.ldc + col;
@@ -152,29 +253,37 @@ __device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoor
 
 // SwiGLU epilogue: the tile's first 128 columns are gate rows, the last 128 the matching up rows (the stacked weight is
 // stored in such 256-row groups); writes act = silu(gate) * up, bf16, [rows][N/2].
-__device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok, int half)
+__device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok, int half,
+                                                uint32_t stage, int lane, int rows_ok)
 {
-    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(g.C) + (size_t)row * g.ldc + tc.col / 2;
-#pragma unroll 1
-    for (int c0 = half * (BN / 4); c0 < (half + 1) * (BN / 4); c0 += 32) {
+    static_assert(BN / 4 == 64, "one staging pass per warp: 64 bf16 outputs = 128 bytes per row");
+    const int c_base = half * (BN / 4);
+#pragma unroll
+    for (int part = 0; part < 2; ++part) {
+        const int c0 = c_base + 32 * part;
         uint32_t gv[32], uv[32];
         tc_ld32(t_row + c0, gv);
         tc_ld32(t_row + BN / 2 + c0, uv);
         tc_wait_ld();
-        if (!row_ok) continue;
-        float f[32];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-            const float a = __uint_as_float(gv[e]);
-            f[e] = a / (1.f + __expf(-a)) * __uint_as_float(uv[e]);
+        for (int j = 0; j < 4; ++j) {
+            float f[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float a = __uint_as_float(gv[8 * j + e]);
+                f[e] = a / (1.f + __expf(-a)) * __uint_as_float(uv[8 * j + e]);
+            }
+            stage_put(stage, lane, 4 * part + j, pack_bf16x8(f));
         }
-        store_bf16x32(out + c0, f);
     }
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(g.C) + (size_t)(row - lane) * g.ldc + tc.col / 2 + c_base;
+    stage_flush(stage, lane, reinterpret_cast<unsigned char*>(out), (size_t)g.ldc * 2, rows_ok);
 }
 
 // QKV epilogue: heads of width dh; q and k heads get the rotary embedding (pairs (j, j + dh/2)); q goes to C (bf16,
 // [rows][N]), k and v go to the paged cache slot of the row's position.  Rows with a negative position write nothing.
-__device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok, int part)
+__device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok, int part,
+                                             uint32_t stage, int lane)
 {
     const int half = g.dh / 2;
     int p = -1, blk = -1, slot = 0;
@@ -188,15 +297,27 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord&
         const int col = tc.col + hb;
         if (col >= g.N) break;                                           // warp-uniform
         const int head = col / g.dh;
+        // where this thread's row of the head goes (0: nowhere): q into C, k and v into the cache slot of the row's position
+        const bool is_k = head < g.Hq + g.Hkv;
+        unsigned long long dst = 0;
+        if (p >= 0) {
+            if (head < g.Hq) {
+                dst = reinterpret_cast<unsigned long long>(static_cast<__nv_bfloat16*>(g.C) + (size_t)row * g.ldc + col);
+            } else if (blk >= 0) {
+                const int kh = is_k ? head - g.Hq : head - g.Hq - g.Hkv;
+                const size_t at = (((size_t)blk * g.Hkv + kh) * g.block_tokens + slot) * g.dh;
+                dst = g.kv_fp8 ? reinterpret_cast<unsigned long long>(reinterpret_cast<unsigned char*>(is_k ? g.k_pool : g.v_pool) + at)
+                               : reinterpret_cast<unsigned long long>((is_k ? g.k_pool : g.v_pool) + at);
+            }
+        }
 #pragma unroll 1
         for (int j0 = 0; j0 < half; j0 += 32) {
             uint32_t lo[32], hi[32];
             tc_ld32(t_row + hb + j0, lo);
             tc_ld32(t_row + hb + half + j0, hi);
             tc_wait_ld();
-            if (p < 0) continue;
             float a[32], b[32];
-            if (head < g.Hq + g.Hkv) {
+            if (is_k) {                                                  // q and k heads: rotary embedding
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                     const float2 t = cs[(size_t)(j0 + e) * g.M];
@@ -208,25 +329,32 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord&
 #pragma unroll
                 for (int e = 0; e < 32; ++e) { a[e] = __uint_as_float(lo[e]); b[e] = __uint_as_float(hi[e]); }
             }
-            __nv_bfloat16* dst;
-            if (head < g.Hq) {
-                dst = static_cast<__nv_bfloat16*>(g.C) + (size_t)row * g.ldc + col;
-            } else {
-                if (blk < 0) continue;
-                const bool is_k = head < g.Hq + g.Hkv;
-                const int kh = is_k ? head - g.Hq : head - g.Hq - g.Hkv;
-                const size_t at = (((size_t)blk * g.Hkv + kh) * g.block_tokens + slot) * g.dh;
-                if (g.kv_fp8) {
-                    unsigned char* d8 = reinterpret_cast<unsigned char*>(is_k ? g.k_pool : g.v_pool) + at;
+            if (g.kv_fp8 && head >= g.Hq) {
+                if (dst) {
+                    unsigned char* d8 = reinterpret_cast<unsigned char*>(dst);
                     const float sc = is_k ? g.k_scale : g.v_scale;
                     store_e4m3x32(d8 + j0, a, sc);
                     store_e4m3x32(d8 + half + j0, b, sc);
-                    continue;
                 }
-                dst = (is_k ? g.k_pool : g.v_pool) + at;
+                continue;
             }
-            store_bf16x32(dst + j0, a);
-            store_bf16x32(dst + half + j0, b);
+            // bf16: the row's two 64-byte pieces (columns j0.. and half + j0..) side by side in the staging area, then four
+            // rows per store instruction
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                stage_put(stage, lane, j, pack_bf16x8(a + 8 * j));
+                stage_put(stage, lane, 4 + j, pack_bf16x8(b + 8 * j));
+            }
+            __syncwarp();
+            const int piece = lane & 7;
+            const int off = piece < 4 ? j0 + piece * 8 : half + j0 + (piece - 4) * 8;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = i * 4 + (lane >> 3);
+                const unsigned long long rp = __shfl_sync(0xffffffffu, dst, r);
+                if (rp) *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(rp) + off) = stage_get(stage, r, piece);
+            }
+            __syncwarp();
         }
     }
 }
@@ -267,7 +395,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;                        // 1024-byte aligned stage ring
-    Ctl* ctl = reinterpret_cast<Ctl*>(smem_raw + (tiles - raw) + STAGES * STAGE_BYTES);
+    const uint32_t out_stage = tiles + STAGES * STAGE_BYTES;              // epilogue warps' staging areas
+    Ctl* ctl = reinterpret_cast<Ctl*>(smem_raw + (tiles - raw) + STAGES * STAGE_BYTES + (kEpiThreads / 32) * kOutStageBytes);
     volatile int* abort_flag = &ctl->abort;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -356,15 +485,25 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             if (!tile_coord(g, w, m_tiles, n_tiles, tc)) continue;
             const uint32_t acc = it & 1, acc_ph = (it >> 1) & 1;
             ++it;
-            if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_ph, abort_flag)) { ok = false; break; }
-            tc_fence_after();
             const int row_in_tile = quarter * 32 + lane;
             const int row = tc.c_row + row_in_tile;
             const bool row_ok = row_in_tile < tc.rows_valid;
+            const int rows_ok = min(32, tc.rows_valid - quarter * 32);       // valid rows among this warp's 32 (may be <= 0)
+            uint4 resid[8];
+            if constexpr (EPI == EPI_PLAIN) {
+                // += residual in fp32: ask for the first block of the residual before waiting for the accumulator
+                const int col = tc.col + half * (BN / 2);
+                if (g.out_f32 && g.accumulate && col + 32 <= g.N)
+                    residual_get(resid, lane, reinterpret_cast<const unsigned char*>(static_cast<const float*>(g.C) + (size_t)(row - lane) * g.ldc + col),
+                                 (size_t)g.ldc * 4, rows_ok);
+            }
+            if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_ph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-            if constexpr (EPI == EPI_SWIGLU) epilogue_swiglu(g, tc, t_row, row, row_ok, half);
-            else if constexpr (EPI == EPI_QKV) epilogue_qkv(g, tc, t_row, row, row_ok, half);
-            else epilogue_plain(g, tc, t_row, row, row_ok, half);
+            const uint32_t stage = out_stage + (warp - 2) * kOutStageBytes;
+            if constexpr (EPI == EPI_SWIGLU) epilogue_swiglu(g, tc, t_row, row, row_ok, half, stage, lane, rows_ok);
+            else if constexpr (EPI == EPI_QKV) epilogue_qkv(g, tc, t_row, row, row_ok, half, stage, lane);
+            else epilogue_plain(g, tc, t_row, row, row_ok, half, stage, lane, rows_ok, resid);
             tc_fence_before();
             mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
         }
