@@ -113,6 +113,64 @@ def moe_mlp(lw, m, top_k, router_logits=None):
     return out
 
 
+def ep_receive_layout(ids_by_rank, n_experts, ep_size):
+    """Expert parallelism over ep_size ranks (the paper's 235B-A22B configuration spans many GPUs, Section 5.1): rank r
+    owns the experts [r * E/ep_size, (r+1) * E/ep_size) and every rank routes its own tokens.  ids_by_rank[s] is the
+    [M_s][top_k] expert choice of source rank s.  Returns, for every destination rank d, the rows it receives, in the
+    order it stores them: its experts ascending; within an expert the source ranks ascending; within a source the
+    entries (token, slot) in row-major order.  Each row is (expert, source rank, source token, slot).  Also returns
+    recv_off[d][local expert][source] = index of the first row of that (expert, source) run."""
+    assert n_experts % ep_size == 0
+    per = n_experts // ep_size
+    rows, recv_off = [], []
+    for d in range(ep_size):
+        r, off = [], np.zeros((per, ep_size), np.int64)
+        for el in range(per):
+            e = d * per + el
+            for s in range(ep_size):
+                off[el, s] = len(r)
+                ids = np.asarray(ids_by_rank[s])
+                for m in range(ids.shape[0]):
+                    for j in range(ids.shape[1]):
+                        if ids[m, j] == e:
+                            r.append((e, s, m, j))
+        rows.append(r)
+        recv_off.append(off)
+    return rows, recv_off
+
+
+def ep_moe_mlp(lw, m_by_rank, top_k, ep_size, router_logits_by_rank=None):
+    """The mixture-of-experts MLP computed the expert-parallel way: route locally, send every (token, slot) row to the
+    rank that owns its expert, run each local expert on the rows it received, return the outputs to the source rank and
+    add them there in slot order with the routing weights.  Returns the list of per-rank outputs [M_s][d]."""
+    E = np.asarray(lw["router"]).shape[0]
+    ids_by, wts_by = [], []
+    for s in range(ep_size):
+        m = np.asarray(m_by_rank[s], F64)
+        lg = m @ np.asarray(lw["router"], F64).T if router_logits_by_rank is None else np.asarray(router_logits_by_rank[s], F64)
+        ids, wts = moe_route(lg, top_k)
+        ids_by.append(ids)
+        wts_by.append(wts)
+    rows, _ = ep_receive_layout(ids_by, E, ep_size)
+    back = [dict() for _ in range(ep_size)]                  # per source rank: (token, slot) -> expert output row
+    for d in range(ep_size):
+        for (e, s, t, j) in rows[d]:
+            x = np.asarray(m_by_rank[s], F64)[t]                                     # dispatch: the row crosses to rank d
+            g = np.asarray(lw["experts_gate"][e], F64)
+            u = np.asarray(lw["experts_up"][e], F64)
+            dn = np.asarray(lw["experts_down"][e], F64)
+            back[s][(t, j)] = (silu(g @ x) * (u @ x)) @ dn.T                          # combine: the row crosses back
+    out = []
+    for s in range(ep_size):
+        m = np.asarray(m_by_rank[s], F64)
+        o = np.zeros_like(m)
+        for t in range(m.shape[0]):
+            for j in range(top_k):
+                o[t] += wts_by[s][t, j] * back[s][(t, j)]
+        out.append(o)
+    return out
+
+
 def kv_as_cached(cfg, k, v):
     """What the attention reads back for freshly computed keys and values: themselves, or, with an 8-bit cache
     (cfg["kv_fp8"] = (k_scale, v_scale)), their e4m3 codes times the scale - for the new positions as for the old ones,

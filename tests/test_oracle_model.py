@@ -226,3 +226,39 @@ def test_ngram_propose_worked_examples():
                 best = t[max(hits) + n]
                 break
         assert d == (best if best is not None else t[-1])
+
+
+def test_ep_receive_layout_hand_worked():
+    # 2 ranks, 4 experts (rank 0 owns 0 and 1, rank 1 owns 2 and 3), top-2.
+    # rank 0 tokens: t0 -> (2, 0), t1 -> (1, 2), t2 -> (0, 1);   rank 1 tokens: t0 -> (3, 0), t1 -> (2, 3)
+    ids = [np.array([[2, 0], [1, 2], [0, 1]]), np.array([[3, 0], [2, 3]])]
+    rows, off = model.ep_receive_layout(ids, 4, 2)
+    # worked by hand: expert 0 gets (r0,t0,slot1), (r0,t2,slot0), then (r1,t0,slot1); expert 1 gets (r0,t1,slot0), (r0,t2,slot1)
+    assert rows[0] == [(0, 0, 0, 1), (0, 0, 2, 0), (0, 1, 0, 1), (1, 0, 1, 0), (1, 0, 2, 1)]
+    # expert 2 gets (r0,t0,slot0), (r0,t1,slot1), then (r1,t1,slot0); expert 3 gets (r1,t0,slot0), (r1,t1,slot1)
+    assert rows[1] == [(2, 0, 0, 0), (2, 0, 1, 1), (2, 1, 1, 0), (3, 1, 0, 0), (3, 1, 1, 1)]
+    assert off[0].tolist() == [[0, 2], [3, 5]] and off[1].tolist() == [[0, 2], [3, 3]]
+    # every (rank, token, slot) entry is received exactly once, by the owner of its expert
+    seen = sorted((s, t, j) for r in rows for (_, s, t, j) in r)
+    assert seen == sorted((s, t, j) for s in range(2) for t in range(ids[s].shape[0]) for j in range(2))
+    assert all(e // 2 == d for d in range(2) for (e, _, _, _) in rows[d])
+
+
+@pytest.mark.parametrize("ep_size", [1, 2, 4])
+def test_ep_moe_equals_unsharded_moe(ep_size):
+    # sharding invariance: what a token gets back does not depend on where its experts live or who else is in the batch
+    d, E, Fe, topk = 32, 8, 16, 3
+    cfg = dict(inputs.model_config("c5"), d_model=d, n_experts=E, d_expert_ffn=Fe, experts_top_k=topk,
+               n_q_heads=2, n_kv_heads=1, head_dim=16, dtype="f32")
+    lw = inputs.make_layer_weights(cfg, np.random.default_rng(14), std=0.2)
+    lw["router"] = (lw["router"] * 8).astype(np.float32)
+    rng = np.random.default_rng(15)
+    ms = [rng.standard_normal((n, d)) for n in [5, 0, 7, 3][:ep_size]]
+    got = model.ep_moe_mlp(lw, ms, topk, ep_size)
+    worst = 0.0
+    for s in range(ep_size):
+        ref = model.moe_mlp(lw, ms[s], topk)
+        assert got[s].shape == ref.shape
+        if ref.size:
+            worst = max(worst, float(np.max(np.abs(got[s] - ref))))
+    assert worst < 1e-12
