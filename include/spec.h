@@ -30,7 +30,7 @@
 extern "C" {
 #endif
 
-#define SPEC_ABI_VERSION 4u
+#define SPEC_ABI_VERSION 5u
 
 typedef struct spec_ctx spec_ctx; /* opaque */
 
@@ -46,7 +46,8 @@ typedef enum {
     SPEC_ERR_KV_EXHAUSTED = -16,
     SPEC_ERR_TOKEN_RANGE = -17,
     SPEC_ERR_BAD_PROB = -18,
-    SPEC_ERR_TIMEOUT = -19
+    SPEC_ERR_TIMEOUT = -19,
+    SPEC_ERR_EP_CAPACITY = -20
 } spec_status;
 
 enum { SPEC_DTYPE_BF16 = 0, SPEC_DTYPE_F32 = 1 };
@@ -297,6 +298,75 @@ size_t spec_attention_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int m
 spec_status spec_attention_noalloc(int B, int R, int Hq, int Hkv, int dh, int block_tokens, int max_blocks,
                                    const void* q, const void* k_pool, const void* v_pool, const int32_t* block_table,
                                    const int32_t* seq_len, void* out, int dtype, void* stream);
+
+/* ---- expert-parallel mixture-of-experts MLP (bf16) -----------------------------------------------------------
+ *
+ * The paper's largest configuration (Qwen3-235B-A22B, Section 5.1) does not fit one GPU: its experts are spread over
+ * the GPUs of an NVLink domain while every GPU keeps its own sequences.  These three calls are one MoE MLP block
+ * (router top-k, SwiGLU experts, weighted sum into the residual; the same arithmetic as the single-GPU block) for that
+ * arrangement.  Rank r of ep_size owns the experts [r * n_experts / ep_size, (r + 1) * n_experts / ep_size) and holds
+ * only their weights.  Data crosses between ranks by LOADS FROM PEER MEMORY inside the gather and combine kernels
+ * (each rank pulls what it needs; nothing is pushed, no kernel waits on another rank):
+ *
+ *   spec_ep_route    (on every rank)  router logits, top-k, and the per-expert lists of this rank's entries; copies
+ *                                     the rank's input rows into its window.  Reads and writes the own window only.
+ *   -- barrier: every rank's route has completed --
+ *   spec_ep_experts  (on every rank)  pulls the rows routed to the local experts out of all ranks' windows into local
+ *                                     memory (expert ascending, source rank ascending, the source's entry order), runs
+ *                                     the two grouped tensor-core GEMMs, leaves the expert outputs in the own window.
+ *   -- barrier: every rank's experts pass has completed --
+ *   spec_ep_combine  (on every rank)  for each own token pulls its top_k expert outputs from the owners' windows and
+ *                                     adds them to the residual in slot order (x += sum_j w_j * y_j, fused multiply-adds).
+ *   -- barrier before the next spec_ep_route reuses the windows --
+ *
+ * The barriers are the caller's (stream-ordered: a collective on the same stream, or a host barrier after a stream
+ * synchronise); on one GPU with several windows, stream order alone is the barrier.  A WINDOW is a caller-owned device
+ * buffer of spec_ep_sizes.window_bytes, 256-byte aligned, that the other ranks can address: peer_windows_host [ep_size]
+ * holds, in rank order, the device addresses under which THIS process sees every rank's window (its own included), e.g.
+ * from spec_ipc_open or from peer access between devices of one process.  scratch is private to the rank.
+ * Results do not depend on ep_size: a token's output is bit-identical to what the single-rank call computes for it.
+ *
+ * status [4] int32 (device, may be NULL): SPEC_ERR_EP_CAPACITY when more rows were routed to this rank than
+ * cap_rows (the surplus rows are dropped: their outputs are missing from the sums), SPEC_ERR_TIMEOUT from the GEMMs.
+ * Host errors: INVALID_ARG (NULL pointers, rank out of range), SHAPE (n_experts % ep_size, n_experts > 256, top_k > 32,
+ * d % 256, 2 * d_expert_ffn % 256, d_expert_ffn % 64, M > max_rows), UNSUPPORTED (ep_size > 16).  Every rank passes
+ * the same spec_ep_config except for ep_rank (the window layout is derived from it). */
+typedef struct spec_ep_config {
+    int32_t ep_size, ep_rank;
+    int32_t n_experts, top_k;
+    int32_t d, d_expert_ffn;
+    int32_t max_rows;           /* most rows (tokens) any rank routes per call                                          */
+    int32_t cap_rows;           /* most rows this rank can receive; ep_size * max_rows * min(top_k, local experts) is safe */
+} spec_ep_config;
+typedef struct spec_ep_sizes { size_t window_bytes, scratch_bytes; } spec_ep_sizes;
+enum {
+    SPEC_EP_T_IDS = 0,          /* window: [M][top_k] int32 selected experts, best first                               */
+    SPEC_EP_T_WTS,              /* window: [M][top_k] fp32 renormalised mixture weights                                 */
+    SPEC_EP_T_COUNTS,           /* window: [n_experts] int32 entries of this rank per expert                            */
+    SPEC_EP_T_RECV_OFF,         /* window: [local experts][ep_size] int32 first received row of each (expert, source)   */
+    SPEC_EP_T_RECV_TOTAL,       /* window: [1] int32 rows received (before clamping to cap_rows)                        */
+    SPEC_EP_T_EXPERT_OUT,       /* window: [cap_rows][d] fp32 expert outputs in receive order                           */
+    SPEC_EP_T_RECV_ROWS         /* scratch: [cap_rows][d] bf16 received rows in receive order                           */
+};
+spec_status spec_ep_query_sizes(const spec_ep_config* cfg, spec_ep_sizes* out);
+spec_status spec_ep_tensor(const spec_ep_config* cfg, void* window, void* scratch, int tensor_id, void** dev_ptr, size_t* bytes);
+/* h [M][d] bf16: the block's (normed) input rows; router_w [n_experts][d] bf16. */
+spec_status spec_ep_route(const spec_ep_config* cfg, void* window, void* scratch, int M, const void* h,
+                          const void* router_w, void* stream);
+/* w_gateup [local experts][2 * d_expert_ffn][d] (each expert grouped like SPEC_T_EXPERTS_GATEUP), w_down
+ * [local experts][d][d_expert_ffn]: the LOCAL experts only. */
+spec_status spec_ep_experts(const spec_ep_config* cfg, void* const* peer_windows_host, void* scratch,
+                            const void* w_gateup, const void* w_down, int32_t* status, void* stream);
+/* x [M][d] fp32 residual of this rank's rows (M as given to spec_ep_route). */
+spec_status spec_ep_combine(const spec_ep_config* cfg, void* const* peer_windows_host, int M, float* x, void* stream);
+
+/* Plumbing for windows in other processes (CUDA inter-process memory handles; the device memory must come from a
+ * plain device allocation).  spec_ipc_export fills handle_host [64] and the offset of dev_ptr inside its allocation;
+ * spec_ipc_open maps the allocation of a handle exported by ANOTHER process and returns its base address (add the
+ * offset); spec_ipc_close unmaps it.  Errors: INVALID_ARG, CUDA. */
+spec_status spec_ipc_export(void* dev_ptr, unsigned char* handle_host, uint64_t* offset_host);
+spec_status spec_ipc_open(const unsigned char* handle_host, void** base_dev_ptr);
+spec_status spec_ipc_close(void* base_dev_ptr);
 
 /* Optional per-pass device timing.  When enabled, the step functions bracket the passes selected by `mask` (bit 0
  * attention, bit 1 GEMMs, bit 2 softmax + sampling, bit 3 everything else) with CUDA events on the call's stream.

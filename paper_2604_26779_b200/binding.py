@@ -12,14 +12,15 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libspec.so")
 
-SPEC_ABI_VERSION = 4
+SPEC_ABI_VERSION = 5
 SPEC_DTYPE_BF16, SPEC_DTYPE_F32 = 0, 1
 SPEC_KV_MODEL, SPEC_KV_E4M3 = 0, 1
 SPEC_DRAFT_NONE, SPEC_DRAFT_EAGLE3, SPEC_DRAFT_MTP, SPEC_DRAFT_NGRAM = 0, 1, 2, 3
 
 STATUS_NAMES = {0: "SPEC_OK", -1: "SPEC_ERR_INVALID_ARG", -2: "SPEC_ERR_SHAPE", -3: "SPEC_ERR_UNSUPPORTED",
                 -4: "SPEC_ERR_STATE", -5: "SPEC_ERR_CUDA", -16: "SPEC_ERR_KV_EXHAUSTED",
-                -17: "SPEC_ERR_TOKEN_RANGE", -18: "SPEC_ERR_BAD_PROB", -19: "SPEC_ERR_TIMEOUT"}
+                -17: "SPEC_ERR_TOKEN_RANGE", -18: "SPEC_ERR_BAD_PROB", -19: "SPEC_ERR_TIMEOUT",
+                -20: "SPEC_ERR_EP_CAPACITY"}
 
 # tensor ids (spec.h)
 T = dict(EMBED=0, LM_HEAD=1, FINAL_NORM=2, ATTN_NORM=3, WQKV=4, WO=5, MLP_NORM=6, WGATEUP=7, WDOWN=8, ROUTER=9,
@@ -65,6 +66,17 @@ class spec_timing(C.Structure):
     _fields_ = [("ms", C.c_float * 4), ("passes", C.c_int32 * 4), ("dropped", C.c_int32)]
 
 
+class spec_ep_config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("ep_size", "ep_rank", "n_experts", "top_k", "d", "d_expert_ffn", "max_rows", "cap_rows")]
+
+
+class spec_ep_sizes(C.Structure):
+    _fields_ = [("window_bytes", C.c_size_t), ("scratch_bytes", C.c_size_t)]
+
+
+EP_T = dict(IDS=0, WTS=1, COUNTS=2, RECV_OFF=3, RECV_TOTAL=4, EXPERT_OUT=5, RECV_ROWS=6)
+
+
 class spec_step_report(C.Structure):
     _fields_ = [("device_status", C.c_int32), ("device_detail", C.c_int32), ("steps", C.c_int64),
                 ("emitted_tokens", C.c_int64), ("accepted_drafts", C.c_int64)]
@@ -98,6 +110,14 @@ SIGNATURES = {
     "spec_set_timing": (_i, [_vp, _u32]),
     "spec_get_timing": (_i, [_vp, C.POINTER(spec_timing), _vp]),
     "spec_selftest_bounded_wait": (_i, [_vp, _vp, _vp]),
+    "spec_ep_query_sizes": (_i, [C.POINTER(spec_ep_config), C.POINTER(spec_ep_sizes)]),
+    "spec_ep_tensor": (_i, [C.POINTER(spec_ep_config), _vp, _vp, _i, C.POINTER(_vp), C.POINTER(_sz)]),
+    "spec_ep_route": (_i, [C.POINTER(spec_ep_config), _vp, _vp, _i, _vp, _vp, _vp]),
+    "spec_ep_experts": (_i, [C.POINTER(spec_ep_config), C.POINTER(_vp), _vp, _vp, _vp, _vp, _vp]),
+    "spec_ep_combine": (_i, [C.POINTER(spec_ep_config), C.POINTER(_vp), _i, _vp, _vp]),
+    "spec_ipc_export": (_i, [_vp, _vp, C.POINTER(_u64)]),
+    "spec_ipc_open": (_i, [_vp, C.POINTER(_vp)]),
+    "spec_ipc_close": (_i, [_vp]),
     "spec_launch_count": (C.c_int64, []),
     "spec_version": (C.c_char_p, []),
 }
@@ -212,6 +232,55 @@ def spec_attention_noalloc(q, k_pool, v_pool, block_table, seq_len, out, stream=
     _check(lib().spec_attention_noalloc(B, R, Hq, Hkv, dh, bt, block_table.shape[1], _ptr(q), _ptr(k_pool), _ptr(v_pool),
                                         _ptr(block_table), _ptr(seq_len), _ptr(out), dt, _stream(stream)),
            "spec_attention_noalloc")
+
+
+def spec_ep_query_sizes(cfg):
+    out = spec_ep_sizes()
+    _check(lib().spec_ep_query_sizes(C.byref(cfg), C.byref(out)), "spec_ep_query_sizes")
+    return out
+
+
+def spec_ep_tensor(cfg, window, scratch, tensor_id):
+    """(device address, bytes) of one piece of a window / scratch."""
+    p, n = _vp(), _sz()
+    _check(lib().spec_ep_tensor(C.byref(cfg), _ptr(window), _ptr(scratch), tensor_id, C.byref(p), C.byref(n)), "spec_ep_tensor")
+    return p.value, n.value
+
+
+def _peer_array(peer_windows):
+    return (_vp * len(peer_windows))(*[_ptr(w) for w in peer_windows])
+
+
+def spec_ep_route(cfg, window, scratch, M, h, router_w, stream=None):
+    _check(lib().spec_ep_route(C.byref(cfg), _ptr(window), _ptr(scratch), M, _ptr(h), _ptr(router_w), _stream(stream)), "spec_ep_route")
+
+
+def spec_ep_experts(cfg, peer_windows, scratch, w_gateup, w_down, status=None, stream=None):
+    _check(lib().spec_ep_experts(C.byref(cfg), _peer_array(peer_windows), _ptr(scratch), _ptr(w_gateup), _ptr(w_down),
+                                 _ptr(status), _stream(stream)), "spec_ep_experts")
+
+
+def spec_ep_combine(cfg, peer_windows, M, x, stream=None):
+    _check(lib().spec_ep_combine(C.byref(cfg), _peer_array(peer_windows), M, _ptr(x), _stream(stream)), "spec_ep_combine")
+
+
+def spec_ipc_export(dev_ptr):
+    """(64-byte handle, offset of dev_ptr inside its allocation)."""
+    h = (C.c_ubyte * 64)()
+    off = _u64()
+    _check(lib().spec_ipc_export(_ptr(dev_ptr), h, C.byref(off)), "spec_ipc_export")
+    return bytes(h), off.value
+
+
+def spec_ipc_open(handle):
+    buf = (C.c_ubyte * 64).from_buffer_copy(handle)
+    p = _vp()
+    _check(lib().spec_ipc_open(buf, C.byref(p)), "spec_ipc_open")
+    return p.value
+
+
+def spec_ipc_close(base):
+    _check(lib().spec_ipc_close(base), "spec_ipc_close")
 
 
 def spec_version():

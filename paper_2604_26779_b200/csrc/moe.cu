@@ -133,6 +133,13 @@ spec_status launch_moe_route(int M, int E, int top_k, const float* logits, int32
     return launch_status();
 }
 
+// Ranks n_entries routed entries inside their experts (entry order) and counts them per expert; n_entries may be 0.
+spec_status launch_moe_rank(int n_entries, int E, const int32_t* ids, int32_t* rank, int32_t* counts, cudaStream_t st)
+{
+    moe_rank_kernel<<<E, 256, 0, st>>>(n_entries, ids, rank, counts);
+    return launch_status();
+}
+
 spec_status launch_moe_permute(int M, int E, int top_k, int d, const int32_t* ids, int32_t* rank, int32_t* counts,
                                int32_t* offsets, int32_t* inv, const void* h, void* a_perm, cudaStream_t st)
 {

@@ -45,7 +45,13 @@ def make_spec_config(cfg: dict, *, draft_kind: str = "none", k_max: int = 3, max
 
 def stack_gate_up(gate, up):
     """[.., F, d] gate and up -> the library's stacked layout [.., 2F, d]: 256-row groups of 128 gate rows followed by
-    the matching 128 up rows."""
+    the matching 128 up rows.  numpy arrays or torch tensors."""
+    if hasattr(gate, "data_ptr"):
+        F, d = gate.shape[-2:]
+        lead = tuple(gate.shape[:-2])
+        g = gate.reshape(lead + (F // 128, 128, d))
+        u = up.reshape(lead + (F // 128, 128, d))
+        return torch.cat([g, u], dim=-2).reshape(lead + (2 * F, d))
     gate, up = np.asarray(gate), np.asarray(up)
     F, d = gate.shape[-2:]
     lead = gate.shape[:-2]
