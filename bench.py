@@ -304,6 +304,77 @@ def run_sampler_microbench(args):
     return 0
 
 
+def run_ep_microbench(args):
+    """The expert-parallel MoE block of the 235B-A22B shape (128 experts, top-8, d 4096, expert FFN 1536) with `--ep` ranks
+    emulated inside this process on one GPU: every rank routes B*(k+1) rows, owns 128/ep experts, and pulls rows / expert
+    outputs from the other ranks' windows - which here live on the same GPU, so the pulls run at HBM speed and the line
+    also gives the time the same bytes would need on NVLink at the measured peer-copy rate.  Phases are timed with CUDA
+    events over all ranks and divided by the number of ranks (what one GPU of the group would spend)."""
+    import torch
+    from paper_2604_26779_b200 import expert_parallel as ep
+    from paper_2604_26779_b200.engine import stack_gate_up
+    R, E, top_k, d, Fe = args.ep, 128, 8, 4096, 1536
+    M = args.batch * (args.k + 1)
+    per = E // R
+    cap = min(ep.safe_cap_rows(R, E, top_k, M), int(args.ep_capacity * M * top_k))
+    gen = torch.Generator(device="cuda"); gen.manual_seed(2604026779 + 5000)
+    rn = lambda shape, scale: (torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32) * scale).to(torch.bfloat16)
+    router = rn((E, d), 1.0 / d ** 0.5)                       # router logits ~ N(0, 1), as in the c5 recipe
+    gus, dns = [], []
+    for r in range(R):
+        gus.append(stack_gate_up(rn((per, Fe, d), d ** -0.5), rn((per, Fe, d), d ** -0.5)).contiguous())
+        dns.append(rn((per, d, Fe), Fe ** -0.5))
+    hs = [rn((M, d), 1.0) for _ in range(R)]
+    xs = [torch.zeros((M, d), dtype=torch.float32, device="cuda") for _ in range(R)]
+    ranks = [ep.EpRank(R, r, E, top_k, d, Fe, M, cap) for r in range(R)]
+    addrs = [r.window.data_ptr() for r in ranks]
+    for r in ranks:
+        r.set_peers(addrs)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    acc = [0.0, 0.0, 0.0]
+    clocks = ClockSampler(torch.cuda.current_device())
+    for it in range(args.warmup + args.steps):
+        if it == args.warmup:
+            clocks.start()
+        ev[0].record()
+        for r, h in zip(ranks, hs):
+            r.route(h, router)
+        ev[1].record()
+        for r, gu, dn in zip(ranks, gus, dns):
+            r.experts(gu, dn)
+        ev[2].record()
+        for r, x in zip(ranks, xs):
+            r.combine(x)
+        ev[3].record()
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            for i in range(3):
+                acc[i] += ev[i].elapsed_time(ev[i + 1])
+    ck = clocks.stop()
+    for r in ranks:
+        r.check_status()
+    ms = [a / args.steps / R for a in acc]
+    recv = [int(r.tensor("RECV_TOTAL")[0]) for r in ranks]
+    rows = sum(recv) / R
+    remote = (R - 1) / R
+    disp_b, comb_b = rows * d * 2, M * top_k * d * 4
+    nvl = 770.0e9
+    hbm_peak, _, kind = measured_peaks()
+    print(json.dumps({
+        "metric": "expert-parallel MoE block, 235B-A22B shape, ranks emulated on one GPU (not the headline)", "unit": "ms per rank",
+        "n_gpus": 1, "ep_size": R, "rows_per_rank": M, "experts_per_rank": per, "cap_rows": cap, "steps": args.steps, "warmup": args.warmup,
+        "ms_route": ms[0], "ms_experts": ms[1], "ms_combine": ms[2], "ms_block": sum(ms),
+        "rows_received": {"mean": rows, "min": min(recv), "max": max(recv)},
+        "dispatch_bytes_per_rank": disp_b, "combine_bytes_per_rank": comb_b,
+        "combine_GBps_local": comb_b / ms[2] / 1e6 if ms[2] > 0 else None,
+        "nvlink_ms_at_770GBps": {"dispatch": disp_b * remote / nvl * 1e3, "combine": comb_b * remote / nvl * 1e3},
+        "expert_gemm_tflops": rows * (2 * 2 * Fe * d + 2 * d * Fe) / ms[1] / 1e9 if ms[1] > 0 else None,
+        "peak_GBps": hbm_peak, "peak_source": kind, "dtype": "bf16", "data": "synthetic", "clocks": ck,
+        "config": {"workload": "c5ep: one MoE MLP block, 128 experts top-8, d=4096, expert FFN 1536, router logits ~N(0,1)",
+                   "l2": "weights + windows of all ranks exceed L2"}}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -328,7 +399,10 @@ def main():
     ap.add_argument("--k-sweep", default=None,
                     help="comma-separated draft lengths, e.g. 1,3,5,7: times the c3 step at each k on one engine built for the "
                          "largest (not the headline run: prints its own JSON line)")
-    ap.add_argument("--workload", default="c3", choices=["c3", "c4", "c5", "c2"],
+    ap.add_argument("--ep", type=int, default=8, help="c5ep only: ranks of the expert-parallel group (emulated on one GPU)")
+    ap.add_argument("--ep-capacity", type=float, default=2.0,
+                    help="c5ep only: receive capacity per rank as a multiple of the mean load rows*top_k (capped by the worst case)")
+    ap.add_argument("--workload", default="c3", choices=["c3", "c4", "c5", "c2", "c5ep"],
                     help="c3 = the headline 8B + EAGLE-3 workload; c4 = 8B + MTP head, B=512, lognormal lengths; "
                          "c5 = one 235B-A22B-shaped MoE layer + LM head, B=256, cache length 8192 (measurement of the "
                          "other configurations; the reported metric line is c3)")
@@ -345,6 +419,8 @@ def main():
     torch.cuda.set_device(local)
     if args.workload == "c2":
         return run_sampler_microbench(args) if rank == 0 else 0
+    if args.workload == "c5ep":
+        return run_ep_microbench(args) if rank == 0 else 0
     if args.k_sweep:
         return run_k_sweep(args, [int(x) for x in args.k_sweep.split(",")]) if rank == 0 else 0
     dist = None

@@ -28,15 +28,18 @@ constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTE
 constexpr int kThreads = 320;          // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue (two per tensor-memory lane quarter)
 constexpr int kEpiThreads = 256;
 constexpr uint32_t kTmemCols = 512;
+constexpr int kMaxGroups = 256;          // grouped mode: most groups per launch
 constexpr int kOutStageBytes = 32 * 128;  // per epilogue warp: 32 rows x 128 bytes, where a warp turns its row-per-thread
                                           // accumulator fragments into row-contiguous 128-byte pieces before they go to memory
-constexpr int kSmemBytes = STAGES * STAGE_BYTES + (kEpiThreads / 32) * kOutStageBytes + 1024 + 256;
+constexpr int kSmemBytes = STAGES * STAGE_BYTES + (kEpiThreads / 32) * kOutStageBytes + 1024 + 128 + (kMaxGroups + 1) * 4;
+static_assert(kSmemBytes <= 232448, "shared memory per CTA");
 #define TRY_LAUNCH(expr) do { spec_status s__ = (expr); if (s__ != SPEC_OK) return s__; } while (0)
 
 struct Ctl {
     uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain;
     uint32_t tmem_base;
     int abort;
+    int pref[kMaxGroups + 1];          // grouped mode: m-tiles of the groups before group e (pref[E] = all m-tiles)
 };
 
 // Shared-memory matrix descriptor of a K-major tile whose rows are 64 bf16 (128 bytes) wide, 128-byte swizzle:
@@ -360,30 +363,33 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord&
 }
 
 // Decodes work item w into (m-tile, n-tile, group) and the tile's row window.  Returns false for an empty tile.
-__device__ __forceinline__ bool tile_coord(const GemmArgs& g, int w, int m_tiles, int n_tiles, TileCoord& t)
+// Grouped mode enumerates only the m-tiles that exist (pref = running count of ceil(counts / BM)): group by group, within
+// a group the n-tiles in turn, within an n-tile the group's m-tiles next to each other, so the CTAs that run at the same
+// time share weight tiles (a group with several m-tiles reads its weights from memory once, not once per m-tile) and no
+// CTA spends turns on tiles that do not exist.
+__device__ __forceinline__ bool tile_coord(const GemmArgs& g, int w, int m_tiles, int n_tiles, const int* pref, TileCoord& t)
 {
     const int kb_count = (g.K + BK - 1) / BK;
     t.kb0 = 0; t.kb1 = kb_count;
     int split = 0;
-    if (g.splits > 1) { split = w % g.splits; w /= g.splits; t.kb0 = split * g.kb_per; t.kb1 = min(kb_count, t.kb0 + g.kb_per); }
-    int mt = w % m_tiles, nt = (w / m_tiles) % n_tiles;
     if (g.E > 0) {
-        // grouped: m-tile index slowest.  Most groups fill only their first m-tile, so the non-empty items are the first
-        // E * n_tiles ones and the round-robin over CTAs spreads them evenly (with the m-tile fastest, a stride of 148
-        // would hand every non-empty item to a quarter of the CTAs)
-        const int per = n_tiles * g.E, rem = w % per;
-        mt = w / per;
-        nt = rem % n_tiles;
-        const int e = rem / n_tiles;
-        const int cnt = g.counts[e];
-        if (mt * BM >= cnt) return false;
-        const int off = g.offsets[e];
+        int lo = 0, hi = g.E - 1;                            // last group whose first item is <= w
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (pref[mid] * n_tiles <= w) lo = mid; else hi = mid - 1;
+        }
+        const int e = lo, mts = pref[e + 1] - pref[e], r = w - pref[e] * n_tiles;
+        const int nt = r / mts, mt = r - nt * mts;
+        const int cnt = g.counts[e], off = g.offsets[e];
         t.a_row = off + mt * BM; t.c_row = t.a_row; t.rows_valid = cnt - mt * BM;
         t.b_row = e * g.N + nt * BN;
-    } else {
-        t.a_row = mt * BM; t.c_row = t.a_row + split * g.M; t.rows_valid = g.M - mt * BM;
-        t.b_row = nt * BN;
+        t.col = nt * BN;
+        return true;
     }
+    if (g.splits > 1) { split = w % g.splits; w /= g.splits; t.kb0 = split * g.kb_per; t.kb1 = min(kb_count, t.kb0 + g.kb_per); }
+    const int mt = w % m_tiles, nt = (w / m_tiles) % n_tiles;
+    t.a_row = mt * BM; t.c_row = t.a_row + split * g.M; t.rows_valid = g.M - mt * BM;
+    t.b_row = nt * BN;
     t.col = nt * BN;
     return true;
 }
@@ -400,8 +406,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     volatile int* abort_flag = &ctl->abort;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    const int m_tiles = g.E > 0 ? g.max_m_tiles : (g.M + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
-    const int n_work = m_tiles * n_tiles * (g.E > 0 ? g.E : 1) * (g.splits > 1 ? g.splits : 1);
+    const int m_tiles = (g.M + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
+    if (g.E > 0 && threadIdx.x == 64) {                     // grouped: the m-tile prefix table (counts live on the device)
+        int run = 0;
+        for (int e = 0; e < g.E; ++e) { ctl->pref[e] = run; run += (min(g.counts[e], g.max_m_tiles * BM) + BM - 1) / BM; }
+        ctl->pref[g.E] = run;
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
@@ -419,6 +429,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    const int* pref = ctl->pref;
+    const int n_work = g.E > 0 ? pref[g.E] * n_tiles : m_tiles * n_tiles * (g.splits > 1 ? g.splits : 1);
 
     if (warp == 0) {
         // ---- TMA producer ----
@@ -427,7 +439,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             bool ok = true;
             for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
                 TileCoord tc;
-                if (!tile_coord(g, w, m_tiles, n_tiles, tc)) continue;
+                if (!tile_coord(g, w, m_tiles, n_tiles, pref, tc)) continue;
                 for (int kb = tc.kb0; kb < tc.kb1; ++kb) {
                     if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t bar = smem_u32(&ctl->full[s]);
@@ -450,7 +462,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             int it = 0;
             for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
                 TileCoord tc;
-                if (!tile_coord(g, w, m_tiles, n_tiles, tc)) continue;
+                if (!tile_coord(g, w, m_tiles, n_tiles, pref, tc)) continue;
                 const uint32_t acc = it & 1, acc_ph = (it >> 1) & 1;
                 ++it;
                 if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -482,7 +494,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         int it = 0;
         for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
             TileCoord tc;
-            if (!tile_coord(g, w, m_tiles, n_tiles, tc)) continue;
+            if (!tile_coord(g, w, m_tiles, n_tiles, pref, tc)) continue;
             const uint32_t acc = it & 1, acc_ph = (it >> 1) & 1;
             ++it;
             const int row_in_tile = quarter * 32 + lane;
@@ -704,7 +716,7 @@ spec_status launch_gemm_grouped(int rows_total, int max_rows_per_group, int E, i
                                 int32_t* status, cudaStream_t st)
 {
     if (rows_total == 0 || E == 0) return SPEC_OK;
-    if (N % BN != 0 || K % 8 != 0) return SPEC_ERR_SHAPE;
+    if (N % BN != 0 || K % 8 != 0 || E > kMaxGroups) return SPEC_ERR_SHAPE;
     if (!init_once()) return SPEC_ERR_CUDA;
     CUtensorMap ma, mb;
     if (!make_map(&ma, A, (uint64_t)rows_total, (uint64_t)K, (uint64_t)K, BM)) return SPEC_ERR_CUDA;
