@@ -83,7 +83,7 @@ __device__ __forceinline__ void e4m3x4_to_f16x4(uint32_t w, uint32_t& lo, uint32
 }
 // One CTA = 4 warps, each taking one 16-token block of every 64-token tile (16 query rows per KV head at most).
 template <int STAGES>
-__global__ void __launch_bounds__(kThreads) attn_fp8_kernel(const Fp8Args a)
+__global__ void __launch_bounds__(kThreads, 4) attn_fp8_kernel(const Fp8Args a)
 {
     constexpr int DH = 128, WM = 1, WN = 4;
     constexpr int CH = DH / 8;                               // 16-byte chunks per fp16 row
