@@ -160,7 +160,7 @@ __global__ void __launch_bounds__(256) ep_combine_kernel(Peers peers, EpLayout L
         const int owner = e / per, el = e % per;
         const int row = reinterpret_cast<const int32_t*>(peers.win[owner] + L.recv_off)[el * R + me] +
                         reinterpret_cast<const int32_t*>(peers.win[me] + L.rank)[i];
-        s_row[threadIdx.x] = row < cap_rows ? reinterpret_cast<const float*>(peers.win[owner] + L.y) + (size_t)row * d : nullptr;
+        s_row[threadIdx.x] = (row >= 0 && row < cap_rows) ? reinterpret_cast<const float*>(peers.win[owner] + L.y) + (size_t)row * d : nullptr;
         s_w[threadIdx.x] = reinterpret_cast<const float*>(peers.win[me] + L.wts)[i];
     }
     __syncthreads();
@@ -270,7 +270,6 @@ extern "C" spec_status spec_ep_experts(const spec_ep_config* cfg, void* const* p
     if (peer_windows_host == nullptr || scratch == nullptr || w_gateup == nullptr || w_down == nullptr) return SPEC_ERR_INVALID_ARG;
     Peers peers;
     if (!fill_peers(*cfg, peer_windows_host, peers)) return SPEC_ERR_INVALID_ARG;
-    if (cfg->cap_rows == 0) return SPEC_OK;
     const EpLayout l = make_layout(*cfg);
     cudaStream_t st = (cudaStream_t)stream;
     unsigned char* sc = static_cast<unsigned char*>(scratch);
@@ -288,7 +287,7 @@ extern "C" spec_status spec_ep_experts(const spec_ep_config* cfg, void* const* p
     const int grid = (int)(want < cfg->cap_rows ? want : (cfg->cap_rows > 0 ? cfg->cap_rows : 1));
     ep_pull_kernel<<<grid, 256, 0, st>>>(peers, l, R, me, E, cfg->top_k, d, cfg->cap_rows, a_perm, gc, go, status);
     spec_status r = launch_status();
-    if (r != SPEC_OK) return r;
+    if (r != SPEC_OK || cfg->cap_rows == 0) return r;      // capacity 0: the offsets and the status are published, nothing to compute
     const long long most = (long long)R * cfg->max_rows;
     const int max_per_group = (int)(most < cfg->cap_rows ? most : cfg->cap_rows);
     r = launch_gemm_grouped(cfg->cap_rows, max_per_group, per, 2 * Fe, d, a_perm, w_gateup, sc + l.act, SPEC_DTYPE_BF16, 1, gc, go, status, st);
