@@ -198,6 +198,18 @@ spec_status spec_seq_replace(spec_ctx* ctx, int n, const int32_t* slots_host, co
 
 /* ---- one speculation step (Introduction, third paragraph) ------------------------------------------------- */
 
+/* Renumbers the running sequences so that the batch shrinks: new slot j takes over everything of old slot
+ * keep_slots_host[j] (strictly ascending old slots), every slot that is not listed is retired first (its blocks
+ * go back to the free stack in slot order, logical block order, as spec_seq_replace does) and the context
+ * continues with n_keep sequences - every later pass (projections, attention plan, sampler) then works on
+ * n_keep * (k+1) rows instead of carrying the retired slots' inert rows: what the long tail of a rollout needs
+ * (paper: Section 5.2, thin batches).  Between steps only.  The uniforms are drawn per slot, so a moved sequence
+ * continues on its new slot's stream.  The logits and hidden-state tensors of the last step are not renumbered
+ * (read them before); token, log-probability and block tables are.  The batch cannot grow again without
+ * spec_seq_init.  Synchronises `stream`.  Errors: INVALID_ARG (order, range), SHAPE, STATE (a verified step is
+ * waiting for its commit). */
+spec_status spec_seq_compact(spec_ctx* ctx, int n_keep, const int32_t* keep_slots_host, void* stream);
+
 /* S1 draft propose.  Runs the draft head: pass 0 consumes the (tapped hidden state, next token) pairs of the
  * positions committed by the previous step, passes 1..k-1 feed the head its own output; fills draft tokens
  * d_1..d_k (d_i drawn from q_i with the stream-1 uniforms), draft logits and their row statistics.

@@ -186,6 +186,19 @@ def kv_replace(slots, new_len, block_tokens, seq_len, block_table, free_stack, f
                                         _p(free_stack, ctypes.c_int32), _p(free_top, ctypes.c_int32))
 
 
+def kv_compact(keep, block_tokens, seq_len, block_table, free_stack, free_top):
+    """Shrinks the batch to the sequences in the (strictly ascending) slots `keep`: every other slot is retired in slot
+    order (kv_replace with a negative length: its blocks go back to the free stack in logical order), then new slot j takes
+    old slot keep[j]'s length and table row.  Returns (seq_len, block_table) of the len(keep) remaining sequences; the free
+    stack is updated in place.  (Continuous batching, paper Section 5.2: the long tail of a rollout runs on a thin batch.)"""
+    keep = [int(k) for k in keep]
+    assert all(a < b for a, b in zip(keep, keep[1:])) and all(0 <= k < seq_len.shape[0] for k in keep)
+    dropped = [b for b in range(seq_len.shape[0]) if b not in keep]
+    if dropped:
+        assert kv_replace(dropped, [-1] * len(dropped), block_tokens, seq_len, block_table, free_stack, free_top) == 0
+    return seq_len[keep].copy(), block_table[keep].copy()
+
+
 def e4m3_quantize(x, scale=1.0):
     """e4m3 codes (uint8) of x / scale: round to nearest even, saturating at 448."""
     xf = _f32(x)

@@ -92,6 +92,7 @@ SIGNATURES = {
     "spec_tensor": (_i, [_vp, _i, _i, C.POINTER(_vp), C.POINTER(_sz)]),
     "spec_seq_init": (_i, [_vp, _i, _vp, _vp, _vp, _vp]),
     "spec_seq_replace": (_i, [_vp, _i, _vp, _vp, _vp, _vp]),
+    "spec_seq_compact": (_i, [_vp, _i, _vp, _vp]),
     "spec_draft": (_i, [_vp, _i, _vp]),
     "spec_verify": (_i, [_vp, _i, _vp, _vp]),
     "spec_reject_sample": (_i, [_vp, _i, _vp, _vp]),

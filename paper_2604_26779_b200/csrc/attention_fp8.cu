@@ -319,8 +319,8 @@ spec_status launch_attention_fp8(const AttnArgs& a, cudaStream_t st)
     constexpr int kStages = STAGES * (4 * kBT * 128 * 2), kMerge = 4 * 16 * 130 * 4;
     constexpr int smem = kStages > kMerge ? kStages : kMerge;      // code stages; the unit-end merge of the four warps reuses them
     const int group = a.Hq / a.Hkv;
-    const int max_chunks = max_chunks_for(a.max_kv_len);
     if (a.scratch_bytes < attention_mma_scratch_bytes(a.B, a.R, a.Hq, a.Hkv, a.dh, a.max_kv_len)) return SPEC_ERR_SHAPE;
+    const int max_chunks = max_chunks_for(a.max_kv_len);
     const PlanView pv = carve_plan(a.scratch, a.B, a.Hkv, 16, a.dh, max_chunks);
     auto kern = attn_fp8_kernel<STAGES>;
     static bool configured = false;
@@ -332,7 +332,7 @@ spec_status launch_attention_fp8(const AttnArgs& a, cudaStream_t st)
               a.block_table, a.max_blocks, a.pos, a.R, group, a.Hkv, (__nv_bfloat16*)a.out, a.out_row_stride,
               1.4426950408889634f / sqrtf((float)a.dh) * a.k_scale, a.v_scale, pv, a.launch_index % kCounters};
     if (a.launch_index % kCounters == 0) {
-        const spec_status s = launch_attn_plan(a.B, a.R, a.pos, max_chunks, pv, st);
+        const spec_status s = launch_attn_plan(a.B, a.R, a.pos, a.Hkv, 4 * 148, max_chunks, pv, st);
         if (s != SPEC_OK) return s;
     }
     int sms = 0, dev = 0;

@@ -50,11 +50,35 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 }
 
 // ---- planning: one CTA, sequences in index order -------------------------------------------------------------------
-__global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(int B, int R, const int32_t* __restrict__ pos,
-                                                                 int max_chunks, PlanView pv)
+__global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(int B, int R, const int32_t* __restrict__ pos, int Hkv, int n_ctas,
+                                                                 int cap_entries, PlanView pv)
 {
     __shared__ int s_warp[33];
+    __shared__ long long s_tot[2];
     for (int i = threadIdx.x; i < kCounters; i += kPlanThreads) pv.counters[i] = 0;
+    if (threadIdx.x == 0) { s_tot[0] = 0; s_tot[1] = 0; }
+    __syncthreads();
+    // Chunk length of this launch.  With a full batch there are far more units than CTAs and kChunk-token chunks are best; a
+    // thin batch (the long tail of a rollout: most slots retired) would leave most CTAs without a unit, so the chunk is halved
+    // while the unit count stays under two per CTA - as long as the unit list still fits what the scratch was sized for.
+    {
+        long long tok = 0, act = 0;
+        for (int b = threadIdx.x; b < B; b += kPlanThreads) {
+            int ntok = 0;
+            for (int i = 0; i < R; ++i) ntok = max(ntok, pos[(size_t)b * R + i] + 1);
+            tok += ntok; act += ntok > 0;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { tok += __shfl_xor_sync(0xffffffffu, tok, o); act += __shfl_xor_sync(0xffffffffu, act, o); }
+        if ((threadIdx.x & 31) == 0) { atomicAdd(reinterpret_cast<unsigned long long*>(&s_tot[0]), (unsigned long long)tok);
+                                       atomicAdd(reinterpret_cast<unsigned long long*>(&s_tot[1]), (unsigned long long)act); }
+    }
+    __syncthreads();
+    int chunk = kChunk;
+    {
+        const long long tok = s_tot[0], act = s_tot[1];
+        while (chunk > kChunkMin && (tok / chunk + act) * Hkv < 2LL * n_ctas && tok / (chunk / 2) + act <= cap_entries) chunk >>= 1;
+    }
     int carry = 0;
     for (int base = 0; base < B; base += kPlanThreads) {
         const int b = base + threadIdx.x;
@@ -63,12 +87,11 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(int B, int R, c
             for (int i = 0; i < R; ++i) ntok = max(ntok, pos[(size_t)b * R + i] + 1);
             // a few tokens past a multiple of the chunk length (the k+1 new rows on top of a round cache length) do not
             // open another chunk: a chunk may run up to kChunkSlack tokens over
-            nc = ntok > 0 ? max(1, (ntok - kChunkSlack + kChunk - 1) / kChunk) : 0;
+            nc = ntok > 0 ? max(1, (ntok - kChunkSlack + chunk - 1) / chunk) : 0;
             if (nc > 0) {
                 per = ((ntok + nc - 1) / nc + kTileTok - 1) / kTileTok * kTileTok;
-                nc = (ntok + per - 1) / per;
+                nc = (ntok + per - 1) / per;                 // <= ntok / chunk + 1, so the list holds at most tok / chunk + act units
             }
-            nc = min(nc, max_chunks);
         }
         // exclusive scan of nc over the block
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -390,7 +413,7 @@ spec_status run_mma(const MmaArgs& m, int B, bool plan, int max_chunks, cudaStre
         configured = true;
     }
     if (plan) {
-        attn_plan_kernel<<<1, kPlanThreads, 0, st>>>(B, m.R, m.pos, max_chunks, m.pv);
+        attn_plan_kernel<<<1, kPlanThreads, 0, st>>>(B, m.R, m.pos, m.Hkv, 2 * sm_count(), B * max_chunks, m.pv);
         if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
     }
     const int ctas_per_sm = (228 * 1024) / (smem + 2048);
@@ -411,15 +434,12 @@ bool attention_mma_supported(const AttnArgs& a)
 
 size_t attention_mma_scratch_bytes(int B, int R, int Hq, int Hkv, int dh, int max_kv_len)
 {
-    const int rows_alloc = rows_alloc_for(R * (Hq / Hkv));
-    const size_t entries = (size_t)B * max_chunks_for(max_kv_len);
-    return align_up((size_t)kCounters * 4 + 4, 256) + 2 * align_up((size_t)B * 4, 256) + align_up(entries * sizeof(Unit), 256) +
-           align_up(entries * Hkv * rows_alloc * dh * 4, 256) + align_up(entries * Hkv * rows_alloc * 8, 256);
+    return plan_scratch_bytes(B, Hkv, rows_alloc_for(R * (Hq / Hkv)), dh, max_chunks_for(max_kv_len));
 }
 
-spec_status attn::launch_attn_plan(int B, int R, const int32_t* pos, int max_chunks, const PlanView& pv, cudaStream_t st)
+spec_status attn::launch_attn_plan(int B, int R, const int32_t* pos, int Hkv, int n_ctas, int max_chunks, const PlanView& pv, cudaStream_t st)
 {
-    attn_plan_kernel<<<1, kPlanThreads, 0, st>>>(B, R, pos, max_chunks, pv);
+    attn_plan_kernel<<<1, kPlanThreads, 0, st>>>(B, R, pos, Hkv, n_ctas, B * max_chunks, pv);
     return launch_status();
 }
 
@@ -436,8 +456,8 @@ spec_status launch_attention_mma(const AttnArgs& a, cudaStream_t st)
 {
     const int group = a.Hq / a.Hkv, rows = a.R * group;
     const int rows_alloc = rows_alloc_for(rows);
-    const int max_chunks = max_chunks_for(a.max_kv_len);
     if (a.scratch_bytes < attention_mma_scratch_bytes(a.B, a.R, a.Hq, a.Hkv, a.dh, a.max_kv_len)) return SPEC_ERR_SHAPE;
+    const int max_chunks = max_chunks_for(a.max_kv_len);
     const PlanView pv = carve_plan(a.scratch, a.B, a.Hkv, rows_alloc, a.dh, max_chunks);
     MmaArgs m{(const __nv_bfloat16*)a.q, a.q_row_stride, (const __nv_bfloat16*)a.k_pool, (const __nv_bfloat16*)a.v_pool,
               a.block_table, a.max_blocks, a.pos, a.R, group, a.Hkv, (__nv_bfloat16*)a.out, a.out_row_stride,

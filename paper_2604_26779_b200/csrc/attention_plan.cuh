@@ -7,6 +7,7 @@ namespace spec {
 namespace attn {
 
 constexpr int kChunk = 4096;        // KV tokens per unit (upper bound); 4096 measured 3 % faster than 2048 and 1 % faster than 8192
+constexpr int kChunkMin = 1024;     // thin batches cut finer, down to this (decided by the planning kernel)
 constexpr int kChunkSlack = 128;    // ... plus this much, rather than opening one more chunk
 constexpr int kTileTok = 64;        // chunk lengths are multiples of this
 constexpr int kBT = 16;             // tokens per KV block
@@ -27,6 +28,14 @@ struct PlanView {                    // carved out of the scratch buffer
 inline int rows_alloc_for(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 64 ? 64 : 128; }
 inline int max_chunks_for(int max_kv_len) { return (max_kv_len + kTileTok + kChunk - 1) / kChunk + 1; }
 
+// Bytes of scratch a plan with max_chunks chunks per sequence needs (the layout of carve_plan).
+inline size_t plan_scratch_bytes(int B, int Hkv, int rows_alloc, int dh, int max_chunks)
+{
+    const size_t entries = (size_t)B * max_chunks;
+    return align_up((size_t)kCounters * 4 + 4, 256) + 2 * align_up((size_t)B * 4, 256) + align_up(entries * sizeof(Unit), 256) +
+           align_up(entries * Hkv * rows_alloc * dh * 4, 256) + align_up(entries * Hkv * rows_alloc * 8, 256);
+}
+
 inline PlanView carve_plan(void* scratch, int B, int Hkv, int rows_alloc, int dh, int max_chunks)
 {
     const size_t entries = (size_t)B * max_chunks;
@@ -43,8 +52,9 @@ inline PlanView carve_plan(void* scratch, int B, int Hkv, int rows_alloc, int dh
     return pv;
 }
 
-// One CTA: splits every sequence into equal chunks and writes the unit list; resets the work counters.
-spec_status launch_attn_plan(int B, int R, const int32_t* pos, int max_chunks, const PlanView& pv, cudaStream_t st);
+// One CTA: picks the chunk length (kChunk, or finer when the batch is thin: n_ctas = CTAs of the attention launch), splits every
+// sequence into equal chunks and writes the unit list (at most B * max_chunks units); resets the work counters.
+spec_status launch_attn_plan(int B, int R, const int32_t* pos, int Hkv, int n_ctas, int max_chunks, const PlanView& pv, cudaStream_t st);
 // Log-sum-exp merge of the chunks of multi-chunk sequences (head_dim 128); zeros for sequences without visible positions.
 spec_status launch_attn_merge128(int B, int rows_alloc, int Hkv, int R, int group, void* out, int out_row_stride,
                                  const PlanView& pv, cudaStream_t st);

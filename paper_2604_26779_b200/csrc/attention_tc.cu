@@ -513,8 +513,8 @@ spec_status launch_attention_tc(const AttnArgs& a, cudaStream_t st)
 {
     const int group = a.Hq / a.Hkv, rows = a.R * group;
     const int rows_alloc = rows_alloc_for(rows);
-    const int max_chunks = max_chunks_for(a.max_kv_len);
     if (a.scratch_bytes < attention_mma_scratch_bytes(a.B, a.R, a.Hq, a.Hkv, a.dh, a.max_kv_len)) return SPEC_ERR_SHAPE;
+    const int max_chunks = max_chunks_for(a.max_kv_len);
     const PlanView pv = carve_plan(a.scratch, a.B, a.Hkv, rows_alloc, a.dh, max_chunks);
     static bool configured = false;
     if (!configured) {
@@ -532,7 +532,7 @@ spec_status launch_attention_tc(const AttnArgs& a, cudaStream_t st)
              (__nv_bfloat16*)a.out, a.out_row_stride, 1.4426950408889634f / sqrtf((float)a.dh), pv, a.launch_index % kCounters,
              a.status};
     if (a.launch_index % kCounters == 0) {
-        spec_status s = launch_attn_plan(a.B, a.R, a.pos, max_chunks, pv, st);
+        spec_status s = launch_attn_plan(a.B, a.R, a.pos, a.Hkv, tc_sm_count(), max_chunks, pv, st);
         if (s != SPEC_OK) return s;
     }
     if (rows <= 64) attn_tc_kernel<1><<<tc_sm_count(), kThreadsTc, kSmemTc, st>>>(mk, mv, t);

@@ -548,6 +548,64 @@ extern "C" spec_status spec_seq_replace(spec_ctx* c, int n, const int32_t* slots
     return SPEC_OK;
 }
 
+extern "C" spec_status spec_seq_compact(spec_ctx* c, int n_keep, const int32_t* keep_slots_host, void* stream)
+{
+    if (c == nullptr || n_keep < 0 || (n_keep > 0 && keep_slots_host == nullptr)) return SPEC_ERR_INVALID_ARG;
+    const spec_config& g = c->cfg;
+    if (c->verified) return fail(c, SPEC_ERR_STATE, "spec_seq_compact: a verified step is waiting for its commit");
+    if (n_keep > c->B) return fail(c, SPEC_ERR_SHAPE, "spec_seq_compact: more slots listed than sequences running");
+    for (int j = 0; j < n_keep; ++j)
+        if (keep_slots_host[j] < 0 || keep_slots_host[j] >= c->B || (j > 0 && keep_slots_host[j] <= keep_slots_host[j - 1]))
+            return fail(c, SPEC_ERR_INVALID_ARG, "spec_seq_compact: kept slots must be in range and strictly ascending");
+    if (n_keep == c->B) return SPEC_OK;                     // ascending and complete: the identity
+    const int B_old = c->B, bt = g.kv_block_tokens, mb = g.max_blocks_per_seq;
+    const size_t Bm = g.max_batch;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* sb = static_cast<char*>(c->buf.state);
+    char* ws = static_cast<char*>(c->buf.workspace);
+    int32_t* args = at<int32_t>(sb, c->replace_args);
+    // 1. every slot that is not kept is retired (its blocks go back in slot order, logical block order)
+    std::vector<int32_t> dropped, minus(B_old, -1), zeros(B_old, 0);
+    for (int b = 0, j = 0; b < B_old; ++b) {
+        if (j < n_keep && keep_slots_host[j] == b) { ++j; continue; }
+        dropped.push_back(b);
+    }
+    const int nd = (int)dropped.size();
+    SPEC_CUDA_OK(cudaMemcpyAsync(args, dropped.data(), (size_t)nd * 4, cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_OK(cudaMemcpyAsync(args + Bm, minus.data(), (size_t)nd * 4, cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_OK(cudaMemcpyAsync(args + 2 * Bm, zeros.data(), (size_t)nd * 4, cudaMemcpyHostToDevice, st));
+    TRY(launch_kv_replace(nd, args, args + Bm, args + 2 * Bm, bt, mb, at<int32_t>(sb, c->seq_len), at<int32_t>(sb, c->last_token),
+                          at<int32_t>(sb, c->block_table), at<int32_t>(sb, c->owned), at<int32_t>(sb, c->free_stack),
+                          at<int32_t>(sb, c->free_top), at<int32_t>(sb, c->n_emitted), at<int32_t>(sb, c->pending_base),
+                          at<int32_t>(sb, c->status), st));
+    // 2. per-slot state moves to the front
+    SPEC_CUDA_OK(cudaMemcpyAsync(args, keep_slots_host, (size_t)n_keep * 4, cudaMemcpyHostToDevice, st));
+    const int R = c->k_last >= 0 ? c->k_last + 1 : 1;
+    const bool ngram = g.draft_kind == SPEC_DRAFT_NGRAM;
+    TRY(launch_seq_compact(n_keep, B_old, args, mb, R, ngram ? mb * bt : 0, at<int32_t>(sb, c->seq_len), at<int32_t>(sb, c->last_token),
+                           at<int32_t>(sb, c->owned), at<int32_t>(sb, c->pending_base), at<int32_t>(sb, c->n_emitted),
+                           at<int32_t>(sb, c->block_table), at<int32_t>(sb, c->out_tokens), at<float>(sb, c->out_logp),
+                           ngram ? at<int32_t>(sb, c->history) : nullptr, st));
+    // 3. what the draft head absorbs from the last verify (EAGLE-3: the tapped hidden states; MTP: the last-layer residual),
+    //    row blocks of R per slot; permuted through the logits buffer, which the next verify overwrites anyway
+    if (c->have_pending && c->k_last >= 0 && n_keep > 0) {
+        const size_t es = g.dtype == SPEC_DTYPE_F32 ? 4 : 2;
+        void* tmp = ws + c->logits.off;
+        if (g.draft_kind == SPEC_DRAFT_EAGLE3) {
+            const size_t row = (size_t)g.n_taps * g.d_model * es;
+            TRY(launch_permute_rows(n_keep, R, row, args, ws + c->taps.off, tmp, st));
+            SPEC_CUDA_OK(cudaMemcpyAsync(ws + c->taps.off, tmp, (size_t)n_keep * R * row, cudaMemcpyDeviceToDevice, st));
+        } else if (g.draft_kind == SPEC_DRAFT_MTP) {
+            const size_t row = (size_t)g.d_model * 4;
+            TRY(launch_permute_rows(n_keep, R, row, args, ws + c->x.off, tmp, st));
+            SPEC_CUDA_OK(cudaMemcpyAsync(ws + c->x.off, tmp, (size_t)n_keep * R * row, cudaMemcpyDeviceToDevice, st));
+        }
+    }
+    SPEC_CUDA_OK(cudaStreamSynchronize(st));          // the host lists go out of scope here
+    c->B = n_keep;
+    return SPEC_OK;
+}
+
 extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_tokens, void* stream)
 {
     if (c == nullptr) return SPEC_ERR_INVALID_ARG;

@@ -401,6 +401,53 @@ __global__ void kv_replace_kernel(int n, const int32_t* __restrict__ slots, cons
     *free_top = top;
 }
 
+// Renumbering of the running sequences (new slot j <- old slot keep[j], keep strictly ascending, so j <= keep[j] and a row
+// is never overwritten before it has been read when the slots are walked in order).  One CTA: the scalars by one thread in
+// slot order, the table / token rows slot by slot with the threads across a row.
+struct CompactArgs {
+    int n_keep, B_old, max_blocks, out_stride, hist_len;
+    const int32_t* keep;
+    int32_t *seq_len, *last_token, *owned, *pending_base, *n_emitted, *table, *out_tokens, *history;
+    float* out_logp;
+};
+__global__ void __launch_bounds__(256) seq_compact_kernel(const CompactArgs a)
+{
+    if (threadIdx.x == 0) {
+        for (int j = 0; j < a.n_keep; ++j) {
+            const int s = a.keep[j];
+            a.seq_len[j] = a.seq_len[s]; a.last_token[j] = a.last_token[s]; a.owned[j] = a.owned[s];
+            a.pending_base[j] = a.pending_base[s]; a.n_emitted[j] = a.n_emitted[s];
+        }
+        for (int j = a.n_keep; j < a.B_old; ++j) {          // the vacated tail: retired, owning nothing
+            a.seq_len[j] = -1; a.last_token[j] = 0; a.owned[j] = 0; a.pending_base[j] = 0; a.n_emitted[j] = 0;
+        }
+    }
+    for (int j = 0; j < a.n_keep; ++j) {
+        const int s = a.keep[j];
+        if (s == j) continue;
+        for (int c = threadIdx.x; c < a.max_blocks; c += blockDim.x) a.table[(size_t)j * a.max_blocks + c] = a.table[(size_t)s * a.max_blocks + c];
+        for (int c = threadIdx.x; c < a.out_stride; c += blockDim.x) {
+            a.out_tokens[(size_t)j * a.out_stride + c] = a.out_tokens[(size_t)s * a.out_stride + c];
+            a.out_logp[(size_t)j * a.out_stride + c] = a.out_logp[(size_t)s * a.out_stride + c];
+        }
+        if (a.history != nullptr)
+            for (int c = threadIdx.x; c < a.hist_len; c += blockDim.x) a.history[(size_t)j * a.hist_len + c] = a.history[(size_t)s * a.hist_len + c];
+        __syncthreads();                                    // a later slot may read what this one's source row held: keep the order
+    }
+    __syncthreads();
+    for (int j = a.n_keep + (int)(threadIdx.x / 32); j < a.B_old; j += blockDim.x / 32)
+        for (int c = threadIdx.x % 32; c < a.max_blocks; c += 32) a.table[(size_t)j * a.max_blocks + c] = -1;
+}
+// dst row j*R + i <- src row keep[j]*R + i (16-byte pieces); dst and src do not overlap.
+__global__ void __launch_bounds__(256) permute_rows_kernel(int R, size_t row_bytes, const int32_t* __restrict__ keep,
+                                                           const unsigned char* __restrict__ src, unsigned char* __restrict__ dst)
+{
+    const int j = blockIdx.x / R, i = blockIdx.x % R;
+    const uint4* s4 = reinterpret_cast<const uint4*>(src + ((size_t)keep[j] * R + i) * row_bytes);
+    uint4* d4 = reinterpret_cast<uint4*>(dst + (size_t)blockIdx.x * row_bytes);
+    for (size_t c = threadIdx.x; c < row_bytes / 16; c += blockDim.x) d4[c] = s4[c];
+}
+
 }  // namespace
 
 #define DISPATCH_T(dtype, ...)                                            \
@@ -499,6 +546,24 @@ spec_status launch_kv_replace(int n, const int32_t* slots, const int32_t* new_le
     if (n == 0) return SPEC_OK;
     kv_replace_kernel<<<1, 32, 0, st>>>(n, slots, new_len, new_last, bt, max_blocks, seq_len, last_token, table, owned,
                                         free_stack, free_top, n_emitted, pending_base, status);
+    return launch_status();
+}
+
+spec_status launch_seq_compact(int n_keep, int B_old, const int32_t* keep, int max_blocks, int out_stride, int hist_len, int32_t* seq_len,
+                               int32_t* last_token, int32_t* owned, int32_t* pending_base, int32_t* n_emitted, int32_t* table,
+                               int32_t* out_tokens, float* out_logp, int32_t* history, cudaStream_t st)
+{
+    CompactArgs a{n_keep, B_old, max_blocks, out_stride, hist_len, keep, seq_len, last_token, owned, pending_base, n_emitted, table,
+                  out_tokens, history, out_logp};
+    seq_compact_kernel<<<1, 256, 0, st>>>(a);
+    return launch_status();
+}
+
+spec_status launch_permute_rows(int n_keep, int R, size_t row_bytes, const int32_t* keep, const void* src, void* dst, cudaStream_t st)
+{
+    if (n_keep * R == 0 || row_bytes == 0) return SPEC_OK;
+    if (row_bytes % 16 != 0) return SPEC_ERR_SHAPE;
+    permute_rows_kernel<<<n_keep * R, 256, 0, st>>>(R, row_bytes, keep, (const unsigned char*)src, (unsigned char*)dst);
     return launch_status();
 }
 

@@ -73,6 +73,11 @@ spec_status launch_kv_replace(int n, const int32_t* slots, const int32_t* new_le
                               int32_t* free_stack, int32_t* free_top, int32_t* n_emitted,
                               int32_t* pending_base, int32_t* status, cudaStream_t st);
 
+spec_status launch_seq_compact(int n_keep, int B_old, const int32_t* keep, int max_blocks, int out_stride, int hist_len, int32_t* seq_len,
+                               int32_t* last_token, int32_t* owned, int32_t* pending_base, int32_t* n_emitted, int32_t* table,
+                               int32_t* out_tokens, float* out_logp, int32_t* history, cudaStream_t st);
+spec_status launch_permute_rows(int n_keep, int R, size_t row_bytes, const int32_t* keep, const void* src, void* dst, cudaStream_t st);
+
 // model-free drafting: continue the most recent earlier occurrence of the trailing n-gram of (history[0..len), last token)
 spec_status launch_ngram_draft(int B, int k, int n_max, const int32_t* history, int max_hist, const int32_t* seq_len,
                                const int32_t* last_token, int32_t* draft_tokens, int draft_stride, cudaStream_t st);

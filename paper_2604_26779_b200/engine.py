@@ -184,6 +184,12 @@ class SpecStep:
         B._check(self.lib.spec_seq_replace(self.ctx, sl.shape[0], sl.ctypes.data, ln.ctypes.data, lt.ctypes.data,
                                            B._stream(stream)), "spec_seq_replace")
 
+    def seq_compact(self, keep_slots, stream=None):
+        """Shrinks the batch to the listed (ascending) slots; everything else is retired.  Updates self.B."""
+        ks = np.ascontiguousarray(keep_slots, np.int32)
+        B._check(self.lib.spec_seq_compact(self.ctx, ks.shape[0], ks.ctypes.data if ks.shape[0] else None, B._stream(stream)), "spec_seq_compact")
+        self.B = int(ks.shape[0])
+
     def draft(self, k, stream=None):
         B._check(self.lib.spec_draft(self.ctx, k, B._stream(stream)), "spec_draft")
 

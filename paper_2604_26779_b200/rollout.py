@@ -3,7 +3,9 @@
 Responses of one rollout batch end at very different lengths (the long tail the paper's Section 5.1 describes), so a
 fixed batch would run mostly empty towards the end.  Here every slot whose sequence is done takes the next prompt
 (`spec_seq_replace`); the new prompt prefills through forced verify steps, k+1 prompt tokens per step, while the other
-slots keep speculating; when no prompt is left the slot is retired.  The draft length k may change from step to step
+slots keep speculating; when no prompt is left the slot is retired, and once the queue is empty and few enough slots are
+still running the batch is compacted (`spec_seq_compact`) so that the long tail does not drag the retired slots' rows through
+every projection.  The draft length k may change from step to step
 (`k_policy`), which is how a caller acts on the paper's observation that the useful k is narrow and depends on how
 full the batch is (Section 4.2, Section 5.2).
 
@@ -50,6 +52,7 @@ class SequenceRecord:
     first_decode_step: int          # value of the step counter at this sequence's first sampled step
     tokens: list                    # response tokens (truncated to the requested length)
     ks: list                        # k of each of its decode steps
+    slots: list = dataclasses.field(default_factory=list)   # slot it occupied at each decode step (compaction moves it)
 
 
 @dataclasses.dataclass
@@ -73,7 +76,9 @@ class Rollout:
     """Generates `response_lens[i]` tokens after `prompts[i]` for every i, with at most `eng.sc.max_batch` sequences in
     flight.  `k_policy(step, n_active, alpha_estimate) -> k` picks the draft length of each step (default: k_max)."""
 
-    def __init__(self, eng, prompts, response_lens, free_stack, k_policy=None):
+    def __init__(self, eng, prompts, response_lens, free_stack, k_policy=None, compact_fraction=0.0):
+        """compact_fraction: once the prompt queue is empty, the batch is compacted whenever the running sequences are
+        at most this fraction of the slots (0 = never; 0.5 halves the batch at most log2(slots) times)."""
         assert len(prompts) == len(response_lens) and len(prompts) > 0
         self.eng, self.sc = eng, eng.sc
         self.queue = [(i, np.ascontiguousarray(p, np.int32), int(w)) for i, (p, w) in enumerate(zip(prompts, response_lens))]
@@ -94,6 +99,8 @@ class Rollout:
         self.step = 0
         self.k_trace, self.active_trace = [], []
         self._acc = [0, 0]          # accepted drafts, tried draft positions
+        self.compact_fraction = float(compact_fraction)
+        self.compactions = []       # (step, slots before, slots after)
 
     @staticmethod
     def _assign(slot, item):
@@ -148,6 +155,7 @@ class Rollout:
             if s.rec.first_decode_step < 0:
                 s.rec.first_decode_step = self.step
             s.rec.ks.append(k)
+            s.rec.slots.append(b)
             s.rec.tokens += [int(t) for t in out[b, : n_em[b]]]
             self._acc[0] += int(n_em[b]) - 1
             self._acc[1] += min(int(n_em[b]), k)
@@ -170,6 +178,14 @@ class Rollout:
                     lens.append(-1)
                     lasts.append(0)
             eng.seq_replace(replace, lens, lasts)
+        if not self.queue and self.compact_fraction > 0.0:
+            live = [b for b, s in enumerate(self.slots) if s.active]
+            if 0 < len(live) <= self.compact_fraction * len(self.slots):
+                eng.seq_compact(live)
+                self.compactions.append((self.step, len(self.slots), len(live)))
+                self.slots = [self.slots[b] for b in live]
+                for j, s in enumerate(self.slots):
+                    s.rec.slot = j
         self.k_trace.append(k)
         self.active_trace.append(n_active)
         self.step += 1

@@ -12,8 +12,8 @@ torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("kind", ["eagle3", "ngram"])
-def test_rollout_with_refill_matches_oracle_chains(kind):
+@pytest.mark.parametrize("kind,compact", [("eagle3", 0.0), ("ngram", 0.0), ("eagle3", 0.7), ("ngram", 0.7)])
+def test_rollout_with_refill_matches_oracle_chains(kind, compact):
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from paper_2604_26779_b200 import engine, rollout
@@ -32,7 +32,8 @@ def test_rollout_with_refill_matches_oracle_chains(kind):
     if H is not None:
         eng.load_draft_weights(H)
     order = inputs.make_block_order(sc.kv_num_blocks, inputs.sub_seed(3, 3))
-    ro = rollout.Rollout(eng, prompts, wants, order, k_policy=lambda step, n_active, alpha: 1 + step % k_max)
+    ro = rollout.Rollout(eng, prompts, wants, order, k_policy=lambda step, n_active, alpha: 1 + step % k_max,
+                         compact_fraction=compact)
     done = ro.run(max_steps=400)
     assert sorted(done) == list(range(7))
     assert max(ro.active_trace) == slots and min(ro.active_trace) >= 1
@@ -40,10 +41,12 @@ def test_rollout_with_refill_matches_oracle_chains(kind):
     for i in range(7):
         rec = done[i]
         assert len(rec.tokens) == wants[i]
-        ch = ChainOracle(cfg, W, H, kind, seed, rec.slot, prompts[i], step0=rec.first_decode_step)
-        # the sequence's decode steps are consecutive device steps, so the chain's step counter follows by itself
+        ch = ChainOracle(cfg, W, H, kind, seed, rec.slots[0], prompts[i], step0=rec.first_decode_step)
+        # the sequence's decode steps are consecutive device steps, so the chain's step counter follows by itself; the slot
+        # (and with it the Philox stream) changes when the batch is compacted
         got, ref = rec.tokens, []
-        for k in rec.ks:
+        for k, slot in zip(rec.ks, rec.slots):
+            ch.seq = slot
             r = ch.step_once(k)
             new = [int(t) for t in r["out_tokens"][: r["n_emitted"]]]
             n_have = len(ref)
@@ -55,8 +58,10 @@ def test_rollout_with_refill_matches_oracle_chains(kind):
             ref += new
     print(f"rollout {kind}: {ro.step} steps, k trace {ro.k_trace[:8]}..., boundary {boundary}")
     assert boundary <= 1
+    if compact:
+        assert len(ro.compactions) >= 1 and ro.compactions[-1][2] < slots
     # everything is retired and every block is back
-    assert eng.seq_len().cpu().tolist() == [-1] * slots
+    assert eng.seq_len().cpu().tolist() == [-1] * eng.B
     assert int(eng.tensor("FREE_TOP", 0, torch.int32, (1,)).item()) == sc.kv_num_blocks
     free = eng.tensor("FREE_STACK", 0, torch.int32, (sc.kv_num_blocks,)).cpu().numpy()
     assert sorted(free.tolist()) == list(range(sc.kv_num_blocks))

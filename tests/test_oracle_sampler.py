@@ -477,3 +477,25 @@ def test_e4m3_codes_match_the_library_cast():
     x = rng.normal(0, 3, 1000).astype(np.float32)
     assert np.array_equal(oracle.e4m3_roundtrip(x, 0.25), oracle.e4m3_dequantize(oracle.e4m3_quantize(x / np.float32(0.25))) * np.float32(0.25))
     assert np.max(np.abs(oracle.e4m3_roundtrip(x) - x) / np.maximum(np.abs(x), 2.0 ** -6)) <= 2.0 ** -4 + 1e-7
+
+
+def test_kv_compact_hand_worked():
+    # 4 slots, 16-token blocks, 10 blocks.  Slot 0 holds 20 tokens (blocks 9, 8), slot 1 holds 5 (block 7), slot 2 is retired,
+    # slot 3 holds 33 (blocks 6, 5, 4); free stack below the top: [0, 1, 2, 3].
+    bt = 16
+    seq_len = np.array([20, 5, -1, 33], np.int32)
+    table = np.full((4, 4), -1, np.int32)
+    table[0, :2] = [9, 8]; table[1, :1] = [7]; table[3, :3] = [6, 5, 4]
+    free = np.array([0, 1, 2, 3, -1, -1, -1, -1, -1, -1], np.int32)
+    top = np.array([4], np.int32)
+    new_len, new_table = oracle.kv_compact([1, 3], bt, seq_len, table, free, top)
+    # worked by hand: slot 0 is dropped (its blocks 9 then 8 are pushed), slot 2 owns nothing; slots 1 and 3 move to 0 and 1
+    assert top[0] == 6 and free[:6].tolist() == [0, 1, 2, 3, 9, 8]
+    assert new_len.tolist() == [5, 33]
+    assert new_table.tolist() == [[7, -1, -1, -1], [6, 5, 4, -1]]
+    # blocks are conserved: free ones plus owned ones are all ten, none twice
+    owned = [b for row in new_table for b in row if b >= 0]
+    assert sorted(free[: top[0]].tolist() + owned) == list(range(10))
+    # keeping everything is the identity
+    l2, t2 = oracle.kv_compact([0, 1], bt, new_len.copy(), new_table.copy(), free, top)
+    assert l2.tolist() == [5, 33] and t2.tolist() == new_table.tolist() and top[0] == 6
