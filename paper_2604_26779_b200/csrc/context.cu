@@ -286,7 +286,11 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
     void* ws = c.buf.workspace;
     int32_t* status_word = at<int32_t>(c.buf.state, c.status);
     const bool tc = gemm_tc_supported(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt);
-    if (tc && (dh == 64 || dh == 128)) {
+    // very few rows (the thin tail of a rollout): plain weight-streaming projections + the small element-wise kernels beat
+    // the fused tensor-core epilogues, which have too few tiles to pull the weights at the HBM rate
+    const bool thin = g.kv_dtype != SPEC_KV_E4M3 && gemm_skinny_supported(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, dt) &&
+                      gemm_skinny_supported(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, dt);
+    if (tc && !thin && (dh == 64 || dh == 128)) {
         // projection, rotary embedding and the append into the paged cache in one kernel
         QkvEpilogue e{Hq, Hkv, dh, R, g.max_blocks_per_seq, g.kv_block_tokens, pos, at<int32_t>(c.buf.state, c.block_table),
                       at<float>(ws, c.rope), k_pool, v_pool};
@@ -321,7 +325,7 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
         TRY(launch_moe_combine(M, tk, d, at<float>(ws, c.moe_wts), at<int32_t>(ws, c.moe_inv), at<float>(ws, c.moe_out), res, st));
         return SPEC_OK;
     }
-    if (gemm_tc_supported(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.act), d_ffn, dt, dt)) {
+    if (!thin && gemm_tc_supported(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.act), d_ffn, dt, dt)) {
         TIMED(c, CLS_GEMM, launch_gemm_swiglu_tc(M, d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.act), status_word, st));
     } else {
         TIMED(c, CLS_GEMM, launch_gemm(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.gu), 2 * d_ffn, dt, dt, 0, st));

@@ -731,6 +731,7 @@ spec_status launch_gemm_grouped(int rows_total, int max_rows_per_group, int E, i
 spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int dtype_in,
                         int out_dtype, int accumulate, cudaStream_t st)
 {
+    if (gemm_skinny_supported(M, N, K, A, lda, W, dtype_in)) return launch_gemm_skinny(M, N, K, A, lda, W, C, ldc, out_dtype, accumulate, st);
     if (gemm_tc_supported(M, N, K, A, lda, W, C, ldc, dtype_in, out_dtype))
         return launch_gemm_tc(M, N, K, A, lda, W, C, ldc, out_dtype, accumulate, nullptr, st);
     return launch_gemm_simt(M, N, K, A, lda, W, C, ldc, dtype_in, out_dtype, accumulate, st);

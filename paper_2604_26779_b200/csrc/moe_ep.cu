@@ -246,7 +246,11 @@ extern "C" spec_status spec_ep_route(const spec_ep_config* cfg, void* window, vo
     unsigned char* sc = static_cast<unsigned char*>(scratch);
     const int E = cfg->n_experts, tk = cfg->top_k, d = cfg->d;
     if (M > 0 && cudaMemcpyAsync(w + l.h, h, (size_t)M * d * 2, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return SPEC_ERR_CUDA;
-    spec_status r = launch_gemm(M, E, d, w + l.h, d, router_w, sc + l.logits, E, SPEC_DTYPE_BF16, SPEC_DTYPE_F32, 0, st);
+    // always the tensor-core tile kernel, whatever M is: a row's router logits (and with them its mixture weights) must not
+    // depend on how many other rows this rank happens to hold, or the block's output would change with ep_size
+    spec_status r = gemm_tc_supported(M, E, d, w + l.h, d, router_w, sc + l.logits, E, SPEC_DTYPE_BF16, SPEC_DTYPE_F32)
+                        ? launch_gemm_tc(M, E, d, w + l.h, d, router_w, sc + l.logits, E, SPEC_DTYPE_F32, 0, nullptr, st)
+                        : launch_gemm(M, E, d, w + l.h, d, router_w, sc + l.logits, E, SPEC_DTYPE_BF16, SPEC_DTYPE_F32, 0, st);
     if (r != SPEC_OK) return r;
     r = launch_moe_route(M, E, tk, reinterpret_cast<const float*>(sc + l.logits), reinterpret_cast<int32_t*>(w + l.ids),
                          reinterpret_cast<float*>(w + l.wts), st);

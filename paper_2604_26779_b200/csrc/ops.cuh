@@ -89,9 +89,15 @@ spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void*
                         int out_dtype, int accumulate, cudaStream_t st);
 
 // swiglu != 0: W holds [2F] rows per group in 256-row gate/up groups and C is the activation [rows][N/2] (bf16)
+// very few rows (M <= 16): the weights are the MMA's M operand, one CTA per 32 weight rows (gemm_skinny.cu)
+bool gemm_skinny_supported(int M, int N, int K, const void* A, int lda, const void* W, int dtype_in);
+spec_status launch_gemm_skinny(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int out_dtype,
+                               int accumulate, cudaStream_t st);
 spec_status launch_gemm_grouped(int rows_total, int max_rows_per_group, int E, int N, int K, const void* A, const void* W,
                                 void* C, int out_dtype, int swiglu, const int32_t* counts, const int32_t* offsets,
                                 int32_t* status, cudaStream_t st);
+spec_status launch_gemm_tc(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int out_dtype,
+                           int accumulate, int32_t* status, cudaStream_t st);
 bool gemm_tc_supported(int M, int N, int K, const void* A, int lda, const void* W, const void* C, int ldc, int dtype_in,
                        int out_dtype);
 spec_status launch_gemm_swiglu_tc(int M, int F, int K, const void* A, int lda, const void* W, void* act, int32_t* status,

@@ -98,6 +98,16 @@ def test_paged_attention_matches_oracle(api, lens, R, Hq, Hkv, dh, dtype):
     (1000, 520, 192, torch.bfloat16, torch.bfloat16, False),       # ragged M and N tails
     (77, 1000, 4096, torch.bfloat16, torch.float32, False),
     (1024, 16384, 1024, torch.bfloat16, torch.float32, False),     # LM-head-like slice: fp32 logits
+    # very few rows (thin-batch kernel: weights as the MMA's M operand): every token-tile width, ragged M and N, both outputs
+    (1, 4096, 4096, torch.bfloat16, torch.float32, False),
+    (7, 96, 256, torch.bfloat16, torch.bfloat16, False),
+    (8, 6144, 4096, torch.bfloat16, torch.bfloat16, False),
+    (9, 1000, 512, torch.bfloat16, torch.float32, True),
+    (16, 4096, 14336, torch.bfloat16, torch.float32, True),
+    (17, 28672, 4096, torch.bfloat16, torch.bfloat16, False),
+    (31, 50, 768, torch.bfloat16, torch.bfloat16, True),
+    (32, 16384, 4096, torch.bfloat16, torch.float32, False),
+    (32, 4096, 320, torch.bfloat16, torch.float32, False),         # K not a multiple of 256: stays on the tensor-core tile kernel
 ])
 def test_gemm_matches_fp64(api, M, N, K, din, dout, acc):
     kind = "bf16" if din == torch.bfloat16 else "f32"
@@ -110,7 +120,7 @@ def test_gemm_matches_fp64(api, M, N, K, din, dout, acc):
     api.spec_gemm(dA, dW, dC, accumulate=acc)
     torch.cuda.synchronize()
     # fp64 reference on sampled rows (all rows when small)
-    rows = np.arange(M) if M * N * K < 2e9 else np.unique(np.concatenate([np.arange(0, M, 37), [M - 1, M - 2, 127, 128]]))
+    rows = np.arange(M) if M * N * K < 2e9 or M <= 128 else np.unique(np.concatenate([np.arange(0, M, 37), [M - 1, M - 2, 127, 128]]))
     ref = A[rows].astype(np.float64) @ W.astype(np.float64).T + (C0[rows].astype(np.float64) if acc else 0.0)
     got = dC.float().cpu().numpy()[rows]
     err = np.abs(got - ref).max(-1) / np.abs(ref).max(-1)
