@@ -178,8 +178,8 @@ spec_status run_skinny(int M, int N, int K, const void* A, int lda, const void* 
 
 bool gemm_skinny_supported(int M, int N, int K, const void* A, int lda, const void* W, int dtype_in)
 {
-    // (the 32-row instantiation works but measured slower than the tensor-core tile kernel: its activation slice per stage is
-    // as large as the weight slice)
+    // (17..32 rows measured slower than the tensor-core tile kernel in two forms - 32 weight rows per CTA, and 64 rows with two
+    // CTAs of a cluster splitting K: at four token tiles per weight tile the legacy MMA path no longer hides behind the stream)
     return dtype_in == SPEC_DTYPE_BF16 && M >= 1 && M <= 16 && K >= kStageK && K % kStageK == 0 && lda % 8 == 0 && N >= 1 &&
            (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && (reinterpret_cast<uintptr_t>(W) & 15u) == 0;
 }
