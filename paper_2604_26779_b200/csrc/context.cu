@@ -288,8 +288,11 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
     const bool tc = gemm_tc_supported(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt);
     // very few rows (the thin tail of a rollout): plain weight-streaming projections + the small element-wise kernels beat
     // the fused tensor-core epilogues, which have too few tiles to pull the weights at the HBM rate
-    const bool thin = g.kv_dtype != SPEC_KV_E4M3 && gemm_skinny_supported(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, dt) &&
-                      gemm_skinny_supported(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, dt);
+    const bool thin = g.kv_dtype != SPEC_KV_E4M3 &&
+                      (gemm_skinny_supported(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, dt) ||
+                       gemm_tc_thin_supported(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt)) &&
+                      (gemm_skinny_supported(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, dt) ||
+                       gemm_tc_thin_supported(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.gu), 2 * d_ffn, dt, dt));
     if (tc && !thin && (dh == 64 || dh == 128)) {
         // projection, rotary embedding and the append into the paged cache in one kernel
         QkvEpilogue e{Hq, Hkv, dh, R, g.max_blocks_per_seq, g.kv_block_tokens, pos, at<int32_t>(c.buf.state, c.block_table),
@@ -300,7 +303,8 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
         if (g.kv_dtype == SPEC_KV_E4M3) return SPEC_ERR_UNSUPPORTED;    // the 8-bit cache is written by the fused epilogue only
         TIMED(c, CLS_GEMM, launch_gemm(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt, 0, st));
         TRY(launch_rope_append(B, R, Hq, Hkv, dh, g.rope_theta, at(ws, c.qkv), pos, k_pool, v_pool,
-                               at<int32_t>(c.buf.state, c.block_table), g.max_blocks_per_seq, g.kv_block_tokens, dt, st));
+                               at<int32_t>(c.buf.state, c.block_table), g.max_blocks_per_seq, g.kv_block_tokens, dt, st,
+                               at<float>(ws, c.rope)));
     }
     AttnArgs a{B, R, Hq, Hkv, dh, g.kv_block_tokens, g.max_blocks_per_seq, at(ws, c.qkv), qkv_n, k_pool, v_pool,
                at<int32_t>(c.buf.state, c.block_table), pos, at(ws, c.attn_out), Hq * dh, dt, at(ws, c.attn_scratch),

@@ -52,7 +52,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr)
 // Instruction descriptor: D fp32, A and B bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
-struct TileCoord { int a_row, b_row, c_row, rows_valid, col, kb0, kb1; };
+struct TileCoord { int a_row, b_row, c_row, rows_valid, col, kb0, kb1, split; };
 
 struct GemmArgs {
     int M, N, K;
@@ -71,9 +71,13 @@ struct GemmArgs {
     const int32_t* pos; const int32_t* block_table; const float2* rope;   // rope [dh/2][M] (cos, sin) of each row's position
     __nv_bfloat16* k_pool; __nv_bfloat16* v_pool;
     int kv_fp8; float k_scale, v_scale;           // 8-bit cache: k and v are stored as e4m3 codes of x / scale
+    // EPI_THIN (17..64 activation rows): the operands are swapped - the WEIGHT rows are the MMA's M operand (M = features here),
+    // the activation rows its N operand (N = tokens <= bn, bn = 32 or 64: one narrow n-tile) - and the epilogue writes the
+    // transposed tile, C[token][feature]
+    int bn;
 };
 
-enum { EPI_PLAIN = 0, EPI_SWIGLU = 1, EPI_QKV = 2 };
+enum { EPI_PLAIN = 0, EPI_SWIGLU = 1, EPI_QKV = 2, EPI_THIN = 3 };
 
 __device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float (&f)[32])
 {
@@ -362,6 +366,39 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord&
     }
 }
 
+// Thin epilogue (operands swapped): this thread's tensor-memory lane is a FEATURE (weight row), the columns are tokens.
+// For every token the warp's 32 lanes hold 32 consecutive features: each store (and residual load) instruction covers one
+// contiguous piece of a row of C.  With split K the piece goes to partial s of the scratch, [splits][tokens][features] fp32.
+__device__ __forceinline__ void epilogue_thin(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int feature, bool feature_ok, int half)
+{
+    const int tokens = g.N;
+#pragma unroll 1
+    for (int c0 = half * 32; c0 < g.bn; c0 += 64) {
+        if (c0 >= tokens) break;                            // warp-uniform
+        uint32_t v[32];
+        tc_ld32(t_row + c0, v);
+        tc_wait_ld();
+        if (!feature_ok) continue;
+        if (g.out_f32) {
+            float* cp = static_cast<float*>(g.C) + (size_t)tc.split * tokens * g.ldc + (size_t)c0 * g.ldc + feature;
+#pragma unroll
+            for (int t = 0; t < 32; ++t)
+                if (c0 + t < tokens) {
+                    const float x = __uint_as_float(v[t]);
+                    cp[(size_t)t * g.ldc] = g.accumulate ? cp[(size_t)t * g.ldc] + x : x;
+                }
+        } else {
+            __nv_bfloat16* cp = static_cast<__nv_bfloat16*>(g.C) + (size_t)c0 * g.ldc + feature;
+#pragma unroll
+            for (int t = 0; t < 32; ++t)
+                if (c0 + t < tokens) {
+                    const float x = __uint_as_float(v[t]);
+                    cp[(size_t)t * g.ldc] = __float2bfloat16_rn(g.accumulate ? __bfloat162float(cp[(size_t)t * g.ldc]) + x : x);
+                }
+        }
+    }
+}
+
 // Decodes work item w into (m-tile, n-tile, group) and the tile's row window.  Returns false for an empty tile.
 // Grouped mode enumerates only the m-tiles that exist (pref = running count of ceil(counts / BM)): group by group, within
 // a group the n-tiles in turn, within an n-tile the group's m-tiles next to each other, so the CTAs that run at the same
@@ -370,7 +407,7 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord&
 __device__ __forceinline__ bool tile_coord(const GemmArgs& g, int w, int m_tiles, int n_tiles, const int* pref, TileCoord& t)
 {
     const int kb_count = (g.K + BK - 1) / BK;
-    t.kb0 = 0; t.kb1 = kb_count;
+    t.kb0 = 0; t.kb1 = kb_count; t.split = 0;
     int split = 0;
     if (g.E > 0) {
         int lo = 0, hi = g.E - 1;                            // last group whose first item is <= w
@@ -386,7 +423,7 @@ __device__ __forceinline__ bool tile_coord(const GemmArgs& g, int w, int m_tiles
         t.col = nt * BN;
         return true;
     }
-    if (g.splits > 1) { split = w % g.splits; w /= g.splits; t.kb0 = split * g.kb_per; t.kb1 = min(kb_count, t.kb0 + g.kb_per); }
+    if (g.splits > 1) { split = w % g.splits; w /= g.splits; t.kb0 = split * g.kb_per; t.kb1 = min(kb_count, t.kb0 + g.kb_per); t.split = split; }
     const int mt = w % m_tiles, nt = (w / m_tiles) % n_tiles;
     t.a_row = mt * BM; t.c_row = t.a_row + split * g.M; t.rows_valid = g.M - mt * BM;
     t.b_row = nt * BN;
@@ -443,7 +480,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
                 for (int kb = tc.kb0; kb < tc.kb1; ++kb) {
                     if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t bar = smem_u32(&ctl->full[s]);
-                    mbar_expect_tx(bar, STAGE_BYTES);
+                    mbar_expect_tx(bar, EPI == EPI_THIN ? (uint32_t)(A_BYTES + g.bn * BK * 2) : (uint32_t)STAGE_BYTES);
                     tma_load_2d(tiles + s * STAGE_BYTES, &map_a, kb * BK, tc.a_row, bar);
                     tma_load_2d(tiles + s * STAGE_BYTES + A_BYTES, &map_b, kb * BK, tc.b_row, bar);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -460,6 +497,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             uint32_t s = 0, ph = 0;
             bool ok = true;
             int it = 0;
+            // instruction descriptor; the thin variant's n extent is the activation tile (32 or 64 rows)
+            const uint32_t idesc = EPI == EPI_THIN ? ((kIdesc & ~(0x3fu << 17)) | ((uint32_t)(g.bn >> 3) << 17)) : kIdesc;
             for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
                 TileCoord tc;
                 if (!tile_coord(g, w, m_tiles, n_tiles, pref, tc)) continue;
@@ -474,7 +513,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
                     const uint32_t sa = tiles + s * STAGE_BYTES, sb = sa + A_BYTES;
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k)
-                        tc_mma(d_tmem, smem_desc(sa + k * UMMA_K * 2), smem_desc(sb + k * UMMA_K * 2), kIdesc, (kb > tc.kb0 || k > 0) ? 1u : 0u);
+                        tc_mma(d_tmem, smem_desc(sa + k * UMMA_K * 2), smem_desc(sb + k * UMMA_K * 2), idesc, (kb > tc.kb0 || k > 0) ? 1u : 0u);
                     tc_commit(smem_u32(&ctl->empty[s]));            // stage reusable once these MMAs have read it
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -513,7 +552,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             tc_fence_after();
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
             const uint32_t stage = out_stage + (warp - 2) * kOutStageBytes;
-            if constexpr (EPI == EPI_SWIGLU) epilogue_swiglu(g, tc, t_row, row, row_ok, half, stage, lane, rows_ok);
+            if constexpr (EPI == EPI_THIN) epilogue_thin(g, tc, t_row, tc.a_row + row_in_tile, row_ok, half);
+            else if constexpr (EPI == EPI_SWIGLU) epilogue_swiglu(g, tc, t_row, row, row_ok, half, stage, lane, rows_ok);
             else if constexpr (EPI == EPI_QKV) epilogue_qkv(g, tc, t_row, row, row_ok, half, stage, lane);
             else epilogue_plain(g, tc, t_row, row, row_ok, half, stage, lane, rows_ok, resid);
             tc_fence_before();
@@ -587,6 +627,7 @@ bool init_once()
     if (cudaFuncSetAttribute(gemm_tc_kernel<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return false;
     if (cudaFuncSetAttribute(gemm_tc_kernel<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return false;
     if (cudaFuncSetAttribute(gemm_tc_kernel<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return false;
+    if (cudaFuncSetAttribute(gemm_tc_kernel<EPI_THIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return false;
     g_encode = reinterpret_cast<EncodeFn>(fn);
     return true;
 }
@@ -596,6 +637,7 @@ spec_status run_kernel(int epi, const CUtensorMap& ma, const CUtensorMap& mb, co
     const int grid = n_work < g_sms ? (int)n_work : g_sms;
     if (epi == EPI_SWIGLU)   gemm_tc_kernel<EPI_SWIGLU><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, g);
     else if (epi == EPI_QKV) gemm_tc_kernel<EPI_QKV><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, g);
+    else if (epi == EPI_THIN) gemm_tc_kernel<EPI_THIN><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, g);
     else                     gemm_tc_kernel<EPI_PLAIN><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, g);
     return launch_status();
 }
@@ -675,6 +717,46 @@ spec_status launch_gemm_tc(int M, int N, int K, const void* A, int lda, const vo
     return run_kernel(EPI_PLAIN, ma, mb, g, n_work, st);
 }
 
+// 17..64 activation rows: operands swapped (see GemmArgs::bn).  One work item per 128 weight rows (x splits of K when that
+// leaves SMs idle and the caller gave scratch; the partials are summed in split order by the reduction kernel).
+bool gemm_tc_thin_supported(int M, int N, int K, const void* A, int lda, const void* W, const void* C, int ldc, int dtype_in, int out_dtype)
+{
+    return M > 16 && M <= 64 && K % BK == 0 && gemm_tc_supported(M, N, K, A, lda, W, C, ldc, dtype_in, out_dtype);
+}
+
+spec_status launch_gemm_tc_thin(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int out_dtype,
+                                int accumulate, int32_t* status, cudaStream_t st)
+{
+    if (!init_once()) return SPEC_ERR_CUDA;
+    const int bn = M <= 32 ? 32 : 64;
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, BM)) return SPEC_ERR_CUDA;            // weights: the M operand
+    if (!make_map(&mb, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, (uint32_t)bn)) return SPEC_ERR_CUDA;   // activations: the N operand
+    const int n_work = (N + BM - 1) / BM, kb_count = K / BK;
+    GemmArgs g{};
+    g.M = N; g.N = M; g.K = K; g.C = C; g.ldc = ldc; g.out_f32 = out_dtype == SPEC_DTYPE_F32 ? 1 : 0; g.accumulate = accumulate;
+    g.status = status; g.bn = bn;
+    const GemmScratch& sc = gemm_scratch();
+    int splits = 1;
+    if (sc.ptr != nullptr && n_work * 2 <= g_sms && N % 4 == 0) {
+        splits = g_sms / n_work;
+        if (splits > 8) splits = 8;
+        while (splits > 1 && (kb_count / splits < 8 || (size_t)splits * M * N * 4 > sc.bytes)) --splits;
+    }
+    if (splits > 1) {
+        g.C = sc.ptr; g.ldc = N; g.out_f32 = 1; g.accumulate = 0;
+        g.splits = splits; g.kb_per = (kb_count + splits - 1) / splits;
+        TRY_LAUNCH(run_kernel(EPI_THIN, ma, mb, g, (long long)n_work * splits, st));
+        const size_t n4 = (size_t)M * N / 4;
+        if (out_dtype == SPEC_DTYPE_F32)
+            splitk_reduce_kernel<float><<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(M, N, splits, (const float*)sc.ptr, (float*)C, ldc, accumulate);
+        else
+            splitk_reduce_kernel<__nv_bfloat16><<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(M, N, splits, (const float*)sc.ptr, (__nv_bfloat16*)C, ldc, accumulate);
+        return launch_status();
+    }
+    return run_kernel(EPI_THIN, ma, mb, g, n_work, st);
+}
+
 // gate/up projection with the SwiGLU applied in the epilogue: W [2F][K] stored in 256-row groups (128 gate rows, then the
 // matching 128 up rows), act [M][F] bf16.
 spec_status launch_gemm_swiglu_tc(int M, int F, int K, const void* A, int lda, const void* W, void* act, int32_t* status,
@@ -732,6 +814,8 @@ spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void*
                         int out_dtype, int accumulate, cudaStream_t st)
 {
     if (gemm_skinny_supported(M, N, K, A, lda, W, dtype_in)) return launch_gemm_skinny(M, N, K, A, lda, W, C, ldc, out_dtype, accumulate, st);
+    if (gemm_tc_thin_supported(M, N, K, A, lda, W, C, ldc, dtype_in, out_dtype))
+        return launch_gemm_tc_thin(M, N, K, A, lda, W, C, ldc, out_dtype, accumulate, nullptr, st);
     if (gemm_tc_supported(M, N, K, A, lda, W, C, ldc, dtype_in, out_dtype))
         return launch_gemm_tc(M, N, K, A, lda, W, C, ldc, out_dtype, accumulate, nullptr, st);
     return launch_gemm_simt(M, N, K, A, lda, W, C, ldc, dtype_in, out_dtype, accumulate, st);

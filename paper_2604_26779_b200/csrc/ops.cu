@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(256) rope_append_kernel(int R, int Hq, int Hkv
                                                           T* __restrict__ qkv, const int32_t* __restrict__ pos,
                                                           T* __restrict__ k_pool, T* __restrict__ v_pool,
                                                           const int32_t* __restrict__ block_table, int max_blocks,
-                                                          int block_tokens)
+                                                          int block_tokens, const float2* __restrict__ table, int M)
 {
     extern __shared__ float s_cs[];                       // cos [dh/2], sin [dh/2]
     const int m = blockIdx.x;
@@ -110,6 +110,11 @@ __global__ void __launch_bounds__(256) rope_append_kernel(int R, int Hq, int Hkv
     const int b = m / R;
     const int half = dh / 2;
     for (int j = threadIdx.x; j < half; j += blockDim.x) {
+        if (table != nullptr) {                           // the forward's (cos, sin) table [dh/2][M]: the same fp32 values
+            const float2 t = table[(size_t)j * M + m];
+            s_cs[j] = t.x; s_cs[half + j] = t.y;
+            continue;
+        }
         // the angle is formed in fp64: at positions of 10^4 an fp32 product would already be off by 10^-3 rad
         const double inv = exp2(-2.0 * (double)j / (double)dh * log2((double)theta));
         double s, c;
@@ -481,11 +486,12 @@ spec_status launch_rmsnorm(int M, int d, const float* in, const float* w, float 
 
 spec_status launch_rope_append(int B, int R, int Hq, int Hkv, int dh, float theta, void* qkv, const int32_t* pos,
                                void* k_pool, void* v_pool, const int32_t* block_table, int max_blocks,
-                               int block_tokens, int dtype, cudaStream_t st)
+                               int block_tokens, int dtype, cudaStream_t st, const float* rope_table)
 {
     if (B * R == 0) return SPEC_OK;
     DISPATCH_T(dtype, rope_append_kernel<T><<<B * R, 256, dh * sizeof(float), st>>>(
-                          R, Hq, Hkv, dh, theta, (T*)qkv, pos, (T*)k_pool, (T*)v_pool, block_table, max_blocks, block_tokens));
+                          R, Hq, Hkv, dh, theta, (T*)qkv, pos, (T*)k_pool, (T*)v_pool, block_table, max_blocks, block_tokens,
+                          reinterpret_cast<const float2*>(rope_table), B * R));
     return launch_status();
 }
 

@@ -42,7 +42,7 @@ spec_status launch_rmsnorm(int M, int d, const float* in, const float* w, float 
 // rotates q and k of qkv [M][(Hq+2Hkv)*dh] in place and writes k, v into the paged cache at the rows' positions
 spec_status launch_rope_append(int B, int R, int Hq, int Hkv, int dh, float theta, void* qkv, const int32_t* pos,
                                void* k_pool, void* v_pool, const int32_t* block_table, int max_blocks,
-                               int block_tokens, int dtype, cudaStream_t st);
+                               int block_tokens, int dtype, cudaStream_t st, const float* rope_table = nullptr);   // rope_table: [dh/2][B*R] (cos, sin) of pos, or NULL
 spec_status launch_swiglu(int M, int F, const void* gate_up, void* out, int dtype, cudaStream_t st);
 spec_status launch_copy_rows_f32_to(int M, int d, const float* x, void* out, int ld_out, int col0, int dtype,
                                     cudaStream_t st);
@@ -93,6 +93,8 @@ spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void*
 bool gemm_skinny_supported(int M, int N, int K, const void* A, int lda, const void* W, int dtype_in);
 spec_status launch_gemm_skinny(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int out_dtype,
                                int accumulate, cudaStream_t st);
+// 17..64 rows: the tensor-core kernel with the operands swapped (weights as the M operand, one narrow tile of activation rows)
+bool gemm_tc_thin_supported(int M, int N, int K, const void* A, int lda, const void* W, const void* C, int ldc, int dtype_in, int out_dtype);
 spec_status launch_gemm_grouped(int rows_total, int max_rows_per_group, int E, int N, int K, const void* A, const void* W,
                                 void* C, int out_dtype, int swiglu, const int32_t* counts, const int32_t* offsets,
                                 int32_t* status, cudaStream_t st);

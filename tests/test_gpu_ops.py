@@ -107,10 +107,13 @@ def test_paged_attention_matches_oracle(api, lens, R, Hq, Hkv, dh, dtype):
     (17, 28672, 4096, torch.bfloat16, torch.bfloat16, False),
     (31, 50, 768, torch.bfloat16, torch.bfloat16, True),
     (32, 16384, 4096, torch.bfloat16, torch.float32, False),
-    (32, 4096, 4096, torch.bfloat16, torch.float32, True),         # 17..32 rows: back on the tensor-core tile kernel
+    (32, 4096, 4096, torch.bfloat16, torch.float32, True),         # 17..64 rows: the tensor-core kernel with swapped operands (weights as the M operand)
     (20, 6144, 4096, torch.bfloat16, torch.bfloat16, False),
     (25, 4000, 14336, torch.bfloat16, torch.float32, True),
-    (32, 4096, 320, torch.bfloat16, torch.float32, False),         # K not a multiple of 256: stays on the tensor-core tile kernel
+    (32, 4096, 320, torch.bfloat16, torch.float32, False),
+    (33, 1000, 512, torch.bfloat16, torch.float32, False),         # 64-wide token tile, ragged features
+    (48, 6144, 4096, torch.bfloat16, torch.bfloat16, True),
+    (64, 4096, 4096, torch.bfloat16, torch.float32, True),
 ])
 def test_gemm_matches_fp64(api, M, N, K, din, dout, acc):
     kind = "bf16" if din == torch.bfloat16 else "f32"
