@@ -140,6 +140,8 @@ struct MmaArgs {
 template <int DH, int WM, int WN, int STAGES>
 __global__ void __launch_bounds__(kThreads) attn_mma_kernel(const MmaArgs a)
 {
+    pdl_trigger();
+    pdl_wait();
     static_assert(WM * WN == 4, "four warps");
     constexpr int CH = DH / 8;                               // 16-byte chunks per row
     constexpr int kBlkBytes = kBT * DH * 2;                  // one KV block of one head
@@ -362,6 +364,8 @@ __global__ void __launch_bounds__(kThreads) attn_mma_kernel(const MmaArgs a)
 template <int DH>
 __global__ void __launch_bounds__(128) attn_merge_kernel(int B, int rows_alloc, const MmaArgs a)
 {
+    pdl_trigger();
+    pdl_wait();
     const int b = blockIdx.x / a.Hkv, g = blockIdx.x % a.Hkv;
     const int nc = a.pv.nc[b], first = a.pv.first[b];
     const int n_rows_valid = a.R * a.group;
@@ -417,9 +421,9 @@ spec_status run_mma(const MmaArgs& m, int B, bool plan, int max_chunks, cudaStre
         if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
     }
     const int ctas_per_sm = (228 * 1024) / (smem + 2048);
-    kern<<<sm_count() * (ctas_per_sm < 1 ? 1 : ctas_per_sm), kThreads, smem, st>>>(m);
+    launch_pdl(kern, dim3(sm_count() * (ctas_per_sm < 1 ? 1 : ctas_per_sm)), dim3(kThreads), (size_t)smem, st, m);
     if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
-    attn_merge_kernel<DH><<<B * m.Hkv, 128, 0, st>>>(B, 16 * WM, m);
+    launch_pdl(attn_merge_kernel<DH>, dim3(B * m.Hkv), dim3(128), 0, st, B, 16 * WM, m);
     return launch_status(plan ? 3 : 2);
 }
 
@@ -448,7 +452,7 @@ spec_status attn::launch_attn_merge128(int B, int rows_alloc, int Hkv, int R, in
 {
     MmaArgs m{};
     m.R = R; m.group = group; m.Hkv = Hkv; m.out = static_cast<__nv_bfloat16*>(out); m.out_row_stride = out_row_stride; m.pv = pv;
-    attn_merge_kernel<128><<<B * Hkv, 128, 0, st>>>(B, rows_alloc, m);
+    launch_pdl(attn_merge_kernel<128>, dim3(B * Hkv), dim3(128), 0, st, B, rows_alloc, m);
     return launch_status();
 }
 

@@ -30,6 +30,25 @@ inline spec_status launch_status(int n_launched = 1)
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }
 
+// Programmatic dependent launch.  A kernel launched through launch_pdl may be scheduled before the kernel in front of it
+// in the stream has finished (as soon as that one has called pdl_trigger, or has exited), which hides the launch latency
+// between the many short dependent kernels of a step; it must call pdl_wait before it touches global memory (the wait
+// returns once the kernel in front has completed and its writes are visible).  Both calls are no-ops in a kernel that
+// was launched the ordinary way.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Per-thread scratch for split-K GEMMs, set by the context entry points (the stateless spec_gemm has none and never splits).
 struct GemmScratch { void* ptr = nullptr; size_t bytes = 0; };
 GemmScratch& gemm_scratch();

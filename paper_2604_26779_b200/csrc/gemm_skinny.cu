@@ -51,6 +51,8 @@ __global__ void __launch_bounds__(kThreads) gemm_skinny_kernel(int M, int N, int
     constexpr int TOK = 8 * NT;
     constexpr int W_SUB = kRows * 128, A_SUB = TOK * 128;
     constexpr int STAGE = 4 * (W_SUB + A_SUB);
+    pdl_trigger();
+    pdl_wait();
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t base = smem_u32(smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -169,8 +171,8 @@ spec_status run_skinny(int M, int N, int K, const void* A, int lda, const void* 
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SPEC_ERR_CUDA;
         configured = true;
     }
-    kern<<<(N + kRows - 1) / kRows, kThreads, smem, st>>>(M, N, K, (const __nv_bfloat16*)A, lda, (const __nv_bfloat16*)W, C, ldc,
-                                                          out_dtype == SPEC_DTYPE_F32 ? 1 : 0, accumulate);
+    launch_pdl(kern, dim3((N + kRows - 1) / kRows), dim3(kThreads), (size_t)smem, st, M, N, K, (const __nv_bfloat16*)A, lda,
+               (const __nv_bfloat16*)W, C, ldc, out_dtype == SPEC_DTYPE_F32 ? 1 : 0, accumulate);
     return launch_status();
 }
 

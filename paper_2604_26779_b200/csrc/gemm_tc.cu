@@ -435,6 +435,7 @@ template <int EPI>
 __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a,
                                                               const __grid_constant__ CUtensorMap map_b, const GemmArgs g)
 {
+    pdl_trigger();                                                        // the next kernel may be scheduled behind this one
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;                        // 1024-byte aligned stage ring
@@ -444,6 +445,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     const int m_tiles = (g.M + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
+    if (g.E > 0) pdl_wait();                                // the counts are another kernel's output
     if (g.E > 0 && threadIdx.x == 64) {                     // grouped: the m-tile prefix table (counts live on the device)
         int run = 0;
         for (int e = 0; e < g.E; ++e) { ctl->pref[e] = run; run += (min(g.counts[e], g.max_m_tiles * BM) + BM - 1) / BM; }
@@ -467,6 +469,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int* pref = ctl->pref;
+    pdl_wait();                                                           // from here on global memory of the kernels in front is read
     const int n_work = g.E > 0 ? pref[g.E] * n_tiles : m_tiles * n_tiles * (g.splits > 1 ? g.splits : 1);
 
     if (warp == 0) {
@@ -595,6 +598,8 @@ template <class TC>
 __global__ void splitk_reduce_kernel(int M, int N, int splits, const float* __restrict__ part, TC* __restrict__ C, int ldc,
                                      int accumulate)
 {
+    pdl_trigger();
+    pdl_wait();
     const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= (size_t)M * N) return;
     const int m = (int)(i / N), n = (int)(i % N);
@@ -635,10 +640,10 @@ bool init_once()
 spec_status run_kernel(int epi, const CUtensorMap& ma, const CUtensorMap& mb, const GemmArgs& g, long long n_work, cudaStream_t st)
 {
     const int grid = n_work < g_sms ? (int)n_work : g_sms;
-    if (epi == EPI_SWIGLU)   gemm_tc_kernel<EPI_SWIGLU><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, g);
-    else if (epi == EPI_QKV) gemm_tc_kernel<EPI_QKV><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, g);
-    else if (epi == EPI_THIN) gemm_tc_kernel<EPI_THIN><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, g);
-    else                     gemm_tc_kernel<EPI_PLAIN><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, g);
+    if (epi == EPI_SWIGLU)   launch_pdl(gemm_tc_kernel<EPI_SWIGLU>, dim3(grid), dim3(kThreads), (size_t)kSmemBytes, st, ma, mb, g);
+    else if (epi == EPI_QKV) launch_pdl(gemm_tc_kernel<EPI_QKV>, dim3(grid), dim3(kThreads), (size_t)kSmemBytes, st, ma, mb, g);
+    else if (epi == EPI_THIN) launch_pdl(gemm_tc_kernel<EPI_THIN>, dim3(grid), dim3(kThreads), (size_t)kSmemBytes, st, ma, mb, g);
+    else                     launch_pdl(gemm_tc_kernel<EPI_PLAIN>, dim3(grid), dim3(kThreads), (size_t)kSmemBytes, st, ma, mb, g);
     return launch_status();
 }
 

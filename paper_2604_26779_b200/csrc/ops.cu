@@ -68,6 +68,8 @@ template <class T>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(int d, const float* __restrict__ in, const float* __restrict__ w,
                                                       float eps, T* __restrict__ out, int ld_out, int col0)
 {
+    pdl_trigger();
+    pdl_wait();
     const int m = blockIdx.x;
     const float* xr = in + (size_t)m * d;
     __shared__ float s_part[8];
@@ -103,6 +105,8 @@ __global__ void __launch_bounds__(256) rope_append_kernel(int R, int Hq, int Hkv
                                                           const int32_t* __restrict__ block_table, int max_blocks,
                                                           int block_tokens, const float2* __restrict__ table, int M)
 {
+    pdl_trigger();
+    pdl_wait();
     extern __shared__ float s_cs[];                       // cos [dh/2], sin [dh/2]
     const int m = blockIdx.x;
     const int p = pos[m];
@@ -153,6 +157,8 @@ __global__ void __launch_bounds__(256) rope_append_kernel(int R, int Hq, int Hkv
 template <class T>
 __global__ void swiglu_kernel(size_t total4, int F, const T* __restrict__ gu, T* __restrict__ out)
 {
+    pdl_trigger();
+    pdl_wait();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= total4) return;
     const size_t e = i * 4;
@@ -185,6 +191,8 @@ __global__ void rope_table_kernel(int M, int half, int dh, float theta, const in
 template <class T>
 __global__ void copy_rows_kernel(int d, const float* __restrict__ x, T* __restrict__ out, int ld_out, int col0)
 {
+    pdl_trigger();
+    pdl_wait();
     const int m = blockIdx.x;
     for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
         float v[4];
@@ -480,7 +488,7 @@ spec_status launch_rmsnorm(int M, int d, const float* in, const float* w, float 
                            int dtype, cudaStream_t st)
 {
     if (M == 0) return SPEC_OK;
-    DISPATCH_T(dtype, rmsnorm_kernel<T><<<M, 256, 0, st>>>(d, in, w, eps, (T*)out, ld_out, col0));
+    DISPATCH_T(dtype, launch_pdl(rmsnorm_kernel<T>, dim3(M), dim3(256), 0, st, d, in, w, eps, (T*)out, ld_out, col0));
     return launch_status();
 }
 
@@ -489,7 +497,7 @@ spec_status launch_rope_append(int B, int R, int Hq, int Hkv, int dh, float thet
                                int block_tokens, int dtype, cudaStream_t st, const float* rope_table)
 {
     if (B * R == 0) return SPEC_OK;
-    DISPATCH_T(dtype, rope_append_kernel<T><<<B * R, 256, dh * sizeof(float), st>>>(
+    DISPATCH_T(dtype, launch_pdl(rope_append_kernel<T>, dim3(B * R), dim3(256), dh * sizeof(float), st,
                           R, Hq, Hkv, dh, theta, (T*)qkv, pos, (T*)k_pool, (T*)v_pool, block_table, max_blocks, block_tokens,
                           reinterpret_cast<const float2*>(rope_table), B * R));
     return launch_status();
@@ -499,7 +507,7 @@ spec_status launch_swiglu(int M, int F, const void* gate_up, void* out, int dtyp
 {
     const size_t total4 = (size_t)M * F / 4;
     if (total4 == 0) return SPEC_OK;
-    DISPATCH_T(dtype, swiglu_kernel<T><<<(unsigned)((total4 + 255) / 256), 256, 0, st>>>(total4, F, (const T*)gate_up, (T*)out));
+    DISPATCH_T(dtype, launch_pdl(swiglu_kernel<T>, dim3((unsigned)((total4 + 255) / 256)), dim3(256), 0, st, total4, F, (const T*)gate_up, (T*)out));
     return launch_status();
 }
 
@@ -515,7 +523,7 @@ spec_status launch_copy_rows_f32_to(int M, int d, const float* x, void* out, int
                                     cudaStream_t st)
 {
     if (M == 0) return SPEC_OK;
-    DISPATCH_T(dtype, copy_rows_kernel<T><<<M, 256, 0, st>>>(d, x, (T*)out, ld_out, col0));
+    DISPATCH_T(dtype, launch_pdl(copy_rows_kernel<T>, dim3(M), dim3(256), 0, st, d, x, (T*)out, ld_out, col0));
     return launch_status();
 }
 
