@@ -366,15 +366,19 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(int B, int rows_alloc, 
 {
     pdl_trigger();
     pdl_wait();
+    // blockIdx.x = (sequence, KV head); blockIdx.y = a slice of 128 (row, 4-column) elements, so that a thin batch still
+    // spreads over many SMs
     const int b = blockIdx.x / a.Hkv, g = blockIdx.x % a.Hkv;
     const int nc = a.pv.nc[b], first = a.pv.first[b];
     const int n_rows_valid = a.R * a.group;
     if (nc == 1) return;
-    for (int e = threadIdx.x; e < n_rows_valid * (DH / 4); e += 128) {
+    for (int e = blockIdx.y * 128 + threadIdx.x; e < n_rows_valid * (DH / 4); e += 128 * gridDim.y) {
         const int r = e / (DH / 4), c4 = (e % (DH / 4)) * 4;
         float acc[4] = {0.f, 0.f, 0.f, 0.f}, L = 0.f, M = -INFINITY;
+#pragma unroll 4
         for (int c = 0; c < nc; ++c) M = fmaxf(M, a.pv.part_ml[(((size_t)(first + c) * a.Hkv + g) * rows_alloc + r) * 2]);
-        for (int c = 0; c < nc; ++c) {
+#pragma unroll 4
+        for (int c = 0; c < nc; ++c) {                       // chunk order: the sum does not depend on who computed what when
             const size_t ps = ((size_t)(first + c) * a.Hkv + g) * rows_alloc + r;
             const float mw = a.pv.part_ml[ps * 2];
             const float f = (mw == -INFINITY) ? 0.f : exp2f(mw - M);
@@ -423,7 +427,7 @@ spec_status run_mma(const MmaArgs& m, int B, bool plan, int max_chunks, cudaStre
     const int ctas_per_sm = (228 * 1024) / (smem + 2048);
     launch_pdl(kern, dim3(sm_count() * (ctas_per_sm < 1 ? 1 : ctas_per_sm)), dim3(kThreads), (size_t)smem, st, m);
     if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
-    launch_pdl(attn_merge_kernel<DH>, dim3(B * m.Hkv), dim3(128), 0, st, B, 16 * WM, m);
+    launch_pdl(attn_merge_kernel<DH>, dim3(B * m.Hkv, (m.R * m.group * (DH / 4) + 127) / 128), dim3(128), 0, st, B, 16 * WM, m);
     return launch_status(plan ? 3 : 2);
 }
 
@@ -452,7 +456,7 @@ spec_status attn::launch_attn_merge128(int B, int rows_alloc, int Hkv, int R, in
 {
     MmaArgs m{};
     m.R = R; m.group = group; m.Hkv = Hkv; m.out = static_cast<__nv_bfloat16*>(out); m.out_row_stride = out_row_stride; m.pv = pv;
-    launch_pdl(attn_merge_kernel<128>, dim3(B * Hkv), dim3(128), 0, st, B, rows_alloc, m);
+    launch_pdl(attn_merge_kernel<128>, dim3(B * Hkv, (R * group * 32 + 127) / 128), dim3(128), 0, st, B, rows_alloc, m);
     return launch_status();
 }
 
