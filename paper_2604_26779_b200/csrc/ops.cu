@@ -130,6 +130,42 @@ __global__ void __launch_bounds__(256) rope_append_kernel(int R, int Hq, int Hkv
     T* row = qkv + (size_t)m * (Hq + 2 * Hkv) * dh;
     const int blk = block_table[(size_t)b * max_blocks + p / block_tokens];
     const int slot = p % block_tokens;
+    if constexpr (sizeof(T) == 2) {
+        if (half % 8 == 0) {
+            // bf16: eight pairs per thread, 16-byte loads and stores (the scalar loop below is latency-bound at small batch)
+            const int vec = half / 8;
+            for (int idx = threadIdx.x; idx < (Hq + Hkv) * vec; idx += blockDim.x) {
+                const int h = idx / vec, j = (idx % vec) * 8;
+                T* hp = row + (size_t)h * dh;
+                uint4 ua = *reinterpret_cast<const uint4*>(hp + j), ub = *reinterpret_cast<const uint4*>(hp + j + half);
+                T* pa = reinterpret_cast<T*>(&ua);
+                T* pb = reinterpret_cast<T*>(&ub);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float a = to_f32(pa[e]), bb = to_f32(pb[e]);
+                    const float c = s_cs[j + e], sn = s_cs[half + j + e];
+                    pa[e] = from_f32<T>(a * c - bb * sn);
+                    pb[e] = from_f32<T>(bb * c + a * sn);
+                }
+                T* dst = nullptr;
+                if (h < Hq) dst = hp;
+                else if (blk >= 0) dst = k_pool + (((size_t)blk * Hkv + (h - Hq)) * block_tokens + slot) * dh;
+                if (dst != nullptr) {
+                    *reinterpret_cast<uint4*>(dst + j) = ua;
+                    *reinterpret_cast<uint4*>(dst + j + half) = ub;
+                }
+            }
+            if (blk >= 0) {
+                const T* vsrc = row + (size_t)(Hq + Hkv) * dh;
+                for (int idx = threadIdx.x; idx < Hkv * dh / 8; idx += blockDim.x) {
+                    const int h = (idx * 8) / dh, j = (idx * 8) % dh;
+                    *reinterpret_cast<uint4*>(v_pool + (((size_t)blk * Hkv + h) * block_tokens + slot) * dh + j) =
+                        *reinterpret_cast<const uint4*>(vsrc + (size_t)idx * 8);
+                }
+            }
+            return;
+        }
+    }
     // q and k heads: rotate pairs
     for (int idx = threadIdx.x; idx < (Hq + Hkv) * half; idx += blockDim.x) {
         const int h = idx / half, j = idx % half;
