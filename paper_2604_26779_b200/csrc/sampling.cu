@@ -331,6 +331,89 @@ __global__ void __launch_bounds__(kThreads) softmax_rows_kernel(int rows, int V,
     }
 }
 
+// The same statistics (and probabilities) by a cluster of kStatCtas CTAs per row: with few rows (a thin batch) one CTA per
+// row reads its 0.5 MB of logits far below the memory rate.  Every CTA reduces a quarter-aligned slice of the row, hands its
+// (m, z) pair to the first CTA through distributed shared memory, and that one combines the pairs in rank order.
+constexpr int kStatCtas = 8;
+__global__ void __launch_bounds__(kThreads) softmax_rows_cluster_kernel(int rows, int V, const float* __restrict__ logits,
+                                                                        size_t row_stride, float inv_t,
+                                                                        float* __restrict__ stats, size_t stats_stride,
+                                                                        float* __restrict__ probs)
+{
+    const int row = blockIdx.x / kStatCtas;
+    const uint32_t rank = cluster_cta_rank();
+    const float* l = logits + (size_t)row * row_stride;
+    const bool vec = row_vec_ok(l, V);
+    __shared__ float s_m[kWarps], s_z[kWarps];
+    __shared__ float s_pair[2 * kStatCtas];                  // first CTA: (m, z) of every rank
+    __shared__ float s_fin[2];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int slice = (((V + kStatCtas - 1) / kStatCtas) + 3) & ~3;
+    const int lo = min(V, (int)rank * slice), hi = min(V, lo + slice);
+
+    float m = -INFINITY, z = 0.f;
+    for (int base = lo + threadIdx.x * 4; base < hi; base += kThreads * 4) {
+        float a[4];
+        load4(l, base, hi, vec, -INFINITY, a);
+        const float mx = fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3]));
+        if (mx > m) { z *= __expf(__fmul_rn(__fsub_rn(m, mx), inv_t)); m = mx; }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) z += __expf(__fmul_rn(__fsub_rn(a[e], m), inv_t));
+    }
+    const float wm = warp_max(m);
+    z = (m == -INFINITY) ? 0.f : z * __expf(__fmul_rn(__fsub_rn(m, wm), inv_t));
+    z = warp_sum(z);
+    if (lane == 0) { s_m[warp] = wm; s_z[warp] = z; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float bm = s_m[0];
+        for (int w = 1; w < kWarps; ++w) bm = fmaxf(bm, s_m[w]);
+        float bz = 0.f;
+        for (int w = 0; w < kWarps; ++w)
+            bz += (s_m[w] == -INFINITY) ? 0.f : s_z[w] * __expf(__fmul_rn(__fsub_rn(s_m[w], bm), inv_t));
+        uint32_t remote;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(&s_pair[2 * rank])), "r"(0));
+        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(bm) : "memory");
+        asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote + 4u), "f"(bz) : "memory");
+    }
+    cluster_sync_all();
+    if (rank == 0 && threadIdx.x == 0) {
+        float bm = s_pair[0];
+        for (int r = 1; r < kStatCtas; ++r) bm = fmaxf(bm, s_pair[2 * r]);
+        float bz = 0.f;
+        for (int r = 0; r < kStatCtas; ++r)
+            bz += (s_pair[2 * r] == -INFINITY) ? 0.f : s_pair[2 * r + 1] * __expf(__fmul_rn(__fsub_rn(s_pair[2 * r], bm), inv_t));
+        s_fin[0] = bm; s_fin[1] = bz;
+        if (stats) { stats[2 * (size_t)row * stats_stride] = bm; stats[2 * (size_t)row * stats_stride + 1] = bz; }
+    }
+    if (probs == nullptr) return;                            // uniform over the cluster: no CTA waits below for one that left
+    cluster_sync_all();
+    float bm, bz;
+    {
+        uint32_t remote;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(&s_fin[0])), "r"(0));
+        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(bm) : "r"(remote) : "memory");
+        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(bz) : "r"(remote + 4u) : "memory");
+    }
+    const float inv_z = __frcp_rn(bz);
+    float* pr = probs + (size_t)row * V;
+    const bool vec_out = vec && ((reinterpret_cast<uintptr_t>(pr) & 15u) == 0);
+    for (int base = lo + threadIdx.x * 4; base < hi; base += kThreads * 4) {
+        float a[4];
+        load4(l, base, hi, vec, -INFINITY, a);
+        float o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[e] = prob_from_logit(a[e], bm, inv_t, inv_z);
+        if (vec_out && base + 3 < hi) {
+            *reinterpret_cast<float4*>(pr + base) = make_float4(o[0], o[1], o[2], o[3]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) if (base + e < hi) pr[base + e] = o[e];
+        }
+    }
+    cluster_sync_all();                                      // the first CTA's shared memory is read until here
+}
+
 // ---- one token per row by inverse CDF -----------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads) sample_rows_kernel(int V, const float* __restrict__ probs, uint64_t seed,
                                                                uint32_t step, uint32_t slot, uint32_t stream_tag,
@@ -563,6 +646,17 @@ spec_status launch_softmax_rows(int rows, int V, const float* logits, size_t row
                                 size_t stats_stride, float* probs, cudaStream_t st)
 {
     if (rows == 0) return SPEC_OK;
+    if (rows <= 128 && V >= 8192) {                          // few rows: a cluster of CTAs per row
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)rows * kStatCtas); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute attr{};
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = kStatCtas; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr; cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, softmax_rows_cluster_kernel, rows, V, logits, row_stride, 1.0f / temperature, stats, stats_stride, probs) !=
+            cudaSuccess) { cudaGetLastError(); return SPEC_ERR_CUDA; }
+        return launch_status();
+    }
     softmax_rows_kernel<<<rows, kThreads, 0, st>>>(rows, V, logits, row_stride, 1.0f / temperature, stats, stats_stride, probs);
     return launch_status();
 }
