@@ -375,6 +375,47 @@ def run_ep_microbench(args):
     return 0
 
 
+def run_rollout_bench(args):
+    """A whole rollout batch on the 8B shape with continuous batching: `--rollout-prompts` prompts through `--batch` slots,
+    long-tailed response lengths (lognormal), prompts prefilled through forced verify steps, finished slots refilled, then
+    retired.  Run twice, without and with batch compaction, to show what the thin tail costs.  Wall clock over the whole
+    rollout, every step followed by a device-to-host read of the emitted tokens (the driver needs them)."""
+    import torch
+    from paper_2604_26779_b200 import rollout, workloads
+    slots, n_prompts, k = args.batch, args.rollout_prompts, args.k
+    rng = np.random.default_rng(2604026779 % (2 ** 32))
+    p_lens = rng.integers(16, 64, n_prompts)
+    wants = np.clip(np.exp(rng.normal(np.log(args.rollout_median), 1.0, n_prompts)).astype(np.int64), 8, args.rollout_max)
+    cap = int(p_lens.max() + wants.max() + k + 2)
+    out = {}
+    for label, frac in (("no_compaction", 0.0), ("compaction", 0.5)):
+        eng, info = workloads.build_dense_workload("c3", lens=np.full(slots, cap, np.int32), k=k, n_layers=args.layers, steps_budget=2)
+        vocab = info["cfg"]["vocab"]
+        prng = np.random.default_rng(7)
+        prompts = [prng.integers(0, vocab, n).astype(np.int32) for n in p_lens]
+        ro = rollout.Rollout(eng, prompts, [int(w) for w in wants], info["block_order"], compact_fraction=frac)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        done = ro.run(max_steps=200000)
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - t0
+        assert len(done) == n_prompts and eng.status().device_status == 0
+        tokens = sum(len(r.tokens) for r in done.values())
+        thin = sum(1 for a in ro.active_trace if a <= slots // 8)
+        out[label] = {"seconds": wall, "response_tokens": tokens, "tokens_per_s": tokens / wall, "steps": ro.step,
+                      "steps_with_at_most_an_eighth_of_the_slots_live": thin, "compactions": ro.compactions,
+                      "acceptance_rate": rollout.acceptance_rate(*ro._acc)}
+        eng.close(); del eng
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "rollout of a whole batch with continuous batching (8B shape; not the headline)", "unit": "response tokens/s",
+                      "n_gpus": 1, "slots": slots, "prompts": n_prompts, "k": k, "layers": args.layers,
+                      "response_lengths": {"distribution": "lognormal", "median": args.rollout_median, "sigma": 1.0, "max": int(wants.max()),
+                                           "mean": float(wants.mean())},
+                      "data": "synthetic", "dtype": "bf16", **out,
+                      "speedup_from_compaction": out["compaction"]["tokens_per_s"] / out["no_compaction"]["tokens_per_s"]}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -402,7 +443,10 @@ def main():
     ap.add_argument("--ep", type=int, default=8, help="c5ep only: ranks of the expert-parallel group (emulated on one GPU)")
     ap.add_argument("--ep-capacity", type=float, default=2.0,
                     help="c5ep only: receive capacity per rank as a multiple of the mean load rows*top_k (capped by the worst case)")
-    ap.add_argument("--workload", default="c3", choices=["c3", "c4", "c5", "c2", "c5ep"],
+    ap.add_argument("--rollout-prompts", type=int, default=256, help="rollout only: prompts in the batch")
+    ap.add_argument("--rollout-median", type=float, default=96.0, help="rollout only: median response length")
+    ap.add_argument("--rollout-max", type=int, default=1024, help="rollout only: longest response")
+    ap.add_argument("--workload", default="c3", choices=["c3", "c4", "c5", "c2", "c5ep", "rollout"],
                     help="c3 = the headline 8B + EAGLE-3 workload; c4 = 8B + MTP head, B=512, lognormal lengths; "
                          "c5 = one 235B-A22B-shaped MoE layer + LM head, B=256, cache length 8192 (measurement of the "
                          "other configurations; the reported metric line is c3)")
@@ -421,6 +465,8 @@ def main():
         return run_sampler_microbench(args) if rank == 0 else 0
     if args.workload == "c5ep":
         return run_ep_microbench(args) if rank == 0 else 0
+    if args.workload == "rollout":
+        return run_rollout_bench(args) if rank == 0 else 0
     if args.k_sweep:
         return run_k_sweep(args, [int(x) for x in args.k_sweep.split(",")]) if rank == 0 else 0
     dist = None
