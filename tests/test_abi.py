@@ -45,6 +45,17 @@ def test_host_side_argument_checks(built_lib):
     assert L.spec_query_sizes(None, None) < 0
     # context entry points refuse a missing context before touching anything
     assert L.spec_seq_replace(None, 1, None, None, None, None) == -1
+    assert L.spec_seq_compact(None, 1, None, None) == -1
+    # expert-parallel block and window plumbing: NULL pointers and impossible shapes are refused on the host
+    assert L.spec_ep_query_sizes(None, None) == -1
+    assert L.spec_ep_route(None, None, None, 0, None, None, None) == -1
+    assert L.spec_ep_experts(None, None, None, None, None, None, None) == -1
+    assert L.spec_ep_combine(None, None, 0, None, None) == -1
+    cfg = binding.spec_ep_config(2, 0, 16, 4, 512, 128, 64, 256)
+    sizes = binding.spec_ep_query_sizes(cfg)
+    assert sizes.window_bytes > 64 * 512 * 2 and sizes.scratch_bytes > 0
+    assert L.spec_ep_route(ctypes.byref(cfg), None, None, 1, None, None, None) == -1
+    assert L.spec_ipc_export(None, None, None) == -1 and L.spec_ipc_open(None, None) == -1 and L.spec_ipc_close(None) == -1
     assert L.spec_seq_init(None, 1, None, None, None, None) == -1
     assert L.spec_verify(None, 0, None, None) == -1
     assert L.spec_draft(None, 1, None) == -1
