@@ -632,6 +632,12 @@ def main():
         eng.set_timing(0)
         ms_vs = timed(lambda: workloads_spec_step(eng, k, with_draft=False), 3)
         ms_dec = timed(lambda: workloads.bootstrap(eng), 3)
+        eng.set_timing(15)
+        eng.get_timing()
+        for _ in range(2):
+            workloads.bootstrap(eng)
+        tmd = eng.get_timing()
+        eng.set_timing(0)
         # the same step captured once into a CUDA graph and replayed (the step functions only enqueue, so capture works)
         ms_graph = None
         try:
@@ -663,6 +669,9 @@ def main():
                           "projected_tokens_per_s_at_paper_AL": {"2.77": 2.77 * B / (ms_total / args.steps / 1000.0),
                                                                  "3.32": 3.32 * B / (ms_total / args.steps / 1000.0)},
                           "ms_by_class_per_step": {"attention": tm.ms[0] / 2, "gemm": tm.ms[1] / 2, "softmax_sampling": tm.ms[2] / 2},
+                          "ms_by_class_plain_decode_step": {"attention": tmd.ms[0] / 2, "gemm": tmd.ms[1] / 2, "softmax_sampling": tmd.ms[2] / 2},
+                          "plain_decode_gemm_bound_ms": {"tensor": gemm_flops_per_step(cfg, B, 0, "none") / (tf_peak * 1e12) * 1e3,
+                                                         "weights_once_from_hbm": gemm_flops_per_step(cfg, 1, 0, "none") / (hbm_peak * 1e9) * 1e3},
                           "gemm_tflops_in_step": gemm_flops_per_step(cfg, B, k, info["draft"]) / (tm.ms[1] / 2 * 1e-3) / 1e12,
                           "gemm_frac_of_measured_sustained_bf16": gemm_flops_per_step(cfg, B, k, info["draft"]) / (tm.ms[1] / 2 * 1e-3) / 1e12 / tf_peak,
                           }
