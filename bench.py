@@ -378,7 +378,8 @@ def run_ep_microbench(args):
 def run_rollout_bench(args):
     """A whole rollout batch on the 8B shape with continuous batching: `--rollout-prompts` prompts through `--batch` slots,
     long-tailed response lengths (lognormal), prompts prefilled through forced verify steps, finished slots refilled, then
-    retired.  Run twice, without and with batch compaction, to show what the thin tail costs.  Wall clock over the whole
+    retired.  Run three times - without batch compaction, with it, and with it plus CUDA-graph replay of the steps in which
+    no slot is prefilling - to show what the thin tail costs.  Wall clock over the whole
     rollout, every step followed by a device-to-host read of the emitted tokens (the driver needs them)."""
     import torch
     from paper_2604_26779_b200 import rollout, workloads
@@ -388,12 +389,12 @@ def run_rollout_bench(args):
     wants = np.clip(np.exp(rng.normal(np.log(args.rollout_median), 1.0, n_prompts)).astype(np.int64), 8, args.rollout_max)
     cap = int(p_lens.max() + wants.max() + k + 2)
     out = {}
-    for label, frac in (("no_compaction", 0.0), ("compaction", 0.5)):
+    for label, frac, graphs in (("no_compaction", 0.0, False), ("compaction", 0.5, False), ("compaction_and_graphs", 0.5, True)):
         eng, info = workloads.build_dense_workload("c3", lens=np.full(slots, cap, np.int32), k=k, n_layers=args.layers, steps_budget=2)
         vocab = info["cfg"]["vocab"]
         prng = np.random.default_rng(7)
         prompts = [prng.integers(0, vocab, n).astype(np.int32) for n in p_lens]
-        ro = rollout.Rollout(eng, prompts, [int(w) for w in wants], info["block_order"], compact_fraction=frac)
+        ro = rollout.Rollout(eng, prompts, [int(w) for w in wants], info["block_order"], compact_fraction=frac, use_graphs=graphs)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         done = ro.run(max_steps=200000)
@@ -403,7 +404,7 @@ def run_rollout_bench(args):
         tokens = sum(len(r.tokens) for r in done.values())
         thin = sum(1 for a in ro.active_trace if a <= slots // 8)
         out[label] = {"seconds": wall, "response_tokens": tokens, "tokens_per_s": tokens / wall, "steps": ro.step,
-                      "steps_with_at_most_an_eighth_of_the_slots_live": thin, "compactions": ro.compactions,
+                      "steps_with_at_most_an_eighth_of_the_slots_live": thin, "compactions": ro.compactions, "graph_steps": ro.graph_steps,
                       "acceptance_rate": rollout.acceptance_rate(*ro._acc)}
         eng.close(); del eng
         torch.cuda.empty_cache()
@@ -412,7 +413,8 @@ def run_rollout_bench(args):
                       "response_lengths": {"distribution": "lognormal", "median": args.rollout_median, "sigma": 1.0, "max": int(wants.max()),
                                            "mean": float(wants.mean())},
                       "data": "synthetic", "dtype": "bf16", **out,
-                      "speedup_from_compaction": out["compaction"]["tokens_per_s"] / out["no_compaction"]["tokens_per_s"]}))
+                      "speedup_from_compaction": out["compaction"]["tokens_per_s"] / out["no_compaction"]["tokens_per_s"],
+                      "speedup_from_compaction_and_graphs": out["compaction_and_graphs"]["tokens_per_s"] / out["no_compaction"]["tokens_per_s"]}))
     return 0
 
 

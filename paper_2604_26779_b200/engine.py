@@ -190,6 +190,25 @@ class SpecStep:
         B._check(self.lib.spec_seq_compact(self.ctx, ks.shape[0], ks.ctypes.data if ks.shape[0] else None, B._stream(stream)), "spec_seq_compact")
         self.B = int(ks.shape[0])
 
+    def capture_step(self, k, with_draft=True):
+        """Captures draft(k) -> verify(k) -> reject_sample(k) -> kv_commit() into a CUDA graph (the step functions only
+        enqueue work, and the step counter and all sequence state live on the device) and returns the graph; `replay()` it
+        on the current stream in place of the four calls.  Worth it when the batch is thin and the step is a chain of
+        hundreds of short kernels.  The graph is tied to the current batch size: capture again after seq_init or
+        seq_compact.  A plain step with the same k must have run before (lazy one-time initialisation happens outside a
+        capture), and no forced commit or caller-supplied drafts can go through a captured step."""
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            if with_draft:
+                self.draft(k)
+            self.verify(k)
+            self.reject_sample(k)
+            self.kv_commit()
+        torch.cuda.current_stream().wait_stream(side)
+        return graph
+
     def draft(self, k, stream=None):
         B._check(self.lib.spec_draft(self.ctx, k, B._stream(stream)), "spec_draft")
 

@@ -12,8 +12,9 @@ torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("kind,compact", [("eagle3", 0.0), ("ngram", 0.0), ("eagle3", 0.7), ("ngram", 0.7)])
-def test_rollout_with_refill_matches_oracle_chains(kind, compact):
+@pytest.mark.parametrize("kind,compact,graphs", [("eagle3", 0.0, False), ("ngram", 0.0, False), ("eagle3", 0.7, False), ("ngram", 0.7, False),
+                                                 ("eagle3", 0.7, True), ("ngram", 0.0, True)])
+def test_rollout_with_refill_matches_oracle_chains(kind, compact, graphs):
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from paper_2604_26779_b200 import engine, rollout
@@ -33,7 +34,7 @@ def test_rollout_with_refill_matches_oracle_chains(kind, compact):
         eng.load_draft_weights(H)
     order = inputs.make_block_order(sc.kv_num_blocks, inputs.sub_seed(3, 3))
     ro = rollout.Rollout(eng, prompts, wants, order, k_policy=lambda step, n_active, alpha: 1 + step % k_max,
-                         compact_fraction=compact)
+                         compact_fraction=compact, use_graphs=graphs)
     done = ro.run(max_steps=400)
     assert sorted(done) == list(range(7))
     assert max(ro.active_trace) == slots and min(ro.active_trace) >= 1
@@ -58,6 +59,8 @@ def test_rollout_with_refill_matches_oracle_chains(kind, compact):
             ref += new
     print(f"rollout {kind}: {ro.step} steps, k trace {ro.k_trace[:8]}..., boundary {boundary}")
     assert boundary <= 1
+    if graphs:
+        assert ro.graph_steps >= 1
     if compact:
         assert len(ro.compactions) >= 1 and ro.compactions[-1][2] < slots
     # everything is retired and every block is back
