@@ -610,7 +610,14 @@ def main():
                 "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": attn_ms, "launches_timed": attn_passes,
                 "share_of_step": float(timing.ms[0]) / ms_total, "frac_of_nominal_8TBs": achieved / 8000.0}
 
-    line = {"metric": METRIC + (" [8-bit KV cache variant]" if cfg.get("kv_fp8") else ""), "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+    metric = METRIC
+    if args.workload == "c4":
+        metric = f"accepted tokens/s per B200 (8B-shape + MTP head, B=512, lognormal lengths, k={k}; not the headline)"
+    elif args.workload == "c5":
+        metric = f"accepted tokens/s per B200 (one 235B-A22B-shaped MoE layer + LM head, k={k}; not the headline)"
+    elif k != 3 or B != 256:
+        metric = f"accepted tokens/s per B200 (8B-shape verify+sample, k={k}, B={B}; not the headline configuration)"
+    line = {"metric": metric + (" [8-bit KV cache variant]" if cfg.get("kv_fp8") else ""), "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": int(launches),
             "roofline": roofline,
