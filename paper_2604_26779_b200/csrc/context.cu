@@ -649,10 +649,22 @@ extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_toke
         if (has_tap(g, l + 1)) TRY(launch_copy_rows_f32_to(M, d, x, at(ws, c->taps), tapw, tap_slot(g, l + 1) * d, dt, st));
     }
     TRY(launch_rmsnorm(M, d, x, at<const float>(c->buf.weights, c->final_norm), g.rms_eps, at(ws, c->h), d, 0, dt, st));
-    TIMED(*c, CLS_GEMM, launch_gemm(M, g.vocab, d, at(ws, c->h), d, at(c->buf.weights, c->lm_head), at(ws, c->logits), g.vocab, dt,
-                                    SPEC_DTYPE_F32, 0, st));
-    TIMED(*c, CLS_SAMPLE, launch_softmax_rows(M, g.vocab, at<float>(ws, c->logits), (size_t)g.vocab, g.temperature,
-                                              at<float>(ws, c->row_stats), 1, nullptr, st));
+    // LM head with the row statistics taken in its epilogue; shapes the tile kernel does not take go the two-pass way
+    spec_status fused = SPEC_ERR_UNSUPPORTED;
+    {
+        Timed t__(*c, CLS_GEMM, st);
+        fused = launch_gemm_lm_head_stats(M, g.vocab, d, at(ws, c->h), d, at(c->buf.weights, c->lm_head), at<float>(ws, c->logits), g.vocab, dt,
+                                          g.temperature, at<float>(ws, c->splitk), c->splitk.bytes, at<float>(ws, c->row_stats), 1,
+                                          at<int32_t>(sb, c->status), st);
+    }
+    if (fused == SPEC_ERR_UNSUPPORTED) {
+        TIMED(*c, CLS_GEMM, launch_gemm(M, g.vocab, d, at(ws, c->h), d, at(c->buf.weights, c->lm_head), at(ws, c->logits), g.vocab, dt,
+                                        SPEC_DTYPE_F32, 0, st));
+        TIMED(*c, CLS_SAMPLE, launch_softmax_rows(M, g.vocab, at<float>(ws, c->logits), (size_t)g.vocab, g.temperature,
+                                                  at<float>(ws, c->row_stats), 1, nullptr, st));
+    } else {
+        TRY(fused);
+    }
     c->k_last = k;
     c->verified = true;
     return SPEC_OK;
@@ -790,12 +802,18 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
         const float* nf = eagle ? at<const float>(dw, c->d_norm_f) : at<const float>(c->buf.weights, c->final_norm);
         const void* lm = eagle ? at<const void>(dw, c->d_lm_head) : at<const void>(c->buf.weights, c->lm_head);
         TRY(launch_rmsnorm(B, d, hid, nf, g.rms_eps, at(ws, c->h), d, 0, dt, st));
-        TRY(launch_gemm(B, Vd, d, at(ws, c->h), d, lm, dlog + (size_t)j * Vd, k * Vd, dt, SPEC_DTYPE_F32, 0, st));
+        spec_status fused = SPEC_ERR_UNSUPPORTED;
+        if (!g.draft_greedy)
+            fused = launch_gemm_lm_head_stats(B, Vd, d, at(ws, c->h), d, lm, dlog + (size_t)j * Vd, k * Vd, dt, g.temperature,
+                                              at<float>(ws, c->splitk), c->splitk.bytes, dstats + 2 * j, k, status, st);
+        if (fused == SPEC_ERR_UNSUPPORTED) TRY(launch_gemm(B, Vd, d, at(ws, c->h), d, lm, dlog + (size_t)j * Vd, k * Vd, dt, SPEC_DTYPE_F32, 0, st));
+        else TRY(fused);
         int32_t* tok_out = mapped ? dred + j : dtoks + j;          // reduced ids first when the head has its own vocabulary
         if (g.draft_greedy) {
             TRY(launch_argmax_rows(B, Vd, dlog + (size_t)j * Vd, (size_t)k * Vd, tok_out, kstride, st));
         } else {
-            TRY(launch_softmax_rows(B, Vd, dlog + (size_t)j * Vd, (size_t)k * Vd, g.temperature, dstats + 2 * j, k, nullptr, st));
+            if (fused == SPEC_ERR_UNSUPPORTED)
+                TRY(launch_softmax_rows(B, Vd, dlog + (size_t)j * Vd, (size_t)k * Vd, g.temperature, dstats + 2 * j, k, nullptr, st));
             TRY(launch_sample_logits(B, Vd, dlog + (size_t)j * Vd, (size_t)k * Vd, dstats + 2 * j, k, g.temperature, g.seed,
                                      at<uint32_t>(sb, c->step), (uint32_t)j, 1u, tok_out, kstride, status, st));
         }

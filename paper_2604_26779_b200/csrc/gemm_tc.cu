@@ -75,6 +75,10 @@ struct GemmArgs {
     // the activation rows its N operand (N = tokens <= bn, bn = 32 or 64: one narrow n-tile) - and the epilogue writes the
     // transposed tile, C[token][feature]
     int bn;
+    // plain epilogue with fp32 output (an LM head): every (row, 128-column piece) also leaves the pair (max, sum of
+    // exp((l - max) * inv_t)) of its logits in stat_part [rows][stat_pairs][2], piece index = 2 * n-tile + column half;
+    // a small kernel combines the pairs of a row, so the row statistics cost no second pass over the logits
+    float* stat_part; int stat_pairs; float inv_t;
 };
 
 enum { EPI_PLAIN = 0, EPI_SWIGLU = 1, EPI_QKV = 2, EPI_THIN = 3 };
@@ -178,6 +182,7 @@ __device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoor
     // resid (fp32 output added to what C holds, whole 32-column blocks): the residual block of the first 32 columns, loaded by the caller before it
     // waited for the accumulator; each later block is requested as soon as the previous one has been stored
     const int row0 = row - lane;                            // first row of this warp's 32
+    float sm = -INFINITY, sz = 0.f;                         // running (max, sum of exponentials) of this row's piece
 #pragma unroll 1
     for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
         const int col = tc.col + c0;
@@ -204,6 +209,14 @@ __device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoor
             continue;
         }
         tc_wait_ld();
+        if (g.stat_part != nullptr) {
+            float cm = -INFINITY;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) if (col + e < g.N) cm = fmaxf(cm, __uint_as_float(v[e]));
+            if (cm > sm) { sz *= __expf(__fmul_rn(__fsub_rn(sm, cm), g.inv_t)); sm = cm; }
+#pragma unroll
+            for (int e = 0; e < 32; ++e) if (col + e < g.N) sz += __expf(__fmul_rn(__fsub_rn(__uint_as_float(v[e]), sm), g.inv_t));
+        }
         if (g.out_f32 && col + 32 <= g.N) {                 // fp32: 32 columns = 128 bytes per row
 #pragma unroll
             for (int j = 0; j < 8; ++j) stage_put(stage, lane, j, make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]));
@@ -255,6 +268,10 @@ __device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoor
                     cp[j] = __float2bfloat16_rn(__uint_as_float(v[j]) + (g.accumulate ? __bfloat162float(cp[j]) : 0.f));
             }
         }
+    }
+    if (g.stat_part != nullptr && row_ok) {
+        float* sp = g.stat_part + ((size_t)row * g.stat_pairs + 2 * (tc.col / BN) + half) * 2;
+        sp[0] = sm; sp[1] = sz;
     }
 }
 
@@ -760,6 +777,59 @@ spec_status launch_gemm_tc_thin(int M, int N, int K, const void* A, int lda, con
         return launch_status();
     }
     return run_kernel(EPI_THIN, ma, mb, g, n_work, st);
+}
+
+// Row statistics from the pairs an LM-head launch left behind: (m, Z) with Z = sum_v exp((l_v - m) * inv_t), pairs merged in a
+// fixed order (each lane takes every 32nd pair in turn, then a shuffle tree).
+__global__ void __launch_bounds__(256) stat_combine_kernel(int rows, int pairs, const float* __restrict__ part, float inv_t,
+                                                           float* __restrict__ stats, size_t stats_stride)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    const float* p = part + (size_t)row * pairs * 2;
+    float m = -INFINITY, z = 0.f;
+    for (int i = lane; i < pairs; i += 32) {
+        const float pm = p[2 * i], pz = p[2 * i + 1];
+        if (pm > m) { z *= __expf(__fmul_rn(__fsub_rn(m, pm), inv_t)); m = pm; }
+        if (pm != -INFINITY) z += pz * __expf(__fmul_rn(__fsub_rn(pm, m), inv_t));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, o), oz = __shfl_xor_sync(0xffffffffu, z, o);
+        const float nm = fmaxf(m, om);
+        const float a = (m == -INFINITY) ? 0.f : z * __expf(__fmul_rn(__fsub_rn(m, nm), inv_t));
+        const float b = (om == -INFINITY) ? 0.f : oz * __expf(__fmul_rn(__fsub_rn(om, nm), inv_t));
+        // both lanes of a pair must form the same sum: add the lower lane's term first
+        z = (lane & o) ? b + a : a + b;
+        m = nm;
+    }
+    if (lane == 0) { stats[2 * (size_t)row * stats_stride] = m; stats[2 * (size_t)row * stats_stride + 1] = z; }
+}
+
+// LM head: logits [M][N] fp32 = A W^T and the row statistics (m, Z) of logits / temperature in stats [row * stats_stride][2],
+// the statistics taken in the GEMM epilogue.  part: scratch of at least M * 2 * ceil(N / 256) * 8 bytes.  Returns
+// SPEC_ERR_UNSUPPORTED (nothing launched) when the shape does not run on the tile kernel; the caller then takes the two-pass way.
+spec_status launch_gemm_lm_head_stats(int M, int N, int K, const void* A, int lda, const void* W, float* logits, int ldc, int dtype_in,
+                                      float temperature, float* part, size_t part_bytes, float* stats, size_t stats_stride,
+                                      int32_t* status, cudaStream_t st)
+{
+    if (M == 0 || N == 0) return SPEC_OK;
+    const int pairs = 2 * ((N + BN - 1) / BN);
+    if (M <= 64 || part == nullptr || (size_t)M * pairs * 8 > part_bytes ||
+        !gemm_tc_supported(M, N, K, A, lda, W, logits, ldc, dtype_in, SPEC_DTYPE_F32))
+        return SPEC_ERR_UNSUPPORTED;
+    if (!init_once()) return SPEC_ERR_CUDA;
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM)) return SPEC_ERR_CUDA;
+    if (!make_map(&mb, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
+    GemmArgs g{};
+    g.M = M; g.N = N; g.K = K; g.C = logits; g.ldc = ldc; g.out_f32 = 1; g.status = status;
+    g.stat_part = part; g.stat_pairs = pairs; g.inv_t = 1.0f / temperature;
+    TRY_LAUNCH(run_kernel(EPI_PLAIN, ma, mb, g, (long long)((M + BM - 1) / BM) * ((N + BN - 1) / BN), st));
+    launch_pdl(stat_combine_kernel, dim3((M + 7) / 8), dim3(256), 0, st, M, pairs, (const float*)part, g.inv_t, stats, stats_stride);
+    return launch_status();
 }
 
 // gate/up projection with the SwiGLU applied in the epilogue: W [2F][K] stored in 256-row groups (128 gate rows, then the

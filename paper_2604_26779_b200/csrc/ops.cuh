@@ -95,6 +95,9 @@ spec_status launch_gemm_skinny(int M, int N, int K, const void* A, int lda, cons
                                int accumulate, cudaStream_t st);
 // 17..64 rows: the tensor-core kernel with the operands swapped (weights as the M operand, one narrow tile of activation rows)
 bool gemm_tc_thin_supported(int M, int N, int K, const void* A, int lda, const void* W, const void* C, int ldc, int dtype_in, int out_dtype);
+spec_status launch_gemm_lm_head_stats(int M, int N, int K, const void* A, int lda, const void* W, float* logits, int ldc, int dtype_in,
+                                      float temperature, float* part, size_t part_bytes, float* stats, size_t stats_stride,
+                                      int32_t* status, cudaStream_t st);
 spec_status launch_gemm_grouped(int rows_total, int max_rows_per_group, int E, int N, int K, const void* A, const void* W,
                                 void* C, int out_dtype, int swiglu, const int32_t* counts, const int32_t* offsets,
                                 int32_t* status, cudaStream_t st);
