@@ -716,6 +716,7 @@ def main():
     wall = time.perf_counter() - t0
     wall, total_e2e = replicas.reduce_job(wall, float(total_e2e), dist, "cuda")
     line["e2e"] = {"value": total_e2e / wall, "unit": UNIT, "h2d_bytes_per_step": int(h2d / e2e_steps),
+                   "tokens": total_e2e, "seconds": wall,
                    "d2h_bytes_per_step": int(pinned_out.numel() * 4 + pinned_n.numel() * 4), "steps": e2e_steps,
                    "note": "host arrays -> spec_seq_init (H2D) + one plain decode step + steps, each with a D2H read of the emitted "
                            "tokens and a synchronize; every emitted token counted, the decode step's included; wall clock, max over ranks"}
