@@ -51,6 +51,8 @@ def lib():
         L.spec_oracle_kv_replace.argtypes = [c.c_int, i32p, i32p, c.c_int, c.c_int, i32p, i32p, i32p, i32p]
         L.spec_oracle_kv_replace.restype = c.c_int
         L.spec_oracle_e4m3_quantize.argtypes = [c.c_size_t, c.POINTER(c.c_float), c.c_float, c.POINTER(c.c_uint8)]
+        L.spec_oracle_e4m3_quantize_rows.argtypes = [c.c_size_t, c.c_size_t, c.POINTER(c.c_float), c.POINTER(c.c_float), c.POINTER(c.c_uint8)]
+        L.spec_oracle_e4m3_quantize_rows.restype = None
         L.spec_oracle_e4m3_dequantize.argtypes = [c.c_size_t, c.POINTER(c.c_uint8), c.c_float, c.POINTER(c.c_float)]
         _lib = L
     return _lib
@@ -205,6 +207,22 @@ def e4m3_quantize(x, scale=1.0):
     out = np.empty(xf.shape, np.uint8)
     lib().spec_oracle_e4m3_quantize(xf.size, _p(xf, ctypes.c_float), float(scale), _p(out, ctypes.c_uint8))
     return out
+
+
+def e4m3_quantize_rows(x):
+    """Per-row e4m3 codes and scales of a matrix [rows][k]: scale = amax(row) / 448 (1 for a zero row)."""
+    xf = _f32(x)
+    assert xf.ndim == 2
+    codes = np.empty(xf.shape, np.uint8)
+    scales = np.empty(xf.shape[0], np.float32)
+    lib().spec_oracle_e4m3_quantize_rows(xf.shape[0], xf.shape[1], _p(xf, ctypes.c_float), _p(scales, ctypes.c_float), _p(codes, ctypes.c_uint8))
+    return codes, scales
+
+
+def e4m3_rows_roundtrip(x):
+    """x with every row replaced by its 8-bit representation (codes times the row's scale), fp32."""
+    codes, scales = e4m3_quantize_rows(x)
+    return (e4m3_dequantize(codes, 1.0).reshape(codes.shape) * scales[:, None]).astype(np.float32)
 
 
 def e4m3_dequantize(codes, scale=1.0):

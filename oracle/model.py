@@ -82,8 +82,10 @@ def silu(x):
     return x / (1.0 + np.exp(-x))
 
 
-def dense_mlp(lw, m):
-    return (silu(m @ np.asarray(lw["wgate"], F64).T) * (m @ np.asarray(lw["wup"], F64).T)) @ np.asarray(lw["wdown"], F64).T
+def dense_mlp(lw, m, cfg=None):
+    if cfg is None or not cfg.get("w_fp8"):
+        return (silu(m @ np.asarray(lw["wgate"], F64).T) * (m @ np.asarray(lw["wup"], F64).T)) @ np.asarray(lw["wdown"], F64).T
+    return proj(cfg, silu(proj(cfg, m, lw["wgate"])) * proj(cfg, m, lw["wup"]), lw["wdown"])
 
 
 def moe_route(router_logits, top_k):
@@ -171,6 +173,25 @@ def ep_moe_mlp(lw, m_by_rank, top_k, ep_size, router_logits_by_rank=None):
     return out
 
 
+def _bf16_round(x):
+    """fp32 values rounded to bf16 (round to nearest even), as fp32."""
+    u = np.ascontiguousarray(x, np.float32).view(np.uint32)
+    r = ((u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)).view(np.float32)
+    return r
+
+
+def proj(cfg, x, W):
+    """x W^T of a target projection.  With cfg["w_fp8"] both operands go through the 8-bit format first (the precision the
+    paper's simulator assumes, Section 5.1): the activation rows as the 16-bit values the layer before produced, each row
+    of x and each row of W with its own scale amax / 448; the product itself is exact."""
+    if not cfg.get("w_fp8"):
+        return x @ np.asarray(W, F64).T
+    import oracle
+    xq = oracle.e4m3_rows_roundtrip(_bf16_round(np.asarray(x, np.float32))).astype(F64)
+    wq = oracle.e4m3_rows_roundtrip(np.asarray(W, np.float32)).astype(F64)
+    return xq @ wq.T
+
+
 def kv_as_cached(cfg, k, v):
     """What the attention reads back for freshly computed keys and values: themselves, or, with an 8-bit cache
     (cfg["kv_fp8"] = (k_scale, v_scale)), their e4m3 codes times the scale - for the new positions as for the old ones,
@@ -192,7 +213,7 @@ def decoder_layer(cfg, lw, x, pos, past_k=None, past_v=None, attn_in=None, route
     Hq, Hkv, dh = cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"]
     T = x.shape[0]
     h = rmsnorm(x, lw["attn_norm"], cfg["rms_eps"]) if attn_in is None else attn_in
-    qkv = h @ np.asarray(lw["wqkv"], F64).T
+    qkv = proj(cfg, h, lw["wqkv"])
     q = qkv[:, : Hq * dh].reshape(T, Hq, dh)
     k = qkv[:, Hq * dh : (Hq + Hkv) * dh].reshape(T, Hkv, dh)
     v = qkv[:, (Hq + Hkv) * dh :].reshape(T, Hkv, dh)
@@ -203,12 +224,12 @@ def decoder_layer(cfg, lw, x, pos, past_k=None, past_v=None, attn_in=None, route
     k_all = k if n_past == 0 else np.concatenate([np.asarray(past_k, F64), k], axis=0)
     v_all = v if n_past == 0 else np.concatenate([np.asarray(past_v, F64), v], axis=0)
     att = attention(q, k_all, v_all, n_past).reshape(T, Hq * dh)
-    x = x + att @ np.asarray(lw["wo"], F64).T
+    x = x + proj(cfg, att, lw["wo"])
     m = rmsnorm(x, lw["mlp_norm"], cfg["rms_eps"])
     if cfg.get("n_experts", 0) > 0:
         x = x + moe_mlp(lw, m, cfg["experts_top_k"], router_logits)
     else:
-        x = x + dense_mlp(lw, m)
+        x = x + dense_mlp(lw, m, cfg)
     return x, k, v
 
 
@@ -232,7 +253,7 @@ def target_forward(cfg, W, tokens, past=None, start_pos=0, tap_layers=(), router
         new_kv.append((k, v))
         if (l + 1) in tap_layers:
             taps[l + 1] = x
-    logits = rmsnorm(x, W["final_norm"], cfg["rms_eps"]) @ np.asarray(W["lm_head"], F64).T
+    logits = proj(cfg, rmsnorm(x, W["final_norm"], cfg["rms_eps"]), W["lm_head"])
     tap_cat = np.concatenate([taps[t] for t in tap_layers], axis=-1) if tap_layers else np.zeros((T, 0))
     return {"logits": logits, "taps": tap_cat, "final": x, "new_kv": new_kv}
 

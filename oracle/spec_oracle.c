@@ -343,6 +343,20 @@ void spec_oracle_e4m3_quantize(size_t n, const float* x, float scale, uint8_t* c
     for (size_t i = 0; i < n; ++i) codes[i] = e4m3_from_float(x[i] / scale);
 }
 
+/* 8-bit operands of a projection (the precision the paper's simulator assumes, Section 5.1): every row of a matrix gets
+ * its own scale, the largest magnitude of the row mapped to the largest e4m3 value, scale = amax / 448 in fp32 (1 for an
+ * all-zero row); code = round_e4m3(x / scale). */
+void spec_oracle_e4m3_quantize_rows(size_t rows, size_t k, const float* x, float* scales, uint8_t* codes)
+{
+    for (size_t r = 0; r < rows; ++r) {
+        float amax = 0.0f;
+        for (size_t i = 0; i < k; ++i) { const float a = fabsf(x[r * k + i]); if (a > amax) amax = a; }
+        const float sc = amax > 0.0f ? amax / 448.0f : 1.0f;
+        scales[r] = sc;
+        for (size_t i = 0; i < k; ++i) codes[r * k + i] = e4m3_from_float(x[r * k + i] / sc);
+    }
+}
+
 void spec_oracle_e4m3_dequantize(size_t n, const uint8_t* codes, float scale, float* x)
 {
     for (size_t i = 0; i < n; ++i) x[i] = e4m3_to_float(codes[i]) * scale;

@@ -262,3 +262,39 @@ def test_ep_moe_equals_unsharded_moe(ep_size):
         if ref.size:
             worst = max(worst, float(np.max(np.abs(got[s] - ref))))
     assert worst < 1e-12
+
+
+def test_e4m3_row_quantisation_hand_worked():
+    import oracle
+    x = np.array([[448.0, -224.0, 1.0, 0.0],          # amax 448: scale 1, the values are their own codes' values
+                  [1.0, 0.5, -0.25, 0.0],             # amax 1: scale 1/448; x / scale = 448, 224, -112: all exact e4m3 values
+                  [0.0, 0.0, 0.0, 0.0],               # zero row: scale 1, codes 0
+                  [3.0, 1.0, 0.1, -3.0]], np.float32)
+    codes, scales = oracle.e4m3_quantize_rows(x)
+    assert scales[0] == 1.0 and scales[1] == np.float32(1.0) / np.float32(448.0) and scales[2] == 1.0
+    assert scales[3] == np.float32(3.0) / np.float32(448.0)
+    back = oracle.e4m3_rows_roundtrip(x)
+    assert np.array_equal(back[0], x[0]) and np.array_equal(back[2], x[2])
+    assert np.allclose(back[1], x[1], rtol=1e-6, atol=0)
+    # a general row: every element within half an e4m3 step (2^-4 relative for normal values) of the original, the extreme exact
+    assert abs(back[3][0] - 3.0) < 1e-6 and abs(back[3][3] + 3.0) < 1e-6
+    assert abs(back[3][1] - 1.0) <= 1.0 * 2.0 ** -4 and abs(back[3][2] - 0.1) <= 0.1 * 2.0 ** -4
+    # the codes are those of the per-tensor routine called row by row with the row's scale
+    for r in range(4):
+        assert np.array_equal(codes[r], oracle.e4m3_quantize(x[r], float(scales[r])))
+
+
+def test_fp8_projection_error_is_what_the_format_allows():
+    # a random projection through the 8-bit path stays within the few-percent error two 4-bit-significand operands allow,
+    # and is exact when both operands are representable (powers of two)
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((5, 256)).astype(np.float32)
+    W = (rng.standard_normal((7, 256)) * 0.05).astype(np.float32)
+    ref = x.astype(np.float64) @ W.astype(np.float64).T
+    got = model.proj({"w_fp8": True}, x, W)
+    assert np.max(np.abs(got - ref)) / np.max(np.abs(ref)) < 0.06
+    assert np.max(np.abs(got - ref)) > 0
+    xp = np.ldexp(1.0, rng.integers(-3, 3, (4, 64))).astype(np.float32) * rng.choice([-1.0, 1.0], (4, 64)).astype(np.float32)
+    Wp = np.ldexp(1.0, rng.integers(-3, 3, (6, 64))).astype(np.float32)
+    assert np.array_equal(model.proj({"w_fp8": True}, xp, Wp), xp.astype(np.float64) @ Wp.astype(np.float64).T)
+    assert np.array_equal(model.proj({}, xp, Wp), xp.astype(np.float64) @ Wp.astype(np.float64).T)
