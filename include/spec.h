@@ -30,7 +30,7 @@
 extern "C" {
 #endif
 
-#define SPEC_ABI_VERSION 5u
+#define SPEC_ABI_VERSION 6u
 
 typedef struct spec_ctx spec_ctx; /* opaque */
 
@@ -52,6 +52,7 @@ typedef enum {
 
 enum { SPEC_DTYPE_BF16 = 0, SPEC_DTYPE_F32 = 1 };
 enum { SPEC_KV_MODEL = 0, SPEC_KV_E4M3 = 1 };
+enum { SPEC_W_MODEL = 0, SPEC_W_E4M3 = 1 };
 enum { SPEC_DRAFT_NONE = 0, SPEC_DRAFT_EAGLE3 = 1, SPEC_DRAFT_MTP = 2, SPEC_DRAFT_NGRAM = 3 };
 
 /* Model and run description.  n_experts = 0 selects the dense SwiGLU MLP. */
@@ -87,7 +88,12 @@ typedef struct {
                                 /* (the precision of the paper's deployment simulator, Section 5.1).  bf16 models with     */
                                 /* head_dim 128 and at most 16 query rows per KV head; a reduced-precision mode            */
     float kv_scale_k, kv_scale_v; /* > 0 with SPEC_KV_E4M3: one scale for all keys (after the rotary embedding), one for values */
-    int32_t reserved_;
+    int32_t weight_dtype;       /* SPEC_W_MODEL: the projections run in `dtype`; SPEC_W_E4M3: the target's QKV, O, gate/up, down  */
+                                /* and LM-head weights are stored as e4m3 codes with one fp32 scale per output row (the     */
+                                /* *_SCALE tensors; code = round_e4m3(w / scale), scale = amax(row) / 448), activations are */
+                                /* quantised the same way per row on the fly, and the products run on the 8-bit tensor-core */
+                                /* path with fp32 accumulation (the precision of the paper's simulator, Section 5.1).       */
+                                /* bf16 dense models, draft kind NONE / EAGLE3 / NGRAM; a reduced-precision mode            */
 } spec_config;
 
 /* Byte sizes of the caller-owned device arenas for a configuration. */
@@ -111,6 +117,8 @@ enum {
     SPEC_T_ROUTER,              /* [n_experts][d]                                                      */
     SPEC_T_EXPERTS_GATEUP,      /* [n_experts][2*d_expert_ffn][d], each expert grouped like WGATEUP    */
     SPEC_T_EXPERTS_DOWN,        /* [n_experts][d][d_expert_ffn]                                        */
+    /* SPEC_W_E4M3: fp32 [rows of the weight] scales; the weight tensors themselves then hold one byte per element */
+    SPEC_T_LM_HEAD_SCALE = 16, SPEC_T_WQKV_SCALE, SPEC_T_WO_SCALE, SPEC_T_WGATEUP_SCALE, SPEC_T_WDOWN_SCALE,
     /* draft head weights (arena `draft_weights`) */
     SPEC_T_D_WFC = 32,          /* EAGLE3: [d][n_taps*d]                                               */
     SPEC_T_D_WPROJ,             /* MTP: [d][2d] acting on concat(norm_g(g), norm_e(e))                 */
@@ -274,11 +282,22 @@ spec_status spec_reject_sample_logits(int B, int k, int V, const float* p_logits
 spec_status spec_uniforms(uint64_t seed, uint32_t step, uint32_t stream_tag, int n_seq, int n_slots, float* u,
                           void* stream);
 
+/* Per-row e4m3 quantisation of a bf16 matrix x [rows][K] (K % 16 == 0): scales [rows] = amax(row) / 448 (1 for a zero
+ * row), codes [rows][K] = round_e4m3(x / scale), round to nearest even, saturating.  What SPEC_W_E4M3 contexts expect in
+ * their weight tensors, and what they do to activations. */
+spec_status spec_quantize_rows(int rows, int K, const void* x_bf16, void* codes, float* scales, void* stream);
+
 /* C[M][N] = A[M][K] * W[N][K]^T (+ C when accumulate != 0).  dtype_in selects bf16 (tensor-core path, fp32
  * accumulation) or fp32 inputs; out_dtype the type of C.  All leading dimensions are the natural ones.
  * bf16 requires K % 64 == 0 and N % 8 == 0. */
 spec_status spec_gemm(int M, int N, int K, const void* A, const void* W, void* C, int dtype_in, int out_dtype,
                       int accumulate, void* stream);
+
+/* The same product with 8-bit operands: a8 [M][K] and w8 [N][K] e4m3 codes (as spec_quantize_rows writes them), a_scale
+ * [M] and w_scale [N] their row scales; C[m][n] (+)= a_scale[m] * w_scale[n] * sum_k a8[m][k] * w8[n][k], accumulated in
+ * fp32 on the 8-bit tensor-core path.  K % 16 == 0, N % 8 == 0; pointers 16-byte aligned. */
+spec_status spec_gemm_e4m3(int M, int N, int K, const void* a8, const float* a_scale, const void* w8, const float* w_scale,
+                           void* C, int out_dtype, int accumulate, void* stream);
 
 /* Paged attention of R = rows_per_seq query rows per sequence (query row i at position seq_len[b] + i sees
  * cache positions <= seq_len[b] + i), grouped-query heads.  q [B][R][Hq][dh], out the same shape and type;

@@ -12,9 +12,10 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libspec.so")
 
-SPEC_ABI_VERSION = 5
+SPEC_ABI_VERSION = 6
 SPEC_DTYPE_BF16, SPEC_DTYPE_F32 = 0, 1
 SPEC_KV_MODEL, SPEC_KV_E4M3 = 0, 1
+SPEC_W_MODEL, SPEC_W_E4M3 = 0, 1
 SPEC_DRAFT_NONE, SPEC_DRAFT_EAGLE3, SPEC_DRAFT_MTP, SPEC_DRAFT_NGRAM = 0, 1, 2, 3
 
 STATUS_NAMES = {0: "SPEC_OK", -1: "SPEC_ERR_INVALID_ARG", -2: "SPEC_ERR_SHAPE", -3: "SPEC_ERR_UNSUPPORTED",
@@ -24,7 +25,7 @@ STATUS_NAMES = {0: "SPEC_OK", -1: "SPEC_ERR_INVALID_ARG", -2: "SPEC_ERR_SHAPE", 
 
 # tensor ids (spec.h)
 T = dict(EMBED=0, LM_HEAD=1, FINAL_NORM=2, ATTN_NORM=3, WQKV=4, WO=5, MLP_NORM=6, WGATEUP=7, WDOWN=8, ROUTER=9,
-         EXPERTS_GATEUP=10, EXPERTS_DOWN=11,
+         EXPERTS_GATEUP=10, EXPERTS_DOWN=11, LM_HEAD_SCALE=16, WQKV_SCALE=17, WO_SCALE=18, WGATEUP_SCALE=19, WDOWN_SCALE=20,
          D_WFC=32, D_WPROJ=33, D_NORM_E=34, D_NORM_G=35, D_NORM_F=36, D_ATTN_NORM=37, D_WQKV=38, D_WO=39,
          D_MLP_NORM=40, D_WGATEUP=41, D_WDOWN=42, D_LM_HEAD=43, D_D2T=44,
          KV_K=64, KV_V=65, DRAFT_KV_K=66, DRAFT_KV_V=67,
@@ -50,7 +51,7 @@ class spec_config(C.Structure):
                 ("k_max", C.c_int32), ("max_batch", C.c_int32), ("kv_block_tokens", C.c_int32),
                 ("kv_num_blocks", C.c_int32), ("max_blocks_per_seq", C.c_int32), ("kv_layer_pools", C.c_int32),
                 ("temperature", C.c_float), ("seed", C.c_uint64), ("ngram_n", C.c_int32), ("draft_greedy", C.c_int32), ("draft_vocab", C.c_int32), ("kv_dtype", C.c_int32),
-                ("kv_scale_k", C.c_float), ("kv_scale_v", C.c_float), ("reserved_", C.c_int32)]
+                ("kv_scale_k", C.c_float), ("kv_scale_v", C.c_float), ("weight_dtype", C.c_int32)]
 
 
 class spec_sizes(C.Structure):
@@ -104,7 +105,9 @@ SIGNATURES = {
     "spec_reject_sample_probs": (_i, [_i, _i, _i, _vp, _vp, _vp, _u64, _u32, _vp, _vp, _vp, _vp]),
     "spec_reject_sample_logits": (_i, [_i, _i, _i, _vp, _vp, _vp, _vp, _vp, _f, _u64, _u32, _vp, _vp, _vp, _vp]),
     "spec_uniforms": (_i, [_u64, _u32, _u32, _i, _i, _vp, _vp]),
+    "spec_quantize_rows": (_i, [_i, _i, _vp, _vp, _vp, _vp]),
     "spec_gemm": (_i, [_i, _i, _i, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "spec_gemm_e4m3": (_i, [_i, _i, _i, _vp, _vp, _vp, _vp, _vp, _i, _i, _vp]),
     "spec_attention": (_i, [_i, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
     "spec_attention_scratch_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
     "spec_attention_noalloc": (_i, [_i, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp]),
@@ -199,6 +202,11 @@ def spec_uniforms(seed, step, stream_tag, u, stream=None):
     _check(lib().spec_uniforms(seed, step, stream_tag, n_seq, n_slots, _ptr(u), _stream(stream)), "spec_uniforms")
 
 
+def spec_quantize_rows(x, codes, scales, stream=None):
+    rows, K = x.shape
+    _check(lib().spec_quantize_rows(rows, K, _ptr(x), _ptr(codes), _ptr(scales), _stream(stream)), "spec_quantize_rows")
+
+
 def spec_gemm(A, W, Cout, accumulate=False, stream=None):
     import torch
     M, K = A.shape
@@ -207,6 +215,15 @@ def spec_gemm(A, W, Cout, accumulate=False, stream=None):
     dout = SPEC_DTYPE_F32 if Cout.dtype == torch.float32 else SPEC_DTYPE_BF16
     _check(lib().spec_gemm(M, N, K, _ptr(A), _ptr(W), _ptr(Cout), din, dout, int(accumulate), _stream(stream)),
            "spec_gemm")
+
+
+def spec_gemm_e4m3(a8, a_scale, w8, w_scale, Cout, accumulate=False, stream=None):
+    import torch
+    M, K = a8.shape
+    N = w8.shape[0]
+    out_dt = SPEC_DTYPE_BF16 if Cout.dtype == torch.bfloat16 else SPEC_DTYPE_F32
+    _check(lib().spec_gemm_e4m3(M, N, K, _ptr(a8), _ptr(a_scale), _ptr(w8), _ptr(w_scale), _ptr(Cout), out_dt, int(accumulate), _stream(stream)),
+           "spec_gemm_e4m3")
 
 
 def spec_attention_scratch_bytes(B, R, Hq, Hkv, dh, max_kv_len):

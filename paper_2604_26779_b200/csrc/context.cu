@@ -9,14 +9,14 @@
 
 struct Loc { size_t off = 0, bytes = 0; };
 
-struct LayerLoc { Loc attn_norm, wqkv, wo, mlp_norm, wgateup, wdown, router, exp_gateup, exp_down; };
+struct LayerLoc { Loc attn_norm, wqkv, wo, mlp_norm, wgateup, wdown, router, exp_gateup, exp_down, wqkv_s, wo_s, wgateup_s, wdown_s; };
 
 struct spec_ctx {
     spec_config cfg;
     spec_buffers buf;
     int Mmax;                       // max_batch * (k_max + 1)
     // weights
-    Loc embed, lm_head, final_norm;
+    Loc embed, lm_head, final_norm, lm_head_s;
     std::vector<LayerLoc> layers;
     size_t weights_bytes = 0;
     // draft weights
@@ -34,7 +34,7 @@ struct spec_ctx {
     Loc tokens_in, pos, x, h, qkv, attn_out, gu, act, logits, draft_logits, row_stats, draft_row_stats, taps,
         attn_scratch, dg, dx, d_hidden, d_tok, d_pos,
         moe_logits, moe_ids, moe_wts, moe_rank, moe_counts, moe_offsets, moe_inv, moe_a, moe_gu, moe_act, moe_out, rope, splitk,
-        t2d, draft_red;
+        t2d, draft_red, a8, a8_scale;
     size_t workspace_bytes = 0;
     // host-side run state
     int B = 0;
@@ -94,6 +94,11 @@ spec_status check_config(const spec_config* c)
     if (c->kv_dtype != SPEC_KV_MODEL && (c->kv_dtype != SPEC_KV_E4M3 || c->dtype != SPEC_DTYPE_BF16 || c->head_dim != 128 ||
                                          !(c->kv_scale_k > 0.f) || !(c->kv_scale_v > 0.f) ||
                                          (c->k_max + 1) * (c->n_q_heads / c->n_kv_heads) > 16)) return SPEC_ERR_UNSUPPORTED;
+    if (c->weight_dtype != SPEC_W_MODEL &&
+        (c->weight_dtype != SPEC_W_E4M3 || c->dtype != SPEC_DTYPE_BF16 || c->n_experts > 0 || c->draft_kind == SPEC_DRAFT_MTP ||
+         c->d_model % 128 != 0 || c->d_ffn % 128 != 0 || (c->n_q_heads * c->head_dim) % 128 != 0 || (c->head_dim != 64 && c->head_dim != 128) ||
+         c->vocab % 8 != 0))
+        return SPEC_ERR_UNSUPPORTED;
     if (c->draft_vocab != 0 && (c->draft_kind != SPEC_DRAFT_EAGLE3 || c->draft_vocab < 8 || c->draft_vocab > c->vocab ||
                                 c->draft_vocab % 8 != 0)) return SPEC_ERR_SHAPE;
     return SPEC_OK;
@@ -107,22 +112,27 @@ void build_layout(spec_ctx& x)
     x.Mmax = c.max_batch * (c.k_max + 1);
     {
         Arena a;
+        const bool w8 = c.weight_dtype == SPEC_W_E4M3;        // 8-bit projections: one byte per weight + one fp32 scale per row
+        const size_t ws = w8 ? 1 : es;
         x.embed = a.take((size_t)c.vocab * d * es);
-        x.lm_head = a.take((size_t)c.vocab * d * es);
+        x.lm_head = a.take((size_t)c.vocab * d * ws);
+        if (w8) x.lm_head_s = a.take((size_t)c.vocab * 4);
         x.final_norm = a.take(d * 4);
         x.layers.resize(c.n_layers);
         for (auto& L : x.layers) {
             L.attn_norm = a.take(d * 4);
-            L.wqkv = a.take(qkv_n * d * es);
-            L.wo = a.take(d * od * es);
+            L.wqkv = a.take(qkv_n * d * ws);
+            L.wo = a.take(d * od * ws);
+            if (w8) { L.wqkv_s = a.take(qkv_n * 4); L.wo_s = a.take(d * 4); }
             L.mlp_norm = a.take(d * 4);
             if (c.n_experts > 0) {
                 L.router = a.take((size_t)c.n_experts * d * es);
                 L.exp_gateup = a.take((size_t)c.n_experts * 2 * c.d_expert_ffn * d * es);
                 L.exp_down = a.take((size_t)c.n_experts * d * c.d_expert_ffn * es);
             } else {
-                L.wgateup = a.take((size_t)2 * c.d_ffn * d * es);
-                L.wdown = a.take(d * (size_t)c.d_ffn * es);
+                L.wgateup = a.take((size_t)2 * c.d_ffn * d * ws);
+                L.wdown = a.take(d * (size_t)c.d_ffn * ws);
+                if (w8) { L.wgateup_s = a.take((size_t)2 * c.d_ffn * 4); L.wdown_s = a.take(d * 4); }
             }
         }
         x.weights_bytes = a.top;
@@ -188,6 +198,11 @@ void build_layout(spec_ctx& x)
         x.attn_out = a.take(M * od * es);
         x.gu = a.take(M * 2 * Fmax * es);
         x.act = a.take(M * Fmax * es);
+        if (c.weight_dtype == SPEC_W_E4M3) {                  // activations as e4m3 codes + one scale per row, rewritten before every projection
+            const size_t kmax = (size_t)(c.d_ffn > (int)od ? c.d_ffn : od) > d ? (size_t)(c.d_ffn > (int)od ? c.d_ffn : od) : d;
+            x.a8 = a.take(M * kmax);
+            x.a8_scale = a.take(M * 4);
+        }
         x.logits = a.take(M * (size_t)c.vocab * 4);
         x.draft_logits = a.take(Bm * (size_t)(c.k_max > 0 ? c.k_max : 1) * c.vocab * 4);   // sized for the whole vocabulary
         if (c.draft_vocab) {
@@ -227,14 +242,17 @@ void build_layout(spec_ctx& x)
 template <class T = void> T* at(void* base, const Loc& l) { return reinterpret_cast<T*>(static_cast<char*>(base) + l.off); }
 
 struct LayerPtrs { const float* attn_norm; const void* wqkv; const void* wo; const float* mlp_norm; const void* wgateup; const void* wdown;
-                   const void* router; const void* exp_gateup; const void* exp_down; };
+                   const void* router; const void* exp_gateup; const void* exp_down;
+                   const float* wqkv_s; const float* wo_s; const float* wgateup_s; const float* wdown_s; };   // 8-bit weights: row scales
 
 LayerPtrs layer_ptrs(void* base, const LayerLoc& L)
 {
     return {at<const float>(base, L.attn_norm), at<const void>(base, L.wqkv), at<const void>(base, L.wo),
             at<const float>(base, L.mlp_norm), at<const void>(base, L.wgateup), at<const void>(base, L.wdown),
             L.router.bytes ? at<const void>(base, L.router) : nullptr, at<const void>(base, L.exp_gateup),
-            at<const void>(base, L.exp_down)};
+            at<const void>(base, L.exp_down),
+            L.wqkv_s.bytes ? at<const float>(base, L.wqkv_s) : nullptr, L.wo_s.bytes ? at<const float>(base, L.wo_s) : nullptr,
+            L.wgateup_s.bytes ? at<const float>(base, L.wgateup_s) : nullptr, L.wdown_s.bytes ? at<const float>(base, L.wdown_s) : nullptr};
 }
 
 #define TRY(expr) do { spec_status s__ = (expr); if (s__ != SPEC_OK) return s__; } while (0)
@@ -428,6 +446,14 @@ extern "C" spec_status spec_tensor(spec_ctx* c, int id, int layer, void** dev_pt
         l = id == SPEC_T_ATTN_NORM ? L.attn_norm : id == SPEC_T_WQKV ? L.wqkv : id == SPEC_T_WO ? L.wo :
             id == SPEC_T_MLP_NORM ? L.mlp_norm : id == SPEC_T_WGATEUP ? L.wgateup : id == SPEC_T_WDOWN ? L.wdown :
             id == SPEC_T_ROUTER ? L.router : id == SPEC_T_EXPERTS_GATEUP ? L.exp_gateup : L.exp_down;
+        break;
+    }
+    case SPEC_T_LM_HEAD_SCALE: base = c->buf.weights; l = c->lm_head_s; break;
+    case SPEC_T_WQKV_SCALE: case SPEC_T_WO_SCALE: case SPEC_T_WGATEUP_SCALE: case SPEC_T_WDOWN_SCALE: {
+        if (!layer_ok()) return SPEC_ERR_INVALID_ARG;
+        const LayerLoc& L = c->layers[layer];
+        base = c->buf.weights;
+        l = id == SPEC_T_WQKV_SCALE ? L.wqkv_s : id == SPEC_T_WO_SCALE ? L.wo_s : id == SPEC_T_WGATEUP_SCALE ? L.wgateup_s : L.wdown_s;
         break;
     }
     case SPEC_T_D_WFC: base = c->buf.draft_weights; l = c->d_wfc; break;

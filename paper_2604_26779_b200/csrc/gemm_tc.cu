@@ -51,6 +51,8 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr)
 }
 // Instruction descriptor: D fp32, A and B bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// The same for e4m3 operands (format code 0 for A and B).
+constexpr uint32_t kIdescF8 = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 struct TileCoord { int a_row, b_row, c_row, rows_valid, col, kb0, kb1, split; };
 
@@ -79,6 +81,10 @@ struct GemmArgs {
     // exp((l - max) * inv_t)) of its logits in stat_part [rows][stat_pairs][2], piece index = 2 * n-tile + column half;
     // a small kernel combines the pairs of a row, so the row statistics cost no second pass over the logits
     float* stat_part; int stat_pairs; float inv_t;
+    // 8-bit operands (fp8 != 0): A and W hold e4m3 codes, one byte per element, a k-block is 128 elements (the same 128 bytes
+    // per row as 64 bf16), K counts byte PAIRS of a row (elements / 2) so that the k-block arithmetic is unchanged, and every
+    // accumulator is multiplied by a_scale[row] * w_scale[weight row] before the epilogue does anything else with it
+    int fp8; const float* a_scale; const float* w_scale;
 };
 
 enum { EPI_PLAIN = 0, EPI_SWIGLU = 1, EPI_QKV = 2, EPI_THIN = 3 };
@@ -175,6 +181,26 @@ __device__ __forceinline__ void stage_flush(uint32_t stage, int lane, unsigned c
     stage_flush<false>(stage, lane, dst, row_stride_bytes, rows_ok, none);
 }
 
+// 8-bit operands: accumulator columns [w0, w0 + 32) of this thread's row times the row's activation scale and the weight
+// rows' scales (weight rows past n_w get 0).
+__device__ __forceinline__ void scale32(const GemmArgs& g, uint32_t (&v)[32], float row_scale, int w0, int n_w)
+{
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        float4 ws = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (w0 + 4 * j + 3 < n_w) ws = __ldg(reinterpret_cast<const float4*>(g.w_scale + w0) + j);
+        else {
+            if (w0 + 4 * j < n_w) ws.x = g.w_scale[w0 + 4 * j];
+            if (w0 + 4 * j + 1 < n_w) ws.y = g.w_scale[w0 + 4 * j + 1];
+            if (w0 + 4 * j + 2 < n_w) ws.z = g.w_scale[w0 + 4 * j + 2];
+        }
+        v[4 * j] = __float_as_uint(__uint_as_float(v[4 * j]) * (row_scale * ws.x));
+        v[4 * j + 1] = __float_as_uint(__uint_as_float(v[4 * j + 1]) * (row_scale * ws.y));
+        v[4 * j + 2] = __float_as_uint(__uint_as_float(v[4 * j + 2]) * (row_scale * ws.z));
+        v[4 * j + 3] = __float_as_uint(__uint_as_float(v[4 * j + 3]) * (row_scale * ws.w));
+    }
+}
+
 // Plain epilogue: C (+)= accumulator, fp32 or bf16, ragged N handled element-wise.
 __device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoord& tc, uint32_t t_row, int row, bool row_ok, int half,
                                                uint32_t stage, int lane, int rows_ok, uint4 (&resid)[8])
@@ -193,6 +219,7 @@ __device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoor
             uint32_t v2[32];
             tc_ld32(t_row + c0 + 32, v2);
             tc_wait_ld();
+            if (g.fp8) { const float rs = row_ok ? g.a_scale[row] : 0.f; scale32(g, v, rs, col, g.N); scale32(g, v2, rs, col + 32, g.N); }
             float f[8];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -209,6 +236,7 @@ __device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoor
             continue;
         }
         tc_wait_ld();
+        if (g.fp8) scale32(g, v, row_ok ? g.a_scale[row] : 0.f, col, g.N);
         if (g.stat_part != nullptr) {
             float cm = -INFINITY;
 #pragma unroll
@@ -289,6 +317,11 @@ __device__ __forceinline__ void epilogue_swiglu(const GemmArgs& g, const TileCoo
         tc_ld32(t_row + c0, gv);
         tc_ld32(t_row + BN / 2 + c0, uv);
         tc_wait_ld();
+        if (g.fp8) {
+            const float rs = row_ok ? g.a_scale[row] : 0.f;
+            scale32(g, gv, rs, tc.b_row + c0, 0x7fffffff);
+            scale32(g, uv, rs, tc.b_row + BN / 2 + c0, 0x7fffffff);
+        }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             float f[8];
@@ -340,6 +373,11 @@ __device__ __forceinline__ void epilogue_qkv(const GemmArgs& g, const TileCoord&
             tc_ld32(t_row + hb + j0, lo);
             tc_ld32(t_row + hb + half + j0, hi);
             tc_wait_ld();
+            if (g.fp8) {
+                const float rs = row_ok ? g.a_scale[row] : 0.f;
+                scale32(g, lo, rs, col + j0, g.N);
+                scale32(g, hi, rs, col + half + j0, g.N);
+            }
             float a[32], b[32];
             if (is_k) {                                                  // q and k heads: rotary embedding
 #pragma unroll
@@ -501,8 +539,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
                     if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t bar = smem_u32(&ctl->full[s]);
                     mbar_expect_tx(bar, EPI == EPI_THIN ? (uint32_t)(A_BYTES + g.bn * BK * 2) : (uint32_t)STAGE_BYTES);
-                    tma_load_2d(tiles + s * STAGE_BYTES, &map_a, kb * BK, tc.a_row, bar);
-                    tma_load_2d(tiles + s * STAGE_BYTES + A_BYTES, &map_b, kb * BK, tc.b_row, bar);
+                    const int kx = g.fp8 ? kb * BK * 2 : kb * BK;               // first element of the k-block (8-bit: 128 per block)
+                    tma_load_2d(tiles + s * STAGE_BYTES, &map_a, kx, tc.a_row, bar);
+                    tma_load_2d(tiles + s * STAGE_BYTES + A_BYTES, &map_b, kx, tc.b_row, bar);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
@@ -518,7 +557,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             bool ok = true;
             int it = 0;
             // instruction descriptor; the thin variant's n extent is the activation tile (32 or 64 rows)
-            const uint32_t idesc = EPI == EPI_THIN ? ((kIdesc & ~(0x3fu << 17)) | ((uint32_t)(g.bn >> 3) << 17)) : kIdesc;
+            const uint32_t idesc = EPI == EPI_THIN ? ((kIdesc & ~(0x3fu << 17)) | ((uint32_t)(g.bn >> 3) << 17)) : g.fp8 ? kIdescF8 : kIdesc;
             for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
                 TileCoord tc;
                 if (!tile_coord(g, w, m_tiles, n_tiles, pref, tc)) continue;
@@ -533,7 +572,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
                     const uint32_t sa = tiles + s * STAGE_BYTES, sb = sa + A_BYTES;
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k)
-                        tc_mma(d_tmem, smem_desc(sa + k * UMMA_K * 2), smem_desc(sb + k * UMMA_K * 2), idesc, (kb > tc.kb0 || k > 0) ? 1u : 0u);
+                        if (g.fp8) tc_mma_f8(d_tmem, smem_desc(sa + k * UMMA_K * 2), smem_desc(sb + k * UMMA_K * 2), idesc, (kb > tc.kb0 || k > 0) ? 1u : 0u);
+                        else tc_mma(d_tmem, smem_desc(sa + k * UMMA_K * 2), smem_desc(sb + k * UMMA_K * 2), idesc, (kb > tc.kb0 || k > 0) ? 1u : 0u);
                     tc_commit(smem_u32(&ctl->empty[s]));            // stage reusable once these MMAs have read it
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -664,6 +704,9 @@ spec_status run_kernel(int epi, const CUtensorMap& ma, const CUtensorMap& mb, co
     return launch_status();
 }
 
+// 2-D map over a row-major [rows][cols] matrix of e4m3 codes (bytes) with row pitch ld bytes; box = 128 columns x box_rows rows:
+// the same 128-byte-wide, 128B-swizzled tile in shared memory as 64 bf16 columns.
+bool make_map8(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows);
 // 2-D map over a row-major [rows][cols] bf16 matrix with row pitch ld elements; box = 64 columns x box_rows rows.
 bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows)
 {
@@ -672,6 +715,17 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, u
     const cuuint32_t box[2] = {BK, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool make_map8(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows)
+{
+    const cuuint64_t gdim[2] = {cols, rows};
+    const cuuint64_t gstride[1] = {ld};
+    const cuuint32_t box[2] = {2 * BK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -866,6 +920,76 @@ spec_status launch_gemm_qkv_tc(int M, int K, const void* A, int lda, const void*
     return run_kernel(EPI_QKV, ma, mb, g, (long long)((M + BM - 1) / BM) * ((N + BN - 1) / BN), st);
 }
 
+// ---- 8-bit (e4m3) operands: A [M][K] and W [N][K] are codes with one fp32 scale per row; K % 16 == 0 ------------------
+namespace {
+bool fp8_ok(int K, const void* a8, const void* w8) { return K % 16 == 0 && ((reinterpret_cast<uintptr_t>(a8) | reinterpret_cast<uintptr_t>(w8)) & 15u) == 0; }
+void fp8_args(GemmArgs& g, int M, int N, int K, const float* a_scale, const float* w_scale, int32_t* status)
+{
+    g.M = M; g.N = N; g.K = K / 2;                          // K in byte pairs: ceil(g.K / 64) = ceil(K / 128) k-blocks
+    g.status = status; g.fp8 = 1; g.a_scale = a_scale; g.w_scale = w_scale;
+}
+}  // namespace
+
+// C (+)= (A W^T) scaled; with part != nullptr (fp32 logits) the row statistics go to stats as in launch_gemm_lm_head_stats.
+spec_status launch_gemm8_tc(int M, int N, int K, const void* a8, const float* a_scale, const void* w8, const float* w_scale, void* C, int ldc,
+                            int out_dtype, int accumulate, float temperature, float* part, size_t part_bytes, float* stats,
+                            size_t stats_stride, int32_t* status, cudaStream_t st)
+{
+    if (M == 0 || N == 0) return SPEC_OK;
+    if (!fp8_ok(K, a8, w8)) return SPEC_ERR_SHAPE;
+    if (!init_once()) return SPEC_ERR_CUDA;
+    CUtensorMap ma, mb;
+    if (!make_map8(&ma, a8, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM)) return SPEC_ERR_CUDA;
+    if (!make_map8(&mb, w8, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
+    GemmArgs g{};
+    fp8_args(g, M, N, K, a_scale, w_scale, status);
+    g.C = C; g.ldc = ldc; g.out_f32 = out_dtype == SPEC_DTYPE_F32 ? 1 : 0; g.accumulate = accumulate;
+    const int pairs = 2 * ((N + BN - 1) / BN);
+    const bool with_stats = part != nullptr && g.out_f32 && (size_t)M * pairs * 8 <= part_bytes;
+    if (with_stats) { g.stat_part = part; g.stat_pairs = pairs; g.inv_t = 1.0f / temperature; }
+    TRY_LAUNCH(run_kernel(EPI_PLAIN, ma, mb, g, (long long)((M + BM - 1) / BM) * ((N + BN - 1) / BN), st));
+    if (with_stats) {
+        launch_pdl(stat_combine_kernel, dim3((M + 7) / 8), dim3(256), 0, st, M, pairs, (const float*)part, g.inv_t, stats, stats_stride);
+        return launch_status();
+    }
+    return part != nullptr ? SPEC_ERR_UNSUPPORTED : SPEC_OK;   // statistics wanted but the scratch is too small: the caller falls back
+}
+
+spec_status launch_gemm8_swiglu_tc(int M, int F, int K, const void* a8, const float* a_scale, const void* w8, const float* w_scale, void* act,
+                                   int32_t* status, cudaStream_t st)
+{
+    if (M == 0 || F == 0) return SPEC_OK;
+    if (!fp8_ok(K, a8, w8)) return SPEC_ERR_SHAPE;
+    if (!init_once()) return SPEC_ERR_CUDA;
+    CUtensorMap ma, mb;
+    if (!make_map8(&ma, a8, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM)) return SPEC_ERR_CUDA;
+    if (!make_map8(&mb, w8, (uint64_t)2 * F, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
+    GemmArgs g{};
+    fp8_args(g, M, 2 * F, K, a_scale, w_scale, status);
+    g.C = act; g.ldc = F;
+    return run_kernel(EPI_SWIGLU, ma, mb, g, (long long)((M + BM - 1) / BM) * (2 * F / BN), st);
+}
+
+spec_status launch_gemm8_qkv_tc(int M, int K, const void* a8, const float* a_scale, const void* w8, const float* w_scale, void* qkv,
+                                const QkvEpilogue& e, int32_t* status, cudaStream_t st)
+{
+    const int N = (e.Hq + 2 * e.Hkv) * e.dh;
+    if (M == 0) return SPEC_OK;
+    if (!fp8_ok(K, a8, w8)) return SPEC_ERR_SHAPE;
+    if (!init_once()) return SPEC_ERR_CUDA;
+    CUtensorMap ma, mb;
+    if (!make_map8(&ma, a8, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM)) return SPEC_ERR_CUDA;
+    if (!make_map8(&mb, w8, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
+    GemmArgs g{};
+    fp8_args(g, M, N, K, a_scale, w_scale, status);
+    g.C = qkv; g.ldc = N;
+    g.Hq = e.Hq; g.Hkv = e.Hkv; g.dh = e.dh; g.R = e.R; g.max_blocks = e.max_blocks; g.block_tokens = e.block_tokens;
+    g.pos = e.pos; g.block_table = e.block_table; g.rope = reinterpret_cast<const float2*>(e.rope);
+    g.k_pool = static_cast<__nv_bfloat16*>(e.k_pool); g.v_pool = static_cast<__nv_bfloat16*>(e.v_pool);
+    g.kv_fp8 = e.kv_fp8; g.k_scale = e.k_scale; g.v_scale = e.v_scale;
+    return run_kernel(EPI_QKV, ma, mb, g, (long long)((M + BM - 1) / BM) * ((N + BN - 1) / BN), st);
+}
+
 // Grouped form: A [rows_total][K] holds the groups' rows back to back (group e at offsets[e], counts[e] rows, both on
 // the device; no group has more than max_rows_per_group rows), W [E][N][K], C [rows_total][N].  N % 256 == 0.
 spec_status launch_gemm_grouped(int rows_total, int max_rows_per_group, int E, int N, int K, const void* A, const void* W,
@@ -912,4 +1036,15 @@ extern "C" spec_status spec_gemm(int M, int N, int K, const void* A, const void*
     if (M == 0 || N == 0) return SPEC_OK;
     if (!A || !W || !C) return SPEC_ERR_INVALID_ARG;
     return spec::launch_gemm(M, N, K, A, K, W, C, N, dtype_in, out_dtype, accumulate, (cudaStream_t)stream);
+}
+
+extern "C" spec_status spec_gemm_e4m3(int M, int N, int K, const void* a8, const float* a_scale, const void* w8, const float* w_scale,
+                                      void* C, int out_dtype, int accumulate, void* stream)
+{
+    if (M < 0 || N < 0 || K <= 0) return SPEC_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return SPEC_OK;
+    if (!a8 || !a_scale || !w8 || !w_scale || !C) return SPEC_ERR_INVALID_ARG;
+    if (N % 8 != 0 || (reinterpret_cast<uintptr_t>(C) & 15u) != 0) return SPEC_ERR_SHAPE;
+    return spec::launch_gemm8_tc(M, N, K, a8, a_scale, w8, w_scale, C, N, out_dtype, accumulate, 1.0f, nullptr, 0, nullptr, 0, nullptr,
+                                 (cudaStream_t)stream);
 }

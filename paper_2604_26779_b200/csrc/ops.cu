@@ -497,6 +497,52 @@ __global__ void __launch_bounds__(256) permute_rows_kernel(int R, size_t row_byt
     for (size_t c = threadIdx.x; c < row_bytes / 16; c += blockDim.x) d4[c] = s4[c];
 }
 
+// Per-row e4m3 quantisation of a bf16 matrix: one CTA per row.  scale = amax / 448 in fp32 (1 for a zero row), codes =
+// round_e4m3(x / scale) with an exact fp32 division, round to nearest even, saturating: the same steps as the oracle's.
+__global__ void __launch_bounds__(256) quantize_rows_kernel(int K, const __nv_bfloat16* __restrict__ x, unsigned char* __restrict__ codes,
+                                                            float* __restrict__ scales)
+{
+    pdl_trigger();
+    pdl_wait();
+    __shared__ float s_w[8];
+    __shared__ float s_scale;
+    const int row = blockIdx.x;
+    const __nv_bfloat16* xr = x + (size_t)row * K;
+    float amax = 0.f;
+    for (int i = threadIdx.x * 8; i < K; i += 256 * 8) {
+        const uint4 v = *reinterpret_cast<const uint4*>(xr + i);
+        const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) amax = fmaxf(amax, fmaxf(fabsf(__low2float(p[e])), fabsf(__high2float(p[e]))));
+    }
+    amax = warp_max(amax);
+    if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float m = s_w[0];
+        for (int w = 1; w < 8; ++w) m = fmaxf(m, s_w[w]);
+        const float sc = m > 0.f ? __fdiv_rn(m, 448.f) : 1.f;
+        s_scale = sc;
+        scales[row] = sc;
+    }
+    __syncthreads();
+    const float sc = s_scale;
+    unsigned char* cr = codes + (size_t)row * K;
+    for (int i = threadIdx.x * 8; i < K; i += 256 * 8) {
+        const uint4 v = *reinterpret_cast<const uint4*>(xr + i);
+        const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+        uint32_t w[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            unsigned short lo, hi;                           // cvt packs its first source into the upper byte
+            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(__fdiv_rn(__high2float(p[2 * h]), sc)), "f"(__fdiv_rn(__low2float(p[2 * h]), sc)));
+            asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(__fdiv_rn(__high2float(p[2 * h + 1]), sc)), "f"(__fdiv_rn(__low2float(p[2 * h + 1]), sc)));
+            w[h] = (uint32_t)lo | ((uint32_t)hi << 16);
+        }
+        *reinterpret_cast<uint2*>(cr + i) = make_uint2(w[0], w[1]);
+    }
+}
+
 }  // namespace
 
 #define DISPATCH_T(dtype, ...)                                            \
@@ -617,6 +663,14 @@ spec_status launch_permute_rows(int n_keep, int R, size_t row_bytes, const int32
     return launch_status();
 }
 
+spec_status launch_quantize_rows(int rows, int K, const void* x_bf16, void* codes, float* scales, cudaStream_t st)
+{
+    if (rows == 0) return SPEC_OK;
+    if (K <= 0 || K % 8 != 0) return SPEC_ERR_SHAPE;
+    launch_pdl(quantize_rows_kernel, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales);
+    return launch_status();
+}
+
 spec_status launch_kv_commit(const CommitArgs& a, cudaStream_t st)
 {
     if (a.B == 0) return SPEC_OK;
@@ -625,3 +679,11 @@ spec_status launch_kv_commit(const CommitArgs& a, cudaStream_t st)
 }
 
 }  // namespace spec
+
+extern "C" spec_status spec_quantize_rows(int rows, int K, const void* x_bf16, void* codes, float* scales, void* stream)
+{
+    if (rows < 0 || K <= 0) return SPEC_ERR_INVALID_ARG;
+    if (rows == 0) return SPEC_OK;
+    if (!x_bf16 || !codes || !scales) return SPEC_ERR_INVALID_ARG;
+    return spec::launch_quantize_rows(rows, K, x_bf16, codes, scales, (cudaStream_t)stream);
+}

@@ -44,6 +44,7 @@ spec_status launch_rope_append(int B, int R, int Hq, int Hkv, int dh, float thet
                                void* k_pool, void* v_pool, const int32_t* block_table, int max_blocks,
                                int block_tokens, int dtype, cudaStream_t st, const float* rope_table = nullptr);   // rope_table: [dh/2][B*R] (cos, sin) of pos, or NULL
 spec_status launch_swiglu(int M, int F, const void* gate_up, void* out, int dtype, cudaStream_t st);
+spec_status launch_quantize_rows(int rows, int K, const void* x_bf16, void* codes, float* scales, cudaStream_t st);
 spec_status launch_copy_rows_f32_to(int M, int d, const float* x, void* out, int ld_out, int col0, int dtype,
                                     cudaStream_t st);
 // dst[b] = src[b*R + idx[b]-1] rows of width d (fp32); idx = rows valid per sequence
@@ -89,6 +90,12 @@ spec_status launch_gemm(int M, int N, int K, const void* A, int lda, const void*
                         int out_dtype, int accumulate, cudaStream_t st);
 
 // swiglu != 0: W holds [2F] rows per group in 256-row gate/up groups and C is the activation [rows][N/2] (bf16)
+// 8-bit (e4m3) operands with per-row scales: plain (optionally with the LM head's row statistics), SwiGLU and QKV epilogues
+spec_status launch_gemm8_tc(int M, int N, int K, const void* a8, const float* a_scale, const void* w8, const float* w_scale, void* C, int ldc,
+                            int out_dtype, int accumulate, float temperature, float* part, size_t part_bytes, float* stats,
+                            size_t stats_stride, int32_t* status, cudaStream_t st);
+spec_status launch_gemm8_swiglu_tc(int M, int F, int K, const void* a8, const float* a_scale, const void* w8, const float* w_scale, void* act,
+                                   int32_t* status, cudaStream_t st);
 // very few rows (M <= 16): the weights are the MMA's M operand, one CTA per 32 weight rows (gemm_skinny.cu)
 bool gemm_skinny_supported(int M, int N, int K, const void* A, int lda, const void* W, int dtype_in);
 spec_status launch_gemm_skinny(int M, int N, int K, const void* A, int lda, const void* W, void* C, int ldc, int out_dtype,
@@ -117,6 +124,8 @@ struct QkvEpilogue {
 };
 spec_status launch_gemm_qkv_tc(int M, int K, const void* A, int lda, const void* W, void* qkv, const QkvEpilogue& e,
                                int32_t* status, cudaStream_t st);
+spec_status launch_gemm8_qkv_tc(int M, int K, const void* a8, const float* a_scale, const void* w8, const float* w_scale, void* qkv,
+                                const QkvEpilogue& e, int32_t* status, cudaStream_t st);
 // (cos, sin) table of the rows' positions for the fused QKV epilogue
 spec_status launch_rope_table(int M, int dh, float theta, const int32_t* pos, float* table, cudaStream_t st);
 

@@ -148,3 +148,37 @@ def test_bounded_wait_times_out_cleanly(api):
     api.spec_gemm(A, W, Cc)
     torch.cuda.synchronize()
     assert torch.allclose(Cc, A.float() @ W.float().t(), atol=1e-2, rtol=1e-3)
+
+
+@pytest.mark.parametrize("M,N,K,dout,acc", [
+    (128, 256, 128, torch.float32, False),             # one tile, one k-block
+    (1024, 4096, 4096, torch.bfloat16, False),
+    (300, 1000, 14336, torch.float32, True),           # ragged M and N, long K
+    (64, 512, 272, torch.float32, False),              # K not a multiple of the 128-element k-block
+])
+def test_gemm_e4m3_matches_oracle(api, M, N, K, dout, acc):
+    """8-bit projection: the row quantiser's codes and scales equal the oracle's bit for bit (same bf16 inputs), and the
+    product of the codes - exact integer-like arithmetic in fp32 accumulation - matches the oracle's fp64 product of the
+    dequantised operands to fp32 rounding."""
+    import oracle
+    A = inputs.round_to_bf16(inputs.make_kv_values((M, K), 11, "bf16"))
+    W = inputs.round_to_bf16(inputs.make_kv_values((N, K), 12, "bf16") * np.float32(0.05))
+    C0 = inputs.make_kv_values((M, N), 13, "bf16" if dout == torch.bfloat16 else "f32")
+    dA, dW = torch.from_numpy(A).cuda().to(torch.bfloat16), torch.from_numpy(W).cuda().to(torch.bfloat16)
+    a8, w8 = torch.empty((M, K), dtype=torch.uint8, device="cuda"), torch.empty((N, K), dtype=torch.uint8, device="cuda")
+    sa, sw = torch.empty(M, dtype=torch.float32, device="cuda"), torch.empty(N, dtype=torch.float32, device="cuda")
+    api.spec_quantize_rows(dA, a8, sa)
+    api.spec_quantize_rows(dW, w8, sw)
+    oa, osa = oracle.e4m3_quantize_rows(A)
+    ow, osw = oracle.e4m3_quantize_rows(W)
+    assert np.array_equal(a8.cpu().numpy(), oa) and np.array_equal(sa.cpu().numpy(), osa)
+    assert np.array_equal(w8.cpu().numpy(), ow) and np.array_equal(sw.cpu().numpy(), osw)
+    dC = torch.from_numpy(C0).cuda().to(dout)
+    api.spec_gemm_e4m3(a8, sa, w8, sw, dC, accumulate=acc)
+    torch.cuda.synchronize()
+    rows = np.arange(M) if M <= 300 else np.unique(np.concatenate([np.arange(0, M, 37), [M - 1, 127, 128]]))
+    ref = model.proj({"w_fp8": True}, A[rows], W) + (C0[rows].astype(np.float64) if acc else 0.0)
+    got = dC.float().cpu().numpy()[rows]
+    err = np.abs(got - ref).max(-1) / np.abs(ref).max(-1)
+    print(f"e4m3 gemm {M}x{N}x{K} ->{dout} acc={acc}: worst row error {err.max():.2e}")
+    assert err.max() < (1e-2 if dout == torch.bfloat16 else 1e-5)
