@@ -439,6 +439,9 @@ def main():
     ap.add_argument("--kv-fp8", action="store_true",
                     help="c3 only: 8-bit (e4m3) KV cache, scales 1/16 - a reduced-precision variant, reported under its own "
                          "metric name and never the headline")
+    ap.add_argument("--w-fp8", action="store_true",
+                    help="c3 only: the target's projections and LM head in 8-bit (e4m3) with one scale per weight row and per "
+                         "activation row - a reduced-precision variant, reported under its own metric name and never the headline")
     ap.add_argument("--k-sweep", default=None,
                     help="comma-separated draft lengths, e.g. 1,3,5,7: times the c3 step at each k on one engine built for the "
                          "largest (not the headline run: prints its own JSON line)")
@@ -487,7 +490,8 @@ def main():
                                                    steps_budget=steps_budget, device=f"cuda:{local}",
                                                    seed=replicas.replica_seed(rank),
                                                    cfg_over=dict(**(dict(draft_vocab=args.draft_vocab) if args.draft_vocab else {}),
-                                                                 **(dict(kv_fp8=(0.0625, 0.0625)) if args.kv_fp8 else {})) or None)
+                                                                 **(dict(kv_fp8=(0.0625, 0.0625)) if args.kv_fp8 else {}),
+                                                                 **(dict(w_fp8=True) if args.w_fp8 else {})) or None)
         wl_name = ("c3: 8B dense verify (32 layers, d=4096, 32q/8kv, dh=128, FFN 14336, V=128256, bf16), "
                    "EAGLE-3-style 1-layer draft head, cache lengths ~U[1024,16384], 16-token pages")
     elif args.workload == "c4":
@@ -527,6 +531,8 @@ def main():
         config["draft_vocab"] = args.draft_vocab
     if args.workload == "c3" and args.kv_fp8:
         config["kv_cache"] = "e4m3 codes, scales 1/16 (REDUCED PRECISION: not the headline configuration)"
+    if args.workload == "c3" and args.w_fp8:
+        config["weights"] = "target projections and LM head as e4m3 codes with per-row scales (REDUCED PRECISION: not the headline configuration)"
     if args.workload != "c3":
         args.no_cpu_baseline = True
 
@@ -617,9 +623,10 @@ def main():
         metric = f"accepted tokens/s per B200 (one 235B-A22B-shaped MoE layer + LM head, k={k}; not the headline)"
     elif k != 3 or B != 256:
         metric = f"accepted tokens/s per B200 (8B-shape verify+sample, k={k}, B={B}; not the headline configuration)"
-    line = {"metric": metric + (" [8-bit KV cache variant]" if cfg.get("kv_fp8") else ""), "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+    line = {"metric": metric + (" [8-bit KV cache variant]" if cfg.get("kv_fp8") else "") + (" [8-bit weights variant]" if cfg.get("w_fp8") else ""),
+            "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": int(launches),
+            "dtype": "e4m3 projections, bf16 attention" if cfg.get("w_fp8") else "bf16", "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": int(launches),
             "roofline": roofline,
             "acceptance_length": emitted / float(args.steps * B), "accepted_drafts_per_step": accepted / float(args.steps * B)}
 
@@ -682,7 +689,9 @@ def main():
                           "plain_decode_gemm_bound_ms": {"tensor": gemm_flops_per_step(cfg, B, 0, "none") / (tf_peak * 1e12) * 1e3,
                                                          "weights_once_from_hbm": gemm_flops_per_step(cfg, 1, 0, "none") / (hbm_peak * 1e9) * 1e3},
                           "gemm_tflops_in_step": gemm_flops_per_step(cfg, B, k, info["draft"]) / (tm.ms[1] / 2 * 1e-3) / 1e12,
-                          "gemm_frac_of_measured_sustained_bf16": gemm_flops_per_step(cfg, B, k, info["draft"]) / (tm.ms[1] / 2 * 1e-3) / 1e12 / tf_peak,
+                          # 8-bit weights: the target's products run at the e4m3 rate, nominally twice the bf16 one (the draft head's stay bf16)
+                          ("gemm_frac_of_2x_measured_sustained_bf16_nominal_e4m3_ratio" if cfg.get("w_fp8") else "gemm_frac_of_measured_sustained_bf16"):
+                              gemm_flops_per_step(cfg, B, k, info["draft"]) / (tm.ms[1] / 2 * 1e-3) / 1e12 / (tf_peak * (2 if cfg.get("w_fp8") else 1)),
                           }
 
         if args.workload == "c3":

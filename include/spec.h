@@ -154,7 +154,12 @@ enum {
     SPEC_T_HIDDEN,              /* [B*(k+1)][d] fp32 residual stream after the last layer              */
     SPEC_T_MOE_LOGITS,          /* [B*(k+1)][n_experts] fp32 router logits of the last MoE layer run   */
     SPEC_T_MOE_IDS,             /* [B*(k+1)][experts_top_k] int32 selected experts, best first         */
-    SPEC_T_MOE_WTS              /* [B*(k+1)][experts_top_k] fp32 renormalised mixture weights          */
+    SPEC_T_MOE_WTS,             /* [B*(k+1)][experts_top_k] fp32 renormalised mixture weights          */
+    /* SPEC_W_E4M3 only: the quantised rows a projection consumed in the last pass.  `layer` names the     */
+    /* slot: 0 QKV, 1 O, 2 gate/up, 3 down (of the last layer that ran), 4 LM head.  Row r of a slot has   */
+    /* K codes at byte r*K (K = that projection's input width) and its scale at ACT_SCALES[r].             */
+    SPEC_T_ACT_CODES,           /* uint8 e4m3 codes, rows back to back                                 */
+    SPEC_T_ACT_SCALES           /* fp32 [rows]                                                         */
 };
 
 /* Counters returned by spec_get_status (host struct). */

@@ -25,6 +25,20 @@ def _split_gate_up(gu):
     return t[:, :128].reshape(F2 // 2, d), t[:, 128:].reshape(F2 // 2, d)
 
 
+def _w8(eng):
+    """True for a context that stores the target's projections as e4m3 codes with one scale per row."""
+    return int(getattr(eng.sc, "weight_dtype", 0)) == 1
+
+
+def _projection(eng, name, layer, shape):
+    """A projection weight as the oracle takes it: fp32 copies of the 16-bit values, or the stored codes and scales."""
+    import torch
+    if not _w8(eng):
+        return _np(eng.tensor(name, layer, eng.tdtype, shape))
+    return model.QuantRows(eng.tensor(name, layer, torch.uint8, shape).cpu().numpy(),
+                           eng.tensor(name + "_SCALE", layer, torch.float32, (shape[0],)).cpu().numpy())
+
+
 class _LazyRows:
     """Per-expert weight matrices [E][rows][cols] fetched from the device one expert at a time; `part` picks the gate
     (0) or up (1) half of a stacked gate/up matrix, None the whole matrix."""
@@ -59,7 +73,7 @@ class LazyLayers:
         od = cfg["n_q_heads"] * cfg["head_dim"]
         td = eng.tdtype
         lw = dict(attn_norm=_np(eng.tensor("ATTN_NORM", l, torch.float32, (d,))),
-                  wqkv=_np(eng.tensor("WQKV", l, td, (qn, d))), wo=_np(eng.tensor("WO", l, td, (d, od))),
+                  wqkv=_projection(eng, "WQKV", l, (qn, d)), wo=_projection(eng, "WO", l, (d, od)),
                   mlp_norm=_np(eng.tensor("MLP_NORM", l, torch.float32, (d,))))
         if cfg.get("n_experts", 0) > 0:
             E, Fe = cfg["n_experts"], cfg["d_expert_ffn"]
@@ -68,8 +82,13 @@ class LazyLayers:
             lw.update(router=_np(eng.tensor("ROUTER", l, td, (E, d))), experts_gate=_LazyRows(gu, 0),
                       experts_up=_LazyRows(gu, 1), experts_down=_LazyRows(dn))
         else:
-            gate, up = _split_gate_up(_np(eng.tensor("WGATEUP", l, td, (2 * F, d))))
-            lw.update(wgate=gate, wup=up, wdown=_np(eng.tensor("WDOWN", l, td, (d, F))))
+            gu = _projection(eng, "WGATEUP", l, (2 * F, d))
+            if isinstance(gu, model.QuantRows):
+                (cg, cu), (sg, su) = _split_gate_up(gu.codes), _split_gate_up(gu.scales[:, None])
+                gate, up = model.QuantRows(cg, sg[:, 0]), model.QuantRows(cu, su[:, 0])
+            else:
+                gate, up = _split_gate_up(gu)
+            lw.update(wgate=gate, wup=up, wdown=_projection(eng, "WDOWN", l, (d, F)))
         return lw
 
 
@@ -98,7 +117,7 @@ class LazyPast:
 def device_weights(eng, cfg, n_layers=None):
     import torch
     d, V, td = cfg["d_model"], cfg["vocab"], eng.tdtype
-    return dict(embed=_np(eng.tensor("EMBED", 0, td, (V, d))), lm_head=_np(eng.tensor("LM_HEAD", 0, td, (V, d))),
+    return dict(embed=_np(eng.tensor("EMBED", 0, td, (V, d))), lm_head=_projection(eng, "LM_HEAD", 0, (V, d)),
                 final_norm=_np(eng.tensor("FINAL_NORM", 0, torch.float32, (d,))), layers=LazyLayers(eng, cfg, n_layers))
 
 

@@ -85,7 +85,7 @@ def silu(x):
 def dense_mlp(lw, m, cfg=None):
     if cfg is None or not cfg.get("w_fp8"):
         return (silu(m @ np.asarray(lw["wgate"], F64).T) * (m @ np.asarray(lw["wup"], F64).T)) @ np.asarray(lw["wdown"], F64).T
-    return proj(cfg, silu(proj(cfg, m, lw["wgate"])) * proj(cfg, m, lw["wup"]), lw["wdown"])
+    return proj(cfg, silu(proj(cfg, m, lw["wgate"], "gateup")) * proj(cfg, m, lw["wup"], "gateup"), lw["wdown"], "down")
 
 
 def moe_route(router_logits, top_k):
@@ -180,15 +180,47 @@ def _bf16_round(x):
     return r
 
 
-def proj(cfg, x, W):
+class QuantRows:
+    """A weight matrix that is already stored in the 8-bit format: e4m3 codes [rows][k] and one fp32 scale per row.  Its
+    value is the exact product code x scale; proj() uses it as it stands instead of quantising 16-bit weights again."""
+
+    def __init__(self, codes, scales):
+        self.codes = np.ascontiguousarray(codes, np.uint8)
+        self.scales = np.ascontiguousarray(scales, np.float32)
+        assert self.codes.ndim == 2 and self.scales.shape == (self.codes.shape[0],)
+
+    def values(self):
+        import oracle
+        return oracle.e4m3_dequantize(self.codes).reshape(self.codes.shape).astype(F64) * self.scales.astype(F64)[:, None]
+
+
+def rows_8bit(x):
+    """Every row of x as its 8-bit representation: e4m3 codes of x / scale times the row's scale amax / 448, in fp64."""
+    import oracle
+    codes, scales = oracle.e4m3_quantize_rows(np.asarray(x, np.float32))
+    return QuantRows(codes, scales).values()
+
+
+def proj(cfg, x, W, stage=None):
     """x W^T of a target projection.  With cfg["w_fp8"] both operands go through the 8-bit format first (the precision the
     paper's simulator assumes, Section 5.1): the activation rows as the 16-bit values the layer before produced, each row
-    of x and each row of W with its own scale amax / 448; the product itself is exact."""
+    of x and each row of W with its own scale amax / 448; the product itself is exact.  W is either the 16-bit matrix
+    (quantised here) or a QuantRows holding the stored codes and scales.
+
+    Quantising is a step function of its input, so two computations whose activations differ in the last 16-bit place
+    drift apart by whole code steps.  For checks that must not depend on that, `stage` names the projection ("qkv", "o",
+    "gateup", "down", "lm_head"): cfg["record"][stage], when the dict is there, receives the rows as quantised here, and
+    cfg["forced"][stage], when present, is a QuantRows that replaces them in the product (single-layer calls only: every
+    layer of a multi-layer forward would see the same entry)."""
     if not cfg.get("w_fp8"):
         return x @ np.asarray(W, F64).T
     import oracle
-    xq = oracle.e4m3_rows_roundtrip(_bf16_round(np.asarray(x, np.float32))).astype(F64)
-    wq = oracle.e4m3_rows_roundtrip(np.asarray(W, np.float32)).astype(F64)
+    own = QuantRows(*oracle.e4m3_quantize_rows(_bf16_round(np.asarray(x, np.float32))))
+    if stage is not None and cfg.get("record") is not None:
+        cfg["record"][stage] = own
+    forced = (cfg.get("forced") or {}).get(stage) if stage is not None else None
+    xq = (own if forced is None else forced).values()
+    wq = W.values() if isinstance(W, QuantRows) else rows_8bit(W)
     return xq @ wq.T
 
 
@@ -213,7 +245,7 @@ def decoder_layer(cfg, lw, x, pos, past_k=None, past_v=None, attn_in=None, route
     Hq, Hkv, dh = cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"]
     T = x.shape[0]
     h = rmsnorm(x, lw["attn_norm"], cfg["rms_eps"]) if attn_in is None else attn_in
-    qkv = proj(cfg, h, lw["wqkv"])
+    qkv = proj(cfg, h, lw["wqkv"], "qkv")
     q = qkv[:, : Hq * dh].reshape(T, Hq, dh)
     k = qkv[:, Hq * dh : (Hq + Hkv) * dh].reshape(T, Hkv, dh)
     v = qkv[:, (Hq + Hkv) * dh :].reshape(T, Hkv, dh)
@@ -224,7 +256,7 @@ def decoder_layer(cfg, lw, x, pos, past_k=None, past_v=None, attn_in=None, route
     k_all = k if n_past == 0 else np.concatenate([np.asarray(past_k, F64), k], axis=0)
     v_all = v if n_past == 0 else np.concatenate([np.asarray(past_v, F64), v], axis=0)
     att = attention(q, k_all, v_all, n_past).reshape(T, Hq * dh)
-    x = x + proj(cfg, att, lw["wo"])
+    x = x + proj(cfg, att, lw["wo"], "o")
     m = rmsnorm(x, lw["mlp_norm"], cfg["rms_eps"])
     if cfg.get("n_experts", 0) > 0:
         x = x + moe_mlp(lw, m, cfg["experts_top_k"], router_logits)
@@ -253,7 +285,7 @@ def target_forward(cfg, W, tokens, past=None, start_pos=0, tap_layers=(), router
         new_kv.append((k, v))
         if (l + 1) in tap_layers:
             taps[l + 1] = x
-    logits = proj(cfg, rmsnorm(x, W["final_norm"], cfg["rms_eps"]), W["lm_head"])
+    logits = proj(cfg, rmsnorm(x, W["final_norm"], cfg["rms_eps"]), W["lm_head"], "lm_head")
     tap_cat = np.concatenate([taps[t] for t in tap_layers], axis=-1) if tap_layers else np.zeros((T, 0))
     return {"logits": logits, "taps": tap_cat, "final": x, "new_kv": new_kv}
 

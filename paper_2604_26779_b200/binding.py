@@ -31,7 +31,8 @@ T = dict(EMBED=0, LM_HEAD=1, FINAL_NORM=2, ATTN_NORM=3, WQKV=4, WO=5, MLP_NORM=6
          KV_K=64, KV_V=65, DRAFT_KV_K=66, DRAFT_KV_V=67,
          SEQ_LEN=96, LAST_TOKEN=97, BLOCK_TABLE=98, FREE_STACK=99, FREE_TOP=100, DRAFT_TOKENS=101, OUT_TOKENS=102,
          N_EMITTED=103, STATUS=104, STEP=105, TOKEN_HISTORY=106, OUT_LOGP=107,
-         LOGITS=128, DRAFT_LOGITS=129, ROW_STATS=130, DRAFT_ROW_STATS=131, TAPS=132, HIDDEN=133, MOE_LOGITS=134, MOE_IDS=135, MOE_WTS=136)
+         LOGITS=128, DRAFT_LOGITS=129, ROW_STATS=130, DRAFT_ROW_STATS=131, TAPS=132, HIDDEN=133, MOE_LOGITS=134, MOE_IDS=135, MOE_WTS=136,
+         ACT_CODES=137, ACT_SCALES=138)
 
 
 class SpecError(RuntimeError):

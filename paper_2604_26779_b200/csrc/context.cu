@@ -8,6 +8,7 @@
 #include "ops.cuh"
 
 struct Loc { size_t off = 0, bytes = 0; };
+constexpr int kActSlots = 5;         // quantised activation buffers of an 8-bit-weights context: QKV, O, gate/up, down, LM head
 
 struct LayerLoc { Loc attn_norm, wqkv, wo, mlp_norm, wgateup, wdown, router, exp_gateup, exp_down, wqkv_s, wo_s, wgateup_s, wdown_s; };
 
@@ -200,8 +201,10 @@ void build_layout(spec_ctx& x)
         x.act = a.take(M * Fmax * es);
         if (c.weight_dtype == SPEC_W_E4M3) {                  // activations as e4m3 codes + one scale per row, rewritten before every projection
             const size_t kmax = (size_t)(c.d_ffn > (int)od ? c.d_ffn : od) > d ? (size_t)(c.d_ffn > (int)od ? c.d_ffn : od) : d;
-            x.a8 = a.take(M * kmax);
-            x.a8_scale = a.take(M * 4);
+            // five slots, one per projection of a layer (QKV, O, gate/up, down) and one for the LM head, so that what the last
+            // layer and the LM head consumed stays readable after the pass (SPEC_T_ACT_CODES / SPEC_T_ACT_SCALES)
+            x.a8 = a.take(kActSlots * M * kmax);
+            x.a8_scale = a.take(kActSlots * M * 4);
         }
         x.logits = a.take(M * (size_t)c.vocab * 4);
         x.draft_logits = a.take(Bm * (size_t)(c.k_max > 0 ? c.k_max : 1) * c.vocab * 4);   // sized for the whole vocabulary
@@ -303,6 +306,35 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
     const int qkv_n = (Hq + 2 * Hkv) * dh, dt = g.dtype;
     void* ws = c.buf.workspace;
     int32_t* status_word = at<int32_t>(c.buf.state, c.status);
+    const bool w8 = g.weight_dtype == SPEC_W_E4M3 && W.wqkv_s != nullptr;   // the target's layers with 8-bit weights (the draft head has none)
+    if (w8) {
+        const size_t slot_bytes = c.a8.bytes / kActSlots, slot_rows = c.a8_scale.bytes / kActSlots / 4;
+        auto a8_of = [&](int slot) { return at<unsigned char>(ws, c.a8) + slot * slot_bytes; };
+        auto a8s_of = [&](int slot) { return at<float>(ws, c.a8_scale) + slot * slot_rows; };
+        // every projection: its input rows to e4m3 with a scale per row, then the 8-bit tensor-core product; the epilogues
+        // are the usual ones (rotary + cache append, residual add, SwiGLU) on the rescaled accumulators
+        QkvEpilogue e{Hq, Hkv, dh, R, g.max_blocks_per_seq, g.kv_block_tokens, pos, at<int32_t>(c.buf.state, c.block_table),
+                      at<float>(ws, c.rope), k_pool, v_pool};
+        if (g.kv_dtype == SPEC_KV_E4M3) { e.kv_fp8 = 1; e.k_scale = g.kv_scale_k; e.v_scale = g.kv_scale_v; }
+        TRY(launch_quantize_rows(M, qkv_k, qkv_in, a8_of(0), a8s_of(0), st));
+        TIMED(c, CLS_GEMM, launch_gemm8_qkv_tc(M, qkv_k, a8_of(0), a8s_of(0), W.wqkv, W.wqkv_s, at(ws, c.qkv), e, status_word, st));
+        AttnArgs a{B, R, Hq, Hkv, dh, g.kv_block_tokens, g.max_blocks_per_seq, at(ws, c.qkv), qkv_n, k_pool, v_pool,
+                   at<int32_t>(c.buf.state, c.block_table), pos, at(ws, c.attn_out), Hq * dh, dt, at(ws, c.attn_scratch),
+                   c.attn_scratch.bytes, g.max_blocks_per_seq * g.kv_block_tokens, launch_index};
+        a.status = status_word;
+        if (g.kv_dtype == SPEC_KV_E4M3) { a.kv_fp8 = 1; a.k_scale = g.kv_scale_k; a.v_scale = g.kv_scale_v; }
+        TIMED(c, CLS_ATTN, launch_attention(a, st));
+        TRY(launch_quantize_rows(M, Hq * dh, at(ws, c.attn_out), a8_of(1), a8s_of(1), st));
+        TIMED(c, CLS_GEMM, launch_gemm8_tc(M, d, Hq * dh, a8_of(1), a8s_of(1), W.wo, W.wo_s, res, d, SPEC_DTYPE_F32, 1, 1.f, nullptr, 0, nullptr, 0,
+                                           status_word, st));
+        TRY(launch_rmsnorm(M, d, res, W.mlp_norm, g.rms_eps, at(ws, c.h), d, 0, dt, st));
+        TRY(launch_quantize_rows(M, d, at(ws, c.h), a8_of(2), a8s_of(2), st));
+        TIMED(c, CLS_GEMM, launch_gemm8_swiglu_tc(M, d_ffn, d, a8_of(2), a8s_of(2), W.wgateup, W.wgateup_s, at(ws, c.act), status_word, st));
+        TRY(launch_quantize_rows(M, d_ffn, at(ws, c.act), a8_of(3), a8s_of(3), st));
+        TIMED(c, CLS_GEMM, launch_gemm8_tc(M, d, d_ffn, a8_of(3), a8s_of(3), W.wdown, W.wdown_s, res, d, SPEC_DTYPE_F32, 1, 1.f, nullptr, 0, nullptr, 0,
+                                           status_word, st));
+        return SPEC_OK;
+    }
     const bool tc = gemm_tc_supported(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt);
     // very few rows (the thin tail of a rollout): plain weight-streaming projections + the small element-wise kernels beat
     // the fused tensor-core epilogues, which have too few tiles to pull the weights at the HBM rate
@@ -500,6 +532,15 @@ extern "C" spec_status spec_tensor(spec_ctx* c, int id, int layer, void** dev_pt
     case SPEC_T_MOE_LOGITS: base = c->buf.workspace; l = c->moe_logits; break;
     case SPEC_T_MOE_IDS: base = c->buf.workspace; l = c->moe_ids; break;
     case SPEC_T_MOE_WTS: base = c->buf.workspace; l = c->moe_wts; break;
+    case SPEC_T_ACT_CODES: case SPEC_T_ACT_SCALES: {
+        // `layer` selects the slot: 0 QKV, 1 O, 2 gate/up, 3 down (of the last layer run), 4 LM head
+        if (layer < 0 || layer >= kActSlots) return SPEC_ERR_INVALID_ARG;
+        const Loc& whole = id == SPEC_T_ACT_CODES ? c->a8 : c->a8_scale;
+        base = c->buf.workspace;
+        l.bytes = whole.bytes / kActSlots;
+        l.off = whole.off + layer * l.bytes;
+        break;
+    }
     default: return SPEC_ERR_INVALID_ARG;
     }
     if (base == nullptr || l.bytes == 0) return SPEC_ERR_INVALID_ARG;
@@ -677,7 +718,20 @@ extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_toke
     TRY(launch_rmsnorm(M, d, x, at<const float>(c->buf.weights, c->final_norm), g.rms_eps, at(ws, c->h), d, 0, dt, st));
     // LM head with the row statistics taken in its epilogue; shapes the tile kernel does not take go the two-pass way
     spec_status fused = SPEC_ERR_UNSUPPORTED;
-    {
+    if (g.weight_dtype == SPEC_W_E4M3) {
+        unsigned char* a8 = at<unsigned char>(ws, c->a8) + (kActSlots - 1) * (c->a8.bytes / kActSlots);
+        float* a8s = at<float>(ws, c->a8_scale) + (kActSlots - 1) * (c->a8_scale.bytes / kActSlots / 4);
+        TRY(launch_quantize_rows(M, d, at(ws, c->h), a8, a8s, st));
+        Timed t__(*c, CLS_GEMM, st);
+        fused = launch_gemm8_tc(M, g.vocab, d, a8, a8s, at(c->buf.weights, c->lm_head), at<const float>(c->buf.weights, c->lm_head_s),
+                                at(ws, c->logits), g.vocab, SPEC_DTYPE_F32, 0, g.temperature, at<float>(ws, c->splitk), c->splitk.bytes,
+                                at<float>(ws, c->row_stats), 1, at<int32_t>(sb, c->status), st);
+        if (fused == SPEC_ERR_UNSUPPORTED) {                  // logits are written; only the statistics still need their pass
+            cudaGetLastError();
+            fused = launch_softmax_rows(M, g.vocab, at<float>(ws, c->logits), (size_t)g.vocab, g.temperature, at<float>(ws, c->row_stats), 1,
+                                        nullptr, st);
+        }
+    } else {
         Timed t__(*c, CLS_GEMM, st);
         fused = launch_gemm_lm_head_stats(M, g.vocab, d, at(ws, c->h), d, at(c->buf.weights, c->lm_head), at<float>(ws, c->logits), g.vocab, dt,
                                           g.temperature, at<float>(ws, c->splitk), c->splitk.bytes, at<float>(ws, c->row_stats), 1,

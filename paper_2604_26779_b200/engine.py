@@ -16,8 +16,9 @@ from .binding import T
 def make_spec_config(cfg: dict, *, draft_kind: str = "none", k_max: int = 3, max_batch: int = 4, kv_num_blocks: int = 64,
                      max_blocks_per_seq: int = 16, kv_block_tokens: int = 16, kv_layer_pools: int | None = None,
                      seed: int = 0, draft_d_ffn: int | None = None, ngram_n: int = 3, draft_greedy: bool = False,
-                     draft_vocab: int = 0, kv_fp8=None) -> B.spec_config:
-    """kv_fp8: None for a cache in the model's dtype, or (k_scale, v_scale) for the 8-bit e4m3 cache."""
+                     draft_vocab: int = 0, kv_fp8=None, w_fp8: bool = False) -> B.spec_config:
+    """kv_fp8: None for a cache in the model's dtype, or (k_scale, v_scale) for the 8-bit e4m3 cache.
+    w_fp8: the target's projections and LM head in e4m3 with per-row scales (a reduced-precision mode)."""
     sc = B.spec_config()
     sc.struct_size, sc.abi_version = C.sizeof(B.spec_config), B.SPEC_ABI_VERSION
     for name in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn", "vocab", "n_experts",
@@ -32,6 +33,7 @@ def make_spec_config(cfg: dict, *, draft_kind: str = "none", k_max: int = 3, max
     sc.draft_vocab = int(draft_vocab) if draft_kind == "eagle3" else 0
     if kv_fp8:
         sc.kv_dtype, sc.kv_scale_k, sc.kv_scale_v = B.SPEC_KV_E4M3, float(kv_fp8[0]), float(kv_fp8[1])
+    sc.weight_dtype = B.SPEC_W_E4M3 if (w_fp8 or cfg.get("w_fp8")) else B.SPEC_W_MODEL
     taps = tuple(cfg.get("tap_layers", ())) if draft_kind == "eagle3" else ()
     sc.n_taps = len(taps)
     for i, t in enumerate(taps):
@@ -128,23 +130,36 @@ class SpecStep:
         assert src.numel() <= dst.numel(), (name, src.numel(), dst.numel())
         dst[: src.numel()].copy_(src)
 
+    def put_projection(self, name: str, layer: int, array):
+        """A projection weight [rows][K]: stored as it is, or - in a context with 8-bit weights - as e4m3 codes with one
+        scale per row, quantised on the device by the library (spec_quantize_rows) from the 16-bit values."""
+        if self.sc.weight_dtype != B.SPEC_W_E4M3:
+            return self.put(name, layer, array)
+        w = torch.from_numpy(np.ascontiguousarray(array)).to(self.device).to(torch.bfloat16)
+        w = w.reshape(-1, w.shape[-1]).contiguous()
+        codes = self.tensor(name, layer, torch.uint8)
+        scales = self.tensor(name + "_SCALE", layer, torch.float32)
+        assert codes.numel() == w.numel() and scales.numel() == w.shape[0], (name, codes.numel(), w.numel(), scales.numel())
+        B.spec_quantize_rows(w, codes.view(w.shape), scales)
+        torch.cuda.synchronize()
+
     def load_target_weights(self, W: dict):
         f32 = torch.float32
         self.put("EMBED", 0, W["embed"])
-        self.put("LM_HEAD", 0, W["lm_head"])
+        self.put_projection("LM_HEAD", 0, W["lm_head"])
         self.put("FINAL_NORM", 0, W["final_norm"], f32)
         for l, lw in enumerate(W["layers"]):
             self.put("ATTN_NORM", l, lw["attn_norm"], f32)
-            self.put("WQKV", l, lw["wqkv"])
-            self.put("WO", l, lw["wo"])
+            self.put_projection("WQKV", l, lw["wqkv"])
+            self.put_projection("WO", l, lw["wo"])
             self.put("MLP_NORM", l, lw["mlp_norm"], f32)
             if "router" in lw:
                 self.put("ROUTER", l, lw["router"])
                 self.put("EXPERTS_GATEUP", l, stack_gate_up(lw["experts_gate"], lw["experts_up"]))
                 self.put("EXPERTS_DOWN", l, lw["experts_down"])
             else:
-                self.put("WGATEUP", l, stack_gate_up(lw["wgate"], lw["wup"]))
-                self.put("WDOWN", l, lw["wdown"])
+                self.put_projection("WGATEUP", l, stack_gate_up(lw["wgate"], lw["wup"]))
+                self.put_projection("WDOWN", l, lw["wdown"])
 
     def load_draft_weights(self, H: dict):
         f32 = torch.float32

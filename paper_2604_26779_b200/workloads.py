@@ -7,7 +7,7 @@ from __future__ import annotations
 import numpy as np
 import torch
 
-from . import engine, inputs
+from . import binding, engine, inputs
 
 
 def _fill_normal(t: torch.Tensor, std: float, gen: torch.Generator):
@@ -57,7 +57,7 @@ def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, l
         sc = engine.make_spec_config(cfg, draft_kind=draft, k_max=k, max_batch=B, kv_num_blocks=num_blocks,
                                      max_blocks_per_seq=max_blocks, kv_layer_pools=G, seed=seed,
                                      draft_vocab=int(cfg.get("draft_vocab") or 0), draft_greedy=bool(cfg.get("draft_greedy")),
-                                     kv_fp8=cfg.get("kv_fp8"))
+                                     kv_fp8=cfg.get("kv_fp8"), w_fp8=bool(cfg.get("w_fp8")))
         from . import binding as Bd
         import ctypes as C
         s = Bd.spec_sizes()
@@ -78,8 +78,20 @@ def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, l
     gen.manual_seed(seed)
     bf = eng.tdtype
     f32 = torch.float32
+    w8 = bool(cfg.get("w_fp8"))
+
+    def fill_projection(name, layer, rows, k):
+        # N(0, 0.02) weights; with 8-bit weights they are drawn in bf16 and quantised row by row on the device by the library
+        if not w8:
+            return _fill_normal(eng.tensor(name, layer, bf), 0.02, gen)
+        tmp = torch.empty((rows, k), dtype=torch.bfloat16, device=device)
+        _fill_normal(tmp, 0.02, gen)
+        binding.spec_quantize_rows(tmp, eng.tensor(name, layer, torch.uint8, (rows, k)), eng.tensor(name + "_SCALE", layer, f32, (rows,)))
+        torch.cuda.synchronize()
+
+    d_, qn_, od_ = cfg["d_model"], (cfg["n_q_heads"] + 2 * cfg["n_kv_heads"]) * cfg["head_dim"], cfg["n_q_heads"] * cfg["head_dim"]
     _fill_normal(eng.tensor("EMBED", 0, bf), 0.02, gen)
-    _fill_normal(eng.tensor("LM_HEAD", 0, bf), 0.02, gen)
+    fill_projection("LM_HEAD", 0, cfg["vocab"], d_)
     eng.tensor("FINAL_NORM", 0, f32).fill_(1.0)
     for l in range(L):
         eng.tensor("ATTN_NORM", l, f32).fill_(1.0)
@@ -90,8 +102,10 @@ def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, l
             # router rows ~ N(0, 1/d): unit-RMS inputs give router logits ~ N(0, 1)
             _fill_normal(eng.tensor("ROUTER", l, bf), float(cfg["d_model"]) ** -0.5, gen)
         else:
-            for nm in ("WQKV", "WO", "WGATEUP", "WDOWN"):
-                _fill_normal(eng.tensor(nm, l, bf), 0.02, gen)
+            fill_projection("WQKV", l, qn_, d_)
+            fill_projection("WO", l, d_, od_)
+            fill_projection("WGATEUP", l, 2 * cfg["d_ffn"], d_)
+            fill_projection("WDOWN", l, d_, cfg["d_ffn"])
     if draft != "none":
         for nm in ("D_NORM_E", "D_NORM_G", "D_MLP_NORM") + (("D_NORM_F",) if draft == "eagle3" else ("D_ATTN_NORM",)):
             eng.tensor(nm, 0, f32).fill_(1.0)

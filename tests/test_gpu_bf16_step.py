@@ -46,10 +46,12 @@ def draft_head_weights(eng, cfg, kind):
     return H
 
 
-@pytest.mark.parametrize("kind,k,head_dim,kv_fp8", [("eagle3", 3, 64, None), ("mtp", 2, 64, None), ("eagle3", 7, 64, None),
-                                                     ("eagle3", 5, 128, None), ("mtp", 7, 128, None),
-                                                     ("eagle3", 3, 128, (1.0, 1.0)), ("mtp", 3, 128, (0.05, 0.03))])
-def test_bf16_steps_stage_by_stage(kind, k, head_dim, kv_fp8):
+@pytest.mark.parametrize("kind,k,head_dim,kv_fp8,w_fp8", [("eagle3", 3, 64, None, False), ("mtp", 2, 64, None, False),
+                                                           ("eagle3", 7, 64, None, False), ("eagle3", 5, 128, None, False),
+                                                           ("mtp", 7, 128, None, False), ("eagle3", 3, 128, (1.0, 1.0), False),
+                                                           ("mtp", 3, 128, (0.05, 0.03), False), ("eagle3", 3, 128, None, True),
+                                                           ("eagle3", 3, 128, (1.0, 1.0), True)])
+def test_bf16_steps_stage_by_stage(kind, k, head_dim, kv_fp8, w_fp8):
     """head_dim 64: 16 or 32 query rows per KV head on the register-fragment attention kernel; head_dim 128 with k = 5 / 7:
     24 / 32 rows on the tcgen05 kernel, including the draft head's first pass, whose rows past the committed count carry
     position -1."""
@@ -59,6 +61,15 @@ def test_bf16_steps_stage_by_stage(kind, k, head_dim, kv_fp8):
     over = dict(d_model=512, n_q_heads=8, n_kv_heads=2, head_dim=head_dim, d_ffn=1024)
     if kv_fp8:                 # 8-bit cache: the oracle rounds every key and value to e4m3 exactly where the device stores it
         over["kv_fp8"] = kv_fp8
+    if w_fp8:
+        # 8-bit projections.  Quantising an activation row is a step function (a row maximum that rounds to the neighbouring
+        # 16-bit value moves the whole row's codes), so two forwards that differ in one last place drift apart by about the
+        # format's own noise: on the oracle alone, a 2^-12 relative perturbation of the activations moves the logits of this
+        # model by 7 % of the row maximum, and the 8-bit forward sits 11 % from the 16-bit one.  The whole-forward logit bar
+        # below therefore only catches gross errors; the products and quantisers are checked exactly, projection by projection
+        # with the device's own rows, in test_gpu_w_fp8.py.  Draft, sampler and bookkeeping bars are unchanged.
+        over["w_fp8"] = True
+    logit_bar = 0.25 if w_fp8 else 2e-2
     n_layers = 3
     lens = np.array([5, 40, 100, 17, 300], np.int32)
     eng, info = workloads.build_dense_workload("c3", lens=lens, k=k, draft=kind, steps_budget=8, n_layers=n_layers,
@@ -134,6 +145,7 @@ def test_bf16_steps_stage_by_stage(kind, k, head_dim, kv_fp8):
         assert eng.status().device_status == 0
         assert np.array_equal(eng.seq_len().cpu().numpy(), seq_len + g_n)
         k_prev = k
-    print(f"bf16 {kind} k={k} dh={head_dim} kv_fp8={kv_fp8}: draft logits {worst_d:.2e}, verify logits {worst_v:.2e}, boundary cases {boundary}")
-    assert worst_d < 2e-2 and worst_v < 2e-2 and boundary <= 2
+    print(f"bf16 {kind} k={k} dh={head_dim} kv_fp8={kv_fp8} w_fp8={w_fp8}: draft logits {worst_d:.2e}, verify logits {worst_v:.2e}, "
+          f"boundary cases {boundary}")
+    assert worst_d < 2e-2 and worst_v < logit_bar and boundary <= 2
     eng.close()

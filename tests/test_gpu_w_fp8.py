@@ -1,0 +1,125 @@
+"""GPU parity of a verify pass with 8-bit (e4m3) projections, projection by projection.
+
+Quantising an activation row is a step function (a row maximum that rounds to the neighbouring 16-bit value moves the
+row's scale and with it many codes), so logits of two whole forwards that differ in the last place of one activation
+drift apart by about the format's own noise; an end-to-end bar would say nothing.  Instead the context keeps the rows every
+projection of its last layer (and the LM head) consumed, and each stage is checked with those rows forced into the oracle:
+
+  product     forced rows x stored weight codes, exact in the oracle: cache entries (after the rotary embedding) to bf16
+              rounding, residual stream and logits to fp32 accumulation error
+  quantiser   what the oracle quantises from ITS result of the stage before against the device's rows of the next stage:
+              scales within one 16-bit step, nearly all codes equal, none further than one code step
+"""
+import numpy as np
+import pytest
+
+import oracle
+from oracle import harness, model
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+def act_rows(eng, slot, M, K):
+    codes = eng.tensor("ACT_CODES", slot, torch.uint8)[: M * K].view(M, K).cpu().numpy()
+    scales = eng.tensor("ACT_SCALES", slot, torch.float32)[:M].cpu().numpy()
+    return model.QuantRows(codes, scales)
+
+
+def rows_of(qr, r0, r1):
+    return model.QuantRows(qr.codes[r0:r1], qr.scales[r0:r1])
+
+
+def compare_rows(dev, ref, what, min_equal, abs_rms=0.0):
+    """Device rows against the oracle's: scales within one bf16 step of the row maximum, values within one e4m3 step of
+    the element (at most 2^-3 of it; sub-normal codes: 2^-9 of the scale) plus the effect of that scale difference, plus
+    abs_rms times the row's RMS where the 16-bit input itself carries an absolute error (attention probabilities in bf16)."""
+    assert np.all(np.abs(dev.scales - ref.scales) <= 2.0 ** -7 * ref.scales), what
+    a, b = dev.values(), ref.values()
+    tol = 0.135 * np.abs(b) + 2.0 ** -9 * ref.scales[:, None] + abs_rms * np.sqrt(np.mean(b * b, -1, keepdims=True))
+    assert np.all(np.abs(a - b) <= tol), (what, float(np.max(np.abs(a - b) - tol)))
+    same = float(np.mean(dev.codes == ref.codes))
+    assert same >= min_equal, (what, same)
+    return same
+
+
+@pytest.mark.parametrize("n_layers,head_dim,kv_fp8", [(1, 128, None), (3, 128, None), (1, 64, None), (2, 128, (0.25, 0.25))])
+def test_w_fp8_verify_projection_by_projection(n_layers, head_dim, kv_fp8):
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_26779_b200 import workloads
+    k = 3
+    over = dict(d_model=512, n_q_heads=8, n_kv_heads=2, head_dim=head_dim, d_ffn=1024, w_fp8=True)
+    if kv_fp8:
+        over["kv_fp8"] = kv_fp8
+    lens = np.array([5, 40, 100, 17, 300, 64, 33], np.int32)
+    eng, info = workloads.build_dense_workload("c3", lens=lens, k=k, draft="eagle3", steps_budget=8, n_layers=n_layers,
+                                               vocab=2048, cfg_over=over)
+    cfg = dict(info["cfg"], n_layers=n_layers)
+    B, d, V, F = eng.B, cfg["d_model"], cfg["vocab"], cfg["d_ffn"]
+    Hq, Hkv, dh = cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"]
+    W = harness.device_weights(eng, cfg)
+    assert isinstance(W["lm_head"], model.QuantRows)
+    lw = W["layers"][n_layers - 1]
+    workloads.bootstrap(eng)
+    eng.draft(k); eng.verify(k); eng.reject_sample(k); eng.kv_commit()      # one whole step first: state past the bootstrap
+    seq_len = eng.seq_len().cpu().numpy().copy()
+    last = eng.tensor("LAST_TOKEN", 0, torch.int32, (B,)).cpu().numpy().copy()
+    eng.draft(k)
+    drafts = eng.draft_tokens().cpu().numpy()[:, :k].copy()
+    eng.verify(k)
+    assert eng.status().device_status == 0
+    table = eng.block_table().cpu().numpy().copy()
+    R, M = k + 1, B * (k + 1)
+    dev = {"qkv": act_rows(eng, 0, M, d), "o": act_rows(eng, 1, M, Hq * dh), "gateup": act_rows(eng, 2, M, d),
+           "down": act_rows(eng, 3, M, F), "lm_head": act_rows(eng, 4, M, d)}
+    hidden = eng.tensor("HIDDEN", 0, torch.float32, (M, d)).cpu().numpy().astype(np.float64)
+    logits = eng.logits(k).cpu().numpy().reshape(M, V).astype(np.float64)
+    stats = eng.tensor("ROW_STATS", 0, torch.float32, (M, 2)).cpu().numpy()
+    embed = W["embed"]
+    worst_kv = worst_x = worst_l = 0.0
+    equal = {"qkv": 1.0, "o": 1.0, "gateup": 1.0, "down": 1.0, "lm_head": 1.0}
+    for b in range(B):
+        r0, r1 = b * R, (b + 1) * R
+        n_past = int(seq_len[b])
+        tokens = [int(last[b])] + [int(t) for t in drafts[b]]
+        pos = np.arange(n_past, n_past + R)
+        record = {}
+        cfg_f = dict(cfg, forced={s: rows_of(q, r0, r1) for s, q in dev.items()}, record=record)
+        past = harness.LazyPast(eng, cfg, table[b], n_past, info["kv_pools"], n_layers)[n_layers - 1]
+        # a one-layer model starts from the embedding rows, which the oracle knows exactly; deeper ones: the layer's input is
+        # not kept, so what depends on it (the residual stream) is left to the one-layer cases
+        x_in = embed[tokens].astype(np.float64) if n_layers == 1 else np.zeros((R, d))
+        x_out, k_new, v_new = model.decoder_layer(cfg_f, lw, x_in, pos, past[0] if n_past else None, past[1] if n_past else None)
+        # -- QKV product + rotary embedding + cache append: the device's cache entries of the new positions
+        got = harness.LazyPast(eng, cfg, table[b], n_past + R, info["kv_pools"], n_layers)[n_layers - 1]
+        for g_, ref in ((got[0][n_past:], k_new), (got[1][n_past:], v_new)):
+            if kv_fp8:      # the oracle's values are already rounded to the cache format: one code step where fp32 and fp64 results straddle a boundary
+                assert np.all(np.abs(g_ - ref) <= 0.126 * np.abs(ref) + 2.0 ** -9 * kv_fp8[0])
+                assert np.mean(g_ == ref.astype(np.float32)) > 0.97
+            else:
+                err = np.abs(g_ - ref) / (np.abs(ref) + 1e-3 * np.abs(ref).max())
+                worst_kv = max(worst_kv, float(err.max()))
+        # -- attention output as the O projection consumed it (q went through the same epilogue as k)
+        equal["o"] = min(equal["o"], compare_rows(rows_of(dev["o"], r0, r1), record["o"], "o", 0.80, abs_rms=8e-3))
+        # -- SwiGLU of the forced gate/up input, as the down projection consumed it
+        equal["down"] = min(equal["down"], compare_rows(rows_of(dev["down"], r0, r1), record["down"], "down", 0.97))
+        if n_layers == 1:
+            equal["qkv"] = min(equal["qkv"], compare_rows(rows_of(dev["qkv"], r0, r1), record["qkv"], "qkv", 0.99))
+            equal["gateup"] = min(equal["gateup"], compare_rows(rows_of(dev["gateup"], r0, r1), record["gateup"], "gateup", 0.99))
+            # -- O and down products with their residual adds: the fp32 residual stream after the layer
+            worst_x = max(worst_x, float(np.abs(hidden[r0:r1] - x_out).max() / np.abs(x_out).max()))
+        # -- final norm of the device's residual stream, quantised, then the LM head product and its row statistics
+        rec2 = {}
+        cfg_l = dict(cfg, forced={"lm_head": rows_of(dev["lm_head"], r0, r1)}, record=rec2)
+        ref_logits = model.proj(cfg_l, model.rmsnorm(hidden[r0:r1], W["final_norm"], cfg["rms_eps"]), W["lm_head"], "lm_head")
+        equal["lm_head"] = min(equal["lm_head"], compare_rows(rows_of(dev["lm_head"], r0, r1), rec2["lm_head"], "lm_head", 0.99))
+        worst_l = max(worst_l, float((np.abs(logits[r0:r1] - ref_logits).max(-1) / np.abs(ref_logits).max(-1)).max()))
+        for j in range(R):
+            m_o, z_o = oracle.softmax_stats(logits[r0 + j].astype(np.float32), 1.0)
+            assert stats[r0 + j, 0] == m_o and abs(stats[r0 + j, 1] - z_o) <= 1e-4 * z_o
+    print(f"w_fp8 L={n_layers} dh={head_dim} kv_fp8={kv_fp8}: cache entries {worst_kv:.2e}, residual stream {worst_x:.2e}, "
+          f"logits {worst_l:.2e}, equal codes {equal}")
+    assert worst_kv < 2.0 ** -7          # bf16 rounding of the stored value (2^-9 .. 2^-8) plus fp32 accumulation
+    assert worst_x < 1e-5 and worst_l < 1e-5
+    eng.close()

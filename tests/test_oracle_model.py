@@ -286,7 +286,10 @@ def test_e4m3_row_quantisation_hand_worked():
 
 def test_fp8_projection_error_is_what_the_format_allows():
     # a random projection through the 8-bit path stays within the few-percent error two 4-bit-significand operands allow,
-    # and is exact when both operands are representable (powers of two)
+    # and is exact when both operands are representable with a power-of-two scale: every row holds 14 = 448 * 2^-5 (so its
+    # scale is exactly 2^-5) and powers of two between 1/8 and 4 (codes 4 .. 128 after scaling).  With any other row maximum
+    # the fp32 scale amax / 448 is itself rounded, and the represented value code * scale is 2^-24-relative off the input:
+    # that rounding belongs to the format and the product of the represented values carries it.
     rng = np.random.default_rng(3)
     x = rng.standard_normal((5, 256)).astype(np.float32)
     W = (rng.standard_normal((7, 256)) * 0.05).astype(np.float32)
@@ -296,5 +299,18 @@ def test_fp8_projection_error_is_what_the_format_allows():
     assert np.max(np.abs(got - ref)) > 0
     xp = np.ldexp(1.0, rng.integers(-3, 3, (4, 64))).astype(np.float32) * rng.choice([-1.0, 1.0], (4, 64)).astype(np.float32)
     Wp = np.ldexp(1.0, rng.integers(-3, 3, (6, 64))).astype(np.float32)
+    xp[:, 0], Wp[:, 5] = 14.0, 14.0
     assert np.array_equal(model.proj({"w_fp8": True}, xp, Wp), xp.astype(np.float64) @ Wp.astype(np.float64).T)
     assert np.array_equal(model.proj({}, xp, Wp), xp.astype(np.float64) @ Wp.astype(np.float64).T)
+    # stored codes and scales are taken as they stand: the same product as quantising the 16-bit matrix here
+    codes, scales = oracle.e4m3_quantize_rows(W)
+    assert np.array_equal(model.proj({"w_fp8": True}, x, model.QuantRows(codes, scales)), got)
+    # recording returns the rows as quantised; forcing them back reproduces the product; forcing other rows replaces x
+    rec = {}
+    assert np.array_equal(model.proj({"w_fp8": True, "record": rec}, x, W, "qkv"), got)
+    xc, xs = oracle.e4m3_quantize_rows(model._bf16_round(x))      # activations enter as 16-bit values
+    assert np.array_equal(rec["qkv"].codes, xc) and np.array_equal(rec["qkv"].scales, xs)
+    assert np.array_equal(model.proj({"w_fp8": True, "forced": {"qkv": rec["qkv"]}}, np.zeros_like(x), W, "qkv"), got)
+    assert np.array_equal(model.proj({"w_fp8": True, "forced": {"o": rec["qkv"]}}, np.zeros_like(x), W, "qkv"), np.zeros_like(got))
+    one = model.QuantRows(np.full((1, 256), 0x38, np.uint8), np.array([2.0], np.float32))      # 0x38 = 1.0: a row of twos
+    assert np.allclose(model.proj({"w_fp8": True, "forced": {"qkv": one}}, x[:1], W, "qkv")[0], 2.0 * model.rows_8bit(W).sum(-1), rtol=1e-12)
