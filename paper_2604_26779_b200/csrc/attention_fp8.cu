@@ -86,7 +86,6 @@ template <int STAGES>
 __global__ void __launch_bounds__(kThreads, 4) attn_fp8_kernel(const Fp8Args a)
 {
     constexpr int DH = 128, WM = 1, WN = 4;
-    constexpr int CH = DH / 8;                               // 16-byte chunks per fp16 row
     constexpr int kCodeBlk = kBT * DH;                       // the same block as e4m3 codes
     constexpr int kStageBytes = 4 * kCodeBlk * 2;            // 4 blocks, K and V, as codes
     constexpr int ROWS = 16 * WM;

@@ -316,7 +316,8 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
         QkvEpilogue e{Hq, Hkv, dh, R, g.max_blocks_per_seq, g.kv_block_tokens, pos, at<int32_t>(c.buf.state, c.block_table),
                       at<float>(ws, c.rope), k_pool, v_pool};
         if (g.kv_dtype == SPEC_KV_E4M3) { e.kv_fp8 = 1; e.k_scale = g.kv_scale_k; e.v_scale = g.kv_scale_v; }
-        TRY(launch_quantize_rows(M, qkv_k, qkv_in, a8_of(0), a8s_of(0), st));
+        if (qkv_in == nullptr) TRY(launch_rmsnorm_quantize(M, d, res, W.attn_norm, g.rms_eps, a8_of(0), a8s_of(0), st));   // norm fused with the quantiser
+        else TRY(launch_quantize_rows(M, qkv_k, qkv_in, a8_of(0), a8s_of(0), st));
         TIMED(c, CLS_GEMM, launch_gemm8_qkv_tc(M, qkv_k, a8_of(0), a8s_of(0), W.wqkv, W.wqkv_s, at(ws, c.qkv), e, status_word, st));
         AttnArgs a{B, R, Hq, Hkv, dh, g.kv_block_tokens, g.max_blocks_per_seq, at(ws, c.qkv), qkv_n, k_pool, v_pool,
                    at<int32_t>(c.buf.state, c.block_table), pos, at(ws, c.attn_out), Hq * dh, dt, at(ws, c.attn_scratch),
@@ -327,8 +328,7 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
         TRY(launch_quantize_rows(M, Hq * dh, at(ws, c.attn_out), a8_of(1), a8s_of(1), st));
         TIMED(c, CLS_GEMM, launch_gemm8_tc(M, d, Hq * dh, a8_of(1), a8s_of(1), W.wo, W.wo_s, res, d, SPEC_DTYPE_F32, 1, 1.f, nullptr, 0, nullptr, 0,
                                            status_word, st));
-        TRY(launch_rmsnorm(M, d, res, W.mlp_norm, g.rms_eps, at(ws, c.h), d, 0, dt, st));
-        TRY(launch_quantize_rows(M, d, at(ws, c.h), a8_of(2), a8s_of(2), st));
+        TRY(launch_rmsnorm_quantize(M, d, res, W.mlp_norm, g.rms_eps, a8_of(2), a8s_of(2), st));
         TIMED(c, CLS_GEMM, launch_gemm8_swiglu_tc(M, d_ffn, d, a8_of(2), a8s_of(2), W.wgateup, W.wgateup_s, at(ws, c.act), status_word, st));
         TRY(launch_quantize_rows(M, d_ffn, at(ws, c.act), a8_of(3), a8s_of(3), st));
         TIMED(c, CLS_GEMM, launch_gemm8_tc(M, d, d_ffn, a8_of(3), a8s_of(3), W.wdown, W.wdown_s, res, d, SPEC_DTYPE_F32, 1, 1.f, nullptr, 0, nullptr, 0,
@@ -709,19 +709,20 @@ extern "C" spec_status spec_verify(spec_ctx* c, int k, const int32_t* draft_toke
     if (has_tap(g, 0)) TRY(launch_copy_rows_f32_to(M, d, x, at(ws, c->taps), tapw, tap_slot(g, 0) * d, dt, st));
     for (int l = 0; l < g.n_layers; ++l) {
         const LayerPtrs W = layer_ptrs(c->buf.weights, c->layers[l]);
-        TRY(launch_rmsnorm(M, d, x, W.attn_norm, g.rms_eps, at(ws, c->h), d, 0, dt, st));
+        const bool w8 = g.weight_dtype == SPEC_W_E4M3;       // 8-bit projections: the layer body norms and quantises x itself
+        if (!w8) TRY(launch_rmsnorm(M, d, x, W.attn_norm, g.rms_eps, at(ws, c->h), d, 0, dt, st));
         const int pool = l % g.kv_layer_pools;
         char* kp = static_cast<char*>(c->buf.kv) + (size_t)pool * 2 * c->kv_pool_bytes;
-        TRY(run_layer_body(*c, W, g.d_ffn, x, at(ws, c->h), d, B, R, rows.pos, kp, kp + c->kv_pool_bytes, l, st));
+        TRY(run_layer_body(*c, W, g.d_ffn, x, w8 ? nullptr : at(ws, c->h), d, B, R, rows.pos, kp, kp + c->kv_pool_bytes, l, st));
         if (has_tap(g, l + 1)) TRY(launch_copy_rows_f32_to(M, d, x, at(ws, c->taps), tapw, tap_slot(g, l + 1) * d, dt, st));
     }
-    TRY(launch_rmsnorm(M, d, x, at<const float>(c->buf.weights, c->final_norm), g.rms_eps, at(ws, c->h), d, 0, dt, st));
+    if (g.weight_dtype != SPEC_W_E4M3) TRY(launch_rmsnorm(M, d, x, at<const float>(c->buf.weights, c->final_norm), g.rms_eps, at(ws, c->h), d, 0, dt, st));
     // LM head with the row statistics taken in its epilogue; shapes the tile kernel does not take go the two-pass way
     spec_status fused = SPEC_ERR_UNSUPPORTED;
     if (g.weight_dtype == SPEC_W_E4M3) {
         unsigned char* a8 = at<unsigned char>(ws, c->a8) + (kActSlots - 1) * (c->a8.bytes / kActSlots);
         float* a8s = at<float>(ws, c->a8_scale) + (kActSlots - 1) * (c->a8_scale.bytes / kActSlots / 4);
-        TRY(launch_quantize_rows(M, d, at(ws, c->h), a8, a8s, st));
+        TRY(launch_rmsnorm_quantize(M, d, x, at<const float>(c->buf.weights, c->final_norm), g.rms_eps, a8, a8s, st));
         Timed t__(*c, CLS_GEMM, st);
         fused = launch_gemm8_tc(M, g.vocab, d, a8, a8s, at(c->buf.weights, c->lm_head), at<const float>(c->buf.weights, c->lm_head_s),
                                 at(ws, c->logits), g.vocab, SPEC_DTYPE_F32, 0, g.temperature, at<float>(ws, c->splitk), c->splitk.bytes,

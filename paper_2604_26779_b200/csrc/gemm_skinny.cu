@@ -191,7 +191,7 @@ spec_status launch_gemm_skinny(int M, int N, int K, const void* A, int lda, cons
 {
     if (M <= 8) return run_skinny<1, 4>(M, N, K, A, lda, W, C, ldc, out_dtype, accumulate, st);
     if (M <= 16) return run_skinny<2, 4>(M, N, K, A, lda, W, C, ldc, out_dtype, accumulate, st);
-    return run_skinny<4, 3>(M, N, K, A, lda, W, C, ldc, out_dtype, accumulate, st);
+    return SPEC_ERR_UNSUPPORTED;                            // callers ask gemm_skinny_supported first
 }
 
 }  // namespace spec

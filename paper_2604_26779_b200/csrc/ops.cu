@@ -543,6 +543,62 @@ __global__ void __launch_bounds__(256) quantize_rows_kernel(int K, const __nv_bf
     }
 }
 
+
+// RMSNorm of an fp32 row followed by the per-row e4m3 quantisation of its bf16-rounded result, in one kernel: the same
+// values, scale and codes as rmsnorm_kernel<bf16> followed by quantize_rows_kernel (the 16-bit row itself is not written:
+// in a context with 8-bit projections nothing else reads it).  d % 4 == 0.
+__global__ void __launch_bounds__(256) rmsnorm_quantize_kernel(int d, const float* __restrict__ in, const float* __restrict__ w, float eps,
+                                                               unsigned char* __restrict__ codes, float* __restrict__ scales)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int m = blockIdx.x;
+    const float* xr = in + (size_t)m * d;
+    __shared__ float s_part[8];
+    __shared__ float s_max[8];
+    float ss = 0.f;
+    for (int c = threadIdx.x * 4; c < d; c += 256 * 4) {
+        float v[4];
+        Vec4<float>::load(xr + c, v);
+        ss += v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) tot += s_part[i];
+    const float r = rsqrtf(tot / (float)d + eps);
+    float amax = 0.f;
+    for (int c = threadIdx.x * 4; c < d; c += 256 * 4) {
+        float v[4], g[4];
+        Vec4<float>::load(xr + c, v);
+        Vec4<float>::load(w + c, g);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) amax = fmaxf(amax, fabsf(__bfloat162float(__float2bfloat16_rn(v[e] * r * g[e]))));
+    }
+    amax = warp_max(amax);
+    if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    float mx = s_max[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) mx = fmaxf(mx, s_max[i]);
+    const float sc = mx > 0.f ? __fdiv_rn(mx, 448.f) : 1.f;
+    if (threadIdx.x == 0) scales[m] = sc;
+    unsigned char* cr = codes + (size_t)m * d;
+    for (int c = threadIdx.x * 4; c < d; c += 256 * 4) {
+        float v[4], g[4];
+        Vec4<float>::load(xr + c, v);
+        Vec4<float>::load(w + c, g);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = __fdiv_rn(__bfloat162float(__float2bfloat16_rn(v[e] * r * g[e])), sc);
+        unsigned short lo, hi;                               // cvt packs its first source into the upper byte
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(v[1]), "f"(v[0]));
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(v[3]), "f"(v[2]));
+        *reinterpret_cast<uint32_t*>(cr + c) = (uint32_t)lo | ((uint32_t)hi << 16);
+    }
+}
+
 }  // namespace
 
 #define DISPATCH_T(dtype, ...)                                            \
@@ -668,6 +724,14 @@ spec_status launch_quantize_rows(int rows, int K, const void* x_bf16, void* code
     if (rows == 0) return SPEC_OK;
     if (K <= 0 || K % 8 != 0) return SPEC_ERR_SHAPE;
     launch_pdl(quantize_rows_kernel, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales);
+    return launch_status();
+}
+
+spec_status launch_rmsnorm_quantize(int M, int d, const float* in, const float* w, float eps, void* codes, float* scales, cudaStream_t st)
+{
+    if (M == 0) return SPEC_OK;
+    if (d <= 0 || d % 4 != 0) return SPEC_ERR_SHAPE;
+    launch_pdl(rmsnorm_quantize_kernel, dim3(M), dim3(256), 0, st, d, in, w, eps, (unsigned char*)codes, scales);
     return launch_status();
 }
 
