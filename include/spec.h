@@ -15,7 +15,9 @@
  *   - step functions only enqueue work on `stream`; they do not synchronise (spec_get_status does);
  *   - a host-detectable problem returns a negative spec_status and launches nothing; a problem found on
  *     the device is recorded in a status word (first error wins) and never traps;
- *   - a context is not thread-safe.
+ *   - a context is not thread-safe: serialise the calls on one context.  Different contexts may be driven from different
+ *     host threads and on different devices of one process (one-time kernel set-up is kept per device); the stateless
+ *     operators are reentrant.
  *
  * Layouts: a weight matrix is [out][in] row-major; token ids, lengths and tables are int32; logits and
  * probabilities are fp32; activations, weights and KV are bf16 (SPEC_DTYPE_BF16) or fp32 (SPEC_DTYPE_F32).

@@ -322,10 +322,11 @@ spec_status launch_attention_fp8(const AttnArgs& a, cudaStream_t st)
     const int max_chunks = max_chunks_for(a.max_kv_len);
     const PlanView pv = carve_plan(a.scratch, a.B, a.Hkv, 16, a.dh, max_chunks);
     auto kern = attn_fp8_kernel<STAGES>;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    int dev__ = 0;
+    if (configured.needed(&dev__)) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SPEC_ERR_CUDA;
-        configured = true;
+        configured.done(dev__);
     }
     Fp8Args f{(const __nv_bfloat16*)a.q, a.q_row_stride, (const unsigned char*)a.k_pool, (const unsigned char*)a.v_pool,
               a.block_table, a.max_blocks, a.pos, a.R, group, a.Hkv, (__nv_bfloat16*)a.out, a.out_row_stride,

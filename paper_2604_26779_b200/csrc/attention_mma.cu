@@ -396,16 +396,18 @@ __global__ void __launch_bounds__(128) attn_merge_kernel(int B, int rows_alloc, 
     }
 }
 
-int g_sm_count = 0;
 int sm_count()
 {
-    if (g_sm_count == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (g_sm_count <= 0) g_sm_count = 148;
+    static std::atomic<int> cached[64];                      // per device ordinal; 0 = not asked yet
+    int dev = 0;
+    cudaGetDevice(&dev);
+    int n = cached[dev & 63].load(std::memory_order_relaxed);
+    if (n == 0) {
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+        cached[dev & 63].store(n, std::memory_order_relaxed);
     }
-    return g_sm_count;
+    return n;
 }
 
 template <int DH, int WM, int WN>
@@ -415,10 +417,11 @@ spec_status run_mma(const MmaArgs& m, int B, bool plan, int max_chunks, cudaStre
     constexpr int smem = STAGES * (4 * kBT * DH * 2 * 2);
     static_assert(smem >= WN * 16 * WM * (DH + 2) * 4, "merge buffer fits in the stages");
     auto kern = attn_mma_kernel<DH, WM, WN, STAGES>;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    int dev__ = 0;
+    if (configured.needed(&dev__)) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SPEC_ERR_CUDA;
-        configured = true;
+        configured.done(dev__);
     }
     if (plan) {
         attn_plan_kernel<<<1, kPlanThreads, 0, st>>>(B, m.R, m.pos, m.Hkv, 2 * sm_count(), B * max_chunks, m.pv);

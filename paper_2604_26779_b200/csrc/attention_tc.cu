@@ -516,12 +516,13 @@ spec_status launch_attention_tc(const AttnArgs& a, cudaStream_t st)
     if (a.scratch_bytes < attention_mma_scratch_bytes(a.B, a.R, a.Hq, a.Hkv, a.dh, a.max_kv_len)) return SPEC_ERR_SHAPE;
     const int max_chunks = max_chunks_for(a.max_kv_len);
     const PlanView pv = carve_plan(a.scratch, a.B, a.Hkv, rows_alloc, a.dh, max_chunks);
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    int dev__ = 0;
+    if (configured.needed(&dev__)) {
         if (cudaFuncSetAttribute(attn_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc) != cudaSuccess ||
             cudaFuncSetAttribute(attn_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTc) != cudaSuccess)
             return SPEC_ERR_CUDA;
-        configured = true;
+        configured.done(dev__);
     }
     // the pools as matrices of 128-column rows ((block, head, token) flattened); one box = 64 columns x 16 tokens
     CUtensorMap mk, mv;

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/spec.h"
 
 namespace spec {
@@ -23,12 +25,28 @@ __device__ __forceinline__ void set_status(int32_t* status, int code, int detail
     } while (0)
 
 // Number of kernels this library has launched in this process (every launcher reports through launch_status()).
-long long& launch_counter();
+std::atomic<long long>& launch_counter();
 inline spec_status launch_status(int n_launched = 1)
 {
     launch_counter() += n_launched;
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }
+
+// Kernel attributes (dynamic shared memory limits) are set per device: one bit per device ordinal records where a call site
+// has done its one-time set-up, so a process that drives several devices configures each of them, and two host threads that
+// arrive together at worst both do the (idempotent) set-up.
+struct PerDeviceOnce {
+    std::atomic<unsigned long long> seen{0};
+    // true when the current device still needs the set-up; call done() after it succeeded
+    bool needed(int* dev_out)
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        *dev_out = dev;
+        return (seen.load(std::memory_order_acquire) & (1ull << (dev & 63))) == 0;
+    }
+    void done(int dev) { seen.fetch_or(1ull << (dev & 63), std::memory_order_release); }
+};
 
 // Programmatic dependent launch.  A kernel launched through launch_pdl may be scheduled before the kernel in front of it
 // in the stream has finished (as soon as that one has called pdl_trigger, or has exited), which hides the launch latency

@@ -927,13 +927,13 @@ spec::GemmScratch& spec::gemm_scratch()
     return s;
 }
 
-long long& spec::launch_counter()
+std::atomic<long long>& spec::launch_counter()
 {
-    static long long n = 0;
+    static std::atomic<long long> n{0};
     return n;
 }
 
-extern "C" int64_t spec_launch_count(void) { return (int64_t)spec::launch_counter(); }
+extern "C" int64_t spec_launch_count(void) { return (int64_t)spec::launch_counter().load(std::memory_order_relaxed); }
 
 extern "C" spec_status spec_set_timing(spec_ctx* c, uint32_t mask)
 {

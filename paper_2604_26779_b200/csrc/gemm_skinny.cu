@@ -166,10 +166,11 @@ spec_status run_skinny(int M, int N, int K, const void* A, int lda, const void* 
 {
     constexpr int smem = STAGES * 4 * (kRows * 128 + 8 * NT * 128);
     auto kern = gemm_skinny_kernel<NT, STAGES>;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    int dev__ = 0;
+    if (configured.needed(&dev__)) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SPEC_ERR_CUDA;
-        configured = true;
+        configured.done(dev__);
     }
     launch_pdl(kern, dim3((N + kRows - 1) / kRows), dim3(kThreads), (size_t)smem, st, M, N, K, (const __nv_bfloat16*)A, lda,
                (const __nv_bfloat16*)W, C, ldc, out_dtype == SPEC_DTYPE_F32 ? 1 : 0, accumulate);

@@ -46,3 +46,46 @@ def test_two_runs_agree_bit_for_bit(name, cfg_over, draft, n_layers, vocab):
         assert torch.equal(pa.view(torch.uint8), pb.view(torch.uint8))
     assert torch.equal(a[2], b[2])
     assert int(a[2].sum()) > int(sum(lens))                                     # tokens were committed
+
+
+def test_two_contexts_on_two_host_threads_match_the_single_threaded_run():
+    """Different contexts may be driven from different host threads (each on its own stream): the calls hold no shared
+    mutable state beyond per-device one-time set-up, so every context produces the bits it produces alone."""
+    import threading
+    from paper_2604_26779_b200 import workloads
+    lens = [300, 37, 4096, 900, 1, 260, 64, 2000]
+    kw = dict(k=3, draft="eagle3", steps_budget=6, n_layers=2, vocab=2048,      # as run_once builds it: the same pools, the same synthetic cache
+              cfg_over=dict(d_model=512, n_q_heads=8, n_kv_heads=2, head_dim=128, d_ffn=1024))
+    alone = run_once("c3", kw["cfg_over"], "eagle3", lens, 3, 4, 2, 2048)
+    engines = [workloads.build_dense_workload("c3", lens=np.array(lens, np.int32), **kw)[0] for _ in range(2)]
+    torch.cuda.synchronize()                                     # the weights were filled on the default stream
+    results, errors = [None, None], []
+
+    def work(i):
+        try:
+            torch.cuda.set_device(0)
+            with torch.cuda.stream(torch.cuda.Stream()):
+                eng = engines[i]
+                workloads.bootstrap(eng)
+                outs = []
+                for _ in range(4):
+                    workloads.spec_step(eng, 3)
+                    outs.append((eng.logits(3).clone(), eng.out_tokens(3).clone(), eng.n_emitted().clone()))
+                torch.cuda.current_stream().synchronize()
+                results[i] = outs
+        except Exception as e:                                   # surfaced in the main thread below
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for outs in results:
+        for (la, ta, na), (lb, tb, nb) in zip(alone[0], outs):
+            assert torch.equal(na, nb) and torch.equal(ta, tb)
+            assert torch.equal(la.view(torch.int32), lb.view(torch.int32))
+    for eng in engines:
+        assert eng.status().device_status == 0
+        eng.close()
