@@ -124,7 +124,7 @@ def cpu_oracle_sample(eng, info, k, n_layers_sample, step_index):
     # split the forward time: time the head alone (final norm + LM head over k+1 rows) to scale only the layer part
     from oracle import model
     t1 = time.perf_counter()
-    model.rmsnorm(r["final"], W["final_norm"], cfg["rms_eps"]) @ np.asarray(W["lm_head"], np.float64).T
+    model.proj(cfg, model.rmsnorm(r["final"], W["final_norm"], cfg["rms_eps"]), W["lm_head"], "lm_head")
     head_s = time.perf_counter() - t1
     layers_s = max(r["seconds_forward"] - head_s, 0.0)
     total = layers_s * (L / n_layers_sample) + head_s + r["seconds_sample"]
