@@ -33,7 +33,9 @@ def rows_of(qr, r0, r1):
 def compare_rows(dev, ref, what, min_equal, abs_rms=0.0):
     """Device rows against the oracle's: scales within one bf16 step of the row maximum, values within one e4m3 step of
     the element (at most 2^-3 of it; sub-normal codes: 2^-9 of the scale) plus the effect of that scale difference, plus
-    abs_rms times the row's RMS where the 16-bit input itself carries an absolute error (attention probabilities in bf16)."""
+    abs_rms times the row's RMS where the 16-bit input itself carries an absolute error: the attention output, whose
+    probabilities and queries are bf16 on the device (each about 2^-9 relative, together about 3e-3 of the row's RMS as a
+    standard deviation; the bar of 2e-2 is six of those, for the maximum over tens of thousands of elements)."""
     assert np.all(np.abs(dev.scales - ref.scales) <= 2.0 ** -7 * ref.scales), what
     a, b = dev.values(), ref.values()
     tol = 0.135 * np.abs(b) + 2.0 ** -9 * ref.scales[:, None] + abs_rms * np.sqrt(np.mean(b * b, -1, keepdims=True))
@@ -101,7 +103,7 @@ def test_w_fp8_verify_projection_by_projection(n_layers, head_dim, kv_fp8):
                 err = np.abs(g_ - ref) / (np.abs(ref) + 1e-3 * np.abs(ref).max())
                 worst_kv = max(worst_kv, float(err.max()))
         # -- attention output as the O projection consumed it (q went through the same epilogue as k)
-        equal["o"] = min(equal["o"], compare_rows(rows_of(dev["o"], r0, r1), record["o"], "o", 0.80, abs_rms=8e-3))
+        equal["o"] = min(equal["o"], compare_rows(rows_of(dev["o"], r0, r1), record["o"], "o", 0.80, abs_rms=2e-2))
         # -- SwiGLU of the forced gate/up input, as the down projection consumed it
         equal["down"] = min(equal["down"], compare_rows(rows_of(dev["down"], r0, r1), record["down"], "down", 0.97))
         if n_layers == 1:
@@ -122,4 +124,64 @@ def test_w_fp8_verify_projection_by_projection(n_layers, head_dim, kv_fp8):
           f"logits {worst_l:.2e}, equal codes {equal}")
     assert worst_kv < 2.0 ** -7          # bf16 rounding of the stored value (2^-9 .. 2^-8) plus fp32 accumulation
     assert worst_x < 1e-5 and worst_l < 1e-5
+    eng.close()
+
+
+def test_w_fp8_full_size_sampled():
+    """The benchmark's configuration with 8-bit projections (8B shape, 32 layers, B = 256, cache lengths ~U[1024,16384], k = 3):
+    sampled sequences, the last layer and the LM head, with the device's own quantised rows forced into the oracle."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60e9:
+        pytest.skip("needs a device with > 60 GB free")
+    from paper_2604_26779_b200 import workloads
+    k, B = 3, 256
+    eng, info = workloads.build_dense_workload("c3", B=B, k=k, steps_budget=8, cfg_over=dict(w_fp8=True))
+    cfg = info["cfg"]
+    L, d, V, F = cfg["n_layers"], cfg["d_model"], cfg["vocab"], cfg["d_ffn"]
+    Hq, dh = cfg["n_q_heads"], cfg["head_dim"]
+    assert L == 32 and d == 4096 and V == 128256 and cfg.get("w_fp8")
+    workloads.bootstrap(eng)
+    workloads.spec_step(eng, k)
+    seq_len = eng.seq_len().cpu().numpy().copy()
+    eng.draft(k)
+    eng.verify(k)
+    assert eng.status().device_status == 0
+    table = eng.block_table().cpu().numpy().copy()
+    R, M = k + 1, B * (k + 1)
+    W = harness.device_weights(eng, cfg)
+    lw = W["layers"][L - 1]
+    worst_kv = worst_l = 0.0
+    low = {"o": 1.0, "down": 1.0, "lm_head": 1.0}
+    for b in (0, 101, 255):
+        r0, r1 = b * R, (b + 1) * R
+        n_past = int(seq_len[b])
+        forced = {}
+        for s, (slot, K) in {"qkv": (0, d), "o": (1, Hq * dh), "gateup": (2, d), "down": (3, F), "lm_head": (4, d)}.items():
+            codes = eng.tensor("ACT_CODES", slot, torch.uint8)[: M * K].view(M, K)[r0:r1].cpu().numpy()
+            scales = eng.tensor("ACT_SCALES", slot, torch.float32)[r0:r1].cpu().numpy()
+            forced[s] = model.QuantRows(codes, scales)
+        record = {}
+        cfg_f = dict(cfg, forced=forced, record=record)
+        past = harness.LazyPast(eng, cfg, table[b], n_past, info["kv_pools"], L)[L - 1]
+        pos = np.arange(n_past, n_past + R)
+        _, k_new, v_new = model.decoder_layer(cfg_f, lw, np.zeros((R, d)), pos, past[0], past[1])
+        got = harness.LazyPast(eng, cfg, table[b], n_past + R, info["kv_pools"], L)[L - 1]
+        for g_, ref in ((got[0][n_past:], k_new), (got[1][n_past:], v_new)):
+            worst_kv = max(worst_kv, float((np.abs(g_ - ref) / (np.abs(ref) + 1e-3 * np.abs(ref).max())).max()))
+        low["o"] = min(low["o"], compare_rows(forced["o"], record["o"], "o", 0.80, abs_rms=2e-2))
+        low["down"] = min(low["down"], compare_rows(forced["down"], record["down"], "down", 0.97))
+        hidden = eng.tensor("HIDDEN", 0, torch.float32, (M, d))[r0:r1].cpu().numpy().astype(np.float64)
+        rec2 = {}
+        ref_logits = model.proj(dict(cfg, forced={"lm_head": forced["lm_head"]}, record=rec2),
+                                model.rmsnorm(hidden, W["final_norm"], cfg["rms_eps"]), W["lm_head"], "lm_head")
+        low["lm_head"] = min(low["lm_head"], compare_rows(forced["lm_head"], rec2["lm_head"], "lm_head", 0.99))
+        logits = eng.logits(k)[b].cpu().numpy().reshape(R, V).astype(np.float64)
+        worst_l = max(worst_l, float((np.abs(logits - ref_logits).max(-1) / np.abs(ref_logits).max(-1)).max()))
+    print(f"w_fp8 full size: cache entries {worst_kv:.2e}, logits {worst_l:.2e}, equal codes {low}")
+    assert worst_kv < 2.0 ** -7 and worst_l < 1e-5
     eng.close()
