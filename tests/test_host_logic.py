@@ -106,3 +106,27 @@ def test_k_policy_arithmetic():
             ks = list(range(1, 8))
             rates = [rollout.expected_tokens_per_step(a, k) / cost(B, k) for k in ks]
             assert rollout.choose_k(a, B, cost, ks) == ks[int(np.argmax(rates))]
+
+
+def test_sizes_and_refusals_with_8bit_projections():
+    """SPEC_W_E4M3: one byte per projection weight + one fp32 scale per weight row (embedding, norms and the draft head stay
+    16-bit); refused for the combinations the 8-bit path does not cover."""
+    cfg = inputs.model_config("c3")
+    kw = dict(draft_kind="eagle3", k_max=3, max_batch=256, kv_num_blocks=1000, max_blocks_per_seq=64, kv_layer_pools=16)
+    code16, s16 = sizes_of(engine.make_spec_config(cfg, **kw))
+    code8, s8 = sizes_of(engine.make_spec_config(cfg, w_fp8=True, **kw))
+    assert code16 == 0 and code8 == 0
+    per_layer = 4096 * 6144 + 4096 * 4096 + 3 * 4096 * 14336
+    rows = 32 * (6144 + 4096 + 2 * 14336 + 4096) + 128256                        # one scale per weight row
+    want = 32 * per_layer + 128256 * 4096 + rows * 4 + 128256 * 4096 * 2       # codes + scales + the 16-bit embedding
+    assert want <= s8.weights_bytes <= want + (32 * 10 + 4) * 256 + 33 * 2 * 4096 * 4 + 4096
+    assert s8.draft_weights_bytes == s16.draft_weights_bytes and s8.kv_bytes == s16.kv_bytes
+    assert s8.workspace_bytes >= s16.workspace_bytes + 5 * 1024 * 14336          # five quantised-activation slots
+    for change in (dict(draft_kind=B.SPEC_DRAFT_MTP, draft_d_ffn=14336),
+                   dict(dtype=B.SPEC_DTYPE_F32),
+                   dict(n_experts=8, experts_top_k=2, d_expert_ffn=1536), dict(weight_dtype=7)):
+        sc = engine.make_spec_config(cfg, w_fp8=True, **kw)
+        for k, v in change.items():
+            setattr(sc, k, v)
+        got, _ = sizes_of(sc)
+        assert got == -3, (change, got)
