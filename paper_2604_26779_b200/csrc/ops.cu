@@ -499,37 +499,50 @@ __global__ void __launch_bounds__(256) permute_rows_kernel(int R, size_t row_byt
 
 // Per-row e4m3 quantisation of a bf16 matrix: one CTA per row.  scale = amax / 448 in fp32 (1 for a zero row), codes =
 // round_e4m3(x / scale) with an exact fp32 division, round to nearest even, saturating: the same steps as the oracle's.
+template <int CHUNKS>
 __global__ void __launch_bounds__(256) quantize_rows_kernel(int K, const __nv_bfloat16* __restrict__ x, unsigned char* __restrict__ codes,
                                                             float* __restrict__ scales)
 {
+    // CHUNKS > 0: the row (K <= 256 * 8 * CHUNKS) stays in registers between the maximum and the conversion, one global read;
+    // CHUNKS == 0: any K, the row is read twice (the second time from cache)
     pdl_trigger();
     pdl_wait();
     __shared__ float s_w[8];
-    __shared__ float s_scale;
     const int row = blockIdx.x;
     const __nv_bfloat16* xr = x + (size_t)row * K;
+    constexpr int NV = CHUNKS > 0 ? CHUNKS : 1;
+    uint4 held[NV];
     float amax = 0.f;
-    for (int i = threadIdx.x * 8; i < K; i += 256 * 8) {
-        const uint4 v = *reinterpret_cast<const uint4*>(xr + i);
-        const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+    if constexpr (CHUNKS > 0) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) amax = fmaxf(amax, fmaxf(fabsf(__low2float(p[e])), fabsf(__high2float(p[e]))));
+        for (int j = 0; j < CHUNKS; ++j) {
+            const int i = (j * 256 + threadIdx.x) * 8;
+            held[j] = i < K ? *reinterpret_cast<const uint4*>(xr + i) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int j = 0; j < CHUNKS; ++j) {
+            const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&held[j]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) amax = fmaxf(amax, fmaxf(fabsf(__low2float(p[e])), fabsf(__high2float(p[e]))));
+        }
+    } else {
+        for (int i = threadIdx.x * 8; i < K; i += 256 * 8) {
+            const uint4 v = *reinterpret_cast<const uint4*>(xr + i);
+            const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) amax = fmaxf(amax, fmaxf(fabsf(__low2float(p[e])), fabsf(__high2float(p[e]))));
+        }
     }
     amax = warp_max(amax);
     if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = amax;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        float m = s_w[0];
-        for (int w = 1; w < 8; ++w) m = fmaxf(m, s_w[w]);
-        const float sc = m > 0.f ? __fdiv_rn(m, 448.f) : 1.f;
-        s_scale = sc;
-        scales[row] = sc;
-    }
-    __syncthreads();
-    const float sc = s_scale;
+    float m = s_w[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) m = fmaxf(m, s_w[w]);
+    const float sc = m > 0.f ? __fdiv_rn(m, 448.f) : 1.f;
+    if (threadIdx.x == 0) scales[row] = sc;
     unsigned char* cr = codes + (size_t)row * K;
-    for (int i = threadIdx.x * 8; i < K; i += 256 * 8) {
-        const uint4 v = *reinterpret_cast<const uint4*>(xr + i);
+    auto convert = [&](const uint4& v, int i) {
         const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
         uint32_t w[2];
 #pragma unroll
@@ -540,9 +553,17 @@ __global__ void __launch_bounds__(256) quantize_rows_kernel(int K, const __nv_bf
             w[h] = (uint32_t)lo | ((uint32_t)hi << 16);
         }
         *reinterpret_cast<uint2*>(cr + i) = make_uint2(w[0], w[1]);
+    };
+    if constexpr (CHUNKS > 0) {
+#pragma unroll
+        for (int j = 0; j < CHUNKS; ++j) {
+            const int i = (j * 256 + threadIdx.x) * 8;
+            if (i < K) convert(held[j], i);
+        }
+    } else {
+        for (int i = threadIdx.x * 8; i < K; i += 256 * 8) convert(*reinterpret_cast<const uint4*>(xr + i), i);
     }
 }
-
 
 // RMSNorm of an fp32 row followed by the per-row e4m3 quantisation of its bf16-rounded result, in one kernel: the same
 // values, scale and codes as rmsnorm_kernel<bf16> followed by quantize_rows_kernel (the 16-bit row itself is not written:
@@ -723,7 +744,9 @@ spec_status launch_quantize_rows(int rows, int K, const void* x_bf16, void* code
 {
     if (rows == 0) return SPEC_OK;
     if (K <= 0 || K % 8 != 0) return SPEC_ERR_SHAPE;
-    launch_pdl(quantize_rows_kernel, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales);
+    if (K <= 256 * 8 * 2)      launch_pdl(quantize_rows_kernel<2>, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales);
+    else if (K <= 256 * 8 * 8) launch_pdl(quantize_rows_kernel<8>, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales);
+    else                       launch_pdl(quantize_rows_kernel<0>, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales);
     return launch_status();
 }
 
