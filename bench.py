@@ -440,7 +440,7 @@ def main():
                     help="c3 only: 8-bit (e4m3) KV cache, scales 1/16 - a reduced-precision variant, reported under its own "
                          "metric name and never the headline")
     ap.add_argument("--w-fp8", action="store_true",
-                    help="c3 only: the target's projections and LM head in 8-bit (e4m3) with one scale per weight row and per "
+                    help="c3 / c4: the target's projections and LM head in 8-bit (e4m3) with one scale per weight row and per "
                          "activation row - a reduced-precision variant, reported under its own metric name and never the headline")
     ap.add_argument("--k-sweep", default=None,
                     help="comma-separated draft lengths, e.g. 1,3,5,7: times the c3 step at each k on one engine built for the "
@@ -500,7 +500,7 @@ def main():
         lens = inputs.make_seq_lens_lognormal(B, 4096, float(np.log(2.0)), 16, 32768, replicas.replica_seed(rank, 4))
         eng, info = workloads.build_dense_workload("c4", lens=lens, k=k, n_layers=args.layers, kv_pools=args.kv_pools, draft="mtp",
                                                    steps_budget=steps_budget, device=f"cuda:{local}",
-                                                   seed=replicas.replica_seed(rank, 4))
+                                                   seed=replicas.replica_seed(rank, 4), cfg_over=dict(w_fp8=True) if args.w_fp8 else None)
         wl_name = "c4: 8B dense verify + MTP head (one decoder layer, shared LM head), cache lengths lognormal(median 4096, sigma ln 2, clip [16, 32768])"
     else:
         lens = np.full(B, 8192, np.int32)
@@ -531,7 +531,7 @@ def main():
         config["draft_vocab"] = args.draft_vocab
     if args.workload == "c3" and args.kv_fp8:
         config["kv_cache"] = "e4m3 codes, scales 1/16 (REDUCED PRECISION: not the headline configuration)"
-    if args.workload == "c3" and args.w_fp8:
+    if args.workload in ("c3", "c4") and args.w_fp8:
         config["weights"] = "target projections and LM head as e4m3 codes with per-row scales (REDUCED PRECISION: not the headline configuration)"
     if args.workload != "c3":
         args.no_cpu_baseline = True

@@ -95,7 +95,8 @@ typedef struct {
                                 /* *_SCALE tensors; code = round_e4m3(w / scale), scale = amax(row) / 448), activations are */
                                 /* quantised the same way per row on the fly, and the products run on the 8-bit tensor-core */
                                 /* path with fp32 accumulation (the precision of the paper's simulator, Section 5.1).       */
-                                /* bf16 dense models, draft kind NONE / EAGLE3 / NGRAM; a reduced-precision mode            */
+                                /* bf16 dense models; the draft heads' own weights stay 16-bit (the MTP head scores with    */
+                                /* the target's 8-bit LM head); a reduced-precision mode                                    */
 } spec_config;
 
 /* Byte sizes of the caller-owned device arenas for a configuration. */
@@ -158,7 +159,8 @@ enum {
     SPEC_T_MOE_IDS,             /* [B*(k+1)][experts_top_k] int32 selected experts, best first         */
     SPEC_T_MOE_WTS,             /* [B*(k+1)][experts_top_k] fp32 renormalised mixture weights          */
     /* SPEC_W_E4M3 only: the quantised rows a projection consumed in the last pass.  `layer` names the     */
-    /* slot: 0 QKV, 1 O, 2 gate/up, 3 down (of the last layer that ran), 4 LM head.  Row r of a slot has   */
+    /* slot: 0 QKV, 1 O, 2 gate/up, 3 down (of the last layer that ran), 4 LM head (the last LM-head     */
+    /* product: the target's, or an MTP head's last pass).  Row r of a slot has                            */
     /* K codes at byte r*K (K = that projection's input width) and its scale at ACT_SCALES[r].             */
     SPEC_T_ACT_CODES,           /* uint8 e4m3 codes, rows back to back                                 */
     SPEC_T_ACT_SCALES           /* fp32 [rows]                                                         */

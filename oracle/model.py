@@ -330,7 +330,7 @@ def mtp_slots(cfg, W, H, g, tokens_next, pos, past_k=None, past_v=None):
 
 
 def mtp_logits(cfg, W, h):
-    return rmsnorm(h, W["final_norm"], cfg["rms_eps"]) @ np.asarray(W["lm_head"], F64).T
+    return proj(cfg, rmsnorm(h, W["final_norm"], cfg["rms_eps"]), W["lm_head"], "lm_head")     # the target's LM head, in its format
 
 
 def draft_propose(cfg, W, H, kind, true_feat, tokens, k, sample_fn, past_k=None, past_v=None, first_slot=0):

@@ -96,7 +96,7 @@ spec_status check_config(const spec_config* c)
                                          !(c->kv_scale_k > 0.f) || !(c->kv_scale_v > 0.f) ||
                                          (c->k_max + 1) * (c->n_q_heads / c->n_kv_heads) > 16)) return SPEC_ERR_UNSUPPORTED;
     if (c->weight_dtype != SPEC_W_MODEL &&
-        (c->weight_dtype != SPEC_W_E4M3 || c->dtype != SPEC_DTYPE_BF16 || c->n_experts > 0 || c->draft_kind == SPEC_DRAFT_MTP ||
+        (c->weight_dtype != SPEC_W_E4M3 || c->dtype != SPEC_DTYPE_BF16 || c->n_experts > 0 ||
          c->d_model % 128 != 0 || c->d_ffn % 128 != 0 || (c->n_q_heads * c->head_dim) % 128 != 0 || (c->head_dim != 64 && c->head_dim != 128) ||
          c->vocab % 8 != 0))
         return SPEC_ERR_UNSUPPORTED;
@@ -882,13 +882,28 @@ extern "C" spec_status spec_draft(spec_ctx* c, int k, void* stream)
         // logits of this slot, their statistics, and the draft token d_{j+1} ~ q_{j+1} (stream-1 uniform, slot j)
         const float* nf = eagle ? at<const float>(dw, c->d_norm_f) : at<const float>(c->buf.weights, c->final_norm);
         const void* lm = eagle ? at<const void>(dw, c->d_lm_head) : at<const void>(c->buf.weights, c->lm_head);
-        TRY(launch_rmsnorm(B, d, hid, nf, g.rms_eps, at(ws, c->h), d, 0, dt, st));
+        const bool lm8 = !eagle && g.weight_dtype == SPEC_W_E4M3;    // the MTP head scores with the target's (8-bit) LM head
         spec_status fused = SPEC_ERR_UNSUPPORTED;
-        if (!g.draft_greedy)
+        if (lm8) {
+            unsigned char* a8 = at<unsigned char>(ws, c->a8) + (kActSlots - 1) * (c->a8.bytes / kActSlots);
+            float* a8s = at<float>(ws, c->a8_scale) + (kActSlots - 1) * (c->a8_scale.bytes / kActSlots / 4);
+            TRY(launch_rmsnorm_quantize(B, d, hid, nf, g.rms_eps, a8, a8s, st));
+            fused = launch_gemm8_tc(B, Vd, d, a8, a8s, lm, at<const float>(c->buf.weights, c->lm_head_s), dlog + (size_t)j * Vd, k * Vd,
+                                    SPEC_DTYPE_F32, 0, g.temperature, g.draft_greedy ? nullptr : at<float>(ws, c->splitk), c->splitk.bytes,
+                                    dstats + 2 * j, k, status, st);
+            if (fused != SPEC_OK && fused != SPEC_ERR_UNSUPPORTED) return fused;
+            if (g.draft_greedy) fused = SPEC_ERR_UNSUPPORTED;        // no statistics wanted; the logits are written
+        } else {
+            TRY(launch_rmsnorm(B, d, hid, nf, g.rms_eps, at(ws, c->h), d, 0, dt, st));
+        }
+        if (!g.draft_greedy && !lm8)
             fused = launch_gemm_lm_head_stats(B, Vd, d, at(ws, c->h), d, lm, dlog + (size_t)j * Vd, k * Vd, dt, g.temperature,
                                               at<float>(ws, c->splitk), c->splitk.bytes, dstats + 2 * j, k, status, st);
-        if (fused == SPEC_ERR_UNSUPPORTED) TRY(launch_gemm(B, Vd, d, at(ws, c->h), d, lm, dlog + (size_t)j * Vd, k * Vd, dt, SPEC_DTYPE_F32, 0, st));
-        else TRY(fused);
+        if (fused == SPEC_ERR_UNSUPPORTED) {
+            if (!lm8) TRY(launch_gemm(B, Vd, d, at(ws, c->h), d, lm, dlog + (size_t)j * Vd, k * Vd, dt, SPEC_DTYPE_F32, 0, st));
+        } else {
+            TRY(fused);
+        }
         int32_t* tok_out = mapped ? dred + j : dtoks + j;          // reduced ids first when the head has its own vocabulary
         if (g.draft_greedy) {
             TRY(launch_argmax_rows(B, Vd, dlog + (size_t)j * Vd, (size_t)k * Vd, tok_out, kstride, st));

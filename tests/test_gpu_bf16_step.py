@@ -51,7 +51,8 @@ def draft_head_weights(eng, cfg, kind):
                                                            ("eagle3", 7, 64, None, False), ("eagle3", 5, 128, None, False),
                                                            ("mtp", 7, 128, None, False), ("eagle3", 3, 128, (1.0, 1.0), False),
                                                            ("mtp", 3, 128, (0.05, 0.03), False), ("eagle3", 3, 128, None, True),
-                                                           ("eagle3", 3, 128, (1.0, 1.0), True)])
+                                                           ("eagle3", 3, 128, (1.0, 1.0), True),
+                                                           ("mtp", 2, 128, None, True)])
 def test_bf16_steps_stage_by_stage(kind, k, head_dim, kv_fp8, w_fp8):
     """head_dim 64: 16 or 32 query rows per KV head on the register-fragment attention kernel; head_dim 128 with k = 5 / 7:
     24 / 32 rows on the tcgen05 kernel, including the draft head's first pass, whose rows past the committed count carry
@@ -75,6 +76,7 @@ def test_bf16_steps_stage_by_stage(kind, k, head_dim, kv_fp8, w_fp8):
         # with the device's own rows, in test_gpu_w_fp8.py.  Draft, sampler and bookkeeping bars are unchanged.
         over["w_fp8"] = True
     logit_bar = 0.25 if w_fp8 else 2e-2
+    draft_bar = 0.25 if (w_fp8 and kind == "mtp") else 2e-2      # the MTP head scores with the 8-bit LM head: the same step-function drift
     n_layers = 3
     lens = np.array([5, 40, 100, 17, 300], np.int32)
     if many:
@@ -155,5 +157,5 @@ def test_bf16_steps_stage_by_stage(kind, k, head_dim, kv_fp8, w_fp8):
         k_prev = k
     print(f"bf16 {kind} k={k} dh={head_dim} kv_fp8={kv_fp8} w_fp8={w_fp8}: draft logits {worst_d:.2e}, verify logits {worst_v:.2e}, "
           f"boundary cases {boundary}")
-    assert worst_d < 2e-2 and worst_v < logit_bar and boundary <= 2
+    assert worst_d < draft_bar and worst_v < logit_bar and boundary <= 2
     eng.close()

@@ -185,3 +185,29 @@ def test_w_fp8_full_size_sampled():
     print(f"w_fp8 full size: cache entries {worst_kv:.2e}, logits {worst_l:.2e}, equal codes {low}")
     assert worst_kv < 2.0 ** -7 and worst_l < 1e-5
     eng.close()
+
+
+def test_w_fp8_mtp_head_scores_with_the_8bit_lm_head():
+    """The MTP head's logits are the target's LM head applied to its own hidden state: with 8-bit projections that product
+    takes the head's rows quantised per row; the last pass's rows stay in slot 4 until the verify pass overwrites them."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_26779_b200 import workloads
+    k = 3
+    over = dict(d_model=512, n_q_heads=8, n_kv_heads=2, head_dim=128, d_ffn=1024, w_fp8=True)
+    lens = np.array([5, 40, 100, 17, 300, 64, 33], np.int32)
+    eng, info = workloads.build_dense_workload("c3", lens=lens, k=k, draft="mtp", steps_budget=8, n_layers=2, vocab=2048, cfg_over=over)
+    cfg = dict(info["cfg"], n_layers=2)
+    B, d, V = eng.B, cfg["d_model"], cfg["vocab"]
+    W = harness.device_weights(eng, cfg)
+    workloads.bootstrap(eng)
+    workloads.spec_step(eng, k)
+    eng.draft(k)
+    assert eng.status().device_status == 0
+    rows = act_rows(eng, 4, B, d)
+    dlog = eng.draft_logits(k).cpu().numpy().astype(np.float64)[:, k - 1]
+    ref = model.proj(dict(cfg, forced={"lm_head": rows}), np.zeros((B, d)), W["lm_head"], "lm_head")
+    err = float((np.abs(dlog - ref).max(-1) / np.abs(ref).max(-1)).max())
+    print(f"w_fp8 MTP head: last pass logits {err:.2e}")
+    assert err < 1e-5
+    eng.close()

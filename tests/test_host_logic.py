@@ -122,8 +122,9 @@ def test_sizes_and_refusals_with_8bit_projections():
     assert want <= s8.weights_bytes <= want + (32 * 10 + 4) * 256 + 33 * 2 * 4096 * 4 + 4096
     assert s8.draft_weights_bytes == s16.draft_weights_bytes and s8.kv_bytes == s16.kv_bytes
     assert s8.workspace_bytes >= s16.workspace_bytes + 5 * 1024 * 14336          # five quantised-activation slots
-    for change in (dict(draft_kind=B.SPEC_DRAFT_MTP, draft_d_ffn=14336),
-                   dict(dtype=B.SPEC_DTYPE_F32),
+    sc = engine.make_spec_config(cfg, w_fp8=True, **dict(kw, draft_kind="mtp", draft_d_ffn=14336))
+    assert sizes_of(sc)[0] == 0                                                  # the MTP head scores with the 8-bit LM head
+    for change in (dict(dtype=B.SPEC_DTYPE_F32),
                    dict(n_experts=8, experts_top_k=2, d_expert_ffn=1536), dict(weight_dtype=7)):
         sc = engine.make_spec_config(cfg, w_fp8=True, **kw)
         for k, v in change.items():
