@@ -440,7 +440,7 @@ def main():
                     help="c3 only: 8-bit (e4m3) KV cache, scales 1/16 - a reduced-precision variant, reported under its own "
                          "metric name and never the headline")
     ap.add_argument("--w-fp8", action="store_true",
-                    help="c3 / c4: the target's projections and LM head in 8-bit (e4m3) with one scale per weight row and per "
+                    help="c3 / c4 / c5: the target's projections (experts included; the router stays 16-bit) and LM head in 8-bit (e4m3) with one scale per weight row and per "
                          "activation row - a reduced-precision variant, reported under its own metric name and never the headline")
     ap.add_argument("--k-sweep", default=None,
                     help="comma-separated draft lengths, e.g. 1,3,5,7: times the c3 step at each k on one engine built for the "
@@ -506,7 +506,7 @@ def main():
         lens = np.full(B, 8192, np.int32)
         eng, info = workloads.build_dense_workload("c5", lens=lens, k=k, draft="none", kv_pools=args.kv_pools,
                                                    steps_budget=steps_budget, device=f"cuda:{local}",
-                                                   seed=replicas.replica_seed(rank, 5))
+                                                   seed=replicas.replica_seed(rank, 5), cfg_over=dict(w_fp8=True) if args.w_fp8 else None)
         g = torch.Generator(device=f"cuda:{local}"); g.manual_seed(5)
         ext_drafts = (torch.randint(0, info["cfg"]["vocab"], (B, k), dtype=torch.int32, device="cuda", generator=g),
                       torch.randn((B, k, info["cfg"]["vocab"]), dtype=torch.float32, device="cuda", generator=g))
@@ -531,7 +531,7 @@ def main():
         config["draft_vocab"] = args.draft_vocab
     if args.workload == "c3" and args.kv_fp8:
         config["kv_cache"] = "e4m3 codes, scales 1/16 (REDUCED PRECISION: not the headline configuration)"
-    if args.workload in ("c3", "c4") and args.w_fp8:
+    if args.workload in ("c3", "c4", "c5") and args.w_fp8:
         config["weights"] = "target projections and LM head as e4m3 codes with per-row scales (REDUCED PRECISION: not the headline configuration)"
     if args.workload != "c3":
         args.no_cpu_baseline = True

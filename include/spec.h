@@ -95,7 +95,8 @@ typedef struct {
                                 /* *_SCALE tensors; code = round_e4m3(w / scale), scale = amax(row) / 448), activations are */
                                 /* quantised the same way per row on the fly, and the products run on the 8-bit tensor-core */
                                 /* path with fp32 accumulation (the precision of the paper's simulator, Section 5.1).       */
-                                /* bf16 dense models; the draft heads' own weights stay 16-bit (the MTP head scores with    */
+                                /* bf16 models (in a mixture-of-experts layer the router stays 16-bit, the experts' gate/up */
+                                /* and down weights are 8-bit); the draft heads' own weights stay 16-bit (the MTP head scores with    */
                                 /* the target's 8-bit LM head); a reduced-precision mode                                    */
 } spec_config;
 
@@ -122,6 +123,8 @@ enum {
     SPEC_T_EXPERTS_DOWN,        /* [n_experts][d][d_expert_ffn]                                        */
     /* SPEC_W_E4M3: fp32 [rows of the weight] scales; the weight tensors themselves then hold one byte per element */
     SPEC_T_LM_HEAD_SCALE = 16, SPEC_T_WQKV_SCALE, SPEC_T_WO_SCALE, SPEC_T_WGATEUP_SCALE, SPEC_T_WDOWN_SCALE,
+    SPEC_T_EXPERTS_GATEUP_SCALE, /* [n_experts][2*d_expert_ffn] (the router stays 16-bit)                  */
+    SPEC_T_EXPERTS_DOWN_SCALE,  /* [n_experts][d]                                                       */
     /* draft head weights (arena `draft_weights`) */
     SPEC_T_D_WFC = 32,          /* EAGLE3: [d][n_taps*d]                                               */
     SPEC_T_D_WPROJ,             /* MTP: [d][2d] acting on concat(norm_g(g), norm_e(e))                 */
@@ -162,8 +165,10 @@ enum {
     /* slot: 0 QKV, 1 O, 2 gate/up, 3 down (of the last layer that ran), 4 LM head (the last LM-head     */
     /* product: the target's, or an MTP head's last pass).  Row r of a slot has                            */
     /* K codes at byte r*K (K = that projection's input width) and its scale at ACT_SCALES[r].             */
+    /* In a mixture-of-experts layer slots 2 and 3 hold the rows in expert order (top_k entries per row). */
     SPEC_T_ACT_CODES,           /* uint8 e4m3 codes, rows back to back                                 */
-    SPEC_T_ACT_SCALES           /* fp32 [rows]                                                         */
+    SPEC_T_ACT_SCALES,          /* fp32 [rows]                                                         */
+    SPEC_T_MOE_INV              /* [B*(k+1)][experts_top_k] int32: where (row, slot) sits in expert order */
 };
 
 /* Counters returned by spec_get_status (host struct). */

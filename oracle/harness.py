@@ -51,6 +51,20 @@ class _LazyRows:
         return m if self.part is None else _split_gate_up(m)[self.part]
 
 
+class _LazyQuantRows:
+    """Per-expert 8-bit weight matrices: codes [E][rows][cols] and scales [E][rows] on the device, fetched one expert at a
+    time as a QuantRows; `part` picks the gate (0) or up (1) half of a stacked gate/up matrix."""
+
+    def __init__(self, codes, scales, part=None):
+        self.codes, self.scales, self.part = codes, scales, part
+
+    def __getitem__(self, e):
+        c, s = self.codes[int(e)].cpu().numpy(), self.scales[int(e)].cpu().numpy()
+        if self.part is None:
+            return model.QuantRows(c, s)
+        return model.QuantRows(_split_gate_up(c)[self.part], _split_gate_up(s[:, None])[self.part][:, 0])
+
+
 class LazyLayers:
     """Sequence of per-layer weight dicts fetched from the device on access (fp32 copies of the stored values)."""
 
@@ -77,10 +91,16 @@ class LazyLayers:
                   mlp_norm=_np(eng.tensor("MLP_NORM", l, torch.float32, (d,))))
         if cfg.get("n_experts", 0) > 0:
             E, Fe = cfg["n_experts"], cfg["d_expert_ffn"]
-            gu = eng.tensor("EXPERTS_GATEUP", l, td, (E, 2 * Fe, d))
-            dn = eng.tensor("EXPERTS_DOWN", l, td, (E, d, Fe))
-            lw.update(router=_np(eng.tensor("ROUTER", l, td, (E, d))), experts_gate=_LazyRows(gu, 0),
-                      experts_up=_LazyRows(gu, 1), experts_down=_LazyRows(dn))
+            lw.update(router=_np(eng.tensor("ROUTER", l, td, (E, d))))
+            if _w8(eng):
+                u8, f32 = torch.uint8, torch.float32
+                gu, gs = eng.tensor("EXPERTS_GATEUP", l, u8, (E, 2 * Fe, d)), eng.tensor("EXPERTS_GATEUP_SCALE", l, f32, (E, 2 * Fe))
+                dn, ds = eng.tensor("EXPERTS_DOWN", l, u8, (E, d, Fe)), eng.tensor("EXPERTS_DOWN_SCALE", l, f32, (E, d))
+                lw.update(experts_gate=_LazyQuantRows(gu, gs, 0), experts_up=_LazyQuantRows(gu, gs, 1), experts_down=_LazyQuantRows(dn, ds))
+            else:
+                gu = eng.tensor("EXPERTS_GATEUP", l, td, (E, 2 * Fe, d))
+                dn = eng.tensor("EXPERTS_DOWN", l, td, (E, d, Fe))
+                lw.update(experts_gate=_LazyRows(gu, 0), experts_up=_LazyRows(gu, 1), experts_down=_LazyRows(dn))
         else:
             gu = _projection(eng, "WGATEUP", l, (2 * F, d))
             if isinstance(gu, model.QuantRows):

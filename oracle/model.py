@@ -101,17 +101,30 @@ def moe_route(router_logits, top_k):
     return ids, wts
 
 
-def moe_mlp(lw, m, top_k, router_logits=None):
+def moe_mlp(lw, m, top_k, router_logits=None, cfg=None):
     """router_logits, when given, replaces W_r m as the input of the top-k decision (used to take that integer
-    decision on the same numbers as an implementation under test)."""
+    decision on the same numbers as an implementation under test).
+
+    With cfg["w_fp8"] the experts' three projections go through the 8-bit format (proj), the router does not.  For checks
+    on given quantised rows, cfg["forced_moe"](t, j) returns the `forced` dict of token t's j-th expert entry, and
+    cfg["record_moe"][(t, j)] receives what was quantised here."""
     ids, wts = moe_route(m @ np.asarray(lw["router"], F64).T if router_logits is None else np.asarray(router_logits, F64), top_k)
     out = np.zeros_like(m)
+    w8 = cfg is not None and cfg.get("w_fp8")
     for t in range(m.shape[0]):
-        for e, w in zip(ids[t], wts[t]):
-            g = np.asarray(lw["experts_gate"][e], F64)
-            u = np.asarray(lw["experts_up"][e], F64)
-            d = np.asarray(lw["experts_down"][e], F64)
-            out[t] += w * ((silu(g @ m[t]) * (u @ m[t])) @ d.T)
+        for j, (e, w) in enumerate(zip(ids[t], wts[t])):
+            if not w8:
+                g = np.asarray(lw["experts_gate"][e], F64)
+                u = np.asarray(lw["experts_up"][e], F64)
+                d = np.asarray(lw["experts_down"][e], F64)
+                out[t] += w * ((silu(g @ m[t]) * (u @ m[t])) @ d.T)
+                continue
+            c = dict(cfg, forced=cfg["forced_moe"](t, j) if cfg.get("forced_moe") else None, record={})
+            row = m[t : t + 1]
+            act = silu(proj(c, row, lw["experts_gate"][e], "gateup")) * proj(c, row, lw["experts_up"][e], "gateup")
+            out[t] += w * proj(c, act, lw["experts_down"][e], "down")[0]
+            if cfg.get("record_moe") is not None:
+                cfg["record_moe"][(t, j)] = c["record"]
     return out
 
 
@@ -259,7 +272,7 @@ def decoder_layer(cfg, lw, x, pos, past_k=None, past_v=None, attn_in=None, route
     x = x + proj(cfg, att, lw["wo"], "o")
     m = rmsnorm(x, lw["mlp_norm"], cfg["rms_eps"])
     if cfg.get("n_experts", 0) > 0:
-        x = x + moe_mlp(lw, m, cfg["experts_top_k"], router_logits)
+        x = x + moe_mlp(lw, m, cfg["experts_top_k"], router_logits, cfg)
     else:
         x = x + dense_mlp(lw, m, cfg)
     return x, k, v

@@ -25,14 +25,14 @@ STATUS_NAMES = {0: "SPEC_OK", -1: "SPEC_ERR_INVALID_ARG", -2: "SPEC_ERR_SHAPE", 
 
 # tensor ids (spec.h)
 T = dict(EMBED=0, LM_HEAD=1, FINAL_NORM=2, ATTN_NORM=3, WQKV=4, WO=5, MLP_NORM=6, WGATEUP=7, WDOWN=8, ROUTER=9,
-         EXPERTS_GATEUP=10, EXPERTS_DOWN=11, LM_HEAD_SCALE=16, WQKV_SCALE=17, WO_SCALE=18, WGATEUP_SCALE=19, WDOWN_SCALE=20,
+         EXPERTS_GATEUP=10, EXPERTS_DOWN=11, LM_HEAD_SCALE=16, WQKV_SCALE=17, WO_SCALE=18, WGATEUP_SCALE=19, WDOWN_SCALE=20, EXPERTS_GATEUP_SCALE=21, EXPERTS_DOWN_SCALE=22,
          D_WFC=32, D_WPROJ=33, D_NORM_E=34, D_NORM_G=35, D_NORM_F=36, D_ATTN_NORM=37, D_WQKV=38, D_WO=39,
          D_MLP_NORM=40, D_WGATEUP=41, D_WDOWN=42, D_LM_HEAD=43, D_D2T=44,
          KV_K=64, KV_V=65, DRAFT_KV_K=66, DRAFT_KV_V=67,
          SEQ_LEN=96, LAST_TOKEN=97, BLOCK_TABLE=98, FREE_STACK=99, FREE_TOP=100, DRAFT_TOKENS=101, OUT_TOKENS=102,
          N_EMITTED=103, STATUS=104, STEP=105, TOKEN_HISTORY=106, OUT_LOGP=107,
          LOGITS=128, DRAFT_LOGITS=129, ROW_STATS=130, DRAFT_ROW_STATS=131, TAPS=132, HIDDEN=133, MOE_LOGITS=134, MOE_IDS=135, MOE_WTS=136,
-         ACT_CODES=137, ACT_SCALES=138)
+         ACT_CODES=137, ACT_SCALES=138, MOE_INV=139)
 
 
 class SpecError(RuntimeError):

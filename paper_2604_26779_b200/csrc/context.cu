@@ -10,7 +10,8 @@
 struct Loc { size_t off = 0, bytes = 0; };
 constexpr int kActSlots = 5;         // quantised activation buffers of an 8-bit-weights context: QKV, O, gate/up, down, LM head
 
-struct LayerLoc { Loc attn_norm, wqkv, wo, mlp_norm, wgateup, wdown, router, exp_gateup, exp_down, wqkv_s, wo_s, wgateup_s, wdown_s; };
+struct LayerLoc { Loc attn_norm, wqkv, wo, mlp_norm, wgateup, wdown, router, exp_gateup, exp_down, wqkv_s, wo_s, wgateup_s, wdown_s,
+                  exp_gateup_s, exp_down_s; };
 
 struct spec_ctx {
     spec_config cfg;
@@ -96,8 +97,8 @@ spec_status check_config(const spec_config* c)
                                          !(c->kv_scale_k > 0.f) || !(c->kv_scale_v > 0.f) ||
                                          (c->k_max + 1) * (c->n_q_heads / c->n_kv_heads) > 16)) return SPEC_ERR_UNSUPPORTED;
     if (c->weight_dtype != SPEC_W_MODEL &&
-        (c->weight_dtype != SPEC_W_E4M3 || c->dtype != SPEC_DTYPE_BF16 || c->n_experts > 0 ||
-         c->d_model % 128 != 0 || c->d_ffn % 128 != 0 || (c->n_q_heads * c->head_dim) % 128 != 0 || (c->head_dim != 64 && c->head_dim != 128) ||
+        (c->weight_dtype != SPEC_W_E4M3 || c->dtype != SPEC_DTYPE_BF16 ||
+         c->d_model % 128 != 0 || (c->n_experts > 0 ? c->d_expert_ffn % 128 != 0 : c->d_ffn % 128 != 0) || (c->n_q_heads * c->head_dim) % 128 != 0 || (c->head_dim != 64 && c->head_dim != 128) ||
          c->vocab % 8 != 0))
         return SPEC_ERR_UNSUPPORTED;
     if (c->draft_vocab != 0 && (c->draft_kind != SPEC_DRAFT_EAGLE3 || c->draft_vocab < 8 || c->draft_vocab > c->vocab ||
@@ -128,8 +129,9 @@ void build_layout(spec_ctx& x)
             L.mlp_norm = a.take(d * 4);
             if (c.n_experts > 0) {
                 L.router = a.take((size_t)c.n_experts * d * es);
-                L.exp_gateup = a.take((size_t)c.n_experts * 2 * c.d_expert_ffn * d * es);
-                L.exp_down = a.take((size_t)c.n_experts * d * c.d_expert_ffn * es);
+                L.exp_gateup = a.take((size_t)c.n_experts * 2 * c.d_expert_ffn * d * ws);     // the router stays 16-bit
+                L.exp_down = a.take((size_t)c.n_experts * d * c.d_expert_ffn * ws);
+                if (w8) { L.exp_gateup_s = a.take((size_t)c.n_experts * 2 * c.d_expert_ffn * 4); L.exp_down_s = a.take((size_t)c.n_experts * d * 4); }
             } else {
                 L.wgateup = a.take((size_t)2 * c.d_ffn * d * ws);
                 L.wdown = a.take(d * (size_t)c.d_ffn * ws);
@@ -200,11 +202,15 @@ void build_layout(spec_ctx& x)
         x.gu = a.take(M * 2 * Fmax * es);
         x.act = a.take(M * Fmax * es);
         if (c.weight_dtype == SPEC_W_E4M3) {                  // activations as e4m3 codes + one scale per row, rewritten before every projection
-            const size_t kmax = (size_t)(c.d_ffn > (int)od ? c.d_ffn : od) > d ? (size_t)(c.d_ffn > (int)od ? c.d_ffn : od) : d;
+            const size_t f8 = c.n_experts > 0 ? (size_t)c.d_expert_ffn : (size_t)c.d_ffn;
+            const size_t kmax = (f8 > od ? f8 : od) > d ? (f8 > od ? f8 : od) : d;
+            // a mixture-of-experts layer quantises its rows in expert order: top_k entries per row, + one tile of slack rows
+            // for the last group's TMA box
+            const size_t rows8 = c.n_experts > 0 ? M * c.experts_top_k + 128 : M;
             // five slots, one per projection of a layer (QKV, O, gate/up, down) and one for the LM head, so that what the last
             // layer and the LM head consumed stays readable after the pass (SPEC_T_ACT_CODES / SPEC_T_ACT_SCALES)
-            x.a8 = a.take(kActSlots * M * kmax);
-            x.a8_scale = a.take(kActSlots * M * 4);
+            x.a8 = a.take(kActSlots * rows8 * kmax);
+            x.a8_scale = a.take(kActSlots * rows8 * 4);
         }
         x.logits = a.take(M * (size_t)c.vocab * 4);
         x.draft_logits = a.take(Bm * (size_t)(c.k_max > 0 ? c.k_max : 1) * c.vocab * 4);   // sized for the whole vocabulary
@@ -246,7 +252,8 @@ template <class T = void> T* at(void* base, const Loc& l) { return reinterpret_c
 
 struct LayerPtrs { const float* attn_norm; const void* wqkv; const void* wo; const float* mlp_norm; const void* wgateup; const void* wdown;
                    const void* router; const void* exp_gateup; const void* exp_down;
-                   const float* wqkv_s; const float* wo_s; const float* wgateup_s; const float* wdown_s; };   // 8-bit weights: row scales
+                   const float* wqkv_s; const float* wo_s; const float* wgateup_s; const float* wdown_s;       // 8-bit weights: row scales
+                   const float* exp_gateup_s; const float* exp_down_s; };
 
 LayerPtrs layer_ptrs(void* base, const LayerLoc& L)
 {
@@ -255,7 +262,9 @@ LayerPtrs layer_ptrs(void* base, const LayerLoc& L)
             L.router.bytes ? at<const void>(base, L.router) : nullptr, at<const void>(base, L.exp_gateup),
             at<const void>(base, L.exp_down),
             L.wqkv_s.bytes ? at<const float>(base, L.wqkv_s) : nullptr, L.wo_s.bytes ? at<const float>(base, L.wo_s) : nullptr,
-            L.wgateup_s.bytes ? at<const float>(base, L.wgateup_s) : nullptr, L.wdown_s.bytes ? at<const float>(base, L.wdown_s) : nullptr};
+            L.wgateup_s.bytes ? at<const float>(base, L.wgateup_s) : nullptr, L.wdown_s.bytes ? at<const float>(base, L.wdown_s) : nullptr,
+            L.exp_gateup_s.bytes ? at<const float>(base, L.exp_gateup_s) : nullptr,
+            L.exp_down_s.bytes ? at<const float>(base, L.exp_down_s) : nullptr};
 }
 
 #define TRY(expr) do { spec_status s__ = (expr); if (s__ != SPEC_OK) return s__; } while (0)
@@ -328,6 +337,24 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
         TRY(launch_quantize_rows(M, Hq * dh, at(ws, c.attn_out), a8_of(1), a8s_of(1), st));
         TIMED(c, CLS_GEMM, launch_gemm8_tc(M, d, Hq * dh, a8_of(1), a8s_of(1), W.wo, W.wo_s, res, d, SPEC_DTYPE_F32, 1, 1.f, nullptr, 0, nullptr, 0,
                                            status_word, st));
+        if (W.router != nullptr) {
+            // mixture of experts: the router decides on the 16-bit rows; the rows are quantised in expert order (slot 2), the
+            // SwiGLU outputs again (slot 3); both grouped products run on the 8-bit path with the experts' row scales
+            const int E = g.n_experts, tk = g.experts_top_k, Fe = g.d_expert_ffn, n = M * tk;
+            TRY(launch_rmsnorm(M, d, res, W.mlp_norm, g.rms_eps, at(ws, c.h), d, 0, dt, st));
+            TIMED(c, CLS_GEMM, launch_gemm(M, E, d, at(ws, c.h), d, W.router, at(ws, c.moe_logits), E, dt, SPEC_DTYPE_F32, 0, st));
+            TRY(launch_moe_route(M, E, tk, at<float>(ws, c.moe_logits), at<int32_t>(ws, c.moe_ids), at<float>(ws, c.moe_wts), st));
+            TRY(launch_moe_permute(M, E, tk, d, at<int32_t>(ws, c.moe_ids), at<int32_t>(ws, c.moe_rank), at<int32_t>(ws, c.moe_counts),
+                                   at<int32_t>(ws, c.moe_offsets), at<int32_t>(ws, c.moe_inv), at(ws, c.h), at(ws, c.moe_a), st));
+            TRY(launch_quantize_rows(n, d, at(ws, c.moe_a), a8_of(2), a8s_of(2), st));
+            TIMED(c, CLS_GEMM, launch_gemm8_grouped(n, M, E, 2 * Fe, d, a8_of(2), a8s_of(2), W.exp_gateup, W.exp_gateup_s, at(ws, c.moe_act), dt, 1,
+                                                    at<int32_t>(ws, c.moe_counts), at<int32_t>(ws, c.moe_offsets), status_word, st));
+            TRY(launch_quantize_rows(n, Fe, at(ws, c.moe_act), a8_of(3), a8s_of(3), st));
+            TIMED(c, CLS_GEMM, launch_gemm8_grouped(n, M, E, d, Fe, a8_of(3), a8s_of(3), W.exp_down, W.exp_down_s, at(ws, c.moe_out), SPEC_DTYPE_F32, 0,
+                                                    at<int32_t>(ws, c.moe_counts), at<int32_t>(ws, c.moe_offsets), status_word, st));
+            TRY(launch_moe_combine(M, tk, d, at<float>(ws, c.moe_wts), at<int32_t>(ws, c.moe_inv), at<float>(ws, c.moe_out), res, st));
+            return SPEC_OK;
+        }
         TRY(launch_rmsnorm_quantize(M, d, res, W.mlp_norm, g.rms_eps, a8_of(2), a8s_of(2), st));
         TIMED(c, CLS_GEMM, launch_gemm8_swiglu_tc(M, d_ffn, d, a8_of(2), a8s_of(2), W.wgateup, W.wgateup_s, at(ws, c.act), status_word, st));
         TRY(launch_quantize_rows(M, d_ffn, at(ws, c.act), a8_of(3), a8s_of(3), st));
@@ -532,6 +559,13 @@ extern "C" spec_status spec_tensor(spec_ctx* c, int id, int layer, void** dev_pt
     case SPEC_T_MOE_LOGITS: base = c->buf.workspace; l = c->moe_logits; break;
     case SPEC_T_MOE_IDS: base = c->buf.workspace; l = c->moe_ids; break;
     case SPEC_T_MOE_WTS: base = c->buf.workspace; l = c->moe_wts; break;
+    case SPEC_T_MOE_INV: base = c->buf.workspace; l = c->moe_inv; break;
+    case SPEC_T_EXPERTS_GATEUP_SCALE: case SPEC_T_EXPERTS_DOWN_SCALE: {
+        if (!layer_ok()) return SPEC_ERR_INVALID_ARG;
+        base = c->buf.weights;
+        l = id == SPEC_T_EXPERTS_GATEUP_SCALE ? c->layers[layer].exp_gateup_s : c->layers[layer].exp_down_s;
+        break;
+    }
     case SPEC_T_ACT_CODES: case SPEC_T_ACT_SCALES: {
         // `layer` selects the slot: 0 QKV, 1 O, 2 gate/up, 3 down (of the last layer run), 4 LM head
         if (layer < 0 || layer >= kActSlots) return SPEC_ERR_INVALID_ARG;

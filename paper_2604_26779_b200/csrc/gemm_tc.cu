@@ -219,7 +219,7 @@ __device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoor
             uint32_t v2[32];
             tc_ld32(t_row + c0 + 32, v2);
             tc_wait_ld();
-            if (g.fp8) { const float rs = row_ok ? g.a_scale[row] : 0.f; scale32(g, v, rs, col, g.N); scale32(g, v2, rs, col + 32, g.N); }
+            if (g.fp8) { const float rs = row_ok ? g.a_scale[row] : 0.f; const int wo = tc.b_row - tc.col; scale32(g, v, rs, wo + col, wo + g.N); scale32(g, v2, rs, wo + col + 32, wo + g.N); }
             float f[8];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -236,7 +236,7 @@ __device__ __forceinline__ void epilogue_plain(const GemmArgs& g, const TileCoor
             continue;
         }
         tc_wait_ld();
-        if (g.fp8) scale32(g, v, row_ok ? g.a_scale[row] : 0.f, col, g.N);
+        if (g.fp8) scale32(g, v, row_ok ? g.a_scale[row] : 0.f, tc.b_row - tc.col + col, tc.b_row - tc.col + g.N);   // grouped: the group's weight rows
         if (g.stat_part != nullptr) {
             float cm = -INFINITY;
 #pragma unroll
@@ -997,6 +997,26 @@ spec_status launch_gemm8_qkv_tc(int M, int K, const void* a8, const float* a_sca
     g.k_pool = static_cast<__nv_bfloat16*>(e.k_pool); g.v_pool = static_cast<__nv_bfloat16*>(e.v_pool);
     g.kv_fp8 = e.kv_fp8; g.k_scale = e.k_scale; g.v_scale = e.v_scale;
     return run_kernel(EPI_QKV, ma, mb, g, (long long)((M + BM - 1) / BM) * ((N + BN - 1) / BN), st);
+}
+
+// Grouped product on 8-bit operands: as launch_gemm_grouped with A [rows_total][K] and W [E][N][K] as e4m3 codes, a_scale one
+// per row of A, w_scale [E][N].
+spec_status launch_gemm8_grouped(int rows_total, int max_rows_per_group, int E, int N, int K, const void* a8, const float* a_scale,
+                                 const void* w8, const float* w_scale, void* C, int out_dtype, int swiglu, const int32_t* counts,
+                                 const int32_t* offsets, int32_t* status, cudaStream_t st)
+{
+    if (rows_total == 0 || E == 0) return SPEC_OK;
+    if (N % BN != 0 || E > kMaxGroups || !fp8_ok(K, a8, w8)) return SPEC_ERR_SHAPE;
+    if (!init_once()) return SPEC_ERR_CUDA;
+    CUtensorMap ma, mb;
+    if (!make_map8(&ma, a8, (uint64_t)rows_total, (uint64_t)K, (uint64_t)K, BM)) return SPEC_ERR_CUDA;
+    if (!make_map8(&mb, w8, (uint64_t)E * N, (uint64_t)K, (uint64_t)K, BN)) return SPEC_ERR_CUDA;
+    const int max_m_tiles = (max_rows_per_group + BM - 1) / BM;
+    GemmArgs g{};
+    fp8_args(g, rows_total, N, K, a_scale, w_scale, status);
+    g.C = C; g.ldc = swiglu ? N / 2 : N; g.out_f32 = out_dtype == SPEC_DTYPE_F32 ? 1 : 0;
+    g.E = E; g.max_m_tiles = max_m_tiles; g.counts = counts; g.offsets = offsets;
+    return run_kernel(swiglu ? EPI_SWIGLU : EPI_PLAIN, ma, mb, g, (long long)E * max_m_tiles * (N / BN), st);
 }
 
 // Grouped form: A [rows_total][K] holds the groups' rows back to back (group e at offsets[e], counts[e] rows, both on

@@ -128,6 +128,9 @@ spec_status launch_gemm_qkv_tc(int M, int K, const void* A, int lda, const void*
                                int32_t* status, cudaStream_t st);
 spec_status launch_gemm8_qkv_tc(int M, int K, const void* a8, const float* a_scale, const void* w8, const float* w_scale, void* qkv,
                                 const QkvEpilogue& e, int32_t* status, cudaStream_t st);
+spec_status launch_gemm8_grouped(int rows_total, int max_rows_per_group, int E, int N, int K, const void* a8, const float* a_scale,
+                                 const void* w8, const float* w_scale, void* C, int out_dtype, int swiglu, const int32_t* counts,
+                                 const int32_t* offsets, int32_t* status, cudaStream_t st);
 // (cos, sin) table of the rows' positions for the fused QKV epilogue
 spec_status launch_rope_table(int M, int dh, float theta, const int32_t* pos, float* table, cudaStream_t st);
 

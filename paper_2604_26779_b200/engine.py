@@ -135,8 +135,9 @@ class SpecStep:
         scale per row, quantised on the device by the library (spec_quantize_rows) from the 16-bit values."""
         if self.sc.weight_dtype != B.SPEC_W_E4M3:
             return self.put(name, layer, array)
-        w = torch.from_numpy(np.ascontiguousarray(array)).to(self.device).to(torch.bfloat16)
-        w = w.reshape(-1, w.shape[-1]).contiguous()
+        w = array if torch.is_tensor(array) else torch.from_numpy(np.ascontiguousarray(array))
+        w = w.to(self.device).to(torch.bfloat16)
+        w = w.reshape(-1, w.shape[-1]).contiguous()                # experts [E][rows][K]: every row of every expert has its scale
         codes = self.tensor(name, layer, torch.uint8)
         scales = self.tensor(name + "_SCALE", layer, torch.float32)
         assert codes.numel() == w.numel() and scales.numel() == w.shape[0], (name, codes.numel(), w.numel(), scales.numel())
@@ -155,8 +156,8 @@ class SpecStep:
             self.put("MLP_NORM", l, lw["mlp_norm"], f32)
             if "router" in lw:
                 self.put("ROUTER", l, lw["router"])
-                self.put("EXPERTS_GATEUP", l, stack_gate_up(lw["experts_gate"], lw["experts_up"]))
-                self.put("EXPERTS_DOWN", l, lw["experts_down"])
+                self.put_projection("EXPERTS_GATEUP", l, stack_gate_up(lw["experts_gate"], lw["experts_up"]))
+                self.put_projection("EXPERTS_DOWN", l, lw["experts_down"])
             else:
                 self.put_projection("WGATEUP", l, stack_gate_up(lw["wgate"], lw["wup"]))
                 self.put_projection("WDOWN", l, lw["wdown"])

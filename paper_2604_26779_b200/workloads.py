@@ -97,8 +97,11 @@ def build_dense_workload(name="c3", *, B=256, k=3, n_layers=None, len_lo=1024, l
         eng.tensor("ATTN_NORM", l, f32).fill_(1.0)
         eng.tensor("MLP_NORM", l, f32).fill_(1.0)
         if cfg.get("n_experts", 0) > 0:
-            for nm in ("WQKV", "WO", "EXPERTS_GATEUP", "EXPERTS_DOWN"):
-                _fill_normal(eng.tensor(nm, l, bf), 0.02, gen)
+            E_, Fe_ = cfg["n_experts"], cfg["d_expert_ffn"]
+            fill_projection("WQKV", l, qn_, d_)
+            fill_projection("WO", l, d_, od_)
+            fill_projection("EXPERTS_GATEUP", l, E_ * 2 * Fe_, d_)
+            fill_projection("EXPERTS_DOWN", l, E_ * d_, Fe_)
             # router rows ~ N(0, 1/d): unit-RMS inputs give router logits ~ N(0, 1)
             _fill_normal(eng.tensor("ROUTER", l, bf), float(cfg["d_model"]) ** -0.5, gen)
         else:

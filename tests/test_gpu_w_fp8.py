@@ -211,3 +211,67 @@ def test_w_fp8_mtp_head_scores_with_the_8bit_lm_head():
     print(f"w_fp8 MTP head: last pass logits {err:.2e}")
     assert err < 1e-5
     eng.close()
+
+
+@pytest.mark.parametrize("shape", ["small", "235b"])
+def test_w_fp8_moe_layer_projection_by_projection(shape):
+    """One mixture-of-experts decoder layer + LM head with 8-bit projections (the router stays 16-bit and decides on the
+    device's own fp32 logits): the rows every expert entry consumed - in expert order, found through MOE_INV - are forced into
+    the oracle; products to fp32 accumulation error, quantiser decisions compared where the oracle reproduces the input."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_26779_b200 import inputs, workloads
+    k = 3
+    if shape == "small":
+        over = dict(d_model=512, n_q_heads=8, n_kv_heads=2, head_dim=64, n_experts=16, experts_top_k=4, d_expert_ffn=128, w_fp8=True)
+        lens, vocab, checked = [3, 40, 100, 300, 20, 1], 1024, range(6)
+    else:           # d=4096, 64 q / 4 KV heads of 128, 128 experts top-8, expert FFN 1536, LM head over 151936
+        over, lens, vocab, checked = dict(w_fp8=True), [8192, 700, 33, 2500, 8192, 1200, 64, 5000], None, (1, 2)
+    eng, info = workloads.build_dense_workload("c5", lens=np.array(lens, np.int32), k=k, draft="none", steps_budget=2, vocab=vocab, cfg_over=over)
+    cfg = info["cfg"]
+    assert cfg["n_layers"] == 1 and cfg["n_experts"] > 0
+    B, d, V, Fe, E, tk = eng.B, cfg["d_model"], cfg["vocab"], cfg["d_expert_ffn"], cfg["n_experts"], cfg["experts_top_k"]
+    Hq, dh = cfg["n_q_heads"], cfg["head_dim"]
+    R, M = k + 1, B * (k + 1)
+    n = M * tk
+    drafts = torch.from_numpy(inputs.make_prompts(B, k, V, seed=77)).cuda()
+    seq_len = eng.seq_len().cpu().numpy().copy()
+    last = eng.tensor("LAST_TOKEN", 0, torch.int32, (B,)).cpu().numpy().copy()
+    eng.verify(k, drafts)
+    assert eng.status().device_status == 0
+    drafts = drafts.cpu().numpy()
+    table = eng.block_table().cpu().numpy().copy()
+    W = harness.device_weights(eng, cfg)
+    lw = W["layers"][0]
+    rl = eng.tensor("MOE_LOGITS", 0, torch.float32, (M, E)).cpu().numpy()
+    ids = eng.tensor("MOE_IDS", 0, torch.int32, (M, tk)).cpu().numpy()
+    o_ids, _ = model.moe_route(rl, tk)
+    assert np.array_equal(o_ids, ids)
+    inv = eng.tensor("MOE_INV", 0, torch.int32, (M, tk)).cpu().numpy()
+    assert np.array_equal(np.sort(inv.reshape(-1)), np.arange(n))                 # a permutation of the entries
+    dev = {"qkv": act_rows(eng, 0, M, d), "o": act_rows(eng, 1, M, Hq * dh), "gateup": act_rows(eng, 2, n, d),
+           "down": act_rows(eng, 3, n, Fe), "lm_head": act_rows(eng, 4, M, d)}
+    hidden = eng.tensor("HIDDEN", 0, torch.float32, (M, d)).cpu().numpy().astype(np.float64)
+    worst_x = worst_l = 0.0
+    low = {"gateup": 1.0, "down": 1.0}
+    for b in checked:
+        r0, r1 = b * R, (b + 1) * R
+        n_past = int(seq_len[b])
+        tokens = [int(last[b])] + [int(t) for t in drafts[b]]
+        rec = {}
+        entry = lambda t, j: {s: rows_of(dev[s], int(inv[r0 + t, j]), int(inv[r0 + t, j]) + 1) for s in ("gateup", "down")}
+        cfg_f = dict(cfg, forced={s: rows_of(dev[s], r0, r1) for s in ("qkv", "o")}, forced_moe=entry, record_moe=rec)
+        past = harness.LazyPast(eng, cfg, table[b], n_past, info["kv_pools"], 1)[0]
+        x_out, _, _ = model.decoder_layer(cfg_f, lw, W["embed"][tokens].astype(np.float64), np.arange(n_past, n_past + R),
+                                          past[0] if n_past else None, past[1] if n_past else None, router_logits=rl[r0:r1])
+        worst_x = max(worst_x, float(np.abs(hidden[r0:r1] - x_out).max() / np.abs(x_out).max()))
+        for (t, j), rr in rec.items():
+            p = int(inv[r0 + t, j])
+            low["gateup"] = min(low["gateup"], compare_rows(rows_of(dev["gateup"], p, p + 1), rr["gateup"], "gateup", 0.98))
+            low["down"] = min(low["down"], compare_rows(rows_of(dev["down"], p, p + 1), rr["down"], "down", 0.90))
+        ref_logits = model.proj(dict(cfg, forced={"lm_head": rows_of(dev["lm_head"], r0, r1)}), np.zeros((R, d)), W["lm_head"], "lm_head")
+        logits = eng.logits(k)[b].cpu().numpy().reshape(R, V).astype(np.float64)
+        worst_l = max(worst_l, float((np.abs(logits - ref_logits).max(-1) / np.abs(ref_logits).max(-1)).max()))
+    print(f"w_fp8 MoE layer ({shape}): residual stream {worst_x:.2e}, logits {worst_l:.2e}, equal codes {low}")
+    assert worst_x < 1e-5 and worst_l < 1e-5
+    eng.close()

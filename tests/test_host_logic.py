@@ -124,8 +124,13 @@ def test_sizes_and_refusals_with_8bit_projections():
     assert s8.workspace_bytes >= s16.workspace_bytes + 5 * 1024 * 14336          # five quantised-activation slots
     sc = engine.make_spec_config(cfg, w_fp8=True, **dict(kw, draft_kind="mtp", draft_d_ffn=14336))
     assert sizes_of(sc)[0] == 0                                                  # the MTP head scores with the 8-bit LM head
-    for change in (dict(dtype=B.SPEC_DTYPE_F32),
-                   dict(n_experts=8, experts_top_k=2, d_expert_ffn=1536), dict(weight_dtype=7)):
+    moe = inputs.model_config("c5")
+    c16, m16 = sizes_of(engine.make_spec_config(moe, draft_kind="none", k_max=3, max_batch=8, kv_num_blocks=100, max_blocks_per_seq=16))
+    c8, m8 = sizes_of(engine.make_spec_config(moe, draft_kind="none", k_max=3, max_batch=8, kv_num_blocks=100, max_blocks_per_seq=16, w_fp8=True))
+    assert c16 == 0 and c8 == 0
+    experts = moe["n_experts"] * 3 * moe["d_expert_ffn"] * moe["d_model"]           # gate, up, down: one byte instead of two
+    assert m16.weights_bytes - m8.weights_bytes > experts * 0.99
+    for change in (dict(dtype=B.SPEC_DTYPE_F32), dict(weight_dtype=7)):
         sc = engine.make_spec_config(cfg, w_fp8=True, **kw)
         for k, v in change.items():
             setattr(sc, k, v)

@@ -314,3 +314,29 @@ def test_fp8_projection_error_is_what_the_format_allows():
     assert np.array_equal(model.proj({"w_fp8": True, "forced": {"o": rec["qkv"]}}, np.zeros_like(x), W, "qkv"), np.zeros_like(got))
     one = model.QuantRows(np.full((1, 256), 0x38, np.uint8), np.array([2.0], np.float32))      # 0x38 = 1.0: a row of twos
     assert np.allclose(model.proj({"w_fp8": True, "forced": {"qkv": one}}, x[:1], W, "qkv")[0], 2.0 * model.rows_8bit(W).sum(-1), rtol=1e-12)
+
+
+def test_8bit_expert_block_reduces_to_the_dense_8bit_mlp():
+    # one expert, top-1: the mixture weight is 1 and the block is the dense SwiGLU MLP through the same 8-bit projections;
+    # with several experts, forcing back the rows the block itself quantised reproduces it, and the router is untouched
+    rng = np.random.default_rng(11)
+    d, Fe, T = 64, 48, 5
+    m = rng.standard_normal((T, d))
+    g, u, dn = (rng.standard_normal((Fe, d)) * 0.2).astype(np.float32), (rng.standard_normal((Fe, d)) * 0.2).astype(np.float32), \
+        (rng.standard_normal((d, Fe)) * 0.2).astype(np.float32)
+    cfg = {"w_fp8": True}
+    one = dict(router=np.zeros((1, d), np.float32), experts_gate=[g], experts_up=[u], experts_down=[dn])
+    # (row-at-a-time against whole-matrix products: equal up to the fp64 summation order of the library matmul)
+    assert np.allclose(model.moe_mlp(one, m, 1, cfg=cfg), model.dense_mlp(dict(wgate=g, wup=u, wdown=dn), m, cfg), rtol=1e-12, atol=1e-14)
+    E, topk = 4, 2
+    lw = dict(router=rng.standard_normal((E, d)).astype(np.float32),
+              experts_gate=[(rng.standard_normal((Fe, d)) * 0.2).astype(np.float32) for _ in range(E)],
+              experts_up=[(rng.standard_normal((Fe, d)) * 0.2).astype(np.float32) for _ in range(E)],
+              experts_down=[(rng.standard_normal((d, Fe)) * 0.2).astype(np.float32) for _ in range(E)])
+    rec = {}
+    a = model.moe_mlp(lw, m, topk, cfg=dict(cfg, record_moe=rec))
+    assert set(rec) == {(t, j) for t in range(T) for j in range(topk)} and all(set(v) == {"gateup", "down"} for v in rec.values())
+    b = model.moe_mlp(lw, np.zeros_like(m), topk, router_logits=m @ lw["router"].astype(np.float64).T,
+                      cfg=dict(cfg, forced_moe=lambda t, j: rec[(t, j)]))
+    assert np.array_equal(a, b)
+    assert np.max(np.abs(a - model.moe_mlp(lw, m, topk))) / np.max(np.abs(a)) < 0.1 and not np.array_equal(a, model.moe_mlp(lw, m, topk))
