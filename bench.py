@@ -324,6 +324,16 @@ def run_ep_microbench(args):
     for r in range(R):
         gus.append(stack_gate_up(rn((per, Fe, d), d ** -0.5), rn((per, Fe, d), d ** -0.5)).contiguous())
         dns.append(rn((per, d, Fe), Fe ** -0.5))
+    scales = [None] * R
+    if args.w_fp8:                                            # 8-bit expert weights: quantised row by row by the library
+        from paper_2604_26779_b200 import binding
+        for r in range(R):
+            gu8, dn8 = torch.empty(gus[r].shape, dtype=torch.uint8, device="cuda"), torch.empty(dns[r].shape, dtype=torch.uint8, device="cuda")
+            gs, ds = torch.empty(per * 2 * Fe, dtype=torch.float32, device="cuda"), torch.empty(per * d, dtype=torch.float32, device="cuda")
+            binding.spec_quantize_rows(gus[r].view(-1, d), gu8.view(-1, d), gs)
+            binding.spec_quantize_rows(dns[r].contiguous().view(-1, Fe), dn8.view(-1, Fe), ds)
+            torch.cuda.synchronize()
+            gus[r], dns[r], scales[r] = gu8, dn8, (gs, ds)
     hs = [rn((M, d), 1.0) for _ in range(R)]
     xs = [torch.zeros((M, d), dtype=torch.float32, device="cuda") for _ in range(R)]
     ranks = [ep.EpRank(R, r, E, top_k, d, Fe, M, cap) for r in range(R)]
@@ -340,8 +350,8 @@ def run_ep_microbench(args):
         for r, h in zip(ranks, hs):
             r.route(h, router)
         ev[1].record()
-        for r, gu, dn in zip(ranks, gus, dns):
-            r.experts(gu, dn)
+        for r, gu, dn, sc in zip(ranks, gus, dns, scales):
+            r.experts(gu, dn, scales=sc)
         ev[2].record()
         for r, x in zip(ranks, xs):
             r.combine(x)
@@ -369,7 +379,7 @@ def run_ep_microbench(args):
         "combine_GBps_local": comb_b / ms[2] / 1e6 if ms[2] > 0 else None,
         "nvlink_ms_at_770GBps": {"dispatch": disp_b * remote / nvl * 1e3, "combine": comb_b * remote / nvl * 1e3},
         "expert_gemm_tflops": rows * (2 * 2 * Fe * d + 2 * d * Fe) / ms[1] / 1e9 if ms[1] > 0 else None,
-        "peak_GBps": hbm_peak, "peak_source": kind, "dtype": "bf16", "data": "synthetic", "clocks": ck,
+        "peak_GBps": hbm_peak, "peak_source": kind, "dtype": "e4m3 experts, bf16 router" if args.w_fp8 else "bf16", "data": "synthetic", "clocks": ck,
         "config": {"workload": "c5ep: one MoE MLP block, 128 experts top-8, d=4096, expert FFN 1536, router logits ~N(0,1)",
                    "l2": "weights + windows of all ranks exceed L2"}}))
     return 0

@@ -402,6 +402,13 @@ spec_status spec_ep_route(const spec_ep_config* cfg, void* window, void* scratch
  * [local experts][d][d_expert_ffn]: the LOCAL experts only. */
 spec_status spec_ep_experts(const spec_ep_config* cfg, void* const* peer_windows_host, void* scratch,
                             const void* w_gateup, const void* w_down, int32_t* status, void* stream);
+/* The same with 8-bit expert weights: w_gateup / w_down hold e4m3 codes (one byte per element, same shapes),
+ * w_gateup_scale [local experts][2 * d_expert_ffn] and w_down_scale [local experts][d] one fp32 scale per weight row
+ * (spec_quantize_rows produces both).  The received rows and the SwiGLU outputs are quantised per row on this rank;
+ * a row gives the same codes wherever its expert lives, so the result does not depend on ep_size. */
+spec_status spec_ep_experts_e4m3(const spec_ep_config* cfg, void* const* peer_windows_host, void* scratch,
+                                 const void* w_gateup, const float* w_gateup_scale, const void* w_down,
+                                 const float* w_down_scale, int32_t* status, void* stream);
 /* x [M][d] fp32 residual of this rank's rows (M as given to spec_ep_route). */
 spec_status spec_ep_combine(const spec_ep_config* cfg, void* const* peer_windows_host, int M, float* x, void* stream);
 

@@ -119,6 +119,7 @@ SIGNATURES = {
     "spec_ep_tensor": (_i, [C.POINTER(spec_ep_config), _vp, _vp, _i, C.POINTER(_vp), C.POINTER(_sz)]),
     "spec_ep_route": (_i, [C.POINTER(spec_ep_config), _vp, _vp, _i, _vp, _vp, _vp]),
     "spec_ep_experts": (_i, [C.POINTER(spec_ep_config), C.POINTER(_vp), _vp, _vp, _vp, _vp, _vp]),
+    "spec_ep_experts_e4m3": (_i, [C.POINTER(spec_ep_config), C.POINTER(_vp), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "spec_ep_combine": (_i, [C.POINTER(spec_ep_config), C.POINTER(_vp), _i, _vp, _vp]),
     "spec_ipc_export": (_i, [_vp, _vp, C.POINTER(_u64)]),
     "spec_ipc_open": (_i, [_vp, C.POINTER(_vp)]),
@@ -277,6 +278,11 @@ def spec_ep_route(cfg, window, scratch, M, h, router_w, stream=None):
 def spec_ep_experts(cfg, peer_windows, scratch, w_gateup, w_down, status=None, stream=None):
     _check(lib().spec_ep_experts(C.byref(cfg), _peer_array(peer_windows), _ptr(scratch), _ptr(w_gateup), _ptr(w_down),
                                  _ptr(status), _stream(stream)), "spec_ep_experts")
+
+
+def spec_ep_experts_e4m3(cfg, peer_windows, scratch, w_gateup, w_gateup_scale, w_down, w_down_scale, status=None, stream=None):
+    _check(lib().spec_ep_experts_e4m3(C.byref(cfg), _peer_array(peer_windows), _ptr(scratch), _ptr(w_gateup), _ptr(w_gateup_scale),
+                                      _ptr(w_down), _ptr(w_down_scale), _ptr(status), _stream(stream)), "spec_ep_experts_e4m3")
 
 
 def spec_ep_combine(cfg, peer_windows, M, x, stream=None):

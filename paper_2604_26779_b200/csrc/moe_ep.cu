@@ -24,7 +24,7 @@ struct Peers { unsigned char* win[kMaxRanks]; };
 // Byte offsets inside a window / the scratch.  Every piece starts on a 256-byte boundary.
 struct EpLayout {
     size_t hdr, h, ids, wts, rank, src_of, counts, offsets, recv_off, y, window_bytes;
-    size_t logits, a_perm, act, grp_counts, grp_offsets, scratch_bytes;
+    size_t logits, a_perm, act, grp_counts, grp_offsets, a8, a8_scale, scratch_bytes;
 };
 enum { HDR_M = 0, HDR_RECV_TOTAL = 1 };
 
@@ -53,6 +53,9 @@ EpLayout make_layout(const spec_ep_config& c)
     l.act = take((cap + 128) * c.d_expert_ffn * 2);
     l.grp_counts = take(E * 4);
     l.grp_offsets = take(E * 4);
+    // 8-bit experts (spec_ep_experts_e4m3): the received rows, then the SwiGLU outputs, as e4m3 codes with one scale per row
+    l.a8 = take((cap + 128) * (size_t)(c.d > c.d_expert_ffn ? c.d : c.d_expert_ffn));
+    l.a8_scale = take((cap + 128) * 4);
     l.scratch_bytes = at;
     return l;
 }
@@ -266,12 +269,16 @@ extern "C" spec_status spec_ep_route(const spec_ep_config* cfg, void* window, vo
     return launch_status();
 }
 
-extern "C" spec_status spec_ep_experts(const spec_ep_config* cfg, void* const* peer_windows_host, void* scratch,
-                                       const void* w_gateup, const void* w_down, int32_t* status, void* stream)
+namespace {
+// Shared body of spec_ep_experts and spec_ep_experts_e4m3 (scales != nullptr: 8-bit expert weights).
+spec_status ep_experts(const spec_ep_config* cfg, void* const* peer_windows_host, void* scratch, const void* w_gateup, const float* gateup_scale,
+                       const void* w_down, const float* down_scale, int32_t* status, void* stream)
 {
     const spec_status s = check(cfg);
     if (s != SPEC_OK) return s;
     if (peer_windows_host == nullptr || scratch == nullptr || w_gateup == nullptr || w_down == nullptr) return SPEC_ERR_INVALID_ARG;
+    const bool w8 = gateup_scale != nullptr;
+    if (w8 && (down_scale == nullptr || cfg->d % 16 != 0 || cfg->d_expert_ffn % 16 != 0)) return SPEC_ERR_INVALID_ARG;
     Peers peers;
     if (!fill_peers(*cfg, peer_windows_host, peers)) return SPEC_ERR_INVALID_ARG;
     const EpLayout l = make_layout(*cfg);
@@ -294,10 +301,41 @@ extern "C" spec_status spec_ep_experts(const spec_ep_config* cfg, void* const* p
     if (r != SPEC_OK || cfg->cap_rows == 0) return r;      // capacity 0: the offsets and the status are published, nothing to compute
     const long long most = (long long)R * cfg->max_rows;
     const int max_per_group = (int)(most < cfg->cap_rows ? most : cfg->cap_rows);
+    if (w8) {
+        // rows are quantised where they are computed on: a row gives the same codes on whichever rank its expert lives
+        unsigned char* a8 = sc + l.a8;
+        float* a8s = reinterpret_cast<float*>(sc + l.a8_scale);
+        // only the rows that arrived (the count sits in this rank's window header; past the capacity nothing was stored)
+        const int32_t* n_recv = reinterpret_cast<const int32_t*>(peers.win[me] + l.hdr) + HDR_RECV_TOTAL;
+        r = launch_quantize_rows(cfg->cap_rows, d, a_perm, a8, a8s, st, n_recv);
+        if (r != SPEC_OK) return r;
+        r = launch_gemm8_grouped(cfg->cap_rows, max_per_group, per, 2 * Fe, d, a8, a8s, w_gateup, gateup_scale, sc + l.act, SPEC_DTYPE_BF16, 1, gc, go,
+                                 status, st);
+        if (r != SPEC_OK) return r;
+        r = launch_quantize_rows(cfg->cap_rows, Fe, sc + l.act, a8, a8s, st, n_recv);
+        if (r != SPEC_OK) return r;
+        return launch_gemm8_grouped(cfg->cap_rows, max_per_group, per, d, Fe, a8, a8s, w_down, down_scale, peers.win[me] + l.y, SPEC_DTYPE_F32, 0, gc, go,
+                                    status, st);
+    }
     r = launch_gemm_grouped(cfg->cap_rows, max_per_group, per, 2 * Fe, d, a_perm, w_gateup, sc + l.act, SPEC_DTYPE_BF16, 1, gc, go, status, st);
     if (r != SPEC_OK) return r;
     return launch_gemm_grouped(cfg->cap_rows, max_per_group, per, d, Fe, sc + l.act, w_down, peers.win[me] + l.y, SPEC_DTYPE_F32, 0, gc, go,
                                status, st);
+}
+}  // namespace
+
+extern "C" spec_status spec_ep_experts(const spec_ep_config* cfg, void* const* peer_windows_host, void* scratch,
+                                       const void* w_gateup, const void* w_down, int32_t* status, void* stream)
+{
+    return ep_experts(cfg, peer_windows_host, scratch, w_gateup, nullptr, w_down, nullptr, status, stream);
+}
+
+extern "C" spec_status spec_ep_experts_e4m3(const spec_ep_config* cfg, void* const* peer_windows_host, void* scratch,
+                                            const void* w_gateup, const float* w_gateup_scale, const void* w_down,
+                                            const float* w_down_scale, int32_t* status, void* stream)
+{
+    if (w_gateup_scale == nullptr || w_down_scale == nullptr) return SPEC_ERR_INVALID_ARG;
+    return ep_experts(cfg, peer_windows_host, scratch, w_gateup, w_gateup_scale, w_down, w_down_scale, status, stream);
 }
 
 extern "C" spec_status spec_ep_combine(const spec_ep_config* cfg, void* const* peer_windows_host, int M, float* x, void* stream)

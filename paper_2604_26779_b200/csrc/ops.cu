@@ -501,14 +501,16 @@ __global__ void __launch_bounds__(256) permute_rows_kernel(int R, size_t row_byt
 // round_e4m3(x / scale) with an exact fp32 division, round to nearest even, saturating: the same steps as the oracle's.
 template <int CHUNKS>
 __global__ void __launch_bounds__(256) quantize_rows_kernel(int K, const __nv_bfloat16* __restrict__ x, unsigned char* __restrict__ codes,
-                                                            float* __restrict__ scales)
+                                                            float* __restrict__ scales, const int32_t* __restrict__ rows_valid)
 {
+    // rows_valid (may be null): a device-side count; rows at or past it are left alone
     // CHUNKS > 0: the row (K <= 256 * 8 * CHUNKS) stays in registers between the maximum and the conversion, one global read;
     // CHUNKS == 0: any K, the row is read twice (the second time from cache)
     pdl_trigger();
     pdl_wait();
     __shared__ float s_w[8];
     const int row = blockIdx.x;
+    if (rows_valid != nullptr && row >= *rows_valid) return;
     const __nv_bfloat16* xr = x + (size_t)row * K;
     constexpr int NV = CHUNKS > 0 ? CHUNKS : 1;
     uint4 held[NV];
@@ -740,13 +742,13 @@ spec_status launch_permute_rows(int n_keep, int R, size_t row_bytes, const int32
     return launch_status();
 }
 
-spec_status launch_quantize_rows(int rows, int K, const void* x_bf16, void* codes, float* scales, cudaStream_t st)
+spec_status launch_quantize_rows(int rows, int K, const void* x_bf16, void* codes, float* scales, cudaStream_t st, const int32_t* rows_valid)
 {
     if (rows == 0) return SPEC_OK;
     if (K <= 0 || K % 8 != 0) return SPEC_ERR_SHAPE;
-    if (K <= 256 * 8 * 2)      launch_pdl(quantize_rows_kernel<2>, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales);
-    else if (K <= 256 * 8 * 8) launch_pdl(quantize_rows_kernel<8>, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales);
-    else                       launch_pdl(quantize_rows_kernel<0>, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales);
+    if (K <= 256 * 8 * 2)      launch_pdl(quantize_rows_kernel<2>, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales, rows_valid);
+    else if (K <= 256 * 8 * 8) launch_pdl(quantize_rows_kernel<8>, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales, rows_valid);
+    else                       launch_pdl(quantize_rows_kernel<0>, dim3(rows), dim3(256), 0, st, K, (const __nv_bfloat16*)x_bf16, (unsigned char*)codes, scales, rows_valid);
     return launch_status();
 }
 
@@ -772,5 +774,5 @@ extern "C" spec_status spec_quantize_rows(int rows, int K, const void* x_bf16, v
     if (rows < 0 || K <= 0) return SPEC_ERR_INVALID_ARG;
     if (rows == 0) return SPEC_OK;
     if (!x_bf16 || !codes || !scales) return SPEC_ERR_INVALID_ARG;
-    return spec::launch_quantize_rows(rows, K, x_bf16, codes, scales, (cudaStream_t)stream);
+    return spec::launch_quantize_rows(rows, K, x_bf16, codes, scales, (cudaStream_t)stream, nullptr);
 }

@@ -44,7 +44,9 @@ spec_status launch_rope_append(int B, int R, int Hq, int Hkv, int dh, float thet
                                void* k_pool, void* v_pool, const int32_t* block_table, int max_blocks,
                                int block_tokens, int dtype, cudaStream_t st, const float* rope_table = nullptr);   // rope_table: [dh/2][B*R] (cos, sin) of pos, or NULL
 spec_status launch_swiglu(int M, int F, const void* gate_up, void* out, int dtype, cudaStream_t st);
-spec_status launch_quantize_rows(int rows, int K, const void* x_bf16, void* codes, float* scales, cudaStream_t st);
+// rows_valid: optional device-side count of the rows that hold data (the others are skipped)
+spec_status launch_quantize_rows(int rows, int K, const void* x_bf16, void* codes, float* scales, cudaStream_t st,
+                                 const int32_t* rows_valid = nullptr);
 // RMSNorm of fp32 rows [M][d] + per-row e4m3 quantisation of the bf16-rounded result (same codes and scales as the two separate kernels).
 spec_status launch_rmsnorm_quantize(int M, int d, const float* in, const float* w, float eps, void* codes, float* scales, cudaStream_t st);
 spec_status launch_copy_rows_f32_to(int M, int d, const float* x, void* out, int ld_out, int col0, int dtype,

@@ -48,9 +48,14 @@ class EpRank:
         self.M = int(h.shape[0])
         api.spec_ep_route(self.cfg, self.window, self.scratch, self.M, h if self.M else None, router_w, stream)
 
-    def experts(self, w_gateup, w_down, stream=None):
+    def experts(self, w_gateup, w_down, stream=None, scales=None):
+        """scales: None for 16-bit expert weights, or (gate/up scales, down scales) with the weights as e4m3 codes."""
         assert self.peers is not None, "set_peers first"
-        api.spec_ep_experts(self.cfg, self.peers, self.scratch, w_gateup, w_down, self.status, stream)
+        if scales is None:
+            api.spec_ep_experts(self.cfg, self.peers, self.scratch, w_gateup, w_down, self.status, stream)
+        else:
+            assert w_gateup.dtype == torch.uint8 and w_down.dtype == torch.uint8
+            api.spec_ep_experts_e4m3(self.cfg, self.peers, self.scratch, w_gateup, scales[0], w_down, scales[1], self.status, stream)
 
     def combine(self, x, stream=None):
         assert x.dtype == torch.float32 and tuple(x.shape) == (self.M, self.cfg.d)
@@ -108,7 +113,7 @@ def stream_barrier(dist, group=None, device_tensor=None):
     dist.barrier(group=group)
 
 
-def run_block_single_process(ranks, hs, router_w, w_gateups, w_downs, xs, stream=None):
+def run_block_single_process(ranks, hs, router_w, w_gateups, w_downs, xs, stream=None, scales=None):
     """All ranks of a group inside one process (their windows on one GPU): phase by phase on one stream."""
     addresses = [r.window.data_ptr() for r in ranks]
     for r in ranks:
@@ -116,7 +121,7 @@ def run_block_single_process(ranks, hs, router_w, w_gateups, w_downs, xs, stream
             r.set_peers(addresses)
     for r, h in zip(ranks, hs):
         r.route(h, router_w, stream)
-    for r, gu, dn in zip(ranks, w_gateups, w_downs):
-        r.experts(gu, dn, stream)
+    for i, (r, gu, dn) in enumerate(zip(ranks, w_gateups, w_downs)):
+        r.experts(gu, dn, stream, None if scales is None else scales[i])
     for r, x in zip(ranks, xs):
         r.combine(x, stream)

@@ -173,3 +173,64 @@ def test_ep_block_235b_shape_sampled():
         worst = max(worst, float(np.abs(got - ref).max() / np.abs(ref).max()))
     print(f"235B-shape expert-parallel block, 4 ranks: worst sampled relative error {worst:.2e}")
     assert worst < 2e-2
+
+
+def run_ep_8bit(lw, hs, xs, ep_size, top_k):
+    """The block with 8-bit expert weights: every rank's local experts quantised row by row on the device."""
+    from paper_2604_26779_b200 import binding as api, expert_parallel as ep
+    from paper_2604_26779_b200.engine import stack_gate_up
+    E, Fe, d = lw["experts_gate"].shape
+    per = E // ep_size
+    max_rows = max(max(h.shape[0] for h in hs), 1)
+    ranks = [ep.EpRank(ep_size, r, E, top_k, d, Fe, max_rows) for r in range(ep_size)]
+    gus, dns, scales = [], [], []
+    for r in range(ep_size):
+        gu = stack_gate_up(lw["experts_gate"][r * per : (r + 1) * per], lw["experts_up"][r * per : (r + 1) * per]).contiguous().cuda()
+        dn = lw["experts_down"][r * per : (r + 1) * per].contiguous().cuda()
+        gu8, dn8 = torch.empty(gu.shape, dtype=torch.uint8, device="cuda"), torch.empty(dn.shape, dtype=torch.uint8, device="cuda")
+        gs = torch.empty(per * 2 * Fe, dtype=torch.float32, device="cuda")
+        ds = torch.empty(per * d, dtype=torch.float32, device="cuda")
+        api.spec_quantize_rows(gu.view(-1, d), gu8.view(-1, d), gs)
+        api.spec_quantize_rows(dn.view(-1, Fe), dn8.view(-1, Fe), ds)
+        gus.append(gu8); dns.append(dn8); scales.append((gs, ds))
+    xd = [x.clone().cuda() for x in xs]
+    ep.run_block_single_process(ranks, [h.cuda() for h in hs], lw["router"].cuda(), gus, dns, xd, scales=scales)
+    torch.cuda.synchronize()
+    for r in ranks:
+        r.check_status()
+    return ranks, xd
+
+
+def test_ep_block_with_8bit_experts():
+    """8-bit expert weights (Section 5.1 names FP8 as the precision of the paper's large-scale projection): bit-identical for
+    every ep_size, and against the oracle's 8-bit block routed with the device's decisions.  The block's input rows are
+    given, so both sides quantise the same rows; what is left is the rare SwiGLU output that rounds to the neighbouring
+    bf16 value on one side (a code step in one element, or - for a row maximum - a 2^-8 shift of that row's scale):
+    bar 1e-2 of the row maximum."""
+    E, top_k, d, Fe = 16, 4, 512, 128
+    rows = [70, 3, 129, 40]
+    lw, hs, xs = make_case(E, top_k, d, Fe, rows, seed=21)
+    r4, x4 = run_ep_8bit(lw, hs, xs, 4, top_k)
+    _, x2 = run_ep_8bit(lw, [torch.cat(hs[:2]), torch.cat(hs[2:])], [torch.cat(xs[:2]), torch.cat(xs[2:])], 2, top_k)
+    _, x1 = run_ep_8bit(lw, [torch.cat(hs)], [torch.cat(xs)], 1, top_k)
+    a = torch.cat([x.cpu() for x in x4])
+    assert torch.equal(a, torch.cat([x.cpu() for x in x2])) and torch.equal(a, x1[0].cpu())
+    _, x16 = run_ep(lw, hs, xs, 4, top_k)
+    assert not torch.equal(a, torch.cat([x.cpu() for x in x16]))                   # the 8-bit path really ran
+    lw64 = {k: f64(v) for k, v in lw.items()}
+    lwo = dict(router=lw64["router"], experts_gate=list(lw64["experts_gate"]), experts_up=list(lw64["experts_up"]),
+               experts_down=list(lw64["experts_down"]))
+    worst = 0.0
+    for s in range(4):
+        n = rows[s]
+        ids = r4[s].tensor("IDS")[:n].cpu().numpy()
+        wts = r4[s].tensor("WTS")[:n].cpu().numpy()
+        # hand the oracle the device's decisions: logits that reproduce ids in order and the device's weights
+        fake = np.full((n, E), -1e9)
+        for t in range(n):
+            fake[t, ids[t]] = np.log(wts[t].astype(np.float64))
+        ref = model.moe_mlp(lwo, f64(hs[s]), top_k, router_logits=fake, cfg={"w_fp8": True})
+        got = x4[s].cpu().numpy().astype(np.float64) - xs[s].numpy().astype(np.float64)
+        worst = max(worst, float((np.abs(got - ref).max(-1) / np.abs(ref).max(-1)).max()))
+    print(f"expert-parallel block, 8-bit experts: worst relative error {worst:.2e}")
+    assert worst < 1e-2
