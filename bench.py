@@ -633,6 +633,8 @@ def main():
         metric = f"accepted tokens/s per B200 (one 235B-A22B-shaped MoE layer + LM head, k={k}; not the headline)"
     elif k != 3 or B != 256:
         metric = f"accepted tokens/s per B200 (8B-shape verify+sample, k={k}, B={B}; not the headline configuration)"
+    if args.workload == "c3" and args.draft_vocab:
+        metric += f" [draft head with its own {args.draft_vocab}-row vocabulary: not the headline configuration]"
     line = {"metric": metric + (" [8-bit KV cache variant]" if cfg.get("kv_fp8") else "") + (" [8-bit weights variant]" if cfg.get("w_fp8") else ""),
             "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -148,6 +148,16 @@ def test_ep_host_errors():
         with pytest.raises(api.SpecError) as e:
             api.spec_ep_query_sizes(bad)
         assert e.value.code == code
+    # the 8-bit form wants both scale arrays
+    sizes = api.spec_ep_query_sizes(ok)
+    win = torch.zeros(sizes.window_bytes, dtype=torch.uint8, device="cuda")
+    scr = torch.zeros(sizes.scratch_bytes, dtype=torch.uint8, device="cuda")
+    w = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    sc = torch.ones(16, dtype=torch.float32, device="cuda")
+    for gs, ds in ((None, sc), (sc, None)):
+        with pytest.raises(api.SpecError) as e:
+            api.spec_ep_experts_e4m3(ok, [win.data_ptr(), win.data_ptr()], scr, w, gs, w, ds)
+        assert e.value.code == -1
 
 
 def test_ep_block_235b_shape_sampled():
