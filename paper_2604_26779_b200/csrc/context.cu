@@ -316,24 +316,32 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
     void* ws = c.buf.workspace;
     int32_t* status_word = at<int32_t>(c.buf.state, c.status);
     const bool w8 = g.weight_dtype == SPEC_W_E4M3 && W.wqkv_s != nullptr;   // the target's layers with 8-bit weights (the draft head has none)
+    // what the fused QKV epilogue needs (rotary table, cache slots), and the attention launch: the same for every weight format
+    auto qkv_epilogue = [&]() {
+        QkvEpilogue e{Hq, Hkv, dh, R, g.max_blocks_per_seq, g.kv_block_tokens, pos, at<int32_t>(c.buf.state, c.block_table),
+                      at<float>(ws, c.rope), k_pool, v_pool};
+        if (g.kv_dtype == SPEC_KV_E4M3) { e.kv_fp8 = 1; e.k_scale = g.kv_scale_k; e.v_scale = g.kv_scale_v; }
+        return e;
+    };
+    auto attention = [&]() -> spec_status {
+        AttnArgs a{B, R, Hq, Hkv, dh, g.kv_block_tokens, g.max_blocks_per_seq, at(ws, c.qkv), qkv_n, k_pool, v_pool,
+                   at<int32_t>(c.buf.state, c.block_table), pos, at(ws, c.attn_out), Hq * dh, dt, at(ws, c.attn_scratch),
+                   c.attn_scratch.bytes, g.max_blocks_per_seq * g.kv_block_tokens, launch_index};
+        a.status = status_word;
+        if (g.kv_dtype == SPEC_KV_E4M3) { a.kv_fp8 = 1; a.k_scale = g.kv_scale_k; a.v_scale = g.kv_scale_v; }
+        Timed t__(c, CLS_ATTN, st);
+        return launch_attention(a, st);
+    };
     if (w8) {
         const size_t slot_bytes = c.a8.bytes / kActSlots, slot_rows = c.a8_scale.bytes / kActSlots / 4;
         auto a8_of = [&](int slot) { return at<unsigned char>(ws, c.a8) + slot * slot_bytes; };
         auto a8s_of = [&](int slot) { return at<float>(ws, c.a8_scale) + slot * slot_rows; };
         // every projection: its input rows to e4m3 with a scale per row, then the 8-bit tensor-core product; the epilogues
         // are the usual ones (rotary + cache append, residual add, SwiGLU) on the rescaled accumulators
-        QkvEpilogue e{Hq, Hkv, dh, R, g.max_blocks_per_seq, g.kv_block_tokens, pos, at<int32_t>(c.buf.state, c.block_table),
-                      at<float>(ws, c.rope), k_pool, v_pool};
-        if (g.kv_dtype == SPEC_KV_E4M3) { e.kv_fp8 = 1; e.k_scale = g.kv_scale_k; e.v_scale = g.kv_scale_v; }
         if (qkv_in == nullptr) TRY(launch_rmsnorm_quantize(M, d, res, W.attn_norm, g.rms_eps, a8_of(0), a8s_of(0), st));   // norm fused with the quantiser
         else TRY(launch_quantize_rows(M, qkv_k, qkv_in, a8_of(0), a8s_of(0), st));
-        TIMED(c, CLS_GEMM, launch_gemm8_qkv_tc(M, qkv_k, a8_of(0), a8s_of(0), W.wqkv, W.wqkv_s, at(ws, c.qkv), e, status_word, st));
-        AttnArgs a{B, R, Hq, Hkv, dh, g.kv_block_tokens, g.max_blocks_per_seq, at(ws, c.qkv), qkv_n, k_pool, v_pool,
-                   at<int32_t>(c.buf.state, c.block_table), pos, at(ws, c.attn_out), Hq * dh, dt, at(ws, c.attn_scratch),
-                   c.attn_scratch.bytes, g.max_blocks_per_seq * g.kv_block_tokens, launch_index};
-        a.status = status_word;
-        if (g.kv_dtype == SPEC_KV_E4M3) { a.kv_fp8 = 1; a.k_scale = g.kv_scale_k; a.v_scale = g.kv_scale_v; }
-        TIMED(c, CLS_ATTN, launch_attention(a, st));
+        TIMED(c, CLS_GEMM, launch_gemm8_qkv_tc(M, qkv_k, a8_of(0), a8s_of(0), W.wqkv, W.wqkv_s, at(ws, c.qkv), qkv_epilogue(), status_word, st));
+        TRY(attention());
         TRY(launch_quantize_rows(M, Hq * dh, at(ws, c.attn_out), a8_of(1), a8s_of(1), st));
         TIMED(c, CLS_GEMM, launch_gemm8_tc(M, d, Hq * dh, a8_of(1), a8s_of(1), W.wo, W.wo_s, res, d, SPEC_DTYPE_F32, 1, 1.f, nullptr, 0, nullptr, 0,
                                            status_word, st));
@@ -372,10 +380,7 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
                        gemm_tc_thin_supported(M, 2 * d_ffn, d, at(ws, c.h), d, W.wgateup, at(ws, c.gu), 2 * d_ffn, dt, dt));
     if (tc && !thin && (dh == 64 || dh == 128)) {
         // projection, rotary embedding and the append into the paged cache in one kernel
-        QkvEpilogue e{Hq, Hkv, dh, R, g.max_blocks_per_seq, g.kv_block_tokens, pos, at<int32_t>(c.buf.state, c.block_table),
-                      at<float>(ws, c.rope), k_pool, v_pool};
-        if (g.kv_dtype == SPEC_KV_E4M3) { e.kv_fp8 = 1; e.k_scale = g.kv_scale_k; e.v_scale = g.kv_scale_v; }
-        TIMED(c, CLS_GEMM, launch_gemm_qkv_tc(M, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), e, status_word, st));
+        TIMED(c, CLS_GEMM, launch_gemm_qkv_tc(M, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_epilogue(), status_word, st));
     } else {
         if (g.kv_dtype == SPEC_KV_E4M3) return SPEC_ERR_UNSUPPORTED;    // the 8-bit cache is written by the fused epilogue only
         TIMED(c, CLS_GEMM, launch_gemm(M, qkv_n, qkv_k, qkv_in, qkv_k, W.wqkv, at(ws, c.qkv), qkv_n, dt, dt, 0, st));
@@ -383,12 +388,7 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
                                at<int32_t>(c.buf.state, c.block_table), g.max_blocks_per_seq, g.kv_block_tokens, dt, st,
                                at<float>(ws, c.rope)));
     }
-    AttnArgs a{B, R, Hq, Hkv, dh, g.kv_block_tokens, g.max_blocks_per_seq, at(ws, c.qkv), qkv_n, k_pool, v_pool,
-               at<int32_t>(c.buf.state, c.block_table), pos, at(ws, c.attn_out), Hq * dh, dt, at(ws, c.attn_scratch),
-               c.attn_scratch.bytes, g.max_blocks_per_seq * g.kv_block_tokens, launch_index};
-    a.status = status_word;
-    if (g.kv_dtype == SPEC_KV_E4M3) { a.kv_fp8 = 1; a.k_scale = g.kv_scale_k; a.v_scale = g.kv_scale_v; }
-    TIMED(c, CLS_ATTN, launch_attention(a, st));
+    TRY(attention());
     TIMED(c, CLS_GEMM, launch_gemm(M, d, Hq * dh, at(ws, c.attn_out), Hq * dh, W.wo, res, d, dt, SPEC_DTYPE_F32, 1, st));
     TRY(launch_rmsnorm(M, d, res, W.mlp_norm, g.rms_eps, at(ws, c.h), d, 0, dt, st));
     if (W.router != nullptr) {
