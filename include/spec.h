@@ -298,7 +298,10 @@ spec_status spec_uniforms(uint64_t seed, uint32_t step, uint32_t stream_tag, int
 
 /* Per-row e4m3 quantisation of a bf16 matrix x [rows][K] (K % 16 == 0): scales [rows] = amax(row) / 448 (1 for a zero
  * row), codes [rows][K] = round_e4m3(x / scale), round to nearest even, saturating.  What SPEC_W_E4M3 contexts expect in
- * their weight tensors, and what they do to activations. */
+ * their weight tensors, and what they do to activations (the 8-bit precision the paper's large-scale projection assumes,
+ * Section 5.1; the paper gives no scaling rule, this one is ours).  All pointers are device memory owned by the caller,
+ * x and codes 16-byte aligned; rows == 0 is a no-op; a null pointer or K <= 0 returns SPEC_ERR_INVALID_ARG and
+ * K % 8 != 0 SPEC_ERR_SHAPE, both before anything is launched. */
 spec_status spec_quantize_rows(int rows, int K, const void* x_bf16, void* codes, float* scales, void* stream);
 
 /* C[M][N] = A[M][K] * W[N][K]^T (+ C when accumulate != 0).  dtype_in selects bf16 (tensor-core path, fp32
@@ -309,7 +312,9 @@ spec_status spec_gemm(int M, int N, int K, const void* A, const void* W, void* C
 
 /* The same product with 8-bit operands: a8 [M][K] and w8 [N][K] e4m3 codes (as spec_quantize_rows writes them), a_scale
  * [M] and w_scale [N] their row scales; C[m][n] (+)= a_scale[m] * w_scale[n] * sum_k a8[m][k] * w8[n][k], accumulated in
- * fp32 on the 8-bit tensor-core path.  K % 16 == 0, N % 8 == 0; pointers 16-byte aligned. */
+ * fp32 on the 8-bit tensor-core path.  K % 16 == 0, N % 8 == 0; pointers 16-byte aligned; C is fp32 or bf16 (out_dtype),
+ * caller-owned device memory like the operands.  M == 0 or N == 0 is a no-op; a null pointer returns
+ * SPEC_ERR_INVALID_ARG, a shape or alignment the kernel does not take SPEC_ERR_SHAPE, nothing launched in either case. */
 spec_status spec_gemm_e4m3(int M, int N, int K, const void* a8, const float* a_scale, const void* w8, const float* w_scale,
                            void* C, int out_dtype, int accumulate, void* stream);
 

@@ -136,3 +136,18 @@ def test_sizes_and_refusals_with_8bit_projections():
             setattr(sc, k, v)
         got, _ = sizes_of(sc)
         assert got == -3, (change, got)
+
+
+def test_8bit_operator_argument_checks_need_no_device():
+    """spec_quantize_rows / spec_gemm_e4m3 refuse bad arguments on the host, before anything is launched."""
+    L = B.lib()
+    fake = 4096                                                 # non-null, 16-byte aligned, never dereferenced on the host
+    assert L.spec_quantize_rows(0, 64, None, None, None, None) == 0
+    assert L.spec_quantize_rows(4, 0, fake, fake, fake, None) == -1
+    assert L.spec_quantize_rows(4, 64, None, fake, fake, None) == -1
+    assert L.spec_quantize_rows(4, 12, fake, fake, fake, None) == -2
+    assert L.spec_gemm_e4m3(0, 64, 64, None, None, None, None, None, 1, 0, None) == 0
+    assert L.spec_gemm_e4m3(4, 64, 64, fake, None, fake, fake, fake, 1, 0, None) == -1
+    assert L.spec_gemm_e4m3(4, 60, 64, fake, fake, fake, fake, fake, 1, 0, None) == -2
+    assert L.spec_gemm_e4m3(4, 64, 24, fake, fake, fake, fake, fake, 1, 0, None) == -2       # K % 16
+    assert L.spec_gemm_e4m3(4, 64, 64, fake + 8, fake, fake, fake, fake, 1, 0, None) == -2   # operand alignment
