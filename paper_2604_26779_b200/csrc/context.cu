@@ -352,9 +352,11 @@ spec_status run_layer_body(spec_ctx& c, const LayerPtrs& W, int d_ffn, float* re
             TRY(launch_rmsnorm(M, d, res, W.mlp_norm, g.rms_eps, at(ws, c.h), d, 0, dt, st));
             TIMED(c, CLS_GEMM, launch_gemm(M, E, d, at(ws, c.h), d, W.router, at(ws, c.moe_logits), E, dt, SPEC_DTYPE_F32, 0, st));
             TRY(launch_moe_route(M, E, tk, at<float>(ws, c.moe_logits), at<int32_t>(ws, c.moe_ids), at<float>(ws, c.moe_wts), st));
-            TRY(launch_moe_permute(M, E, tk, d, at<int32_t>(ws, c.moe_ids), at<int32_t>(ws, c.moe_rank), at<int32_t>(ws, c.moe_counts),
-                                   at<int32_t>(ws, c.moe_offsets), at<int32_t>(ws, c.moe_inv), at(ws, c.h), at(ws, c.moe_a), st));
-            TRY(launch_quantize_rows(n, d, at(ws, c.moe_a), a8_of(2), a8s_of(2), st));
+            // the rows are quantised once (parked in slot 3, which the SwiGLU outputs take over later) and their codes and
+            // scales permuted into expert order: the same codes as quantising every permuted copy, an eighth of the work
+            TRY(launch_quantize_rows(M, d, at(ws, c.h), a8_of(3), a8s_of(3), st));
+            TRY(launch_moe_permute(M, E, tk, d / 2, at<int32_t>(ws, c.moe_ids), at<int32_t>(ws, c.moe_rank), at<int32_t>(ws, c.moe_counts),
+                                   at<int32_t>(ws, c.moe_offsets), at<int32_t>(ws, c.moe_inv), a8_of(3), a8_of(2), st, a8s_of(3), a8s_of(2)));
             TIMED(c, CLS_GEMM, launch_gemm8_grouped(n, M, E, 2 * Fe, d, a8_of(2), a8s_of(2), W.exp_gateup, W.exp_gateup_s, at(ws, c.moe_act), dt, 1,
                                                     at<int32_t>(ws, c.moe_counts), at<int32_t>(ws, c.moe_offsets), status_word, st));
             TRY(launch_quantize_rows(n, Fe, at(ws, c.moe_act), a8_of(3), a8s_of(3), st));

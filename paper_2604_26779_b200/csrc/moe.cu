@@ -84,7 +84,8 @@ template <class T>
 __global__ void __launch_bounds__(256) moe_gather_kernel(int E, int top_k, int d, const int32_t* __restrict__ ids,
                                                          const int32_t* __restrict__ rank, const int32_t* __restrict__ counts,
                                                          int32_t* __restrict__ offsets, int32_t* __restrict__ inv,
-                                                         const T* __restrict__ h, T* __restrict__ a_perm)
+                                                         const T* __restrict__ h, T* __restrict__ a_perm,
+                                                         const float* __restrict__ row_scale, float* __restrict__ perm_scale)
 {
     __shared__ int s_off;
     const int i = blockIdx.x, e = ids[i];
@@ -100,7 +101,10 @@ __global__ void __launch_bounds__(256) moe_gather_kernel(int E, int top_k, int d
     }
     __syncthreads();
     const int pos = s_off + rank[i];
-    if (threadIdx.x == 0) inv[i] = pos;
+    if (threadIdx.x == 0) {
+        inv[i] = pos;
+        if (row_scale != nullptr) perm_scale[pos] = row_scale[i / top_k];   // 8-bit rows travel with their scale
+    }
     const T* src = h + (size_t)(i / top_k) * d;
     T* dst = a_perm + (size_t)pos * d;
     for (int c = threadIdx.x * 8; c < d; c += 256 * 8)
@@ -141,14 +145,15 @@ spec_status launch_moe_rank(int n_entries, int E, const int32_t* ids, int32_t* r
 }
 
 spec_status launch_moe_permute(int M, int E, int top_k, int d, const int32_t* ids, int32_t* rank, int32_t* counts,
-                               int32_t* offsets, int32_t* inv, const void* h, void* a_perm, cudaStream_t st)
+                               int32_t* offsets, int32_t* inv, const void* h, void* a_perm, cudaStream_t st,
+                               const float* row_scale, float* perm_scale)
 {
     const int n = M * top_k;
     if (n == 0) return SPEC_OK;
     moe_rank_kernel<<<E, 256, 0, st>>>(n, ids, rank, counts);
     if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
     moe_gather_kernel<__nv_bfloat16><<<n, 256, 0, st>>>(E, top_k, d, ids, rank, counts, offsets, inv,
-                                                       (const __nv_bfloat16*)h, (__nv_bfloat16*)a_perm);
+                                                       (const __nv_bfloat16*)h, (__nv_bfloat16*)a_perm, row_scale, perm_scale);
     return launch_status(2);
 }
 

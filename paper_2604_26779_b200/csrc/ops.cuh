@@ -139,8 +139,10 @@ spec_status launch_rope_table(int M, int dh, float theta, const int32_t* pos, fl
 // moe.cu: router top-k, permutation into expert order, weighted combination
 spec_status launch_moe_route(int M, int E, int top_k, const float* logits, int32_t* ids, float* wts, cudaStream_t st);
 spec_status launch_moe_rank(int n_entries, int E, const int32_t* ids, int32_t* rank, int32_t* counts, cudaStream_t st);
+// h rows of d 16-bit elements (8-bit code rows: pass d / 2 and the rows' scales, which are then permuted along)
 spec_status launch_moe_permute(int M, int E, int top_k, int d, const int32_t* ids, int32_t* rank, int32_t* counts,
-                               int32_t* offsets, int32_t* inv, const void* h, void* a_perm, cudaStream_t st);
+                               int32_t* offsets, int32_t* inv, const void* h, void* a_perm, cudaStream_t st,
+                               const float* row_scale = nullptr, float* perm_scale = nullptr);
 spec_status launch_moe_combine(int M, int top_k, int d, const float* wts, const int32_t* inv, const float* out_perm,
                                float* x, cudaStream_t st);
 
