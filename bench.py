@@ -348,7 +348,7 @@ def run_ep_microbench(args):
             clocks.start()
         ev[0].record()
         for r, h in zip(ranks, hs):
-            r.route(h, router)
+            r.route(h, router, rows8=args.w_fp8)
         ev[1].record()
         for r, gu, dn, sc in zip(ranks, gus, dns, scales):
             r.experts(gu, dn, scales=sc)
@@ -367,7 +367,7 @@ def run_ep_microbench(args):
     recv = [int(r.tensor("RECV_TOTAL")[0]) for r in ranks]
     rows = sum(recv) / R
     remote = (R - 1) / R
-    disp_b, comb_b = rows * d * 2, M * top_k * d * 4
+    disp_b, comb_b = rows * (d + 4 if args.w_fp8 else d * 2), M * top_k * d * 4      # 8-bit dispatch: codes + one scale per row
     nvl = 770.0e9
     hbm_peak, _, kind = measured_peaks()
     print(json.dumps({

@@ -407,10 +407,17 @@ spec_status spec_ep_route(const spec_ep_config* cfg, void* window, void* scratch
  * [local experts][d][d_expert_ffn]: the LOCAL experts only. */
 spec_status spec_ep_experts(const spec_ep_config* cfg, void* const* peer_windows_host, void* scratch,
                             const void* w_gateup, const void* w_down, int32_t* status, void* stream);
-/* The same with 8-bit expert weights: w_gateup / w_down hold e4m3 codes (one byte per element, same shapes),
- * w_gateup_scale [local experts][2 * d_expert_ffn] and w_down_scale [local experts][d] one fp32 scale per weight row
- * (spec_quantize_rows produces both).  The received rows and the SwiGLU outputs are quantised per row on this rank;
- * a row gives the same codes wherever its expert lives, so the result does not depend on ep_size. */
+/* The block with 8-bit expert weights and 8-bit dispatch (the precision of the paper's large-scale projection, Section 5.1).
+ * spec_ep_route_e4m3 is spec_ep_route that also publishes the rank's rows as e4m3 codes with one scale per row
+ * (spec_quantize_rows' rule; d % 16 == 0), quantised once at their source.  spec_ep_experts_e4m3 pulls those codes and
+ * scales (half the bytes of the 16-bit rows) and multiplies them with w_gateup / w_down given as e4m3 codes (one byte per
+ * element, same shapes as above) and w_gateup_scale [local experts][2 * d_expert_ffn], w_down_scale [local experts][d] (one
+ * fp32 scale per weight row; spec_quantize_rows produces both); the SwiGLU outputs are quantised per row on this rank.  A
+ * row gives the same codes wherever its expert lives, so the result does not depend on ep_size.  Every rank of the group
+ * must have routed with spec_ep_route_e4m3: a source that did not is reported as SPEC_ERR_STATE (detail = its rank) in
+ * `status`.  spec_ep_combine is unchanged. */
+spec_status spec_ep_route_e4m3(const spec_ep_config* cfg, void* window, void* scratch, int M, const void* h,
+                               const void* router_w, void* stream);
 spec_status spec_ep_experts_e4m3(const spec_ep_config* cfg, void* const* peer_windows_host, void* scratch,
                                  const void* w_gateup, const float* w_gateup_scale, const void* w_down,
                                  const float* w_down_scale, int32_t* status, void* stream);

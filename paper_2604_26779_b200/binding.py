@@ -118,6 +118,7 @@ SIGNATURES = {
     "spec_ep_query_sizes": (_i, [C.POINTER(spec_ep_config), C.POINTER(spec_ep_sizes)]),
     "spec_ep_tensor": (_i, [C.POINTER(spec_ep_config), _vp, _vp, _i, C.POINTER(_vp), C.POINTER(_sz)]),
     "spec_ep_route": (_i, [C.POINTER(spec_ep_config), _vp, _vp, _i, _vp, _vp, _vp]),
+    "spec_ep_route_e4m3": (_i, [C.POINTER(spec_ep_config), _vp, _vp, _i, _vp, _vp, _vp]),
     "spec_ep_experts": (_i, [C.POINTER(spec_ep_config), C.POINTER(_vp), _vp, _vp, _vp, _vp, _vp]),
     "spec_ep_experts_e4m3": (_i, [C.POINTER(spec_ep_config), C.POINTER(_vp), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "spec_ep_combine": (_i, [C.POINTER(spec_ep_config), C.POINTER(_vp), _i, _vp, _vp]),
@@ -273,6 +274,10 @@ def _peer_array(peer_windows):
 
 def spec_ep_route(cfg, window, scratch, M, h, router_w, stream=None):
     _check(lib().spec_ep_route(C.byref(cfg), _ptr(window), _ptr(scratch), M, _ptr(h), _ptr(router_w), _stream(stream)), "spec_ep_route")
+
+
+def spec_ep_route_e4m3(cfg, window, scratch, M, h, router_w, stream=None):
+    _check(lib().spec_ep_route_e4m3(C.byref(cfg), _ptr(window), _ptr(scratch), M, _ptr(h), _ptr(router_w), _stream(stream)), "spec_ep_route_e4m3")
 
 
 def spec_ep_experts(cfg, peer_windows, scratch, w_gateup, w_down, status=None, stream=None):

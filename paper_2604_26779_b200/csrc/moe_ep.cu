@@ -23,10 +23,10 @@ struct Peers { unsigned char* win[kMaxRanks]; };
 
 // Byte offsets inside a window / the scratch.  Every piece starts on a 256-byte boundary.
 struct EpLayout {
-    size_t hdr, h, ids, wts, rank, src_of, counts, offsets, recv_off, y, window_bytes;
+    size_t hdr, h, h8, h8_scale, ids, wts, rank, src_of, counts, offsets, recv_off, y, window_bytes;
     size_t logits, a_perm, act, grp_counts, grp_offsets, a8, a8_scale, scratch_bytes;
 };
-enum { HDR_M = 0, HDR_RECV_TOTAL = 1 };
+enum { HDR_M = 0, HDR_RECV_TOTAL = 1, HDR_ROWS8 = 2 };   // HDR_ROWS8: 1 when the rows were also published as e4m3 codes
 
 size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -38,6 +38,8 @@ EpLayout make_layout(const spec_ep_config& c)
     auto take = [&](size_t bytes) { const size_t o = at; at = up256(at + bytes); return o; };
     l.hdr = take(64 * 4);
     l.h = take((size_t)c.max_rows * c.d * 2);
+    l.h8 = take((size_t)c.max_rows * c.d);                   // the same rows as e4m3 codes + one scale each (spec_ep_route_e4m3)
+    l.h8_scale = take((size_t)c.max_rows * 4);
     l.ids = take(n * 4);
     l.wts = take(n * 4);
     l.rank = take(n * 4);
@@ -77,7 +79,7 @@ spec_status check(const spec_ep_config* c)
 __global__ void __launch_bounds__(256) ep_publish_kernel(int M, int E, int top_k, const int32_t* __restrict__ ids,
                                                          const int32_t* __restrict__ rank, const int32_t* __restrict__ counts,
                                                          int32_t* __restrict__ offsets, int32_t* __restrict__ src_of,
-                                                         int32_t* __restrict__ hdr)
+                                                         int32_t* __restrict__ hdr, int rows8)
 {
     __shared__ int s_off[kMaxExperts];
     if (threadIdx.x == 0) {
@@ -87,7 +89,7 @@ __global__ void __launch_bounds__(256) ep_publish_kernel(int M, int E, int top_k
     __syncthreads();
     if (blockIdx.x == 0) {
         for (int e = threadIdx.x; e < E; e += blockDim.x) offsets[e] = s_off[e];
-        if (threadIdx.x == 0) hdr[HDR_M] = M;
+        if (threadIdx.x == 0) { hdr[HDR_M] = M; hdr[HDR_ROWS8] = rows8; }
     }
     const int n = M * top_k;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
@@ -99,8 +101,10 @@ __global__ void __launch_bounds__(256) ep_publish_kernel(int M, int E, int top_k
 // the sources' published counts, then the CTAs copy rows: one row per CTA per turn, 16 bytes per thread per load.
 __global__ void __launch_bounds__(256) ep_pull_kernel(Peers peers, EpLayout L, int R, int me, int E, int top_k, int d, int cap_rows,
                                                       __nv_bfloat16* __restrict__ a_perm, int32_t* __restrict__ grp_counts,
-                                                      int32_t* __restrict__ grp_offsets, int32_t* status)
+                                                      int32_t* __restrict__ grp_offsets, int32_t* status,
+                                                      unsigned char* __restrict__ a8, float* __restrict__ a8_scale)
 {
+    // a8 != nullptr: pull the rows as e4m3 codes + scale (what spec_ep_route_e4m3 published) instead of the 16-bit rows
     __shared__ int s_cnt[kMaxExperts], s_off[kMaxExperts + 1], s_src_start[kMaxExperts];
     const int per = E / R, e0 = me * per;
     for (int u = threadIdx.x; u < E; u += blockDim.x) {
@@ -129,6 +133,9 @@ __global__ void __launch_bounds__(256) ep_pull_kernel(Peers peers, EpLayout L, i
         if (threadIdx.x == 0) {
             reinterpret_cast<int32_t*>(peers.win[me] + L.hdr)[HDR_RECV_TOTAL] = total;
             if (total > cap_rows) set_status(status, SPEC_ERR_EP_CAPACITY, total);
+            if (a8 != nullptr)                                       // every source must have published codes
+                for (int s = 0; s < R; ++s)
+                    if (reinterpret_cast<const int32_t*>(peers.win[s] + L.hdr)[HDR_ROWS8] != 1) set_status(status, SPEC_ERR_STATE, s);
         }
     }
     const int rows = min(total, cap_rows);
@@ -142,6 +149,13 @@ __global__ void __launch_bounds__(256) ep_pull_kernel(Peers peers, EpLayout L, i
         const int u = lo, s = u % R, j = t - s_off[u];
         const int32_t* src_of = reinterpret_cast<const int32_t*>(peers.win[s] + L.src_of);
         const int m = src_of[s_src_start[u] + j] / top_k;
+        if (a8 != nullptr) {
+            const uint4* src8 = reinterpret_cast<const uint4*>(peers.win[s] + L.h8 + (size_t)m * d);
+            uint4* dst8 = reinterpret_cast<uint4*>(a8 + (size_t)t * d);
+            for (int c = threadIdx.x; c < d / 16; c += blockDim.x) dst8[c] = src8[c];
+            if (threadIdx.x == 0) a8_scale[t] = reinterpret_cast<const float*>(peers.win[s] + L.h8_scale)[m];
+            continue;
+        }
         const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(peers.win[s] + L.h) + (size_t)m * d);
         uint4* dst = reinterpret_cast<uint4*>(a_perm + (size_t)t * d);
         for (int c = threadIdx.x; c < d / 8; c += blockDim.x) dst[c] = src[c];
@@ -236,8 +250,8 @@ extern "C" spec_status spec_ep_tensor(const spec_ep_config* cfg, void* window, v
     return SPEC_OK;
 }
 
-extern "C" spec_status spec_ep_route(const spec_ep_config* cfg, void* window, void* scratch, int M, const void* h,
-                                     const void* router_w, void* stream)
+namespace {
+spec_status ep_route(const spec_ep_config* cfg, void* window, void* scratch, int M, const void* h, const void* router_w, int rows8, void* stream)
 {
     const spec_status s = check(cfg);
     if (s != SPEC_OK) return s;
@@ -265,8 +279,25 @@ extern "C" spec_status spec_ep_route(const spec_ep_config* cfg, void* window, vo
     ep_publish_kernel<<<n > 0 ? (n + 255) / 256 : 1, 256, 0, st>>>(
         M, E, tk, reinterpret_cast<const int32_t*>(w + l.ids), reinterpret_cast<const int32_t*>(w + l.rank),
         reinterpret_cast<const int32_t*>(w + l.counts), reinterpret_cast<int32_t*>(w + l.offsets),
-        reinterpret_cast<int32_t*>(w + l.src_of), reinterpret_cast<int32_t*>(w + l.hdr));
-    return launch_status();
+        reinterpret_cast<int32_t*>(w + l.src_of), reinterpret_cast<int32_t*>(w + l.hdr), rows8);
+    r = launch_status();
+    if (r != SPEC_OK || !rows8 || M == 0) return r;
+    // 8-bit dispatch: a row is quantised once, here, and travels as codes + scale (half the bytes of the 16-bit row)
+    return launch_quantize_rows(M, d, w + l.h, w + l.h8, reinterpret_cast<float*>(w + l.h8_scale), st);
+}
+}  // namespace
+
+extern "C" spec_status spec_ep_route(const spec_ep_config* cfg, void* window, void* scratch, int M, const void* h,
+                                     const void* router_w, void* stream)
+{
+    return ep_route(cfg, window, scratch, M, h, router_w, 0, stream);
+}
+
+extern "C" spec_status spec_ep_route_e4m3(const spec_ep_config* cfg, void* window, void* scratch, int M, const void* h,
+                                          const void* router_w, void* stream)
+{
+    if (cfg != nullptr && cfg->d % 16 != 0) return SPEC_ERR_SHAPE;
+    return ep_route(cfg, window, scratch, M, h, router_w, 1, stream);
 }
 
 namespace {
@@ -296,19 +327,18 @@ spec_status ep_experts(const spec_ep_config* cfg, void* const* peer_windows_host
     }
     const long long want = (long long)sms * 8;
     const int grid = (int)(want < cfg->cap_rows ? want : (cfg->cap_rows > 0 ? cfg->cap_rows : 1));
-    ep_pull_kernel<<<grid, 256, 0, st>>>(peers, l, R, me, E, cfg->top_k, d, cfg->cap_rows, a_perm, gc, go, status);
+    ep_pull_kernel<<<grid, 256, 0, st>>>(peers, l, R, me, E, cfg->top_k, d, cfg->cap_rows, a_perm, gc, go, status,
+                                         w8 ? sc + l.a8 : nullptr, w8 ? reinterpret_cast<float*>(sc + l.a8_scale) : nullptr);
     spec_status r = launch_status();
     if (r != SPEC_OK || cfg->cap_rows == 0) return r;      // capacity 0: the offsets and the status are published, nothing to compute
     const long long most = (long long)R * cfg->max_rows;
     const int max_per_group = (int)(most < cfg->cap_rows ? most : cfg->cap_rows);
     if (w8) {
-        // rows are quantised where they are computed on: a row gives the same codes on whichever rank its expert lives
+        // the rows arrived as codes + scale, quantised once at their source: a row gives the same codes on whichever rank its
+        // expert lives, and half the bytes cross between ranks
         unsigned char* a8 = sc + l.a8;
         float* a8s = reinterpret_cast<float*>(sc + l.a8_scale);
-        // only the rows that arrived (the count sits in this rank's window header; past the capacity nothing was stored)
         const int32_t* n_recv = reinterpret_cast<const int32_t*>(peers.win[me] + l.hdr) + HDR_RECV_TOTAL;
-        r = launch_quantize_rows(cfg->cap_rows, d, a_perm, a8, a8s, st, n_recv);
-        if (r != SPEC_OK) return r;
         r = launch_gemm8_grouped(cfg->cap_rows, max_per_group, per, 2 * Fe, d, a8, a8s, w_gateup, gateup_scale, sc + l.act, SPEC_DTYPE_BF16, 1, gc, go,
                                  status, st);
         if (r != SPEC_OK) return r;

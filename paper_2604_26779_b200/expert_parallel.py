@@ -43,10 +43,12 @@ class EpRank:
         self.peers = [a if isinstance(a, int) else a.data_ptr() for a in addresses]
         assert self.peers[self.cfg.ep_rank] == self.window.data_ptr()
 
-    def route(self, h, router_w, stream=None):
+    def route(self, h, router_w, stream=None, rows8=False):
+        """rows8: also publish the rows as e4m3 codes + scales (what experts(..., scales=...) pulls)."""
         assert h.dtype == torch.bfloat16 and router_w.dtype == torch.bfloat16 and h.shape[1] == self.cfg.d
         self.M = int(h.shape[0])
-        api.spec_ep_route(self.cfg, self.window, self.scratch, self.M, h if self.M else None, router_w, stream)
+        fn = api.spec_ep_route_e4m3 if rows8 else api.spec_ep_route
+        fn(self.cfg, self.window, self.scratch, self.M, h if self.M else None, router_w, stream)
 
     def experts(self, w_gateup, w_down, stream=None, scales=None):
         """scales: None for 16-bit expert weights, or (gate/up scales, down scales) with the weights as e4m3 codes."""
@@ -120,7 +122,7 @@ def run_block_single_process(ranks, hs, router_w, w_gateups, w_downs, xs, stream
         if r.peers is None:
             r.set_peers(addresses)
     for r, h in zip(ranks, hs):
-        r.route(h, router_w, stream)
+        r.route(h, router_w, stream, rows8=scales is not None)
     for i, (r, gu, dn) in enumerate(zip(ranks, w_gateups, w_downs)):
         r.experts(gu, dn, stream, None if scales is None else scales[i])
     for r, x in zip(ranks, xs):

@@ -244,3 +244,24 @@ def test_ep_block_with_8bit_experts():
         worst = max(worst, float((np.abs(got - ref).max(-1) / np.abs(ref).max(-1)).max()))
     print(f"expert-parallel block, 8-bit experts: worst relative error {worst:.2e}")
     assert worst < 1e-2
+
+
+def test_8bit_experts_after_a_16bit_route_is_reported():
+    """spec_ep_experts_e4m3 pulls the codes spec_ep_route_e4m3 publishes; a source that routed with the 16-bit call is
+    reported in the status word (SPEC_ERR_STATE, detail = the source's rank), nothing faults."""
+    from paper_2604_26779_b200 import binding as api, expert_parallel as ep
+    E, top_k, d, Fe = 16, 4, 512, 128
+    lw, hs, xs = make_case(E, top_k, d, Fe, [20, 20], seed=5)
+    ranks = [ep.EpRank(2, r, E, top_k, d, Fe, 20) for r in range(2)]
+    addrs = [r.window.data_ptr() for r in ranks]
+    for r in ranks:
+        r.set_peers(addrs)
+    ranks[0].route(hs[0].cuda(), lw["router"].cuda(), rows8=True)
+    ranks[1].route(hs[1].cuda(), lw["router"].cuda(), rows8=False)              # this rank did not publish codes
+    w8 = torch.zeros((8, 2 * Fe, d), dtype=torch.uint8, device="cuda")
+    d8 = torch.zeros((8, d, Fe), dtype=torch.uint8, device="cuda")
+    sc = (torch.ones(8 * 2 * Fe, dtype=torch.float32, device="cuda"), torch.ones(8 * d, dtype=torch.float32, device="cuda"))
+    ranks[0].experts(w8, d8, scales=sc)
+    torch.cuda.synchronize()
+    st = ranks[0].status.cpu().tolist()
+    assert st[0] == -4 and st[1] == 1 and api.STATUS_NAMES[-4] == "SPEC_ERR_STATE"
