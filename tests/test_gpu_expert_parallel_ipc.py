@@ -30,7 +30,7 @@ def _case():
     return lw, hs, xs
 
 
-def _worker(rank, world, port, out):
+def _worker(rank, world, port, out, w8):
     from paper_2604_26779_b200 import expert_parallel as ep
     from paper_2604_26779_b200.engine import stack_gate_up
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
@@ -49,9 +49,11 @@ def _worker(rank, world, port, out):
     gu = stack_gate_up(lw["experts_gate"][rank * per : (rank + 1) * per], lw["experts_up"][rank * per : (rank + 1) * per]).contiguous().cuda()
     dn = lw["experts_down"][rank * per : (rank + 1) * per].contiguous().cuda()
     x = xs[rank].clone().cuda()
-    me.route(hs[rank].cuda(), lw["router"].cuda())
+    quant = lambda g_, d_: _quantised(g_, d_) if w8 else (g_, d_, None)      # 8-bit experts and 8-bit dispatch through the same windows
+    gu, dn, sc = quant(gu, dn)
+    me.route(hs[rank].cuda(), lw["router"].cuda(), rows8=w8)
     ep.stream_barrier(dist)
-    me.experts(gu, dn)
+    me.experts(gu, dn, scales=sc)
     ep.stream_barrier(dist)
     me.combine(x)
     ep.stream_barrier(dist)
@@ -61,18 +63,35 @@ def _worker(rank, world, port, out):
     gus = [stack_gate_up(lw["experts_gate"][r * per : (r + 1) * per], lw["experts_up"][r * per : (r + 1) * per]).contiguous().cuda() for r in range(world)]
     dns = [lw["experts_down"][r * per : (r + 1) * per].contiguous().cuda() for r in range(world)]
     xd = [t.clone().cuda() for t in xs]
-    ep.run_block_single_process(ranks, [h.cuda() for h in hs], lw["router"].cuda(), gus, dns, xd)
+    scs = None
+    if w8:
+        trip = [_quantised(g_, d_) for g_, d_ in zip(gus, dns)]
+        gus, dns, scs = [t[0] for t in trip], [t[1] for t in trip], [t[2] for t in trip]
+    ep.run_block_single_process(ranks, [h.cuda() for h in hs], lw["router"].cuda(), gus, dns, xd, scales=scs)
     torch.cuda.synchronize()
     out[rank] = ("ok", bool(torch.equal(x, xd[rank])), bool(torch.equal(x.cpu(), xs[rank])))
     dist.barrier()
     dist.destroy_process_group()
 
 
-def test_two_processes_one_gpu():
+def _quantised(gu, dn):
+    """Expert weights as e4m3 codes + one scale per row, by the library's quantiser."""
+    from paper_2604_26779_b200 import binding as api
+    g8, d8 = torch.empty(gu.shape, dtype=torch.uint8, device="cuda"), torch.empty(dn.shape, dtype=torch.uint8, device="cuda")
+    gs = torch.empty(gu.shape[0] * gu.shape[1], dtype=torch.float32, device="cuda")
+    ds = torch.empty(dn.shape[0] * dn.shape[1], dtype=torch.float32, device="cuda")
+    api.spec_quantize_rows(gu.view(-1, gu.shape[-1]), g8.view(-1, gu.shape[-1]), gs)
+    api.spec_quantize_rows(dn.view(-1, dn.shape[-1]), d8.view(-1, dn.shape[-1]), ds)
+    torch.cuda.synchronize()
+    return g8, d8, (gs, ds)
+
+
+@pytest.mark.parametrize("w8", [False, True])
+def test_two_processes_one_gpu(w8):
     s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
     with mp.Manager() as m:
         out = m.dict()
-        mp.spawn(_worker, args=(2, port, out), nprocs=2, join=True)
+        mp.spawn(_worker, args=(2, port, out, w8), nprocs=2, join=True)
         res = dict(out)
     if any(v[0] == "no-ipc" for v in res.values()):
         pytest.skip(f"inter-process memory handles are not available here: {[v for v in res.values() if v[0] == 'no-ipc'][0][1]}")
